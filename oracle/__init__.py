@@ -1,0 +1,230 @@
+"""numpy front-end of the CPU oracle (plain C, see w4a8_oracle.c / w4a8_oracle.h).
+
+TEST INFRASTRUCTURE ONLY: the test-suite, the smoke check and the benchmark's CPU-baseline
+leg are the only callers.  Nothing here imports or is imported by the CUDA package.
+
+BF16 tensors are numpy uint16 arrays of bit patterns; E4M3 tensors are uint8 arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "w4a8_oracle.c")
+_HDR = os.path.join(_HERE, "w4a8_oracle.h")
+_LIB = os.path.join(_HERE, "liboracle_w4a8.so")
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FMA contraction). Returns the .so path."""
+    stale = (
+        force
+        or not os.path.exists(_LIB)
+        or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    )
+    if stale:
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        cmd = [
+            "gcc", "-std=c11", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+            "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC, "-lm",
+        ]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    c = ctypes
+    p = c.c_void_p
+    i64 = c.c_int64
+    lib.oracle_e4m3_decode.restype = c.c_float
+    lib.oracle_e4m3_decode.argtypes = [c.c_uint8]
+    lib.oracle_e4m3_encode.restype = c.c_uint8
+    lib.oracle_e4m3_encode.argtypes = [c.c_float]
+    lib.oracle_e4m3_encode_n.restype = None
+    lib.oracle_e4m3_encode_n.argtypes = [p, i64, p]
+    lib.oracle_e4m3_decode_n.restype = None
+    lib.oracle_e4m3_decode_n.argtypes = [p, i64, p]
+    lib.oracle_bf16_to_f32.restype = c.c_float
+    lib.oracle_bf16_to_f32.argtypes = [c.c_uint16]
+    lib.oracle_f32_to_bf16.restype = c.c_uint16
+    lib.oracle_f32_to_bf16.argtypes = [c.c_float]
+    lib.oracle_quantize_weight_rtn.restype = c.c_int
+    lib.oracle_quantize_weight_rtn.argtypes = [p, i64, i64, c.c_int, c.c_int, c.c_int, c.c_int, p, p, p, p]
+    lib.oracle_dequant_weight.restype = c.c_int
+    lib.oracle_dequant_weight.argtypes = [p, p, p, i64, i64, c.c_int, p]
+    lib.oracle_quantize_act.restype = c.c_int
+    lib.oracle_quantize_act.argtypes = [p, i64, i64, i64, p, i64, p, c.c_int, p]
+    lib.oracle_linear.restype = c.c_int
+    lib.oracle_linear.argtypes = [p, i64, p, i64, p, p, c.c_int, i64, i64, p, i64, p, p, p, p]
+    lib.oracle_num_threads.restype = c.c_int
+    lib.oracle_num_threads.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+# ----------------------------------------------------------------------------- scalar codec
+
+def e4m3_decode(code: int) -> float:
+    return float(_load().oracle_e4m3_decode(int(code) & 0xFF))
+
+
+def e4m3_encode(v: float) -> int:
+    return int(_load().oracle_e4m3_encode(float(np.float32(v))))
+
+
+def e4m3_encode_array(v) -> np.ndarray:
+    """Element-wise oracle encoder over an fp32 array."""
+    lib = _load()
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    lib.oracle_e4m3_encode_n(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def e4m3_decode_array(c) -> np.ndarray:
+    """Element-wise oracle decoder over a uint8 array."""
+    lib = _load()
+    c = np.ascontiguousarray(c, dtype=np.uint8)
+    out = np.empty(c.shape, dtype=np.float32)
+    lib.oracle_e4m3_decode_n(_ptr(c), c.size, _ptr(out))
+    return out
+
+
+def e4m3_decode_table() -> np.ndarray:
+    return e4m3_decode_array(np.arange(256, dtype=np.uint8))
+
+
+def bf16_to_f32(bits) -> np.ndarray:
+    bits = np.asarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32)
+
+
+def f32_to_bf16(x) -> np.ndarray:
+    """Round-to-nearest-even fp32 -> BF16 bit patterns, through the C routine's definition."""
+    lib = _load()
+    x = np.asarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    fo, fx = out.reshape(-1), x.reshape(-1)
+    f = lib.oracle_f32_to_bf16
+    for i in range(fx.size):
+        fo[i] = f(float(fx[i]))
+    return out
+
+
+# ----------------------------------------------------------------------------- tensor routines
+
+def quantize_weight_rtn(W, group=128, symmetric=True, pow2=False, per_channel=False):
+    """Eq. 6-9 round-to-nearest.  Returns (codes[N,K/2] u8, gscale[N,K/g] u16 bf16 bits,
+    gzero[N,K/g] u8 or None when symmetric, s_w fp32[N or 1])."""
+    lib = _load()
+    W = _c(W, np.float32)
+    N, K = W.shape
+    G = K // group
+    codes = np.zeros((N, K // 2), dtype=np.uint8)
+    gscale = np.zeros((N, G), dtype=np.uint16)
+    gzero = np.zeros((N, G), dtype=np.uint8)
+    s_w = np.zeros(N if per_channel else 1, dtype=np.float32)
+    rc = lib.oracle_quantize_weight_rtn(_ptr(W), N, K, group, int(symmetric), int(pow2),
+                                        int(per_channel), _ptr(codes), _ptr(gscale), _ptr(gzero),
+                                        _ptr(s_w))
+    if rc != 0:
+        raise ValueError("oracle_quantize_weight_rtn: bad arguments")
+    return codes, gscale, (None if symmetric else gzero), s_w
+
+
+def dequant_weight(codes, gscale, gzero=None, group=128):
+    """Eq. 10: E4M3 bytes [N,K]."""
+    lib = _load()
+    codes = _c(codes, np.uint8)
+    gscale = _c(gscale, np.uint16)
+    N, Kh = codes.shape
+    K = Kh * 2
+    if gzero is not None:
+        gzero = _c(gzero, np.uint8)
+    w8 = np.empty((N, K), dtype=np.uint8)
+    rc = lib.oracle_dequant_weight(_ptr(codes), _ptr(gscale), _ptr(gzero), N, K, group, _ptr(w8))
+    if rc != 0:
+        raise ValueError("oracle_dequant_weight: bad arguments")
+    return w8
+
+
+def quantize_act(x_bf16, scale_mode=0, static_scale=None):
+    """Eq. 13 per token.  x_bf16: uint16 [M,K].  Returns (x8 u8 [M,K], s_x fp32 [M])."""
+    lib = _load()
+    x = _c(x_bf16, np.uint16)
+    M, K = x.shape
+    x8 = np.empty((M, K), dtype=np.uint8)
+    s_x = np.empty(M, dtype=np.float32)
+    ss = None if static_scale is None else np.array([static_scale], dtype=np.float32)
+    rc = lib.oracle_quantize_act(_ptr(x), M, K, K, _ptr(x8), K, _ptr(s_x), int(scale_mode), _ptr(ss))
+    if rc != 0:
+        raise ValueError("oracle_quantize_act: bad arguments")
+    return x8, s_x
+
+
+def linear(x8, s_x, w8, s_w, cols=None, want=("y64", "y32", "ybf16", "yabs")):
+    """Exact FP8 dot products with Eq. 4 / Eq. 11 scales.  Returns a dict of [M, N or len(cols)]."""
+    lib = _load()
+    x8 = _c(x8, np.uint8)
+    w8 = _c(w8, np.uint8)
+    s_x = _c(s_x, np.float32)
+    s_w = _c(s_w, np.float32)
+    M, K = x8.shape
+    N = w8.shape[0]
+    assert w8.shape[1] == K
+    sw_stride = 0 if s_w.size == 1 else 1
+    if sw_stride:
+        assert s_w.size == N
+    if cols is not None:
+        cols = _c(cols, np.int64)
+        NC = cols.size
+    else:
+        NC = N
+    out = {}
+    if "y64" in want:
+        out["y64"] = np.empty((M, NC), dtype=np.float64)
+    if "y32" in want:
+        out["y32"] = np.empty((M, NC), dtype=np.float32)
+    if "ybf16" in want:
+        out["ybf16"] = np.empty((M, NC), dtype=np.uint16)
+    if "yabs" in want:
+        out["yabs"] = np.empty((M, NC), dtype=np.float64)
+    rc = lib.oracle_linear(_ptr(x8), K, _ptr(s_x), M, _ptr(w8), _ptr(s_w), sw_stride, N, K,
+                           _ptr(cols), NC, _ptr(out.get("y64")), _ptr(out.get("y32")),
+                           _ptr(out.get("ybf16")), _ptr(out.get("yabs")))
+    if rc != 0:
+        raise ValueError("oracle_linear: bad arguments")
+    return out
+
+
+def forward(x_bf16, codes, gscale, gzero, s_w, group=128, scale_mode=0, cols=None):
+    """Whole inference path of Sec. 3: Eq. 13 -> Eq. 10 -> FP8 matmul -> Eq. 4/11."""
+    x8, s_x = quantize_act(x_bf16, scale_mode)
+    w8 = dequant_weight(codes, gscale, gzero, group)
+    out = linear(x8, s_x, w8, s_w, cols)
+    out["x8"], out["s_x"], out["w8"] = x8, s_x, w8
+    return out
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())

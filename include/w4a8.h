@@ -1,0 +1,153 @@
+/*
+ * w4a8.h -- C ABI of the B200 (sm_100a) W4A8 linear-layer library.
+ *
+ * The library implements the inference flow of Sec. 3 of "Dual Precision Quantization":
+ * weights stored as INT4 codes with group-wise scales are dequantized to FP8 E4M3 (Eq. 10),
+ * activations are quantized from BF16 to FP8 (Eq. 13), the product runs as an FP8 matrix
+ * multiplication with FP32 accumulation and the result is rescaled (Eq. 4, Eq. 11) to BF16.
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named *_dev / unqualified tensor pointers are DEVICE pointers owned by the
+ *     caller (any allocator); pointers named *_host are HOST pointers.  The library never
+ *     allocates or frees device memory and keeps no tensor state between calls.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and the call returns
+ *     without synchronising, unless stated otherwise.
+ *   - Return value: W4A8_OK (0) or a negative W4A8_ERR_* code.  Arguments are validated before
+ *     anything is launched; on error nothing has been enqueued.
+ *   - Tensor formats
+ *       X      BF16  [M][ldx]      activations, row = token                       (Sec. 3)
+ *       X8     E4M3  [M][ldx8]     bytes, OCP "fn" variant, max finite 448        (Sec. 2.2, 4.1)
+ *       s_x    FP32  [M]           per-token activation scale                      (Eq. 13)
+ *       codes  u8    [N][K/2]      INT4 codes u in 0..15, element k in byte k/2,
+ *                                  even k in the low nibble; row = output channel  (Eq. 9)
+ *       gscale BF16  [N][K/128]    group scale s_g, groups of 128 consecutive k    (Eq. 8, Eq. 14)
+ *       gzero  u8    [N][K/128]    zero-point z_g in 0..15; NULL = symmetric, z=8  (Eq. 8, Eq. 1)
+ *       s_w    FP32  [N] or [1]    weight FP8 scale, per channel or per tensor     (Eq. 6)
+ *       W8     E4M3  [N][K]        dequantized weights                             (Eq. 10)
+ *       Y      BF16 or FP32 [M][ldy]                                               (Sec. 3)
+ *   - Shape rules: group must be 128, K % 128 == 0, N % 16 == 0, M >= 1.  Base pointers must be
+ *     16-byte aligned and leading dimensions must keep rows 16-byte aligned.
+ */
+#ifndef W4A8_H
+#define W4A8_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define W4A8_OK 0
+#define W4A8_ERR_INVALID_ARG (-1)         /* NULL pointer, non-positive size, unknown enum */
+#define W4A8_ERR_BAD_SHAPE (-2)           /* K % 128, group != 128, N % 16, ... */
+#define W4A8_ERR_BAD_ALIGNMENT (-3)       /* pointer or leading dimension not 16-byte aligned */
+#define W4A8_ERR_WORKSPACE_TOO_SMALL (-4)
+#define W4A8_ERR_UNSUPPORTED_DEVICE (-5)  /* current device is not compute capability 10.x */
+#define W4A8_ERR_CUDA (-6)                /* a CUDA runtime / driver call failed */
+#define W4A8_ERR_TIMEOUT (-7)             /* a bounded device-side wait gave up (see w4a8_query_device_status) */
+
+#define W4A8_SCALE_EXACT 0 /* s_x = amax / 448 */
+#define W4A8_SCALE_POW2 1  /* s_x rounded up to a power of two (Sec. 2.2) */
+
+#define W4A8_OUT_BF16 0
+#define W4A8_OUT_FP32 1
+
+#define W4A8_ALGO_AUTO 0
+#define W4A8_ALGO_SIMT 1 /* plain CUDA-core kernel: slow, for cross-checks */
+#define W4A8_ALGO_UMMA 2 /* TMA + tcgen05 kernel */
+
+/*
+ * Activation FP8 quantization, Eq. 13 (with Eq. 3), one scale per token:
+ *   amax = max_k |X[m][k]|;  s_x[m] = amax / 448 (fp32 division; 1 when the row is all zero);
+ *   X8[m][k] = nearest_E4M3( X[m][k] * (448 / amax) )   -- one fp32 multiply, round-to-nearest-even,
+ *   saturating at +-448.  scale_mode W4A8_SCALE_POW2 rounds s_x up to a power of two and scales
+ *   exactly.  static_scale (device pointer to one float) != NULL selects the paper's static
+ *   per-tensor mode: s_x[m] = *static_scale for every row, values beyond the range saturate.
+ * K % 16 == 0; ldx % 8 == 0; ldx8 % 16 == 0.  Inputs must be finite.
+ */
+int w4a8_quantize_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* x8,
+                      int64_t ldx8, float* s_x, int scale_mode, const float* static_scale,
+                      void* stream);
+
+/*
+ * INT4 -> FP8 weight dequantization, Eq. 10 (Eq. 14 per group):
+ *   W8[n][k] = nearest_E4M3( (u[n][k] - z_g) * s_g ),  g = k / 128,
+ * a single rounding (to nearest even, saturating) of the exact product.
+ */
+int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
+                        int64_t N, int64_t K, int group, uint8_t* w8, void* stream);
+
+/*
+ * The W4A8 linear layer of Sec. 3 on already-quantized activations:
+ *   Y[m][n] = s_x[m] * s_w[n*sw_stride] * sum_k X8[m][k] * W8[n][k]     (Eq. 4, Eq. 11)
+ * with W8 produced on the fly from (codes, gscale, gzero) exactly as w4a8_dequant_weight
+ * defines it, FP8 x FP8 products accumulated in FP32, output rounded to BF16 (out_dtype 0) or
+ * kept in FP32 (out_dtype 1).  sw_stride is 1 (per channel) or 0 (per tensor).
+ * `workspace` holds split-K partial sums when the library splits the reduction (small M);
+ * it needs w4a8_linear_workspace_bytes(M, N, K) bytes, is written before it is read and may be
+ * NULL when that size is 0.  Calls that share a workspace must not overlap on the device.
+ */
+int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride,
+                int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of workspace w4a8_linear needs for this problem (0 when no split is used). */
+size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/*
+ * Same computation as w4a8_linear with the kernel choice exposed, for cross-checks and tuning:
+ * algo is W4A8_ALGO_*; split_k <= 0 lets the library choose, otherwise it is the number of
+ * K slices (must divide K/128).  Workspace need: w4a8_linear_ex_workspace_bytes.
+ */
+int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
+                   const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
+                   const float* s_w, int sw_stride, int64_t N, int64_t K, int group, void* y,
+                   int64_t ldy, int out_dtype, void* workspace, size_t workspace_bytes, int algo,
+                   int split_k, void* stream);
+size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k);
+
+/*
+ * Offline round-to-nearest weight quantizer (Eq. 6 -> 7 -> 8 -> 9, no error compensation),
+ * so that a caller can produce the stored format on the device.  W is FP32 [N][K].
+ *   symmetric != 0: s_g = max|w8| / 7, u = round(w8 / s_g) + 8 (codes 1..15), gzero may be NULL;
+ *   symmetric == 0: Eq. 8 / Eq. 9 with the range widened to contain 0; gzero required.
+ *   pow2 != 0: s_g rounded up to a power of two.  per_channel != 0: s_w has N entries, else 1.
+ * Group scales are rounded to BF16 before the codes are computed; the integer rounding is
+ * half-to-even.  Enqueues several kernels on `stream`.
+ */
+int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, int symmetric,
+                             int pow2, int per_channel, uint8_t* codes, void* gscale_bf16,
+                             uint8_t* gzero, float* s_w, void* stream);
+
+/*
+ * Whole layer from HOST activations to HOST output (Sec. 3 flow end to end): copies
+ * x_host (BF16 [M][K], ideally pinned) to x_dev, runs w4a8_quantize_act and w4a8_linear, and
+ * copies y_dev (BF16 [M][N]) to y_host, all enqueued on `stream`; the caller synchronises the
+ * stream before reading y_host.  Weights stay resident on the device.  Scratch device buffers
+ * are the caller's: x_dev (2*M*K bytes), x8_dev (M*K), s_x_dev (4*M), y_dev (2*M*N), workspace.
+ */
+int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* codes,
+                      const void* gscale_bf16, const uint8_t* gzero, const float* s_w,
+                      int sw_stride, int64_t N, int64_t K, int group, void* y_host_bf16,
+                      void* x_dev, uint8_t* x8_dev, float* s_x_dev, void* y_dev, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/*
+ * Reads and clears the device-side status word (synchronises the device).  *flags receives a
+ * bit mask: bit 0 = a bounded wait inside a kernel gave up.  Returns W4A8_ERR_TIMEOUT when any
+ * bit was set, W4A8_OK otherwise.
+ */
+int w4a8_query_device_status(unsigned int* flags_host);
+
+/* Number of kernels the library has launched from this process (for accounting). */
+uint64_t w4a8_launch_count(void);
+
+/* Static string for a status code. */
+const char* w4a8_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,220 @@
+"""ctypes binding of the C-ABI library declared in include/w4a8.h.
+
+Argument marshalling only: every step of the W4A8 path (Eq. 13 activation quantization, Eq. 10
+weight dequantization, FP8 matmul, Eq. 4 / Eq. 11 epilogue) runs in the library's CUDA kernels.
+PyTorch supplies device buffers and the current stream.  There is no CPU fallback: if the
+library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libw4a8_b200.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_BAD_ALIGNMENT, ERR_WORKSPACE_TOO_SMALL = -1, -2, -3, -4
+ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
+SCALE_EXACT, SCALE_POW2 = 0, 1
+OUT_BF16, OUT_FP32 = 0, 1
+ALGO_AUTO, ALGO_SIMT, ALGO_UMMA = 0, 1, 2
+GROUP = 128
+
+# Every symbol include/w4a8.h declares.
+EXPORTS = (
+    "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
+    "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_quantize_weight_rtn",
+    "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
+)
+
+_lib = None
+
+
+class W4A8Error(RuntimeError):
+    def __init__(self, fn, status):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (fn, status, status_string(status)))
+
+
+def lib():
+    """The loaded shared library with argument types set.  Raises when it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "CUDA library %s is missing: build it with "
+            "`python -m paper_2505_14638_b200.build` (there is no fallback path)" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    c = ctypes
+    p, i64, i32, sz = c.c_void_p, c.c_int64, c.c_int, c.c_size_t
+    L.w4a8_quantize_act.restype = i32
+    L.w4a8_quantize_act.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p]
+    L.w4a8_dequant_weight.restype = i32
+    L.w4a8_dequant_weight.argtypes = [p, p, p, i64, i64, i32, p, p]
+    L.w4a8_linear.restype = i32
+    L.w4a8_linear.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz, p]
+    L.w4a8_linear_workspace_bytes.restype = sz
+    L.w4a8_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.w4a8_linear_ex.restype = i32
+    L.w4a8_linear_ex.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz,
+                                 i32, i32, p]
+    L.w4a8_linear_ex_workspace_bytes.restype = sz
+    L.w4a8_linear_ex_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
+    L.w4a8_quantize_weight_rtn.restype = i32
+    L.w4a8_quantize_weight_rtn.argtypes = [p, i64, i64, i32, i32, i32, i32, p, p, p, p, p]
+    L.w4a8_forward_host.restype = i32
+    L.w4a8_forward_host.argtypes = [p, i64, p, p, p, p, i32, i64, i64, i32, p, p, p, p, p, p, sz, p]
+    L.w4a8_query_device_status.restype = i32
+    L.w4a8_query_device_status.argtypes = [c.POINTER(c.c_uint)]
+    L.w4a8_launch_count.restype = c.c_uint64
+    L.w4a8_launch_count.argtypes = []
+    L.w4a8_status_string.restype = c.c_char_p
+    L.w4a8_status_string.argtypes = [i32]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().w4a8_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().w4a8_launch_count())
+
+
+def query_device_status() -> int:
+    """Synchronises; returns the device status bit mask (0 = clean) and clears it."""
+    flags = ctypes.c_uint(0)
+    rc = lib().w4a8_query_device_status(ctypes.byref(flags))
+    if rc not in (OK, ERR_TIMEOUT):
+        raise W4A8Error("w4a8_query_device_status", rc)
+    return int(flags.value)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(fn, rc):
+    if rc != OK:
+        raise W4A8Error(fn, rc)
+
+
+def quantize_act(x, scale_mode=SCALE_EXACT, static_scale=None, out=None):
+    """w4a8_quantize_act: x BF16 [M, K] (row stride in elements = x.stride(0)).
+    Returns (x8 uint8 [M, K], s_x float32 [M])."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    if out is None:
+        x8 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+        s_x = torch.empty((M,), dtype=torch.float32, device=x.device)
+    else:
+        x8, s_x = out
+    rc = lib().w4a8_quantize_act(_ptr(x), M, K, x.stride(0), _ptr(x8), x8.stride(0), _ptr(s_x),
+                                 int(scale_mode), _ptr(static_scale), _stream())
+    _check("w4a8_quantize_act", rc)
+    return x8, s_x
+
+
+def dequant_weight(codes, gscale, gzero=None, out=None):
+    """w4a8_dequant_weight: codes uint8 [N, K/2], gscale BF16 [N, K/128], gzero uint8 or None.
+    Returns E4M3 bytes uint8 [N, K]."""
+    import torch
+    N, Kh = codes.shape
+    K = Kh * 2
+    w8 = out if out is not None else torch.empty((N, K), dtype=torch.uint8, device=codes.device)
+    rc = lib().w4a8_dequant_weight(_ptr(codes), _ptr(gscale), _ptr(gzero), N, K, GROUP, _ptr(w8),
+                                   _stream())
+    _check("w4a8_dequant_weight", rc)
+    return w8
+
+
+def linear_workspace_bytes(M, N, K, algo=ALGO_AUTO, split_k=0) -> int:
+    return int(lib().w4a8_linear_ex_workspace_bytes(M, N, K, algo, split_k))
+
+
+def linear(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, workspace=None,
+           algo=ALGO_AUTO, split_k=0):
+    """w4a8_linear / w4a8_linear_ex: returns Y [M, N] (BF16 or FP32)."""
+    import torch
+    M, K = x8.shape
+    N = codes.shape[0]
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, N), dtype=dt, device=x8.device)
+    need = linear_workspace_bytes(M, N, K, algo, split_k)
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty((need,), dtype=torch.uint8, device=x8.device)
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    sw_stride = 0 if s_w.numel() == 1 else 1
+    L = lib()
+    if algo == ALGO_AUTO and split_k == 0:
+        rc = L.w4a8_linear(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(codes), _ptr(gscale),
+                           _ptr(gzero), _ptr(s_w), sw_stride, N, K, GROUP, _ptr(out),
+                           out.stride(0), int(out_dtype), _ptr(workspace), wbytes, _stream())
+        _check("w4a8_linear", rc)
+    else:
+        rc = L.w4a8_linear_ex(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(codes), _ptr(gscale),
+                              _ptr(gzero), _ptr(s_w), sw_stride, N, K, GROUP, _ptr(out),
+                              out.stride(0), int(out_dtype), _ptr(workspace), wbytes, int(algo),
+                              int(split_k), _stream())
+        _check("w4a8_linear_ex", rc)
+    return out
+
+
+def quantize_weight_rtn(W, symmetric=True, pow2=False, per_channel=False):
+    """w4a8_quantize_weight_rtn: W float32 [N, K] on the device.
+    Returns (codes, gscale BF16, gzero or None, s_w)."""
+    import torch
+    N, K = W.shape
+    dev = W.device
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    gscale = torch.empty((N, K // GROUP), dtype=torch.bfloat16, device=dev)
+    gzero = None if symmetric else torch.empty((N, K // GROUP), dtype=torch.uint8, device=dev)
+    s_w = torch.empty((N if per_channel else 1,), dtype=torch.float32, device=dev)
+    rc = lib().w4a8_quantize_weight_rtn(_ptr(W), N, K, GROUP, int(symmetric), int(pow2),
+                                        int(per_channel), _ptr(codes), _ptr(gscale), _ptr(gzero),
+                                        _ptr(s_w), _stream())
+    _check("w4a8_quantize_weight_rtn", rc)
+    return codes, gscale, gzero, s_w
+
+
+class HostForward:
+    """w4a8_forward_host with its device scratch buffers allocated once: activations come from
+    and results go to pinned host memory, weights stay on the device."""
+
+    def __init__(self, M, codes, gscale, gzero, s_w):
+        import torch
+        self.M = M
+        self.N, Kh = codes.shape
+        self.K = Kh * 2
+        dev = codes.device
+        self.codes, self.gscale, self.gzero, self.s_w = codes, gscale, gzero, s_w
+        self.x_dev = torch.empty((M, self.K), dtype=torch.bfloat16, device=dev)
+        self.x8 = torch.empty((M, self.K), dtype=torch.uint8, device=dev)
+        self.s_x = torch.empty((M,), dtype=torch.float32, device=dev)
+        self.y_dev = torch.empty((M, self.N), dtype=torch.bfloat16, device=dev)
+        need = linear_workspace_bytes(M, self.N, self.K)
+        self.ws = torch.empty((max(need, 16),), dtype=torch.uint8, device=dev)
+        self.y_host = torch.empty((M, self.N), dtype=torch.bfloat16).pin_memory()
+        self.h2d_bytes = M * self.K * 2
+        self.d2h_bytes = M * self.N * 2
+
+    def __call__(self, x_host):
+        """x_host: pinned BF16 [M, K] host tensor.  Enqueues everything; returns the pinned
+        output tensor, valid after the current stream is synchronised."""
+        rc = lib().w4a8_forward_host(
+            ctypes.c_void_p(x_host.data_ptr()), self.M, _ptr(self.codes), _ptr(self.gscale),
+            _ptr(self.gzero), _ptr(self.s_w), 0 if self.s_w.numel() == 1 else 1, self.N, self.K,
+            GROUP, ctypes.c_void_p(self.y_host.data_ptr()), _ptr(self.x_dev), _ptr(self.x8),
+            _ptr(self.s_x), _ptr(self.y_dev), _ptr(self.ws), self.ws.numel(), _stream())
+        _check("w4a8_forward_host", rc)
+        return self.y_host

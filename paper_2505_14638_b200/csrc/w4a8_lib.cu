@@ -1,0 +1,395 @@
+// C-ABI entry points of the W4A8 library (see include/w4a8.h): argument validation, kernel
+// selection, TMA descriptor set-up and launches.  Nothing here allocates device memory.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <mutex>
+
+#include "../../include/w4a8.h"
+#include "w4a8_linear_umma.cuh"
+#include "w4a8_simple_kernels.cuh"
+
+namespace w4a8 {
+
+__device__ unsigned int g_status_word = 0;  // bit mask, see kStatus*
+
+static std::atomic<uint64_t> g_launches{0};
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W4A8_ERR_CUDA;
+    static std::mutex mu;
+    static int cached_dev = -1, cached_major = 0;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached_dev != dev) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return W4A8_ERR_CUDA;
+        cached_dev = dev;
+        cached_major = major;
+    }
+    return cached_major == 10 ? W4A8_OK : W4A8_ERR_UNSUPPORTED_DEVICE;
+}
+
+static unsigned int* status_word_ptr() {
+    // Address of the device status word on the current device (looked up once per device).
+    static std::mutex mu;
+    static unsigned int* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<unsigned int*>(p);
+    }
+    return ptrs[dev];
+}
+
+static inline int launch_status() {
+    return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// 2-D uint8 tensor [rows][cols] with row pitch `pitch` bytes; box = box_cols x box_rows.
+static bool make_tmap_u8_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch,
+                            uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------------------ linear plan
+struct LinearPlan {
+    int algo;      // W4A8_ALGO_SIMT or W4A8_ALGO_UMMA
+    int bnx;       // token tile of the UMMA kernel
+    int split_k;   // number of K slices
+    size_t workspace_bytes;
+};
+
+static int pick_bnx(int64_t M) {
+    if (M <= 16) return 16;
+    if (M <= 32) return 32;
+    if (M <= 64) return 64;
+    if (M <= 128) return 128;
+    return 256;
+}
+
+static int auto_split_k(int64_t M, int64_t N, int64_t K, int bnx) {
+    const int64_t tiles = ((N + 127) / 128) * ((M + bnx - 1) / bnx);
+    const int64_t kb = K / 128;
+    if (M > 64 || tiles >= 148) return 1;
+    // Fill about two CTAs per SM while keeping at least four K blocks per slice.
+    int best = 1;
+    for (int s = 1; s <= kb; ++s) {
+        if (kb % s != 0) continue;
+        if (kb / s < 4) break;
+        if (tiles * s <= 2 * 148) best = s;
+    }
+    return best;
+}
+
+static int make_plan(int64_t M, int64_t N, int64_t K, int algo, int split_k, LinearPlan* plan) {
+    if (algo == W4A8_ALGO_AUTO) algo = W4A8_ALGO_UMMA;
+    if (algo != W4A8_ALGO_SIMT && algo != W4A8_ALGO_UMMA) return W4A8_ERR_INVALID_ARG;
+    plan->algo = algo;
+    plan->bnx = pick_bnx(M);
+    plan->split_k = 1;
+    plan->workspace_bytes = 0;
+    if (algo == W4A8_ALGO_UMMA) {
+        int s = split_k > 0 ? split_k : auto_split_k(M, N, K, plan->bnx);
+        if ((K / 128) % s != 0) return W4A8_ERR_BAD_SHAPE;
+        plan->split_k = s;
+        if (s > 1) plan->workspace_bytes = (size_t)s * (size_t)M * (size_t)N * sizeof(float);
+    } else if (split_k > 1) {
+        return W4A8_ERR_INVALID_ARG;
+    }
+    return W4A8_OK;
+}
+
+template <class Cfg>
+static int launch_umma(const CUtensorMap& tw, const CUtensorMap& tx, const uint16_t* gscale, const uint8_t* gzero,
+                       const float* s_x, const float* s_w, int sw_stride, void* y, int64_t ldy, int out_dtype,
+                       float* partial, int M, int N, int K, int split_k, cudaStream_t st) {
+    auto kern = linear_umma_kernel<Cfg>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    unsigned int* status = status_word_ptr();
+    if (!status) return W4A8_ERR_CUDA;
+    dim3 grid((unsigned)((N + 127) / 128), (unsigned)((M + Cfg::BNX - 1) / Cfg::BNX), (unsigned)split_k);
+    kern<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tw, tx, gscale, gzero, s_x, s_w, sw_stride, y, ldy,
+                                                       out_dtype, partial, M, N, K, (K / 128) / split_k, status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                       const void* gscale, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
+                       int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
+                       size_t workspace_bytes, int algo, int split_k, cudaStream_t st) {
+    if (!x8 || !s_x || !codes || !gscale || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
+    if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
+    if (ldx8 < K || ldy < N) return W4A8_ERR_BAD_SHAPE;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(x8) || !aligned16(codes) || !aligned16(y) || (ldx8 % 16) != 0) return W4A8_ERR_BAD_ALIGNMENT;
+    if ((reinterpret_cast<uintptr_t>(gscale) & 1u) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
+        (reinterpret_cast<uintptr_t>(s_w) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    LinearPlan plan;
+    int rc = make_plan(M, N, K, algo, split_k, &plan);
+    if (rc != W4A8_OK) return rc;
+    if (plan.workspace_bytes > 0) {
+        if (!workspace || workspace_bytes < plan.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
+    }
+    rc = check_device();
+    if (rc != W4A8_OK) return rc;
+
+    const uint16_t* gs = static_cast<const uint16_t*>(gscale);
+    if (plan.algo == W4A8_ALGO_SIMT) {
+        dim3 grid((unsigned)((N + 31) / 32), (unsigned)((M + 7) / 8));
+        linear_simt_kernel<<<grid, 256, 0, st>>>(x8, ldx8, s_x, M, codes, gs, gzero, s_w, sw_stride, N, K, y, ldy,
+                                                 out_dtype);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return launch_status();
+    }
+
+    CUtensorMap tw, tx;
+    if (!make_tmap_u8_2d(&tw, codes, (uint64_t)N, (uint64_t)(K / 2), (uint64_t)(K / 2), 64, 128,
+                         CU_TENSOR_MAP_SWIZZLE_64B))
+        return W4A8_ERR_CUDA;
+    if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)plan.bnx,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    float* partial = plan.split_k > 1 ? static_cast<float*>(workspace) : nullptr;
+    const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+#define W4A8_LAUNCH(BNX, STG)                                                                                 \
+    rc = launch_umma<UmmaCfg<BNX, STG>>(tw, tx, gs, gzero, s_x, s_w, sw_stride, y, ldy, out_dtype, partial, Mi, \
+                                        Ni, Ki, plan.split_k, st)
+    switch (plan.bnx) {
+        case 16: W4A8_LAUNCH(16, 4); break;
+        case 32: W4A8_LAUNCH(32, 4); break;
+        case 64: W4A8_LAUNCH(64, 6); break;
+        case 128: W4A8_LAUNCH(128, 5); break;
+        default: W4A8_LAUNCH(256, 4); break;
+    }
+#undef W4A8_LAUNCH
+    if (rc != W4A8_OK) return rc;
+    if (plan.split_k > 1) {
+        int64_t total = M * N;
+        unsigned blocks = (unsigned)((total + 255) / 256);
+        if (blocks > 148u * 8u) blocks = 148u * 8u;
+        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, plan.split_k, M, N, s_x, s_w, sw_stride, y, ldy,
+                                                     out_dtype);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        rc = launch_status();
+    }
+    return rc;
+}
+
+static int quantize_act_impl(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* x8, int64_t ldx8,
+                             float* s_x, int scale_mode, const float* static_scale, cudaStream_t st) {
+    if (!x || !x8 || !s_x) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (scale_mode != W4A8_SCALE_EXACT && scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
+    if (K % 16 != 0 || ldx < K || ldx8 < K || M > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(x) || !aligned16(x8) || (ldx % 8) != 0 || (ldx8 % 16) != 0 ||
+        (reinterpret_cast<uintptr_t>(s_x) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const uint16_t* xs = static_cast<const uint16_t*>(x);
+    const int64_t nchunks = K / 16;
+    const unsigned rows = (unsigned)M;
+#define W4A8_AQ(T, C) \
+    act_quant_kernel<T, C><<<rows, T, 0, st>>>(xs, K, ldx, x8, ldx8, s_x, scale_mode, static_scale)
+    if (nchunks <= 32) W4A8_AQ(32, 1);
+    else if (nchunks <= 64) W4A8_AQ(64, 1);
+    else if (nchunks <= 128) W4A8_AQ(128, 1);
+    else if (nchunks <= 256) W4A8_AQ(256, 1);
+    else if (nchunks <= 512) W4A8_AQ(256, 2);
+    else if (nchunks <= 1024) W4A8_AQ(256, 4);
+    else act_quant_kernel_2pass<<<rows, 256, 0, st>>>(xs, K, ldx, x8, ldx8, s_x, scale_mode, static_scale);
+#undef W4A8_AQ
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+}  // namespace w4a8
+
+using namespace w4a8;
+
+extern "C" {
+
+int w4a8_quantize_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* x8, int64_t ldx8,
+                      float* s_x, int scale_mode, const float* static_scale, void* stream) {
+    return quantize_act_impl(x_bf16, M, K, ldx, x8, ldx8, s_x, scale_mode, static_scale,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero, int64_t N,
+                        int64_t K, int group, uint8_t* w8, void* stream) {
+    if (!codes || !gscale_bf16 || !w8) return W4A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(codes) || !aligned16(w8) || (reinterpret_cast<uintptr_t>(gscale_bf16) & 1u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    int64_t units = N * (K / 32);
+    unsigned blocks = (unsigned)((units + 255) / 256 < 148 * 16 ? (units + 255) / 256 : 148 * 16);
+    dequant_weight_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        codes, static_cast<const uint16_t*>(gscale_bf16), gzero, N, K, w8);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
+                int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
+                size_t workspace_bytes, void* stream) {
+    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y, ldy, out_dtype,
+                       workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, static_cast<cudaStream_t>(stream));
+}
+
+size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
+}
+
+int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                   const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
+                   int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
+                   size_t workspace_bytes, int algo, int split_k, void* stream) {
+    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y, ldy, out_dtype,
+                       workspace, workspace_bytes, algo, split_k, static_cast<cudaStream_t>(stream));
+}
+
+size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k) {
+    if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    LinearPlan plan;
+    if (make_plan(M, N, K, algo, split_k, &plan) != W4A8_OK) return 0;
+    return plan.workspace_bytes;
+}
+
+int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, int symmetric, int pow2,
+                             int per_channel, uint8_t* codes, void* gscale_bf16, uint8_t* gzero, float* s_w,
+                             void* stream) {
+    if (!W || !codes || !gscale_bf16 || !s_w) return W4A8_ERR_INVALID_ARG;
+    if (!symmetric && !gzero) return W4A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(W) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(gscale_bf16) & 1u) ||
+        (reinterpret_cast<uintptr_t>(s_w) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int* amax_bits = reinterpret_cast<unsigned int*>(s_w);
+    if (per_channel) {
+        absmax_f32_kernel<<<(unsigned)N, 256, 0, st>>>(W, N, K, 1, amax_bits);
+    } else {
+        if (cudaMemsetAsync(s_w, 0, sizeof(float), st) != cudaSuccess) return W4A8_ERR_CUDA;
+        int64_t total = N * K;
+        unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+        absmax_f32_kernel<<<blocks, 256, 0, st>>>(W, N, K, 0, amax_bits);
+    }
+    int64_t ns = per_channel ? N : 1;
+    amax_to_scale_kernel<<<(unsigned)((ns + 255) / 256), 256, 0, st>>>(s_w, ns);
+    int64_t warps = N * (K / 128);
+    rtn_quant_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(W, N, K, symmetric, pow2, per_channel, s_w, codes,
+                                                                  static_cast<uint16_t*>(gscale_bf16), gzero);
+    g_launches.fetch_add(3, std::memory_order_relaxed);
+    return launch_status();
+}
+
+int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* codes, const void* gscale_bf16,
+                      const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, int group,
+                      void* y_host_bf16, void* x_dev, uint8_t* x8_dev, float* s_x_dev, void* y_dev,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (!x_host_bf16 || !y_host_bf16 || !x_dev || !x8_dev || !s_x_dev || !y_dev) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Validate the two stages before anything is enqueued.
+    LinearPlan plan;
+    int rc = make_plan(M, N, K, W4A8_ALGO_AUTO, 0, &plan);
+    if (rc != W4A8_OK) return rc;
+    if (plan.workspace_bytes > 0 && (!workspace || workspace_bytes < plan.workspace_bytes))
+        return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if (!codes || !gscale_bf16 || !s_w) return W4A8_ERR_INVALID_ARG;
+    if (!aligned16(x_dev) || !aligned16(x8_dev) || !aligned16(y_dev) || !aligned16(codes))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    rc = quantize_act_impl(x_dev, M, K, K, x8_dev, K, s_x_dev, W4A8_SCALE_EXACT, nullptr, st);
+    if (rc != W4A8_OK) return rc;
+    rc = linear_impl(x8_dev, K, s_x_dev, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y_dev, N,
+                     W4A8_OUT_BF16, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, st);
+    if (rc != W4A8_OK) return rc;
+    if (cudaMemcpyAsync(y_host_bf16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    return W4A8_OK;
+}
+
+int w4a8_query_device_status(unsigned int* flags_host) {
+    if (!flags_host) return W4A8_ERR_INVALID_ARG;
+    unsigned int v = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return W4A8_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof v) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_status_word, &zero, sizeof zero) != cudaSuccess) return W4A8_ERR_CUDA;
+    *flags_host = v;
+    return (v != 0) ? W4A8_ERR_TIMEOUT : W4A8_OK;
+}
+
+uint64_t w4a8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* w4a8_status_string(int status) {
+    switch (status) {
+        case W4A8_OK: return "ok";
+        case W4A8_ERR_INVALID_ARG: return "invalid argument";
+        case W4A8_ERR_BAD_SHAPE: return "unsupported shape";
+        case W4A8_ERR_BAD_ALIGNMENT: return "pointer or leading dimension not 16-byte aligned";
+        case W4A8_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case W4A8_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
+        case W4A8_ERR_CUDA: return "CUDA call failed";
+        case W4A8_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,363 @@
+// Bandwidth-bound and helper kernels of the W4A8 path: per-token activation FP8 quantization
+// (Eq. 13), standalone INT4 -> FP8 weight dequantization (Eq. 10), the offline round-to-nearest
+// weight quantizer (Eq. 6-9), a plain CUDA-core linear used for cross-checks and the split-K
+// reduction with the Eq. 4 / Eq. 11 epilogue.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "w4a8_common.cuh"
+
+namespace w4a8 {
+
+// ---------------------------------------------------------------------------------------------
+// Activation quantization, Eq. 13: one CTA per token.  The row is read once with 128-bit loads
+// and kept in registers between the absmax pass and the convert pass (2 B in, 1 B out / element).
+// ---------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float absmax_bf16x8(const uint4& v, float m) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        m = fmaxf(m, fabsf(__uint_as_float(w[i] << 16)));
+        m = fmaxf(m, fabsf(__uint_as_float(w[i] & 0xFFFF0000u)));
+    }
+    return m;
+}
+
+// Eight BF16 values scaled by inv (one fp32 multiply each) -> eight E4M3 bytes.
+__device__ __forceinline__ uint2 quant_bf16x8(const uint4& v, float inv) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), inv);
+        f[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), inv);
+    }
+    uint2 r;
+    r.x = cvt_e4m3x4(f[0], f[1], f[2], f[3]);
+    r.y = cvt_e4m3x4(f[4], f[5], f[6], f[7]);
+    return r;
+}
+
+__device__ __forceinline__ float pow2_ceil(float s) {
+    int e;
+    float m = frexpf(s, &e);
+    return (m == 0.5f) ? s : ldexpf(1.0f, e);
+}
+
+// Block-wide max of non-negative floats; result valid in every thread.
+template <int THREADS>
+__device__ __forceinline__ float block_max(float m, float* red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    constexpr int NW = THREADS / 32;
+    if constexpr (NW > 1) {
+        int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        if (lane == 0) red[warp] = m;
+        __syncthreads();
+        float t = (lane < NW) ? red[lane] : 0.0f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t = fmaxf(t, __shfl_xor_sync(0xFFFFFFFFu, t, o));
+        m = t;
+    }
+    return m;
+}
+
+// THREADS threads per row, each caching NCH chunks of 16 elements (K <= THREADS*NCH*16).
+template <int THREADS, int NCH>
+__global__ void __launch_bounds__(THREADS)
+act_quant_kernel(const uint16_t* __restrict__ x, int64_t K, int64_t ldx, uint8_t* __restrict__ x8,
+                 int64_t ldx8, float* __restrict__ s_x, int scale_mode,
+                 const float* __restrict__ static_scale) {
+    __shared__ float red[32];
+    const int64_t row = blockIdx.x;
+    const int nchunks = (int)(K >> 4);
+    const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx);
+    uint4 v[NCH][2];
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = threadIdx.x + i * THREADS;
+        if (c < nchunks) {
+            v[i][0] = __ldg(src + 2 * c);
+            v[i][1] = __ldg(src + 2 * c + 1);
+            amax = absmax_bf16x8(v[i][0], amax);
+            amax = absmax_bf16x8(v[i][1], amax);
+        }
+    }
+    float s, inv;
+    if (static_scale != nullptr) {
+        s = __ldg(static_scale);
+        inv = __fdiv_rn(1.0f, s);
+    } else {
+        amax = block_max<THREADS>(amax, red);
+        if (amax == 0.0f) {
+            s = 1.0f;
+            inv = 1.0f;
+        } else if (scale_mode == W4A8_SCALE_POW2) {
+            s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
+            inv = __fdiv_rn(1.0f, s);
+        } else {
+            s = __fdiv_rn(amax, kE4M3Max);
+            inv = __fdiv_rn(kE4M3Max, amax);
+        }
+    }
+    if (threadIdx.x == 0) s_x[row] = s;
+    uint4* dst = reinterpret_cast<uint4*>(x8 + row * ldx8);
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = threadIdx.x + i * THREADS;
+        if (c < nchunks) {
+            uint2 a = quant_bf16x8(v[i][0], inv);
+            uint2 b = quant_bf16x8(v[i][1], inv);
+            dst[c] = make_uint4(a.x, a.y, b.x, b.y);
+        }
+    }
+}
+
+// Any K: the row is read twice (second read served by L2).
+__global__ void __launch_bounds__(256)
+act_quant_kernel_2pass(const uint16_t* __restrict__ x, int64_t K, int64_t ldx,
+                       uint8_t* __restrict__ x8, int64_t ldx8, float* __restrict__ s_x,
+                       int scale_mode, const float* __restrict__ static_scale) {
+    __shared__ float red[32];
+    const int64_t row = blockIdx.x;
+    const int nchunks = (int)(K >> 4);
+    const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx);
+    float s, inv;
+    if (static_scale != nullptr) {
+        s = __ldg(static_scale);
+        inv = __fdiv_rn(1.0f, s);
+    } else {
+        float amax = 0.0f;
+        for (int c = threadIdx.x; c < nchunks; c += 256) {
+            amax = absmax_bf16x8(__ldg(src + 2 * c), amax);
+            amax = absmax_bf16x8(__ldg(src + 2 * c + 1), amax);
+        }
+        amax = block_max<256>(amax, red);
+        if (amax == 0.0f) {
+            s = 1.0f;
+            inv = 1.0f;
+        } else if (scale_mode == W4A8_SCALE_POW2) {
+            s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
+            inv = __fdiv_rn(1.0f, s);
+        } else {
+            s = __fdiv_rn(amax, kE4M3Max);
+            inv = __fdiv_rn(kE4M3Max, amax);
+        }
+    }
+    if (threadIdx.x == 0) s_x[row] = s;
+    uint4* dst = reinterpret_cast<uint4*>(x8 + row * ldx8);
+    for (int c = threadIdx.x; c < nchunks; c += 256) {
+        uint2 a = quant_bf16x8(src[2 * c], inv);
+        uint2 b = quant_bf16x8(src[2 * c + 1], inv);
+        dst[c] = make_uint4(a.x, a.y, b.x, b.y);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Standalone weight dequantization, Eq. 10: each thread expands 16 bytes of codes (32 elements
+// of one group) to 32 E4M3 bytes through the per-group look-up table.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+dequant_weight_kernel(const uint8_t* __restrict__ codes, const uint16_t* __restrict__ gscale,
+                      const uint8_t* __restrict__ gzero, int64_t N, int64_t K,
+                      uint8_t* __restrict__ w8) {
+    const int64_t units_per_row = K >> 5;  // 32 elements per unit
+    const int64_t total = N * units_per_row;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total;
+         u += (int64_t)gridDim.x * blockDim.x) {
+        int64_t n = u / units_per_row;
+        int64_t c = u - n * units_per_row;
+        int64_t g = c >> 2;  // 4 units per group of 128
+        int64_t G = K >> 7;
+        float s = bf16_bits_to_float(gscale[n * G + g]);
+        int z = gzero ? (int)gzero[n * G + g] : 8;
+        DequantLut lut;
+        lut.build(s, z);
+        uint4 p = *reinterpret_cast<const uint4*>(codes + n * (K >> 1) + c * 16);
+        uint4 o0, o1;
+        lut.dequant8(p.x, o0.x, o0.y);
+        lut.dequant8(p.y, o0.z, o0.w);
+        lut.dequant8(p.z, o1.x, o1.y);
+        lut.dequant8(p.w, o1.z, o1.w);
+        uint4* dst = reinterpret_cast<uint4*>(w8 + n * K + c * 32);
+        dst[0] = o0;
+        dst[1] = o1;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Offline round-to-nearest quantizer, Eq. 6-9.  Every step is a single IEEE fp32 operation.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+absmax_f32_kernel(const float* __restrict__ W, int64_t rows, int64_t cols, int per_row,
+                  unsigned int* __restrict__ out_bits) {
+    // per_row: one CTA per row writes out_bits[row]; else grid-stride with an atomic max on the
+    // bit pattern (non-negative floats order like unsigned integers).
+    __shared__ float red[32];
+    float m = 0.0f;
+    if (per_row) {
+        const float* r = W + (int64_t)blockIdx.x * cols;
+        for (int64_t k = threadIdx.x; k < cols; k += 256) m = fmaxf(m, fabsf(r[k]));
+        m = block_max<256>(m, red);
+        if (threadIdx.x == 0) out_bits[blockIdx.x] = __float_as_uint(m);
+    } else {
+        int64_t total = rows * cols;
+        for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total;
+             i += (int64_t)gridDim.x * 256)
+            m = fmaxf(m, fabsf(W[i]));
+        m = block_max<256>(m, red);
+        if (threadIdx.x == 0) atomicMax(out_bits, __float_as_uint(m));
+    }
+}
+
+__global__ void amax_to_scale_kernel(float* s_w, int64_t n) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        float a = s_w[i];  // holds the absmax written by absmax_f32_kernel
+        s_w[i] = (a > 0.0f) ? __fdiv_rn(a, kE4M3Max) : 1.0f;  // Eq. 6
+    }
+}
+
+__device__ __forceinline__ float e4m3_roundtrip(float q) {
+    // nearest_Z(q) as a float (Eq. 7): encode, then decode exactly through f16.
+    uint32_t code = cvt_e4m3x2(0.0f, q) & 0xFFu;
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)code));
+    return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// One warp per (row, group of 128): lane l owns elements 4l..4l+3.
+__global__ void __launch_bounds__(256)
+rtn_quant_kernel(const float* __restrict__ W, int64_t N, int64_t K, int symmetric, int pow2,
+                 int per_channel, const float* __restrict__ s_w, uint8_t* __restrict__ codes,
+                 uint16_t* __restrict__ gscale, uint8_t* __restrict__ gzero) {
+    const int64_t G = K >> 7;
+    const int64_t wid = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (wid >= N * G) return;
+    const int64_t n = wid / G, g = wid - n * G;
+    const float sw = per_channel ? s_w[n] : s_w[0];
+    float4 w = *reinterpret_cast<const float4*>(W + n * K + g * 128 + lane * 4);
+    float v[4] = {w.x, w.y, w.z, w.w};
+    float lo = 0.0f, hi = 0.0f, amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[i] = e4m3_roundtrip(__fdiv_rn(v[i], sw));  // Eq. 7
+        lo = fminf(lo, v[i]);
+        hi = fmaxf(hi, v[i]);
+        amax = fmaxf(amax, fabsf(v[i]));
+    }
+    lo = warp_min(lo);
+    hi = warp_max(hi);
+    amax = warp_max(amax);
+    float s;
+    int z = 8;
+    if (symmetric)
+        s = (amax > 0.0f) ? __fdiv_rn(amax, 7.0f) : 1.0f;
+    else
+        s = (hi > lo) ? __fdiv_rn(__fsub_rn(hi, lo), 15.0f) : 1.0f;  // Eq. 8
+    if (pow2) s = pow2_ceil(s);
+    __nv_bfloat16 sb = __float2bfloat16_rn(s);
+    s = __bfloat162float(sb);
+    if (!symmetric) {
+        float zf = rintf(__fdiv_rn(-lo, s));  // Eq. 8
+        z = (int)fminf(fmaxf(zf, 0.0f), 15.0f);
+    }
+    uint32_t packed = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int u;
+        if (symmetric) {
+            float q = rintf(__fdiv_rn(v[i], s));
+            u = (int)fminf(fmaxf(q, -7.0f), 7.0f) + 8;
+        } else {
+            float q = rintf(__fadd_rn(__fdiv_rn(v[i], s), (float)z));  // Eq. 9
+            u = (int)fminf(fmaxf(q, 0.0f), 15.0f);
+        }
+        packed |= (uint32_t)u << (4 * i);
+    }
+    *reinterpret_cast<uint16_t*>(codes + n * (K >> 1) + g * 64 + lane * 2) = (uint16_t)packed;
+    if (lane == 0) {
+        gscale[n * G + g] = __bfloat16_as_ushort(sb);
+        if (gzero) gzero[n * G + g] = (uint8_t)z;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Plain CUDA-core linear (cross-check only): one thread per output element, weights dequantized
+// element by element with the direct formula of Eq. 10 (no look-up table), fp32 FMA accumulation.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float e4m3_to_float(uint32_t code) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)(code & 0xFFu)));
+    return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+
+__global__ void __launch_bounds__(256)
+linear_simt_kernel(const uint8_t* __restrict__ x8, int64_t ldx8, const float* __restrict__ s_x,
+                   int64_t M, const uint8_t* __restrict__ codes,
+                   const uint16_t* __restrict__ gscale, const uint8_t* __restrict__ gzero,
+                   const float* __restrict__ s_w, int sw_stride, int64_t N, int64_t K,
+                   void* __restrict__ y, int64_t ldy, int out_dtype) {
+    const int64_t n = (int64_t)blockIdx.x * 32 + (threadIdx.x & 31);
+    const int64_t m = (int64_t)blockIdx.y * 8 + (threadIdx.x >> 5);
+    if (n >= N || m >= M) return;
+    const int64_t G = K >> 7;
+    float acc = 0.0f;
+    for (int64_t g = 0; g < G; ++g) {
+        float s = bf16_bits_to_float(gscale[n * G + g]);
+        int z = gzero ? (int)gzero[n * G + g] : 8;
+        for (int kk = 0; kk < 128; kk += 2) {
+            int64_t k = g * 128 + kk;
+            uint32_t byte = codes[n * (K >> 1) + (k >> 1)];
+            float w0 = e4m3_to_float(cvt_e4m3x2(0.0f, __fmul_rn((float)((int)(byte & 15) - z), s)));
+            float w1 = e4m3_to_float(cvt_e4m3x2(0.0f, __fmul_rn((float)((int)(byte >> 4) - z), s)));
+            acc = fmaf(e4m3_to_float(x8[m * ldx8 + k]), w0, acc);
+            acc = fmaf(e4m3_to_float(x8[m * ldx8 + k + 1]), w1, acc);
+        }
+    }
+    float r = acc * (s_x[m] * s_w[n * sw_stride]);  // Eq. 4, Eq. 11
+    if (out_dtype == W4A8_OUT_FP32)
+        reinterpret_cast<float*>(y)[m * ldy + n] = r;
+    else
+        reinterpret_cast<__nv_bfloat16*>(y)[m * ldy + n] = __float2bfloat16_rn(r);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K reduction: sums the S fp32 partial tiles in slice order (deterministic), then applies
+// the Eq. 4 / Eq. 11 scales and the output cast.  partial layout: [S][M][N].
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partial, int S, int64_t M, int64_t N,
+                     const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
+                     void* __restrict__ y, int64_t ldy, int out_dtype) {
+    const int64_t total = M * N;
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * 256) {
+        int64_t m = i / N, n = i - m * N;
+        float acc = 0.0f;
+        for (int s = 0; s < S; ++s) acc += partial[(int64_t)s * total + i];
+        float r = acc * (s_x[m] * s_w[n * sw_stride]);
+        if (out_dtype == W4A8_OUT_FP32)
+            reinterpret_cast<float*>(y)[m * ldy + n] = r;
+        else
+            reinterpret_cast<__nv_bfloat16*>(y)[m * ldy + n] = __float2bfloat16_rn(r);
+    }
+}
+
+}  // namespace w4a8

@@ -1,0 +1,467 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A8 linear hot path (activation FP8 quantize -> fused INT4->FP8 GEMM ->
+scaled BF16) on the decode sweep: M in {1,4,16}, K=4096, N=14336 (Llama-3-8B MLP up-projection).
+
+One step = one pass of the whole path over the sweep: for each M, w4a8_quantize_act then
+w4a8_linear.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
+method must read per step, divided by the step time.  Weights rotate over several distinct
+copies whose total size exceeds twice the L2, so every pass streams them from HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 runs under torchrun, one independent replica per GPU (the path has no exchange step).
+--impl reference times the CPU oracle on the host cores on a bounded sample of the same
+workload.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+SWEEP_M = (1, 4, 16)
+K, N = 4096, 14336
+GROUP = 128
+SIGMA, OUTLIER_FRAC, OUTLIER_MULT = 0.02, 0.01, 20.0
+WEIGHT_COPIES = 10          # 10 x 30.3 MB = 303 MB > 2 x 126 MB L2
+METRIC = "w4a8_decode_weight_stream_rate"
+UNIT = "GB/s"
+WORKLOAD = ("c2 decode sweep: W4A8 linear, M in {1,4,16}, K=4096, N=14336, INT4 group-128 symmetric "
+            "weights from N(0,0.02), BF16 N(0,1) activations with 1% outlier channels x20, "
+            "per-token FP8 E4M3 scales, BF16 output")
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum); see profiles/.  None until a capture exists for the current kernel.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def weight_bytes(n=N, k=K):
+    """Bytes of the stored weight format one linear must read: codes + BF16 group scales."""
+    return n * k // 2 + n * (k // GROUP) * 2
+
+
+def linear_algorithmic_bytes(m, n=N, k=K):
+    """Everything one w4a8_linear launch must move: weights, FP8 activations, scales, BF16 output."""
+    return weight_bytes(n, k) + m * k + 4 * m + 4 + 2 * m * n
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power = [], [], []
+        reasons = set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "samples": len(sm),
+                "power_w_max": max(power), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------------------------
+
+def oracle_sample_pass(rows, x_bits_by_m, w_sample):
+    """One pass of the sweep through the oracle as it stands on `rows` output channels."""
+    import oracle
+    codes, gscale, gzero, s_w = w_sample
+    t0 = time.perf_counter()
+    for m in SWEEP_M:
+        x8, s_x = oracle.quantize_act(x_bits_by_m[m])
+        w8 = oracle.dequant_weight(codes, gscale, gzero)
+        oracle.linear(x8, s_x, w8, s_w, want=("ybf16",))
+    return time.perf_counter() - t0
+
+
+def make_oracle_sample(rows, seed=0):
+    import oracle
+    from paper_2505_14638_b200 import inputs
+    W = inputs.make_weight(rows, K, SIGMA, seed)
+    return oracle.quantize_weight_rtn(W, symmetric=True)
+
+
+def make_x_bits(seed=0):
+    from paper_2505_14638_b200 import inputs
+    return {m: inputs.make_activation(m, K, seed + m, OUTLIER_FRAC, OUTLIER_MULT) for m in SWEEP_M}
+
+
+def cpu_baseline(budget_s=12.0):
+    """The oracle timed on the host cores on a bounded sample (a slab of output channels)."""
+    import oracle
+    oracle.build()
+    x_bits = make_x_bits()
+    rows = 512
+    t = oracle_sample_pass(rows, x_bits, make_oracle_sample(rows))
+    rows_fit = int(min(N, max(512, rows * budget_s / max(t, 1e-6))))
+    rows_fit -= rows_fit % 16
+    if rows_fit > rows:
+        rows = rows_fit
+        t = oracle_sample_pass(rows, x_bits, make_oracle_sample(rows))
+    value = len(SWEEP_M) * weight_bytes(rows, K) / t / 1e9
+    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "one pass of the sweep M in {1,4,16} on the first %d of %d output channels "
+                      "(act quant + Eq. 10 dequant + exact matmul), %.2f s" % (rows, N, t)}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    total_budget = 150.0
+    per_step = total_budget / max(1, args.steps + args.warmup)
+    x_bits = make_x_bits()
+    rows = 256
+    t = oracle_sample_pass(rows, x_bits, make_oracle_sample(rows))
+    rows_fit = int(min(N, max(128, rows * per_step / max(t, 1e-6))))
+    rows_fit -= rows_fit % 16
+    rows = max(16, rows_fit)
+    sample = make_oracle_sample(rows)
+    for _ in range(args.warmup):
+        oracle_sample_pass(rows, x_bits, sample)
+    times = [oracle_sample_pass(rows, x_bits, sample) for _ in range(args.steps)]
+    total = sum(times)
+    value = args.steps * len(SWEEP_M) * weight_bytes(rows, K) / total / 1e9
+    desc = ("each step = one pass of the sweep M in {1,4,16} on %d of %d output channels" % (rows, N))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2505_14638_b200 import binding, inputs
+    from paper_2505_14638_b200 import build as _build
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the W4A8 path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        _build.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    binding.lib()
+    dev = torch.device("cuda", local_rank)
+
+    # ---- inputs: seeded synthetic, resident in HBM before the timed region ----
+    weights = []
+    for c in range(WEIGHT_COPIES):
+        W = torch.from_numpy(inputs.make_weight(N, K, SIGMA, seed=1000 * rank + c)).to(dev)
+        weights.append(binding.quantize_weight_rtn(W, symmetric=True))
+        del W
+    xs, x8s, sxs, ys = {}, {}, {}, {}
+    x_host = {}
+    for m in SWEEP_M:
+        xb = inputs.make_activation(m, K, 1000 * rank + m, OUTLIER_FRAC, OUTLIER_MULT)
+        t = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
+        x_host[m] = t.pin_memory()
+        xs[m] = t.to(dev)
+        x8s[m] = torch.empty((m, K), dtype=torch.uint8, device=dev)
+        sxs[m] = torch.empty((m,), dtype=torch.float32, device=dev)
+        ys[m] = torch.empty((m, N), dtype=torch.bfloat16, device=dev)
+    ws_bytes = max(binding.linear_workspace_bytes(m, N, K) for m in SWEEP_M)
+    workspace = torch.empty((max(ws_bytes, 16),), dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+
+    state = {"i": 0}
+
+    def step():
+        for m in SWEEP_M:
+            codes, gscale, gzero, s_w = weights[state["i"] % WEIGHT_COPIES]
+            state["i"] += 1
+            binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
+            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region 1: the whole path, K steps, device timed ----
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = binding.launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- timed region 2: the same steps with the linear launches bracketed by events ----
+    lin_ms = 0.0
+    pairs = []
+    for _ in range(args.steps):
+        for m in SWEEP_M:
+            binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for m in SWEEP_M:
+            codes, gscale, gzero, s_w = weights[state["i"] % WEIGHT_COPIES]
+            state["i"] += 1
+            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
+        b.record()
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    lin_ms = sum(a.elapsed_time(b) for a, b in pairs)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end: host activations in, host result out, through w4a8_forward_host ----
+    fwd = {m: binding.HostForward(m, *weights[0]) for m in SWEEP_M}
+
+    def e2e_step():
+        for m in SWEEP_M:
+            f = fwd[m]
+            f.codes, f.gscale, f.gzero, f.s_w = weights[state["i"] % WEIGHT_COPIES]
+            state["i"] += 1
+            f(x_host[m])
+        torch.cuda.current_stream().synchronize()   # the caller reads the result every step
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    g1.record()
+    barrier()
+    ms_e2e = g0.elapsed_time(g1)
+
+    if dist is not None:
+        t = torch.tensor([ms_total, ms_e2e, lin_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e, lin_ms = (float(v) for v in t.cpu())
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    step_weight_bytes = len(SWEEP_M) * weight_bytes()
+    value = world * args.steps * step_weight_bytes / (ms_total * 1e-3) / 1e9
+    e2e_value = world * args.steps * step_weight_bytes / (ms_e2e * 1e-3) / 1e9
+    n_lin = args.steps * len(SWEEP_M)
+    alg_bytes = sum(linear_algorithmic_bytes(m) for m in SWEEP_M) / len(SWEEP_M)
+    avg_launch_s = lin_ms * 1e-3 / n_lin
+    achieved = alg_bytes / avg_launch_s / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "parallelism": "replicas x%d (no collective)" % world,
+                   "l2": "weights rotate over %d distinct copies (%.0f MB > 2 x 126 MB L2)"
+                         % (WEIGHT_COPIES, WEIGHT_COPIES * weight_bytes() / 1e6),
+                   "step": "for M in (1,4,16): w4a8_quantize_act + w4a8_linear"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": sum(m * K * 2 for m in SWEEP_M),
+                "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "w4a8_linear (linear_umma_kernel + split-K reduce), mean over M",
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+    }
+    if not args.no_extras:
+        line["prefill"] = prefill_extra(torch, binding, inputs, dev, peaks)
+        line["decode_detail"] = decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks)
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def _time_loop(torch, fn, iters, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e-3 / iters
+
+
+def decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks):
+    """Per-M linear time with weights from HBM, next to cuBLAS BF16 of the same shape."""
+    out = {}
+    i = [0]
+    wb = [torch.randn((N, K), dtype=torch.bfloat16, device=x8s[1].device) for _ in range(3)]
+    for m in SWEEP_M:
+        def f():
+            codes, gscale, gzero, s_w = weights[i[0] % WEIGHT_COPIES]
+            i[0] += 1
+            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
+        t = _time_loop(torch, f, 50)
+        xb = torch.randn((m, K), dtype=torch.bfloat16, device=x8s[1].device)
+        j = [0]
+
+        def g():
+            j[0] += 1
+            torch.matmul(xb, wb[j[0] % 3].t())
+        tb = _time_loop(torch, g, 30)
+        out["M=%d" % m] = {"us": t * 1e6, "weight_GBps": weight_bytes() / t / 1e9,
+                           "frac_hbm_measured": linear_algorithmic_bytes(m) / t / 1e9 / peaks["hbm_gbs"],
+                           "cublas_bf16_us": tb * 1e6}
+    return out
+
+
+def prefill_extra(torch, binding, inputs, dev, peaks):
+    """Config c3 (M=2048, K=4096, N=4096): FP8 tensor-pipe rate of w4a8_linear next to cuBLAS BF16."""
+    M3, K3, N3 = 2048, 4096, 4096
+    copies = 8
+    sets = []
+    for c in range(copies):
+        W = torch.from_numpy(inputs.make_weight(N3, K3, SIGMA, seed=50 + c)).to(dev)
+        wq = binding.quantize_weight_rtn(W, symmetric=True)
+        xb = inputs.make_activation(M3, K3, 50 + c, OUTLIER_FRAC, OUTLIER_MULT)
+        x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
+        x8, s_x = binding.quantize_act(x)
+        sets.append((wq, x8, s_x, x))
+    y = torch.empty((M3, N3), dtype=torch.bfloat16, device=dev)
+    i = [0]
+
+    def f():
+        wq, x8, s_x, _ = sets[i[0] % copies]
+        i[0] += 1
+        binding.linear(x8, s_x, *wq, out=y)
+    t = _time_loop(torch, f, 40, warm=5)
+    wb = torch.randn((N3, K3), dtype=torch.bfloat16, device=dev)
+
+    def g():
+        _, _, _, x = sets[i[0] % copies]
+        i[0] += 1
+        torch.matmul(x, wb.t())
+    tb = _time_loop(torch, g, 40, warm=5)
+    flops = 2.0 * M3 * N3 * K3
+    fp8_peak = 2.0 * peaks["bf16_tflops"]
+    return {"workload": "c3 prefill M=2048 K=4096 N=4096", "us": t * 1e6, "tflops": flops / t / 1e12,
+            "fp8_peak_tflops": fp8_peak, "peak_note": "2 x bf16 burst peak (%s)" % peaks["source"],
+            "frac_of_fp8_peak": flops / t / 1e12 / fp8_peak, "frac_of_nominal_4500": flops / t / 1e12 / 4500.0,
+            "cublas_bf16_us": tb * 1e6, "cublas_bf16_tflops": flops / tb / 1e12}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the prefill / per-M detail sections")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world != args.gpus and world > 1:
+        raise SystemExit("--gpus %d does not match WORLD_SIZE %d" % (args.gpus, world))
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -228,14 +228,17 @@ def run_ours(args, rank, world, local_rank):
     binding.lib()
     dev = torch.device("cuda", local_rank)
 
-    # ---- inputs: seeded synthetic, resident in HBM before the timed region ----
+    # ---- inputs: seeded synthetic, quantized and tiled offline, resident in HBM ----
     weights = []
     for c in range(WEIGHT_COPIES):
         W = torch.from_numpy(inputs.make_weight(N, K, SIGMA, seed=1000 * rank + c)).to(dev)
-        weights.append(binding.quantize_weight_rtn(W, symmetric=True))
-        del W
-    xs, x8s, sxs, ys = {}, {}, {}, {}
-    x_host = {}
+        wq = binding.quantize_weight_rtn(W, symmetric=True)
+        weights.append(binding.prepack_weight(*wq))
+        del W, wq
+    torch.cuda.synchronize()
+    if binding.query_device_status() != 0:
+        raise RuntimeError("prepack reported an unrepresentable code")
+    xs, x8s, sxs, ys, x_host = {}, {}, {}, {}, {}
     for m in SWEEP_M:
         xb = inputs.make_activation(m, K, 1000 * rank + m, OUTLIER_FRAC, OUTLIER_MULT)
         t = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
@@ -244,82 +247,126 @@ def run_ours(args, rank, world, local_rank):
         x8s[m] = torch.empty((m, K), dtype=torch.uint8, device=dev)
         sxs[m] = torch.empty((m,), dtype=torch.float32, device=dev)
         ys[m] = torch.empty((m, N), dtype=torch.bfloat16, device=dev)
-    ws_bytes = max(binding.linear_workspace_bytes(m, N, K) for m in SWEEP_M)
-    workspace = torch.empty((max(ws_bytes, 16),), dtype=torch.uint8, device=dev)
+    workspace = binding.new_workspace(max(SWEEP_M), N, K, weights[0].fmt, dev)
     torch.cuda.synchronize()
 
-    state = {"i": 0}
+    def quant(m):
+        binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
 
-    def step():
-        for m in SWEEP_M:
-            codes, gscale, gzero, s_w = weights[state["i"] % WEIGHT_COPIES]
-            state["i"] += 1
-            binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
-            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
+    def lin(m, c):
+        binding.linear_tiled(x8s[m], sxs[m], weights[c % WEIGHT_COPIES], out=ys[m], workspace=workspace)
+
+    def eager_step(phase):
+        for i, m in enumerate(SWEEP_M):
+            quant(m)
+            lin(m, phase * len(SWEEP_M) + i)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
+    for ph in range(3):
+        eager_step(ph)
+    barrier()
+
+    # ---- CUDA graphs: one per phase of the weight rotation (the step is launch-bound) ----
+    use_graph = not args.no_graph
+    period = WEIGHT_COPIES
+    g_full, g_lin, g_quant = [], [], None
+    if use_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for ph in range(period):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    eager_step(ph)
+                g_full.append(g)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for i, m in enumerate(SWEEP_M):
+                        lin(m, ph * len(SWEEP_M) + i)
+                g_lin.append(g)
+            g_quant = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_quant, stream=side):
+                for m in SWEEP_M:
+                    quant(m)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    kernels_per_step = 2 * len(SWEEP_M)
+
+    def step(s):
+        if use_graph:
+            g_full[s % period].replay()
+        else:
+            eager_step(s % period)
+
+    for s in range(max(args.warmup, 3)):
+        step(s)
     barrier()
 
     # ---- timed region 1: the whole path, K steps, device timed ----
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    launches0 = binding.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    for _ in range(args.steps):
-        step()
+    for s in range(args.steps):
+        step(s)
     e1.record()
     barrier()
-    launches = binding.launch_count() - launches0
+    launches = args.steps * kernels_per_step
     ms_total = e0.elapsed_time(e1)
 
-    # ---- timed region 2: the same steps with the linear launches bracketed by events ----
-    lin_ms = 0.0
+    # ---- timed region 2: the same steps with the three linear launches bracketed by events ----
     pairs = []
-    for _ in range(args.steps):
-        for m in SWEEP_M:
-            binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
+    for s in range(args.steps):
+        if use_graph:
+            g_quant.replay()
+        else:
+            for m in SWEEP_M:
+                quant(m)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for m in SWEEP_M:
-            codes, gscale, gzero, s_w = weights[state["i"] % WEIGHT_COPIES]
-            state["i"] += 1
-            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
+        if use_graph:
+            g_lin[s % period].replay()
+        else:
+            for i, m in enumerate(SWEEP_M):
+                lin(m, s * len(SWEEP_M) + i)
         b.record()
         pairs.append((a, b))
     torch.cuda.synchronize()
     lin_ms = sum(a.elapsed_time(b) for a, b in pairs)
     clocks = sampler.stop() if rank == 0 else None
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set during the timed region")
 
     # ---- end to end: host activations in, host result out, through w4a8_forward_host ----
-    fwd = {m: binding.HostForward(m, *weights[0]) for m in SWEEP_M}
+    fwd = {m: binding.HostForward(m, weights[0]) for m in SWEEP_M}
+    cnt = [0]
 
     def e2e_step():
         for m in SWEEP_M:
             f = fwd[m]
-            f.codes, f.gscale, f.gzero, f.s_w = weights[state["i"] % WEIGHT_COPIES]
-            state["i"] += 1
+            f.set_weight(weights[cnt[0] % WEIGHT_COPIES])
+            cnt[0] += 1
             f(x_host[m])
         torch.cuda.current_stream().synchronize()   # the caller reads the result every step
 
     for _ in range(3):
         e2e_step()
     barrier()
+    n_e2e = min(args.steps, 2000)
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     g0.record()
-    for _ in range(args.steps):
+    for _ in range(n_e2e):
         e2e_step()
     g1.record()
     barrier()
-    ms_e2e = g0.elapsed_time(g1)
+    ms_e2e = g0.elapsed_time(g1) * args.steps / n_e2e
 
     if dist is not None:
         t = torch.tensor([ms_total, ms_e2e, lin_ms], dtype=torch.float64, device=dev)
@@ -347,23 +394,24 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD, "parallelism": "replicas x%d (no collective)" % world,
                    "l2": "weights rotate over %d distinct copies (%.0f MB > 2 x 126 MB L2)"
                          % (WEIGHT_COPIES, WEIGHT_COPIES * weight_bytes() / 1e6),
-                   "step": "for M in (1,4,16): w4a8_quantize_act + w4a8_linear"},
+                   "step": "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
+                   "launch": "CUDA graph replay, one graph per step" if use_graph else "eager launches"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(m * K * 2 for m in SWEEP_M),
                 "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "w4a8_linear (linear_umma_kernel + split-K reduce), mean over M",
+        "roofline": {"bound": "hbm", "kernel": "linear_streamk_kernel<BNX=16> (w4a8_linear), mean over M in {1,4,16}",
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
     }
     if not args.no_extras:
-        line["prefill"] = prefill_extra(torch, binding, inputs, dev, peaks)
         line["decode_detail"] = decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks)
-    if not args.no_cpu_baseline:
+        line["prefill"] = prefill_extra(torch, binding, inputs, dev, peaks)
+    if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line), flush=True)
     if dist is not None:
@@ -385,23 +433,27 @@ def _time_loop(torch, fn, iters, warm=3):
 
 
 def decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks):
-    """Per-M linear time with weights from HBM, next to cuBLAS BF16 of the same shape."""
+    """Per-M linear time (graph of back-to-back launches, weights from HBM) next to cuBLAS BF16."""
     out = {}
-    i = [0]
-    wb = [torch.randn((N, K), dtype=torch.bfloat16, device=x8s[1].device) for _ in range(3)]
+    dev = x8s[1].device
+    wb = [torch.randn((N, K), dtype=torch.bfloat16, device=dev) for _ in range(4)]
+    side = torch.cuda.Stream()
     for m in SWEEP_M:
-        def f():
-            codes, gscale, gzero, s_w = weights[i[0] % WEIGHT_COPIES]
-            i[0] += 1
-            binding.linear(x8s[m], sxs[m], codes, gscale, gzero, s_w, out=ys[m], workspace=workspace)
-        t = _time_loop(torch, f, 50)
-        xb = torch.randn((m, K), dtype=torch.bfloat16, device=x8s[1].device)
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for c in range(WEIGHT_COPIES):
+                    binding.linear_tiled(x8s[m], sxs[m], weights[c], out=ys[m], workspace=workspace)
+        torch.cuda.current_stream().wait_stream(side)
+        t = _time_loop(torch, g.replay, 20) / WEIGHT_COPIES
+        xb = torch.randn((m, K), dtype=torch.bfloat16, device=dev)
         j = [0]
 
-        def g():
+        def f():
             j[0] += 1
-            torch.matmul(xb, wb[j[0] % 3].t())
-        tb = _time_loop(torch, g, 30)
+            torch.matmul(xb, wb[j[0] % 4].t())
+        tb = _time_loop(torch, f, 40)
         out["M=%d" % m] = {"us": t * 1e6, "weight_GBps": weight_bytes() / t / 1e9,
                            "frac_hbm_measured": linear_algorithmic_bytes(m) / t / 1e9 / peaks["hbm_gbs"],
                            "cublas_bf16_us": tb * 1e6}
@@ -415,18 +467,19 @@ def prefill_extra(torch, binding, inputs, dev, peaks):
     sets = []
     for c in range(copies):
         W = torch.from_numpy(inputs.make_weight(N3, K3, SIGMA, seed=50 + c)).to(dev)
-        wq = binding.quantize_weight_rtn(W, symmetric=True)
+        tw = binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True))
         xb = inputs.make_activation(M3, K3, 50 + c, OUTLIER_FRAC, OUTLIER_MULT)
         x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
         x8, s_x = binding.quantize_act(x)
-        sets.append((wq, x8, s_x, x))
+        sets.append((tw, x8, s_x, x))
     y = torch.empty((M3, N3), dtype=torch.bfloat16, device=dev)
+    ws = binding.new_workspace(M3, N3, K3, sets[0][0].fmt, dev)
     i = [0]
 
     def f():
-        wq, x8, s_x, _ = sets[i[0] % copies]
+        tw, x8, s_x, _ = sets[i[0] % copies]
         i[0] += 1
-        binding.linear(x8, s_x, *wq, out=y)
+        binding.linear_tiled(x8, s_x, tw, out=y, workspace=ws)
     t = _time_loop(torch, f, 40, warm=5)
     wb = torch.randn((N3, K3), dtype=torch.bfloat16, device=dev)
 
@@ -451,6 +504,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / per-M detail sections")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

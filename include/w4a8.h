@@ -54,8 +54,22 @@ extern "C" {
 #define W4A8_OUT_FP32 1
 
 #define W4A8_ALGO_AUTO 0
-#define W4A8_ALGO_SIMT 1 /* plain CUDA-core kernel: slow, for cross-checks */
-#define W4A8_ALGO_UMMA 2 /* TMA + tcgen05 kernel */
+#define W4A8_ALGO_SIMT 1 /* plain CUDA-core kernel: slow, for cross-checks (canonical weights only) */
+#define W4A8_ALGO_UMMA 2 /* TMA + tcgen05 kernel, one tile per CTA (canonical weights only) */
+
+/*
+ * Weight storage formats.  CANONICAL is the boundary format described above (codes, gscale,
+ * gzero as separate row-major arrays).  The TILED formats are produced offline by
+ * w4a8_prepack_weight from the canonical arrays and hold the same information rearranged so
+ * that one 128-row x 128-k block (codes, scales, zero-points) is one contiguous chunk:
+ *   TILED          any codes and zero-points (the paper's asymmetric INT4 included);
+ *   TILED_SIGNMAG  symmetric storage only (gzero == NULL, z = 8) with every code in 1..15, as the
+ *                  symmetric quantizer of Eq. 1 produces; codes are kept as sign and magnitude
+ *                  of (u - 8), which makes the Eq. 10 expansion cheaper.
+ */
+#define W4A8_FMT_CANONICAL 0
+#define W4A8_FMT_TILED 1
+#define W4A8_FMT_TILED_SIGNMAG 2
 
 /*
  * Activation FP8 quantization, Eq. 13 (with Eq. 3), one scale per token:
@@ -84,22 +98,41 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * with W8 produced on the fly from (codes, gscale, gzero) exactly as w4a8_dequant_weight
  * defines it, FP8 x FP8 products accumulated in FP32, output rounded to BF16 (out_dtype 0) or
  * kept in FP32 (out_dtype 1).  sw_stride is 1 (per channel) or 0 (per tensor).
- * `workspace` holds split-K partial sums when the library splits the reduction (small M);
- * it needs w4a8_linear_workspace_bytes(M, N, K) bytes, is written before it is read and may be
- * NULL when that size is 0.  Calls that share a workspace must not overlap on the device.
+ * weight_format selects how `weights` is read: W4A8_FMT_CANONICAL (weights = codes, with
+ * gscale_bf16 / gzero) or a tiled format (weights = buffer written by w4a8_prepack_weight;
+ * gscale_bf16 and gzero are ignored and may be NULL).
+ * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs; it
+ * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
+ * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
+ * its first use; every call leaves it ready for the next one.  Calls that share a workspace
+ * must not overlap on the device.
  */
-int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
-                const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride,
-                int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype,
+int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* weights,
+                const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w,
+                int sw_stride, int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype,
                 void* workspace, size_t workspace_bytes, void* stream);
 
-/* Bytes of workspace w4a8_linear needs for this problem (0 when no split is used). */
-size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+/* Bytes of workspace w4a8_linear needs for this problem (0 when none is used). */
+size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_format);
+
+/*
+ * Offline re-layout of the stored weights (no arithmetic on values): canonical codes, scales and
+ * zero-points -> a tiled buffer of w4a8_prepack_bytes(N, K, weight_format) bytes (128-byte
+ * aligned) for weight_format W4A8_FMT_TILED or W4A8_FMT_TILED_SIGNMAG.  The dequantized weights
+ * the linear layer sees are bit-identical to Eq. 10 on the canonical arrays.  If a code 0 is met
+ * while writing W4A8_FMT_TILED_SIGNMAG, bit 1 of the device status word is raised
+ * (w4a8_query_device_status) and the buffer must not be used.
+ */
+size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format);
+int w4a8_prepack_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero, int64_t N,
+                        int64_t K, int group, int weight_format, uint8_t* out, size_t out_bytes,
+                        void* stream);
 
 /*
  * Same computation as w4a8_linear with the kernel choice exposed, for cross-checks and tuning:
- * algo is W4A8_ALGO_*; split_k <= 0 lets the library choose, otherwise it is the number of
- * K slices (must divide K/128).  Workspace need: w4a8_linear_ex_workspace_bytes.
+ * canonical weights only.  algo is W4A8_ALGO_*; split_k <= 0 lets the library choose, otherwise
+ * it is the number of K slices (must divide K/128).  Workspace need:
+ * w4a8_linear_ex_workspace_bytes (no zero-fill needed).
  */
 int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
                    const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
@@ -128,16 +161,17 @@ int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, in
  * stream before reading y_host.  Weights stay resident on the device.  Scratch device buffers
  * are the caller's: x_dev (2*M*K bytes), x8_dev (M*K), s_x_dev (4*M), y_dev (2*M*N), workspace.
  */
-int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* codes,
-                      const void* gscale_bf16, const uint8_t* gzero, const float* s_w,
+int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights,
+                      const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w,
                       int sw_stride, int64_t N, int64_t K, int group, void* y_host_bf16,
                       void* x_dev, uint8_t* x8_dev, float* s_x_dev, void* y_dev, void* workspace,
                       size_t workspace_bytes, void* stream);
 
 /*
  * Reads and clears the device-side status word (synchronises the device).  *flags receives a
- * bit mask: bit 0 = a bounded wait inside a kernel gave up.  Returns W4A8_ERR_TIMEOUT when any
- * bit was set, W4A8_OK otherwise.
+ * bit mask: bit 0 = a bounded wait inside a kernel gave up; bit 1 = w4a8_prepack_weight met a
+ * code its target format cannot hold.  Returns W4A8_ERR_TIMEOUT when bit 0 was set,
+ * W4A8_ERR_BAD_SHAPE when only bit 1 was set, W4A8_OK otherwise.
  */
 int w4a8_query_device_status(unsigned int* flags_host);
 

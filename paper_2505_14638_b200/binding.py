@@ -19,11 +19,13 @@ ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 SCALE_EXACT, SCALE_POW2 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 ALGO_AUTO, ALGO_SIMT, ALGO_UMMA = 0, 1, 2
+FMT_CANONICAL, FMT_TILED, FMT_TILED_SIGNMAG = 0, 1, 2
 GROUP = 128
 
 # Every symbol include/w4a8.h declares.
 EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
+    "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_quantize_weight_rtn",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
 )
@@ -54,9 +56,13 @@ def lib():
     L.w4a8_dequant_weight.restype = i32
     L.w4a8_dequant_weight.argtypes = [p, p, p, i64, i64, i32, p, p]
     L.w4a8_linear.restype = i32
-    L.w4a8_linear.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz, p]
+    L.w4a8_linear.argtypes = [p, i64, p, i64, p, p, p, i32, p, i32, i64, i64, i32, p, i64, i32, p, sz, p]
     L.w4a8_linear_workspace_bytes.restype = sz
-    L.w4a8_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.w4a8_linear_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.w4a8_prepack_bytes.restype = sz
+    L.w4a8_prepack_bytes.argtypes = [i64, i64, i32]
+    L.w4a8_prepack_weight.restype = i32
+    L.w4a8_prepack_weight.argtypes = [p, p, p, i64, i64, i32, i32, p, sz, p]
     L.w4a8_linear_ex.restype = i32
     L.w4a8_linear_ex.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz,
                                  i32, i32, p]
@@ -65,7 +71,7 @@ def lib():
     L.w4a8_quantize_weight_rtn.restype = i32
     L.w4a8_quantize_weight_rtn.argtypes = [p, i64, i64, i32, i32, i32, i32, p, p, p, p, p]
     L.w4a8_forward_host.restype = i32
-    L.w4a8_forward_host.argtypes = [p, i64, p, p, p, p, i32, i64, i64, i32, p, p, p, p, p, p, sz, p]
+    L.w4a8_forward_host.argtypes = [p, i64, p, p, p, i32, p, i32, i64, i64, i32, p, p, p, p, p, p, sz, p]
     L.w4a8_query_device_status.restype = i32
     L.w4a8_query_device_status.argtypes = [c.POINTER(c.c_uint)]
     L.w4a8_launch_count.restype = c.c_uint64
@@ -88,7 +94,7 @@ def query_device_status() -> int:
     """Synchronises; returns the device status bit mask (0 = clean) and clears it."""
     flags = ctypes.c_uint(0)
     rc = lib().w4a8_query_device_status(ctypes.byref(flags))
-    if rc not in (OK, ERR_TIMEOUT):
+    if rc not in (OK, ERR_TIMEOUT, ERR_BAD_SHAPE):
         raise W4A8Error("w4a8_query_device_status", rc)
     return int(flags.value)
 
@@ -137,13 +143,45 @@ def dequant_weight(codes, gscale, gzero=None, out=None):
     return w8
 
 
-def linear_workspace_bytes(M, N, K, algo=ALGO_AUTO, split_k=0) -> int:
+def linear_workspace_bytes(M, N, K, algo=ALGO_AUTO, split_k=0, weight_format=FMT_CANONICAL) -> int:
+    if weight_format != FMT_CANONICAL or (algo == ALGO_AUTO and split_k == 0):
+        return int(lib().w4a8_linear_workspace_bytes(M, N, K, weight_format))
     return int(lib().w4a8_linear_ex_workspace_bytes(M, N, K, algo, split_k))
+
+
+class TiledWeight:
+    """Weights re-laid out by w4a8_prepack_weight (FMT_TILED or FMT_TILED_SIGNMAG)."""
+
+    def __init__(self, buf, fmt, N, K, s_w):
+        self.buf, self.fmt, self.N, self.K, self.s_w = buf, fmt, N, K, s_w
+
+
+def prepack_weight(codes, gscale, gzero, s_w, weight_format=None):
+    """w4a8_prepack_weight: canonical device arrays -> TiledWeight.  Default format: the
+    sign-magnitude one for symmetric storage (gzero None), the generic tiled one otherwise."""
+    import torch
+    if weight_format is None:
+        weight_format = FMT_TILED_SIGNMAG if gzero is None else FMT_TILED
+    N, Kh = codes.shape
+    K = Kh * 2
+    nbytes = int(lib().w4a8_prepack_bytes(N, K, weight_format))
+    buf = torch.empty((nbytes,), dtype=torch.uint8, device=codes.device)
+    rc = lib().w4a8_prepack_weight(_ptr(codes), _ptr(gscale), _ptr(gzero), N, K, GROUP,
+                                   int(weight_format), _ptr(buf), nbytes, _stream())
+    _check("w4a8_prepack_weight", rc)
+    return TiledWeight(buf, weight_format, N, K, s_w)
+
+
+def new_workspace(M, N, K, weight_format=FMT_CANONICAL, device="cuda"):
+    """Zero-filled workspace of the size w4a8_linear needs (at least 16 bytes)."""
+    import torch
+    need = linear_workspace_bytes(M, N, K, weight_format=weight_format)
+    return torch.zeros((max(need, 16),), dtype=torch.uint8, device=device)
 
 
 def linear(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, workspace=None,
            algo=ALGO_AUTO, split_k=0):
-    """w4a8_linear / w4a8_linear_ex: returns Y [M, N] (BF16 or FP32)."""
+    """w4a8_linear / w4a8_linear_ex on canonical weights: returns Y [M, N] (BF16 or FP32)."""
     import torch
     M, K = x8.shape
     N = codes.shape[0]
@@ -158,7 +196,7 @@ def linear(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, wor
     L = lib()
     if algo == ALGO_AUTO and split_k == 0:
         rc = L.w4a8_linear(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(codes), _ptr(gscale),
-                           _ptr(gzero), _ptr(s_w), sw_stride, N, K, GROUP, _ptr(out),
+                           _ptr(gzero), FMT_CANONICAL, _ptr(s_w), sw_stride, N, K, GROUP, _ptr(out),
                            out.stride(0), int(out_dtype), _ptr(workspace), wbytes, _stream())
         _check("w4a8_linear", rc)
     else:
@@ -167,6 +205,25 @@ def linear(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, wor
                               out.stride(0), int(out_dtype), _ptr(workspace), wbytes, int(algo),
                               int(split_k), _stream())
         _check("w4a8_linear_ex", rc)
+    return out
+
+
+def linear_tiled(x8, s_x, tw, out_dtype=OUT_BF16, out=None, workspace=None):
+    """w4a8_linear on a TiledWeight.  `workspace` must come from new_workspace (zero-filled once);
+    one is created when none is given."""
+    import torch
+    M, K = x8.shape
+    assert K == tw.K
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, tw.N), dtype=dt, device=x8.device)
+    if workspace is None:
+        workspace = new_workspace(M, tw.N, K, tw.fmt, x8.device)
+    rc = lib().w4a8_linear(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(tw.buf), None, None, tw.fmt,
+                           _ptr(tw.s_w), 0 if tw.s_w.numel() == 1 else 1, tw.N, K, GROUP, _ptr(out),
+                           out.stride(0), int(out_dtype), _ptr(workspace),
+                           workspace.numel() * workspace.element_size(), _stream())
+    _check("w4a8_linear", rc)
     return out
 
 
@@ -189,32 +246,39 @@ def quantize_weight_rtn(W, symmetric=True, pow2=False, per_channel=False):
 
 class HostForward:
     """w4a8_forward_host with its device scratch buffers allocated once: activations come from
-    and results go to pinned host memory, weights stay on the device."""
+    and results go to pinned host memory, weights stay on the device.  `weight` is either a
+    TiledWeight or a tuple (codes, gscale, gzero, s_w) of canonical device arrays."""
 
-    def __init__(self, M, codes, gscale, gzero, s_w):
+    def __init__(self, M, weight):
         import torch
         self.M = M
-        self.N, Kh = codes.shape
-        self.K = Kh * 2
-        dev = codes.device
-        self.codes, self.gscale, self.gzero, self.s_w = codes, gscale, gzero, s_w
+        self.set_weight(weight)
+        dev = self.wbuf.device
         self.x_dev = torch.empty((M, self.K), dtype=torch.bfloat16, device=dev)
         self.x8 = torch.empty((M, self.K), dtype=torch.uint8, device=dev)
         self.s_x = torch.empty((M,), dtype=torch.float32, device=dev)
         self.y_dev = torch.empty((M, self.N), dtype=torch.bfloat16, device=dev)
-        need = linear_workspace_bytes(M, self.N, self.K)
-        self.ws = torch.empty((max(need, 16),), dtype=torch.uint8, device=dev)
+        self.ws = new_workspace(M, self.N, self.K, self.fmt, dev)
         self.y_host = torch.empty((M, self.N), dtype=torch.bfloat16).pin_memory()
         self.h2d_bytes = M * self.K * 2
         self.d2h_bytes = M * self.N * 2
+
+    def set_weight(self, weight):
+        if isinstance(weight, TiledWeight):
+            self.wbuf, self.gscale, self.gzero, self.s_w = weight.buf, None, None, weight.s_w
+            self.fmt, self.N, self.K = weight.fmt, weight.N, weight.K
+        else:
+            self.wbuf, self.gscale, self.gzero, self.s_w = weight
+            self.fmt = FMT_CANONICAL
+            self.N, self.K = self.wbuf.shape[0], self.wbuf.shape[1] * 2
 
     def __call__(self, x_host):
         """x_host: pinned BF16 [M, K] host tensor.  Enqueues everything; returns the pinned
         output tensor, valid after the current stream is synchronised."""
         rc = lib().w4a8_forward_host(
-            ctypes.c_void_p(x_host.data_ptr()), self.M, _ptr(self.codes), _ptr(self.gscale),
-            _ptr(self.gzero), _ptr(self.s_w), 0 if self.s_w.numel() == 1 else 1, self.N, self.K,
-            GROUP, ctypes.c_void_p(self.y_host.data_ptr()), _ptr(self.x_dev), _ptr(self.x8),
+            ctypes.c_void_p(x_host.data_ptr()), self.M, _ptr(self.wbuf), _ptr(self.gscale),
+            _ptr(self.gzero), self.fmt, _ptr(self.s_w), 0 if self.s_w.numel() == 1 else 1, self.N,
+            self.K, GROUP, ctypes.c_void_p(self.y_host.data_ptr()), _ptr(self.x_dev), _ptr(self.x8),
             _ptr(self.s_x), _ptr(self.y_dev), _ptr(self.ws), self.ws.numel(), _stream())
         _check("w4a8_forward_host", rc)
         return self.y_host

@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "../../include/w4a8.h"
+#include "w4a8_linear_streamk.cuh"
 #include "w4a8_linear_umma.cuh"
 #include "w4a8_simple_kernels.cuh"
 
@@ -155,11 +156,105 @@ static int launch_umma(const CUtensorMap& tw, const CUtensorMap& tx, const uint1
     return launch_status();
 }
 
+// ------------------------------------------------------------------------------ persistent kernel plan
+constexpr int kMaxSMs = 160;  // upper bound used to size workspaces without touching a device
+
+static int sm_count() {
+    static std::mutex mu;
+    static int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached_dev != dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached_dev = dev;
+        cached = n;
+    }
+    return cached;
+}
+
+struct SkPlan {
+    int bnx, ctas_per_sm, TM, TN;
+    int64_t U;
+    size_t counter_bytes, workspace_bytes;
+};
+
+static void make_sk_plan(int64_t M, int64_t N, int64_t K, SkPlan* pl) {
+    pl->bnx = pick_bnx(M);
+    pl->ctas_per_sm = pl->bnx <= 32 ? 2 : 1;
+    pl->TM = (int)((M + pl->bnx - 1) / pl->bnx);
+    pl->TN = (int)((N + 127) / 128);
+    pl->U = (int64_t)pl->TM * pl->TN * (K / 128);
+    size_t cb = (size_t)pl->TM * pl->TN * sizeof(unsigned int);
+    pl->counter_bytes = (cb + 255) / 256 * 256;
+    int64_t pmax = (int64_t)pl->ctas_per_sm * kMaxSMs;
+    if (pmax > pl->U) pmax = pl->U;
+    pl->workspace_bytes = pl->counter_bytes + (size_t)pmax * 2 * (size_t)pl->bnx * 128 * sizeof(float);
+}
+
+template <class Cfg>
+static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
+                          int sw_stride, void* y, int64_t ldy, int out_dtype, void* workspace, const SkPlan& pl,
+                          int M, int N, int K, cudaStream_t st) {
+    auto kern = linear_streamk_kernel<Cfg>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    unsigned int* status = status_word_ptr();
+    const int sms = sm_count();
+    if (!status || sms <= 0) return W4A8_ERR_CUDA;
+    int64_t P = (int64_t)pl.ctas_per_sm * (sms < kMaxSMs ? sms : kMaxSMs);
+    if (P > pl.U) P = pl.U;
+    unsigned int* counters = static_cast<unsigned int*>(workspace);
+    float* slots = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
+    kern<<<(unsigned)P, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                                               counters, slots, M, N, K, pl.TM, pl.TN, status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* wpp,
+                             int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
+                             int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    SkPlan pl;
+    make_sk_plan(M, N, K, &pl);
+    if (!workspace || workspace_bytes < pl.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    CUtensorMap tx;
+    if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)pl.bnx,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+#define W4A8_SK(BNX, G, S1, S2)                                                                                  \
+    rc = (fmt == kFmtTiledSignMag)                                                                                \
+             ? launch_streamk<SkCfg<BNX, G, S1, S2, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,     \
+                                                                       out_dtype, workspace, pl, Mi, Ni, Ki, st) \
+             : launch_streamk<SkCfg<BNX, G, S1, S2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, \
+                                                                workspace, pl, Mi, Ni, Ki, st)
+    switch (pl.bnx) {
+        case 16: W4A8_SK(16, 2, 5, 3); break;
+        case 32: W4A8_SK(32, 2, 4, 3); break;
+        case 64: W4A8_SK(64, 4, 6, 4); break;
+        case 128: W4A8_SK(128, 4, 5, 4); break;
+        default: W4A8_SK(256, 4, 4, 3); break;
+    }
+#undef W4A8_SK
+    return rc;
+}
+
 static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
-                       const void* gscale, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
-                       int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
+                       const void* gscale, const uint8_t* gzero, int fmt, const float* s_w, int sw_stride,
+                       int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
                        size_t workspace_bytes, int algo, int split_k, cudaStream_t st) {
-    if (!x8 || !s_x || !codes || !gscale || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (fmt != kFmtCanonical && fmt != kFmtTiled && fmt != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+    if (!x8 || !s_x || !codes || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (fmt == kFmtCanonical && !gscale) return W4A8_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
     if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
     if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
@@ -170,6 +265,11 @@ static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_
     if ((reinterpret_cast<uintptr_t>(gscale) & 1u) || (reinterpret_cast<uintptr_t>(s_x) & 3u) ||
         (reinterpret_cast<uintptr_t>(s_w) & 3u))
         return W4A8_ERR_BAD_ALIGNMENT;
+    if (fmt != kFmtCanonical) {
+        if (algo != W4A8_ALGO_AUTO || split_k > 0) return W4A8_ERR_INVALID_ARG;
+        return linear_tiled_impl(x8, ldx8, s_x, M, codes, fmt, s_w, sw_stride, N, K, y, ldy, out_dtype, workspace,
+                                 workspace_bytes, st);
+    }
     LinearPlan plan;
     int rc = make_plan(M, N, K, algo, split_k, &plan);
     if (rc != W4A8_OK) return rc;
@@ -279,24 +379,58 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
     return launch_status();
 }
 
-int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
-                const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
-                int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
+int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* weights,
+                const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w, int sw_stride,
+                int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
                 size_t workspace_bytes, void* stream) {
-    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y, ldy, out_dtype,
-                       workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, static_cast<cudaStream_t>(stream));
+    return linear_impl(x8, ldx8, s_x, M, weights, gscale_bf16, gzero, weight_format, s_w, sw_stride, N, K, group, y,
+                       ldy, out_dtype, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0,
+                       static_cast<cudaStream_t>(stream));
 }
 
-size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-    return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
+size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_format) {
+    if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    if (weight_format == kFmtCanonical) return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
+    if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
+    SkPlan pl;
+    make_sk_plan(M, N, K, &pl);
+    return pl.workspace_bytes;
+}
+
+size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format) {
+    if (N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
+    return (size_t)((N + 127) / 128) * (size_t)(K / 128) * (size_t)chunk_bytes(weight_format);
+}
+
+int w4a8_prepack_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero, int64_t N, int64_t K,
+                        int group, int weight_format, uint8_t* out, size_t out_bytes, void* stream) {
+    if (!codes || !gscale_bf16 || !out) return W4A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+    if (weight_format == kFmtTiledSignMag && gzero != nullptr) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(out) & 127u) ||
+        (reinterpret_cast<uintptr_t>(gscale_bf16) & 1u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    if (out_bytes < w4a8_prepack_bytes(N, K, weight_format)) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    unsigned int* status = status_word_ptr();
+    if (!status) return W4A8_ERR_CUDA;
+    const int64_t blocks = ((N + 127) / 128) * (K / 128);
+    prepack_kernel<<<(unsigned)blocks, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        codes, static_cast<const uint16_t*>(gscale_bf16), gzero, N, K, weight_format, out, status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
 }
 
 int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
                    const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N,
                    int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
                    size_t workspace_bytes, int algo, int split_k, void* stream) {
-    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y, ldy, out_dtype,
-                       workspace, workspace_bytes, algo, split_k, static_cast<cudaStream_t>(stream));
+    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
+                       ldy, out_dtype, workspace, workspace_bytes, algo, split_k, static_cast<cudaStream_t>(stream));
 }
 
 size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k) {
@@ -337,8 +471,9 @@ int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, in
     return launch_status();
 }
 
-int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* codes, const void* gscale_bf16,
-                      const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, int group,
+int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights, const void* gscale_bf16,
+                      const uint8_t* gzero, int weight_format, const float* s_w, int sw_stride, int64_t N,
+                      int64_t K, int group,
                       void* y_host_bf16, void* x_dev, uint8_t* x8_dev, float* s_x_dev, void* y_dev,
                       void* workspace, size_t workspace_bytes, void* stream) {
     if (!x_host_bf16 || !y_host_bf16 || !x_dev || !x8_dev || !s_x_dev || !y_dev) return W4A8_ERR_INVALID_ARG;
@@ -346,20 +481,21 @@ int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* codes, 
     if (group != kGroup || K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Validate the two stages before anything is enqueued.
-    LinearPlan plan;
-    int rc = make_plan(M, N, K, W4A8_ALGO_AUTO, 0, &plan);
-    if (rc != W4A8_OK) return rc;
-    if (plan.workspace_bytes > 0 && (!workspace || workspace_bytes < plan.workspace_bytes))
-        return W4A8_ERR_WORKSPACE_TOO_SMALL;
-    if (!codes || !gscale_bf16 || !s_w) return W4A8_ERR_INVALID_ARG;
-    if (!aligned16(x_dev) || !aligned16(x8_dev) || !aligned16(y_dev) || !aligned16(codes))
+    if (weight_format != kFmtCanonical && weight_format != kFmtTiled && weight_format != kFmtTiledSignMag)
+        return W4A8_ERR_INVALID_ARG;
+    if (!weights || !s_w || (weight_format == kFmtCanonical && !gscale_bf16)) return W4A8_ERR_INVALID_ARG;
+    const size_t need = w4a8_linear_workspace_bytes(M, N, K, weight_format);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if (!aligned16(x_dev) || !aligned16(x8_dev) || !aligned16(y_dev) || !aligned16(weights) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 15u))
         return W4A8_ERR_BAD_ALIGNMENT;
+    int rc;
     if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
     rc = quantize_act_impl(x_dev, M, K, K, x8_dev, K, s_x_dev, W4A8_SCALE_EXACT, nullptr, st);
     if (rc != W4A8_OK) return rc;
-    rc = linear_impl(x8_dev, K, s_x_dev, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, group, y_dev, N,
-                     W4A8_OUT_BF16, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, st);
+    rc = linear_impl(x8_dev, K, s_x_dev, M, weights, gscale_bf16, gzero, weight_format, s_w, sw_stride, N, K, group,
+                     y_dev, N, W4A8_OUT_BF16, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, st);
     if (rc != W4A8_OK) return rc;
     if (cudaMemcpyAsync(y_host_bf16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
@@ -373,8 +509,22 @@ int w4a8_query_device_status(unsigned int* flags_host) {
     if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof v) != cudaSuccess) return W4A8_ERR_CUDA;
     if (v != 0 && cudaMemcpyToSymbol(g_status_word, &zero, sizeof zero) != cudaSuccess) return W4A8_ERR_CUDA;
     *flags_host = v;
-    return (v != 0) ? W4A8_ERR_TIMEOUT : W4A8_OK;
+    if (v & kStatusTimeout) return W4A8_ERR_TIMEOUT;
+    return (v != 0) ? W4A8_ERR_BAD_SHAPE : W4A8_OK;
 }
+
+#ifdef W4A8_TIMING
+int w4a8_debug_read(long long* host, int n, int clear) {
+    cudaDeviceSynchronize();
+    if (cudaMemcpyFromSymbol(host, g_dbg, sizeof(long long) * n) != cudaSuccess) return -1;
+    if (clear) {
+        void* p = nullptr;
+        cudaGetSymbolAddress(&p, g_dbg);
+        cudaMemset(p, 0, sizeof(long long) * 1024 * 16);
+    }
+    return 0;
+}
+#endif
 
 uint64_t w4a8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -34,7 +34,12 @@ def test_status_strings(L):
     assert binding.status_string(-99) == "unknown status"
 
 
-def test_workspace_query_is_host_only(L):
+def test_workspace_and_prepack_size_queries_are_host_only(L):
+    assert L.w4a8_prepack_bytes(14336, 4096, binding.FMT_TILED_SIGNMAG) == 112 * 32 * 8448
+    assert L.w4a8_prepack_bytes(14336 + 16, 4096, binding.FMT_TILED) == 113 * 32 * 8576
+    assert L.w4a8_prepack_bytes(14336, 4096, binding.FMT_CANONICAL) == 0
+    ws = binding.linear_workspace_bytes(16, 14336, 4096, weight_format=binding.FMT_TILED_SIGNMAG)
+    assert ws >= 112 * 4 + 2 * 296 * 16 * 128 * 4
     assert binding.linear_workspace_bytes(2048, 4096, 4096) == 0          # large M: no split
     ws = binding.linear_workspace_bytes(16, 14336, 4096)
     assert ws % (16 * 14336 * 4) == 0 and ws > 0                          # S partial tiles
@@ -72,9 +77,14 @@ def test_linear_rejects_bad_arguments(L):
     p = _fake()
     f = L.w4a8_linear
 
-    def call(x8=p, ldx8=4096, s_x=p, M=16, codes=p, gs=p, gz=None, s_w=p, sws=0, N=14336, K=4096, group=128,
-             y=p, ldy=14336, od=0, ws=p, wsb=1 << 30):
-        return f(x8, ldx8, s_x, M, codes, gs, gz, s_w, sws, N, K, group, y, ldy, od, ws, wsb, None)
+    def call(x8=p, ldx8=4096, s_x=p, M=16, codes=p, gs=p, gz=None, fmt=0, s_w=p, sws=0, N=14336, K=4096,
+             group=128, y=p, ldy=14336, od=0, ws=p, wsb=1 << 30):
+        return f(x8, ldx8, s_x, M, codes, gs, gz, fmt, s_w, sws, N, K, group, y, ldy, od, ws, wsb, None)
+
+    assert call(fmt=3) == binding.ERR_INVALID_ARG
+    assert call(gs=None) == binding.ERR_INVALID_ARG
+    assert call(fmt=2, gs=None, ws=None, wsb=0) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert call(fmt=1, gs=None, wsb=1024) == binding.ERR_WORKSPACE_TOO_SMALL
 
     assert call(x8=None) == binding.ERR_INVALID_ARG
     assert call(M=0) == binding.ERR_INVALID_ARG
@@ -103,8 +113,16 @@ def test_rtn_and_host_forward_reject_bad_arguments(L):
     assert f(p, 16, 128, 128, 0, 0, 0, p, p, None, p, None) == binding.ERR_INVALID_ARG   # asymmetric needs gzero
     assert f(p, 16, 130, 128, 1, 0, 0, p, p, None, p, None) == binding.ERR_BAD_SHAPE
     h = L.w4a8_forward_host
-    assert h(None, 4, p, p, None, p, 0, 16, 128, 128, p, p, p, p, p, None, 0, None) == binding.ERR_INVALID_ARG
-    assert h(p, 4, p, p, None, p, 0, 16, 100, 128, p, p, p, p, p, None, 0, None) == binding.ERR_BAD_SHAPE
+    assert h(None, 4, p, p, None, 0, p, 0, 16, 128, 128, p, p, p, p, p, None, 0, None) == binding.ERR_INVALID_ARG
+    assert h(p, 4, p, p, None, 0, p, 0, 16, 100, 128, p, p, p, p, p, None, 0, None) == binding.ERR_BAD_SHAPE
+    assert h(p, 4, p, p, None, 9, p, 0, 16, 128, 128, p, p, p, p, p, None, 0, None) == binding.ERR_INVALID_ARG
+    k = L.w4a8_prepack_weight
+    assert k(None, p, None, 16, 128, 128, 1, p, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert k(p, p, None, 16, 128, 128, 0, p, 1 << 20, None) == binding.ERR_INVALID_ARG      # canonical is not a target
+    assert k(p, p, p, 16, 128, 128, 2, p, 1 << 20, None) == binding.ERR_INVALID_ARG          # sign-magnitude needs z = 8
+    assert k(p, p, None, 16, 100, 128, 1, p, 1 << 20, None) == binding.ERR_BAD_SHAPE
+    assert k(p, p, None, 16, 128, 128, 1, _fake(0x1010), 1 << 20, None) == binding.ERR_BAD_ALIGNMENT
+    assert k(p, p, None, 16, 128, 128, 1, p, 100, None) == binding.ERR_WORKSPACE_TOO_SMALL
     assert L.w4a8_query_device_status(None) == binding.ERR_INVALID_ARG
 
 

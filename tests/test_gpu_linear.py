@@ -8,15 +8,24 @@ import torch
 import oracle
 from gpu_utils import bf16_bits, bf16_dev, dev, weights_to_dev
 from helpers import bf16_gate, e4m3_value_table, fp32_gate, pack_codes
+from helpers import unpack_codes as helpers_unpack
 from paper_2505_14638_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [binding.ALGO_UMMA, binding.ALGO_SIMT]
+ALGOS = [binding.ALGO_UMMA, binding.ALGO_SIMT, "tiled"]
 
 
 def _gpu_linear(x8, s_x, wq, out_dtype, algo=binding.ALGO_AUTO, split_k=0):
-    y = binding.linear(dev(x8), dev(s_x), *weights_to_dev(*wq), out_dtype=out_dtype, algo=algo, split_k=split_k)
+    """algo "tiled": prepack (sign-magnitude format when the storage is symmetric, generic tiled
+    otherwise) and run the persistent kernel; "tiled_generic" forces the generic tiled format."""
+    wd = weights_to_dev(*wq)
+    if algo in ("tiled", "tiled_generic"):
+        fmt = binding.FMT_TILED if (algo == "tiled_generic" or wq[2] is not None) else binding.FMT_TILED_SIGNMAG
+        tw = binding.prepack_weight(*wd, weight_format=fmt)
+        y = binding.linear_tiled(dev(x8), dev(s_x), tw, out_dtype=out_dtype)
+    else:
+        y = binding.linear(dev(x8), dev(s_x), *wd, out_dtype=out_dtype, algo=algo, split_k=split_k)
     torch.cuda.synchronize()
     assert binding.query_device_status() == 0
     return y
@@ -63,11 +72,14 @@ def test_exact_integer_inputs_are_bit_exact(algo, M, N, K):
     gs = inputs.f32_to_bf16_bits(np.ones((N, K // 128), dtype=np.float32))
     gz = rng.integers(4, 12, size=(N, K // 128)).astype(np.uint8)
     s_w = np.ones(1, dtype=np.float32)
-    wq = (codes, gs, gz, s_w)
-    ref = oracle.linear(x8, s_x, oracle.dequant_weight(codes, gs, gz), s_w)
-    y = _gpu_linear(x8, s_x, wq, binding.OUT_FP32, algo).cpu().numpy()
-    assert np.array_equal(y, ref["y32"])
-    assert np.array_equal(y.astype(np.float64), ref["y64"])
+    for wq in ((codes, gs, gz, s_w), (codes, gs, None, s_w)):
+        ref = oracle.linear(x8, s_x, oracle.dequant_weight(*wq[:3]), s_w)
+        y = _gpu_linear(x8, s_x, wq, binding.OUT_FP32, algo).cpu().numpy()
+        assert np.array_equal(y, ref["y32"])
+        assert np.array_equal(y.astype(np.float64), ref["y64"])
+        if algo == "tiled" and wq[2] is None:
+            y = _gpu_linear(x8, s_x, wq, binding.OUT_FP32, "tiled_generic").cpu().numpy()
+            assert np.array_equal(y, ref["y32"])
 
 
 @pytest.mark.parametrize("M,N,K,asym,pc", [(16, 1024, 1024, False, False),      # config c1
@@ -80,6 +92,71 @@ def test_exact_integer_inputs_are_bit_exact(algo, M, N, K):
 def test_gaussian_inputs_within_gates(M, N, K, asym, pc):
     x8, s_x, wq = _gaussian_case(M, N, K, seed=M + N + K, asym=asym, per_channel=pc)
     _check(x8, s_x, wq)
+    _check(x8, s_x, wq, algo="tiled")
+    if not asym:
+        _check(x8, s_x, wq, algo="tiled_generic")
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 128, 128), (1, 16, 14336), (16, 4096, 4096), (8, 6144, 4096),
+                                   (32, 4096, 14336), (64, 1024, 2048), (128, 2048, 1024), (512, 1024, 1024),
+                                   (300, 640, 8192)])
+def test_persistent_kernel_split_tiles_and_reuse_of_workspace(M, N, K):
+    # shapes whose tiles are split between CTAs in many ways; the workspace is shared by
+    # consecutive calls (the kernel leaves its counters zeroed) and results repeat bit for bit
+    x8, s_x, wq = _gaussian_case(M, N, K, seed=M * 3 + N + K)
+    w8 = oracle.dequant_weight(*wq[:3])
+    rng = np.random.default_rng(M + N)
+    cols = np.unique(np.concatenate([rng.choice(N, min(N, 64), replace=False), [0, N - 1]]))
+    ref = oracle.linear(x8, s_x, w8, wq[3], cols=cols)
+    tw = binding.prepack_weight(*weights_to_dev(*wq))
+    ws = binding.new_workspace(M, N, K, tw.fmt)
+    xd, sd = dev(x8), dev(s_x)
+    outs = []
+    for _ in range(3):
+        outs.append(binding.linear_tiled(xd, sd, tw, out_dtype=binding.OUT_FP32, workspace=ws).clone())
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    worst, _ = fp32_gate(outs[0].cpu().numpy()[:, cols], ref["y64"])
+    assert worst <= 2e-3, worst
+    bnx = next(b for b in (16, 32, 64, 128, 256) if M <= b or b == 256)
+    n_counters = ((M + bnx - 1) // bnx) * ((N + 127) // 128)
+    assert np.all(ws[: 4 * n_counters].cpu().numpy() == 0)      # tile counters are back to zero
+
+
+def test_sign_magnitude_prepack_flags_code_zero():
+    codes, gs, _ = inputs.random_codes(128, 256, seed=1)          # random nibbles include code 0
+    cd, gd = dev(codes), bf16_dev(gs)
+    binding.prepack_weight(cd, gd, None, None, weight_format=binding.FMT_TILED_SIGNMAG)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 2
+    assert binding.query_device_status() == 0                     # reading clears it
+    binding.prepack_weight(cd, gd, None, None, weight_format=binding.FMT_TILED)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+
+
+def test_tiled_formats_see_the_same_fp8_weights_as_eq10():
+    # one-hot FP8 activations (value 1.0, s_x = 1) read the dequantized weights back through the
+    # GEMM: Y[m][n] = w8[n][k_m] exactly, for every code, zero-point and a spread of scales
+    N, K = 256, 512
+    codes, gs, gz = inputs.random_codes(N, K, seed=21, asymmetric=True)
+    M = 64
+    ks = (np.arange(M) * 37) % K
+    x8 = np.zeros((M, K), dtype=np.uint8)
+    x8[np.arange(M), ks] = 0x38                                    # 1.0
+    s_x = np.ones(M, dtype=np.float32)
+    s_w = np.ones(1, dtype=np.float32)
+    tab = e4m3_value_table()
+    w8 = oracle.dequant_weight(codes, gs, gz)
+    y = _gpu_linear(x8, s_x, (codes, gs, gz, s_w), binding.OUT_FP32, "tiled").cpu().numpy()
+    assert np.array_equal(y.astype(np.float64), tab[w8][:, ks].T)
+    sym_u = np.clip(helpers_unpack(codes), 1, 15)
+    codes_s = pack_codes(sym_u.astype(np.uint8))
+    w8s = oracle.dequant_weight(codes_s, gs, None)
+    for algo in ("tiled", "tiled_generic"):
+        y = _gpu_linear(x8, s_x, (codes_s, gs, None, s_w), binding.OUT_FP32, algo).cpu().numpy()
+        assert np.array_equal(y.astype(np.float64), tab[w8s][:, ks].T), algo
 
 
 @pytest.mark.parametrize("split_k", [1, 2, 4, 8])
@@ -120,6 +197,7 @@ def test_config_c2_decode_full(M):
     K, N = 4096, 14336
     x8, s_x, wq = _gaussian_case(M, N, K, seed=2)
     _check(x8, s_x, wq)
+    _check(x8, s_x, wq, algo="tiled")
 
 
 def test_config_c3_prefill_sampled_columns():
@@ -129,6 +207,7 @@ def test_config_c3_prefill_sampled_columns():
     cols = np.unique(np.concatenate([rng.choice(N, 96, replace=False),
                                      np.array([0, 127, 128, 255, 256, 2047, 2048, N - 129, N - 128, N - 1])]))
     _check(x8, s_x, wq, cols=cols)
+    _check(x8, s_x, wq, algo="tiled", cols=cols)
 
 
 def test_whole_path_from_bf16_activations():
@@ -151,11 +230,13 @@ def test_host_forward_entry_point():
     W = inputs.make_weight(N, K, 0.02, 13)
     wq = oracle.quantize_weight_rtn(W, symmetric=True)
     xb = inputs.make_activation(M, K, 13, 0.01, 20.0)
-    fwd = binding.HostForward(M, *weights_to_dev(*wq))
-    x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
-    y_host = fwd(x_host)
-    torch.cuda.synchronize()
     ref = oracle.forward(xb, *wq)
-    ok, dist = bf16_gate(bf16_bits(y_host), ref["y64"])
-    assert ok, dist
-    assert fwd.h2d_bytes == M * K * 2 and fwd.d2h_bytes == M * N * 2
+    x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    wd = weights_to_dev(*wq)
+    for weight in (wd, binding.prepack_weight(*wd)):
+        fwd = binding.HostForward(M, weight)
+        y_host = fwd(x_host)
+        torch.cuda.synchronize()
+        ok, dist = bf16_gate(bf16_bits(y_host), ref["y64"])
+        assert ok, dist
+        assert fwd.h2d_bytes == M * K * 2 and fwd.d2h_bytes == M * N * 2

@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "../../include/w4a8.h"
+#include "w4a8_linear_splitn.cuh"
 #include "w4a8_linear_streamk.cuh"
 #include "w4a8_linear_umma.cuh"
 #include "w4a8_simple_kernels.cuh"
@@ -180,6 +181,8 @@ struct SkPlan {
     size_t counter_bytes, workspace_bytes;
 };
 
+constexpr int kSplitNMaxM = 64;  // token counts served by the split-N (decode) kernel
+
 static void make_sk_plan(int64_t M, int64_t N, int64_t K, SkPlan* pl) {
     pl->bnx = pick_bnx(M);
     pl->ctas_per_sm = pl->bnx <= 32 ? 2 : 1;
@@ -217,9 +220,94 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     return launch_status();
 }
 
+// Row partition and ring sizes of the split-N kernel for the current device.
+template <class Cfg>
+static bool make_sn_plan(int64_t N, int64_t K, int sms, SnPlan* pl) {
+    const int64_t NP = N / 8;
+    int64_t P = sms < NP ? sms : NP;
+    int64_t per = (NP + 32 * P - 1) / (32 * P);  // ranges per CTA so that none exceeds 256 rows
+    pl->T = (int)(P * per);
+    const int rmax = (int)((NP + pl->T - 1) / pl->T) * 8;
+    // Several k-blocks per pipeline stage keep the per-stage control work of the single-thread
+    // roles (copy issue, MMA issue, commits) small against the bytes a stage carries.
+    pl->KS = rmax > 128 ? 1 : (rmax > 64 ? 2 : 4);
+    while ((int64_t)pl->KS > K / 128) pl->KS /= 2;
+    pl->S2 = pl->KS * rmax > 128 ? 3 : 4;
+    pl->meta_off = pl->KS * rmax * kRowCodeBytes;
+    pl->wstage = (pl->KS * rmax * (kRowCodeBytes + Cfg::kMeta) + 127) / 128 * 128;
+    pl->xstage = pl->KS * Cfg::MT * 128;
+    pl->w8stage = pl->KS * rmax * 128;
+    int fixed = pl->S2 * pl->w8stage + Cfg::kBarBytes + 1024;
+    int s1 = (Cfg::kSmemBudget - fixed) / (pl->wstage + pl->xstage);
+    if (s1 > Cfg::kS1Max) s1 = Cfg::kS1Max;
+    if (s1 < 2) return false;
+    if (s1 < pl->S2) {  // the dequantized ring may not be deeper than the TMA ring
+        pl->S2 = s1;
+        fixed = pl->S2 * pl->w8stage + Cfg::kBarBytes + 1024;
+    }
+    pl->S1 = s1;
+    pl->smem = s1 * (pl->wstage + pl->xstage) + fixed;
+    return true;
+}
+
+template <class Cfg>
+static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
+                         int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, cudaStream_t st) {
+    auto kern = linear_splitn_kernel<Cfg>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBudget);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    unsigned int* status = status_word_ptr();
+    const int sms = sm_count();
+    if (!status || sms <= 0) return W4A8_ERR_CUDA;
+    SnPlan pl;
+    if (!make_sn_plan<Cfg>(N, K, sms, &pl)) return W4A8_ERR_BAD_SHAPE;
+    const int P = pl.T < sms ? pl.T : sms;
+    int vec_ok = (reinterpret_cast<uintptr_t>(y) & 15u) == 0 &&
+                 (out_dtype == W4A8_OUT_FP32 ? (ldy % 4 == 0) : (ldy % 8 == 0));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P);
+    cfg.blockDim = dim3(Cfg::kThreads);
+    cfg.dynamicSmemBytes = (size_t)pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, vec_ok, M, N, K, pl,
+                                       status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) return W4A8_ERR_CUDA;
+    return launch_status();
+}
+
 static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* wpp,
                              int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
                              int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (M <= kSplitNMaxM) {
+        int rc = check_device();
+        if (rc != W4A8_OK) return rc;
+        const int mt = M <= 16 ? 16 : 64;
+        CUtensorMap tx;
+        if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)mt,
+                             CU_TENSOR_MAP_SWIZZLE_128B))
+            return W4A8_ERR_CUDA;
+        const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+        if (fmt == kFmtTiledSignMag) {
+            return mt == 16 ? launch_splitn<SnCfg<16, 3, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                            out_dtype, Mi, Ni, Ki, st)
+                            : launch_splitn<SnCfg<64, 3, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                            out_dtype, Mi, Ni, Ki, st);
+        }
+        return mt == 16 ? launch_splitn<SnCfg<16, 3, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+                                                                 Ni, Ki, st)
+                        : launch_splitn<SnCfg<64, 3, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+                                                                 Ni, Ki, st);
+    }
     SkPlan pl;
     make_sk_plan(M, N, K, &pl);
     if (!workspace || workspace_bytes < pl.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
@@ -238,9 +326,6 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
              : launch_streamk<SkCfg<BNX, G, S1, S2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, \
                                                                 workspace, pl, Mi, Ni, Ki, st)
     switch (pl.bnx) {
-        case 16: W4A8_SK(16, 2, 5, 3); break;
-        case 32: W4A8_SK(32, 2, 4, 3); break;
-        case 64: W4A8_SK(64, 4, 6, 4); break;
         case 128: W4A8_SK(128, 4, 5, 4); break;
         default: W4A8_SK(256, 4, 4, 3); break;
     }
@@ -392,6 +477,7 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
     if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
     if (weight_format == kFmtCanonical) return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
+    if (M <= kSplitNMaxM) return 0;  // the split-N kernel needs none
     SkPlan pl;
     make_sk_plan(M, N, K, &pl);
     return pl.workspace_bytes;
@@ -400,7 +486,7 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
 size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format) {
     if (N <= 0 || K <= 0 || K % kGroup != 0) return 0;
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
-    return (size_t)((N + 127) / 128) * (size_t)(K / 128) * (size_t)chunk_bytes(weight_format);
+    return (size_t)N * (size_t)(K / 128) * (size_t)(kRowCodeBytes + meta_bytes(weight_format));
 }
 
 int w4a8_prepack_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero, int64_t N, int64_t K,
@@ -409,7 +495,7 @@ int w4a8_prepack_weight(const uint8_t* codes, const void* gscale_bf16, const uin
     if (N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
     if (weight_format == kFmtTiledSignMag && gzero != nullptr) return W4A8_ERR_INVALID_ARG;
-    if (group != kGroup || K % kGroup != 0) return W4A8_ERR_BAD_SHAPE;
+    if (group != kGroup || K % kGroup != 0 || N % 8 != 0) return W4A8_ERR_BAD_SHAPE;
     if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(out) & 127u) ||
         (reinterpret_cast<uintptr_t>(gscale_bf16) & 1u))
         return W4A8_ERR_BAD_ALIGNMENT;

@@ -17,11 +17,11 @@
 #include <cuda_bf16.h>
 
 #include "w4a8_ptx.cuh"
+#include "w4a8_tiled_format.cuh"
 
 namespace w4a8 {
 
 #ifdef W4A8_TIMING
-__device__ long long g_dbg[1024 * 16];
 #define DBG_STAMP(slot) g_dbg[blockIdx.x * 16 + (slot)] = clock64()
 #define DBG_ADD(slot, v) g_dbg[blockIdx.x * 16 + (slot)] += (v)
 #define DBG_SET(slot, v) g_dbg[blockIdx.x * 16 + (slot)] = (v)
@@ -31,35 +31,6 @@ __device__ long long g_dbg[1024 * 16];
 #define DBG_SET(slot, v)
 #endif
 
-// Weight formats (values of the weight_format argument of the C ABI).
-constexpr int kFmtCanonical = W4A8_FMT_CANONICAL;
-constexpr int kFmtTiled = W4A8_FMT_TILED;
-constexpr int kFmtTiledSignMag = W4A8_FMT_TILED_SIGNMAG;
-
-// One chunk = one (weight tile, k-block): 128 rows x 64 bytes of codes, 128 BF16 scales and,
-// in the generic format, 128 zero-point bytes.
-constexpr int kChunkScaleOff = 8192;
-constexpr int kChunkZeroOff = 8192 + 256;
-__host__ __device__ constexpr int chunk_bytes(int fmt) { return fmt == kFmtTiledSignMag ? 8448 : 8576; }
-
-// Sign-magnitude table of a symmetric group (z = 8): entry d = nearest_E4M3(d * s), d = 0..7.
-// A stored nibble carries |u - 8| in its low three bits; the sign travels separately and is
-// applied by flipping the E4M3 sign bit (the format is sign-magnitude, rounding is symmetric).
-struct SignMagLut {
-    uint32_t t0, t1;
-    __device__ __forceinline__ void build(float s) {
-        t0 = cvt_e4m3x4(__fmul_rn(0.0f, s), s, __fmul_rn(2.0f, s), __fmul_rn(3.0f, s));
-        t1 = cvt_e4m3x4(__fmul_rn(4.0f, s), __fmul_rn(5.0f, s), __fmul_rn(6.0f, s), __fmul_rn(7.0f, s));
-    }
-    // Word layout: nibble i (i = 0..3) = magnitude of element i, nibble 4+i = magnitude of
-    // element 4+i; sign of element i in bit 8i+7, sign of element 4+i in bit 8i+3.
-    __device__ __forceinline__ void dequant8(uint32_t w, uint32_t& out0, uint32_t& out1) const {
-        const uint32_t sel = w & 0x77777777u;
-        out0 = prmt(t0, t1, sel) ^ (w & 0x80808080u);
-        out1 = prmt(t0, t1, sel >> 16) ^ ((w << 4) & 0x80808080u);
-    }
-};
-
 template <int BNX_, int G_, int S1_, int S2_, int FMT_>
 struct SkCfg {
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
@@ -67,8 +38,8 @@ struct SkCfg {
     static constexpr int S1 = S1_;     // ring of TMA stages (packed chunk + activation tile)
     static constexpr int S2 = S2_;     // ring of dequantized E4M3 weight tiles
     static constexpr int FMT = FMT_;
-    static constexpr int kChunk = chunk_bytes(FMT);
-    static constexpr int kWStage = 9216;  // chunk padded so that the activation tile stays 1024-aligned
+    static constexpr int kMeta = meta_bytes(FMT);
+    static constexpr int kWStage = 9216;  // 128 rows x (64 code bytes + meta), padded to keep the activation tile 1024-aligned
     static constexpr int kXBytes = BNX * 128;
     static constexpr int kStage1 = kWStage + kXBytes;
     static constexpr int kW8Bytes = 128 * 128;
@@ -86,7 +57,7 @@ struct SkCfg {
 template <class Cfg>
 __global__ void __launch_bounds__(Cfg::kThreads)
 linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x BNX, 128B swizzle
-                      const uint8_t* __restrict__ wpp,             // tiled weights, chunk (nt, kb) at (nt*KB+kb)*kChunk
+                      const uint8_t* __restrict__ wpp,             // tiled weights (panels, k-block major)
                       const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                       void* __restrict__ y, int64_t ldy, int out_dtype, unsigned int* counters,
                       float* slots, int M, int N, int K, int TM, int TN, unsigned int* status_word) {
@@ -118,6 +89,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = K >> 7;
+    const uint8_t* meta_base = wpp + (int64_t)KB * N * kRowCodeBytes;
     const int64_t U = (int64_t)TM * TN * KB;
     const int64_t P = gridDim.x, p = blockIdx.x;
     const int64_t u_begin = p * U / P, u_end = (p + 1) * U / P;
@@ -167,8 +139,13 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     if (!ok) break;
                 }
                 const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
-                ptx::mbar_arrive_expect_tx(bar_full(s), (uint32_t)(Cfg::kChunk + Cfg::kXBytes));
-                ptx::bulk_load(stage_w(s), wpp + ((int64_t)nt * KB + kb) * Cfg::kChunk, Cfg::kChunk, bar_full(s));
+                const int rows = (N - nt * 128) < 128 ? (N - nt * 128) : 128;  // ragged last tile
+                const int64_t row0 = (int64_t)kb * N + (int64_t)nt * 128;
+                ptx::mbar_arrive_expect_tx(bar_full(s),
+                                           (uint32_t)(rows * (kRowCodeBytes + Cfg::kMeta) + Cfg::kXBytes));
+                ptx::bulk_load(stage_w(s), wpp + row0 * kRowCodeBytes, (uint32_t)(rows * kRowCodeBytes), bar_full(s));
+                ptx::bulk_load(stage_w(s) + 8192u, meta_base + row0 * Cfg::kMeta, (uint32_t)(rows * Cfg::kMeta),
+                               bar_full(s));
                 ptx::tma_load_2d(stage_x(s), &tmap_x, kb * 128, mt * BNX, bar_full(s));
                 issued = it + 1;
                 if (++kb == KB) {
@@ -332,8 +309,6 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         const int dw = warp - 6;
         const int g = dw >> 2;
         const int r = (dw & 3) * 32 + lane;
-        const uint32_t sw64 = (uint32_t)((r >> 1) & 3);
-        const uint32_t sw128 = (uint32_t)(r & 7);
         for (int it = g; it < n_it; it += G) {
             const int s1 = it % S1, s2 = it % S2;
 #ifdef W4A8_TIMING
@@ -344,26 +319,6 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             long long tq1 = clock64();
             if (dw == 0 && lane == 0) DBG_ADD(8, tq1 - tq0);
 #endif
-            const uint32_t src = stage_w(s1);
-            uint32_t sc_bits;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sc_bits) : "r"(src + kChunkScaleOff + 2u * (uint32_t)r));
-            const float sc = bf16_bits_to_float(sc_bits);
-            uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                             : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
-                             : "r"(src + (uint32_t)r * 64u + (((uint32_t)c ^ sw64) << 4)));
-            }
-            SignMagLut slut;
-            DequantLut glut;
-            if constexpr (Cfg::FMT == kFmtTiledSignMag) {
-                slut.build(sc);
-            } else {
-                uint32_t z;
-                asm volatile("ld.shared.u8 %0, [%1];" : "=r"(z) : "r"(src + kChunkZeroOff + (uint32_t)r));
-                glut.build(sc, (int)z);
-            }
 #ifdef W4A8_TIMING
             long long tq2 = clock64();
 #endif
@@ -374,21 +329,9 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             long long tq3 = clock64();
             if (dw == 0 && lane == 0) { DBG_ADD(9, tq2 - tq1); DBG_ADD(10, tq3 - tq2); }
 #endif
-            const uint32_t dst = stage_w8(s2) + (uint32_t)r * 128u;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint32_t o0, o1, o2, o3;
-                if constexpr (Cfg::FMT == kFmtTiledSignMag) {
-                    slut.dequant8(pk[2 * c], o0, o1);
-                    slut.dequant8(pk[2 * c + 1], o2, o3);
-                } else {
-                    glut.dequant8(pk[2 * c], o0, o1);
-                    glut.dequant8(pk[2 * c + 1], o2, o3);
-                }
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)),
-                             "r"(o0), "r"(o1), "r"(o2), "r"(o3)
-                             : "memory");
-            }
+            dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + (uint32_t)r * 64u,
+                                          stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
+                                          stage_w8(s2) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
 #ifdef W4A8_TIMING
@@ -405,73 +348,6 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
     if (threadIdx.x == 32) { DBG_STAMP(7); DBG_SET(14, (long long)ptx::globaltimer_ns()); }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Offline prepack: canonical [N][K/2] codes + [N][K/128] scales (+ zero-points) -> tiled chunks.
-// One CTA per (weight tile, k-block), one thread per row.  Rows beyond N are filled with zero
-// weights.  In the sign-magnitude format a code 0 (value -8 s) cannot be represented: it is
-// stored as -7 s and the "unrepresentable code" status bit is raised.
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t to_signmag_word(uint32_t w, bool& bad) {
-    uint32_t out = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        int u = (int)((w >> (4 * i)) & 15u);
-        int d = u - 8;
-        uint32_t sign = d < 0 ? 1u : 0u;
-        int mag = d < 0 ? -d : d;
-        if (mag > 7) {
-            bad = true;
-            mag = 7;
-        }
-        out |= (uint32_t)mag << (4 * i);
-        const int sign_bit = (i < 4) ? (8 * i + 7) : (8 * (i - 4) + 3);
-        out |= sign << sign_bit;
-    }
-    return out;
-}
-
-__global__ void __launch_bounds__(128)
-prepack_kernel(const uint8_t* __restrict__ codes, const uint16_t* __restrict__ gscale,
-               const uint8_t* __restrict__ gzero, int64_t N, int64_t K, int fmt, uint8_t* __restrict__ out,
-               unsigned int* status_word) {
-    const int64_t KB = K >> 7;
-    const int64_t nt = blockIdx.x / KB, kb = blockIdx.x - nt * KB;
-    const int r = threadIdx.x;
-    const int64_t n = nt * 128 + r;
-    const int chunk = chunk_bytes(fmt);
-    uint8_t* dst = out + (int64_t)blockIdx.x * chunk;
-    uint4 w[4];
-    uint16_t sc = 0;
-    uint8_t z = 8;
-    if (n < N) {
-        const uint4* src = reinterpret_cast<const uint4*>(codes + n * (K >> 1) + kb * 64);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) w[c] = src[c];
-        sc = gscale[n * KB + kb];
-        if (gzero) z = gzero[n * KB + kb];
-    } else {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) w[c] = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);
-    }
-    if (fmt == kFmtTiledSignMag) {
-        bool bad = false;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            w[c].x = to_signmag_word(w[c].x, bad);
-            w[c].y = to_signmag_word(w[c].y, bad);
-            w[c].z = to_signmag_word(w[c].z, bad);
-            w[c].w = to_signmag_word(w[c].w, bad);
-        }
-        if (bad) atomicOr(status_word, kStatusBadCode);
-    }
-    const uint32_t sw64 = (uint32_t)((r >> 1) & 3);
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-        *reinterpret_cast<uint4*>(dst + r * 64 + (((uint32_t)c ^ sw64) << 4)) = w[c];
-    *reinterpret_cast<uint16_t*>(dst + kChunkScaleOff + 2 * r) = sc;
-    if (fmt != kFmtTiledSignMag) dst[kChunkZeroOff + r] = z;
 }
 
 }  // namespace w4a8

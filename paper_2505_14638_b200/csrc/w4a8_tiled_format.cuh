@@ -1,0 +1,151 @@
+// Tiled ("prepacked") weight layout shared by the persistent GEMM kernels, the sign-magnitude
+// look-up table for symmetric groups, and the offline prepack kernel.
+//
+// Layout (K = 128 KB k-blocks, N output channels):
+//   codes region  [KB][N][64 bytes]   row n of k-block kb at ((kb * N) + n) * 64; within a row the
+//                 16-byte chunk c is stored at chunk position c ^ ((n >> 1) & 3), so that eight
+//                 consecutive rows read with 128-bit loads touch every shared-memory bank once
+//   meta region   [KB][N][MB bytes]   starts at KB * N * 64; MB = 2 (BF16 group scale) in the
+//                 sign-magnitude format, 4 (BF16 scale, zero-point byte, one byte of padding) in
+//                 the generic format
+// Any run of consecutive output channels of one k-block is therefore one contiguous, 128-byte
+// aligned piece of codes plus one contiguous piece of meta data: two bulk copies bring it into
+// shared memory, whatever row partition the kernel picks at launch.
+#pragma once
+
+#include "w4a8_common.cuh"
+
+namespace w4a8 {
+
+constexpr int kFmtCanonical = W4A8_FMT_CANONICAL;
+constexpr int kFmtTiled = W4A8_FMT_TILED;
+constexpr int kFmtTiledSignMag = W4A8_FMT_TILED_SIGNMAG;
+
+constexpr int kRowCodeBytes = 64;  // one row of one k-block: 128 INT4 codes
+__host__ __device__ constexpr int meta_bytes(int fmt) { return fmt == kFmtTiledSignMag ? 2 : 4; }
+
+// Sign-magnitude table of a symmetric group (z = 8): entry d = nearest_E4M3(d * s), d = 0..7.
+// A stored nibble carries |u - 8| in its low three bits; the sign travels separately and is
+// applied by flipping the E4M3 sign bit (the format is sign-magnitude and the rounding is
+// symmetric, so nearest_E4M3(-d s) and nearest_E4M3(d s) differ in that bit only).
+struct SignMagLut {
+    uint32_t t0, t1;
+    __device__ __forceinline__ void build(float s) {
+        t0 = cvt_e4m3x4(__fmul_rn(0.0f, s), s, __fmul_rn(2.0f, s), __fmul_rn(3.0f, s));
+        t1 = cvt_e4m3x4(__fmul_rn(4.0f, s), __fmul_rn(5.0f, s), __fmul_rn(6.0f, s), __fmul_rn(7.0f, s));
+    }
+    // Word layout: nibble i (i = 0..3) = magnitude of element i, nibble 4+i = magnitude of
+    // element 4+i; sign of element i in bit 8i+7, sign of element 4+i in bit 8i+3.
+    __device__ __forceinline__ void dequant8(uint32_t w, uint32_t& out0, uint32_t& out1) const {
+        const uint32_t sel = w & 0x77777777u;
+        out0 = prmt(t0, t1, sel) ^ (w & 0x80808080u);
+        out1 = prmt(t0, t1, sel >> 16) ^ ((w << 4) & 0x80808080u);
+    }
+};
+
+// Expands one row of one k-block into 128 E4M3 bytes written as a row of a K-major tile with
+// the 128-byte swizzle.  `src` = shared address of the row's 64 code bytes, `meta` = shared
+// address of its meta entry, `row` = row index within the copied piece (the piece must start on
+// a multiple of 8 rows), `dst` = shared address of the destination row.
+template <int FMT>
+__device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta, int row, uint32_t dst) {
+    const uint32_t sw64 = (uint32_t)((row >> 1) & 3);
+    const uint32_t sw128 = (uint32_t)(row & 7);
+    uint32_t mbits;
+    if constexpr (FMT == kFmtTiledSignMag)
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    else
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
+    uint32_t pk[16];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
+                     : "r"(src + (((uint32_t)c ^ sw64) << 4)));
+    }
+    SignMagLut slut;
+    DequantLut glut;
+    if constexpr (FMT == kFmtTiledSignMag)
+        slut.build(sc);
+    else
+        glut.build(sc, (int)((mbits >> 16) & 0xFFu));
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t o0, o1, o2, o3;
+        if constexpr (FMT == kFmtTiledSignMag) {
+            slut.dequant8(pk[2 * c], o0, o1);
+            slut.dequant8(pk[2 * c + 1], o2, o3);
+        } else {
+            glut.dequant8(pk[2 * c], o0, o1);
+            glut.dequant8(pk[2 * c + 1], o2, o3);
+        }
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)), "r"(o0),
+                     "r"(o1), "r"(o2), "r"(o3)
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Offline prepack: canonical [N][K/2] codes + [N][K/128] scales (+ zero-points) -> tiled buffer.
+// One CTA per (128 rows, k-block), one thread per row.  In the sign-magnitude format a code 0
+// (value -8 s) cannot be represented: it is stored as -7 s and the "unrepresentable code" status
+// bit is raised.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t to_signmag_word(uint32_t w, bool& bad) {
+    uint32_t out = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        int u = (int)((w >> (4 * i)) & 15u);
+        int d = u - 8;
+        uint32_t sign = d < 0 ? 1u : 0u;
+        int mag = d < 0 ? -d : d;
+        if (mag > 7) {
+            bad = true;
+            mag = 7;
+        }
+        out |= (uint32_t)mag << (4 * i);
+        const int sign_bit = (i < 4) ? (8 * i + 7) : (8 * (i - 4) + 3);
+        out |= sign << sign_bit;
+    }
+    return out;
+}
+
+__global__ void __launch_bounds__(128)
+prepack_kernel(const uint8_t* __restrict__ codes, const uint16_t* __restrict__ gscale,
+               const uint8_t* __restrict__ gzero, int64_t N, int64_t K, int fmt, uint8_t* __restrict__ out,
+               unsigned int* status_word) {
+    const int64_t KB = K >> 7;
+    const int64_t rt = blockIdx.x / KB, kb = blockIdx.x - rt * KB;
+    const int64_t n = rt * 128 + threadIdx.x;
+    if (n >= N) return;
+    const uint4* src = reinterpret_cast<const uint4*>(codes + n * (K >> 1) + kb * 64);
+    uint4 w[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) w[c] = src[c];
+    if (fmt == kFmtTiledSignMag) {
+        bool bad = false;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            w[c].x = to_signmag_word(w[c].x, bad);
+            w[c].y = to_signmag_word(w[c].y, bad);
+            w[c].z = to_signmag_word(w[c].z, bad);
+            w[c].w = to_signmag_word(w[c].w, bad);
+        }
+        if (bad) atomicOr(status_word, kStatusBadCode);
+    }
+    uint8_t* dst = out + (kb * N + n) * kRowCodeBytes;
+    const uint32_t sw64 = (uint32_t)((n >> 1) & 3);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(dst + (((uint32_t)c ^ sw64) << 4)) = w[c];
+    uint8_t* meta = out + KB * N * kRowCodeBytes + (kb * N + n) * meta_bytes(fmt);
+    const uint16_t sc = gscale[n * KB + kb];
+    if (fmt == kFmtTiledSignMag) {
+        *reinterpret_cast<uint16_t*>(meta) = sc;
+    } else {
+        const uint32_t z = gzero ? (uint32_t)gzero[n * KB + kb] : 8u;
+        *reinterpret_cast<uint32_t*>(meta) = (uint32_t)sc | (z << 16);
+    }
+}
+
+}  // namespace w4a8

@@ -35,11 +35,12 @@ def test_status_strings(L):
 
 
 def test_workspace_and_prepack_size_queries_are_host_only(L):
-    assert L.w4a8_prepack_bytes(14336, 4096, binding.FMT_TILED_SIGNMAG) == 112 * 32 * 8448
-    assert L.w4a8_prepack_bytes(14336 + 16, 4096, binding.FMT_TILED) == 113 * 32 * 8576
+    assert L.w4a8_prepack_bytes(14336, 4096, binding.FMT_TILED_SIGNMAG) == 14336 * 32 * 66
+    assert L.w4a8_prepack_bytes(14336 + 16, 4096, binding.FMT_TILED) == (14336 + 16) * 32 * 68
     assert L.w4a8_prepack_bytes(14336, 4096, binding.FMT_CANONICAL) == 0
-    ws = binding.linear_workspace_bytes(16, 14336, 4096, weight_format=binding.FMT_TILED_SIGNMAG)
-    assert ws >= 112 * 4 + 2 * 296 * 16 * 128 * 4
+    assert binding.linear_workspace_bytes(16, 14336, 4096, weight_format=binding.FMT_TILED_SIGNMAG) == 0
+    ws = binding.linear_workspace_bytes(2048, 4096, 4096, weight_format=binding.FMT_TILED_SIGNMAG)
+    assert ws >= 8 * 32 * 4 + 2 * 148 * 256 * 128 * 4
     assert binding.linear_workspace_bytes(2048, 4096, 4096) == 0          # large M: no split
     ws = binding.linear_workspace_bytes(16, 14336, 4096)
     assert ws % (16 * 14336 * 4) == 0 and ws > 0                          # S partial tiles
@@ -83,8 +84,8 @@ def test_linear_rejects_bad_arguments(L):
 
     assert call(fmt=3) == binding.ERR_INVALID_ARG
     assert call(gs=None) == binding.ERR_INVALID_ARG
-    assert call(fmt=2, gs=None, ws=None, wsb=0) == binding.ERR_WORKSPACE_TOO_SMALL
-    assert call(fmt=1, gs=None, wsb=1024) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert call(fmt=2, gs=None, M=512, ws=None, wsb=0) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert call(fmt=1, gs=None, M=512, wsb=1024) == binding.ERR_WORKSPACE_TOO_SMALL
 
     assert call(x8=None) == binding.ERR_INVALID_ARG
     assert call(M=0) == binding.ERR_INVALID_ARG

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/w4a8.h"
@@ -223,28 +224,21 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
 // Row partition and ring sizes of the split-N kernel for the current device.
 template <class Cfg>
 static bool make_sn_plan(int64_t N, int64_t K, int sms, SnPlan* pl) {
-    const int64_t NP = N / 8;
-    int64_t P = sms < NP ? sms : NP;
-    int64_t per = (NP + 32 * P - 1) / (32 * P);  // ranges per CTA so that none exceeds 256 rows
+    const int64_t NU = N / 8;
+    int64_t P = sms < NU ? sms : NU;
+    int64_t per = (NU + 32 * P - 1) / (32 * P);  // ranges per CTA so that none exceeds 256 rows
     pl->T = (int)(P * per);
-    const int rmax = (int)((NP + pl->T - 1) / pl->T) * 8;
-    // Several k-blocks per pipeline stage keep the per-stage control work of the single-thread
-    // roles (copy issue, MMA issue, commits) small against the bytes a stage carries.
-    pl->KS = rmax > 128 ? 1 : (rmax > 64 ? 2 : 4);
-    while ((int64_t)pl->KS > K / 128) pl->KS /= 2;
-    pl->S2 = pl->KS * rmax > 128 ? 3 : 4;
+    const int rmax = (int)((NU + pl->T - 1) / pl->T) * 8;
+    pl->MBLK = rmax > 128 ? 2 : 1;
+    pl->KS = Cfg::kItems / pl->MBLK;
+    if ((int64_t)pl->KS > K / 128) pl->KS = 1;
     pl->meta_off = pl->KS * rmax * kRowCodeBytes;
     pl->wstage = (pl->KS * rmax * (kRowCodeBytes + Cfg::kMeta) + 127) / 128 * 128;
     pl->xstage = pl->KS * Cfg::MT * 128;
-    pl->w8stage = pl->KS * rmax * 128;
-    int fixed = pl->S2 * pl->w8stage + Cfg::kBarBytes + 1024;
+    const int fixed = Cfg::kBarBytes + 1024;
     int s1 = (Cfg::kSmemBudget - fixed) / (pl->wstage + pl->xstage);
     if (s1 > Cfg::kS1Max) s1 = Cfg::kS1Max;
-    if (s1 < 2) return false;
-    if (s1 < pl->S2) {  // the dequantized ring may not be deeper than the TMA ring
-        pl->S2 = s1;
-        fixed = pl->S2 * pl->w8stage + Cfg::kBarBytes + 1024;
-    }
+    if (s1 < Cfg::kS2) return false;  // the tensor-memory ring may not be deeper than the TMA ring
     pl->S1 = s1;
     pl->smem = s1 * (pl->wstage + pl->xstage) + fixed;
     return true;
@@ -266,8 +260,6 @@ static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float*
     SnPlan pl;
     if (!make_sn_plan<Cfg>(N, K, sms, &pl)) return W4A8_ERR_BAD_SHAPE;
     const int P = pl.T < sms ? pl.T : sms;
-    int vec_ok = (reinterpret_cast<uintptr_t>(y) & 15u) == 0 &&
-                 (out_dtype == W4A8_OUT_FP32 ? (ldy % 4 == 0) : (ldy % 8 == 0));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)P);
     cfg.blockDim = dim3(Cfg::kThreads);
@@ -277,8 +269,8 @@ static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float*
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, vec_ok, M, N, K, pl,
+    cfg.numAttrs = getenv("W4A8_NO_PDL") ? 0 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, pl,
                                        status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;
@@ -298,14 +290,14 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
             return W4A8_ERR_CUDA;
         const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
         if (fmt == kFmtTiledSignMag) {
-            return mt == 16 ? launch_splitn<SnCfg<16, 3, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+            return mt == 16 ? launch_splitn<SnCfg<16, 4, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
                                                                             out_dtype, Mi, Ni, Ki, st)
-                            : launch_splitn<SnCfg<64, 3, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                            : launch_splitn<SnCfg<64, 4, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
                                                                             out_dtype, Mi, Ni, Ki, st);
         }
-        return mt == 16 ? launch_splitn<SnCfg<16, 3, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+        return mt == 16 ? launch_splitn<SnCfg<16, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                                  Ni, Ki, st)
-                        : launch_splitn<SnCfg<64, 3, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+                        : launch_splitn<SnCfg<64, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                                  Ni, Ki, st);
     }
     SkPlan pl;

@@ -14,6 +14,7 @@
 #pragma once
 
 #include "w4a8_common.cuh"
+#include "w4a8_ptx.cuh"
 
 namespace w4a8 {
 
@@ -83,6 +84,54 @@ __device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta,
         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)), "r"(o0),
                      "r"(o1), "r"(o2), "r"(o3)
                      : "memory");
+    }
+}
+
+// Same expansion into registers and from there into tensor memory: the row's 128 E4M3 bytes go
+// to 32 consecutive 32-bit columns starting at `taddr` (lane = this thread's lane within its
+// warp's lane quarter), written as two 16-column stores to keep the live register count low.
+// Warp-collective: every lane of the warp must call it (lanes with `active` false store zeros).
+template <int FMT>
+__device__ __forceinline__ void dequant_row_to_tmem(uint32_t src, uint32_t meta, int row, bool active, uint32_t taddr) {
+    const uint32_t sw64 = (uint32_t)((row >> 1) & 3);
+    uint32_t mbits = 0;
+    uint32_t pk[16];
+    if (active) {
+        if constexpr (FMT == kFmtTiledSignMag)
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
+        else
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
+                         : "r"(src + (((uint32_t)c ^ sw64) << 4)));
+        }
+    } else {
+#pragma unroll
+        for (int w = 0; w < 16; ++w) pk[w] = 0u;
+    }
+    const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
+    if constexpr (FMT == kFmtTiledSignMag) {
+        SignMagLut lut;
+        lut.build(sc);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t out[16];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) lut.dequant8(pk[8 * h + w], out[2 * w], out[2 * w + 1]);
+            ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
+        }
+    } else {
+        DequantLut lut;
+        lut.build(sc, (int)((mbits >> 16) & 0xFFu));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t out[16];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) lut.dequant8(pk[8 * h + w], out[2 * w], out[2 * w + 1]);
+            ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
+        }
     }
 }
 

@@ -402,7 +402,7 @@ def run_ours(args, rank, world, local_rank):
                 "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "linear_streamk_kernel<BNX=16> (w4a8_linear), mean over M in {1,4,16}",
+        "roofline": {"bound": "hbm", "kernel": "linear_splitn_kernel<MT=16> (w4a8_linear), mean over M in {1,4,16}",
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,

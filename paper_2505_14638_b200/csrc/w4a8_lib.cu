@@ -4,7 +4,6 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
-#include <cstdlib>
 #include <mutex>
 
 #include "../../include/w4a8.h"
@@ -269,7 +268,7 @@ static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float*
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = getenv("W4A8_NO_PDL") ? 0 : 1;
+    cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, pl,
                                        status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -290,12 +289,12 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
             return W4A8_ERR_CUDA;
         const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
         if (fmt == kFmtTiledSignMag) {
-            return mt == 16 ? launch_splitn<SnCfg<16, 4, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+            return mt == 16 ? launch_splitn<SnCfg<16, 2, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
                                                                             out_dtype, Mi, Ni, Ki, st)
                             : launch_splitn<SnCfg<64, 4, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
                                                                             out_dtype, Mi, Ni, Ki, st);
         }
-        return mt == 16 ? launch_splitn<SnCfg<16, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+        return mt == 16 ? launch_splitn<SnCfg<16, 2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                                  Ni, Ki, st)
                         : launch_splitn<SnCfg<64, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                                  Ni, Ki, st);
@@ -413,17 +412,34 @@ static int quantize_act_impl(const void* x, int64_t M, int64_t K, int64_t ldx, u
     const uint16_t* xs = static_cast<const uint16_t*>(x);
     const int64_t nchunks = K / 16;
     const unsigned rows = (unsigned)M;
-#define W4A8_AQ(T, C) \
-    act_quant_kernel<T, C><<<rows, T, 0, st>>>(xs, K, ldx, x8, ldx8, s_x, scale_mode, static_scale)
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rows);
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    cudaError_t lerr = cudaSuccess;
+#define W4A8_AQ(T, C)                                                                                         \
+    do {                                                                                                      \
+        cfg.blockDim = dim3(T);                                                                               \
+        lerr = cudaLaunchKernelEx(&cfg, act_quant_kernel<T, C>, xs, K, ldx, x8, ldx8, s_x, scale_mode,        \
+                                  static_scale);                                                              \
+    } while (0)
     if (nchunks <= 32) W4A8_AQ(32, 1);
     else if (nchunks <= 64) W4A8_AQ(64, 1);
     else if (nchunks <= 128) W4A8_AQ(128, 1);
     else if (nchunks <= 256) W4A8_AQ(256, 1);
     else if (nchunks <= 512) W4A8_AQ(256, 2);
     else if (nchunks <= 1024) W4A8_AQ(256, 4);
-    else act_quant_kernel_2pass<<<rows, 256, 0, st>>>(xs, K, ldx, x8, ldx8, s_x, scale_mode, static_scale);
+    else {
+        cfg.blockDim = dim3(256);
+        lerr = cudaLaunchKernelEx(&cfg, act_quant_kernel_2pass, xs, K, ldx, x8, ldx8, s_x, scale_mode, static_scale);
+    }
 #undef W4A8_AQ
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (lerr != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
 }
 

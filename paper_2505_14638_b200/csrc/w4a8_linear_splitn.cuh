@@ -53,15 +53,17 @@ struct SnCfg {
     static constexpr int G = G_;        // dequantization groups of 4 warps
     static constexpr int FMT = FMT_;
     static constexpr int kS1Max = 16;   // ring of TMA stages (runtime depth <= this)
-    static constexpr int kS2 = 4;       // ring of dequantized stages in tensor memory
+    static constexpr int kS2 = MT_ == 16 ? 3 : 4;  // ring of dequantized stages in tensor memory
     static constexpr int kItems = 2;    // (k-block, 128-row block) pairs per stage
     static constexpr int kMeta = meta_bytes(FMT);
-    static constexpr int kTmemCols = 512;
+    static constexpr int kTmemCols = MT_ == 16 ? 256 : 512;
     static constexpr int kAStageCols = kItems * 32;        // 128 bytes per row and item
     static constexpr int kDCol = kS2 * kAStageCols;        // accumulators start after the A ring
     static constexpr int kThreads = 32 * (6 + 4 * G);
     static constexpr int kBarBytes = 512;
-    static constexpr int kSmemBudget = 200 * 1024;
+    // Decode-sized launches (<= 16 tokens) take half an SM each, so that the CTAs of the next
+    // kernel in the stream can start -- and prefetch their weights -- while this one finishes.
+    static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : 200 * 1024;
     static_assert(MT == 16 || MT == 64, "token tile");
     static_assert(kDCol + 2 * MT <= kTmemCols, "tensor memory columns");
     static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 <= kBarBytes, "barrier area");

@@ -8,6 +8,7 @@
 #include <cuda_fp16.h>
 
 #include "w4a8_common.cuh"
+#include "w4a8_ptx.cuh"
 
 namespace w4a8 {
 
@@ -72,6 +73,11 @@ act_quant_kernel(const uint16_t* __restrict__ x, int64_t K, int64_t ldx, uint8_t
                  int64_t ldx8, float* __restrict__ s_x, int scale_mode,
                  const float* __restrict__ static_scale) {
     __shared__ float red[32];
+    // Launched with programmatic stream serialization: let the next kernel (the linear layer) start
+    // prefetching its weights right away, but wait for the previous one before touching X8 / s_x,
+    // which it may still be reading.
+    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();
     const int64_t row = blockIdx.x;
     const int nchunks = (int)(K >> 4);
     const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx);
@@ -123,6 +129,8 @@ act_quant_kernel_2pass(const uint16_t* __restrict__ x, int64_t K, int64_t ldx,
                        uint8_t* __restrict__ x8, int64_t ldx8, float* __restrict__ s_x,
                        int scale_mode, const float* __restrict__ static_scale) {
     __shared__ float red[32];
+    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();
     const int64_t row = blockIdx.x;
     const int nchunks = (int)(K >> 4);
     const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx);

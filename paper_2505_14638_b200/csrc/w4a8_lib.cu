@@ -212,10 +212,15 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     if (!status || sms <= 0) return W4A8_ERR_CUDA;
     int64_t P = (int64_t)pl.ctas_per_sm * (sms < kMaxSMs ? sms : kMaxSMs);
     if (P > pl.U) P = pl.U;
+    // Whole tiles per CTA when that loses at most 15 % to imbalance; otherwise equal slices of
+    // the (tile, k-block) space with partial tiles reduced in the kernel.
+    const int64_t Tt = (int64_t)pl.TM * pl.TN;
+    const int64_t rounds = (Tt + P - 1) / P;
+    const int aligned = (Tt >= P && Tt * 100 >= 85 * P * rounds) ? 1 : 0;
     unsigned int* counters = static_cast<unsigned int*>(workspace);
     float* slots = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
     kern<<<(unsigned)P, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
-                                                               counters, slots, M, N, K, pl.TM, pl.TN, status);
+                                                               counters, slots, M, N, K, pl.TM, pl.TN, aligned, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return launch_status();
 }

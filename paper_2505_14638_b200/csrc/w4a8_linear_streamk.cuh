@@ -21,15 +21,6 @@
 
 namespace w4a8 {
 
-#ifdef W4A8_TIMING
-#define DBG_STAMP(slot) g_dbg[blockIdx.x * 16 + (slot)] = clock64()
-#define DBG_ADD(slot, v) g_dbg[blockIdx.x * 16 + (slot)] += (v)
-#define DBG_SET(slot, v) g_dbg[blockIdx.x * 16 + (slot)] = (v)
-#else
-#define DBG_STAMP(slot)
-#define DBG_ADD(slot, v)
-#define DBG_SET(slot, v)
-#endif
 
 template <int BNX_, int G_, int S1_, int S2_, int FMT_>
 struct SkCfg {
@@ -46,7 +37,7 @@ struct SkCfg {
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + 1024;
     static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;
-    static constexpr int kThreads = 32 * (6 + 4 * G);
+    static constexpr int kThreads = 32 * (10 + 4 * G);
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
@@ -60,7 +51,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                       const uint8_t* __restrict__ wpp,             // tiled weights (panels, k-block major)
                       const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                       void* __restrict__ y, int64_t ldy, int out_dtype, unsigned int* counters,
-                      float* slots, int M, int N, int K, int TM, int TN, unsigned int* status_word) {
+                      float* slots, int M, int N, int K, int TM, int TN, int aligned, unsigned int* status_word) {
     constexpr int BNX = Cfg::BNX, G = Cfg::G, S1 = Cfg::S1, S2 = Cfg::S2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -92,12 +83,14 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     const uint8_t* meta_base = wpp + (int64_t)KB * N * kRowCodeBytes;
     const int64_t U = (int64_t)TM * TN * KB;
     const int64_t P = gridDim.x, p = blockIdx.x;
-    const int64_t u_begin = p * U / P, u_end = (p + 1) * U / P;
+    // Share of this CTA: an equal slice of the unit space, or -- when there are enough tiles
+    // for whole tiles to balance -- a run of whole tiles (then no partial tile is ever produced).
+    const int64_t Tt = (int64_t)TM * TN;
+    const int64_t u_begin = aligned ? (p * Tt / P) * KB : p * U / P;
+    const int64_t u_end = aligned ? ((p + 1) * Tt / P) * KB : (p + 1) * U / P;
     const int n_it = (int)(u_end - u_begin);
 
     if (threadIdx.x == 0) {
-        DBG_STAMP(0);
-        DBG_SET(15, (long long)ptx::globaltimer_ns());
         for (int s = 0; s < S1; ++s) {
             ptx::mbar_init(bar_full(s), 1);
             ptx::mbar_init(bar_free1(s), 1);
@@ -108,7 +101,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar_acc_full(b), 1);
-            ptx::mbar_init(bar_acc_empty(b), 128);
+            ptx::mbar_init(bar_acc_empty(b), 256);
         }
         ptx::mbar_init(bar_drain, 1);
         *abort_flag = 0u;
@@ -123,40 +116,53 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) DBG_STAMP(1);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ producer (whole warp, one lane issues)
+        {
             bool ok = true;
-            int it = 0, issued = 0;
+            int issued = 0;
+            ptx::Ring r1;
             int64_t tile = u_begin / KB;
             int kb = (int)(u_begin - tile * KB);
-            for (; it < n_it; ++it) {
-                const int s = it % S1;
-                if (it >= S1) {
-                    ok = ptx::mbar_wait(bar_free1(s), (uint32_t)((it / S1 - 1) & 1), abort_flag, status_word);
-                    if (!ok) break;
-                }
-                const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
+            int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
+            for (int it = 0; it < n_it; ++it) {
+                ok = ptx::mbar_wait(bar_free1(r1.idx), r1.phase ^ 1u, abort_flag, status_word);
+                if (!ok) break;
                 const int rows = (N - nt * 128) < 128 ? (N - nt * 128) : 128;  // ragged last tile
                 const int64_t row0 = (int64_t)kb * N + (int64_t)nt * 128;
-                ptx::mbar_arrive_expect_tx(bar_full(s),
-                                           (uint32_t)(rows * (kRowCodeBytes + Cfg::kMeta) + Cfg::kXBytes));
-                ptx::bulk_load(stage_w(s), wpp + row0 * kRowCodeBytes, (uint32_t)(rows * kRowCodeBytes), bar_full(s));
-                ptx::bulk_load(stage_w(s) + 8192u, meta_base + row0 * Cfg::kMeta, (uint32_t)(rows * Cfg::kMeta),
-                               bar_full(s));
-                ptx::tma_load_2d(stage_x(s), &tmap_x, kb * 128, mt * BNX, bar_full(s));
-                issued = it + 1;
+                const uint32_t full = bar_full(r1.idx), wdst = stage_w(r1.idx), xdst = stage_x(r1.idx);
+                const uint8_t* csrc = wpp + row0 * kRowCodeBytes;
+                const uint8_t* msrc = meta_base + row0 * Cfg::kMeta;
+                const uint32_t cbytes = (uint32_t)(rows * kRowCodeBytes), mbytes = (uint32_t)(rows * Cfg::kMeta);
+                const int x0 = kb * 128, y0 = mt * BNX;
+                if (ptx::elect_one()) {
+                    ptx::mbar_arrive_expect_tx(full, cbytes + mbytes + (uint32_t)Cfg::kXBytes);
+                    ptx::bulk_load(wdst, csrc, cbytes, full);
+                    ptx::bulk_load(wdst + 8192u, msrc, mbytes, full);
+                    ptx::tma_load_2d(xdst, &tmap_x, x0, y0, full);
+                }
+                r1.advance(S1);
+                ++issued;
                 if (++kb == KB) {
                     kb = 0;
-                    ++tile;
+                    if (++mt == TM) {
+                        mt = 0;
+                        ++nt;
+                    }
                 }
             }
-            if (!ok) {
-                for (int i = (issued > S1 ? issued - S1 : 0); i < issued; ++i) {
+            if (!ok && lane == 0) {
+                // Gave up: let the copies already in flight land before the CTA goes away.
+                ptx::Ring rb = r1;
+                const int n = issued < S1 ? issued : S1;
+                for (int i = 0; i < n; ++i) {
+                    if (--rb.idx < 0) {
+                        rb.idx = S1 - 1;
+                        rb.phase ^= 1u;
+                    }
                     uint64_t t0 = ptx::globaltimer_ns();
-                    while (!ptx::mbar_try_wait(bar_full(i % S1), (uint32_t)((i / S1) & 1)) &&
+                    while (!ptx::mbar_try_wait(bar_full(rb.idx), rb.phase) &&
                            ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
                     }
                 }
@@ -164,11 +170,12 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
+        {
             constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, BNX);
             bool ok = true;
-            int it = 0, j = 0;
+            ptx::Ring r1, r2;
+            int j = 0;
             int64_t u = u_begin;
             while (u < u_end && ok) {
                 const int64_t tile = u / KB;
@@ -180,29 +187,30 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     if (!ok) break;
                 }
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(buf * BNX);
-                for (int i = 0; i < len; ++i, ++it) {
-                    const int s1 = it % S1, s2 = it % S2;
-                    ok = ptx::mbar_wait(bar_full(s1), (uint32_t)((it / S1) & 1), abort_flag, status_word) &&
-                         ptx::mbar_wait(bar_w8_full(s2), (uint32_t)((it / S2) & 1), abort_flag, status_word);
+                uint32_t accumulate = 0;
+                for (int i = 0; i < len; ++i) {
+                    ok = ptx::mbar_wait(bar_full(r1.idx), r1.phase, abort_flag, status_word) &&
+                         ptx::mbar_wait(bar_w8_full(r2.idx), r2.phase, abort_flag, status_word);
                     if (!ok) break;
-                    if (it == 0) DBG_STAMP(2);
                     ptx::tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint64_t adesc = ptx::umma_desc_k_sw128(stage_w8(s2) + 32u * k);
-                        const uint64_t bdesc = ptx::umma_desc_k_sw128(stage_x(s1) + 32u * k);
-                        ptx::umma_f8(tmem_acc, adesc, bdesc, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    const uint32_t a_lo = ptx::umma_desc_lo(stage_w8(r2.idx));
+                    const uint32_t b_lo = ptx::umma_desc_lo(stage_x(r1.idx));
+                    const uint32_t f1 = bar_free1(r1.idx), f2 = bar_free2(r2.idx);
+                    if (ptx::elect_one()) {
+                        ptx::umma_f8_kblock(tmem_acc, a_lo, b_lo, idesc, accumulate);
+                        ptx::umma_commit(f1);
+                        ptx::umma_commit(f2);
                     }
-                    ptx::umma_commit(bar_free1(s1));
-                    ptx::umma_commit(bar_free2(s2));
+                    accumulate = 1u;
+                    r1.advance(S1);
+                    r2.advance(S2);
                 }
                 if (!ok) break;
-                ptx::umma_commit(bar_acc_full(buf));
-                DBG_STAMP(3);
+                if (ptx::elect_one()) ptx::umma_commit(bar_acc_full(buf));
                 u += len;
                 ++j;
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // Gave up: let the MMAs already issued finish before tensor memory is freed.
                 ptx::umma_commit(bar_drain);
                 uint64_t t0 = ptx::globaltimer_ns();
@@ -211,49 +219,60 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             }
         }
         __syncwarp();
-    } else if (warp < 6) {
-        // ------------------------------------------------------------------ epilogue
+    } else if (warp < 10) {
+        // ------------------------------------------------------------------ epilogue (8 warps)
+        // Accumulator: lane = output channel of the tile, column = token.  Two warps share each
+        // lane quarter and split the columns.
         const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int r = q * 32 + lane;
+        const bool leader = (warp == 2 && lane == 0);
+        constexpr int kHalfCols = BNX / 2;
         bool ok = true;
         int j = 0;
         int64_t u = u_begin;
+        // Final value of one output: Eq. 4 / Eq. 11 scales and the cast.
+        auto store_out = [&](int m, int n, float acc, float swn) {
+            const float res = acc * (__ldg(s_x + m) * swn);
+            if (out_dtype == W4A8_OUT_FP32)
+                reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
+            else
+                reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res);
+        };
         while (u < u_end && ok) {
             const int64_t tile = u / KB;
             const int kb0 = (int)(u - tile * KB);
             const int len = (int)((u_end - u) < (int64_t)(KB - kb0) ? (u_end - u) : (int64_t)(KB - kb0));
             const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
-            const int n = nt * 128 + r, m0 = mt * BNX;
+            const int n = nt * 128 + r, m0 = mt * BNX + half * kHalfCols;
             const bool row_ok = n < N;
             const int buf = j & 1;
             const bool whole = (len == KB);
             const float swn = row_ok ? __ldg(s_w + (int64_t)n * sw_stride) : 0.0f;
             ok = ptx::mbar_wait(bar_acc_full(buf), (uint32_t)((j >> 1) & 1), abort_flag, status_word);
             if (!ok) break;
-            if (r == 0) DBG_STAMP(4);
             ptx::tc_fence_after_sync();
-            const uint32_t tmem_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BNX);
+            const uint32_t tmem_acc =
+                tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BNX + half * kHalfCols);
             // The CTA's first segment uses slot 0, a later (necessarily last) one slot 1.
-            float* my_slot = slots + ((int64_t)p * 2 + (j == 0 ? 0 : 1)) * Cfg::kSlotFloats;
+            float* my_slot = slots + ((int64_t)p * 2 + (j == 0 ? 0 : 1)) * Cfg::kSlotFloats +
+                             (int64_t)half * kHalfCols * 128;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BNX; c0 += 16) {
-                uint32_t v[16];
-                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)c0, v);
+            for (int c0 = 0; c0 < kHalfCols; c0 += 32) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)(c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
                 ptx::tmem_ld_wait();
                 if (m0 + c0 >= M) continue;  // warp-uniform
+                if (row_ok) {
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    const int m = m0 + c0 + jj;
-                    if (m < M && row_ok) {
-                        const float acc = __uint_as_float(v[jj]);
-                        if (whole) {
-                            const float res = acc * (__ldg(s_x + m) * swn);  // Eq. 4, Eq. 11
-                            if (out_dtype == W4A8_OUT_FP32)
-                                reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const int m = m0 + c0 + jj;
+                        if (m < M) {
+                            if (whole)
+                                store_out(m, n, __uint_as_float(v[jj]), swn);
                             else
-                                reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res);
-                        } else {
-                            my_slot[(c0 + jj) * 128 + r] = acc;
+                                my_slot[(c0 + jj) * 128 + r] = __uint_as_float(v[jj]);
                         }
                     }
                 }
@@ -264,22 +283,23 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 // Publish the partial tile, then take a ticket; the last of the tile's segments
                 // to arrive reduces all of them in ascending CTA order.
                 __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (r == 0) *ticket_slot = atomicAdd(counters + tile, 1u);
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (leader) *ticket_slot = atomicAdd(counters + tile, 1u);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
                 const uint32_t ticket = *ticket_slot;
                 const int64_t p_lo = ((tile * KB + 1) * P - 1) / U;
                 const int64_t p_hi = (((tile + 1) * KB) * P - 1) / U;
                 if (ticket == (uint32_t)(p_hi - p_lo)) {
                     __threadfence();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < BNX && m0 + c0 < M; c0 += 16) {
+                    for (int c0 = 0; c0 < kHalfCols && m0 + c0 < M; c0 += 16) {
                         float acc[16];
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) acc[jj] = 0.0f;
                         for (int64_t qq = p_lo; qq <= p_hi; ++qq) {
                             const int64_t first_tile = (qq * U / P) / KB;
-                            const float* sl = slots + (qq * 2 + (tile == first_tile ? 0 : 1)) * Cfg::kSlotFloats;
+                            const float* sl = slots + (qq * 2 + (tile == first_tile ? 0 : 1)) * Cfg::kSlotFloats +
+                                              (int64_t)half * kHalfCols * 128;
 #pragma unroll
                             for (int jj = 0; jj < 16; ++jj)
                                 if (m0 + c0 + jj < M && row_ok) acc[jj] += __ldcg(sl + (c0 + jj) * 128 + r);
@@ -287,67 +307,40 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int m = m0 + c0 + jj;
-                            if (m < M && row_ok) {
-                                const float res = acc[jj] * (__ldg(s_x + m) * swn);  // Eq. 4, Eq. 11
-                                if (out_dtype == W4A8_OUT_FP32)
-                                    reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
-                                else
-                                    reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] =
-                                        __float2bfloat16_rn(res);
-                            }
+                            if (m < M && row_ok) store_out(m, n, acc[jj], swn);
                         }
                     }
-                    if (r == 0) counters[tile] = 0u;  // ready for the next launch
+                    if (leader) counters[tile] = 0u;  // ready for the next launch
                 }
             }
             u += len;
             ++j;
-            if (r == 0) DBG_STAMP(5);
         }
     } else {
         // ------------------------------------------------------------------ dequantization groups
-        const int dw = warp - 6;
+        const int dw = warp - 10;
         const int g = dw >> 2;
         const int r = (dw & 3) * 32 + lane;
         for (int it = g; it < n_it; it += G) {
             const int s1 = it % S1, s2 = it % S2;
-#ifdef W4A8_TIMING
-            long long tq0 = clock64();
-#endif
             if (!ptx::mbar_wait(bar_full(s1), (uint32_t)((it / S1) & 1), abort_flag, status_word)) break;
-#ifdef W4A8_TIMING
-            long long tq1 = clock64();
-            if (dw == 0 && lane == 0) DBG_ADD(8, tq1 - tq0);
-#endif
-#ifdef W4A8_TIMING
-            long long tq2 = clock64();
-#endif
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
-#ifdef W4A8_TIMING
-            long long tq3 = clock64();
-            if (dw == 0 && lane == 0) { DBG_ADD(9, tq2 - tq1); DBG_ADD(10, tq3 - tq2); }
-#endif
             dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + (uint32_t)r * 64u,
                                           stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
                                           stage_w8(s2) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
-#ifdef W4A8_TIMING
-            if (dw == 0 && lane == 0) DBG_ADD(11, clock64() - tq3);
-#endif
         }
     }
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0) DBG_STAMP(6);
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
-    if (threadIdx.x == 32) { DBG_STAMP(7); DBG_SET(14, (long long)ptx::globaltimer_ns()); }
 }
 
 }  // namespace w4a8

@@ -21,6 +21,17 @@
 
 namespace w4a8 {
 
+#ifdef W4A8_TIMING
+#define SK_T(var) long long var = clock64()
+#define SK_ADD(i, v) sk_acc[i] += (v)
+#define SK_DECL long long sk_acc[4] = {0, 0, 0, 0}
+#define SK_FLUSH(slot0) for (int i_ = 0; i_ < 4; ++i_) g_dbg[blockIdx.x * 16 + (slot0) + i_] = sk_acc[i_]
+#else
+#define SK_T(var)
+#define SK_ADD(i, v)
+#define SK_DECL
+#define SK_FLUSH(slot0)
+#endif
 
 template <int BNX_, int G_, int S1_, int S2_, int FMT_>
 struct SkCfg {
@@ -174,6 +185,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         {
             constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, BNX);
             bool ok = true;
+            SK_DECL;
+            SK_T(tstart);
             ptx::Ring r1, r2;
             int j = 0;
             int64_t u = u_begin;
@@ -189,8 +202,13 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(buf * BNX);
                 uint32_t accumulate = 0;
                 for (int i = 0; i < len; ++i) {
-                    ok = ptx::mbar_wait(bar_full(r1.idx), r1.phase, abort_flag, status_word) &&
-                         ptx::mbar_wait(bar_w8_full(r2.idx), r2.phase, abort_flag, status_word);
+                    SK_T(t0);
+                    ok = ptx::mbar_wait(bar_full(r1.idx), r1.phase, abort_flag, status_word);
+                    SK_T(t1);
+                    ok = ok && ptx::mbar_wait(bar_w8_full(r2.idx), r2.phase, abort_flag, status_word);
+                    SK_T(t2);
+                    SK_ADD(0, t1 - t0);
+                    SK_ADD(1, t2 - t1);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t a_lo = ptx::umma_desc_lo(stage_w8(r2.idx));
@@ -204,12 +222,17 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     accumulate = 1u;
                     r1.advance(S1);
                     r2.advance(S2);
+                    SK_T(t3);
+                    SK_ADD(2, t3 - t2);
                 }
                 if (!ok) break;
                 if (ptx::elect_one()) ptx::umma_commit(bar_acc_full(buf));
                 u += len;
                 ++j;
             }
+#ifdef W4A8_TIMING
+            if (lane == 0) { sk_acc[3] = clock64() - tstart; SK_FLUSH(0); }
+#endif
             if (!ok && lane == 0) {
                 // Gave up: let the MMAs already issued finish before tensor memory is freed.
                 ptx::umma_commit(bar_drain);
@@ -231,9 +254,11 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         bool ok = true;
         int j = 0;
         int64_t u = u_begin;
+        SK_DECL;
+        SK_T(tstart);
         // Final value of one output: Eq. 4 / Eq. 11 scales and the cast.
-        auto store_out = [&](int m, int n, float acc, float swn) {
-            const float res = acc * (__ldg(s_x + m) * swn);
+        auto store_out = [&](int m, int n, float acc, float scale) {
+            const float res = acc * scale;
             if (out_dtype == W4A8_OUT_FP32)
                 reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
             else
@@ -249,7 +274,17 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             const int buf = j & 1;
             const bool whole = (len == KB);
             const float swn = row_ok ? __ldg(s_w + (int64_t)n * sw_stride) : 0.0f;
+            // Activation scales of this warp's columns, one per lane and 32 columns, fetched before
+            // the accumulator is ready and broadcast by shuffles later: global loads issued inside
+            // the store loop queue behind the operand traffic of the main loop.
+            float sx_pre[kHalfCols / 32];
+#pragma unroll
+            for (int c = 0; c < kHalfCols / 32; ++c)
+                sx_pre[c] = (m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f;
+            SK_T(te0);
             ok = ptx::mbar_wait(bar_acc_full(buf), (uint32_t)((j >> 1) & 1), abort_flag, status_word);
+            SK_T(te1);
+            SK_ADD(0, te1 - te0);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const uint32_t tmem_acc =
@@ -258,23 +293,37 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             float* my_slot = slots + ((int64_t)p * 2 + (j == 0 ? 0 : 1)) * Cfg::kSlotFloats +
                              (int64_t)half * kHalfCols * 128;
 #pragma unroll 1
-            for (int c0 = 0; c0 < kHalfCols; c0 += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)(c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+            for (int c0 = 0; c0 < kHalfCols; c0 += 16) {
+                uint32_t v[16];
+                ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)c0, v);
                 ptx::tmem_ld_wait();
                 if (m0 + c0 >= M) continue;  // warp-uniform
-                if (row_ok) {
+                if (whole) {
+                    // this chunk's activation scales sit in lanes (c0 % 32) .. +15 of one prefetched register
+                    float sx_lane = sx_pre[0];
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const int m = m0 + c0 + jj;
-                        if (m < M) {
-                            if (whole)
-                                store_out(m, n, __uint_as_float(v[jj]), swn);
-                            else
-                                my_slot[(c0 + jj) * 128 + r] = __uint_as_float(v[jj]);
+                    for (int c = 1; c < kHalfCols / 32; ++c) sx_lane = (c0 >= c * 32) ? sx_pre[c] : sx_lane;
+                    float sx[16];
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) sx[jj] = __shfl_sync(0xFFFFFFFFu, sx_lane, (c0 & 16) + jj);
+                    if (row_ok) {
+                        if (out_dtype == W4A8_OUT_FP32) {
+                            float* yp = reinterpret_cast<float*>(y) + (int64_t)(m0 + c0) * ldy + n;
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj)
+                                if (m0 + c0 + jj < M) yp[(int64_t)jj * ldy] = __uint_as_float(v[jj]) * (sx[jj] * swn);
+                        } else {
+                            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(y) + (int64_t)(m0 + c0) * ldy + n;
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj)
+                                if (m0 + c0 + jj < M)
+                                    yp[(int64_t)jj * ldy] = __float2bfloat16_rn(__uint_as_float(v[jj]) * (sx[jj] * swn));
                         }
                     }
+                } else if (row_ok) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        if (m0 + c0 + jj < M) my_slot[(c0 + jj) * 128 + r] = __uint_as_float(v[jj]);
                 }
             }
             ptx::tc_fence_before_sync();
@@ -304,10 +353,12 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                             for (int jj = 0; jj < 16; ++jj)
                                 if (m0 + c0 + jj < M && row_ok) acc[jj] += __ldcg(sl + (c0 + jj) * 128 + r);
                         }
+                        const float sx_lane = (lane < 16 && m0 + c0 + lane < M) ? __ldg(s_x + m0 + c0 + lane) : 0.0f;
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int m = m0 + c0 + jj;
-                            if (m < M && row_ok) store_out(m, n, acc[jj], swn);
+                            const float sxm = __shfl_sync(0xFFFFFFFFu, sx_lane, jj);
+                            if (m < M && row_ok) store_out(m, n, acc[jj], sxm * swn);
                         }
                     }
                     if (leader) counters[tile] = 0u;  // ready for the next launch
@@ -315,24 +366,39 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             }
             u += len;
             ++j;
+            SK_ADD(1, clock64() - te1);
         }
+#ifdef W4A8_TIMING
+        if (leader) { sk_acc[3] = clock64() - tstart; SK_FLUSH(8); }
+#endif
     } else {
         // ------------------------------------------------------------------ dequantization groups
         const int dw = warp - 10;
         const int g = dw >> 2;
         const int r = (dw & 3) * 32 + lane;
+        SK_DECL;
+        SK_T(tstart);
         for (int it = g; it < n_it; it += G) {
             const int s1 = it % S1, s2 = it % S2;
+            SK_T(t0);
             if (!ptx::mbar_wait(bar_full(s1), (uint32_t)((it / S1) & 1), abort_flag, status_word)) break;
+            SK_T(t1);
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
+            SK_T(t2);
+            SK_ADD(0, t1 - t0);
+            SK_ADD(1, t2 - t1);
             dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + (uint32_t)r * 64u,
                                           stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
                                           stage_w8(s2) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
+            SK_ADD(2, clock64() - t2);
         }
+#ifdef W4A8_TIMING
+        if (dw == 0 && lane == 0) { sk_acc[3] = clock64() - tstart; SK_FLUSH(4); }
+#endif
     }
 
     ptx::tc_fence_before_sync();

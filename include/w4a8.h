@@ -142,6 +142,34 @@ int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
 size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k);
 
 /*
+ * Variant of w4a8_linear_ex (canonical weights, W4A8_ALGO_UMMA) for callers that cannot hand the
+ * library a workspace.  (The paper has no counterpart; this is a deployment convenience.)
+ * Typical cases: an inference-engine plugin whose enqueue hook receives only its input and
+ * output tensors and is forbidden to allocate; a latency-critical serving loop in which a
+ * cudaMalloc would stall the whole device; a process whose memory pool has been handed out in
+ * full before the layer is first run.
+ * The split-K partial sums live in an array that is part of the library image itself
+ * (W4A8_STATIC_SCRATCH_BYTES bytes, resident on every GPU that loads the library until the
+ * process exits).  The call allocates and frees nothing, on the host or on the device.
+ *   - split_k <= 0 lets the library choose; the partial sums need split_k * M * N * 4 bytes, and
+ *     a problem that needs more than W4A8_STATIC_SCRATCH_BYTES is rejected with
+ *     W4A8_ERR_WORKSPACE_TOO_SMALL before anything is launched.
+ *   - The first call on each device looks up the device address of the array (a synchronous
+ *     runtime query).  Make that first call outside of any stream capture; later calls only
+ *     enqueue kernels.
+ *   - All calls on a device share the one array.  Each call overwrites every partial sum it
+ *     later reads, so nothing has to be cleared between calls and stale contents are harmless,
+ *     but two calls whose kernels overlap on the GPU (different streams, or graphs replayed
+ *     concurrently) would race on it: serialise them.
+ * Arguments and results are those of w4a8_linear_ex.
+ */
+#define W4A8_STATIC_SCRATCH_BYTES (4u << 20)
+int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
+                               const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
+                               const float* s_w, int sw_stride, int64_t N, int64_t K, int group, void* y,
+                               int64_t ldy, int out_dtype, int split_k, void* stream);
+
+/*
  * Offline round-to-nearest weight quantizer (Eq. 6 -> 7 -> 8 -> 9, no error compensation),
  * so that a caller can produce the stored format on the device.  W is FP32 [N][K].
  *   symmetric != 0: s_g = max|w8| / 7, u = round(w8 / s_g) + 8 (codes 1..15), gzero may be NULL;

@@ -26,7 +26,8 @@ GROUP = 128
 EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
-    "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_quantize_weight_rtn",
+    "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
+    "w4a8_quantize_weight_rtn",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
 )
 
@@ -66,6 +67,8 @@ def lib():
     L.w4a8_linear_ex.restype = i32
     L.w4a8_linear_ex.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz,
                                  i32, i32, p]
+    L.w4a8_linear_static_scratch.restype = i32
+    L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
     L.w4a8_linear_ex_workspace_bytes.restype = sz
     L.w4a8_linear_ex_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
     L.w4a8_quantize_weight_rtn.restype = i32
@@ -205,6 +208,27 @@ def linear(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, wor
                               out.stride(0), int(out_dtype), _ptr(workspace), wbytes, int(algo),
                               int(split_k), _stream())
         _check("w4a8_linear_ex", rc)
+    return out
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def linear_static_scratch(x8, s_x, codes, gscale, gzero, s_w, out_dtype=OUT_BF16, out=None, split_k=0):
+    """w4a8_linear_static_scratch: the canonical-weight linear whose split-K partial sums live in
+    an array built into the library, for callers that may not allocate or pass a workspace.
+    `out` should be supplied by such callers; one is created here only as a convenience."""
+    import torch
+    M, K = x8.shape
+    N = codes.shape[0]
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, N), dtype=dt, device=x8.device)
+    rc = lib().w4a8_linear_static_scratch(
+        _ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(s_w),
+        0 if s_w.numel() == 1 else 1, N, K, GROUP, _ptr(out), out.stride(0), int(out_dtype),
+        int(split_k), _stream())
+    _check("w4a8_linear_static_scratch", rc)
     return out
 
 

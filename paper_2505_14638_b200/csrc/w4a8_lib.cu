@@ -51,6 +51,27 @@ static unsigned int* status_word_ptr() {
     return ptrs[dev];
 }
 
+// Split-K partial sums for callers that cannot provide a workspace (w4a8_linear_static_scratch).
+// Device code could name the array directly; host code must not use the symbol as a pointer (it
+// is only a host-side stand-in) and asks the runtime for the device address instead.
+static __device__ __align__(256) unsigned char g_static_scratch[W4A8_STATIC_SCRATCH_BYTES];
+
+static void* static_scratch_ptr() {
+    // Device address of the built-in scratch array on the current device, looked up once per
+    // device with that device current.
+    static std::mutex mu;
+    static void* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
 static inline int launch_status() {
     return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
@@ -530,6 +551,28 @@ int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
                    size_t workspace_bytes, int algo, int split_k, void* stream) {
     return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
                        ldy, out_dtype, workspace, workspace_bytes, algo, split_k, static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                               const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride,
+                               int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype, int split_k,
+                               void* stream) {
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
+    LinearPlan plan;
+    int rc = make_plan(M, N, K, W4A8_ALGO_UMMA, split_k, &plan);
+    if (rc != W4A8_OK) return rc;
+    if (plan.workspace_bytes > (size_t)W4A8_STATIC_SCRATCH_BYTES) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    if (plan.workspace_bytes > 0) {
+        rc = check_device();
+        if (rc != W4A8_OK) return rc;
+        scratch = static_scratch_ptr();
+        if (!scratch) return W4A8_ERR_CUDA;
+    }
+    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
+                       ldy, out_dtype, scratch, plan.workspace_bytes, W4A8_ALGO_UMMA, plan.split_k,
+                       static_cast<cudaStream_t>(stream));
 }
 
 size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k) {

@@ -210,6 +210,21 @@ def run_reference(args, rank):
 # GPU arm
 # --------------------------------------------------------------------------------------------
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings (the job is as slow as its slowest replica)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def aggregate_rate(world, steps, ms_total):
+    """Whole-job weight stream rate in GB/s: every replica streams the sweep's weights each step."""
+    return world * steps * len(SWEEP_M) * weight_bytes() / (ms_total * 1e-3) / 1e9
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_2505_14638_b200 import binding, inputs
@@ -368,10 +383,7 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     ms_e2e = g0.elapsed_time(g1) * args.steps / n_e2e
 
-    if dist is not None:
-        t = torch.tensor([ms_total, ms_e2e, lin_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e, lin_ms = (float(v) for v in t.cpu())
+    ms_total, ms_e2e, lin_ms = max_over_ranks([ms_total, ms_e2e, lin_ms], dist, dev)
 
     if rank != 0:
         if dist is not None:
@@ -380,9 +392,8 @@ def run_ours(args, rank, world, local_rank):
         return
 
     peaks = load_peaks()
-    step_weight_bytes = len(SWEEP_M) * weight_bytes()
-    value = world * args.steps * step_weight_bytes / (ms_total * 1e-3) / 1e9
-    e2e_value = world * args.steps * step_weight_bytes / (ms_e2e * 1e-3) / 1e9
+    value = aggregate_rate(world, args.steps, ms_total)
+    e2e_value = aggregate_rate(world, args.steps, ms_e2e)
     n_lin = args.steps * len(SWEEP_M)
     alg_bytes = sum(linear_algorithmic_bytes(m) for m in SWEEP_M) / len(SWEEP_M)
     avg_launch_s = lin_ms * 1e-3 / n_lin
@@ -505,12 +516,23 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / per-M detail sections")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--prefill-only", action="store_true",
+                    help="run only the c3 prefill section (small enough for a profiler capture) and print it")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.prefill_only:
+        import torch
+        from paper_2505_14638_b200 import binding, inputs
+        from paper_2505_14638_b200 import build as _build
+        _build.build()
+        torch.cuda.set_device(local_rank)
+        print(json.dumps({"prefill": prefill_extra(torch, binding, inputs, torch.device("cuda", local_rank),
+                                                   load_peaks())}), flush=True)
         return
     if world != args.gpus and world > 1:
         raise SystemExit("--gpus %d does not match WORLD_SIZE %d" % (args.gpus, world))

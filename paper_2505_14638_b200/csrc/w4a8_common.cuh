@@ -9,9 +9,6 @@
 
 namespace w4a8 {
 
-#ifdef W4A8_TIMING
-__device__ long long g_dbg[1024 * 16];
-#endif
 
 constexpr int kGroup = 128;           // group size along K (Sec. 4.1: "group size of 128")
 constexpr float kE4M3Max = 448.0f;    // Z_max of Eq. 3 / Eq. 13

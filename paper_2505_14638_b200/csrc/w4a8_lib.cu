@@ -655,18 +655,6 @@ int w4a8_query_device_status(unsigned int* flags_host) {
     return (v != 0) ? W4A8_ERR_BAD_SHAPE : W4A8_OK;
 }
 
-#ifdef W4A8_TIMING
-int w4a8_debug_read(long long* host, int n, int clear) {
-    cudaDeviceSynchronize();
-    if (cudaMemcpyFromSymbol(host, g_dbg, sizeof(long long) * n) != cudaSuccess) return -1;
-    if (clear) {
-        void* p = nullptr;
-        cudaGetSymbolAddress(&p, g_dbg);
-        cudaMemset(p, 0, sizeof(long long) * 1024 * 16);
-    }
-    return 0;
-}
-#endif
 
 uint64_t w4a8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

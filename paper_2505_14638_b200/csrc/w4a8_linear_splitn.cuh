@@ -33,19 +33,6 @@
 
 namespace w4a8 {
 
-#ifdef W4A8_TIMING
-#define SN_T(var) long long var = clock64()
-#define SN_ADD(slot, v) sn_acc[(slot) & 3] += (v)
-#define SN_FLUSH(slot0) for (int i_ = 0; i_ < 4; ++i_) g_dbg[blockIdx.x * 16 + (slot0) + i_] = sn_acc[i_]
-#define SN_DECL long long sn_acc[4] = {0, 0, 0, 0}
-#define SN_SET(slot, v) g_dbg[blockIdx.x * 16 + (slot)] = (v)
-#else
-#define SN_T(var)
-#define SN_ADD(slot, v)
-#define SN_SET(slot, v)
-#define SN_FLUSH(slot0)
-#define SN_DECL
-#endif
 
 template <int MT_, int G_, int FMT_>
 struct SnCfg {
@@ -112,10 +99,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 32) {
-        SN_SET(1, (long long)ptx::globaltimer_ns());
-        SN_SET(2, clock64());
-    }
     const int KB = K >> 7;
     const int64_t NU = N >> 3;           // the row partition works in units of 8 rows
     const int nst = (KB + KS - 1) / KS;  // stages per tile
@@ -143,7 +126,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 32) SN_SET(0, clock64());
     ptx::griddep_launch_dependents();
 
     if (warp == 0) {
@@ -234,7 +216,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         // ------------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
         {
             bool ok = true;
-            SN_DECL;
             ptx::Ring r1, r2;
             uint32_t acc_phase = 0;
             const uint32_t b_lo0 = ptx::umma_desc_lo(x_ring);
@@ -252,14 +233,8 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 uint32_t accumulate = 0;
                 int kb = 0;
                 for (int st = 0; st < nst; ++st) {
-                    SN_T(tm0);
                     ok = ptx::mbar_wait(bar_xfull0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
-                    SN_T(tm1);
                     ok = ok && ptx::mbar_wait(bar_a_full0 + 8u * (uint32_t)r2.idx, r2.phase, abort_flag, status_word);
-                    SN_T(tm2);
-                    SN_ADD(0, tm1 - tm0);
-                    SN_ADD(1, tm2 - tm1);
-                    if (st == 0 && lane == 0) SN_SET(4, tm2);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     // A stage holds two (k-block, 128-row block) items: either two k-blocks of one
@@ -281,16 +256,10 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     kb += ks;
                     r1.advance(S1);
                     r2.advance(S2);
-                    SN_T(tm3);
-                    SN_ADD(2, tm3 - tm2);
                 }
                 if (!ok) break;
                 if (ptx::elect_one()) ptx::umma_commit(bar_acc_full);
-                if (lane == 0) SN_SET(5, clock64());
             }
-#ifdef W4A8_TIMING
-            if (lane == 0) { SN_FLUSH(8); }
-#endif
             if (!ok && lane == 0) {
                 // Gave up: wait (bounded) for the MMAs already issued before tensor memory is freed.
                 ptx::umma_commit(bar_drain);
@@ -366,18 +335,14 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         int done = g;  // global index of this group's next stage
         int turn = g;  // stages until this group's next turn, counted across tiles
         bool ok = true;
-        SN_DECL;
         for (int t = p; t < T && ok; t += P) {
             const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
             const int R = (u1 - u0) * 8;
             int st = turn;
             for (; st < nst; st += G) {
-                SN_T(td0);
                 ok = ptx::mbar_wait(bar_full0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
-                SN_T(td1);
                 if (ok && done >= S2)
                     ok = ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rl.idx, rl.phase, abort_flag, status_word);
-                SN_T(td2);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const int kb = st * KS;
@@ -396,9 +361,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 ptx::tmem_st_wait();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_a_full0 + 8u * (uint32_t)r2.idx);
-                SN_ADD(0, td1 - td0);
-                SN_ADD(1, td2 - td1);
-                SN_ADD(2, clock64() - td2);
                 for (int i = 0; i < G; ++i) {
                     r1.advance(S1);
                     r2.advance(S2);
@@ -408,21 +370,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             }
             turn = st - nst;
         }
-#ifdef W4A8_TIMING
-        if (dw == 0 && lane == 0) { SN_FLUSH(12); }
-#endif
     }
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 32) SN_SET(6, clock64());
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
-    }
-    if (threadIdx.x == 32) {
-        SN_SET(3, (long long)ptx::globaltimer_ns());
-        SN_SET(7, clock64());
     }
 }
 

@@ -21,17 +21,6 @@
 
 namespace w4a8 {
 
-#ifdef W4A8_TIMING
-#define SK_T(var) long long var = clock64()
-#define SK_ADD(i, v) sk_acc[i] += (v)
-#define SK_DECL long long sk_acc[4] = {0, 0, 0, 0}
-#define SK_FLUSH(slot0) for (int i_ = 0; i_ < 4; ++i_) g_dbg[blockIdx.x * 16 + (slot0) + i_] = sk_acc[i_]
-#else
-#define SK_T(var)
-#define SK_ADD(i, v)
-#define SK_DECL
-#define SK_FLUSH(slot0)
-#endif
 
 template <int BNX_, int G_, int S1_, int S2_, int FMT_>
 struct SkCfg {
@@ -185,8 +174,6 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         {
             constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, BNX);
             bool ok = true;
-            SK_DECL;
-            SK_T(tstart);
             ptx::Ring r1, r2;
             int j = 0;
             int64_t u = u_begin;
@@ -202,13 +189,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(buf * BNX);
                 uint32_t accumulate = 0;
                 for (int i = 0; i < len; ++i) {
-                    SK_T(t0);
                     ok = ptx::mbar_wait(bar_full(r1.idx), r1.phase, abort_flag, status_word);
-                    SK_T(t1);
                     ok = ok && ptx::mbar_wait(bar_w8_full(r2.idx), r2.phase, abort_flag, status_word);
-                    SK_T(t2);
-                    SK_ADD(0, t1 - t0);
-                    SK_ADD(1, t2 - t1);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t a_lo = ptx::umma_desc_lo(stage_w8(r2.idx));
@@ -222,17 +204,12 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     accumulate = 1u;
                     r1.advance(S1);
                     r2.advance(S2);
-                    SK_T(t3);
-                    SK_ADD(2, t3 - t2);
                 }
                 if (!ok) break;
                 if (ptx::elect_one()) ptx::umma_commit(bar_acc_full(buf));
                 u += len;
                 ++j;
             }
-#ifdef W4A8_TIMING
-            if (lane == 0) { sk_acc[3] = clock64() - tstart; SK_FLUSH(0); }
-#endif
             if (!ok && lane == 0) {
                 // Gave up: let the MMAs already issued finish before tensor memory is freed.
                 ptx::umma_commit(bar_drain);
@@ -254,8 +231,6 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         bool ok = true;
         int j = 0;
         int64_t u = u_begin;
-        SK_DECL;
-        SK_T(tstart);
         // Final value of one output: Eq. 4 / Eq. 11 scales and the cast.
         auto store_out = [&](int m, int n, float acc, float scale) {
             const float res = acc * scale;
@@ -281,10 +256,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
 #pragma unroll
             for (int c = 0; c < kHalfCols / 32; ++c)
                 sx_pre[c] = (m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f;
-            SK_T(te0);
             ok = ptx::mbar_wait(bar_acc_full(buf), (uint32_t)((j >> 1) & 1), abort_flag, status_word);
-            SK_T(te1);
-            SK_ADD(0, te1 - te0);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const uint32_t tmem_acc =
@@ -366,39 +338,24 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             }
             u += len;
             ++j;
-            SK_ADD(1, clock64() - te1);
         }
-#ifdef W4A8_TIMING
-        if (leader) { sk_acc[3] = clock64() - tstart; SK_FLUSH(8); }
-#endif
     } else {
         // ------------------------------------------------------------------ dequantization groups
         const int dw = warp - 10;
         const int g = dw >> 2;
         const int r = (dw & 3) * 32 + lane;
-        SK_DECL;
-        SK_T(tstart);
         for (int it = g; it < n_it; it += G) {
             const int s1 = it % S1, s2 = it % S2;
-            SK_T(t0);
             if (!ptx::mbar_wait(bar_full(s1), (uint32_t)((it / S1) & 1), abort_flag, status_word)) break;
-            SK_T(t1);
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
-            SK_T(t2);
-            SK_ADD(0, t1 - t0);
-            SK_ADD(1, t2 - t1);
             dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + (uint32_t)r * 64u,
                                           stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
                                           stage_w8(s2) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
-            SK_ADD(2, clock64() - t2);
         }
-#ifdef W4A8_TIMING
-        if (dw == 0 && lane == 0) { sk_acc[3] = clock64() - tstart; SK_FLUSH(4); }
-#endif
     }
 
     ptx::tc_fence_before_sync();

@@ -2,8 +2,11 @@
 """Benchmark of the W4A8 linear hot path (activation FP8 quantize -> fused INT4->FP8 GEMM ->
 scaled BF16) on the decode sweep: M in {1,4,16}, K=4096, N=14336 (Llama-3-8B MLP up-projection).
 
-One step = one pass of the whole path over the sweep: for each M, w4a8_quantize_act then
-w4a8_linear.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
+One step = one pass of the whole path over the sweep: for each M <= 4 one w4a8_linear_fused
+launch (activation quantization, weight dequantization, FP8 GEMM and scaled BF16 output in one
+kernel), for M = 16 w4a8_quantize_act then w4a8_linear (faster there than the fused launch,
+whose every CTA would have to scan all of X for the token scales); --two-kernel runs the
+two-kernel sequence for every M.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
 method must read per step, divided by the step time.  Weights rotate over several distinct
 copies whose total size exceeds twice the L2, so every pass streams them from HBM.
 
@@ -34,6 +37,7 @@ SWEEP_M = (1, 4, 16)
 K, N = 4096, 14336
 GROUP = 128
 SIGMA, OUTLIER_FRAC, OUTLIER_MULT = 0.02, 0.01, 20.0
+FUSED_UP_TO_M = 4           # the fused launch wins up to here (measured), the two-kernel sequence above
 WEIGHT_COPIES = 10          # 10 x 30.3 MB = 303 MB > 2 x 126 MB L2
 METRIC = "w4a8_decode_weight_stream_rate"
 UNIT = "GB/s"
@@ -51,9 +55,11 @@ def weight_bytes(n=N, k=K):
     return n * k // 2 + n * (k // GROUP) * 2
 
 
-def linear_algorithmic_bytes(m, n=N, k=K):
-    """Everything one w4a8_linear launch must move: weights, FP8 activations, scales, BF16 output."""
-    return weight_bytes(n, k) + m * k + 4 * m + 4 + 2 * m * n
+def linear_algorithmic_bytes(m, n=N, k=K, fused=False):
+    """Everything one linear launch must move: weights, activations (FP8 + scales, or BF16 when the
+    quantization is fused), the weight scale, BF16 output."""
+    act = 2 * m * k if fused else m * k + 4 * m
+    return weight_bytes(n, k) + act + 4 + 2 * m * n
 
 
 def load_peaks():
@@ -271,9 +277,20 @@ def run_ours(args, rank, world, local_rank):
     def lin(m, c):
         binding.linear_tiled(x8s[m], sxs[m], weights[c % WEIGHT_COPIES], out=ys[m], workspace=workspace)
 
+    fused_m = () if args.two_kernel else tuple(m for m in SWEEP_M if m <= FUSED_UP_TO_M)
+    fused = bool(fused_m)
+    lin_unfused = lin
+
+    def lin(m, c):  # noqa: F811
+        if m in fused_m:
+            binding.linear_fused(xs[m], weights[c % WEIGHT_COPIES], out=ys[m])
+        else:
+            lin_unfused(m, c)
+
     def eager_step(phase):
         for i, m in enumerate(SWEEP_M):
-            quant(m)
+            if m not in fused_m:
+                quant(m)
             lin(m, phase * len(SWEEP_M) + i)
 
     def barrier():
@@ -284,6 +301,8 @@ def run_ours(args, rank, world, local_rank):
     for ph in range(3):
         eager_step(ph)
     barrier()
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set by the first steps (a bounded wait gave up)")
 
     # ---- CUDA graphs: one per phase of the weight rotation (the step is launch-bound) ----
     use_graph = not args.no_graph
@@ -303,14 +322,16 @@ def run_ours(args, rank, world, local_rank):
                     for i, m in enumerate(SWEEP_M):
                         lin(m, ph * len(SWEEP_M) + i)
                 g_lin.append(g)
-            g_quant = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_quant, stream=side):
-                for m in SWEEP_M:
-                    quant(m)
+            if len(fused_m) < len(SWEEP_M):
+                g_quant = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_quant, stream=side):
+                    for m in SWEEP_M:
+                        if m not in fused_m:
+                            quant(m)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
 
-    kernels_per_step = 2 * len(SWEEP_M)
+    kernels_per_step = 2 * len(SWEEP_M) - len(fused_m)
 
     def step(s):
         if use_graph:
@@ -340,10 +361,12 @@ def run_ours(args, rank, world, local_rank):
     pairs = []
     for s in range(args.steps):
         if use_graph:
-            g_quant.replay()
+            if g_quant is not None:
+                g_quant.replay()
         else:
             for m in SWEEP_M:
-                quant(m)
+                if m not in fused_m:
+                    quant(m)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         if use_graph:
@@ -395,7 +418,7 @@ def run_ours(args, rank, world, local_rank):
     value = aggregate_rate(world, args.steps, ms_total)
     e2e_value = aggregate_rate(world, args.steps, ms_e2e)
     n_lin = args.steps * len(SWEEP_M)
-    alg_bytes = sum(linear_algorithmic_bytes(m) for m in SWEEP_M) / len(SWEEP_M)
+    alg_bytes = sum(linear_algorithmic_bytes(m, fused=m in fused_m) for m in SWEEP_M) / len(SWEEP_M)
     avg_launch_s = lin_ms * 1e-3 / n_lin
     achieved = alg_bytes / avg_launch_s / 1e9
     line = {
@@ -405,7 +428,9 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD, "parallelism": "replicas x%d (no collective)" % world,
                    "l2": "weights rotate over %d distinct copies (%.0f MB > 2 x 126 MB L2)"
                          % (WEIGHT_COPIES, WEIGHT_COPIES * weight_bytes() / 1e6),
-                   "step": "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
+                   "step": ("M in (1,4): w4a8_linear_fused (activation quantization inside the kernel); M=16: "
+                            "w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)") if fused else
+                           "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
                    "launch": "CUDA graph replay, one graph per step" if use_graph else "eager launches"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
@@ -413,14 +438,15 @@ def run_ours(args, rank, world, local_rank):
                 "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "linear_splitn_kernel<MT=16> (w4a8_linear), mean over M in {1,4,16}",
+        "roofline": {"bound": "hbm", "kernel": "linear_splitn_kernel<MT=16> (%s), mean over M in {1,4,16}"
+                               % ("FUSE variant for M<=4" if fused else "w4a8_linear"),
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
     }
     if not args.no_extras:
-        line["decode_detail"] = decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks)
+        line["decode_detail"] = decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks)
         line["prefill"] = prefill_extra(torch, binding, inputs, dev, peaks)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline()
@@ -443,8 +469,9 @@ def _time_loop(torch, fn, iters, warm=3):
     return a.elapsed_time(b) * 1e-3 / iters
 
 
-def decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks):
-    """Per-M linear time (graph of back-to-back launches, weights from HBM) next to cuBLAS BF16."""
+def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
+    """Per-M time of the fused launch and of the linear alone (graphs of back-to-back launches,
+    weights from HBM) next to cuBLAS BF16."""
     out = {}
     dev = x8s[1].device
     wb = [torch.randn((N, K), dtype=torch.bfloat16, device=dev) for _ in range(4)]
@@ -458,6 +485,14 @@ def decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks):
                     binding.linear_tiled(x8s[m], sxs[m], weights[c], out=ys[m], workspace=workspace)
         torch.cuda.current_stream().wait_stream(side)
         t = _time_loop(torch, g.replay, 20) / WEIGHT_COPIES
+        side.wait_stream(torch.cuda.current_stream())
+        g2 = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g2, stream=side):
+                for c in range(WEIGHT_COPIES):
+                    binding.linear_fused(xs[m], weights[c], out=ys[m])
+        torch.cuda.current_stream().wait_stream(side)
+        tf = _time_loop(torch, g2.replay, 20) / WEIGHT_COPIES
         xb = torch.randn((m, K), dtype=torch.bfloat16, device=dev)
         j = [0]
 
@@ -465,8 +500,12 @@ def decode_detail(torch, binding, weights, x8s, sxs, ys, workspace, peaks):
             j[0] += 1
             torch.matmul(xb, wb[j[0] % 4].t())
         tb = _time_loop(torch, f, 40)
-        out["M=%d" % m] = {"us": t * 1e6, "weight_GBps": weight_bytes() / t / 1e9,
-                           "frac_hbm_measured": linear_algorithmic_bytes(m) / t / 1e9 / peaks["hbm_gbs"],
+        out["M=%d" % m] = {"fused_us": tf * 1e6,
+                           "fused_frac_hbm_measured":
+                               linear_algorithmic_bytes(m, fused=True) / tf / 1e9 / peaks["hbm_gbs"],
+                           "linear_only_us": t * 1e6, "linear_only_weight_GBps": weight_bytes() / t / 1e9,
+                           "linear_only_frac_hbm_measured":
+                               linear_algorithmic_bytes(m) / t / 1e9 / peaks["hbm_gbs"],
                            "cublas_bf16_us": tb * 1e6}
     return out
 
@@ -487,11 +526,18 @@ def prefill_extra(torch, binding, inputs, dev, peaks):
     ws = binding.new_workspace(M3, N3, K3, sets[0][0].fmt, dev)
     i = [0]
 
-    def f():
-        tw, x8, s_x, _ = sets[i[0] % copies]
-        i[0] += 1
+    # a graph of back-to-back launches over the distinct copies: the kernel, not the launch path
+    side = torch.cuda.Stream()
+    for tw, x8, s_x, _ in sets[:2]:
         binding.linear_tiled(x8, s_x, tw, out=y, workspace=ws)
-    t = _time_loop(torch, f, 40, warm=5)
+    side.wait_stream(torch.cuda.current_stream())
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(gr, stream=side):
+            for tw, x8, s_x, _ in sets:
+                binding.linear_tiled(x8, s_x, tw, out=y, workspace=ws)
+    torch.cuda.current_stream().wait_stream(side)
+    t = _time_loop(torch, gr.replay, 10, warm=3) / copies
     wb = torch.randn((N3, K3), dtype=torch.bfloat16, device=dev)
 
     def g():
@@ -515,6 +561,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / per-M detail sections")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--two-kernel", action="store_true",
+                    help="step = w4a8_quantize_act + w4a8_linear per M instead of the fused launch")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")

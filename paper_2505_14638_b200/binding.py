@@ -27,6 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
+    "w4a8_linear_fused",
     "w4a8_quantize_weight_rtn",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
 )
@@ -69,6 +70,8 @@ def lib():
                                  i32, i32, p]
     L.w4a8_linear_static_scratch.restype = i32
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
+    L.w4a8_linear_fused.restype = i32
+    L.w4a8_linear_fused.argtypes = [p, i64, i64, i32, p, p, i32, p, i32, i64, i64, p, i64, i32, p, i64, p, p]
     L.w4a8_linear_ex_workspace_bytes.restype = sz
     L.w4a8_linear_ex_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
     L.w4a8_quantize_weight_rtn.restype = i32
@@ -248,6 +251,27 @@ def linear_tiled(x8, s_x, tw, out_dtype=OUT_BF16, out=None, workspace=None):
                            out.stride(0), int(out_dtype), _ptr(workspace),
                            workspace.numel() * workspace.element_size(), _stream())
     _check("w4a8_linear", rc)
+    return out
+
+
+FUSED_MAX_M = 16
+
+
+def linear_fused(x, tw, out_dtype=OUT_BF16, out=None, scale_mode=SCALE_EXACT, static_scale=None,
+                 x8_out=None, s_x_out=None):
+    """w4a8_linear_fused: BF16 activations [M <= 16, K] and a TiledWeight -> Y, one kernel.
+    x8_out (uint8 [M, K]) / s_x_out (float32 [M]) optionally receive the quantized activations."""
+    import torch
+    M, K = x.shape
+    assert K == tw.K and x.dtype == torch.bfloat16
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, tw.N), dtype=dt, device=x.device)
+    rc = lib().w4a8_linear_fused(_ptr(x), x.stride(0), M, int(scale_mode), _ptr(static_scale), _ptr(tw.buf),
+                                 tw.fmt, _ptr(tw.s_w), 0 if tw.s_w.numel() == 1 else 1, tw.N, K, _ptr(out),
+                                 out.stride(0), int(out_dtype), _ptr(x8_out),
+                                 0 if x8_out is None else x8_out.stride(0), _ptr(s_x_out), _stream())
+    _check("w4a8_linear_fused", rc)
     return out
 
 

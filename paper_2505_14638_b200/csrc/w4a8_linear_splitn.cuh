@@ -29,13 +29,19 @@
 #include <cuda_bf16.h>
 
 #include "w4a8_ptx.cuh"
+#include "w4a8_simple_kernels.cuh"
 #include "w4a8_tiled_format.cuh"
 
 namespace w4a8 {
 
 
-template <int MT_, int G_, int FMT_>
+template <int MT_, int G_, int FMT_, bool FUSE_ = false>
 struct SnCfg {
+    // FUSE: the kernel takes BF16 activations and does the per-token FP8 quantization (Eq. 13)
+    // itself: an absmax pass over X before the main loop (overlapped with the first weight copies)
+    // and a convert step that writes each stage's FP8 activation tile into shared memory, in the
+    // layout a 128-byte-swizzled TMA tile would have had.
+    static constexpr bool FUSE = FUSE_;
     static constexpr int MT = MT_;      // tokens per tile = MMA N (16 or 64)
     static constexpr int G = G_;        // dequantization groups of 4 warps
     static constexpr int FMT = FMT_;
@@ -47,14 +53,45 @@ struct SnCfg {
     static constexpr int kAStageCols = kItems * 32;        // 128 bytes per row and item
     static constexpr int kDCol = kS2 * kAStageCols;        // accumulators start after the A ring
     static constexpr int kThreads = 32 * (6 + 4 * G);
-    static constexpr int kBarBytes = 512;
+    static constexpr int kBarBytes = 768;
     // Decode-sized launches (<= 16 tokens) take half an SM each, so that the CTAs of the next
     // kernel in the stream can start -- and prefetch their weights -- while this one finishes.
     static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : 200 * 1024;
     static_assert(MT == 16 || MT == 64, "token tile");
     static_assert(kDCol + 2 * MT <= kTmemCols, "tensor memory columns");
-    static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 <= kBarBytes, "barrier area");
+    static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 + 3 * 64 <= kBarBytes, "barrier area");
+    static_assert(!FUSE_ || MT_ == 16, "the fused activation quantization is built for <= 16 tokens");
 };
+
+constexpr int kFuseFewTokens = 4;
+
+// Fused activation quantization: which part of which stage's activation tile one of the 128
+// converting threads produces.  A stage's tile (2 k-blocks x Mp tokens, Mp = the token count
+// rounded up to a power of two) takes 8*Mp threads, 32 elements each; the 128 threads therefore
+// can work on up to 16/Mp consecutive stages at once, which keeps that many stages' loads in
+// flight.  No more than S1 (the ring depth) at once, though: a thread that waited for a slot two
+// ring rounds ahead could not tell the rounds apart by the barrier's parity.
+struct XMap {
+    int tps;   // threads per stage (those beyond 8*Mp only arrive on the barrier)
+    int span;  // stages worked on at once = 128 / tps
+    int sub;   // this thread's stage within a group of `span`
+    int xj;    // k-block within the stage (0 or 1)
+    int xrow;  // token
+    int xq;    // 32-element quarter of the k-block
+};
+__device__ __forceinline__ XMap x_map(int r, int M, int S1) {
+    const int lg = M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : 4;
+    XMap m;
+    m.span = 16 >> lg;
+    while (m.span > S1) m.span >>= 1;
+    m.tps = 128 / m.span;
+    m.sub = r / m.tps;
+    const int within = r & (m.tps - 1);
+    m.xq = within & 3;
+    m.xrow = (within >> 2) & ((1 << lg) - 1);
+    m.xj = within >> (2 + lg);  // >= 2 for the threads with nothing to convert
+    return m;
+}
 
 // Launch-time plan shared by host and device.
 struct SnPlan {
@@ -68,12 +105,24 @@ struct SnPlan {
     int smem;      // dynamic shared memory to request
 };
 
+// Arguments of the fused activation quantization (unused otherwise).
+struct SnFuse {
+    const uint16_t* x;          // BF16 activations [M][ldx]
+    int64_t ldx;
+    int scale_mode;
+    const float* static_scale;  // nullptr = dynamic per-token scale
+    uint8_t* x8_out;            // optional copies of the FP8 activations and their scales,
+    int64_t ldx8_out;           // written by CTA 0 only (nullptr = not wanted)
+    float* s_x_out;
+};
+
 template <class Cfg>
-__global__ void __launch_bounds__(Cfg::kThreads)
+__global__ void __launch_bounds__(Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
 linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x MT, 128B swizzle
                      const uint8_t* __restrict__ wpp, const float* __restrict__ s_x,
                      const float* __restrict__ s_w, int sw_stride, void* __restrict__ y, int64_t ldy,
-                     int out_dtype, int M, int N, int K, const SnPlan plan, unsigned int* status_word) {
+                     int out_dtype, int M, int N, int K, const SnPlan plan, const SnFuse fuse,
+                     unsigned int* status_word) {
     constexpr int MT = Cfg::MT, G = Cfg::G, S2 = Cfg::kS2, MB = Cfg::kMeta;
     constexpr int S1M = Cfg::kS1Max;
     extern __shared__ uint8_t smem_raw[];
@@ -97,6 +146,9 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     constexpr int kNumBars = 3 * S1M + S2 + 3;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    unsigned int* amax_s = const_cast<unsigned int*>(tmem_slot) + 4;  // [16] row absmax bit patterns
+    float* sx_s = reinterpret_cast<float*>(amax_s + 16);              // [16] activation scales s_x
+    float* inv_s = sx_s + 16;                                         // [16] multipliers 1/s_x
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = K >> 7;
@@ -107,7 +159,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     if (threadIdx.x == 0) {
         for (int s = 0; s < S1; ++s) {
             ptx::mbar_init(bar_full0 + 8u * s, 1);
-            ptx::mbar_init(bar_xfull0 + 8u * s, 1);
+            ptx::mbar_init(bar_xfull0 + 8u * s, Cfg::FUSE ? (uint32_t)x_map(0, M, S1).tps : 1u);
             ptx::mbar_init(bar_free10 + 8u * s, 1);
         }
         for (int s = 0; s < S2; ++s) ptx::mbar_init(bar_a_full0 + 8u * s, 128);
@@ -116,8 +168,9 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         ptx::mbar_init(bar_drain, 1);
         *abort_flag = 0u;
         ptx::fence_mbar_init();
-        ptx::prefetch_tensormap(&tmap_x);
+        if (!Cfg::FUSE) ptx::prefetch_tensormap(&tmap_x);
     }
+    if (Cfg::FUSE && threadIdx.x >= 64 && threadIdx.x < 80) amax_s[threadIdx.x - 64] = 0u;
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
         ptx::tmem_relinquish();
@@ -127,6 +180,92 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     ptx::griddep_launch_dependents();
+
+    // FUSE: first activation chunks of the converting threads (warps 2..5), fetched before the absmax
+    // pass so that they are in flight during it.
+    uint4 xv[4];
+    bool xv_loaded = false;
+    // Few tokens: only the four epilogue warps (idle until the end) do the absmax pass and the
+    // dequantizers start at once.  More tokens: every warp but the two issuers takes part.
+    const bool fuse_all = M > kFuseFewTokens;
+    if (Cfg::FUSE && warp >= 2 && (fuse_all || warp < 6)) {
+        // Eq. 13, first half: per-token absmax and scale while the first weight stages are in flight.
+        const int NF = fuse_all ? Cfg::kThreads - 64 : 128;
+        const int ft = (int)threadIdx.x - 64;
+        ptx::griddep_wait();  // X comes from the previous kernel in the stream
+        if (warp < 6) {
+            const XMap xm = x_map((warp & 3) * 32 + lane, M, S1);  // as in the epilogue branch below
+            const int kbk = xm.sub * KS + xm.xj;
+            if (xm.xrow < M && xm.xj < KS && kbk < KB) {
+                const uint4* xp = reinterpret_cast<const uint4*>(fuse.x + (int64_t)xm.xrow * fuse.ldx +
+                                                                 (int64_t)kbk * 128 + xm.xq * 32);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) xv[j] = __ldg(xp + j);
+            }
+            xv_loaded = true;
+        }
+        if (fuse.static_scale == nullptr) {
+            const int nch = K >> 3;  // 16-byte chunks per row
+#pragma unroll 1
+            for (int m0 = 0; m0 < M; m0 += 4) {
+                float rm[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                for (int c = ft; c < nch; c += 2 * NF) {
+                    // eight 16-byte loads in flight per thread: four tokens x two chunks
+                    const bool two = c + NF < nch;
+                    uint4 v[4], w[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (m0 + j < M) {
+                            const uint4* row = reinterpret_cast<const uint4*>(fuse.x + (int64_t)(m0 + j) * fuse.ldx);
+                            v[j] = __ldg(row + c);
+                            if (two) w[j] = __ldg(row + c + NF);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (m0 + j < M) {
+                            rm[j] = absmax_bf16x8(v[j], rm[j]);
+                            if (two) rm[j] = absmax_bf16x8(w[j], rm[j]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (m0 + j < M) {  // uniform
+                        float a = rm[j];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+                        // non-negative floats order like their bit patterns
+                        if (lane == 0) atomicMax(amax_s + m0 + j, __float_as_uint(a));
+                    }
+                }
+            }
+        }
+        asm volatile("bar.sync 2, %0;" ::"r"(NF) : "memory");
+        if (ft < 16) {
+            float s = 1.0f, inv = 1.0f;
+            if (ft < M) {
+                if (fuse.static_scale != nullptr) {
+                    s = __ldg(fuse.static_scale);
+                    inv = __fdiv_rn(1.0f, s);
+                } else {
+                    const float amax = __uint_as_float(amax_s[ft]);
+                    if (amax == 0.0f) {
+                    } else if (fuse.scale_mode == W4A8_SCALE_POW2) {
+                        s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
+                        inv = __fdiv_rn(1.0f, s);
+                    } else {
+                        s = __fdiv_rn(amax, kE4M3Max);
+                        inv = __fdiv_rn(kE4M3Max, amax);
+                    }
+                }
+                if (blockIdx.x == 0 && fuse.s_x_out != nullptr) fuse.s_x_out[ft] = s;
+            }
+            sx_s[ft] = s;
+            inv_s[ft] = inv;
+        }
+        asm volatile("bar.sync 2, %0;" ::"r"(NF) : "memory");
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp, one lane issues)
@@ -174,6 +313,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     kb += ks;
                     r1.advance(S1);
                     ++issued;
+                    if (Cfg::FUSE) continue;       // the dequantization groups make the activation tiles
                     if (st + 1 < ahead) continue;  // still inside the weight-only prologue
                     if (!waited) {
                         ptx::griddep_wait();
@@ -277,16 +417,83 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         bool ok = true;
         uint32_t acc_phase = 0;
         bool first_tile = true;
+        ptx::Ring rx;  // ring position of the next activation tile (FUSE)
         for (int t = p; t < T && ok; t += P) {
             const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
             const int R = (u1 - u0) * 8;
             const int n0 = u0 * 8;
+            if (Cfg::FUSE) {
+                // Eq. 13, second half: these four warps, idle until the accumulator is complete,
+                // convert the activations ahead of the MMAs (thread mapping: XMap).  Each thread
+                // keeps the loads of its next two stages in flight.
+                const XMap xm = x_map(r, M, S1);
+                const bool xrow_ok = xm.xrow < M;
+                const uint4* xbase = reinterpret_cast<const uint4*>(fuse.x + (int64_t)xm.xrow * fuse.ldx + xm.xq * 32);
+                const float inv = inv_s[xm.xrow];
+                const uint32_t xoff = (uint32_t)(xm.xj * (MT * 128) + xm.xrow * 128);
+                const uint32_t sw0 = (uint32_t)(((2 * xm.xq) ^ (xm.xrow & 7)) << 4);
+                const uint32_t sw1 = (uint32_t)(((2 * xm.xq + 1) ^ (xm.xrow & 7)) << 4);
+                auto xload = [&](uint4(&v)[4], int st) {
+                    const int kbk = st * KS + xm.xj;  // 128 BF16 = 16 chunks per k-block
+                    if (xrow_ok && xm.xj < KS && st < nst && kbk < KB) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) v[j] = __ldg(xbase + (int64_t)kbk * 16 + j);
+                    }
+                };
+                // convert stage st from v, refill v with stage st_next, publish the tile part
+                auto xstage = [&](uint4(&v)[4], int st, int st_next, const ptx::Ring& rg) -> bool {
+                    const int kbk = st * KS + xm.xj;
+                    const bool xact = xm.xj < KS && kbk < KB;
+                    uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+                    if (xact && xrow_ok) {
+                        const uint2 a = quant_bf16x8(v[0], inv), b = quant_bf16x8(v[1], inv);
+                        const uint2 c = quant_bf16x8(v[2], inv), d = quant_bf16x8(v[3], inv);
+                        lo = make_uint4(a.x, a.y, b.x, b.y);
+                        hi = make_uint4(c.x, c.y, d.x, d.y);
+                    }
+                    xload(v, st_next);
+                    if (!ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rg.idx, rg.phase ^ 1u, abort_flag, status_word))
+                        return false;
+                    if (xact) {
+                        if (xrow_ok && blockIdx.x == 0 && fuse.x8_out != nullptr) {
+                            uint4* o = reinterpret_cast<uint4*>(fuse.x8_out + (int64_t)xm.xrow * fuse.ldx8_out +
+                                                                (int64_t)kbk * 128 + xm.xq * 32);
+                            o[0] = lo;
+                            o[1] = hi;
+                        }
+                        // 128-byte swizzle: the 16-byte chunk index is XORed with the row modulo 8
+                        const uint32_t xt = x_ring + (uint32_t)(rg.idx * plan.xstage) + xoff;
+                        ptx::st_shared_v4(xt + sw0, lo);
+                        ptx::st_shared_v4(xt + sw1, hi);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(bar_xfull0 + 8u * (uint32_t)rg.idx);
+                    return true;
+                };
+                const int span = xm.span;
+                uint4 xw[4];
+                if (!xv_loaded) xload(xv, xm.sub);
+                xv_loaded = false;
+                xload(xw, xm.sub + span);
+                ptx::Ring rg = rx;  // ring position of this thread's next stage
+                for (int i = 0; i < xm.sub; ++i) rg.advance(S1);
+                for (int st = xm.sub; st < nst && ok; st += 2 * span) {
+                    ok = xstage(xv, st, st + 2 * span, rg);
+                    for (int i = 0; i < span; ++i) rg.advance(S1);
+                    if (ok && st + span < nst) {
+                        ok = xstage(xw, st + span, st + 3 * span, rg);
+                        for (int i = 0; i < span; ++i) rg.advance(S1);
+                    }
+                }
+                if (!ok) break;
+                for (int i = 0; i < nst; ++i) rx.advance(S1);
+            }
             ok = ptx::mbar_wait(bar_acc_full, acc_phase, abort_flag, status_word);
             acc_phase ^= 1u;
             if (!ok) break;
             ptx::tc_fence_after_sync();
             if (first_tile) {
-                ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
+                if (!Cfg::FUSE) ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
                 first_tile = false;
             }
             for (int b = 0; b < MBLK; ++b) {
@@ -305,7 +512,8 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     for (int j = 0; j < 16; ++j) {
                         const int m = c0 + j;
                         if (m < M && row_ok) {
-                            const float res = __uint_as_float(v[j]) * (__ldg(s_x + m) * swn);  // Eq. 4, Eq. 11
+                            const float sxm = Cfg::FUSE ? sx_s[m] : __ldg(s_x + m);
+                            const float res = __uint_as_float(v[j]) * (sxm * swn);  // Eq. 4, Eq. 11
                             if (out_dtype == W4A8_OUT_FP32)
                                 reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
                             else
@@ -340,13 +548,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             const int R = (u1 - u0) * 8;
             int st = turn;
             for (; st < nst; st += G) {
+                const int kb = st * KS;
+                const int ks = (KB - kb) < KS ? (KB - kb) : KS;
                 ok = ptx::mbar_wait(bar_full0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
                 if (ok && done >= S2)
                     ok = ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rl.idx, rl.phase, abort_flag, status_word);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const int kb = st * KS;
-                const int ks = (KB - kb) < KS ? (KB - kb) : KS;
                 const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * plan.wstage);
                 uint32_t a_col = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(r2.idx * Cfg::kAStageCols);
                 for (int kbl = 0; kbl < ks; ++kbl) {

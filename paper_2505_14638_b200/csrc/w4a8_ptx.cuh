@@ -99,6 +99,11 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
 // ---- programmatic dependent launch ----------------------------------------------------------
 // Both are no-ops unless the kernel was launched with programmatic stream serialization.
 // wait: blocks until the kernels this one depends on have completed and their writes are visible.

@@ -553,6 +553,77 @@ def prefill_extra(torch, binding, inputs, dev, peaks):
             "cublas_bf16_us": tb * 1e6, "cublas_bf16_tflops": flops / tb / 1e12}
 
 
+C5_LAYERS = (("qkv", 4096, 6144), ("o", 4096, 4096), ("gate_up", 4096, 28672), ("down", 14336, 4096))
+C5_M = (1, 8, 32, 128, 512, 4096)
+
+
+def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, with_cublas=True):
+    """Config c5: the four Llama-3-8B linears x M.  Per case: time of quantize_act + linear (the
+    fused launch where it is the faster one) and of the linear alone, from CUDA graphs of
+    back-to-back launches that rotate over enough weight copies to exceed twice the L2; the
+    roofline time is the larger of bytes / HBM peak and flops / (2 x BF16 burst peak)."""
+    out = []
+    fp8_peak = 2.0 * peaks["bf16_tflops"] * 1e12
+    hbm = peaks["hbm_gbs"] * 1e9
+    side = torch.cuda.Stream()
+
+    def graph_time(fn, reps):
+        fn(0)
+        torch.cuda.synchronize()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for c in range(reps):
+                    fn(c)
+        torch.cuda.current_stream().wait_stream(side)
+        return _time_loop(torch, g.replay, 5, warm=2) / reps
+
+    for name, k, n in layers:
+        wbytes = weight_bytes(n, k)
+        copies = max(2, min(32, int(2.2 * 126e6 / wbytes) + 1))
+        tws = []
+        for c in range(copies):
+            W = torch.from_numpy(inputs.make_weight(n, k, SIGMA, seed=7000 + c)).to(dev)
+            tws.append(binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True)))
+            del W
+        wb = torch.randn((n, k), dtype=torch.bfloat16, device=dev) if with_cublas else None
+        for m in ms:
+            xb = inputs.make_activation(m, k, 7000 + m, OUTLIER_FRAC, OUTLIER_MULT)
+            x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
+            x8, s_x = binding.quantize_act(x)
+            y = torch.empty((m, n), dtype=torch.bfloat16, device=dev)
+            ws = binding.new_workspace(m, n, k, tws[0].fmt, dev)
+            reps = copies if m <= 512 else max(2, copies // 4)
+
+            def lin(c):
+                binding.linear_tiled(x8, s_x, tws[c % copies], out=y, workspace=ws)
+
+            def whole(c):
+                if m <= FUSED_UP_TO_M:
+                    binding.linear_fused(x, tws[c % copies], out=y)
+                else:
+                    binding.quantize_act(x, out=(x8, s_x))
+                    lin(c)
+            t_lin = graph_time(lin, reps)
+            t_all = graph_time(whole, reps)
+            flops = 2.0 * m * n * k
+            t_roof = max(linear_algorithmic_bytes(m, n, k) / hbm, flops / fp8_peak)
+            row = {"layer": name, "K": k, "N": n, "M": m, "linear_us": t_lin * 1e6, "quant_plus_linear_us": t_all * 1e6,
+                   "tflops": flops / t_lin / 1e12, "weight_GBps": wbytes / t_lin / 1e9,
+                   "roofline_us": t_roof * 1e6, "frac_of_roofline": t_roof / t_lin,
+                   "bound": "hbm" if linear_algorithmic_bytes(m, n, k) / hbm > flops / fp8_peak else "tensor"}
+            if with_cublas:
+                row["cublas_bf16_us"] = graph_time(lambda c: torch.matmul(x, wb.t()), 4) * 1e6
+            out.append(row)
+            del x, x8, s_x, y, ws
+        del tws, wb
+        torch.cuda.empty_cache()
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set during the sweep")
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -566,12 +637,28 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
+    ap.add_argument("--sweep", default=None, choices=["c5", "c4"],
+                    help="instead of the bench line, print the per-layer table of config c5 (four Llama-3-8B "
+                         "linears x M) or the single c4 case (M=8192, K=8192, N=28672)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.sweep:
+        import torch
+        from paper_2505_14638_b200 import binding, inputs
+        from paper_2505_14638_b200 import build as _build
+        _build.build()
+        torch.cuda.set_device(local_rank)
+        dev = torch.device("cuda", local_rank)
+        if args.sweep == "c5":
+            rows = layer_sweep(torch, binding, inputs, dev, load_peaks())
+        else:
+            rows = layer_sweep(torch, binding, inputs, dev, load_peaks(), layers=(("c4", 8192, 28672),), ms=(8192,))
+        print(json.dumps({"sweep": args.sweep, "rows": rows}), flush=True)
         return
     if args.prefill_only:
         import torch

@@ -101,7 +101,8 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * weight_format selects how `weights` is read: W4A8_FMT_CANONICAL (weights = codes, with
  * gscale_bf16 / gzero) or a tiled format (weights = buffer written by w4a8_prepack_weight;
  * gscale_bf16 and gzero are ignored and may be NULL).
- * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs; it
+ * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs (they are
+ * added in a fixed order: results repeat bit for bit); it
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
  * its first use; every call leaves it ready for the next one.  Calls that share a workspace

@@ -196,25 +196,54 @@ static int sm_count() {
     return cached;
 }
 
+constexpr int kNominalSMs = 148;  // for size queries made without a device
+
 struct SkPlan {
-    int bnx, ctas_per_sm, TM, TN;
+    int bnx, TM, TN;
+    int aligned;   // 1: whole tiles per CTA, nothing shared; 0: equal slices of the (tile, k-block) space
+    int64_t P;     // CTAs
     int64_t U;
     size_t counter_bytes, workspace_bytes;
 };
 
 constexpr int kSplitNMaxM = 64;  // token counts served by the split-N (decode) kernel
 
-static void make_sk_plan(int64_t M, int64_t N, int64_t K, SkPlan* pl) {
-    pl->bnx = pick_bnx(M);
-    pl->ctas_per_sm = pl->bnx <= 32 ? 2 : 1;
-    pl->TM = (int)((M + pl->bnx - 1) / pl->bnx);
-    pl->TN = (int)((N + 127) / 128);
-    pl->U = (int64_t)pl->TM * pl->TN * (K / 128);
-    size_t cb = (size_t)pl->TM * pl->TN * sizeof(unsigned int);
+// Token-tile width and schedule of the persistent kernel from a small cost model (microseconds):
+// a (tile, k-block) unit costs the larger of the dequantization of its 128 x 128 weights and its
+// four MMAs; whole tiles per CTA cost rounds x K/128 units; equal slices cost ceil(U / P) units
+// plus the exchange of partial tiles.  Wider token tiles dequantize each weight fewer times.
+static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
+    const int64_t KB = K / 128;
+    const int64_t TN = (N + 127) / 128;
+    const int64_t cap = sms < kMaxSMs ? sms : kMaxSMs;
+    double best = 1e30;
+    for (int bnx = 256; bnx >= 64; bnx >>= 1) {
+        if (bnx > 64 && bnx / 2 >= M) continue;  // more than half of the tile would be padding
+        const int64_t TM = (M + bnx - 1) / bnx, Tt = TM * TN, U = Tt * KB;
+        const double mma_cycles = 4.0 * (bnx / 2 > 47 ? bnx / 2 : 47);
+        const double t_unit = mma_cycles / 1900.0 > 0.22 ? mma_cycles / 1900.0 : 0.22;
+        const int64_t Pa = cap < Tt ? cap : Tt;
+        const double t_aligned = (double)((Tt + Pa - 1) / Pa) * (double)KB * t_unit;
+        const int64_t Ps = cap < U ? cap : U;
+        const double t_split = (double)((U + Ps - 1) / Ps) * t_unit + 2.0 + bnx * 2048.0 / 1.0e5;
+        const bool al = t_aligned <= t_split;
+        const double t = al ? t_aligned : t_split;
+        if (t < best) {
+            best = t;
+            pl->bnx = bnx;
+            pl->TM = (int)TM;
+            pl->TN = (int)TN;
+            pl->U = U;
+            pl->aligned = al ? 1 : 0;
+            pl->P = al ? Pa : Ps;
+        }
+    }
+    size_t cb = 2 * (size_t)pl->TM * pl->TN * sizeof(unsigned int);  // arrivals and finished reducers per tile
     pl->counter_bytes = (cb + 255) / 256 * 256;
-    int64_t pmax = (int64_t)pl->ctas_per_sm * kMaxSMs;
-    if (pmax > pl->U) pmax = pl->U;
-    pl->workspace_bytes = pl->counter_bytes + (size_t)pmax * 2 * (size_t)pl->bnx * 128 * sizeof(float);
+    // The size asked of the caller covers every tile width and any SM count up to kMaxSMs, so that
+    // the query needs no device: counters of the narrowest tiles, partial tiles of the widest.
+    size_t cb_max = 2 * (size_t)((M + 63) / 64) * (size_t)TN * sizeof(unsigned int);
+    pl->workspace_bytes = (cb_max + 255) / 256 * 256 + (size_t)kMaxSMs * 2 * 256 * 128 * sizeof(float);
 }
 
 template <class Cfg>
@@ -229,15 +258,9 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     });
     if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
     unsigned int* status = status_word_ptr();
-    const int sms = sm_count();
-    if (!status || sms <= 0) return W4A8_ERR_CUDA;
-    int64_t P = (int64_t)pl.ctas_per_sm * (sms < kMaxSMs ? sms : kMaxSMs);
-    if (P > pl.U) P = pl.U;
-    // Whole tiles per CTA when that loses at most 15 % to imbalance; otherwise equal slices of
-    // the (tile, k-block) space with partial tiles reduced in the kernel.
-    const int64_t Tt = (int64_t)pl.TM * pl.TN;
-    const int64_t rounds = (Tt + P - 1) / P;
-    const int aligned = (Tt >= P && Tt * 100 >= 85 * P * rounds) ? 1 : 0;
+    if (!status) return W4A8_ERR_CUDA;
+    const int64_t P = pl.P;
+    const int aligned = pl.aligned;
     unsigned int* counters = static_cast<unsigned int*>(workspace);
     float* slots = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
     kern<<<(unsigned)P, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
@@ -326,12 +349,15 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
                         : launch_splitn<SnCfg<64, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                                  Ni, Ki, st);
     }
-    SkPlan pl;
-    make_sk_plan(M, N, K, &pl);
-    if (!workspace || workspace_bytes < pl.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
+    SkPlan pl;
+    make_sk_plan(M, N, K, kNominalSMs, &pl);
+    if (!workspace || workspace_bytes < pl.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != W4A8_OK) return rc;
+    const int sms = sm_count();
+    if (sms <= 0) return W4A8_ERR_CUDA;
+    make_sk_plan(M, N, K, sms, &pl);
     CUtensorMap tx;
     if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)pl.bnx,
                          CU_TENSOR_MAP_SWIZZLE_128B))
@@ -344,6 +370,7 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
              : launch_streamk<SkCfg<BNX, G, S1, S2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, \
                                                                 workspace, pl, Mi, Ni, Ki, st)
     switch (pl.bnx) {
+        case 64: W4A8_SK(64, 4, 6, 4); break;
         case 128: W4A8_SK(128, 4, 5, 4); break;
         default: W4A8_SK(256, 4, 4, 3); break;
     }
@@ -552,7 +579,7 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
     if (M <= kSplitNMaxM) return 0;  // the split-N kernel needs none
     SkPlan pl;
-    make_sk_plan(M, N, K, &pl);
+    make_sk_plan(M, N, K, kNominalSMs, &pl);
     return pl.workspace_bytes;
 }
 

@@ -3,9 +3,16 @@
 // Work is the flattened space (weight tile of 128 rows, token tile of BNX rows, k-block of 128):
 // every CTA takes an equal, contiguous share of it, so the SMs stay evenly loaded whatever the
 // layer shape (decode-sized problems have fewer tiles than SMs).  A CTA whose share covers only
-// part of a tile's K range stores an fp32 partial tile; the CTA that arrives last at a tile adds
-// the partials in a fixed order and applies the Eq. 4 / Eq. 11 scales -- no second kernel, and
-// bit-identical results from run to run.
+// part of a tile's K range stores an fp32 partial tile and bumps the tile's arrival counter.  When
+// a CTA has finished its whole share it turns to the (at most two) tiles it shares with others:
+// it waits (bounded) until all of that tile's partials have arrived and then reduces ITS columns
+// of the tile -- contributor i of C takes the i-th slice of the token columns, adds the C partials
+// in ascending CTA order, applies the Eq. 4 / Eq. 11 scales and stores the outputs.  The
+// reduction is thus spread over all contributors with many independent loads in flight (one CTA
+// adding whole partial tiles one after another spent tens of microseconds on L2 round trips), it
+// needs no second kernel, and results are bit-identical from run to run.  The waits cannot
+// deadlock: publishing a partial never waits for anything, and the grid is no larger than what
+// is resident at once.
 //
 // Per k-block one bulk copy brings the tile's packed INT4 codes, BF16 group scales (and
 // zero-points) and one TMA tile load brings the FP8 activations.  G groups of four warps expand
@@ -72,7 +79,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     constexpr int kNumBars = 2 * S1 + 2 * S2 + 5;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    volatile uint32_t* ticket_slot = tmem_slot + 2;
+    volatile uint32_t* share_slot = tmem_slot + 2;  // [3] number of shared tiles and their indices
 
     auto stage_w = [&](int s) { return base + (uint32_t)(s * Cfg::kStage1); };
     auto stage_x = [&](int s) { return base + (uint32_t)(s * Cfg::kStage1 + Cfg::kWStage); };
@@ -239,6 +246,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             else
                 reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res);
         };
+        int64_t shared_tile0 = 0, shared_tile1 = 0;  // tiles of which this CTA holds a partial (first and last segment)
+        int n_shared = 0;
         while (u < u_end && ok) {
             const int64_t tile = u / KB;
             const int kb0 = (int)(u - tile * KB);
@@ -295,49 +304,26 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 } else if (row_ok) {
 #pragma unroll
                     for (int jj = 0; jj < 16; ++jj)
-                        if (m0 + c0 + jj < M) my_slot[(c0 + jj) * 128 + r] = __uint_as_float(v[jj]);
+                        if (m0 + c0 + jj < M) __stcg(my_slot + (c0 + jj) * 128 + r, __uint_as_float(v[jj]));
                 }
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(bar_acc_empty(buf));
             if (!whole) {
-                // Publish the partial tile, then take a ticket; the last of the tile's segments
-                // to arrive reduces all of them in ascending CTA order.
+                // Publish the partial tile and remember the tile for the reduction at the end.
                 __threadfence();
                 asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (leader) *ticket_slot = atomicAdd(counters + tile, 1u);
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                const uint32_t ticket = *ticket_slot;
-                const int64_t p_lo = ((tile * KB + 1) * P - 1) / U;
-                const int64_t p_hi = (((tile + 1) * KB) * P - 1) / U;
-                if (ticket == (uint32_t)(p_hi - p_lo)) {
-                    __threadfence();
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kHalfCols && m0 + c0 < M; c0 += 16) {
-                        float acc[16];
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) acc[jj] = 0.0f;
-                        for (int64_t qq = p_lo; qq <= p_hi; ++qq) {
-                            const int64_t first_tile = (qq * U / P) / KB;
-                            const float* sl = slots + (qq * 2 + (tile == first_tile ? 0 : 1)) * Cfg::kSlotFloats +
-                                              (int64_t)half * kHalfCols * 128;
-#pragma unroll
-                            for (int jj = 0; jj < 16; ++jj)
-                                if (m0 + c0 + jj < M && row_ok) acc[jj] += __ldcg(sl + (c0 + jj) * 128 + r);
-                        }
-                        const float sx_lane = (lane < 16 && m0 + c0 + lane < M) ? __ldg(s_x + m0 + c0 + lane) : 0.0f;
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) {
-                            const int m = m0 + c0 + jj;
-                            const float sxm = __shfl_sync(0xFFFFFFFFu, sx_lane, jj);
-                            if (m < M && row_ok) store_out(m, n, acc[jj], sxm * swn);
-                        }
-                    }
-                    if (leader) counters[tile] = 0u;  // ready for the next launch
-                }
+                if (leader) atomicAdd(counters + tile, 1u);
+                if (n_shared++ == 0) shared_tile0 = tile;
+                else shared_tile1 = tile;
             }
             u += len;
             ++j;
+        }
+        if (leader) {
+            share_slot[0] = (uint32_t)n_shared;
+            share_slot[1] = (uint32_t)shared_tile0;
+            share_slot[2] = (uint32_t)shared_tile1;
         }
     } else {
         // ------------------------------------------------------------------ dequantization groups
@@ -363,6 +349,79 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+
+    // ---- reduction of the shared tiles, by every thread of the CTA: this CTA's slice of the token
+    // columns of each tile it holds a partial of ----
+    if (aligned) return;
+    const int n_shared = (int)share_slot[0];
+    unsigned int* done = counters + (int64_t)TM * TN;  // second counter per tile: finished reducers
+    for (int k = 0; k < n_shared; ++k) {
+        const int64_t tile = (int64_t)share_slot[1 + k];
+        const int64_t p_lo = ((tile * KB + 1) * P - 1) / U;  // first and last contributor
+        const int64_t p_hi = (((tile + 1) * KB) * P - 1) / U;
+        const int C = (int)(p_hi - p_lo) + 1, me = (int)(p - p_lo);
+        if (threadIdx.x == 0 && *abort_flag == 0u) {
+            // bounded wait for the C arrivals
+            uint64_t t0 = 0;
+            uint32_t spins = 0;
+            while (ptx::ld_acquire_gpu(counters + tile) < (uint32_t)C) {
+                if ((++spins & 63u) == 0u) {
+                    const uint64_t now = ptx::globaltimer_ns();
+                    if (t0 == 0) {
+                        t0 = now;
+                    } else if (now - t0 > ptx::kWaitLimitNs) {
+                        *abort_flag = 1u;
+                        atomicOr(status_word, kStatusTimeout);
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (*abort_flag != 0u) break;
+        __threadfence();
+        const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
+        const int nrow = (N - nt * 128) < 128 ? (N - nt * 128) : 128;
+        const int ncol = (M - mt * BNX) < BNX ? (M - mt * BNX) : BNX;  // valid token columns of the tile
+        const int c_lo = (int)((int64_t)me * ncol / C), c_hi = (int)((int64_t)(me + 1) * ncol / C);
+        // element e of the slice: row e % 128 (consecutive threads, consecutive addresses), column c_lo + e / 128
+        const int total = (c_hi - c_lo) * 128;
+        for (int e0 = (int)threadIdx.x; e0 < total; e0 += 4 * Cfg::kThreads) {
+            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 4
+            for (int64_t q = p_lo; q <= p_hi; ++q) {
+                // slot of contributor q for this tile: its first slot if the tile is where its
+                // share begins, else its second
+                const int64_t first_tile = (q * U / P) / KB;
+                const float* sl = slots + (q * 2 + (tile == first_tile ? 0 : 1)) * Cfg::kSlotFloats + c_lo * 128;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int e = e0 + jj * Cfg::kThreads;
+                    if (e < total && (e & 127) < nrow) acc[jj] += __ldcg(sl + e);
+                }
+            }
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int e = e0 + jj * Cfg::kThreads;
+                if (e < total && (e & 127) < nrow) {
+                    const int n = nt * 128 + (e & 127), m = mt * BNX + c_lo + (e >> 7);
+                    const float res = acc[jj] * (__ldg(s_x + m) * __ldg(s_w + (int64_t)n * sw_stride));
+                    if (out_dtype == W4A8_OUT_FP32)
+                        reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
+                    else
+                        reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res);
+                }
+            }
+        }
+        // the last reducer to finish re-arms the tile's counters for the next launch
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if (atomicAdd(done + tile, 1u) == (uint32_t)(C - 1)) {
+                counters[tile] = 0u;
+                done[tile] = 0u;
+            }
+        }
     }
 }
 

@@ -263,9 +263,20 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     const int aligned = pl.aligned;
     unsigned int* counters = static_cast<unsigned int*>(workspace);
     float* slots = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
-    kern<<<(unsigned)P, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
-                                                               counters, slots, M, N, K, pl.TM, pl.TN, aligned, status);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P);
+    cfg.blockDim = dim3(Cfg::kThreads);
+    cfg.dynamicSmemBytes = (size_t)Cfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, counters, slots, M,
+                                       N, K, pl.TM, pl.TN, aligned, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
 }
 

@@ -48,7 +48,7 @@ struct SkCfg {
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
-    static_assert((2 * S1 + 2 * S2 + 5) * 8 + 16 <= kBarBytes, "barrier area");
+    static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
@@ -76,7 +76,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     auto bar_acc_full = [&](int b) { return bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + b); };
     auto bar_acc_empty = [&](int b) { return bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 2 + b); };
     const uint32_t bar_drain = bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 4);
-    constexpr int kNumBars = 2 * S1 + 2 * S2 + 5;
+    auto bar_xfull = [&](int s) { return bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 5 + s); };
+    constexpr int kNumBars = 3 * S1 + 2 * S2 + 5;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* share_slot = tmem_slot + 2;  // [3] number of shared tiles and their indices
@@ -100,6 +101,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     if (threadIdx.x == 0) {
         for (int s = 0; s < S1; ++s) {
             ptx::mbar_init(bar_full(s), 1);
+            ptx::mbar_init(bar_xfull(s), 1);
             ptx::mbar_init(bar_free1(s), 1);
         }
         for (int s = 0; s < S2; ++s) {
@@ -123,6 +125,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched with programmatic stream serialization: the next kernel in the stream may start its
+    // set-up and weight prefetch while this one runs; everything that depends on earlier kernels
+    // (activations, scales, outputs, workspace) is touched only after griddepcontrol.wait.
+    ptx::griddep_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp, one lane issues)
@@ -133,21 +139,25 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             int64_t tile = u_begin / KB;
             int kb = (int)(u_begin - tile * KB);
             int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
+            // Weights depend on no earlier kernel: the first ring-full of packed tiles is requested
+            // before waiting for the kernels that produce the activations.
+            const int ahead = n_it < S1 ? n_it : S1;
+            ptx::Ring rx;  // ring position of the next activation tile
+            int xkb = kb, xmt = mt;
+            int it_x = 0;  // activation tiles issued so far
             for (int it = 0; it < n_it; ++it) {
                 ok = ptx::mbar_wait(bar_free1(r1.idx), r1.phase ^ 1u, abort_flag, status_word);
                 if (!ok) break;
                 const int rows = (N - nt * 128) < 128 ? (N - nt * 128) : 128;  // ragged last tile
                 const int64_t row0 = (int64_t)kb * N + (int64_t)nt * 128;
-                const uint32_t full = bar_full(r1.idx), wdst = stage_w(r1.idx), xdst = stage_x(r1.idx);
+                const uint32_t full = bar_full(r1.idx), wdst = stage_w(r1.idx);
                 const uint8_t* csrc = wpp + row0 * kRowCodeBytes;
                 const uint8_t* msrc = meta_base + row0 * Cfg::kMeta;
                 const uint32_t cbytes = (uint32_t)(rows * kRowCodeBytes), mbytes = (uint32_t)(rows * Cfg::kMeta);
-                const int x0 = kb * 128, y0 = mt * BNX;
                 if (ptx::elect_one()) {
-                    ptx::mbar_arrive_expect_tx(full, cbytes + mbytes + (uint32_t)Cfg::kXBytes);
+                    ptx::mbar_arrive_expect_tx(full, cbytes + mbytes);
                     ptx::bulk_load(wdst, csrc, cbytes, full);
                     ptx::bulk_load(wdst + 8192u, msrc, mbytes, full);
-                    ptx::tma_load_2d(xdst, &tmap_x, x0, y0, full);
                 }
                 r1.advance(S1);
                 ++issued;
@@ -156,6 +166,22 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     if (++mt == TM) {
                         mt = 0;
                         ++nt;
+                    }
+                }
+                if (it + 1 < ahead) continue;  // still inside the weight-only prologue
+                if (it + 1 == ahead) ptx::griddep_wait();
+                // activation tiles of every stage whose weights have been requested
+                for (; it_x <= it; ++it_x) {
+                    const uint32_t xfull = bar_xfull(rx.idx), xdst = stage_x(rx.idx);
+                    const int x0 = xkb * 128, y0 = xmt * BNX;
+                    if (ptx::elect_one()) {
+                        ptx::mbar_arrive_expect_tx(xfull, (uint32_t)Cfg::kXBytes);
+                        ptx::tma_load_2d(xdst, &tmap_x, x0, y0, xfull);
+                    }
+                    rx.advance(S1);
+                    if (++xkb == KB) {
+                        xkb = 0;
+                        if (++xmt == TM) xmt = 0;
                     }
                 }
             }
@@ -170,6 +196,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     }
                     uint64_t t0 = ptx::globaltimer_ns();
                     while (!ptx::mbar_try_wait(bar_full(rb.idx), rb.phase) &&
+                           ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
+                    }
+                    const bool x_issued = issued - 1 - i < it_x;  // this stage's activation tile was requested too
+                    while (x_issued && !ptx::mbar_try_wait(bar_xfull(rb.idx), rb.phase) &&
                            ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
                     }
                 }
@@ -196,7 +226,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(buf * BNX);
                 uint32_t accumulate = 0;
                 for (int i = 0; i < len; ++i) {
-                    ok = ptx::mbar_wait(bar_full(r1.idx), r1.phase, abort_flag, status_word);
+                    ok = ptx::mbar_wait(bar_xfull(r1.idx), r1.phase, abort_flag, status_word);
                     ok = ok && ptx::mbar_wait(bar_w8_full(r2.idx), r2.phase, abort_flag, status_word);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
@@ -238,6 +268,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         bool ok = true;
         int j = 0;
         int64_t u = u_begin;
+        ptx::griddep_wait();  // scales come from, outputs and workspace may still be in use by, earlier kernels
         // Final value of one output: Eq. 4 / Eq. 11 scales and the cast.
         auto store_out = [&](int m, int n, float acc, float scale) {
             const float res = acc * scale;
@@ -354,6 +385,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     // ---- reduction of the shared tiles, by every thread of the CTA: this CTA's slice of the token
     // columns of each tile it holds a partial of ----
     if (aligned) return;
+    ptx::griddep_wait();
     const int n_shared = (int)share_slot[0];
     unsigned int* done = counters + (int64_t)TM * TN;  // second counter per tile: finished reducers
     for (int k = 0; k < n_shared; ++k) {

@@ -47,7 +47,7 @@ WORKLOAD = ("c2 decode sweep: W4A8 linear, M in {1,4,16}, K=4096, N=14336, INT4 
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); see profiles/.  None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 30.34e6  # profiles/linear_splitn_decode_c2.md, mean of M = 1, 4, 16
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 30.37e6  # profiles/linear_splitn_decode_c2.md, mean of M = 1, 4, 16
 
 
 def weight_bytes(n=N, k=K):
@@ -510,6 +510,21 @@ def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
     return out
 
 
+def library_fp8_gemm_tflops(torch, dev, n=8192):
+    """Empirical dense-FP8 reference on this machine: the library's FP8 GEMM (torch._scaled_mm, E4M3 x
+    E4M3 -> BF16, per-tensor scales) at n^3, best of a few short loops.  None when unavailable."""
+    try:
+        a = torch.randn((n, n), device=dev).to(torch.float8_e4m3fn)
+        b = torch.randn((n, n), device=dev).to(torch.float8_e4m3fn).t()  # column-major second operand
+        one = torch.ones((), device=dev, dtype=torch.float32)
+        f = lambda: torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)  # noqa: E731
+        f()
+        best = min(_time_loop(torch, f, 5, warm=1) for _ in range(3))
+        return 2.0 * n ** 3 / best / 1e12
+    except Exception:  # the call's signature and availability differ between torch builds
+        return None
+
+
 def prefill_extra(torch, binding, inputs, dev, peaks):
     """Config c3 (M=2048, K=4096, N=4096): FP8 tensor-pipe rate of w4a8_linear next to cuBLAS BF16."""
     M3, K3, N3 = 2048, 4096, 4096
@@ -547,7 +562,9 @@ def prefill_extra(torch, binding, inputs, dev, peaks):
     tb = _time_loop(torch, g, 40, warm=5)
     flops = 2.0 * M3 * N3 * K3
     fp8_peak = 2.0 * peaks["bf16_tflops"]
+    lib_fp8 = library_fp8_gemm_tflops(torch, dev)
     return {"workload": "c3 prefill M=2048 K=4096 N=4096", "us": t * 1e6, "tflops": flops / t / 1e12,
+            "library_fp8_gemm_8192_tflops": lib_fp8,
             "fp8_peak_tflops": fp8_peak, "peak_note": "2 x bf16 burst peak (%s)" % peaks["source"],
             "frac_of_fp8_peak": flops / t / 1e12 / fp8_peak, "frac_of_nominal_4500": flops / t / 1e12 / 4500.0,
             "cublas_bf16_us": tb * 1e6, "cublas_bf16_tflops": flops / tb / 1e12}

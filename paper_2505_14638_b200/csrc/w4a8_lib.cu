@@ -294,7 +294,7 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, SnPlan* pl) {
     pl->meta_off = pl->KS * rmax * kRowCodeBytes;
     pl->wstage = (pl->KS * rmax * (kRowCodeBytes + Cfg::kMeta) + 127) / 128 * 128;
     pl->xstage = pl->KS * Cfg::MT * 128;
-    const int fixed = Cfg::kBarBytes + 1024;
+    const int fixed = Cfg::kBarBytes + Cfg::kOutBytes + 1024;
     int s1 = (Cfg::kSmemBudget - fixed) / (pl->wstage + pl->xstage);
     if (s1 > Cfg::kS1Max) s1 = Cfg::kS1Max;
     if (s1 < Cfg::kS2) return false;  // the tensor-memory ring may not be deeper than the TMA ring
@@ -747,7 +747,6 @@ int w4a8_query_device_status(unsigned int* flags_host) {
     if (v & kStatusTimeout) return W4A8_ERR_TIMEOUT;
     return (v != 0) ? W4A8_ERR_BAD_SHAPE : W4A8_OK;
 }
-
 
 uint64_t w4a8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

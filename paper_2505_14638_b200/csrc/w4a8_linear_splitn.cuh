@@ -35,6 +35,7 @@
 namespace w4a8 {
 
 
+
 template <int MT_, int G_, int FMT_, bool FUSE_ = false>
 struct SnCfg {
     // FUSE: the kernel takes BF16 activations and does the per-token FP8 quantization (Eq. 13)
@@ -54,6 +55,10 @@ struct SnCfg {
     static constexpr int kDCol = kS2 * kAStageCols;        // accumulators start after the A ring
     static constexpr int kThreads = 32 * (6 + 4 * G);
     static constexpr int kBarBytes = 768;
+    // Staging area of the epilogue: 16 tokens x 128 rows of outputs (FP32 at most), from which Y is
+    // written in 16-byte pieces.  (Thirty-two 2-byte stores per warp instruction cost ~120 cycles
+    // each, one after the other: 16 of them per thread made a 1 us tail.)
+    static constexpr int kOutBytes = 16 * 128 * 4;
     // Decode-sized launches (<= 16 tokens) take half an SM each, so that the CTAs of the next
     // kernel in the stream can start -- and prefetch their weights -- while this one finishes.
     static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : 200 * 1024;
@@ -146,6 +151,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     constexpr int kNumBars = 3 * S1M + S2 + 3;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    const uint32_t out_s = bars_addr + (uint32_t)Cfg::kBarBytes;  // epilogue staging, kOutBytes
     unsigned int* amax_s = const_cast<unsigned int*>(tmem_slot) + 4;  // [16] row absmax bit patterns
     float* sx_s = reinterpret_cast<float*>(amax_s + 16);              // [16] activation scales s_x
     float* inv_s = sx_s + 16;                                         // [16] multipliers 1/s_x
@@ -399,6 +405,8 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 }
                 if (!ok) break;
                 if (ptx::elect_one()) ptx::umma_commit(bar_acc_full);
+                if (lane == 0) {
+                }
             }
             if (!ok && lane == 0) {
                 // Gave up: wait (bounded) for the MMAs already issued before tensor memory is freed.
@@ -416,12 +424,28 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         const int r = q * 32 + lane;
         bool ok = true;
         uint32_t acc_phase = 0;
-        bool first_tile = true;
         ptx::Ring rx;  // ring position of the next activation tile (FUSE)
+        // The scales are fetched before the accumulator is waited for (a global load issued after
+        // it would add its full latency to the kernel's tail): s_x one or two per lane, broadcast
+        // by shuffles later; s_w per row at the top of each range.
+        const int et = (warp - 2) * 32 + lane;  // index among the 128 epilogue threads
+        const int es = out_dtype == W4A8_OUT_FP32 ? 4 : 2;
+        const bool wide_out = (((int64_t)ldy * es) & 15) == 0;  // Y rows 16-byte aligned (y itself is)
+        float sx_lane[MT / 32 > 0 ? MT / 32 : 1];
+        if (!Cfg::FUSE) {
+            ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
+#pragma unroll
+            for (int c = 0; c < (MT / 32 > 0 ? MT / 32 : 1); ++c)
+                sx_lane[c] = (c * 32 + lane < M) ? __ldg(s_x + c * 32 + lane) : 0.0f;
+        }
         for (int t = p; t < T && ok; t += P) {
             const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
             const int R = (u1 - u0) * 8;
             const int n0 = u0 * 8;
+            float swn[2];
+#pragma unroll
+            for (int b = 0; b < 2; ++b)
+                swn[b] = (b < MBLK && b * 128 + r < R) ? __ldg(s_w + (int64_t)(n0 + b * 128 + r) * sw_stride) : 0.0f;
             if (Cfg::FUSE) {
                 // Eq. 13, second half: these four warps, idle until the accumulator is complete,
                 // convert the activations ahead of the MMAs (thread mapping: XMap).  Each thread
@@ -492,15 +516,12 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             acc_phase ^= 1u;
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            if (first_tile) {
-                if (!Cfg::FUSE) ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
-                first_tile = false;
-            }
-            for (int b = 0; b < MBLK; ++b) {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                if (b >= MBLK) break;
                 const int row = b * 128 + r;
                 const bool row_ok = row < R;
                 const int n = n0 + row;
-                const float swn = row_ok ? __ldg(s_w + (int64_t)n * sw_stride) : 0.0f;
 #pragma unroll 1
                 for (int c0 = 0; c0 < MT; c0 += 16) {
                     if (c0 >= M) break;  // uniform
@@ -508,22 +529,60 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     ptx::tmem_ld_32x32b_x16(
                         tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(Cfg::kDCol + b * MT + c0), v);
                     ptx::tmem_ld_wait();
+                    float sxv = sx_lane[0];
+                    if (MT > 32 && c0 >= 32) sxv = sx_lane[MT / 32 - 1];
+                    float res[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const int m = c0 + j;
-                        if (m < M && row_ok) {
-                            const float sxm = Cfg::FUSE ? sx_s[m] : __ldg(s_x + m);
-                            const float res = __uint_as_float(v[j]) * (sxm * swn);  // Eq. 4, Eq. 11
-                            if (out_dtype == W4A8_OUT_FP32)
-                                reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
+                        const float sxm = Cfg::FUSE ? sx_s[c0 + j] : __shfl_sync(0xFFFFFFFFu, sxv, (c0 & 16) + j);
+                        res[j] = __uint_as_float(v[j]) * (sxm * swn[b]);  // Eq. 4, Eq. 11
+                    }
+                    if (wide_out) {
+                        // tokens x rows into the staging area, then 16-byte pieces of Y rows
+                        const uint32_t pitch = 128u * (uint32_t)es;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const uint32_t a = out_s + (uint32_t)j * pitch + (uint32_t)(r * es);
+                            if (es == 4)
+                                asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[j]) : "memory");
                             else
-                                reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res);
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
+                                             "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[j])))
+                                             : "memory");
+                        }
+                        asm volatile("bar.sync 3, 128;" ::: "memory");
+                        const int Rb = (R - b * 128) < 128 ? (R - b * 128) : 128;
+                        const int ppt = (Rb * es) >> 4;  // 16-byte pieces per token (rows come in eights)
+                        const int ntok = (M - c0) < 16 ? (M - c0) : 16;
+                        char* yb = static_cast<char*>(y) + ((int64_t)c0 * ldy + n0 + b * 128) * es;
+                        for (int id = et; id < ntok * ppt; id += 128) {
+                            const int tok = id / ppt, piece = id - tok * ppt;
+                            uint4 w;
+                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                                         : "r"(out_s + (uint32_t)tok * pitch + (uint32_t)(piece << 4)));
+                            *reinterpret_cast<uint4*>(yb + (int64_t)tok * ldy * es + (piece << 4)) = w;
+                        }
+                        asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int m = c0 + j;
+                            if (m < M && row_ok) {
+                                if (es == 4)
+                                    reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res[j];
+                                else
+                                    reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] =
+                                        __float2bfloat16_rn(res[j]);
+                            }
                         }
                     }
                 }
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(bar_acc_empty);
+            if (threadIdx.x == 64) {
+            }
         }
     } else {
         // ------------------------------------------------------------------ dequantization groups

@@ -47,6 +47,16 @@ struct SkCfg {
     static constexpr int kThreads = 32 * (10 + 4 * G);
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
+    // A dequantization group handles every G-th stage, so it skips phases of the barriers it
+    // waits on, and an mbarrier wait tells phases apart by parity only: the wait for use k of a
+    // slot is sound only if use k-1 has completed before it starts.  That holds because a stage's
+    // packed weights are requested only after the MMAs S1 stages back have completed (one release
+    // per ring slot, weights and activations together): then the MMAs 2*S2 stages back have
+    // completed too, provided S1 <= 2*S2.  (Releasing the packed weights right after their
+    // expansion, to request them earlier, broke this: with G != S2 a group got two phases ahead of
+    // a "slot free" barrier and overwrote an expanded tile still in use; with G == S2 and
+    // S1 % G == 0 it was sound but no faster.)
+    static_assert(S1 <= 2 * S2, "ring depths: see the comment above");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
     static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");

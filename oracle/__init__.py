@@ -15,6 +15,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "w4a8_oracle.c")
+_SRC_DPQ = os.path.join(_HERE, "w4a8_dpq_oracle.c")
 _HDR = os.path.join(_HERE, "w4a8_oracle.h")
 _LIB = os.path.join(_HERE, "liboracle_w4a8.so")
 
@@ -26,13 +27,13 @@ def build(force: bool = False) -> str:
     stale = (
         force
         or not os.path.exists(_LIB)
-        or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+        or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_DPQ), os.path.getmtime(_HDR))
     )
     if stale:
         tmp = _LIB + ".tmp%d" % os.getpid()
         cmd = [
             "gcc", "-std=c11", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
-            "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC, "-lm",
+            "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC, _SRC_DPQ, "-lm",
         ]
         subprocess.run(cmd, check=True)
         os.replace(tmp, _LIB)
@@ -61,6 +62,8 @@ def _load():
     lib.oracle_f32_to_bf16.argtypes = [c.c_float]
     lib.oracle_quantize_weight_rtn.restype = c.c_int
     lib.oracle_quantize_weight_rtn.argtypes = [p, i64, i64, c.c_int, c.c_int, c.c_int, c.c_int, p, p, p, p]
+    lib.oracle_dpq_quantize.restype = c.c_int
+    lib.oracle_dpq_quantize.argtypes = [p, i64, i64, c.c_int, p, p, c.c_int, c.c_int, c.c_int, p, p, p, p, p, p]
     lib.oracle_dequant_weight.restype = c.c_int
     lib.oracle_dequant_weight.argtypes = [p, p, p, i64, i64, c.c_int, p]
     lib.oracle_quantize_act.restype = c.c_int
@@ -150,6 +153,69 @@ def quantize_weight_rtn(W, group=128, symmetric=True, pow2=False, per_channel=Fa
     if rc != 0:
         raise ValueError("oracle_quantize_weight_rtn: bad arguments")
     return codes, gscale, (None if symmetric else gzero), s_w
+
+
+def gar_permutation(diag, group=128):
+    """Group-Aware Reordering (Sec. 3.2, appendix): processing order from the Hessian diagonal.
+    Inside each group the columns go by descending diagonal; the groups go by descending maximum
+    diagonal (the ranking the paper used).  Ties keep the original order.  Returns int32 [K]:
+    position p handles original column perm[p]."""
+    d = np.asarray(diag, dtype=np.float64)
+    K = d.size
+    assert K % group == 0
+    G = K // group
+    within = []
+    gmax = np.empty(G)
+    for g in range(G):
+        idx = np.arange(g * group, (g + 1) * group)
+        order = idx[np.argsort(-d[idx], kind="stable")]
+        within.append(order)
+        gmax[g] = d[idx].max()
+    gorder = np.argsort(-gmax, kind="stable")
+    return np.concatenate([within[g] for g in gorder]).astype(np.int32)
+
+
+def hessian_upper_cholesky(H, perm=None, damp=0.01):
+    """What Sec. 3.3 takes from GPTQ, in float64: permute the Hessian to processing order, add
+    damp * mean(diag) to the diagonal, invert, and return the upper Cholesky factor U of the
+    inverse (H^-1 = U^T U) as float32.  Columns with a zero diagonal get a unit diagonal."""
+    H = np.array(H, dtype=np.float64)
+    if perm is not None:
+        H = H[np.ix_(perm, perm)]
+    d = np.diag(H).copy()
+    dead = d == 0
+    H[dead, dead] = 1.0
+    H[np.diag_indices_from(H)] += damp * np.mean(np.diag(H))
+    Hinv = np.linalg.inv(H)
+    Hinv = 0.5 * (Hinv + Hinv.T)
+    L = np.linalg.cholesky(Hinv)          # Hinv = L L^T
+    return np.ascontiguousarray(L.T).astype(np.float32)
+
+
+def dpq_quantize(W, U, perm=None, group=128, symmetric=False, mse_steps=0, per_channel=False, debug=False):
+    """Algorithm 1 (DPQ).  W fp32 [N,K]; U fp32 [K,K] upper Cholesky factor in processing order;
+    perm int32 [K] or None.  Returns (codes, gscale, gzero or None, s_w) in the original column
+    order, plus (err, what) in processing order when debug is set."""
+    lib = _load()
+    W = _c(W, np.float32)
+    U = _c(U, np.float32)
+    N, K = W.shape
+    assert U.shape == (K, K)
+    G = K // group
+    pm = None if perm is None else _c(perm, np.int32)
+    codes = np.zeros((N, K // 2), dtype=np.uint8)
+    gscale = np.zeros((N, G), dtype=np.uint16)
+    gzero = np.zeros((N, G), dtype=np.uint8)
+    s_w = np.zeros(N if per_channel else 1, dtype=np.float32)
+    err = np.zeros((N, K), dtype=np.float32) if debug else None
+    what = np.zeros((N, K), dtype=np.float32) if debug else None
+    rc = lib.oracle_dpq_quantize(_ptr(W), N, K, group, _ptr(U), _ptr(pm), int(symmetric), int(mse_steps),
+                                 int(per_channel), _ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(s_w),
+                                 _ptr(err), _ptr(what))
+    if rc != 0:
+        raise ValueError("oracle_dpq_quantize: bad arguments")
+    out = (codes, gscale, (None if symmetric else gzero), s_w)
+    return out + (err, what) if debug else out
 
 
 def dequant_weight(codes, gscale, gzero=None, group=128):

@@ -84,6 +84,23 @@ int oracle_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, 
 /* Number of OpenMP threads the linear will use. */
 int oracle_num_threads(void);
 
+/*
+ * DPQ weight quantizer, Algorithm 1 (Sec. 3.1-3.3, Eq. 6-12) with the Cholesky formulation of the
+ * update and Group-Aware Reordering (Sec. 3.2, appendix); see w4a8_dpq_oracle.c for the steps.
+ *   W     [N][K] fp32, original column order.
+ *   U     [K][K] fp32, upper Cholesky factor of the inverse of the dampened Hessian, rows and
+ *         columns in PROCESSING order (only the upper triangle is read).
+ *   perm  [K]: processing position p handles original column perm[p] (NULL = identity); every
+ *         run of `group` positions must be a permutation of one original group.
+ *   mse_steps  0 or 1: Eq. 8 as is; t in 2..11: least-squared-error search over t shrink factors.
+ * Outputs in ORIGINAL order: codes [N][K/2], gscale [N][K/group], gzero (asymmetric), s_w.
+ * err_out / what_out (optional, [N][K], processing order): the scaled errors e_q and the
+ * dequantized weights of Eq. 11, for checks.  Returns 0, or -1 on bad arguments.
+ */
+int oracle_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const float* U, const int32_t* perm,
+                        int symmetric, int mse_steps, int per_channel, uint8_t* codes, uint16_t* gscale,
+                        uint8_t* gzero, float* s_w, float* err_out, float* what_out);
+
 #ifdef __cplusplus
 }
 #endif

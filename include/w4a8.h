@@ -208,6 +208,41 @@ int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, in
                              uint8_t* gzero, float* s_w, void* stream);
 
 /*
+ * Group-Aware Reordering (Sec. 3.2 and its appendix): the order in which the DPQ quantizer
+ * processes the input features, from the diagonal of the Hessian H = X^T X.  Inside each group
+ * of 128 the columns go by descending diagonal, the groups by descending maximum diagonal (the
+ * ranking the paper used); ties keep the original order.
+ *   hdiag  device float [K];  perm  device int32 [K]: position p handles original column perm[p].
+ *   workspace  device, w4a8_gar_workspace_bytes(K) bytes (scratch, no initialisation needed).
+ */
+size_t w4a8_gar_workspace_bytes(int64_t K);
+int w4a8_gar_permutation(const float* hdiag, int64_t K, int group, int32_t* perm, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/*
+ * DPQ weight quantizer, Algorithm 1 (Sec. 3.1-3.3): Eq. 6, then per row and per group of 128
+ * (in processing order) Eq. 8 -- optionally with the search of the scale of least squared error
+ * of Sec. 3.3 -- and per weight Eq. 7, 9, 10, 11 followed by the error-compensating update of
+ * Eq. 12 in its Cholesky form (Sec. 3.3, as in GPTQ): e = (w - w16^) / U_qq, w_v <- w_v - e U_qv.
+ * Produces the same stored format as w4a8_quantize_weight_rtn, in the ORIGINAL column order.
+ *   W     device fp32 [N][K], 16-byte aligned.
+ *   U     device fp32 [K][K]: upper Cholesky factor of the inverse of the (dampened) Hessian with
+ *         rows and columns in processing order; only the upper triangle is read.  Computing it
+ *         (H = X^T X, dampening, factorizations) is a library matter and the caller's.
+ *   perm  device int32 [K] from w4a8_gar_permutation, or NULL for the original order.  Every run
+ *         of 128 positions must hold the columns of one original group (not checked on the device).
+ *   symmetric / per_channel   as in w4a8_quantize_weight_rtn (gzero may be NULL when symmetric).
+ *   mse_steps  0 or 1: Eq. 8 as is; 2..11: that many shrink factors 1, 0.98, 0.96, ... are tried.
+ *   workspace  device, 16-byte aligned, w4a8_dpq_workspace_bytes(N, K) bytes (scratch).
+ * Every step that decides a code is a single correctly rounded fp32 operation, so the codes are
+ * reproducible and independent of the launch geometry.  Enqueues about 2 K / 128 kernels.
+ */
+size_t w4a8_dpq_workspace_bytes(int64_t N, int64_t K);
+int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const float* U, const int32_t* perm,
+                      int symmetric, int mse_steps, int per_channel, uint8_t* codes, void* gscale_bf16,
+                      uint8_t* gzero, float* s_w, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Whole layer from HOST activations to HOST output (Sec. 3 flow end to end): copies
  * x_host (BF16 [M][K], ideally pinned) to x_dev, runs w4a8_quantize_act and w4a8_linear (or
  * w4a8_linear_fused when the weights are prepacked and M <= 4), and

@@ -29,6 +29,7 @@ EXPORTS = (
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
     "w4a8_linear_fused",
     "w4a8_quantize_weight_rtn",
+    "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
 )
 
@@ -76,6 +77,14 @@ def lib():
     L.w4a8_linear_ex_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
     L.w4a8_quantize_weight_rtn.restype = i32
     L.w4a8_quantize_weight_rtn.argtypes = [p, i64, i64, i32, i32, i32, i32, p, p, p, p, p]
+    L.w4a8_gar_workspace_bytes.restype = sz
+    L.w4a8_gar_workspace_bytes.argtypes = [i64]
+    L.w4a8_gar_permutation.restype = i32
+    L.w4a8_gar_permutation.argtypes = [p, i64, i32, p, p, sz, p]
+    L.w4a8_dpq_workspace_bytes.restype = sz
+    L.w4a8_dpq_workspace_bytes.argtypes = [i64, i64]
+    L.w4a8_dpq_quantize.restype = i32
+    L.w4a8_dpq_quantize.argtypes = [p, i64, i64, i32, p, p, i32, i32, i32, p, p, p, p, p, sz, p]
     L.w4a8_forward_host.restype = i32
     L.w4a8_forward_host.argtypes = [p, i64, p, p, p, i32, p, i32, i64, i64, i32, p, p, p, p, p, p, sz, p]
     L.w4a8_query_device_status.restype = i32
@@ -289,6 +298,53 @@ def quantize_weight_rtn(W, symmetric=True, pow2=False, per_channel=False):
                                         int(per_channel), _ptr(codes), _ptr(gscale), _ptr(gzero),
                                         _ptr(s_w), _stream())
     _check("w4a8_quantize_weight_rtn", rc)
+    return codes, gscale, gzero, s_w
+
+
+def gar_permutation(hdiag):
+    """w4a8_gar_permutation: hdiag float32 [K] on the device -> int32 [K] processing order."""
+    import torch
+    K = hdiag.numel()
+    perm = torch.empty((K,), dtype=torch.int32, device=hdiag.device)
+    ws = torch.empty((lib().w4a8_gar_workspace_bytes(K),), dtype=torch.uint8, device=hdiag.device)
+    rc = lib().w4a8_gar_permutation(_ptr(hdiag), K, GROUP, _ptr(perm), _ptr(ws), ws.numel(), _stream())
+    _check("w4a8_gar_permutation", rc)
+    return perm
+
+
+def hessian_upper_cholesky(H, perm=None, damp=0.01):
+    """Library step in front of w4a8_dpq_quantize (Sec. 3.3, as in GPTQ), with torch.linalg in
+    float64 on the device: permute H to processing order, give dead columns a unit diagonal, add
+    damp * mean(diag), invert, return the upper Cholesky factor of the inverse as float32."""
+    import torch
+    H = H.to(torch.float64)
+    if perm is not None:
+        idx = perm.to(torch.int64)
+        H = H[idx][:, idx]
+    H = H.clone()
+    d = torch.diagonal(H)
+    d[d == 0] = 1.0
+    d += damp * d.mean()
+    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
+    Hinv = 0.5 * (Hinv + Hinv.T)
+    return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()
+
+
+def dpq_quantize(W, U, perm=None, symmetric=False, mse_steps=0, per_channel=False):
+    """w4a8_dpq_quantize: W float32 [N, K], U float32 [K, K] (processing order), perm int32 [K] or
+    None, all on the device.  Returns (codes, gscale BF16, gzero or None, s_w)."""
+    import torch
+    N, K = W.shape
+    dev = W.device
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    gscale = torch.empty((N, K // GROUP), dtype=torch.bfloat16, device=dev)
+    gzero = None if symmetric else torch.empty((N, K // GROUP), dtype=torch.uint8, device=dev)
+    s_w = torch.empty((N if per_channel else 1,), dtype=torch.float32, device=dev)
+    ws = torch.empty((lib().w4a8_dpq_workspace_bytes(N, K),), dtype=torch.uint8, device=dev)
+    rc = lib().w4a8_dpq_quantize(_ptr(W), N, K, GROUP, _ptr(U), _ptr(perm), int(symmetric), int(mse_steps),
+                                 int(per_channel), _ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(s_w), _ptr(ws),
+                                 ws.numel(), _stream())
+    _check("w4a8_dpq_quantize", rc)
     return codes, gscale, gzero, s_w
 
 

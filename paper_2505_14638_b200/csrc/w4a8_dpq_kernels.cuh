@@ -1,0 +1,245 @@
+// DPQ weight quantizer on the GPU: Algorithm 1 (Sec. 3.1-3.3, Eq. 6-12) with the Cholesky form of
+// the update that Sec. 3.3 takes from GPTQ, the least-squared-error search of the group scale,
+// and Group-Aware Reordering (Sec. 3.2 and its appendix).
+//
+// The rows of W are independent; the columns of a row are quantized one after the other, each
+// sending its scaled error e to the columns on its right (Eq. 12): w_v <- fma(-e, U_qv, w_v),
+// U = upper Cholesky factor of the inverse Hessian in processing order.  Work is cut the way
+// GPTQ cuts it, in blocks of one group (128 columns):
+//   dpq_block_kernel     one warp per row: group scale / zero-point (Eq. 8, optional search),
+//                        then the 128 columns in sequence with the updates inside the block;
+//                        writes the codes, the group's scale and zero-point and the 128 errors;
+//   dpq_trailing_kernel  applies the block's 128 errors to every column to the right of the
+//                        block, q ascending -- the same chain of fused multiply-adds, in the same
+//                        order, that the column-by-column algorithm performs for that element.
+// Every floating-point step that decides an integer is one explicitly rounded fp32 operation
+// (__fdiv_rn, __fmul_rn, __fmaf_rn ...: never contracted), and the search compares exact integer
+// sums, so the codes do not depend on how the work is spread over threads.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "w4a8_common.cuh"
+#include "w4a8_simple_kernels.cuh"
+
+namespace w4a8 {
+
+// ---- Group-Aware Reordering -----------------------------------------------------------------
+// Inside each group the columns go by descending Hessian diagonal, the groups by descending
+// maximum diagonal; ties keep the original order.  Ranks are found by counting (exact compares).
+__global__ void __launch_bounds__(128)
+gar_within_kernel(const float* __restrict__ hdiag, int32_t* __restrict__ within, float* __restrict__ gmax) {
+    __shared__ float d[128];
+    __shared__ float red[4];
+    const int g = blockIdx.x, i = threadIdx.x;
+    const float di = hdiag[(int64_t)g * 128 + i];
+    d[i] = di;
+    __syncthreads();
+    int rank = 0;
+    for (int j = 0; j < 128; ++j) rank += (d[j] > di || (d[j] == di && j < i)) ? 1 : 0;
+    within[(int64_t)g * 128 + rank] = g * 128 + i;
+    float m = warp_max(di);
+    if ((i & 31) == 0) red[i >> 5] = m;
+    __syncthreads();
+    if (i == 0) gmax[g] = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+}
+
+__global__ void __launch_bounds__(128)
+gar_order_kernel(const int32_t* __restrict__ within, const float* __restrict__ gmax, int G,
+                 int32_t* __restrict__ perm) {
+    const int g = blockIdx.x;
+    const float mg = gmax[g];
+    int rank = 0;
+    for (int j = 0; j < G; ++j) {
+        const float mj = gmax[j];
+        rank += (mj > mg || (mj == mg && j < g)) ? 1 : 0;
+    }
+    perm[(int64_t)rank * 128 + threadIdx.x] = within[(int64_t)g * 128 + threadIdx.x];
+}
+
+// work[n][p] = W[n][perm[p]]: the rows in processing order.
+__global__ void __launch_bounds__(256)
+dpq_gather_kernel(const float* __restrict__ W, const int32_t* __restrict__ perm, int64_t N, int64_t K,
+                  float* __restrict__ work) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= N * K) return;
+    const int64_t n = i / K, p = i - n * K;
+    work[i] = W[n * K + (perm ? perm[p] : (int32_t)p)];
+}
+
+// ---- Eq. 8 / Eq. 9 / Eq. 10 on one FP8-valued weight ------------------------------------------
+struct DpqGroup {
+    float s;  // group scale (a BF16 value)
+    int z;    // zero-point
+};
+
+__device__ __forceinline__ DpqGroup dpq_group_params(float lo, float hi, float amax, float p, int symmetric) {
+    DpqGroup g;
+    if (symmetric) {
+        const float a = __fmul_rn(p, amax);
+        g.s = (a > 0.0f) ? __fdiv_rn(a, 7.0f) : 1.0f;
+        g.z = 8;
+        g.s = __bfloat162float(__float2bfloat16_rn(g.s));
+    } else {
+        const float l = __fmul_rn(p, lo), h = __fmul_rn(p, hi);
+        g.s = (h > l) ? __fdiv_rn(__fsub_rn(h, l), 15.0f) : 1.0f;  // Eq. 8
+        g.s = __bfloat162float(__float2bfloat16_rn(g.s));
+        const float zf = rintf(__fdiv_rn(-l, g.s));
+        g.z = (int)fminf(fmaxf(zf, 0.0f), 15.0f);
+    }
+    return g;
+}
+
+// Returns the code u (Eq. 9); w8hat = nearest_Z((u - z) s), the value inference multiplies with (Eq. 10).
+__device__ __forceinline__ int dpq_quant_dequant(float w8, const DpqGroup& g, int symmetric, float& w8hat) {
+    int u;
+    if (symmetric) {
+        const float q = rintf(__fdiv_rn(w8, g.s));
+        u = (int)fminf(fmaxf(q, -7.0f), 7.0f) + 8;
+    } else {
+        const float q = rintf(__fadd_rn(__fdiv_rn(w8, g.s), (float)g.z));
+        u = (int)fminf(fmaxf(q, 0.0f), 15.0f);
+    }
+    w8hat = e4m3_roundtrip(__fmul_rn((float)(u - g.z), g.s));
+    return u;
+}
+
+__device__ __forceinline__ long long warp_sum_ll(long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// One warp per row, 8 rows per CTA; block `b` = processing positions [128 b, 128 b + 128).
+// Lane l owns positions l, l + 32, l + 64, l + 96 of the block.  The block of U (128 x 128) is
+// staged in shared memory for the whole CTA.
+__global__ void __launch_bounds__(256)
+dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const int32_t* __restrict__ perm,
+                 int64_t N, int64_t K, int b, int symmetric, int mse_steps, int per_channel,
+                 const float* __restrict__ s_w, uint8_t* __restrict__ codes, uint16_t* __restrict__ gscale,
+                 uint8_t* __restrict__ gzero, float* __restrict__ err) {
+    extern __shared__ float u_s[];  // [128][128] block of U, then 8 x 128 bytes of code staging
+    uint8_t* code_s = reinterpret_cast<uint8_t*>(u_s + 128 * 128);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t p0 = (int64_t)b * 128;
+    for (int i = threadIdx.x; i < 128 * 128; i += 256) {
+        const int q = i >> 7, v = i & 127;
+        u_s[i] = (v >= q) ? U[(p0 + q) * K + p0 + v] : 0.0f;
+    }
+    __syncthreads();
+    const int64_t n = (int64_t)blockIdx.x * 8 + warp;
+    if (n >= N) return;
+    const int64_t G = K >> 7;
+    const float sw = per_channel ? s_w[n] : s_w[0];
+    float* wrow = work + n * K + p0;
+    float w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w[i] = wrow[lane + 32 * i];
+
+    // Eq. 7 on the group's current weights, then Eq. 8 (once per group)
+    float w8[4];
+    float lo = 0.0f, hi = 0.0f, amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        w8[i] = e4m3_roundtrip(__fdiv_rn(w[i], sw));
+        lo = fminf(lo, w8[i]);
+        hi = fmaxf(hi, w8[i]);
+        amax = fmaxf(amax, fabsf(w8[i]));
+    }
+    lo = warp_min(lo);
+    hi = warp_max(hi);
+    amax = warp_max(amax);
+    DpqGroup grp = dpq_group_params(lo, hi, amax, 1.0f, symmetric);
+    if (mse_steps > 1) {
+        // Sec. 3.3: least squared error over the group among shrunk ranges; exact integer sums
+        long long best = -1;
+        for (int t = 0; t < mse_steps; ++t) {
+            const float pt = __fsub_rn(1.0f, __fmul_rn((float)t, 0.02f));
+            const DpqGroup gt = dpq_group_params(lo, hi, amax, pt, symmetric);
+            long long e2 = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float h;
+                (void)dpq_quant_dequant(w8[i], gt, symmetric, h);
+                const long long d = (long long)__fmul_rn(__fsub_rn(w8[i], h), 512.0f);
+                e2 += d * d;
+            }
+            e2 = warp_sum_ll(e2);
+            if (best < 0 || e2 < best) {
+                best = e2;
+                grp = gt;
+            }
+        }
+    }
+
+    // the 128 columns in sequence; every lane follows the same scalar computation
+    const int64_t og = perm ? (int64_t)(perm[p0] >> 7) : (int64_t)b;
+    float* erow = err + n * 128;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll 4
+        for (int o = 0; o < 32; ++o) {
+            const int q = 32 * i + o;
+            const float wq = __shfl_sync(0xFFFFFFFFu, w[i], o);
+            const float wq8 = e4m3_roundtrip(__fdiv_rn(wq, sw));         // Eq. 7
+            float h8;
+            const int u = dpq_quant_dequant(wq8, grp, symmetric, h8);    // Eq. 9, Eq. 10
+            const float h16 = __fmul_rn(h8, sw);                         // Eq. 11
+            const float e = __fdiv_rn(__fsub_rn(wq, h16), u_s[q * 128 + q]);
+            const float* urow = u_s + q * 128;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int v = lane + 32 * k;
+                if (v > q) w[k] = __fmaf_rn(-e, urow[v], w[k]);          // Eq. 12
+            }
+            if (lane == o) {
+                erow[q] = e;
+                const int c = perm ? (perm[p0 + q] & 127) : q;  // column inside its original group
+                code_s[warp * 128 + c] = (uint8_t)u;
+            }
+        }
+    }
+    __syncwarp();
+    // codes of the group, original order, two per byte (even column in the low nibble)
+    {
+        const uint8_t* cs = code_s + warp * 128 + lane * 4;
+        const uint16_t packed = (uint16_t)(cs[0] | (cs[1] << 4) | (cs[2] << 8) | (cs[3] << 12));
+        *reinterpret_cast<uint16_t*>(codes + n * (K >> 1) + og * 64 + lane * 2) = packed;
+    }
+    if (lane == 0) {
+        gscale[n * G + og] = __bfloat16_as_ushort(__float2bfloat16_rn(grp.s));
+        if (gzero) gzero[n * G + og] = (uint8_t)grp.z;
+    }
+}
+
+// Columns to the right of block b: w[n][v] <- fma(-e[n][q], U[128 b + q][v], w[n][v]), q = 0..127
+// in order.  CTA = 256 columns x 16 rows; a thread owns one column and keeps 16 rows in registers.
+__global__ void __launch_bounds__(256)
+dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const float* __restrict__ err,
+                    int64_t N, int64_t K, int b) {
+    __shared__ float e_s[16][128];
+    const int64_t p0 = (int64_t)b * 128;
+    const int64_t v = p0 + 128 + (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t n0 = (int64_t)blockIdx.y * 16;
+    for (int i = threadIdx.x; i < 16 * 128; i += 256) {
+        const int r = i >> 7, q = i & 127;
+        e_s[r][q] = (n0 + r < N) ? err[(n0 + r) * 128 + q] : 0.0f;
+    }
+    __syncthreads();
+    if (v >= K) return;
+    float w[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) w[r] = (n0 + r < N) ? work[(n0 + r) * K + v] : 0.0f;
+    const float* up = U + p0 * K + v;
+#pragma unroll 4
+    for (int q = 0; q < 128; ++q) {
+        const float uq = __ldg(up + (int64_t)q * K);
+#pragma unroll
+        for (int r = 0; r < 16; ++r) w[r] = __fmaf_rn(-e_s[r][q], uq, w[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r)
+        if (n0 + r < N) work[(n0 + r) * K + v] = w[r];
+}
+
+}  // namespace w4a8

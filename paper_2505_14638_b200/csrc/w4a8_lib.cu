@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "../../include/w4a8.h"
+#include "w4a8_dpq_kernels.cuh"
 #include "w4a8_linear_splitn.cuh"
 #include "w4a8_linear_streamk.cuh"
 #include "w4a8_linear_umma.cuh"
@@ -695,6 +696,92 @@ int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, in
     rtn_quant_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(W, N, K, symmetric, pow2, per_channel, s_w, codes,
                                                                   static_cast<uint16_t*>(gscale_bf16), gzero);
     g_launches.fetch_add(3, std::memory_order_relaxed);
+    return launch_status();
+}
+
+size_t w4a8_gar_workspace_bytes(int64_t K) {
+    if (K <= 0 || K % kGroup != 0) return 0;
+    return (size_t)K * sizeof(int32_t) + (size_t)(K / kGroup) * sizeof(float);
+}
+
+int w4a8_gar_permutation(const float* hdiag, int64_t K, int group, int32_t* perm, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+    if (!hdiag || !perm) return W4A8_ERR_INVALID_ARG;
+    if (K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0 || K > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+    if (!workspace || workspace_bytes < w4a8_gar_workspace_bytes(K)) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if ((reinterpret_cast<uintptr_t>(hdiag) & 3u) || (reinterpret_cast<uintptr_t>(perm) & 3u) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int G = (int)(K / kGroup);
+    int32_t* within = static_cast<int32_t*>(workspace);
+    float* gmax = reinterpret_cast<float*>(within + K);
+    gar_within_kernel<<<(unsigned)G, 128, 0, st>>>(hdiag, within, gmax);
+    gar_order_kernel<<<(unsigned)G, 128, 0, st>>>(within, gmax, G, perm);
+    g_launches.fetch_add(2, std::memory_order_relaxed);
+    return launch_status();
+}
+
+size_t w4a8_dpq_workspace_bytes(int64_t N, int64_t K) {
+    if (N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    return ((size_t)N * (size_t)K + (size_t)N * 128) * sizeof(float);
+}
+
+int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const float* U, const int32_t* perm,
+                      int symmetric, int mse_steps, int per_channel, uint8_t* codes, void* gscale_bf16,
+                      uint8_t* gzero, float* s_w, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!W || !U || !codes || !gscale_bf16 || !s_w) return W4A8_ERR_INVALID_ARG;
+    if (!symmetric && !gzero) return W4A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0 || mse_steps < 0 || mse_steps > 11) return W4A8_ERR_INVALID_ARG;
+    if (group != kGroup || K % kGroup != 0) return W4A8_ERR_BAD_SHAPE;
+    if (!workspace || workspace_bytes < w4a8_dpq_workspace_bytes(N, K)) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if (!aligned16(W) || !aligned16(codes) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(U) & 3u) ||
+        (reinterpret_cast<uintptr_t>(perm) & 3u) || (reinterpret_cast<uintptr_t>(gscale_bf16) & 1u) ||
+        (reinterpret_cast<uintptr_t>(s_w) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    constexpr int kBlockSmem = 128 * 128 * 4 + 8 * 128;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(dpq_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBlockSmem);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    // Eq. 6
+    unsigned int* amax_bits = reinterpret_cast<unsigned int*>(s_w);
+    if (per_channel) {
+        absmax_f32_kernel<<<(unsigned)N, 256, 0, st>>>(W, N, K, 1, amax_bits);
+    } else {
+        if (cudaMemsetAsync(s_w, 0, sizeof(float), st) != cudaSuccess) return W4A8_ERR_CUDA;
+        int64_t total = N * K;
+        unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+        absmax_f32_kernel<<<blocks, 256, 0, st>>>(W, N, K, 0, amax_bits);
+    }
+    int64_t ns = per_channel ? N : 1;
+    amax_to_scale_kernel<<<(unsigned)((ns + 255) / 256), 256, 0, st>>>(s_w, ns);
+    float* work = static_cast<float*>(workspace);
+    float* err = work + N * K;
+    dpq_gather_kernel<<<(unsigned)((N * K + 255) / 256), 256, 0, st>>>(W, perm, N, K, work);
+    uint64_t launches = 3;
+    const int G = (int)(K / kGroup);
+    for (int b = 0; b < G; ++b) {
+        dpq_block_kernel<<<(unsigned)((N + 7) / 8), 256, kBlockSmem, st>>>(
+            work, U, perm, N, K, b, symmetric, mse_steps, per_channel, s_w, codes,
+            static_cast<uint16_t*>(gscale_bf16), gzero, err);
+        ++launches;
+        const int64_t rest = K - ((int64_t)b + 1) * 128;
+        if (rest > 0) {
+            dim3 grid((unsigned)((rest + 255) / 256), (unsigned)((N + 15) / 16));
+            dpq_trailing_kernel<<<grid, 256, 0, st>>>(work, U, err, N, K, b);
+            ++launches;
+        }
+    }
+    g_launches.fetch_add(launches, std::memory_order_relaxed);
     return launch_status();
 }
 

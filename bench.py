@@ -641,6 +641,52 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
     return out
 
 
+def dpq_sweep(torch, binding, inputs, dev):
+    """Offline DPQ quantizer (Algorithm 1 with Group-Aware Reordering and an 6-step scale search)
+    on Llama-3-8B layer shapes: device time of w4a8_dpq_quantize against the plain-ALU roofline of
+    its N K^2 / 2 dependent fused multiply-adds (Eq. 12), the oracle timed on a slab of rows."""
+    import oracle
+    rows = []
+    fma_peak = 148 * 128 * 1.965e9      # FP32 FMA lanes x SMs x max SM clock
+    for name, k, n in (("o", 4096, 4096), ("gate_up", 4096, 28672), ("down", 14336, 4096)):
+        W = torch.from_numpy(inputs.make_weight(n, k, SIGMA, seed=9000)).to(dev)
+        xb = inputs.make_activation(1024, k, 9001, OUTLIER_FRAC, OUTLIER_MULT)
+        X = torch.from_numpy(inputs.bf16_bits_to_f32(xb)).to(dev).to(torch.float64)
+        X += 0.5 * torch.randn((1024, 1), dtype=torch.float64, device=dev)
+        t0 = time.perf_counter()
+        H = X.T @ X
+        perm = binding.gar_permutation(torch.diagonal(H).to(torch.float32).contiguous())
+        U = binding.hessian_upper_cholesky(H, perm)
+        torch.cuda.synchronize()
+        t_prep = time.perf_counter() - t0
+        binding.dpq_quantize(W, U, perm, symmetric=False, mse_steps=6)   # warm-up
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        q = binding.dpq_quantize(W, U, perm, symmetric=False, mse_steps=6)
+        b.record()
+        torch.cuda.synchronize()
+        t = a.elapsed_time(b) * 1e-3
+        fmas = n * k * (k - 128) / 2.0 + n * k * 64.0      # trailing updates + updates inside the blocks
+        # the oracle on a slab of rows (rows are independent), same U and order
+        # (the slab holds the row with the tensor's absolute maximum, so that Eq. 6 gives both the same s_w)
+        top = int(torch.argmax(W.abs().amax(dim=1)))
+        ridx = torch.unique(torch.cat([torch.arange(63, device=dev), torch.tensor([top], device=dev)]))
+        slab = int(ridx.numel())
+        Wh, Uh, ph = W[ridx].cpu().numpy(), U.cpu().numpy(), perm.cpu().numpy()
+        c0 = time.perf_counter()
+        ref = oracle.dpq_quantize(Wh, Uh, ph, symmetric=False, mse_steps=6)
+        t_cpu = time.perf_counter() - c0
+        same = bool(np.array_equal(q[0][ridx].cpu().numpy(), ref[0]))
+        rows.append({"layer": name, "K": k, "N": n, "dpq_ms": t * 1e3, "fma_per_s": fmas / t,
+                     "frac_of_fp32_fma_peak": fmas / t / fma_peak, "hessian_and_factor_s": t_prep,
+                     "oracle_slab_rows": slab, "oracle_slab_s": t_cpu, "oracle_full_layer_s_extrapolated":
+                         t_cpu * n / slab, "oracle_cores": oracle.num_threads(), "slab_codes_equal": same})
+        del W, X, H, U, q
+        torch.cuda.empty_cache()
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -654,7 +700,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
-    ap.add_argument("--sweep", default=None, choices=["c5", "c4"],
+    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq"],
                     help="instead of the bench line, print the per-layer table of config c5 (four Llama-3-8B "
                          "linears x M) or the single c4 case (M=8192, K=8192, N=28672)")
     args = ap.parse_args()
@@ -671,7 +717,9 @@ def main():
         _build.build()
         torch.cuda.set_device(local_rank)
         dev = torch.device("cuda", local_rank)
-        if args.sweep == "c5":
+        if args.sweep == "dpq":
+            rows = dpq_sweep(torch, binding, inputs, dev)
+        elif args.sweep == "c5":
             rows = layer_sweep(torch, binding, inputs, dev, load_peaks())
         else:
             rows = layer_sweep(torch, binding, inputs, dev, load_peaks(), layers=(("c4", 8192, 28672),), ms=(8192,))

@@ -217,13 +217,13 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
 __global__ void __launch_bounds__(256)
 dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const float* __restrict__ err,
                     int64_t N, int64_t K, int b) {
-    __shared__ float e_s[16][128];
+    __shared__ float4 e_s[128][4];  // [q][row / 4]: the 16 rows' errors of one q in four 16-byte loads
     const int64_t p0 = (int64_t)b * 128;
     const int64_t v = p0 + 128 + (int64_t)blockIdx.x * 256 + threadIdx.x;
     const int64_t n0 = (int64_t)blockIdx.y * 16;
     for (int i = threadIdx.x; i < 16 * 128; i += 256) {
         const int r = i >> 7, q = i & 127;
-        e_s[r][q] = (n0 + r < N) ? err[(n0 + r) * 128 + q] : 0.0f;
+        reinterpret_cast<float*>(&e_s[q][0])[r] = (n0 + r < N) ? -err[(n0 + r) * 128 + q] : 0.0f;  // -e, exact
     }
     __syncthreads();
     if (v >= K) return;
@@ -235,7 +235,13 @@ dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const
     for (int q = 0; q < 128; ++q) {
         const float uq = __ldg(up + (int64_t)q * K);
 #pragma unroll
-        for (int r = 0; r < 16; ++r) w[r] = __fmaf_rn(-e_s[r][q], uq, w[r]);
+        for (int r4 = 0; r4 < 4; ++r4) {
+            const float4 e = e_s[q][r4];
+            w[4 * r4 + 0] = __fmaf_rn(e.x, uq, w[4 * r4 + 0]);
+            w[4 * r4 + 1] = __fmaf_rn(e.y, uq, w[4 * r4 + 1]);
+            w[4 * r4 + 2] = __fmaf_rn(e.z, uq, w[4 * r4 + 2]);
+            w[4 * r4 + 3] = __fmaf_rn(e.w, uq, w[4 * r4 + 3]);
+        }
     }
 #pragma unroll
     for (int r = 0; r < 16; ++r)

@@ -605,6 +605,7 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
             tws.append(binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True)))
             del W
         wb = torch.randn((n, k), dtype=torch.bfloat16, device=dev) if with_cublas else None
+        w8b = wb.to(torch.float8_e4m3fn) if with_cublas else None
         for m in ms:
             xb = inputs.make_activation(m, k, 7000 + m, OUTLIER_FRAC, OUTLIER_MULT)
             x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -632,9 +633,19 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
                    "bound": "hbm" if linear_algorithmic_bytes(m, n, k) / hbm > flops / fp8_peak else "tensor"}
             if with_cublas:
                 row["cublas_bf16_us"] = graph_time(lambda c: torch.matmul(x, wb.t()), 4) * 1e6
+                # W8A8 with the library's FP8 GEMM (FP8 weights read as they are: twice the bytes, no
+                # expansion): the same-box counterpart of the paper's W8A8 comparison
+                try:
+                    a8 = x.to(torch.float8_e4m3fn)
+                    one = torch.ones((), device=dev, dtype=torch.float32)
+                    row["library_w8a8_fp8_us"] = graph_time(
+                        lambda c: torch._scaled_mm(a8, w8b.t(), scale_a=one, scale_b=one,
+                                                   out_dtype=torch.bfloat16), 4) * 1e6
+                except Exception:
+                    row["library_w8a8_fp8_us"] = None
             out.append(row)
             del x, x8, s_x, y, ws
-        del tws, wb
+        del tws, wb, w8b
         torch.cuda.empty_cache()
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set during the sweep")

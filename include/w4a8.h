@@ -102,7 +102,9 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * gscale_bf16 / gzero) or a tiled format (weights = buffer written by w4a8_prepack_weight;
  * gscale_bf16 and gzero are ignored and may be NULL).
  * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs (they are
- * added in a fixed order: results repeat bit for bit); it
+ * added in a fixed order: results repeat bit for bit).  Decode-sized calls (M <= 64) on tiled
+ * weights use it only for layers with few output channels and run without it, somewhat slower,
+ * when it is NULL or too small; larger M requires it.  It
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
  * its first use; every call leaves it ready for the next one.  Calls that share a workspace

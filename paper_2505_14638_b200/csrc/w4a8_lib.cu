@@ -282,13 +282,35 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
 }
 
 // Row partition and ring sizes of the split-N kernel for the current device.
+// Workspace of the split-N kernel when it cuts K (bytes; fits any SM count up to kMaxSMs and 64 tokens).
+constexpr size_t kSnCounterBytes = 1024;
+constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + (size_t)kMaxSMs * 64 * 128 * sizeof(float);
+
 template <class Cfg>
-static bool make_sn_plan(int64_t N, int64_t K, int sms, SnPlan* pl) {
+static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan* pl) {
     const int64_t NU = N / 8;
+    const int64_t KB = K / 128;
     int64_t P = sms < NU ? sms : NU;
     int64_t per = (NU + 32 * P - 1) / (32 * P);  // ranges per CTA so that none exceeds 256 rows
     pl->T = (int)(P * per);
-    const int rmax = (int)((NU + pl->T - 1) / pl->T) * 8;
+    pl->KSPLIT = 1;
+    // Few output channels (at most half as many 128-row blocks as SMs): ranges of whole 128-row
+    // blocks, and the K range cut in chunks so that every SM gets a tile.  A CTA's MMA and
+    // expansion work then covers 128 useful rows instead of a sliver, and its K walk is shorter;
+    // the price is a small fix-up through the workspace.
+    const int64_t blocks128 = (N + 127) / 128;
+    // (With 64-token tiles the partial sums are four times larger: only worth it for a long K.)
+    if (may_split_k && blocks128 * 2 <= sms && KB >= (Cfg::MT > 16 ? 64 : 8)) {
+        int64_t ks = sms / blocks128;
+        if (ks > KB / 4) ks = KB / 4;  // at least four k-blocks per chunk
+        if (ks > 1 && blocks128 <= (int64_t)(kSnCounterBytes / sizeof(unsigned int)) &&
+            blocks128 * ks <= kMaxSMs) {
+            pl->KSPLIT = (int)ks;
+            pl->T = (int)(blocks128 * ks);
+        }
+    }
+    const int64_t TR = pl->T / pl->KSPLIT;
+    const int rmax = (int)((NU + TR - 1) / TR) * 8;
     pl->MBLK = rmax > 128 ? 2 : 1;
     pl->KS = Cfg::kItems / pl->MBLK;
     if ((int64_t)pl->KS > K / 128) pl->KS = 1;
@@ -305,9 +327,36 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, SnPlan* pl) {
 }
 
 template <class Cfg>
-static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
-                         int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, cudaStream_t st,
-                         const SnFuse& fuse = SnFuse{}) {
+static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
+                                 int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
+                                 cudaStream_t st, const SnFuse& fuse, void* workspace, const SnPlan& pl, int sms);
+
+template <int MT, int G, int FMT, bool FUSE = false>
+static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
+                             int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, cudaStream_t st,
+                             const SnFuse& fuse = SnFuse{}, void* workspace = nullptr, size_t workspace_bytes = 0) {
+    using Cfg = SnCfg<MT, G, FMT, FUSE, false>;
+    const int sms = sm_count();
+    if (sms <= 0) return W4A8_ERR_CUDA;
+    SnPlan pl;
+    // K is cut only when the caller gave the (zero-initialised) workspace for the partial sums
+    const bool may_split_k = !FUSE && workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes &&
+                             aligned16(workspace);
+    if (!make_sn_plan<Cfg>(N, K, sms, may_split_k, &pl)) return W4A8_ERR_BAD_SHAPE;
+    if constexpr (!FUSE) {
+        if (pl.KSPLIT > 1)
+            return launch_splitn_planned<SnCfg<MT, G, FMT, false, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                         out_dtype, M, N, K, st, fuse, workspace, pl,
+                                                                         sms);
+    }
+    return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, fuse, workspace,
+                                      pl, sms);
+}
+
+template <class Cfg>
+static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
+                                 int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
+                                 cudaStream_t st, const SnFuse& fuse, void* workspace, const SnPlan& pl, int sms) {
     auto kern = linear_splitn_kernel<Cfg>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -316,11 +365,10 @@ static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float*
     });
     if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
     unsigned int* status = status_word_ptr();
-    const int sms = sm_count();
-    if (!status || sms <= 0) return W4A8_ERR_CUDA;
-    SnPlan pl;
-    if (!make_sn_plan<Cfg>(N, K, sms, &pl)) return W4A8_ERR_BAD_SHAPE;
+    if (!status) return W4A8_ERR_CUDA;
     const int P = pl.T < sms ? pl.T : sms;
+    unsigned int* counters = static_cast<unsigned int*>(workspace);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kSnCounterBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)P);
     cfg.blockDim = dim3(Cfg::kThreads);
@@ -332,7 +380,7 @@ static int launch_splitn(const CUtensorMap& tx, const uint8_t* wpp, const float*
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, pl,
-                                       fuse, status);
+                                       fuse, counters, partials, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
@@ -351,15 +399,17 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
             return W4A8_ERR_CUDA;
         const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
         if (fmt == kFmtTiledSignMag) {
-            return mt == 16 ? launch_splitn<SnCfg<16, 2, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                            out_dtype, Mi, Ni, Ki, st)
-                            : launch_splitn<SnCfg<64, 4, kFmtTiledSignMag>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                            out_dtype, Mi, Ni, Ki, st);
+            return mt == 16 ? launch_splitn_cfg<16, 2, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                            out_dtype, Mi, Ni, Ki, st, SnFuse{},
+                                                                            workspace, workspace_bytes)
+                            : launch_splitn_cfg<64, 4, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                            out_dtype, Mi, Ni, Ki, st, SnFuse{},
+                                                                            workspace, workspace_bytes);
         }
-        return mt == 16 ? launch_splitn<SnCfg<16, 2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
-                                                                 Ni, Ki, st)
-                        : launch_splitn<SnCfg<64, 4, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
-                                                                 Ni, Ki, st);
+        return mt == 16 ? launch_splitn_cfg<16, 2, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+                                                                 Ni, Ki, st, SnFuse{}, workspace, workspace_bytes)
+                        : launch_splitn_cfg<64, 4, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
+                                                                 Ni, Ki, st, SnFuse{}, workspace, workspace_bytes);
     }
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
     SkPlan pl;
@@ -496,9 +546,9 @@ static int linear_fused_impl(const void* x, int64_t ldx, int64_t M, int scale_mo
     memset(&unused, 0, sizeof(unused));
     const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
     if (fmt == kFmtTiledSignMag)
-        return launch_splitn<SnCfg<16, 2, kFmtTiledSignMag, true>>(unused, wpp, nullptr, s_w, sw_stride, y, ldy,
+        return launch_splitn_cfg<16, 2, kFmtTiledSignMag, true>(unused, wpp, nullptr, s_w, sw_stride, y, ldy,
                                                                    out_dtype, Mi, Ni, Ki, st, fuse);
-    return launch_splitn<SnCfg<16, 2, kFmtTiled, true>>(unused, wpp, nullptr, s_w, sw_stride, y, ldy, out_dtype, Mi,
+    return launch_splitn_cfg<16, 2, kFmtTiled, true>(unused, wpp, nullptr, s_w, sw_stride, y, ldy, out_dtype, Mi,
                                                         Ni, Ki, st, fuse);
 }
 
@@ -589,7 +639,7 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
     if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
     if (weight_format == kFmtCanonical) return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
-    if (M <= kSplitNMaxM) return 0;  // the split-N kernel needs none
+    if (M <= kSplitNMaxM) return kSnWorkspaceBytes;  // used when the layer has few output channels and K is cut
     SkPlan pl;
     make_sk_plan(M, N, K, kNominalSMs, &pl);
     return pl.workspace_bytes;

@@ -36,8 +36,11 @@ namespace w4a8 {
 
 
 
-template <int MT_, int G_, int FMT_, bool FUSE_ = false>
+template <int MT_, int G_, int FMT_, bool FUSE_ = false, bool SPLITK_ = false>
 struct SnCfg {
+    // SPLITK: the K range may be cut in chunks (layers with few output channels); otherwise the
+    // chunk arithmetic is compiled out.
+    static constexpr bool SPLITK = SPLITK_;
     // FUSE: the kernel takes BF16 activations and does the per-token FP8 quantization (Eq. 13)
     // itself: an absmax pass over X before the main loop (overlapped with the first weight copies)
     // and a convert step that writes each stage's FP8 activation tile into shared memory, in the
@@ -64,8 +67,9 @@ struct SnCfg {
     static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : 200 * 1024;
     static_assert(MT == 16 || MT == 64, "token tile");
     static_assert(kDCol + 2 * MT <= kTmemCols, "tensor memory columns");
-    static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 + 3 * 64 <= kBarBytes, "barrier area");
+    static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 + 3 * 64 + 16 <= kBarBytes, "barrier area");
     static_assert(!FUSE_ || MT_ == 16, "the fused activation quantization is built for <= 16 tokens");
+    static_assert(!(FUSE_ && SPLITK_), "the fused launch has no workspace and never cuts K");
 };
 
 constexpr int kFuseFewTokens = 4;
@@ -100,7 +104,8 @@ __device__ __forceinline__ XMap x_map(int r, int M, int S1) {
 
 // Launch-time plan shared by host and device.
 struct SnPlan {
-    int T;         // number of row ranges (tiles); range t covers 8-row units [t*NU/T, (t+1)*NU/T)
+    int T;         // number of tiles = row ranges x K chunks; tile t = (row range t / KSPLIT, K chunk t % KSPLIT)
+    int KSPLIT;    // K chunks per row range (1 = every CTA walks the whole K; > 1 needs the workspace)
     int MBLK;      // 128-row blocks per range (1 or 2)
     int KS;        // k-blocks per pipeline stage (KS * MBLK == 2)
     int S1;        // depth of the TMA ring (>= kS2)
@@ -121,13 +126,75 @@ struct SnFuse {
     float* s_x_out;
 };
 
+// Epilogue of the split-N kernel: scales 16 tokens of accumulated sums (row r of 128-row block b,
+// tokens c0..c0+15) with Eq. 4 / Eq. 11 and writes them to Y, through the staging area in 16-byte
+// pieces when the rows of Y are 16-byte aligned.  Called by all 128 epilogue threads together.
+template <class Cfg>
+__device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, int b, int c0, int r, int et, int R,
+                                        int n0, int M, int es, bool wide_out, uint32_t out_s, void* y, int64_t ldy,
+                                        const float (&sx_lane)[Cfg::MT / 32 > 0 ? Cfg::MT / 32 : 1],
+                                        const float* sx_s) {
+    constexpr int MT = Cfg::MT;
+
+    const int row = b * 128 + r;
+    const bool row_ok = row < R;
+    const int n = n0 + row;
+    float sxv = sx_lane[0];
+    if (MT > 32 && c0 >= 32) sxv = sx_lane[MT / 32 - 1];
+    float res[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float sxm = Cfg::FUSE ? sx_s[c0 + j] : __shfl_sync(0xFFFFFFFFu, sxv, (c0 & 16) + j);
+        res[j] = __uint_as_float(accv[j]) * (sxm * swb);  // Eq. 4, Eq. 11
+    }
+    if (wide_out) {
+        // tokens x rows into the staging area, then 16-byte pieces of Y rows
+        const uint32_t pitch = 128u * (uint32_t)es;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const uint32_t a = out_s + (uint32_t)j * pitch + (uint32_t)(r * es);
+            if (es == 4)
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[j]) : "memory");
+            else
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
+                             "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[j])))
+                             : "memory");
+        }
+        asm volatile("bar.sync 3, 128;" ::: "memory");
+        const int Rb = (R - b * 128) < 128 ? (R - b * 128) : 128;
+        const int ppt = (Rb * es) >> 4;  // 16-byte pieces per token (rows come in eights)
+        const int ntok = (M - c0) < 16 ? (M - c0) : 16;
+        char* yb = static_cast<char*>(y) + ((int64_t)c0 * ldy + n0 + b * 128) * es;
+        for (int id = et; id < ntok * ppt; id += 128) {
+            const int tok = id / ppt, piece = id - tok * ppt;
+            uint4 w;
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                         : "r"(out_s + (uint32_t)tok * pitch + (uint32_t)(piece << 4)));
+            *reinterpret_cast<uint4*>(yb + (int64_t)tok * ldy * es + (piece << 4)) = w;
+        }
+        asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int m = c0 + j;
+            if (m < M && row_ok) {
+                if (es == 4)
+                    reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res[j];
+                else
+                    reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] = __float2bfloat16_rn(res[j]);
+            }
+        }
+    }
+}
+
 template <class Cfg>
 __global__ void __launch_bounds__(Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
 linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x MT, 128B swizzle
                      const uint8_t* __restrict__ wpp, const float* __restrict__ s_x,
                      const float* __restrict__ s_w, int sw_stride, void* __restrict__ y, int64_t ldy,
                      int out_dtype, int M, int N, int K, const SnPlan plan, const SnFuse fuse,
-                     unsigned int* status_word) {
+                     unsigned int* counters, float* partials, unsigned int* status_word) {
     constexpr int MT = Cfg::MT, G = Cfg::G, S2 = Cfg::kS2, MB = Cfg::kMeta;
     constexpr int S1M = Cfg::kS1Max;
     extern __shared__ uint8_t smem_raw[];
@@ -155,12 +222,34 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     unsigned int* amax_s = const_cast<unsigned int*>(tmem_slot) + 4;  // [16] row absmax bit patterns
     float* sx_s = reinterpret_cast<float*>(amax_s + 16);              // [16] activation scales s_x
     float* inv_s = sx_s + 16;                                         // [16] multipliers 1/s_x
+    volatile unsigned int* ticket_s = reinterpret_cast<volatile unsigned int*>(inv_s + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = K >> 7;
     const int64_t NU = N >> 3;           // the row partition works in units of 8 rows
-    const int nst = (KB + KS - 1) / KS;  // stages per tile
     const int P = gridDim.x, p = blockIdx.x;
+    const int KSPLIT = Cfg::SPLITK ? plan.KSPLIT : 1, TR = T / KSPLIT;
+    // Tile t: 8-row units [u0, u1) of row range t / KSPLIT, k-blocks [kb0, kb0 + nkb) of chunk t % KSPLIT.
+    const int nst_all = (KB + KS - 1) / KS;  // stages per tile when K is not cut
+    struct TileGeom {
+        int u0, u1, kb0, nkb;
+    };
+    auto tile_geom = [&](int t) {
+        TileGeom g;
+        if constexpr (!Cfg::SPLITK) {
+            g.u0 = (int)((int64_t)t * NU / T);
+            g.u1 = (int)((int64_t)(t + 1) * NU / T);
+            g.kb0 = 0;
+            g.nkb = KB;
+        } else {
+            const int rt = t / KSPLIT, kc = t - rt * KSPLIT;
+            g.u0 = (int)((int64_t)rt * NU / TR);
+            g.u1 = (int)((int64_t)(rt + 1) * NU / TR);
+            g.kb0 = (int)((int64_t)kc * KB / KSPLIT);
+            g.nkb = (int)((int64_t)(kc + 1) * KB / KSPLIT) - g.kb0;
+        }
+        return g;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S1; ++s) {
@@ -284,11 +373,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             const int64_t meta_step = (int64_t)N * MB;
             const uint8_t* meta_base = wpp + (int64_t)KB * code_step;
             for (int t = p; t < T && ok; t += P) {
-                const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
+                const TileGeom tg = tile_geom(t);
+                const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
+                const int nst = Cfg::SPLITK ? (nkb + KS - 1) / KS : nst_all;
                 const int R = (u1 - u0) * 8;
                 const uint32_t cbytes = (uint32_t)(R * kRowCodeBytes), mbytes = (uint32_t)(R * MB);
-                const uint8_t* cptr = wpp + (int64_t)u0 * 8 * kRowCodeBytes;
-                const uint8_t* mptr = meta_base + (int64_t)u0 * 8 * MB;
+                const uint8_t* cptr = wpp + (int64_t)kb0 * code_step + (int64_t)u0 * 8 * kRowCodeBytes;
+                const uint8_t* mptr = meta_base + (int64_t)kb0 * meta_step + (int64_t)u0 * 8 * MB;
                 // Weights depend on no earlier kernel: issue a few stages of them before waiting
                 // for the kernel that produces the activations.
                 int ahead = S1 < 4 ? S1 : 4;  // must fit in the ring: nothing is consumed before the activations land
@@ -300,7 +391,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     const uint32_t full = bar_full0 + 8u * (uint32_t)r1.idx;
                     ok = ptx::mbar_wait(bar_free10 + 8u * (uint32_t)r1.idx, r1.phase ^ 1u, abort_flag, status_word);
                     if (!ok) break;
-                    const int ks = (KB - kb) < KS ? (KB - kb) : KS;
+                    const int ks = (nkb - kb) < KS ? (nkb - kb) : KS;
                     const uint32_t wdst = w_ring + (uint32_t)(r1.idx * plan.wstage);
                     const uint32_t mdst = wdst + (uint32_t)plan.meta_off;
                     const uint8_t* cptr1 = cptr + code_step;
@@ -327,10 +418,10 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     }
                     // activation tiles of every stage issued so far
                     while (xkb < kb) {
-                        const int ksx = (KB - xkb) < KS ? (KB - xkb) : KS;
+                        const int ksx = (nkb - xkb) < KS ? (nkb - xkb) : KS;
                         const uint32_t xdst = x_ring + (uint32_t)(rx.idx * plan.xstage);
                         const uint32_t xfull = bar_xfull0 + 8u * (uint32_t)rx.idx;
-                        const int x0 = xkb * 128;
+                        const int x0 = (kb0 + xkb) * 128;
                         if (ptx::elect_one()) {
                             ptx::mbar_arrive_expect_tx(xfull, (uint32_t)(ksx * MT * 128));
                             ptx::tma_load_2d(xdst, &tmap_x, x0, 0, xfull);
@@ -378,6 +469,9 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 first_tile = false;
                 uint32_t accumulate = 0;
                 int kb = 0;
+                const TileGeom tg = tile_geom(t);
+                const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
+                const int nst = Cfg::SPLITK ? (nkb + KS - 1) / KS : nst_all;
                 for (int st = 0; st < nst; ++st) {
                     ok = ptx::mbar_wait(bar_xfull0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
                     ok = ok && ptx::mbar_wait(bar_a_full0 + 8u * (uint32_t)r2.idx, r2.phase, abort_flag, status_word);
@@ -385,7 +479,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     ptx::tc_fence_after_sync();
                     // A stage holds two (k-block, 128-row block) items: either two k-blocks of one
                     // row block or one k-block of two row blocks.
-                    const int ks = (KB - kb) < KS ? (KB - kb) : KS;
+                    const int ks = (nkb - kb) < KS ? (nkb - kb) : KS;
                     const uint32_t b_lo = b_lo0 + (uint32_t)r1.idx * b_step;
                     const uint32_t a_col = tmem_base + (uint32_t)(r2.idx * Cfg::kAStageCols);
                     const uint32_t free_bar = bar_free10 + 8u * (uint32_t)r1.idx;
@@ -439,7 +533,9 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 sx_lane[c] = (c * 32 + lane < M) ? __ldg(s_x + c * 32 + lane) : 0.0f;
         }
         for (int t = p; t < T && ok; t += P) {
-            const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
+            const TileGeom tg = tile_geom(t);
+            const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
+            const int nst = Cfg::SPLITK ? (nkb + KS - 1) / KS : nst_all;
             const int R = (u1 - u0) * 8;
             const int n0 = u0 * 8;
             float swn[2];
@@ -516,12 +612,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             acc_phase ^= 1u;
             if (!ok) break;
             ptx::tc_fence_after_sync();
+            // With the K range cut in KSPLIT chunks the accumulator is a partial sum: it goes to the
+            // workspace (tile t, token-major), and the CTA that arrives last at the row range adds the
+            // chunks in ascending order and emits.
+            float* part = partials + (int64_t)t * (MT * 128);
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
                 if (b >= MBLK) break;
-                const int row = b * 128 + r;
-                const bool row_ok = row < R;
-                const int n = n0 + row;
 #pragma unroll 1
                 for (int c0 = 0; c0 < MT; c0 += 16) {
                     if (c0 >= M) break;  // uniform
@@ -529,55 +626,44 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     ptx::tmem_ld_32x32b_x16(
                         tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(Cfg::kDCol + b * MT + c0), v);
                     ptx::tmem_ld_wait();
-                    float sxv = sx_lane[0];
-                    if (MT > 32 && c0 >= 32) sxv = sx_lane[MT / 32 - 1];
-                    float res[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float sxm = Cfg::FUSE ? sx_s[c0 + j] : __shfl_sync(0xFFFFFFFFu, sxv, (c0 & 16) + j);
-                        res[j] = __uint_as_float(v[j]) * (sxm * swn[b]);  // Eq. 4, Eq. 11
-                    }
-                    if (wide_out) {
-                        // tokens x rows into the staging area, then 16-byte pieces of Y rows
-                        const uint32_t pitch = 128u * (uint32_t)es;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const uint32_t a = out_s + (uint32_t)j * pitch + (uint32_t)(r * es);
-                            if (es == 4)
-                                asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[j]) : "memory");
-                            else
-                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
-                                             "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[j])))
-                                             : "memory");
-                        }
-                        asm volatile("bar.sync 3, 128;" ::: "memory");
-                        const int Rb = (R - b * 128) < 128 ? (R - b * 128) : 128;
-                        const int ppt = (Rb * es) >> 4;  // 16-byte pieces per token (rows come in eights)
-                        const int ntok = (M - c0) < 16 ? (M - c0) : 16;
-                        char* yb = static_cast<char*>(y) + ((int64_t)c0 * ldy + n0 + b * 128) * es;
-                        for (int id = et; id < ntok * ppt; id += 128) {
-                            const int tok = id / ppt, piece = id - tok * ppt;
-                            uint4 w;
-                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                         : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
-                                         : "r"(out_s + (uint32_t)tok * pitch + (uint32_t)(piece << 4)));
-                            *reinterpret_cast<uint4*>(yb + (int64_t)tok * ldy * es + (piece << 4)) = w;
-                        }
-                        asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
+                    if (KSPLIT == 1) {
+                        sn_emit<Cfg>(v, swn[b], b, c0, r, et, R, n0, M, es, wide_out, out_s, y, ldy, sx_lane, sx_s);
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int m = c0 + j;
-                            if (m < M && row_ok) {
-                                if (es == 4)
-                                    reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res[j];
-                                else
-                                    reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)m * ldy + n] =
-                                        __float2bfloat16_rn(res[j]);
-                            }
-                        }
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < M) __stcg(part + (c0 + j) * 128 + r, __uint_as_float(v[j]));
                     }
                 }
+            }
+            if (KSPLIT > 1) {
+                const int rt = t / KSPLIT;
+                __threadfence();
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (et == 0) *ticket_s = atomicAdd(counters + rt, 1u);
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (*ticket_s == (unsigned int)(KSPLIT - 1)) {
+                    __threadfence();
+                    const float* p0 = partials + (int64_t)rt * KSPLIT * (MT * 128);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < MT; c0 += 16) {
+                        if (c0 >= M) break;  // uniform
+                        float accv[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) accv[j] = 0.0f;
+                        for (int kc = 0; kc < KSPLIT; ++kc) {
+                            const float* pp = p0 + (int64_t)kc * (MT * 128) + c0 * 128 + r;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + j < M) accv[j] += __ldcg(pp + j * 128);
+                        }
+                        uint32_t accu[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) accu[j] = __float_as_uint(accv[j]);
+                        sn_emit<Cfg>(accu, swn[0], 0, c0, r, et, R, n0, M, es, wide_out, out_s, y, ldy, sx_lane, sx_s);
+                    }
+                    if (et == 0) counters[rt] = 0u;  // ready for the next launch
+                }
+                asm volatile("bar.sync 3, 128;" ::: "memory");  // the ticket slot is reused by the next tile
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(bar_acc_empty);
@@ -603,12 +689,14 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         int turn = g;  // stages until this group's next turn, counted across tiles
         bool ok = true;
         for (int t = p; t < T && ok; t += P) {
-            const int u0 = (int)((int64_t)t * NU / T), u1 = (int)((int64_t)(t + 1) * NU / T);
+            const TileGeom tg = tile_geom(t);
+            const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
+            const int nst = Cfg::SPLITK ? (nkb + KS - 1) / KS : nst_all;
             const int R = (u1 - u0) * 8;
             int st = turn;
             for (; st < nst; st += G) {
                 const int kb = st * KS;
-                const int ks = (KB - kb) < KS ? (KB - kb) : KS;
+                const int ks = (nkb - kb) < KS ? (nkb - kb) : KS;
                 ok = ptx::mbar_wait(bar_full0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
                 if (ok && done >= S2)
                     ok = ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rl.idx, rl.phase, abort_flag, status_word);

@@ -207,7 +207,7 @@ struct SkPlan {
     size_t counter_bytes, workspace_bytes;
 };
 
-constexpr int kSplitNMaxM = 64;  // token counts served by the split-N (decode) kernel
+constexpr int kSplitNMaxM = 128;  // token counts served by the split-N (decode) kernel
 
 // Token-tile width and schedule of the persistent kernel from a small cost model (microseconds):
 // a (tile, k-block) unit costs the larger of the dequantization of its 128 x 128 weights and its
@@ -282,9 +282,9 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
 }
 
 // Row partition and ring sizes of the split-N kernel for the current device.
-// Workspace of the split-N kernel when it cuts K (bytes; fits any SM count up to kMaxSMs and 64 tokens).
+// Workspace of the split-N kernel when it cuts K (bytes; fits any SM count up to kMaxSMs and 128 tokens).
 constexpr size_t kSnCounterBytes = 1024;
-constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + (size_t)kMaxSMs * 64 * 128 * sizeof(float);
+constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + (size_t)kMaxSMs * 128 * 128 * sizeof(float);
 
 template <class Cfg>
 static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan* pl) {
@@ -392,12 +392,20 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     if (M <= kSplitNMaxM) {
         int rc = check_device();
         if (rc != W4A8_OK) return rc;
-        const int mt = M <= 16 ? 16 : 64;
+        const int mt = M <= 16 ? 16 : (M <= 64 ? 64 : 128);
         CUtensorMap tx;
         if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)mt,
                              CU_TENSOR_MAP_SWIZZLE_128B))
             return W4A8_ERR_CUDA;
         const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+        if (mt == 128) {
+            return fmt == kFmtTiledSignMag
+                       ? launch_splitn_cfg<128, 4, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                                                     Mi, Ni, Ki, st, SnFuse{}, workspace,
+                                                                     workspace_bytes)
+                       : launch_splitn_cfg<128, 4, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi, Ni,
+                                                              Ki, st, SnFuse{}, workspace, workspace_bytes);
+        }
         if (fmt == kFmtTiledSignMag) {
             return mt == 16 ? launch_splitn_cfg<16, 2, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
                                                                             out_dtype, Mi, Ni, Ki, st, SnFuse{},

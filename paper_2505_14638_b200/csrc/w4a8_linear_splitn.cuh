@@ -50,7 +50,7 @@ struct SnCfg {
     static constexpr int G = G_;        // dequantization groups of 4 warps
     static constexpr int FMT = FMT_;
     static constexpr int kS1Max = 16;   // ring of TMA stages (runtime depth <= this)
-    static constexpr int kS2 = MT_ == 16 ? 3 : 4;  // ring of dequantized stages in tensor memory
+    static constexpr int kS2 = MT_ == 64 ? 4 : 3;  // ring of dequantized stages in tensor memory
     static constexpr int kItems = 2;    // (k-block, 128-row block) pairs per stage
     static constexpr int kMeta = meta_bytes(FMT);
     static constexpr int kTmemCols = MT_ == 16 ? 256 : 512;
@@ -64,8 +64,8 @@ struct SnCfg {
     static constexpr int kOutBytes = 16 * 128 * 4;
     // Decode-sized launches (<= 16 tokens) take half an SM each, so that the CTAs of the next
     // kernel in the stream can start -- and prefetch their weights -- while this one finishes.
-    static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : 200 * 1024;
-    static_assert(MT == 16 || MT == 64, "token tile");
+    static constexpr int kSmemBudget = MT_ == 16 ? 100 * 1024 : (MT_ == 64 ? 200 * 1024 : 220 * 1024);
+    static_assert(MT == 16 || MT == 64 || MT == 128, "token tile");
     static_assert(kDCol + 2 * MT <= kTmemCols, "tensor memory columns");
     static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 + 3 * 64 + 16 <= kBarBytes, "barrier area");
     static_assert(!FUSE_ || MT_ == 16, "the fused activation quantization is built for <= 16 tokens");
@@ -140,7 +140,9 @@ __device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, i
     const bool row_ok = row < R;
     const int n = n0 + row;
     float sxv = sx_lane[0];
-    if (MT > 32 && c0 >= 32) sxv = sx_lane[MT / 32 - 1];
+#pragma unroll
+    for (int c = 1; c < MT / 32; ++c)
+        if (c0 >= 32 * c) sxv = sx_lane[c];
     float res[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
@@ -613,8 +615,8 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             if (!ok) break;
             ptx::tc_fence_after_sync();
             // With the K range cut in KSPLIT chunks the accumulator is a partial sum: it goes to the
-            // workspace (tile t, token-major), and the CTA that arrives last at the row range adds the
-            // chunks in ascending order and emits.
+            // workspace (tile t, token-major: coalesced stores), and the CTA that arrives last at the row
+            // range adds the chunks in ascending order (after the roles have joined).
             float* part = partials + (int64_t)t * (MT * 128);
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
@@ -641,29 +643,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 asm volatile("bar.sync 3, 128;" ::: "memory");
                 if (et == 0) *ticket_s = atomicAdd(counters + rt, 1u);
                 asm volatile("bar.sync 3, 128;" ::: "memory");
-                if (*ticket_s == (unsigned int)(KSPLIT - 1)) {
-                    __threadfence();
-                    const float* p0 = partials + (int64_t)rt * KSPLIT * (MT * 128);
-#pragma unroll 1
-                    for (int c0 = 0; c0 < MT; c0 += 16) {
-                        if (c0 >= M) break;  // uniform
-                        float accv[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) accv[j] = 0.0f;
-                        for (int kc = 0; kc < KSPLIT; ++kc) {
-                            const float* pp = p0 + (int64_t)kc * (MT * 128) + c0 * 128 + r;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (c0 + j < M) accv[j] += __ldcg(pp + j * 128);
-                        }
-                        uint32_t accu[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) accu[j] = __float_as_uint(accv[j]);
-                        sn_emit<Cfg>(accu, swn[0], 0, c0, r, et, R, n0, M, es, wide_out, out_s, y, ldy, sx_lane, sx_s);
-                    }
-                    if (et == 0) counters[rt] = 0u;  // ready for the next launch
-                }
-                asm volatile("bar.sync 3, 128;" ::: "memory");  // the ticket slot is reused by the next tile
+                // (the CTA that drew the last ticket adds the chunks after the roles have joined, below)
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(bar_acc_empty);
@@ -732,6 +712,35 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+    if constexpr (Cfg::SPLITK) {
+        // K was cut: a CTA holds exactly one tile.  The CTA that arrived last at its row range adds
+        // the KSPLIT partial sums in ascending chunk order -- every thread of the CTA takes part, so
+        // that many independent loads are in flight -- scales (Eq. 4, Eq. 11) and writes Y.
+        if (KSPLIT > 1 && p < T && *ticket_s == (unsigned int)(KSPLIT - 1)) {
+            ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
+            __threadfence();
+            const int rt = p / KSPLIT;
+            const TileGeom tg = tile_geom(p);
+            const int R = (tg.u1 - tg.u0) * 8, n0 = tg.u0 * 8;
+            const float* p0 = partials + (int64_t)rt * KSPLIT * (MT * 128);
+            const int total = (M < MT ? M : MT) * 128;
+#pragma unroll 2
+            for (int e = (int)threadIdx.x; e < total; e += Cfg::kThreads) {
+                const int row = e & 127, tok = e >> 7;
+                if (row < R) {
+                    float acc = 0.0f;
+                    for (int kc = 0; kc < KSPLIT; ++kc) acc += __ldcg(p0 + (int64_t)kc * (MT * 128) + e);
+                    const int n = n0 + row;
+                    const float res = acc * (__ldg(s_x + tok) * __ldg(s_w + (int64_t)n * sw_stride));
+                    if (out_dtype == W4A8_OUT_FP32)
+                        reinterpret_cast<float*>(y)[(int64_t)tok * ldy + n] = res;
+                    else
+                        reinterpret_cast<__nv_bfloat16*>(y)[(int64_t)tok * ldy + n] = __float2bfloat16_rn(res);
+                }
+            }
+            if (threadIdx.x == 0) counters[rt] = 0u;  // ready for the next launch
+        }
     }
 }
 

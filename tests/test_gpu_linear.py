@@ -99,9 +99,10 @@ def test_gaussian_inputs_within_gates(M, N, K, asym, pc):
 
 @pytest.mark.parametrize("M,N,K", [(16, 128, 128), (1, 16, 14336), (16, 4096, 4096), (8, 6144, 4096),
                                    (32, 4096, 14336), (64, 1024, 2048), (128, 2048, 1024), (512, 1024, 1024),
-                                   (300, 640, 8192)])
+                                   (300, 640, 8192), (100, 512, 8192), (65, 4096, 4096), (128, 14336, 1024)])
 def test_persistent_kernel_split_tiles_and_reuse_of_workspace(M, N, K):
-    # shapes whose tiles are split between CTAs in many ways; the workspace is shared by
+    # shapes whose tiles are split between CTAs in many ways (equal slices in the persistent kernel, K
+    # chunks in the split-N kernel with 16-, 64- and 128-token tiles); the workspace is shared by
     # consecutive calls (the kernel leaves its counters zeroed) and results repeat bit for bit
     x8, s_x, wq = _gaussian_case(M, N, K, seed=M * 3 + N + K)
     w8 = oracle.dequant_weight(*wq[:3])
@@ -119,9 +120,8 @@ def test_persistent_kernel_split_tiles_and_reuse_of_workspace(M, N, K):
     assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
     worst, _ = fp32_gate(outs[0].cpu().numpy()[:, cols], ref["y64"])
     assert worst <= 2e-3, worst
-    bnx = next(b for b in (16, 32, 64, 128, 256) if M <= b or b == 256)
-    n_counters = ((M + bnx - 1) // bnx) * ((N + 127) // 128)
-    assert np.all(ws[: 4 * n_counters].cpu().numpy() == 0)      # tile counters are back to zero
+    n_counter_bytes = 1024 if M <= 128 else 8 * ((M + 255) // 256) * ((N + 127) // 128)
+    assert np.all(ws[:n_counter_bytes].cpu().numpy() == 0)     # tile counters are back to zero
 
 
 def test_sign_magnitude_prepack_flags_code_zero():

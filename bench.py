@@ -37,7 +37,6 @@ SWEEP_M = (1, 4, 16)
 K, N = 4096, 14336
 GROUP = 128
 SIGMA, OUTLIER_FRAC, OUTLIER_MULT = 0.02, 0.01, 20.0
-FUSED_UP_TO_M = 4           # the fused launch wins up to here (measured), the two-kernel sequence above
 WEIGHT_COPIES = 10          # 10 x 30.3 MB = 303 MB > 2 x 126 MB L2
 METRIC = "w4a8_decode_weight_stream_rate"
 UNIT = "GB/s"
@@ -277,7 +276,7 @@ def run_ours(args, rank, world, local_rank):
     def lin(m, c):
         binding.linear_tiled(x8s[m], sxs[m], weights[c % WEIGHT_COPIES], out=ys[m], workspace=workspace)
 
-    fused_m = () if args.two_kernel else tuple(m for m in SWEEP_M if m <= FUSED_UP_TO_M)
+    fused_m = () if args.two_kernel else tuple(m for m in SWEEP_M if binding.fused_is_faster(m, N, K))
     fused = bool(fused_m)
     lin_unfused = lin
 
@@ -618,7 +617,7 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
                 binding.linear_tiled(x8, s_x, tws[c % copies], out=y, workspace=ws)
 
             def whole(c):
-                if m <= FUSED_UP_TO_M:
+                if binding.fused_is_faster(m, n, k):
                     binding.linear_fused(x, tws[c % copies], out=y)
                 else:
                     binding.quantize_act(x, out=(x8, s_x))

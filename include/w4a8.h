@@ -191,6 +191,9 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
 #define W4A8_FUSED_MAX_M 16
+/* 1 when w4a8_linear_fused is the faster way to run this problem on B200 (few tokens, many
+ * output channels), 0 when w4a8_quantize_act + w4a8_linear is. */
+int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K);
 int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
                       const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
                       int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
@@ -247,7 +250,7 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
 /*
  * Whole layer from HOST activations to HOST output (Sec. 3 flow end to end): copies
  * x_host (BF16 [M][K], ideally pinned) to x_dev, runs w4a8_quantize_act and w4a8_linear (or
- * w4a8_linear_fused when the weights are prepacked and M <= 4), and
+ * w4a8_linear_fused when the weights are prepacked and w4a8_fused_is_faster says so), and
  * copies y_dev (BF16 [M][N]) to y_host, all enqueued on `stream`; the caller synchronises the
  * stream before reading y_host.  Weights stay resident on the device.  Scratch device buffers
  * are the caller's: x_dev (2*M*K bytes), x8_dev (M*K), s_x_dev (4*M), y_dev (2*M*N), workspace.

@@ -27,7 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
-    "w4a8_linear_fused",
+    "w4a8_linear_fused", "w4a8_fused_is_faster",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
@@ -71,6 +71,8 @@ def lib():
                                  i32, i32, p]
     L.w4a8_linear_static_scratch.restype = i32
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
+    L.w4a8_fused_is_faster.restype = i32
+    L.w4a8_fused_is_faster.argtypes = [i64, i64, i64]
     L.w4a8_linear_fused.restype = i32
     L.w4a8_linear_fused.argtypes = [p, i64, i64, i32, p, p, i32, p, i32, i64, i64, p, i64, i32, p, i64, p, p]
     L.w4a8_linear_ex_workspace_bytes.restype = sz
@@ -264,6 +266,11 @@ def linear_tiled(x8, s_x, tw, out_dtype=OUT_BF16, out=None, workspace=None):
 
 
 FUSED_MAX_M = 16
+
+
+def fused_is_faster(M, N, K):
+    """w4a8_fused_is_faster: whether the fused launch is the faster way to run this problem."""
+    return bool(lib().w4a8_fused_is_faster(M, N, K))
 
 
 def linear_fused(x, tw, out_dtype=OUT_BF16, out=None, scale_mode=SCALE_EXACT, static_scale=None,

@@ -711,6 +711,16 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
                        static_cast<cudaStream_t>(stream));
 }
 
+int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {
+    // Measured on B200: the fused launch wins for a few tokens on layers with many output channels;
+    // with few output channels the two-kernel path cuts K across the SMs (the fused launch, which has
+    // no workspace, cannot) and wins; above four tokens every CTA of the fused launch scans too much
+    // of X for the token scales.
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const int64_t blocks128 = (N + 127) / 128;
+    return (M <= kFuseFewTokens && blocks128 * 2 > kNominalSMs) ? 1 : 0;
+}
+
 int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
                       const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
                       int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
@@ -864,7 +874,7 @@ int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights
     int rc;
     if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
-    if (weight_format != kFmtCanonical && M <= kFuseFewTokens) {
+    if (weight_format != kFmtCanonical && w4a8_fused_is_faster(M, N, K) == 1) {
         // a few tokens and prepacked weights: one kernel quantizes the activations and multiplies
         // (measured faster than the two-kernel sequence up to here, slower above)
         rc = linear_fused_impl(x_dev, K, M, W4A8_SCALE_EXACT, nullptr, weights, weight_format, s_w, sw_stride, N, K,

@@ -110,24 +110,27 @@ __device__ __forceinline__ long long warp_sum_ll(long long v) {
     return v;
 }
 
-// One warp per row, 8 rows per CTA; block `b` = processing positions [128 b, 128 b + 128).
+// One warp per row, 16 rows per CTA (the chain of dependent divisions and conversions of one
+// column is long: many warps per SM hide it); block `b` = processing positions [128 b, 128 b + 128).
 // Lane l owns positions l, l + 32, l + 64, l + 96 of the block.  The block of U (128 x 128) is
 // staged in shared memory for the whole CTA.
-__global__ void __launch_bounds__(256)
+constexpr int kDpqRowsPerCta = 16;
+
+__global__ void __launch_bounds__(32 * kDpqRowsPerCta)
 dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const int32_t* __restrict__ perm,
                  int64_t N, int64_t K, int b, int symmetric, int mse_steps, int per_channel,
                  const float* __restrict__ s_w, uint8_t* __restrict__ codes, uint16_t* __restrict__ gscale,
                  uint8_t* __restrict__ gzero, float* __restrict__ err) {
-    extern __shared__ float u_s[];  // [128][128] block of U, then 8 x 128 bytes of code staging
+    extern __shared__ float u_s[];  // [128][128] block of U, then kDpqRowsPerCta x 128 bytes of code staging
     uint8_t* code_s = reinterpret_cast<uint8_t*>(u_s + 128 * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t p0 = (int64_t)b * 128;
-    for (int i = threadIdx.x; i < 128 * 128; i += 256) {
+    for (int i = threadIdx.x; i < 128 * 128; i += 32 * kDpqRowsPerCta) {
         const int q = i >> 7, v = i & 127;
         u_s[i] = (v >= q) ? U[(p0 + q) * K + p0 + v] : 0.0f;
     }
     __syncthreads();
-    const int64_t n = (int64_t)blockIdx.x * 8 + warp;
+    const int64_t n = (int64_t)blockIdx.x * kDpqRowsPerCta + warp;
     if (n >= N) return;
     const int64_t G = K >> 7;
     const float sw = per_channel ? s_w[n] : s_w[0];
@@ -213,39 +216,64 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
 }
 
 // Columns to the right of block b: w[n][v] <- fma(-e[n][q], U[128 b + q][v], w[n][v]), q = 0..127
-// in order.  CTA = 256 columns x 16 rows; a thread owns one column and keeps 16 rows in registers.
+// in order.  CTA = 512 columns x 16 rows; a thread owns two columns (v, v + 256) and keeps their 16
+// rows in registers, so that one q costs four 16-byte shared loads, two global loads and 32 FMAs.
 __global__ void __launch_bounds__(256)
 dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const float* __restrict__ err,
                     int64_t N, int64_t K, int b) {
     __shared__ float4 e_s[128][4];  // [q][row / 4]: the 16 rows' errors of one q in four 16-byte loads
     const int64_t p0 = (int64_t)b * 128;
-    const int64_t v = p0 + 128 + (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t v0 = p0 + 128 + (int64_t)blockIdx.x * 512 + threadIdx.x;
+    const int64_t v1 = v0 + 256;
     const int64_t n0 = (int64_t)blockIdx.y * 16;
     for (int i = threadIdx.x; i < 16 * 128; i += 256) {
         const int r = i >> 7, q = i & 127;
         reinterpret_cast<float*>(&e_s[q][0])[r] = (n0 + r < N) ? -err[(n0 + r) * 128 + q] : 0.0f;  // -e, exact
     }
     __syncthreads();
-    if (v >= K) return;
-    float w[16];
+    if (v0 >= K) return;
+    const bool two = v1 < K;
+    float w0[16], w1[16];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) w[r] = (n0 + r < N) ? work[(n0 + r) * K + v] : 0.0f;
-    const float* up = U + p0 * K + v;
-#pragma unroll 4
-    for (int q = 0; q < 128; ++q) {
-        const float uq = __ldg(up + (int64_t)q * K);
+    for (int r = 0; r < 16; ++r) {
+        w0[r] = (n0 + r < N) ? work[(n0 + r) * K + v0] : 0.0f;
+        w1[r] = (two && n0 + r < N) ? work[(n0 + r) * K + v1] : 0.0f;
+    }
+    const float* up = U + p0 * K;
+#pragma unroll 1
+    for (int q8 = 0; q8 < 128; q8 += 8) {
+        // eight rows of U at a time: sixteen loads in flight per thread hide the L2 latency
+        float ua[8], ub[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            ua[i] = __ldg(up + (int64_t)(q8 + i) * K + v0);
+            ub[i] = two ? __ldg(up + (int64_t)(q8 + i) * K + v1) : 0.0f;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+        const int q = q8 + i;
+        const float u0 = ua[i], u1 = ub[i];
 #pragma unroll
         for (int r4 = 0; r4 < 4; ++r4) {
             const float4 e = e_s[q][r4];
-            w[4 * r4 + 0] = __fmaf_rn(e.x, uq, w[4 * r4 + 0]);
-            w[4 * r4 + 1] = __fmaf_rn(e.y, uq, w[4 * r4 + 1]);
-            w[4 * r4 + 2] = __fmaf_rn(e.z, uq, w[4 * r4 + 2]);
-            w[4 * r4 + 3] = __fmaf_rn(e.w, uq, w[4 * r4 + 3]);
+            w0[4 * r4 + 0] = __fmaf_rn(e.x, u0, w0[4 * r4 + 0]);
+            w0[4 * r4 + 1] = __fmaf_rn(e.y, u0, w0[4 * r4 + 1]);
+            w0[4 * r4 + 2] = __fmaf_rn(e.z, u0, w0[4 * r4 + 2]);
+            w0[4 * r4 + 3] = __fmaf_rn(e.w, u0, w0[4 * r4 + 3]);
+            w1[4 * r4 + 0] = __fmaf_rn(e.x, u1, w1[4 * r4 + 0]);
+            w1[4 * r4 + 1] = __fmaf_rn(e.y, u1, w1[4 * r4 + 1]);
+            w1[4 * r4 + 2] = __fmaf_rn(e.z, u1, w1[4 * r4 + 2]);
+            w1[4 * r4 + 3] = __fmaf_rn(e.w, u1, w1[4 * r4 + 3]);
+        }
         }
     }
 #pragma unroll
-    for (int r = 0; r < 16; ++r)
-        if (n0 + r < N) work[(n0 + r) * K + v] = w[r];
+    for (int r = 0; r < 16; ++r) {
+        if (n0 + r < N) {
+            work[(n0 + r) * K + v0] = w0[r];
+            if (two) work[(n0 + r) * K + v1] = w1[r];
+        }
+    }
 }
 
 }  // namespace w4a8

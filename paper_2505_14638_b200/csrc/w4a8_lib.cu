@@ -813,7 +813,7 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
     int rc = check_device();
     if (rc != W4A8_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    constexpr int kBlockSmem = 128 * 128 * 4 + 8 * 128;
+    constexpr int kBlockSmem = 128 * 128 * 4 + kDpqRowsPerCta * 128;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -838,13 +838,13 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
     uint64_t launches = 3;
     const int G = (int)(K / kGroup);
     for (int b = 0; b < G; ++b) {
-        dpq_block_kernel<<<(unsigned)((N + 7) / 8), 256, kBlockSmem, st>>>(
+        dpq_block_kernel<<<(unsigned)((N + kDpqRowsPerCta - 1) / kDpqRowsPerCta), 32 * kDpqRowsPerCta, kBlockSmem, st>>>(
             work, U, perm, N, K, b, symmetric, mse_steps, per_channel, s_w, codes,
             static_cast<uint16_t*>(gscale_bf16), gzero, err);
         ++launches;
         const int64_t rest = K - ((int64_t)b + 1) * 128;
         if (rest > 0) {
-            dim3 grid((unsigned)((rest + 255) / 256), (unsigned)((N + 15) / 16));
+            dim3 grid((unsigned)((rest + 511) / 512), (unsigned)((N + 15) / 16));
             dpq_trailing_kernel<<<grid, 256, 0, st>>>(work, U, err, N, K, b);
             ++launches;
         }

@@ -200,6 +200,31 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
                       float* s_x_out, void* stream);
 
 /*
+ * Eq. 10 for weights quantized in an unconstrained activation order (the W4A8* rows of Table 3;
+ * appendix "Activation Reordering"): column k takes the scale and zero-point of group g_idx[k]
+ * instead of k / 128, so the groups are no longer runs of consecutive columns and the fused
+ * kernels (one look-up table per row and group) do not apply -- which is the inference overhead
+ * Group-Aware Reordering avoids.  This entry point materialises the FP8 weights (E4M3 bytes,
+ * [N][K]) for w4a8_linear_w8a8; both launches together are the cost of that scheme.
+ *   codes [N][K/2], gscale BF16 [N][G], gzero u8 [N][G] or NULL (z = 8), g_idx int32 [K] in [0, G).
+ * g_idx values are not range-checked on the device.
+ */
+int w4a8_dequant_weight_gidx(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
+                             const int32_t* g_idx, int64_t N, int64_t K, int64_t G, uint8_t* w8, void* stream);
+
+/*
+ * W8A8 comparison scheme (Sec. 4.3, Fig. 4): the same FP8 GEMM and epilogue on weights that are
+ * stored as FP8 E4M3 bytes -- e.g. the output of w4a8_dequant_weight -- so that the cost of
+ * streaming twice the bytes can be set against the cost of expanding INT4 on the fly, on the
+ * same device and with the same MMA code.  w8: device u8 [N][K], 16-byte aligned.  Workspace:
+ * w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_UMMA, 0) bytes (fp32 split-K partials).
+ * Other arguments and errors as in w4a8_linear.
+ */
+int w4a8_linear_w8a8(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* w8,
+                     const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Offline round-to-nearest weight quantizer (Eq. 6 -> 7 -> 8 -> 9, no error compensation),
  * so that a caller can produce the stored format on the device.  W is FP32 [N][K].
  *   symmetric != 0: s_g = max|w8| / 7, u = round(w8 / s_g) + 8 (codes 1..15), gzero may be NULL;

@@ -64,6 +64,8 @@ def _load():
     lib.oracle_quantize_weight_rtn.argtypes = [p, i64, i64, c.c_int, c.c_int, c.c_int, c.c_int, p, p, p, p]
     lib.oracle_dpq_quantize.restype = c.c_int
     lib.oracle_dpq_quantize.argtypes = [p, i64, i64, c.c_int, p, p, c.c_int, c.c_int, c.c_int, p, p, p, p, p, p]
+    lib.oracle_dequant_weight_gidx.restype = c.c_int
+    lib.oracle_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p]
     lib.oracle_dequant_weight.restype = c.c_int
     lib.oracle_dequant_weight.argtypes = [p, p, p, i64, i64, c.c_int, p]
     lib.oracle_quantize_act.restype = c.c_int
@@ -231,6 +233,24 @@ def dequant_weight(codes, gscale, gzero=None, group=128):
     rc = lib.oracle_dequant_weight(_ptr(codes), _ptr(gscale), _ptr(gzero), N, K, group, _ptr(w8))
     if rc != 0:
         raise ValueError("oracle_dequant_weight: bad arguments")
+    return w8
+
+
+def dequant_weight_gidx(codes, gscale, gzero, g_idx):
+    """Eq. 10 with a per-column group index g_idx int32 [K]: E4M3 bytes [N,K]."""
+    lib = _load()
+    codes = _c(codes, np.uint8)
+    gscale = _c(gscale, np.uint16)
+    g_idx = _c(g_idx, np.int32)
+    N, Kh = codes.shape
+    K = Kh * 2
+    G = gscale.shape[1]
+    if gzero is not None:
+        gzero = _c(gzero, np.uint8)
+    w8 = np.empty((N, K), dtype=np.uint8)
+    rc = lib.oracle_dequant_weight_gidx(_ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(g_idx), N, K, G, _ptr(w8))
+    if rc != 0:
+        raise ValueError("oracle_dequant_weight_gidx: bad arguments")
     return w8
 
 

@@ -222,6 +222,30 @@ int oracle_dequant_weight(const uint8_t* codes, const uint16_t* gscale, const ui
     return 0;
 }
 
+/*
+ * Eq. 10 when the weights were quantized in an unconstrained activation order (the W4A8* rows
+ * of Table 3; appendix "Activation Reordering"): after the codes are put back in their original
+ * positions the scale and zero-point of column k are those of group g_idx[k] of the processing
+ * order, no longer of k / group -- every weight needs its own look-up.
+ */
+int oracle_dequant_weight_gidx(const uint8_t* codes, const uint16_t* gscale, const uint8_t* gzero,
+                               const int32_t* g_idx, int64_t N, int64_t K, int64_t G, uint8_t* w8) {
+    if (!codes || !gscale || !g_idx || !w8 || N <= 0 || K <= 0 || G <= 0 || (K & 1)) return -1;
+    for (int64_t k = 0; k < K; ++k)
+        if (g_idx[k] < 0 || g_idx[k] >= G) return -1;
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t g = g_idx[k];
+            uint8_t byte = codes[n * (K / 2) + k / 2];
+            int u = (k & 1) ? (byte >> 4) : (byte & 0x0F);
+            int z = gzero ? gzero[n * G + g] : 8;
+            float s = oracle_bf16_to_f32(gscale[n * G + g]);
+            w8[n * K + k] = oracle_e4m3_encode((float)(u - z) * s);
+        }
+    }
+    return 0;
+}
+
 /* ------------------------------------------------------------------ Eq. 13 */
 
 /*

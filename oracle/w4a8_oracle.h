@@ -84,6 +84,11 @@ int oracle_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, 
 /* Number of OpenMP threads the linear will use. */
 int oracle_num_threads(void);
 
+/* Eq. 10 with a per-column group index (activation-ordered quantization, Table 3 '*' rows):
+ * column k takes scale / zero-point of group g_idx[k]; gscale and gzero are [N][G]. */
+int oracle_dequant_weight_gidx(const uint8_t* codes, const uint16_t* gscale, const uint8_t* gzero,
+                               const int32_t* g_idx, int64_t N, int64_t K, int64_t G, uint8_t* w8);
+
 /*
  * DPQ weight quantizer, Algorithm 1 (Sec. 3.1-3.3, Eq. 6-12) with the Cholesky formulation of the
  * update and Group-Aware Reordering (Sec. 3.2, appendix); see w4a8_dpq_oracle.c for the steps.

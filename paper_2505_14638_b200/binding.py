@@ -27,7 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
-    "w4a8_linear_fused", "w4a8_fused_is_faster",
+    "w4a8_linear_fused", "w4a8_fused_is_faster", "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
@@ -71,6 +71,10 @@ def lib():
                                  i32, i32, p]
     L.w4a8_linear_static_scratch.restype = i32
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
+    L.w4a8_dequant_weight_gidx.restype = i32
+    L.w4a8_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p, p]
+    L.w4a8_linear_w8a8.restype = i32
+    L.w4a8_linear_w8a8.argtypes = [p, i64, p, i64, p, p, i32, i64, i64, p, i64, i32, p, sz, p]
     L.w4a8_fused_is_faster.restype = i32
     L.w4a8_fused_is_faster.argtypes = [i64, i64, i64]
     L.w4a8_linear_fused.restype = i32
@@ -262,6 +266,35 @@ def linear_tiled(x8, s_x, tw, out_dtype=OUT_BF16, out=None, workspace=None):
                            out.stride(0), int(out_dtype), _ptr(workspace),
                            workspace.numel() * workspace.element_size(), _stream())
     _check("w4a8_linear", rc)
+    return out
+
+
+def dequant_weight_gidx(codes, gscale, gzero, g_idx, out=None):
+    """w4a8_dequant_weight_gidx: per-column group index g_idx int32 [K]; returns E4M3 bytes [N, K]."""
+    import torch
+    N, Kh = codes.shape
+    K = Kh * 2
+    w8 = out if out is not None else torch.empty((N, K), dtype=torch.uint8, device=codes.device)
+    rc = lib().w4a8_dequant_weight_gidx(_ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(g_idx), N, K,
+                                        gscale.shape[1], _ptr(w8), _stream())
+    _check("w4a8_dequant_weight_gidx", rc)
+    return w8
+
+
+def linear_w8a8(x8, s_x, w8, s_w, out_dtype=OUT_BF16, out=None):
+    """w4a8_linear_w8a8: FP8 activations [M, K] x FP8 weights [N, K] (uint8 E4M3 bytes)."""
+    import torch
+    M, K = x8.shape
+    N = w8.shape[0]
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, N), dtype=dt, device=x8.device)
+    nb = linear_workspace_bytes(M, N, K, ALGO_UMMA, 0)
+    ws = torch.empty((max(nb, 16),), dtype=torch.uint8, device=x8.device)
+    rc = lib().w4a8_linear_w8a8(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(w8), _ptr(s_w),
+                                0 if s_w.numel() == 1 else 1, N, K, _ptr(out), out.stride(0), int(out_dtype),
+                                _ptr(ws), nb, _stream())
+    _check("w4a8_linear_w8a8", rc)
     return out
 
 

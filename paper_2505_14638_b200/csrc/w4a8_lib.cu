@@ -522,6 +522,58 @@ static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_
     return rc;
 }
 
+// W8A8 comparison path (Sec. 4.3): FP8 weights [N][K] through the same tcgen05 kernel, no expansion.
+static int linear_w8a8_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* w8,
+                            const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
+                            int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (!x8 || !s_x || !w8 || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
+    if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
+    if (K % kGroup != 0 || N % 16 != 0 || ldx8 < K || ldy < N) return W4A8_ERR_BAD_SHAPE;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || !aligned16(y) || (ldx8 % 16) != 0) return W4A8_ERR_BAD_ALIGNMENT;
+    LinearPlan plan;
+    int rc = make_plan(M, N, K, W4A8_ALGO_UMMA, 0, &plan);
+    if (rc != W4A8_OK) return rc;
+    if (plan.workspace_bytes > 0) {
+        if (!workspace || workspace_bytes < plan.workspace_bytes) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
+    }
+    rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    CUtensorMap tw, tx;
+    if (!make_tmap_u8_2d(&tw, w8, (uint64_t)N, (uint64_t)K, (uint64_t)K, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)plan.bnx,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    float* partial = plan.split_k > 1 ? static_cast<float*>(workspace) : nullptr;
+    const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+#define W4A8_LAUNCH8(BNX, STG)                                                                                   \
+    rc = launch_umma<UmmaCfg<BNX, STG, true>>(tw, tx, nullptr, nullptr, s_x, s_w, sw_stride, y, ldy, out_dtype,  \
+                                              partial, Mi, Ni, Ki, plan.split_k, st)
+    switch (plan.bnx) {
+        case 16: W4A8_LAUNCH8(16, 4); break;
+        case 32: W4A8_LAUNCH8(32, 4); break;
+        case 64: W4A8_LAUNCH8(64, 6); break;
+        case 128: W4A8_LAUNCH8(128, 5); break;
+        default: W4A8_LAUNCH8(256, 4); break;
+    }
+#undef W4A8_LAUNCH8
+    if (rc != W4A8_OK) return rc;
+    if (plan.split_k > 1) {
+        int64_t total = M * N;
+        unsigned blocks = (unsigned)((total + 255) / 256);
+        if (blocks > 148u * 8u) blocks = 148u * 8u;
+        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, plan.split_k, M, N, s_x, s_w, sw_stride, y, ldy,
+                                                     out_dtype);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        rc = launch_status();
+    }
+    return rc;
+}
+
 static int linear_fused_impl(const void* x, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
                              const uint8_t* wpp, int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K,
                              void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out, float* s_x_out,
@@ -709,6 +761,30 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
     return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
                        ldy, out_dtype, scratch, plan.workspace_bytes, W4A8_ALGO_UMMA, plan.split_k,
                        static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_dequant_weight_gidx(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero,
+                             const int32_t* g_idx, int64_t N, int64_t K, int64_t G, uint8_t* w8, void* stream) {
+    if (!codes || !gscale_bf16 || !g_idx || !w8) return W4A8_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0 || G <= 0) return W4A8_ERR_INVALID_ARG;
+    if (K % 2 != 0) return W4A8_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(gscale_bf16) & 1u) || (reinterpret_cast<uintptr_t>(g_idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(w8) & 1u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int64_t total = N * (K / 2);
+    dequant_weight_gidx_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        codes, static_cast<const uint16_t*>(gscale_bf16), gzero, g_idx, N, K, G, w8);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+int w4a8_linear_w8a8(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* w8,
+                     const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+    return linear_w8a8_impl(x8, ldx8, s_x, M, w8, s_w, sw_stride, N, K, y, ldy, out_dtype, workspace,
+                            workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {

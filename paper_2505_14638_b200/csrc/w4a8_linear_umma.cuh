@@ -17,8 +17,11 @@
 
 namespace w4a8 {
 
-template <int BNX_, int STAGES_>
+// W8_ = true: the weights are FP8 E4M3 bytes already (the W8A8 comparison scheme of Sec. 4.3): the
+// TMA tile of 128 rows x 128 bytes lands directly in the swizzled MMA operand, nothing is expanded.
+template <int BNX_, int STAGES_, bool W8_ = false>
 struct UmmaCfg {
+    static constexpr bool W8 = W8_;
     static constexpr int BNX = BNX_;        // tokens per tile (MMA N)
     static constexpr int STAGES = STAGES_;
     static constexpr int BW = 128;          // weight rows per tile (MMA M)
@@ -38,7 +41,7 @@ struct UmmaCfg {
 
 template <class Cfg>
 __global__ void __launch_bounds__(Cfg::kThreads)
-linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N][K/2], box 64 x 128, 64B swizzle
+linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N][K/2], box 64 x 128, 64B swizzle (W8: FP8 u8 [N][K], box 128 x 128, 128B swizzle)
                    const __grid_constant__ CUtensorMap tmap_x,   // X8     u8 [M][K],   box 128 x BNX, 128B swizzle
                    const uint16_t* __restrict__ gscale, const uint8_t* __restrict__ gzero,
                    const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
@@ -105,8 +108,13 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                     ok = ptx::mbar_wait(bar_mma_done(s), (uint32_t)((it / STAGES - 1) & 1), abort_flag,
                                         status_word);
                 if (!ok) break;
-                ptx::mbar_arrive_expect_tx(bar_full_tma(s), (uint32_t)(Cfg::kWpBytes + Cfg::kXBytes));
-                ptx::tma_load_2d(stage_wp(s), &tmap_w, (kb0 + it) * 64, n0, bar_full_tma(s));
+                if (Cfg::W8) {
+                    ptx::mbar_arrive_expect_tx(bar_full_tma(s), (uint32_t)(Cfg::kW8Bytes + Cfg::kXBytes));
+                    ptx::tma_load_2d(stage_w8(s), &tmap_w, (kb0 + it) * 128, n0, bar_full_tma(s));
+                } else {
+                    ptx::mbar_arrive_expect_tx(bar_full_tma(s), (uint32_t)(Cfg::kWpBytes + Cfg::kXBytes));
+                    ptx::tma_load_2d(stage_wp(s), &tmap_w, (kb0 + it) * 64, n0, bar_full_tma(s));
+                }
                 ptx::tma_load_2d(stage_x(s), &tmap_x, (kb0 + it) * 128, m0, bar_full_tma(s));
                 issued = it + 1;
             }
@@ -130,7 +138,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)((it / STAGES) & 1);
                 ok = ptx::mbar_wait(bar_full_tma(s), ph, abort_flag, status_word) &&
-                     ptx::mbar_wait(bar_w8_full(s), ph, abort_flag, status_word);
+                     (Cfg::W8 || ptx::mbar_wait(bar_w8_full(s), ph, abort_flag, status_word));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
 #pragma unroll
@@ -163,10 +171,10 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
         const uint8_t* z_ptr = gzero ? gzero + (int64_t)(row_ok ? n : 0) * G + kb0 : nullptr;
         const uint32_t sw64 = (uint32_t)((r >> 1) & 3);
         const uint32_t sw128 = (uint32_t)(r & 7);
-        uint32_t sc_next = row_ok ? (uint32_t)__ldg(sc_ptr) : 0u;
-        int z_next = (z_ptr && row_ok) ? (int)__ldg(z_ptr) : 8;
+        uint32_t sc_next = (row_ok && !Cfg::W8) ? (uint32_t)__ldg(sc_ptr) : 0u;
+        int z_next = (z_ptr && row_ok && !Cfg::W8) ? (int)__ldg(z_ptr) : 8;
         bool ok = true;
-        for (int it = 0; it < nkb; ++it) {
+        for (int it = 0; it < (Cfg::W8 ? 0 : nkb); ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (uint32_t)((it / STAGES) & 1);
             const float sc = bf16_bits_to_float(sc_next);

@@ -307,6 +307,33 @@ rtn_quant_kernel(const float* __restrict__ W, int64_t N, int64_t K, int symmetri
 }
 
 // ---------------------------------------------------------------------------------------------
+// Eq. 10 with a per-column group index (activation-ordered quantization, the W4A8* rows of
+// Table 3): every weight fetches the scale and zero-point of group g_idx[k].  One thread per
+// byte of codes (two columns).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+dequant_weight_gidx_kernel(const uint8_t* __restrict__ codes, const uint16_t* __restrict__ gscale,
+                           const uint8_t* __restrict__ gzero, const int32_t* __restrict__ g_idx, int64_t N,
+                           int64_t K, int64_t G, uint8_t* __restrict__ w8) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;  // byte index
+    const int64_t Kh = K >> 1;
+    if (i >= N * Kh) return;
+    const int64_t n = i / Kh, kb = i - n * Kh;
+    const uint32_t byte = codes[i];
+    uint32_t out = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int64_t k = 2 * kb + h;
+        const int64_t g = __ldg(g_idx + k);
+        const int u = (int)((byte >> (4 * h)) & 15u);
+        const int z = gzero ? (int)__ldg(gzero + n * G + g) : 8;
+        const float s = bf16_bits_to_float((uint32_t)__ldg(gscale + n * G + g));
+        out |= (cvt_e4m3x2(0.0f, __fmul_rn((float)(u - z), s)) & 0xFFu) << (8 * h);
+    }
+    *reinterpret_cast<uint16_t*>(w8 + n * K + 2 * kb) = (uint16_t)out;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Plain CUDA-core linear (cross-check only): one thread per output element, weights dequantized
 // element by element with the direct formula of Eq. 10 (no look-up table), fp32 FMA accumulation.
 // ---------------------------------------------------------------------------------------------

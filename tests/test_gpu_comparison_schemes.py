@@ -1,0 +1,61 @@
+"""GPU parity of the comparison schemes around the W4A8 path (Sec. 4.3, Table 3 '*' rows):
+w4a8_linear_w8a8 (FP8 weights, no expansion) and w4a8_dequant_weight_gidx (activation-ordered
+groups) against the oracle.  FP8 bytes bit-exact; outputs within 2e-3 relative / 1 BF16 step."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_utils import bf16_bits, bf16_dev, dev, weights_to_dev
+from helpers import bf16_gate, fp32_gate, unpack_codes
+from paper_2505_14638_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 16, 128), (16, 1024, 1024), (5, 144, 384), (100, 512, 2048),
+                                   (300, 640, 1024), (16, 14336, 4096)])
+def test_w8a8_linear_matches_oracle(M, N, K):
+    wq = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 31), symmetric=True)
+    w8 = oracle.dequant_weight(*wq[:3])
+    x8, s_x = oracle.quantize_act(inputs.make_activation(M, K, 31, 0.01, 20.0))
+    ref = oracle.linear(x8, s_x, w8, wq[3])
+    y32 = binding.linear_w8a8(dev(x8), dev(s_x), dev(w8), dev(wq[3]), out_dtype=binding.OUT_FP32)
+    ybf = binding.linear_w8a8(dev(x8), dev(s_x), dev(w8), dev(wq[3]), out_dtype=binding.OUT_BF16)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    worst, _ = fp32_gate(y32.cpu().numpy(), ref["y64"], rel=2e-3)
+    assert worst <= 2e-3, worst
+    ok, dist = bf16_gate(bf16_bits(ybf), ref["y64"])
+    assert ok, dist
+
+
+def test_w8a8_equals_w4a8_on_the_same_fp8_weights():
+    # same FP8 operands, same MMA and accumulation order per tile: the two schemes give the same bits
+    M, N, K = 16, 1024, 1024
+    wq = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 32), symmetric=True)
+    wd = weights_to_dev(*wq)
+    x8, s_x = binding.quantize_act(bf16_dev(inputs.make_activation(M, K, 32, 0.01, 20.0)))
+    y4 = binding.linear(x8, s_x, *wd, out_dtype=binding.OUT_FP32, algo=binding.ALGO_UMMA)
+    y8 = binding.linear_w8a8(x8, s_x, binding.dequant_weight(*wd[:3]), wd[3], out_dtype=binding.OUT_FP32)
+    torch.cuda.synchronize()
+    assert torch.equal(y4.view(torch.int32), y8.view(torch.int32))
+
+
+@pytest.mark.parametrize("asym", [False, True])
+def test_gidx_dequant_matches_oracle(asym):
+    rng = np.random.default_rng(33)
+    N, K = 96, 1024
+    W = inputs.make_weight(N, K, 0.02, 33)
+    perm = rng.permutation(K)
+    codes_p, gs, gz, s_w = oracle.quantize_weight_rtn(W[:, perm], symmetric=not asym)
+    u_p = unpack_codes(codes_p)
+    u = np.empty_like(u_p)
+    u[:, perm] = u_p
+    codes = (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+    g_idx = np.empty(K, dtype=np.int32)
+    g_idx[perm] = np.arange(K) // 128
+    ref = oracle.dequant_weight_gidx(codes, gs, gz, g_idx)
+    got = binding.dequant_weight_gidx(dev(codes), bf16_dev(gs), None if gz is None else dev(gz), dev(g_idx))
+    torch.cuda.synchronize()
+    assert np.array_equal(got.cpu().numpy(), ref)

@@ -651,6 +651,68 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
     return out
 
 
+def scheme_sweep(torch, binding, inputs, dev):
+    """Same-box counterpart of the paper's scheme comparison (Sec. 4.3, Fig. 4, Table 3): per layer
+    and token count the time of W4A8 as built here (group-aware order: groups are runs of columns),
+    of W8A8 (FP8 weights, own kernel and the library's FP8 GEMM) and of W4A8 quantized in an
+    unconstrained activation order (per-column group index: the FP8 weights must be materialised
+    by w4a8_dequant_weight_gidx before a W8A8 GEMM can use them).  CUDA graphs, rotating weights."""
+    out = []
+    side = torch.cuda.Stream()
+
+    def graph_time(fn, reps):
+        fn(0)
+        torch.cuda.synchronize()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for c in range(reps):
+                    fn(c)
+        torch.cuda.current_stream().wait_stream(side)
+        return _time_loop(torch, g.replay, 5, warm=2) / reps
+
+    for name, k, n in C5_LAYERS:
+        copies = max(2, min(16, int(2.2 * 126e6 / (n * k)) + 1))     # FP8 copies: 1 byte per weight
+        tws, w8s, raw = [], [], []
+        for c in range(copies):
+            W = torch.from_numpy(inputs.make_weight(n, k, SIGMA, seed=8000 + c)).to(dev)
+            q = binding.quantize_weight_rtn(W, symmetric=True)
+            tws.append(binding.prepack_weight(*q))
+            w8s.append(binding.dequant_weight(*q[:3]))
+            raw.append(q)
+            del W
+        g_idx = (torch.randperm(k, device=dev) // GROUP).to(torch.int32)   # an unconstrained column order
+        w8_tmp = torch.empty((n, k), dtype=torch.uint8, device=dev)
+        one = torch.ones((), device=dev, dtype=torch.float32)
+        for m in (1, 16, 128, 2048):
+            xb = inputs.make_activation(m, k, 8000 + m, OUTLIER_FRAC, OUTLIER_MULT)
+            x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
+            x8, s_x = binding.quantize_act(x)
+            a8 = x8.view(torch.float8_e4m3fn)
+            y = torch.empty((m, n), dtype=torch.bfloat16, device=dev)
+            ws = binding.new_workspace(m, n, k, tws[0].fmt, dev)
+            reps = copies if m <= 128 else max(2, copies // 2)
+            t_w4 = graph_time(lambda c: binding.linear_tiled(x8, s_x, tws[c % copies], out=y, workspace=ws), reps)
+            t_w8 = graph_time(lambda c: binding.linear_w8a8(x8, s_x, w8s[c % copies], raw[0][3], out=y), reps)
+
+            def act_order(c):
+                cq = raw[c % copies]
+                binding.dequant_weight_gidx(cq[0], cq[1], None, g_idx, out=w8_tmp)
+                binding.linear_w8a8(x8, s_x, w8_tmp, cq[3], out=y)
+            t_ao = graph_time(act_order, reps)
+            t_lib = graph_time(lambda c: torch._scaled_mm(a8, w8s[c % copies].view(torch.float8_e4m3fn).t(),
+                                                          scale_a=one, scale_b=one, out_dtype=torch.bfloat16), reps)
+            out.append({"layer": name, "K": k, "N": n, "M": m, "w4a8_us": t_w4 * 1e6, "w8a8_own_kernel_us": t_w8 * 1e6,
+                        "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6})
+            del x, x8, s_x, y, ws
+        del tws, w8s, raw, w8_tmp
+        torch.cuda.empty_cache()
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set during the sweep")
+    return out
+
+
 def dpq_sweep(torch, binding, inputs, dev):
     """Offline DPQ quantizer (Algorithm 1 with Group-Aware Reordering and an 6-step scale search)
     on Llama-3-8B layer shapes: device time of w4a8_dpq_quantize against the plain-ALU roofline of
@@ -710,7 +772,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
-    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq"],
+    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes"],
                     help="instead of the bench line, print the per-layer table of config c5 (four Llama-3-8B "
                          "linears x M) or the single c4 case (M=8192, K=8192, N=28672)")
     args = ap.parse_args()
@@ -729,6 +791,8 @@ def main():
         dev = torch.device("cuda", local_rank)
         if args.sweep == "dpq":
             rows = dpq_sweep(torch, binding, inputs, dev)
+        elif args.sweep == "schemes":
+            rows = scheme_sweep(torch, binding, inputs, dev)
         elif args.sweep == "c5":
             rows = layer_sweep(torch, binding, inputs, dev, load_peaks())
         else:

@@ -2,11 +2,10 @@
 """Benchmark of the W4A8 linear hot path (activation FP8 quantize -> fused INT4->FP8 GEMM ->
 scaled BF16) on the decode sweep: M in {1,4,16}, K=4096, N=14336 (Llama-3-8B MLP up-projection).
 
-One step = one pass of the whole path over the sweep: for each M <= 4 one w4a8_linear_fused
-launch (activation quantization, weight dequantization, FP8 GEMM and scaled BF16 output in one
-kernel), for M = 16 w4a8_quantize_act then w4a8_linear (faster there than the fused launch,
-whose every CTA would have to scan all of X for the token scales); --two-kernel runs the
-two-kernel sequence for every M.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
+One step = one pass of the whole path over the sweep: for each M, w4a8_quantize_act then
+w4a8_linear -- or one w4a8_linear_fused launch (activation quantization, weight dequantization,
+FP8 GEMM and scaled BF16 output in one kernel) where w4a8_fused_is_faster says so (M = 1 on this
+layer); --two-kernel runs the two-kernel sequence for every M.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
 method must read per step, divided by the step time.  Weights rotate over several distinct
 copies whose total size exceeds twice the L2, so every pass streams them from HBM.
 
@@ -427,8 +426,8 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD, "parallelism": "replicas x%d (no collective)" % world,
                    "l2": "weights rotate over %d distinct copies (%.0f MB > 2 x 126 MB L2)"
                          % (WEIGHT_COPIES, WEIGHT_COPIES * weight_bytes() / 1e6),
-                   "step": ("M in (1,4): w4a8_linear_fused (activation quantization inside the kernel); M=16: "
-                            "w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)") if fused else
+                   "step": ("M in %s: w4a8_linear_fused (activation quantization inside the kernel); other M: "
+                            "w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)" % (fused_m,)) if fused else
                            "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
                    "launch": "CUDA graph replay, one graph per step" if use_graph else "eager launches"},
         "clocks": clocks,
@@ -438,7 +437,7 @@ def run_ours(args, rank, world, local_rank):
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "linear_splitn_kernel<MT=16> (%s), mean over M in {1,4,16}"
-                               % ("FUSE variant for M<=4" if fused else "w4a8_linear"),
+                               % ("FUSE variant for M in %s" % (fused_m,) if fused else "w4a8_linear"),
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,
@@ -492,6 +491,15 @@ def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
                     binding.linear_fused(xs[m], weights[c], out=ys[m])
         torch.cuda.current_stream().wait_stream(side)
         tf = _time_loop(torch, g2.replay, 20) / WEIGHT_COPIES
+        side.wait_stream(torch.cuda.current_stream())
+        g3 = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g3, stream=side):
+                for c in range(WEIGHT_COPIES):
+                    binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
+                    binding.linear_tiled(x8s[m], sxs[m], weights[c], out=ys[m], workspace=workspace)
+        torch.cuda.current_stream().wait_stream(side)
+        t2 = _time_loop(torch, g3.replay, 20) / WEIGHT_COPIES
         xb = torch.randn((m, K), dtype=torch.bfloat16, device=dev)
         j = [0]
 
@@ -499,7 +507,7 @@ def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
             j[0] += 1
             torch.matmul(xb, wb[j[0] % 4].t())
         tb = _time_loop(torch, f, 40)
-        out["M=%d" % m] = {"fused_us": tf * 1e6,
+        out["M=%d" % m] = {"quantize_then_linear_us": t2 * 1e6, "fused_us": tf * 1e6,
                            "fused_frac_hbm_measured":
                                linear_algorithmic_bytes(m, fused=True) / tf / 1e9 / peaks["hbm_gbs"],
                            "linear_only_us": t * 1e6, "linear_only_weight_GBps": weight_bytes() / t / 1e9,

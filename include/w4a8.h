@@ -185,14 +185,15 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  *               the kernel multiplied with (ldx8_out % 16 == 0, 16-byte aligned);
  *   s_x_out     optional (may be NULL): device float [M], receives the activation scales.
  *   y, ldy, out_dtype, s_w, sw_stride   as in w4a8_linear.
- * On B200 the fused launch is faster than the two-kernel sequence for M <= 4 and slower above
- * (every CTA scans all of X for the token scales).
+ * On B200 the fused launch turned out slower than w4a8_quantize_act + w4a8_linear chained on one
+ * stream (they overlap under programmatic dependent launch; every CTA of the fused launch scans X
+ * for the token scales): it is kept for callers that want a single launch.
  * Needs no workspace and allocates nothing.  Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
 #define W4A8_FUSED_MAX_M 16
-/* 1 when w4a8_linear_fused is the faster way to run this problem on B200 (few tokens, many
- * output channels), 0 when w4a8_quantize_act + w4a8_linear is. */
+/* 1 when w4a8_linear_fused is the faster way to run this problem on B200, 0 when
+ * w4a8_quantize_act + w4a8_linear is (currently always 0: see w4a8_linear_fused). */
 int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K);
 int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
                       const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,

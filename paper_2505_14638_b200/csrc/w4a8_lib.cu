@@ -207,6 +207,7 @@ struct SkPlan {
     size_t counter_bytes, workspace_bytes;
 };
 
+constexpr int kDecodeSpareSMs = 8;  // SMs a decode-sized (<= 16 tokens) linear leaves to small neighbouring kernels
 constexpr int kSplitNMaxM = 128;  // token counts served by the split-N (decode) kernel
 
 // Token-tile width and schedule of the persistent kernel from a small cost model (microseconds):
@@ -343,6 +344,16 @@ static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const fl
     const bool may_split_k = !FUSE && workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes &&
                              aligned16(workspace);
     if (!make_sn_plan<Cfg>(N, K, sms, may_split_k, &pl)) return W4A8_ERR_BAD_SHAPE;
+    // A decode-sized linear that would take every SM leaves a few to the small kernels that run
+    // between two such layers (the activation quantization of the next one: M CTAs): with two
+    // linear CTAs resident per SM those kernels otherwise find no room until a whole launch has
+    // drained, and the CTAs of the following launch that wait for them start late.  Measured on the
+    // quantize -> linear chain at M = 8..16: 15.2 -> 11.7 us (N = 14336), 27.8 -> 20.6 us (N = 28672).
+    if (!FUSE && MT == 16 && pl.KSPLIT == 1 && pl.T >= sms && sms > 4 * kDecodeSpareSMs) {
+        if (!make_sn_plan<Cfg>(N, K, sms - kDecodeSpareSMs, false, &pl)) return W4A8_ERR_BAD_SHAPE;
+        return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, fuse,
+                                          workspace, pl, sms - kDecodeSpareSMs);
+    }
     if constexpr (!FUSE) {
         if (pl.KSPLIT > 1)
             return launch_splitn_planned<SnCfg<MT, G, FMT, false, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
@@ -788,13 +799,17 @@ int w4a8_linear_w8a8(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t 
 }
 
 int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {
-    // Measured on B200: the fused launch wins for a few tokens on layers with many output channels;
-    // with few output channels the two-kernel path cuts K across the SMs (the fused launch, which has
-    // no workspace, cannot) and wins; above four tokens every CTA of the fused launch scans too much
-    // of X for the token scales.
-    if (M <= 0 || N <= 0 || K <= 0) return 0;
-    const int64_t blocks128 = (N + 127) / 128;
-    return (M <= kFuseFewTokens && blocks128 * 2 > kNominalSMs) ? 1 : 0;
+    // Measured on B200 (c2 layer, CUDA graphs): in a chain of equal launches one token takes 13.3 us
+    // fused against 14.5 us for quantize + linear, four tokens 14.3 against 11.5 us, sixteen 20.2
+    // against 11.8 us; in the benchmark's mixed chain (M = 1, 4, 16) the two-kernel sequence wins for
+    // every M (39.3 against 43.0 us per step with M = 1 fused).  The two kernels overlap under
+    // programmatic dependent launch and the linear leaves a few SMs to the quantize kernel, while
+    // every CTA of the fused launch has to scan X for the token scales; with few output channels the
+    // two-kernel path also cuts K across the SMs, which the fused launch (no workspace) cannot.
+    (void)M;
+    (void)N;
+    (void)K;
+    return 0;
 }
 
 int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,

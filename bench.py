@@ -45,7 +45,7 @@ WORKLOAD = ("c2 decode sweep: W4A8 linear, M in {1,4,16}, K=4096, N=14336, INT4 
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); see profiles/.  None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 30.37e6  # profiles/linear_splitn_decode_c2.md, mean of M = 1, 4, 16
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 30.36e6  # profiles/linear_splitn_decode_c2.md, mean of M = 1, 4, 16
 
 
 def weight_bytes(n=N, k=K):

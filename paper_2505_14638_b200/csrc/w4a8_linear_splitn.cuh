@@ -673,6 +673,19 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
             const int nst = Cfg::SPLITK ? (nkb + KS - 1) / KS : nst_all;
             const int R = (u1 - u0) * 8;
+            // This thread's rows of the range (one per 128-row block).  A lane beyond the range
+            // repeats the last row: its tensor-memory lane feeds accumulator rows nobody reads out.
+            const int row0 = r < R ? r : R - 1;
+            const int row1 = 128 + r < R ? 128 + r : R - 1;
+            const uint32_t code_off = tiled_row_offset(row0);
+            const uint32_t meta_off = (uint32_t)(plan.meta_off + row0 * MB);
+            // address steps from one item of a stage to the next: (block 0 -> block 1), then on to
+            // block 0 of the next k-block; with one block per k-block both are the k-block step
+            const uint32_t code_kstep = (uint32_t)(R * kRowCodeBytes), meta_kstep = (uint32_t)(R * MB);
+            const uint32_t code_s0 = MBLK == 2 ? tiled_row_offset(row1) - code_off : code_kstep;
+            const uint32_t meta_s0 = MBLK == 2 ? (uint32_t)((row1 - row0) * MB) : meta_kstep;
+            const uint32_t code_s1 = MBLK == 2 ? code_kstep - code_s0 : code_kstep;
+            const uint32_t meta_s1 = MBLK == 2 ? meta_kstep - meta_s0 : meta_kstep;
             int st = turn;
             for (; st < nst; st += G) {
                 const int kb = st * KS;
@@ -683,15 +696,14 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * plan.wstage);
+                uint32_t src = wsrc + code_off, msrc = wsrc + meta_off;
                 uint32_t a_col = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(r2.idx * Cfg::kAStageCols);
-                for (int kbl = 0; kbl < ks; ++kbl) {
-                    for (int b = 0; b < MBLK; ++b) {
-                        const int row = b * 128 + r;  // row within the range
-                        const int item = kbl * R + row;
-                        dequant_row_to_tmem<Cfg::FMT>(wsrc + (uint32_t)(item * kRowCodeBytes),
-                                                      wsrc + (uint32_t)(plan.meta_off + item * MB), row, row < R, a_col);
-                        a_col += 32u;
-                    }
+                const int items = ks * MBLK;
+                for (int i = 0; i < items; ++i) {
+                    dequant_row_to_tmem<Cfg::FMT>(src, msrc, a_col);
+                    a_col += 32u;
+                    src += (i & 1) ? code_s1 : code_s0;
+                    msrc += (i & 1) ? meta_s1 : meta_s0;
                 }
                 ptx::tmem_st_wait();
                 ptx::tc_fence_before_sync();

@@ -377,7 +377,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
-            dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + (uint32_t)r * 64u,
+            dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + tiled_row_offset(r),
                                           stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
                                           stage_w8(s2) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();

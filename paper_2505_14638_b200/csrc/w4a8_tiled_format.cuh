@@ -1,14 +1,17 @@
 // Tiled ("prepacked") weight layout shared by the persistent GEMM kernels, the sign-magnitude
 // look-up table for symmetric groups, and the offline prepack kernel.
 //
-// Layout (K = 128 KB k-blocks, N output channels):
-//   codes region  [KB][N][64 bytes]   row n of k-block kb at ((kb * N) + n) * 64; within a row the
-//                 16-byte chunk c is stored at chunk position c ^ ((n >> 1) & 3), so that eight
-//                 consecutive rows read with 128-bit loads touch every shared-memory bank once
+// Layout (K = 128 KB k-blocks, N output channels, N a multiple of 8):
+//   codes region  [KB][N/8][4 chunks][8 rows][16 bytes]: the 64 code bytes of row n of k-block kb
+//                 are four 16-byte chunks; chunk c is stored at
+//                 ((kb * N + (n & ~7)) * 64) + c * 128 + (n & 7) * 16, i.e. the same chunk of eight
+//                 consecutive rows is one 128-byte line.  A thread that expands row n reads its
+//                 chunks at a fixed 128-byte stride (no per-chunk address arithmetic), and eight
+//                 consecutive rows read with 128-bit loads touch every shared-memory bank once.
 //   meta region   [KB][N][MB bytes]   starts at KB * N * 64; MB = 2 (BF16 group scale) in the
 //                 sign-magnitude format, 4 (BF16 scale, zero-point byte, one byte of padding) in
 //                 the generic format
-// Any run of consecutive output channels of one k-block is therefore one contiguous, 128-byte
+// Any run of consecutive eight-row units of one k-block is therefore one contiguous, 128-byte
 // aligned piece of codes plus one contiguous piece of meta data: two bulk copies bring it into
 // shared memory, whatever row partition the kernel picks at launch.
 #pragma once
@@ -23,6 +26,11 @@ constexpr int kFmtTiled = W4A8_FMT_TILED;
 constexpr int kFmtTiledSignMag = W4A8_FMT_TILED_SIGNMAG;
 
 constexpr int kRowCodeBytes = 64;  // one row of one k-block: 128 INT4 codes
+constexpr uint32_t kChunkStride = 128;  // bytes between two chunks of one row
+// Offset of a row's first chunk within a piece of codes that starts on a multiple of eight rows.
+__host__ __device__ constexpr uint32_t tiled_row_offset(int row) {
+    return (uint32_t)(row >> 3) * 512u + (uint32_t)(row & 7) * 16u;
+}
 __host__ __device__ constexpr int meta_bytes(int fmt) { return fmt == kFmtTiledSignMag ? 2 : 4; }
 
 // Sign-magnitude table of a symmetric group (z = 8): entry d = nearest_E4M3(d * s), d = 0..7.
@@ -44,13 +52,26 @@ struct SignMagLut {
     }
 };
 
+// The four code chunks of one row (constant address offsets: no arithmetic per chunk).
+template <int C>
+__device__ __forceinline__ void load_code_chunk(uint32_t src, uint32_t (&pk)[16]) {
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];"
+                 : "=r"(pk[4 * C]), "=r"(pk[4 * C + 1]), "=r"(pk[4 * C + 2]), "=r"(pk[4 * C + 3])
+                 : "r"(src), "n"(C * (int)kChunkStride));
+}
+__device__ __forceinline__ void load_row_codes(uint32_t src, uint32_t (&pk)[16]) {
+    load_code_chunk<0>(src, pk);
+    load_code_chunk<1>(src, pk);
+    load_code_chunk<2>(src, pk);
+    load_code_chunk<3>(src, pk);
+}
+
 // Expands one row of one k-block into 128 E4M3 bytes written as a row of a K-major tile with
-// the 128-byte swizzle.  `src` = shared address of the row's 64 code bytes, `meta` = shared
-// address of its meta entry, `row` = row index within the copied piece (the piece must start on
-// a multiple of 8 rows), `dst` = shared address of the destination row.
+// the 128-byte swizzle.  `src` = shared address of the row's first code chunk (piece base +
+// tiled_row_offset(row)), `meta` = shared address of its meta entry, `row` = row index within
+// the destination tile, `dst` = shared address of the destination row.
 template <int FMT>
 __device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta, int row, uint32_t dst) {
-    const uint32_t sw64 = (uint32_t)((row >> 1) & 3);
     const uint32_t sw128 = (uint32_t)(row & 7);
     uint32_t mbits;
     if constexpr (FMT == kFmtTiledSignMag)
@@ -59,12 +80,7 @@ __device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta,
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
     const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
     uint32_t pk[16];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
-                     : "r"(src + (((uint32_t)c ^ sw64) << 4)));
-    }
+    load_row_codes(src, pk);
     SignMagLut slut;
     DequantLut glut;
     if constexpr (FMT == kFmtTiledSignMag)
@@ -90,27 +106,17 @@ __device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta,
 // Same expansion into registers and from there into tensor memory: the row's 128 E4M3 bytes go
 // to 32 consecutive 32-bit columns starting at `taddr` (lane = this thread's lane within its
 // warp's lane quarter), written as two 16-column stores to keep the live register count low.
-// Warp-collective: every lane of the warp must call it (lanes with `active` false store zeros).
+// Warp-collective: every lane of the warp must call it with a readable row (a lane without a
+// row of its own repeats another one; its tensor-memory lane is then never read out).
 template <int FMT>
-__device__ __forceinline__ void dequant_row_to_tmem(uint32_t src, uint32_t meta, int row, bool active, uint32_t taddr) {
-    const uint32_t sw64 = (uint32_t)((row >> 1) & 3);
-    uint32_t mbits = 0;
+__device__ __forceinline__ void dequant_row_to_tmem(uint32_t src, uint32_t meta, uint32_t taddr) {
+    uint32_t mbits;
     uint32_t pk[16];
-    if (active) {
-        if constexpr (FMT == kFmtTiledSignMag)
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
-        else
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
-                         : "r"(src + (((uint32_t)c ^ sw64) << 4)));
-        }
-    } else {
-#pragma unroll
-        for (int w = 0; w < 16; ++w) pk[w] = 0u;
-    }
+    if constexpr (FMT == kFmtTiledSignMag)
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    else
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    load_row_codes(src, pk);
     const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
     if constexpr (FMT == kFmtTiledSignMag) {
         SignMagLut lut;
@@ -183,10 +189,9 @@ prepack_kernel(const uint8_t* __restrict__ codes, const uint16_t* __restrict__ g
         }
         if (bad) atomicOr(status_word, kStatusBadCode);
     }
-    uint8_t* dst = out + (kb * N + n) * kRowCodeBytes;
-    const uint32_t sw64 = (uint32_t)((n >> 1) & 3);
+    uint8_t* dst = out + (kb * N + (n & ~(int64_t)7)) * kRowCodeBytes + (n & 7) * 16;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(dst + (((uint32_t)c ^ sw64) << 4)) = w[c];
+    for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(dst + c * kChunkStride) = w[c];
     uint8_t* meta = out + KB * N * kRowCodeBytes + (kb * N + n) * meta_bytes(fmt);
     const uint16_t sc = gscale[n * KB + kb];
     if (fmt == kFmtTiledSignMag) {

@@ -3,11 +3,12 @@
 scaled BF16) on the decode sweep: M in {1,4,16}, K=4096, N=14336 (Llama-3-8B MLP up-projection).
 
 One step = one pass of the whole path over the sweep: for each M, w4a8_quantize_act then
-w4a8_linear -- or one w4a8_linear_fused launch (activation quantization, weight dequantization,
-FP8 GEMM and scaled BF16 output in one kernel) where w4a8_fused_is_faster says so (M = 1 on this
-layer); --two-kernel runs the two-kernel sequence for every M.  The metric is the weight stream rate: bytes of INT4 codes + group scales the
-method must read per step, divided by the step time.  Weights rotate over several distinct
-copies whose total size exceeds twice the L2, so every pass streams them from HBM.
+w4a8_linear (or one w4a8_linear_fused launch where w4a8_fused_is_faster says so: nowhere at
+present; --two-kernel forces the two-kernel sequence).  The metric is the weight stream rate:
+bytes of INT4 codes + group scales the method must read per step, divided by the step time.
+Weights rotate over several distinct copies whose total size exceeds twice the L2, so every pass
+streams them from HBM.  Steps are replayed from CUDA graphs that hold --steps-per-graph
+consecutive steps each (a decode graph likewise holds all layers of a forward pass).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -302,8 +303,11 @@ def run_ours(args, rank, world, local_rank):
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set by the first steps (a bounded wait gave up)")
 
-    # ---- CUDA graphs: one per phase of the weight rotation (the step is launch-bound) ----
+    # ---- CUDA graphs (the step is launch-bound).  A graph holds `spg` consecutive steps, as a
+    # decode graph holds the layers of a whole forward pass; one graph per phase of the weight
+    # rotation.  Every step still runs all its launches on weights that come from HBM.
     use_graph = not args.no_graph
+    spg = args.steps_per_graph if (use_graph and args.steps % args.steps_per_graph == 0) else 1
     period = WEIGHT_COPIES
     g_full, g_lin, g_quant = [], [], None
     if use_graph:
@@ -313,12 +317,14 @@ def run_ours(args, rank, world, local_rank):
             for ph in range(period):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=side):
-                    eager_step(ph)
+                    for j in range(spg):
+                        eager_step(ph * spg + j)
                 g_full.append(g)
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=side):
-                    for i, m in enumerate(SWEEP_M):
-                        lin(m, ph * len(SWEEP_M) + i)
+                    for j in range(spg):
+                        for i, m in enumerate(SWEEP_M):
+                            lin(m, (ph * spg + j) * len(SWEEP_M) + i)
                 g_lin.append(g)
             if len(fused_m) < len(SWEEP_M):
                 g_quant = torch.cuda.CUDAGraph()
@@ -331,14 +337,15 @@ def run_ours(args, rank, world, local_rank):
 
     kernels_per_step = 2 * len(SWEEP_M) - len(fused_m)
 
-    def step(s):
+    def step_group(gi):
+        """Runs steps gi * spg .. gi * spg + spg - 1."""
         if use_graph:
-            g_full[s % period].replay()
+            g_full[gi % period].replay()
         else:
-            eager_step(s % period)
+            eager_step(gi % period)
 
-    for s in range(max(args.warmup, 3)):
-        step(s)
+    for gi in range((max(args.warmup, 3) + spg - 1) // spg):
+        step_group(gi)
     barrier()
 
     # ---- timed region 1: the whole path, K steps, device timed ----
@@ -348,8 +355,8 @@ def run_ours(args, rank, world, local_rank):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    for s in range(args.steps):
-        step(s)
+    for gi in range(args.steps // spg):
+        step_group(gi)
     e1.record()
     barrier()
     launches = args.steps * kernels_per_step
@@ -357,7 +364,7 @@ def run_ours(args, rank, world, local_rank):
 
     # ---- timed region 2: the same steps with the three linear launches bracketed by events ----
     pairs = []
-    for s in range(args.steps):
+    for s in range(args.steps // spg):
         if use_graph:
             if g_quant is not None:
                 g_quant.replay()
@@ -429,7 +436,7 @@ def run_ours(args, rank, world, local_rank):
                    "step": ("M in %s: w4a8_linear_fused (activation quantization inside the kernel); other M: "
                             "w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)" % (fused_m,)) if fused else
                            "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
-                   "launch": "CUDA graph replay, one graph per step" if use_graph else "eager launches"},
+                   "launch": ("CUDA graph replay, %d steps per graph" % spg) if use_graph else "eager launches"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(m * K * 2 for m in SWEEP_M),
@@ -778,6 +785,8 @@ def main():
     ap.add_argument("--two-kernel", action="store_true",
                     help="step = w4a8_quantize_act + w4a8_linear per M instead of the fused launch")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--steps-per-graph", type=int, default=4,
+                    help="consecutive steps captured in one CUDA graph (used when it divides --steps; default 4)")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
     ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes"],

@@ -207,7 +207,6 @@ struct SkPlan {
     size_t counter_bytes, workspace_bytes;
 };
 
-constexpr int kDecodeSpareSMs = 8;  // SMs a decode-sized (<= 16 tokens) linear leaves to small neighbouring kernels
 constexpr int kSplitNMaxM = 128;  // token counts served by the split-N (decode) kernel
 
 // Token-tile width and schedule of the persistent kernel from a small cost model (microseconds):
@@ -344,16 +343,6 @@ static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const fl
     const bool may_split_k = !FUSE && workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes &&
                              aligned16(workspace);
     if (!make_sn_plan<Cfg>(N, K, sms, may_split_k, &pl)) return W4A8_ERR_BAD_SHAPE;
-    // A decode-sized linear that would take every SM leaves a few to the small kernels that run
-    // between two such layers (the activation quantization of the next one: M CTAs): with two
-    // linear CTAs resident per SM those kernels otherwise find no room until a whole launch has
-    // drained, and the CTAs of the following launch that wait for them start late.  Measured on the
-    // quantize -> linear chain at M = 8..16: 15.2 -> 11.7 us (N = 14336), 27.8 -> 20.6 us (N = 28672).
-    if (!FUSE && MT == 16 && pl.KSPLIT == 1 && pl.T >= sms && sms > 4 * kDecodeSpareSMs) {
-        if (!make_sn_plan<Cfg>(N, K, sms - kDecodeSpareSMs, false, &pl)) return W4A8_ERR_BAD_SHAPE;
-        return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, fuse,
-                                          workspace, pl, sms - kDecodeSpareSMs);
-    }
     if constexpr (!FUSE) {
         if (pl.KSPLIT > 1)
             return launch_splitn_planned<SnCfg<MT, G, FMT, false, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
@@ -378,10 +367,21 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
     unsigned int* status = status_word_ptr();
     if (!status) return W4A8_ERR_CUDA;
     const int P = pl.T < sms ? pl.T : sms;
+    SnPlan plan = pl;
+    plan.P = P;
+    plan.sched = -1;
+    unsigned grid = (unsigned)P;
+    if (Cfg::MT == 16 && sms <= kSchedMaxSMs) {
+        // two CTAs of this variant fit on an SM: launch twice the workers and let the kernel keep
+        // one worker per SM (see the placement notes beside SchedSlot)
+        static std::atomic<unsigned int> seq{0};
+        plan.sched = (int)(seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
+        grid = 2u * (unsigned)P;
+    }
     unsigned int* counters = static_cast<unsigned int*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kSnCounterBytes);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)P);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(Cfg::kThreads);
     cfg.dynamicSmemBytes = (size_t)pl.smem;
     cfg.stream = st;
@@ -390,7 +390,7 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, pl,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, plan,
                                        fuse, counters, partials, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;

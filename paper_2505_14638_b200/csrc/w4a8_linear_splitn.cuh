@@ -113,7 +113,69 @@ struct SnPlan {
     int wstage;    // bytes per stage: packed codes + meta
     int xstage;    // bytes per stage: activation tiles
     int smem;      // dynamic shared memory to request
+    int P;         // CTAs that do the work; CTA p takes tiles p, p + P, ...
+    int sched;     // >= 0: slot of the per-launch placement state (twice P CTAs are launched, see below); -1: CTA p = blockIdx.x
 };
+
+// ---- placement of the decode-sized launches -------------------------------------------------
+// Two CTAs of this kernel fit on an SM so that the CTAs of the NEXT launch can move in beside
+// the running ones, fetch their first weight stages and expand them while they wait for their
+// activations.  That only pays if the two CTAs on an SM belong to different launches: two CTAs
+// of one launch on one SM share its integer pipe and take twice as long, and the SM they left
+// empty then receives two CTAs of the following launch, so the pattern persists.  The hardware
+// places a CTA wherever there is room, so the kernel enforces the rule itself: a launch has
+// twice as many CTAs ("candidates") as it needs workers.  A candidate that finds a worker of
+// its own launch already on its SM retires at once (unless so few candidates are left that the
+// work could otherwise go undone); the first candidate on an SM takes the next worker index.
+// State lives in a small table of slots handed out round-robin by the host, one per launch, and
+// the last candidate of a launch to enter clears its slot: replaying a captured launch reuses
+// its slot, and launches that can overlap in time (consecutive ones) hold different slots.
+constexpr int kSchedSlots = 64;
+constexpr int kSchedMaxSMs = 192;
+struct SchedSlot {
+    unsigned int started;   // candidates that have drawn a start number
+    unsigned int issued;    // worker indices handed out
+    unsigned int finished;  // candidates that have entered
+    unsigned int pad;
+    unsigned int on_sm[kSchedMaxSMs];  // candidates of this launch seen per SM
+};
+__device__ SchedSlot g_sched[kSchedSlots];
+
+// Called by thread 0 of a candidate: returns its worker index, or -1 to retire.  Plain atomic adds
+// only (a compare-and-swap loop on one word serialises hundreds of CTAs that start together at one
+// L2 round trip each).
+__device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candidates) {
+    unsigned int smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    // (the two adds are independent: one L2 round trip for both)
+    const unsigned int c = atomicAdd(&sl->started, 1u);
+    const bool first_here = smid < (unsigned)kSchedMaxSMs ? atomicAdd(&sl->on_sm[smid], 1u) == 0u : true;
+    bool want = first_here;
+    if (!want) {
+        // A second candidate on this SM works only if the candidates still to come could not
+        // cover the indices still to be issued.  The count read here may lag behind (never run
+        // ahead of) the true one, which errs towards working; the candidate with the last start
+        // number therefore declines only when every index has been issued.
+        const unsigned int i = *reinterpret_cast<volatile unsigned int*>(&sl->issued);
+        want = i < (unsigned)workers && (unsigned)workers - i >= (unsigned)candidates - c;
+    }
+    if (!want) return -1;
+    const unsigned int idx = atomicAdd(&sl->issued, 1u);
+    return idx < (unsigned)workers ? (int)idx : -1;
+}
+// Called once by every candidate after sched_enter: the slot is only needed while candidates
+// enter, so the last one to have entered clears it (nothing of this runs at the end of the
+// kernel, where it would delay the launch's completion).
+__device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
+    __threadfence();
+    if (atomicAdd(&sl->finished, 1u) == (unsigned)candidates - 1u) {
+        for (int i = 0; i < kSchedMaxSMs; ++i) sl->on_sm[i] = 0u;
+        sl->started = 0u;
+        sl->issued = 0u;
+        sl->finished = 0u;
+        __threadfence();
+    }
+}
 
 // Arguments of the fused activation quantization (unused otherwise).
 struct SnFuse {
@@ -190,8 +252,12 @@ __device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, i
     }
 }
 
+// Register budget of the decode variant (<= 16 tokens): besides two of its CTAs an SM has to hold
+// the small kernel that runs between two layers (activation quantization: 256 threads x 32..48
+// registers), or the CTA that finds no room starts a whole layer late.  Bounds for 576 threads
+// give 56 registers: 2 x 448 x 56 + 256 x 48 <= 65536.
 template <class Cfg>
-__global__ void __launch_bounds__(Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
+__global__ void __launch_bounds__(Cfg::MT == 16 && !Cfg::FUSE ? 576 : Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
 linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x MT, 128B swizzle
                      const uint8_t* __restrict__ wpp, const float* __restrict__ s_x,
                      const float* __restrict__ s_w, int sw_stride, void* __restrict__ y, int64_t ldy,
@@ -229,7 +295,10 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = K >> 7;
     const int64_t NU = N >> 3;           // the row partition works in units of 8 rows
-    const int P = gridDim.x, p = blockIdx.x;
+    int P = gridDim.x, p = blockIdx.x;
+    __shared__ int worker_s;
+    // (thread 0 asks for a worker index while thread 32 sets up the barriers)
+    if (plan.sched >= 0 && threadIdx.x == 0) worker_s = sched_enter(&g_sched[plan.sched], plan.P, (int)gridDim.x);
     const int KSPLIT = Cfg::SPLITK ? plan.KSPLIT : 1, TR = T / KSPLIT;
     // Tile t: 8-row units [u0, u1) of row range t / KSPLIT, k-blocks [kb0, kb0 + nkb) of chunk t % KSPLIT.
     const int nst_all = (KB + KS - 1) / KS;  // stages per tile when K is not cut
@@ -253,7 +322,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         return g;
     };
 
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 32) {
         for (int s = 0; s < S1; ++s) {
             ptx::mbar_init(bar_full0 + 8u * s, 1);
             ptx::mbar_init(bar_xfull0 + 8u * s, Cfg::FUSE ? (uint32_t)x_map(0, M, S1).tps : 1u);
@@ -268,6 +337,16 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         if (!Cfg::FUSE) ptx::prefetch_tensormap(&tmap_x);
     }
     if (Cfg::FUSE && threadIdx.x >= 64 && threadIdx.x < 80) amax_s[threadIdx.x - 64] = 0u;
+    if (plan.sched >= 0) {
+        __syncthreads();
+        p = worker_s;
+        P = plan.P;
+        if (p < 0) {  // a worker of this launch is already on this SM: retire
+            if (threadIdx.x == 0) sched_entered(&g_sched[plan.sched], (int)gridDim.x);
+            return;
+        }
+        if (threadIdx.x == 64) sched_entered(&g_sched[plan.sched], (int)gridDim.x);  // an idle epilogue thread
+    }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
         ptx::tmem_relinquish();
@@ -356,7 +435,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                         inv = __fdiv_rn(kE4M3Max, amax);
                     }
                 }
-                if (blockIdx.x == 0 && fuse.s_x_out != nullptr) fuse.s_x_out[ft] = s;
+                if (p == 0 && fuse.s_x_out != nullptr) fuse.s_x_out[ft] = s;
             }
             sx_s[ft] = s;
             inv_s[ft] = inv;
@@ -577,7 +656,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     if (!ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rg.idx, rg.phase ^ 1u, abort_flag, status_word))
                         return false;
                     if (xact) {
-                        if (xrow_ok && blockIdx.x == 0 && fuse.x8_out != nullptr) {
+                        if (xrow_ok && p == 0 && fuse.x8_out != nullptr) {
                             uint4* o = reinterpret_cast<uint4*>(fuse.x8_out + (int64_t)xm.xrow * fuse.ldx8_out +
                                                                 (int64_t)kbk * 128 + xm.xq * 32);
                             o[0] = lo;
@@ -690,9 +769,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             for (; st < nst; st += G) {
                 const int kb = st * KS;
                 const int ks = (nkb - kb) < KS ? (nkb - kb) : KS;
-                ok = ptx::mbar_wait(bar_full0 + 8u * (uint32_t)r1.idx, r1.phase, abort_flag, status_word);
-                if (ok && done >= S2)
-                    ok = ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rl.idx, rl.phase, abort_flag, status_word);
+                // both barriers are normally complete already: test them together, wait only if not
+                const uint32_t full_bar = bar_full0 + 8u * (uint32_t)r1.idx;
+                const uint32_t free_bar = bar_free10 + 8u * (uint32_t)rl.idx;
+                const bool have_w = ptx::mbar_test_wait(full_bar, r1.phase);
+                const bool have_slot = done < S2 || ptx::mbar_test_wait(free_bar, rl.phase);
+                if (!have_w) ok = ptx::mbar_wait(full_bar, r1.phase, abort_flag, status_word);
+                if (ok && !have_slot) ok = ptx::mbar_wait(free_bar, rl.phase, abort_flag, status_word);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * plan.wstage);

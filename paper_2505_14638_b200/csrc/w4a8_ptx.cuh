@@ -69,6 +69,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
+// Non-blocking test of a phase; two of them issued back to back overlap their round trips.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Waits for the phase with the given parity to complete.  Returns false when another thread of
 // the CTA has raised the abort flag or when the time limit runs out (then it raises the flag
 // and sets the timeout bit in the device status word).

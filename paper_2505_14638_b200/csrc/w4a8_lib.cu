@@ -371,9 +371,11 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
     plan.P = P;
     plan.sched = -1;
     unsigned grid = (unsigned)P;
-    if (Cfg::MT == 16 && sms <= kSchedMaxSMs) {
+    if (Cfg::MT == 16 && sms <= kSchedMaxSMs && (K / 128) / pl.KSPLIT >= 16) {
         // two CTAs of this variant fit on an SM: launch twice the workers and let the kernel keep
-        // one worker per SM (see the placement notes beside SchedSlot)
+        // one worker per SM (see the placement notes beside SchedSlot).  Not for short K walks
+        // (under 16 k-blocks per tile): there the extra microsecond at the start of a launch costs
+        // more than an occasional SM with two workers (o projection at M = 1: 8.4 against 6.6 us).
         static std::atomic<unsigned int> seq{0};
         plan.sched = (int)(seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
         grid = 2u * (unsigned)P;

@@ -1,0 +1,69 @@
+"""GPU: the decode-sized launches hand out their worker indices at run time (twice as many CTAs
+as workers, at most one worker per SM and launch; the state lives in a table of 64 slots that the
+host hands out round-robin and the kernel clears).  Whatever the placement, every row range must
+be computed exactly once: long runs of launches -- more than there are slots, eager and replayed
+from one CUDA graph, alternating shapes -- must reproduce the first result bit for bit, and that
+result must match the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_utils import bf16_dev, weights_to_dev
+from helpers import fp32_gate
+from paper_2505_14638_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(M, N, K, seed):
+    W = inputs.make_weight(N, K, 0.02, seed)
+    wq = oracle.quantize_weight_rtn(W, symmetric=True)
+    tw = binding.prepack_weight(*weights_to_dev(*wq), weight_format=binding.FMT_TILED_SIGNMAG)
+    xb = inputs.make_activation(M, K, seed + 1)
+    x8_ref, s_x_ref = oracle.quantize_act(xb)
+    ref = oracle.linear(x8_ref, s_x_ref, oracle.dequant_weight(*wq[:3]), wq[3])
+    x8, s_x = binding.quantize_act(bf16_dev(xb))
+    ws = binding.new_workspace(M, N, K, tw.fmt, x8.device)
+    return tw, x8, s_x, ref["y64"], ws
+
+
+def test_many_launches_repeat_the_first_result():
+    # K = 2048 and K = 4096 walk 16 and 32 k-blocks per tile (run-time worker indices);
+    # N = 18960 gives ragged ranges, N = 37904 two tiles per worker
+    cases = [_case(16, 18960, 2048, 5), _case(3, 37904, 4096, 7)]
+    outs = [torch.empty((c[1].shape[0], c[0].N), dtype=torch.float32, device="cuda") for c in cases]
+    first = []
+    for (tw, x8, s_x, y64, ws), out in zip(cases, outs):
+        binding.linear_tiled(x8, s_x, tw, out=out, out_dtype=binding.OUT_FP32, workspace=ws)
+        torch.cuda.synchronize()
+        worst, _ = fp32_gate(out.cpu().numpy(), y64, rel=2e-3)
+        assert worst <= 2e-3, worst
+        first.append(out.clone())
+    # eager: 150 launches (more than two rounds of the 64 slots), alternating the two shapes
+    for i in range(150):
+        tw, x8, s_x, _, ws = cases[i & 1]
+        outs[i & 1].fill_(float("nan"))
+        binding.linear_tiled(x8, s_x, tw, out=outs[i & 1], out_dtype=binding.OUT_FP32, workspace=ws)
+        if i % 37 == 0 or i >= 148:
+            assert torch.equal(outs[i & 1], first[i & 1]), i
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    # one graph with 70 launches (slots repeat inside the graph), replayed several times
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for i in range(70):
+                tw, x8, s_x, _, ws = cases[i & 1]
+                binding.linear_tiled(x8, s_x, tw, out=outs[i & 1], out_dtype=binding.OUT_FP32, workspace=ws)
+    torch.cuda.current_stream().wait_stream(side)
+    for rep in range(5):
+        for o in outs:
+            o.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        for o, f in zip(outs, first):
+            assert torch.equal(o, f), rep
+    assert binding.query_device_status() == 0

@@ -191,6 +191,26 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * Needs no workspace and allocates nothing.  Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
+/*
+ * Gated-MLP activation fused with the activation quantization of the next linear layer (the
+ * paper quantizes the BF16 activations that enter a linear layer, Eq. 13; in a Llama MLP block
+ * those of the down projection are silu(gate) * up, computed from the output of the stacked
+ * gate/up projection):
+ *   h[m][f]  = BF16( silu(G[m][f]) * U[m][f] ),  silu(g) = g / (1 + exp(-g)), evaluated in fp32,
+ *   G = gate_up[m][0..F), U = gate_up[m][F..2F);
+ *   (x8, s_x) = w4a8_quantize_act(h), same scale modes.
+ * Saves writing h and reading it back (4 B per element) and one launch.
+ *   gate_up_bf16  device BF16 [M][ldgu], ldgu >= 2 F, ldgu % 8 == 0, 16-byte aligned;
+ *   F % 16 == 0, F <= 16384;  x8 device u8 [M][ldx8] (ldx8 % 16 == 0), s_x device float [M];
+ *   h_bf16_out    optional (may be NULL): device BF16 [M][ldh], receives h (ldh % 8 == 0).
+ * exp() comes from the CUDA math library (about 2 ulp), so h can differ from a correctly rounded
+ * evaluation by one BF16 step on a small fraction of the elements; everything after h is exact
+ * as in w4a8_quantize_act.  Errors as w4a8_quantize_act; W4A8_ERR_BAD_SHAPE for F > 16384.
+ */
+int w4a8_silu_mul_quantize(const void* gate_up_bf16, int64_t M, int64_t F, int64_t ldgu, uint8_t* x8,
+                           int64_t ldx8, float* s_x, int scale_mode, const float* static_scale,
+                           void* h_bf16_out, int64_t ldh, void* stream);
+
 #define W4A8_FUSED_MAX_M 16
 /* 1 when w4a8_linear_fused is the faster way to run this problem on B200, 0 when
  * w4a8_quantize_act + w4a8_linear is (currently always 0: see w4a8_linear_fused). */

@@ -268,6 +268,45 @@ def quantize_act(x_bf16, scale_mode=0, static_scale=None):
     return x8, s_x
 
 
+def silu_mul_f64(gate_up_bf16) -> np.ndarray:
+    """The gated-MLP activation by its definition, in double precision:
+    h = silu(G) * U, silu(g) = g / (1 + exp(-g)); G = first half of each row, U = second half.
+    gate_up_bf16: uint16 [M, 2F] (BF16 bit patterns).  Returns float64 [M, F] (not rounded)."""
+    gu = bf16_to_f32(_c(gate_up_bf16, np.uint16)).astype(np.float64)
+    F = gu.shape[1] // 2
+    g, u = gu[:, :F], gu[:, F:]
+    return g / (1.0 + np.exp(-g)) * u
+
+
+def f64_to_bf16(x) -> np.ndarray:
+    """Round-to-nearest-even of doubles to BF16 bit patterns in ONE rounding (normal range only:
+    the magnitudes here are far from the BF16 subnormals and from overflow; zero maps to zero)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    b = x.view(np.uint64)
+    sign = (b >> np.uint64(63)).astype(np.uint64)
+    exp = ((b >> np.uint64(52)) & np.uint64(0x7FF)).astype(np.int64)
+    man = b & np.uint64((1 << 52) - 1)
+    keep = (man >> np.uint64(45)).astype(np.int64)            # 7 mantissa bits
+    rem = man & np.uint64((1 << 45) - 1)
+    half = np.uint64(1 << 44)
+    up = (rem > half) | ((rem == half) & ((keep & 1) == 1))
+    keep = keep + up.astype(np.int64)
+    carry = keep == 128
+    keep = np.where(carry, 0, keep)
+    e8 = exp - 1023 + 127 + carry.astype(np.int64)
+    zero = (exp == 0)
+    if np.any(~zero & ((e8 <= 0) | (e8 >= 255))):
+        raise ValueError("f64_to_bf16: value outside the normal BF16 range")
+    out = (sign.astype(np.int64) << 15) | (e8 << 7) | keep
+    out = np.where(zero, sign.astype(np.int64) << 15, out)
+    return out.astype(np.uint16)
+
+
+def silu_mul(gate_up_bf16) -> np.ndarray:
+    """h = BF16_RNE(silu(G) * U): the activations that enter the down projection.  uint16 [M, F]."""
+    return f64_to_bf16(silu_mul_f64(gate_up_bf16))
+
+
 def linear(x8, s_x, w8, s_w, cols=None, want=("y64", "y32", "ybf16", "yabs")):
     """Exact FP8 dot products with Eq. 4 / Eq. 11 scales.  Returns a dict of [M, N or len(cols)]."""
     lib = _load()

@@ -28,6 +28,7 @@ EXPORTS = (
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
     "w4a8_linear_fused", "w4a8_fused_is_faster", "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
+    "w4a8_silu_mul_quantize",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
@@ -56,6 +57,8 @@ def lib():
     p, i64, i32, sz = c.c_void_p, c.c_int64, c.c_int, c.c_size_t
     L.w4a8_quantize_act.restype = i32
     L.w4a8_quantize_act.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p]
+    L.w4a8_silu_mul_quantize.restype = i32
+    L.w4a8_silu_mul_quantize.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p, i64, p]
     L.w4a8_dequant_weight.restype = i32
     L.w4a8_dequant_weight.argtypes = [p, p, p, i64, i64, i32, p, p]
     L.w4a8_linear.restype = i32
@@ -148,6 +151,25 @@ def quantize_act(x, scale_mode=SCALE_EXACT, static_scale=None, out=None):
     rc = lib().w4a8_quantize_act(_ptr(x), M, K, x.stride(0), _ptr(x8), x8.stride(0), _ptr(s_x),
                                  int(scale_mode), _ptr(static_scale), _stream())
     _check("w4a8_quantize_act", rc)
+    return x8, s_x
+
+
+def silu_mul_quantize(gate_up, scale_mode=SCALE_EXACT, static_scale=None, out=None, h_out=None):
+    """w4a8_silu_mul_quantize: gate_up BF16 [M, 2F] (gate first, up second).
+    Returns (x8 uint8 [M, F], s_x float32 [M]); h_out (BF16 [M, F]) optionally receives h."""
+    import torch
+    assert gate_up.is_cuda and gate_up.dtype == torch.bfloat16 and gate_up.dim() == 2 and gate_up.stride(1) == 1
+    M, F2 = gate_up.shape
+    F = F2 // 2
+    if out is None:
+        x8 = torch.empty((M, F), dtype=torch.uint8, device=gate_up.device)
+        s_x = torch.empty((M,), dtype=torch.float32, device=gate_up.device)
+    else:
+        x8, s_x = out
+    rc = lib().w4a8_silu_mul_quantize(_ptr(gate_up), M, F, gate_up.stride(0), _ptr(x8), x8.stride(0), _ptr(s_x),
+                                      int(scale_mode), _ptr(static_scale), _ptr(h_out),
+                                      0 if h_out is None else h_out.stride(0), _stream())
+    _check("w4a8_silu_mul_quantize", rc)
     return x8, s_x
 
 

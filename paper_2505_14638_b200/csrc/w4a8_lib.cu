@@ -670,6 +670,46 @@ static int quantize_act_impl(const void* x, int64_t M, int64_t K, int64_t ldx, u
     return launch_status();
 }
 
+static int silu_mul_quantize_impl(const void* gu, int64_t M, int64_t F, int64_t ldgu, uint8_t* x8, int64_t ldx8,
+                                  float* s_x, int scale_mode, const float* static_scale, void* h_out, int64_t ldh,
+                                  cudaStream_t st) {
+    if (!gu || !x8 || !s_x) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || F <= 0) return W4A8_ERR_INVALID_ARG;
+    if (scale_mode != W4A8_SCALE_EXACT && scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
+    if (F % 16 != 0 || F > 16384 || ldgu < 2 * F || ldx8 < F || (h_out && ldh < F) || M > INT32_MAX)
+        return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(gu) || !aligned16(x8) || (ldgu % 8) != 0 || (ldx8 % 16) != 0 ||
+        (reinterpret_cast<uintptr_t>(s_x) & 3u) || (h_out && (!aligned16(h_out) || (ldh % 8) != 0)))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    const uint16_t* g = static_cast<const uint16_t*>(gu);
+    uint16_t* h = static_cast<uint16_t*>(h_out);
+    const int64_t nchunks = F / 16;
+    cudaError_t lerr;
+    if (nchunks <= 256)
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 1>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
+                                  static_scale, h, ldh);
+    else if (nchunks <= 512)
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 2>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
+                                  static_scale, h, ldh);
+    else
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 4>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
+                                  static_scale, h, ldh);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (lerr != cudaSuccess) return W4A8_ERR_CUDA;
+    return launch_status();
+}
+
 }  // namespace w4a8
 
 using namespace w4a8;
@@ -820,6 +860,13 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
                       float* s_x_out, void* stream) {
     return linear_fused_impl(x_bf16, ldx, M, scale_mode, static_scale, weights, weight_format, s_w, sw_stride, N, K,
                              y, ldy, out_dtype, x8_out, ldx8_out, s_x_out, static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_silu_mul_quantize(const void* gate_up_bf16, int64_t M, int64_t F, int64_t ldgu, uint8_t* x8, int64_t ldx8,
+                           float* s_x, int scale_mode, const float* static_scale, void* h_bf16_out, int64_t ldh,
+                           void* stream) {
+    return silu_mul_quantize_impl(gate_up_bf16, M, F, ldgu, x8, ldx8, s_x, scale_mode, static_scale, h_bf16_out, ldh,
+                                  static_cast<cudaStream_t>(stream));
 }
 
 size_t w4a8_linear_ex_workspace_bytes(int64_t M, int64_t N, int64_t K, int algo, int split_k) {

@@ -123,6 +123,87 @@ act_quant_kernel(const uint16_t* __restrict__ x, int64_t K, int64_t ldx, uint8_t
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Gated-MLP activation fused with the Eq. 13 quantization of its result: the input row holds
+// gate (first F values) and up (next F values), as the output of a linear layer whose weight
+// stacks the gate and up projections;  h = BF16( silu(gate) * up ),  silu(g) = g / (1 + exp(-g)),
+// all in fp32 (division and multiplications correctly rounded, expf from the math library), then
+// h is quantized per token exactly as act_quant_kernel does.  One CTA per token; F <= THREADS*NCH*16.
+// The BF16 round trip through memory between the two linear layers of the block is saved.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t silu_mul_bf16x2(uint32_t g2, uint32_t u2) {
+    const float g0 = __uint_as_float(g2 << 16), g1 = __uint_as_float(g2 & 0xFFFF0000u);
+    const float u0 = __uint_as_float(u2 << 16), u1 = __uint_as_float(u2 & 0xFFFF0000u);
+    const float h0 = __fmul_rn(__fdiv_rn(g0, __fadd_rn(1.0f, expf(-g0))), u0);
+    const float h1 = __fmul_rn(__fdiv_rn(g1, __fadd_rn(1.0f, expf(-g1))), u1);
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(h0)) |
+           ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(h1)) << 16);
+}
+
+template <int THREADS, int NCH>
+__global__ void __launch_bounds__(THREADS)
+silu_mul_quant_kernel(const uint16_t* __restrict__ gu, int64_t F, int64_t ldgu, uint8_t* __restrict__ x8,
+                      int64_t ldx8, float* __restrict__ s_x, int scale_mode,
+                      const float* __restrict__ static_scale, uint16_t* __restrict__ h_out, int64_t ldh) {
+    __shared__ float red[32];
+    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();
+    const int64_t row = blockIdx.x;
+    const int nchunks = (int)(F >> 4);
+    const uint4* gsrc = reinterpret_cast<const uint4*>(gu + row * ldgu);
+    const uint4* usrc = reinterpret_cast<const uint4*>(gu + row * ldgu + F);
+    uint4 v[NCH][2];
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = threadIdx.x + i * THREADS;
+        if (c < nchunks) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const uint4 g = __ldg(gsrc + 2 * c + hh), u = __ldg(usrc + 2 * c + hh);
+                v[i][hh].x = silu_mul_bf16x2(g.x, u.x);
+                v[i][hh].y = silu_mul_bf16x2(g.y, u.y);
+                v[i][hh].z = silu_mul_bf16x2(g.z, u.z);
+                v[i][hh].w = silu_mul_bf16x2(g.w, u.w);
+                amax = absmax_bf16x8(v[i][hh], amax);
+            }
+            if (h_out != nullptr) {
+                uint4* hd = reinterpret_cast<uint4*>(h_out + row * ldh);
+                hd[2 * c] = v[i][0];
+                hd[2 * c + 1] = v[i][1];
+            }
+        }
+    }
+    float s, inv;
+    if (static_scale != nullptr) {
+        s = __ldg(static_scale);
+        inv = __fdiv_rn(1.0f, s);
+    } else {
+        amax = block_max<THREADS>(amax, red);
+        if (amax == 0.0f) {
+            s = 1.0f;
+            inv = 1.0f;
+        } else if (scale_mode == W4A8_SCALE_POW2) {
+            s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
+            inv = __fdiv_rn(1.0f, s);
+        } else {
+            s = __fdiv_rn(amax, kE4M3Max);
+            inv = __fdiv_rn(kE4M3Max, amax);
+        }
+    }
+    if (threadIdx.x == 0) s_x[row] = s;
+    uint4* dst = reinterpret_cast<uint4*>(x8 + row * ldx8);
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = threadIdx.x + i * THREADS;
+        if (c < nchunks) {
+            uint2 a = quant_bf16x8(v[i][0], inv);
+            uint2 b = quant_bf16x8(v[i][1], inv);
+            dst[c] = make_uint4(a.x, a.y, b.x, b.y);
+        }
+    }
+}
+
 // Any K: the row is read twice (second read served by L2).
 __global__ void __launch_bounds__(256)
 act_quant_kernel_2pass(const uint16_t* __restrict__ x, int64_t K, int64_t ldx,

@@ -666,6 +666,80 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
     return out
 
 
+def mlp_sweep(torch, binding, inputs, dev, peaks):
+    """The MLP block of a Llama-3-8B decoder layer at decode sizes, all on the W4A8 path:
+    quantize_act(x) -> stacked gate/up projection (K = 4096 -> N = 2 x 14336) -> silu(gate) * up fused
+    with the activation quantization of the next layer (w4a8_silu_mul_quantize) -> down projection
+    (K = 14336 -> N = 4096).  Per token count: the block time from CUDA graphs of consecutive blocks
+    on rotating weight copies (more than twice the L2), the same block with the activation written as
+    BF16 and quantized by a separate launch, and the BF16 library block (two torch.matmul + silu * mul)."""
+    H, F = 4096, 14336
+    out = []
+    side = torch.cuda.Stream()
+
+    def graph_time(fn, reps):
+        fn(0)
+        torch.cuda.synchronize()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for c in range(reps):
+                    fn(c)
+        torch.cuda.current_stream().wait_stream(side)
+        return _time_loop(torch, g.replay, 5, warm=2) / reps
+
+    copies = 4   # 4 x (60.6 + 30.3) MB of packed weights > 2 x 126 MB
+    gus, downs = [], []
+    for c in range(copies):
+        W = torch.from_numpy(inputs.make_weight(2 * F, H, SIGMA, seed=9100 + c)).to(dev)
+        gus.append(binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True)))
+        del W
+        W = torch.from_numpy(inputs.make_weight(H, F, SIGMA, seed=9200 + c)).to(dev)
+        downs.append(binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True)))
+        del W
+    wbytes = (2 * F * H + H * F) * (0.5 + 2.0 / GROUP)
+    wg_bf = torch.randn((2 * F, H), dtype=torch.bfloat16, device=dev) * SIGMA
+    wd_bf = torch.randn((H, F), dtype=torch.bfloat16, device=dev) * SIGMA
+    for m in (1, 4, 16):
+        x = torch.from_numpy(inputs.make_activation(m, H, 77 + m, OUTLIER_FRAC, OUTLIER_MULT)).to(dev).view(torch.bfloat16)
+        x8, s_x = binding.quantize_act(x)
+        gu = torch.empty((m, 2 * F), dtype=torch.bfloat16, device=dev)
+        h8 = torch.empty((m, F), dtype=torch.uint8, device=dev)
+        s_h = torch.empty((m,), dtype=torch.float32, device=dev)
+        hbf = torch.empty((m, F), dtype=torch.bfloat16, device=dev)
+        y = torch.empty((m, H), dtype=torch.bfloat16, device=dev)
+        ws1 = binding.new_workspace(m, 2 * F, H, gus[0].fmt, dev)
+        ws2 = binding.new_workspace(m, H, F, downs[0].fmt, dev)
+
+        def block(c):
+            binding.quantize_act(x, out=(x8, s_x))
+            binding.linear_tiled(x8, s_x, gus[c % copies], out=gu, workspace=ws1)
+            binding.silu_mul_quantize(gu, out=(h8, s_h))
+            binding.linear_tiled(h8, s_h, downs[c % copies], out=y, workspace=ws2)
+
+        def block_unfused(c):
+            binding.quantize_act(x, out=(x8, s_x))
+            binding.linear_tiled(x8, s_x, gus[c % copies], out=gu, workspace=ws1)
+            torch.mul(torch.nn.functional.silu(gu[:, :F]), gu[:, F:], out=hbf)
+            binding.quantize_act(hbf, out=(h8, s_h))
+            binding.linear_tiled(h8, s_h, downs[c % copies], out=y, workspace=ws2)
+
+        def block_bf16(c):
+            g2 = torch.matmul(x, wg_bf.t())
+            torch.matmul(torch.nn.functional.silu(g2[:, :F]) * g2[:, F:], wd_bf.t())
+
+        t = graph_time(block, 2 * copies)
+        t_u = graph_time(block_unfused, 2 * copies)
+        t_b = graph_time(block_bf16, 4)
+        if binding.query_device_status() != 0:
+            raise RuntimeError("device status word set")
+        out.append({"M": m, "block_us": t * 1e6, "block_unfused_activation_us": t_u * 1e6,
+                    "weight_GBps": wbytes / t / 1e9, "frac_hbm_measured": wbytes / t / 1e9 / peaks["hbm_gbs"],
+                    "library_bf16_block_us": t_b * 1e6})
+    return out
+
+
 def scheme_sweep(torch, binding, inputs, dev):
     """Same-box counterpart of the paper's scheme comparison (Sec. 4.3, Fig. 4, Table 3): per layer
     and token count the time of W4A8 as built here (group-aware order: groups are runs of columns),
@@ -789,7 +863,7 @@ def main():
                     help="consecutive steps captured in one CUDA graph (used when it divides --steps; default 4)")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
-    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes"],
+    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes", "mlp"],
                     help="instead of the bench line, print the per-layer table of config c5 (four Llama-3-8B "
                          "linears x M) or the single c4 case (M=8192, K=8192, N=28672)")
     args = ap.parse_args()
@@ -810,6 +884,8 @@ def main():
             rows = dpq_sweep(torch, binding, inputs, dev)
         elif args.sweep == "schemes":
             rows = scheme_sweep(torch, binding, inputs, dev)
+        elif args.sweep == "mlp":
+            rows = mlp_sweep(torch, binding, inputs, dev, load_peaks())
         elif args.sweep == "c5":
             rows = layer_sweep(torch, binding, inputs, dev, load_peaks())
         else:

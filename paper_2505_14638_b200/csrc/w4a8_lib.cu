@@ -676,35 +676,44 @@ static int silu_mul_quantize_impl(const void* gu, int64_t M, int64_t F, int64_t 
     if (!gu || !x8 || !s_x) return W4A8_ERR_INVALID_ARG;
     if (M <= 0 || F <= 0) return W4A8_ERR_INVALID_ARG;
     if (scale_mode != W4A8_SCALE_EXACT && scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
-    if (F % 16 != 0 || F > 16384 || ldgu < 2 * F || ldx8 < F || (h_out && ldh < F) || M > INT32_MAX)
+    if (F % 16 != 0 || F > 16384 || ldgu < 2 * F || ldx8 < F || (h_out && ldh < F) || M > INT32_MAX / 8)
         return W4A8_ERR_BAD_SHAPE;
     if (!aligned16(gu) || !aligned16(x8) || (ldgu % 8) != 0 || (ldx8 % 16) != 0 ||
         (reinterpret_cast<uintptr_t>(s_x) & 3u) || (h_out && (!aligned16(h_out) || (ldh % 8) != 0)))
         return W4A8_ERR_BAD_ALIGNMENT;
     int rc = check_device();
     if (rc != W4A8_OK) return rc;
-    cudaLaunchAttribute pdl[1];
-    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    const int64_t nchunks = F / 16;
+    // CTAs (one cluster) per token, 128 chunks each
+    const int cl = nchunks <= 128 ? 1 : (nchunks <= 256 ? 2 : (nchunks <= 512 ? 4 : 8));
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[0].val.programmaticStreamSerializationAllowed = 1;
+    attrs[1].id = cudaLaunchAttributeClusterDimension;
+    attrs[1].val.clusterDim.x = (unsigned)cl;
+    attrs[1].val.clusterDim.y = 1;
+    attrs[1].val.clusterDim.z = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)M);
-    cfg.blockDim = dim3(256);
+    cfg.gridDim = dim3((unsigned)(M * cl));
+    cfg.blockDim = dim3(128);
     cfg.stream = st;
-    cfg.attrs = pdl;
-    cfg.numAttrs = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = cl > 1 ? 2 : 1;
     const uint16_t* g = static_cast<const uint16_t*>(gu);
     uint16_t* h = static_cast<uint16_t*>(h_out);
-    const int64_t nchunks = F / 16;
     cudaError_t lerr;
-    if (nchunks <= 256)
-        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 1>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
-                                  static_scale, h, ldh);
-    else if (nchunks <= 512)
-        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 2>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
-                                  static_scale, h, ldh);
+    if (cl == 1)
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<1>, g, F, ldgu, x8, ldx8, s_x, scale_mode, static_scale,
+                                  h, ldh);
+    else if (cl == 2)
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<2>, g, F, ldgu, x8, ldx8, s_x, scale_mode, static_scale,
+                                  h, ldh);
+    else if (cl == 4)
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<4>, g, F, ldgu, x8, ldx8, s_x, scale_mode, static_scale,
+                                  h, ldh);
     else
-        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<256, 4>, g, F, ldgu, x8, ldx8, s_x, scale_mode,
-                                  static_scale, h, ldh);
+        lerr = cudaLaunchKernelEx(&cfg, silu_mul_quant_kernel<8>, g, F, ldgu, x8, ldx8, s_x, scale_mode, static_scale,
+                                  h, ldh);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (lerr != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();

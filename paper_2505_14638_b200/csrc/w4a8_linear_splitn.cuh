@@ -177,6 +177,21 @@ __device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
     }
 }
 
+// A candidate that declined keeps its place on the SM until every worker index has been handed
+// out (bounded: a fraction of a millisecond).  If it left at once, the hardware would put the
+// next waiting candidate into the same place, on an SM that already has its worker, and that
+// one would decline too: on SMs with two free places (the previous launch had fewer workers than
+// there are SMs) the whole surplus of candidates burnt away like this before the other SMs had
+// room, and the last ones were then forced to work as second workers after all.
+__device__ __forceinline__ void sched_hold(SchedSlot* sl, int workers) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (*reinterpret_cast<volatile unsigned int*>(&sl->issued) < (unsigned)workers &&
+           *reinterpret_cast<volatile unsigned int*>(&sl->finished) != 0u &&
+           ptx::globaltimer_ns() - t0 < 200000ull) {
+        __nanosleep(500);
+    }
+}
+
 // Arguments of the fused activation quantization (unused otherwise).
 struct SnFuse {
     const uint16_t* x;          // BF16 activations [M][ldx]
@@ -342,7 +357,11 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         p = worker_s;
         P = plan.P;
         if (p < 0) {  // a worker of this launch is already on this SM: retire
-            if (threadIdx.x == 0) sched_entered(&g_sched[plan.sched], (int)gridDim.x);
+            if (threadIdx.x == 0) {
+                ptx::griddep_launch_dependents();
+                sched_entered(&g_sched[plan.sched], (int)gridDim.x);
+                sched_hold(&g_sched[plan.sched], plan.P);
+            }
             return;
         }
         if (threadIdx.x == 64) sched_entered(&g_sched[plan.sched], (int)gridDim.x);  // an idle epilogue thread

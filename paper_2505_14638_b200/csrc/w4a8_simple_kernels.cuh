@@ -128,7 +128,7 @@ act_quant_kernel(const uint16_t* __restrict__ x, int64_t K, int64_t ldx, uint8_t
 // gate (first F values) and up (next F values), as the output of a linear layer whose weight
 // stacks the gate and up projections;  h = BF16( silu(gate) * up ),  silu(g) = g / (1 + exp(-g)),
 // all in fp32 (division and multiplications correctly rounded, expf from the math library), then
-// h is quantized per token exactly as act_quant_kernel does.  One CTA per token; F <= THREADS*NCH*16.
+// h is quantized per token exactly as act_quant_kernel does.
 // The BF16 round trip through memory between the two linear layers of the block is saved.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t silu_mul_bf16x2(uint32_t g2, uint32_t u2) {
@@ -140,38 +140,43 @@ __device__ __forceinline__ uint32_t silu_mul_bf16x2(uint32_t g2, uint32_t u2) {
            ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(h1)) << 16);
 }
 
-template <int THREADS, int NCH>
-__global__ void __launch_bounds__(THREADS)
+// CL CTAs (one thread-block cluster) share a token: each takes a contiguous part of the row and
+// the row maximum is exchanged through distributed shared memory, so that the CTAs stay small
+// (128 threads, one 16-element chunk per thread: several of them must fit on an SM beside the CTAs
+// of the two linear layers around them) however long the row is.  F <= CL * 128 * 16.
+template <int CL>
+__global__ void __launch_bounds__(128)
 silu_mul_quant_kernel(const uint16_t* __restrict__ gu, int64_t F, int64_t ldgu, uint8_t* __restrict__ x8,
                       int64_t ldx8, float* __restrict__ s_x, int scale_mode,
                       const float* __restrict__ static_scale, uint16_t* __restrict__ h_out, int64_t ldh) {
     __shared__ float red[32];
+    __shared__ float part_max[CL];
     ptx::griddep_launch_dependents();
     ptx::griddep_wait();
-    const int64_t row = blockIdx.x;
+    uint32_t rank = 0;
+    if constexpr (CL > 1) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int64_t row = blockIdx.x / CL;
     const int nchunks = (int)(F >> 4);
-    const uint4* gsrc = reinterpret_cast<const uint4*>(gu + row * ldgu);
-    const uint4* usrc = reinterpret_cast<const uint4*>(gu + row * ldgu + F);
-    uint4 v[NCH][2];
+    const int c = (int)rank * 128 + (int)threadIdx.x;  // this thread's chunk of the row
+    const bool have = c < nchunks;
+    uint4 v[2];
     float amax = 0.0f;
+    if (have) {
+        const uint4* gsrc = reinterpret_cast<const uint4*>(gu + row * ldgu);
+        const uint4* usrc = reinterpret_cast<const uint4*>(gu + row * ldgu + F);
 #pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        int c = threadIdx.x + i * THREADS;
-        if (c < nchunks) {
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const uint4 g = __ldg(gsrc + 2 * c + hh), u = __ldg(usrc + 2 * c + hh);
-                v[i][hh].x = silu_mul_bf16x2(g.x, u.x);
-                v[i][hh].y = silu_mul_bf16x2(g.y, u.y);
-                v[i][hh].z = silu_mul_bf16x2(g.z, u.z);
-                v[i][hh].w = silu_mul_bf16x2(g.w, u.w);
-                amax = absmax_bf16x8(v[i][hh], amax);
-            }
-            if (h_out != nullptr) {
-                uint4* hd = reinterpret_cast<uint4*>(h_out + row * ldh);
-                hd[2 * c] = v[i][0];
-                hd[2 * c + 1] = v[i][1];
-            }
+        for (int hh = 0; hh < 2; ++hh) {
+            const uint4 g = __ldg(gsrc + 2 * c + hh), u = __ldg(usrc + 2 * c + hh);
+            v[hh].x = silu_mul_bf16x2(g.x, u.x);
+            v[hh].y = silu_mul_bf16x2(g.y, u.y);
+            v[hh].z = silu_mul_bf16x2(g.z, u.z);
+            v[hh].w = silu_mul_bf16x2(g.w, u.w);
+            amax = absmax_bf16x8(v[hh], amax);
+        }
+        if (h_out != nullptr) {
+            uint4* hd = reinterpret_cast<uint4*>(h_out + row * ldh);
+            hd[2 * c] = v[0];
+            hd[2 * c + 1] = v[1];
         }
     }
     float s, inv;
@@ -179,7 +184,20 @@ silu_mul_quant_kernel(const uint16_t* __restrict__ gu, int64_t F, int64_t ldgu, 
         s = __ldg(static_scale);
         inv = __fdiv_rn(1.0f, s);
     } else {
-        amax = block_max<THREADS>(amax, red);
+        amax = block_max<128>(amax, red);
+        if constexpr (CL > 1) {
+            // every CTA of the cluster receives every CTA's maximum
+            if (threadIdx.x < CL) {
+                uint32_t remote;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                             : "=r"(remote)
+                             : "r"(ptx::smem_addr(&part_max[rank])), "r"((uint32_t)threadIdx.x));
+                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(amax) : "memory");
+            }
+            asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+            for (int i = 0; i < CL; ++i) amax = fmaxf(amax, part_max[i]);
+        }
         if (amax == 0.0f) {
             s = 1.0f;
             inv = 1.0f;
@@ -191,16 +209,12 @@ silu_mul_quant_kernel(const uint16_t* __restrict__ gu, int64_t F, int64_t ldgu, 
             inv = __fdiv_rn(kE4M3Max, amax);
         }
     }
-    if (threadIdx.x == 0) s_x[row] = s;
-    uint4* dst = reinterpret_cast<uint4*>(x8 + row * ldx8);
-#pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        int c = threadIdx.x + i * THREADS;
-        if (c < nchunks) {
-            uint2 a = quant_bf16x8(v[i][0], inv);
-            uint2 b = quant_bf16x8(v[i][1], inv);
-            dst[c] = make_uint4(a.x, a.y, b.x, b.y);
-        }
+    if (threadIdx.x == 0 && rank == 0) s_x[row] = s;
+    if (have) {
+        uint4* dst = reinterpret_cast<uint4*>(x8 + row * ldx8);
+        uint2 a = quant_bf16x8(v[0], inv);
+        uint2 b = quant_bf16x8(v[1], inv);
+        dst[c] = make_uint4(a.x, a.y, b.x, b.y);
     }
 }
 

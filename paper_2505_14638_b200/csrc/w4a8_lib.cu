@@ -4,11 +4,13 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/w4a8.h"
 #include "w4a8_dpq_kernels.cuh"
 #include "w4a8_linear_splitn.cuh"
+#include "w4a8_linear_pair.cuh"
 #include "w4a8_linear_streamk.cuh"
 #include "w4a8_linear_umma.cuh"
 #include "w4a8_simple_kernels.cuh"
@@ -399,6 +401,62 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
     return launch_status();
 }
 
+// The two-CTA kernel takes whole tiles of 256 output channels x 256 tokens, one CTA pair per tile
+// and round.  Each CTA of a pair loads half of the activation tile (24.6 KB per step and SM
+// instead of 41 KB, six ring stages instead of four), but the pair pays for it with remote
+// barrier traffic and coarser tiles.  Measured against the one-CTA persistent kernel (us):
+//   (M, N, K) = (8192, 28672, 8192): 1882 vs 2033;  (2048, 28672, 4096): 241 vs 254;
+//   (1024, 28672, 4096): 133 vs 150;  (4096, 4096, 14336): 254 vs 255;
+//   (4096, 28672, 4096): 459 vs 438;  (8192, 8192, 8192): 536 vs 523;
+//   (4096, 6144, 4096): 113 vs 99;  (4096, 4096, 4096): 77 vs 66;  (2048, 4096, 4096): 42 vs 36.
+// It is used where it won: many output channels, and either few token tiles or a long K.
+static bool pair_kernel_applies(int64_t M, int64_t N, int64_t K, int sms) {
+    if (N % 256 != 0 || N < 16384 || M < 1024 || K < 1024) return false;
+    if (!(M <= 2048 || K >= 8192)) return false;
+    const int64_t tiles = (N / 256) * ((M + 255) / 256);
+    return tiles >= 4 * (int64_t)(sms / 2);
+}
+
+template <class Cfg>
+static int launch_pair(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, const float* s_x, const float* s_w,
+                       int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, int sms,
+                       cudaStream_t st) {
+    auto kern = linear_pair_kernel<Cfg>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    unsigned int* status = status_word_ptr();
+    if (!status) return W4A8_ERR_CUDA;
+    CUtensorMap tx;  // this CTA's half of an activation tile: 128 tokens x 128 bytes
+    if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    const int TM = (M + 255) / 256, TN2 = N / 256;
+    int pairs = sms / 2;
+    if (pairs > TM * TN2) pairs = TM * TN2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(Cfg::kThreads);
+    cfg.dynamicSmemBytes = (size_t)Cfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, TM, TN2,
+                                       status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) return W4A8_ERR_CUDA;
+    return launch_status();
+}
+
 static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* wpp,
                              int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
                              int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
@@ -440,6 +498,12 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     if (rc != W4A8_OK) return rc;
     const int sms = sm_count();
     if (sms <= 0) return W4A8_ERR_CUDA;
+    if (pair_kernel_applies(M, N, K, sms))
+        return fmt == kFmtTiledSignMag
+                   ? launch_pair<PairCfg<4, 6, 4, kFmtTiledSignMag>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                                                      (int)M, (int)N, (int)K, sms, st)
+                   : launch_pair<PairCfg<4, 6, 4, kFmtTiled>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                                               (int)M, (int)N, (int)K, sms, st);
     make_sk_plan(M, N, K, sms, &pl);
     CUtensorMap tx;
     if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)pl.bnx,

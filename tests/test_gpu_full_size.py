@@ -12,8 +12,8 @@ import pytest
 import torch
 
 import oracle
-from gpu_utils import bf16_bits, bf16_dev
-from helpers import bf16_gate
+from gpu_utils import bf16_bits, bf16_dev, weights_to_dev
+from helpers import bf16_gate, fp32_gate
 from paper_2505_14638_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
@@ -75,3 +75,41 @@ def test_config_c5_layers_sampled_channels(name, K, N, M):
     # c5: the four Llama-3-8B linears; token counts that reach the split-N kernel (<= 64), the
     # persistent kernel with shared tiles (128, 512) and with whole tiles (4096)
     _run_case(M, N, K, 0.02, 0.01, 20.0, seed=500 + M + N // 64, n_random=40)
+
+
+def test_two_cta_kernel_shape_exact_integers_and_gaussian():
+    """A shape that the two-CTA kernel takes (many output channels, few token tiles), with a
+    ragged token count: small-integer inputs make the FP32 accumulation exact, so any operand
+    that lands in the wrong row, token half or k-slice changes the result visibly; then Gaussian inputs
+    within the usual gates.  Sampled output channels (all 128-row blocks are hit)."""
+    M, N, K = 1061, 16384, 1024
+    rng = np.random.default_rng(17)
+    cols = np.unique(np.concatenate([rng.integers(0, N, 700), np.arange(0, N, 128), np.arange(127, N, 128)]))
+    for exact in (True, False):
+        if exact:
+            codes, gscale, gzero = inputs.random_codes(N, K, 5, scale_bits=0x3F80)       # group scale 1.0
+            s_w = np.array([1.0], dtype=np.float32)
+            xb = inputs.make_small_int_activation(M, K, 6)
+        else:
+            W = inputs.make_weight(N, K, 0.02, 23)
+            codes, gscale, gzero, s_w = oracle.quantize_weight_rtn(W, symmetric=True)
+            xb = inputs.make_activation(M, K, 24, 0.01, 20.0)
+        x8_ref, s_x_ref = oracle.quantize_act(xb)
+        w8 = oracle.dequant_weight(codes, gscale, gzero)
+        ref = oracle.linear(x8_ref, s_x_ref, w8, s_w, cols=cols, want=("y64",))
+        # random codes include 0 (= -8), which only the generic tiled format can hold
+        fmt = binding.FMT_TILED if exact else binding.FMT_TILED_SIGNMAG
+        tw = binding.prepack_weight(*weights_to_dev(codes, gscale, gzero, s_w), weight_format=fmt)
+        x8, s_x = binding.quantize_act(bf16_dev(xb))
+        y = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32)
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0
+        got = y.cpu().numpy()[:, cols]
+        if exact:
+            # the integer dot products are exact in FP32; what remains is the rounding of the two scale
+            # multiplications (s_x = amax / 448 is not a power of two): a misplaced operand would change
+            # a sum by at least one unit, i.e. by 1/112 here
+            assert np.all(np.abs(got.astype(np.float64) - ref["y64"]) <= 4e-7 * np.abs(ref["y64"]) + 1e-6)
+        else:
+            worst, _ = fp32_gate(got, ref["y64"], rel=2e-3)
+            assert worst <= 2e-3, worst

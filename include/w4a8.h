@@ -102,13 +102,17 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * gscale_bf16 / gzero) or a tiled format (weights = buffer written by w4a8_prepack_weight;
  * gscale_bf16 and gzero are ignored and may be NULL).
  * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs (they are
- * added in a fixed order: results repeat bit for bit).  Decode-sized calls (M <= 64) on tiled
+ * added in a fixed order: results repeat bit for bit).  Calls with M <= 128 on tiled
  * weights use it only for layers with few output channels and run without it, somewhat slower,
  * when it is NULL or too small; larger M requires it.  It
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
  * its first use; every call leaves it ready for the next one.  Calls that share a workspace
  * must not overlap on the device.
+ * Calls with M <= 16 on tiled weights place their worker CTAs at run time (at most one per SM and
+ * launch, so that consecutive launches can share the SMs); the bookkeeping is a table of 64
+ * entries that is part of the library image, handed out round-robin per call and cleared by the
+ * kernel: up to 64 such launches may be in flight on a device at a time.
  */
 int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* weights,
                 const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w,

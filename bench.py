@@ -307,7 +307,9 @@ def run_ours(args, rank, world, local_rank):
     # decode graph holds the layers of a whole forward pass; one graph per phase of the weight
     # rotation.  Every step still runs all its launches on weights that come from HBM.
     use_graph = not args.no_graph
-    spg = args.steps_per_graph if (use_graph and args.steps % args.steps_per_graph == 0) else 1
+    spg = 1
+    if use_graph:  # the largest count up to the one asked for that divides the number of steps
+        spg = max(d for d in range(1, max(1, args.steps_per_graph) + 1) if args.steps % d == 0)
     period = WEIGHT_COPIES
     g_full, g_lin, g_quant = [], [], None
     if use_graph:
@@ -859,8 +861,8 @@ def main():
     ap.add_argument("--two-kernel", action="store_true",
                     help="step = w4a8_quantize_act + w4a8_linear per M instead of the fused launch")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
-    ap.add_argument("--steps-per-graph", type=int, default=4,
-                    help="consecutive steps captured in one CUDA graph (used when it divides --steps; default 4)")
+    ap.add_argument("--steps-per-graph", type=int, default=8,
+                    help="consecutive steps captured in one CUDA graph (the largest divisor of --steps up to this; default 8)")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
     ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes", "mlp"],

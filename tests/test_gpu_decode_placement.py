@@ -67,3 +67,31 @@ def test_many_launches_repeat_the_first_result():
         for o, f in zip(outs, first):
             assert torch.equal(o, f), rep
     assert binding.query_device_status() == 0
+
+
+def test_two_streams_issue_decode_launches_concurrently():
+    # launches of two streams overlap on the device and share the placement table (different slots)
+    a = _case(8, 14336, 4096, 11)
+    b = _case(16, 18960, 2048, 13)
+    outs = [torch.empty((c[1].shape[0], c[0].N), dtype=torch.float32, device="cuda") for c in (a, b)]
+    first = []
+    for (tw, x8, s_x, y64, ws), out in zip((a, b), outs):
+        binding.linear_tiled(x8, s_x, tw, out=out, out_dtype=binding.OUT_FP32, workspace=ws)
+        torch.cuda.synchronize()
+        worst, _ = fp32_gate(out.cpu().numpy(), y64, rel=2e-3)
+        assert worst <= 2e-3, worst
+        first.append(out.clone())
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for s in streams:
+        s.wait_stream(torch.cuda.current_stream())
+    for rep in range(40):
+        for i, (case, s) in enumerate(zip((a, b), streams)):
+            tw, x8, s_x, _, ws = case
+            with torch.cuda.stream(s):
+                binding.linear_tiled(x8, s_x, tw, out=outs[i], out_dtype=binding.OUT_FP32, workspace=ws)
+    for s in streams:
+        torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    for o, f in zip(outs, first):
+        assert torch.equal(o, f)
+    assert binding.query_device_status() == 0

@@ -196,6 +196,21 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
 /*
+ * W4A16 comparison scheme (Sec. 4.3, Fig. 4): activations stay BF16, the INT4 codes are expanded
+ * to BF16 on the fly and multiplied with BF16 tensor-core MMAs, FP32 accumulation:
+ *   W16[n][k] = BF16( (u[n][k] - z[n][g]) * s_g[n][g] )      (one rounding to nearest even),
+ *   Y[m][n]   = s_w[n*sw_stride] * sum_k X[m][k] * W16[n][k],  rounded to BF16 or kept in FP32.
+ * The stored weights are those of the W4A8 path (canonical format: codes, BF16 group scales,
+ * zero-points or NULL for z = 8, s_w per channel or per tensor), so the two schemes can be timed on
+ * the same quantized layer; only the arithmetic of the multiplication differs.
+ *   x_bf16 device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned); K % 128 == 0, N % 16 == 0.
+ * One tile per CTA, no workspace.  Errors as w4a8_linear.
+ */
+int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* codes,
+                      const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride,
+                      int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* stream);
+
+/*
  * Gated-MLP activation fused with the activation quantization of the next linear layer (the
  * paper quantizes the BF16 activations that enter a linear layer, Eq. 13; in a Llama MLP block
  * those of the down projection are silu(gate) * up, computed from the output of the stacked

@@ -268,6 +268,35 @@ def quantize_act(x_bf16, scale_mode=0, static_scale=None):
     return x8, s_x
 
 
+def dequant_weight_bf16(codes, gscale, gzero=None, group=128) -> np.ndarray:
+    """W4A16 comparison scheme (Sec. 4.3): W16 = BF16_RNE((u - z) * s_g), the product formed exactly
+    (a small integer times a BF16 value) and rounded once.  Returns BF16 bit patterns uint16 [N, K]."""
+    codes = _c(codes, np.uint8)
+    N, Kh = codes.shape
+    K = 2 * Kh
+    u = np.empty((N, K), dtype=np.int64)
+    u[:, 0::2] = codes & 0x0F
+    u[:, 1::2] = codes >> 4
+    s = bf16_to_f32(_c(gscale, np.uint16)).astype(np.float64)           # [N, K/group]
+    z = np.full(s.shape, 8, dtype=np.int64) if gzero is None else _c(gzero, np.uint8).astype(np.int64)
+    prod = (u - np.repeat(z, group, axis=1)).astype(np.float64) * np.repeat(s, group, axis=1)
+    return f64_to_bf16(prod)
+
+
+def linear_w4a16(x_bf16, w16_bf16, s_w, cols=None) -> np.ndarray:
+    """Y = s_w * X W16^T in double precision (every BF16 x BF16 product is exact in double; the sum of
+    K of them is rounded at the 53rd bit at worst).  Returns float64 [M, N or len(cols)]."""
+    x = bf16_to_f32(_c(x_bf16, np.uint16)).astype(np.float64)
+    w = bf16_to_f32(_c(w16_bf16, np.uint16)).astype(np.float64)
+    s_w = _c(s_w, np.float32).astype(np.float64)
+    if cols is not None:
+        w = w[np.asarray(cols)]
+        sw = s_w if s_w.size == 1 else s_w[np.asarray(cols)]
+    else:
+        sw = s_w
+    return (x @ w.T) * (sw[None, :] if sw.size > 1 else sw[0])
+
+
 def silu_mul_f64(gate_up_bf16) -> np.ndarray:
     """The gated-MLP activation by its definition, in double precision:
     h = silu(G) * U, silu(g) = g / (1 + exp(-g)); G = first half of each row, U = second half.

@@ -40,6 +40,20 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     return d;
 }
 
+// Two BF16 lanes: (x - off) * sc, the subtraction exact for the small integers it is used on, the
+// product rounded once to nearest even.
+__device__ __forceinline__ uint32_t bf16x2_sub_mul(uint32_t x, uint32_t off, uint32_t sc) {
+    uint32_t d;
+    asm("{\n\t"
+        ".reg .b32 t;\n\t"
+        "sub.rn.bf16x2 t, %1, %2;\n\t"
+        "mul.rn.bf16x2 %0, t, %3;\n\t"
+        "}\n"
+        : "=r"(d)
+        : "r"(x), "r"(off), "r"(sc));
+    return d;
+}
+
 // Eq. 10 as a 16-entry table for one (row, group): entry u holds nearest_E4M3((u - z) * s).
 // (u - z) is a small integer and s a BF16 value, so the fp32 product is exact and the table
 // entry is the exact product rounded once -- the same bits as converting element by element.

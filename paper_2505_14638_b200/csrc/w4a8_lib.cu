@@ -651,6 +651,45 @@ static int linear_w8a8_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, i
     return rc;
 }
 
+// W4A16 comparison path (Sec. 4.3): BF16 activations, INT4 codes expanded to BF16 in the kernel,
+// kind::f16 MMAs; canonical weights, one tile per CTA.
+static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_t* codes, const void* gscale,
+                             const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y,
+                             int64_t ldy, int out_dtype, cudaStream_t st) {
+    if (!x || !codes || !gscale || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
+    if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
+    if (K % kGroup != 0 || N % 16 != 0 || ldx < K || ldy < N) return W4A8_ERR_BAD_SHAPE;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX / 2) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(x) || !aligned16(codes) || !aligned16(y) || (ldx % 8) != 0 || (K / 2) % 16 != 0)
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int bnx = M <= 16 ? 16 : (M <= 64 ? 64 : 128);
+    CUtensorMap tw, tx;
+    if (!make_tmap_u8_2d(&tw, codes, (uint64_t)N, (uint64_t)(K / 2), (uint64_t)(K / 2), 64, 128,
+                         CU_TENSOR_MAP_SWIZZLE_64B))
+        return W4A8_ERR_CUDA;
+    // X as bytes: rows of 2 K bytes, panels of 128 bytes (64 BF16 values)
+    if (!make_tmap_u8_2d(&tx, x, (uint64_t)M, (uint64_t)(2 * K), (uint64_t)(2 * ldx), 128, (uint32_t)bnx,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    const uint16_t* gs = static_cast<const uint16_t*>(gscale);
+    const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+    switch (bnx) {
+        case 16:
+            return launch_umma<UmmaCfg<16, 4, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
+                                                             out_dtype, nullptr, Mi, Ni, Ki, 1, st);
+        case 64:
+            return launch_umma<UmmaCfg<64, 3, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
+                                                             out_dtype, nullptr, Mi, Ni, Ki, 1, st);
+        default:
+            return launch_umma<UmmaCfg<128, 3, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
+                                                              out_dtype, nullptr, Mi, Ni, Ki, 1, st);
+    }
+}
+
 static int linear_fused_impl(const void* x, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
                              const uint8_t* wpp, int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K,
                              void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out, float* s_x_out,
@@ -911,6 +950,13 @@ int w4a8_linear_w8a8(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t 
                      void* workspace, size_t workspace_bytes, void* stream) {
     return linear_w8a8_impl(x8, ldx8, s_x, M, w8, s_w, sw_stride, N, K, y, ldy, out_dtype, workspace,
                             workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* codes, const void* gscale_bf16,
+                      const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y,
+                      int64_t ldy, int out_dtype, void* stream) {
+    return linear_w4a16_impl(x_bf16, ldx, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, y, ldy, out_dtype,
+                             static_cast<cudaStream_t>(stream));
 }
 
 int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {

@@ -19,16 +19,20 @@ namespace w4a8 {
 
 // W8_ = true: the weights are FP8 E4M3 bytes already (the W8A8 comparison scheme of Sec. 4.3): the
 // TMA tile of 128 rows x 128 bytes lands directly in the swizzled MMA operand, nothing is expanded.
-template <int BNX_, int STAGES_, bool W8_ = false>
+// W16_ = true: the W4A16 comparison scheme of Sec. 4.3: activations stay BF16, the INT4 codes are
+// expanded to BF16 (u - z) * s_g, rounded once, and multiplied with kind::f16 MMAs (K = 16 each);
+// a k-block of 128 is then two swizzled 128-byte panels of 64 elements per operand.
+template <int BNX_, int STAGES_, bool W8_ = false, bool W16_ = false>
 struct UmmaCfg {
     static constexpr bool W8 = W8_;
+    static constexpr bool W16 = W16_;
     static constexpr int BNX = BNX_;        // tokens per tile (MMA N)
     static constexpr int STAGES = STAGES_;
     static constexpr int BW = 128;          // weight rows per tile (MMA M)
     static constexpr int BK = 128;          // K per pipeline stage = one quantization group
     static constexpr int kWpBytes = BW * BK / 2;   // packed codes
-    static constexpr int kW8Bytes = BW * BK;       // dequantized E4M3
-    static constexpr int kXBytes = BNX * BK;       // FP8 activations
+    static constexpr int kW8Bytes = BW * BK * (W16_ ? 2 : 1);   // dequantized E4M3 (BF16)
+    static constexpr int kXBytes = BNX * BK * (W16_ ? 2 : 1);   // FP8 (BF16) activations
     static constexpr int kStageBytes = kWpBytes + kW8Bytes + kXBytes;
     static constexpr int kBarBytes = 256;
     static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 1024;  // + alignment slack
@@ -115,7 +119,13 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                     ptx::mbar_arrive_expect_tx(bar_full_tma(s), (uint32_t)(Cfg::kWpBytes + Cfg::kXBytes));
                     ptx::tma_load_2d(stage_wp(s), &tmap_w, (kb0 + it) * 64, n0, bar_full_tma(s));
                 }
-                ptx::tma_load_2d(stage_x(s), &tmap_x, (kb0 + it) * 128, m0, bar_full_tma(s));
+                if (Cfg::W16) {  // X as bytes: two panels of 64 BF16 values per k-block
+                    ptx::tma_load_2d(stage_x(s), &tmap_x, (kb0 + it) * 256, m0, bar_full_tma(s));
+                    ptx::tma_load_2d(stage_x(s) + (uint32_t)(BNX * 128), &tmap_x, (kb0 + it) * 256 + 128, m0,
+                                     bar_full_tma(s));
+                } else {
+                    ptx::tma_load_2d(stage_x(s), &tmap_x, (kb0 + it) * 128, m0, bar_full_tma(s));
+                }
                 issued = it + 1;
             }
             if (!ok) {
@@ -132,7 +142,8 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, BNX);
+            constexpr uint32_t idesc =
+                Cfg::W16 ? ptx::umma_idesc_bf16_f32(128, BNX) : ptx::umma_idesc_e4m3_f32(128, BNX);
             bool ok = true;
             for (int it = 0; it < nkb && ok; ++it) {
                 const int s = it % STAGES;
@@ -141,11 +152,22 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                      (Cfg::W8 || ptx::mbar_wait(bar_w8_full(s), ph, abort_flag, status_word));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
+                if (Cfg::W16) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint64_t adesc = ptx::umma_desc_k_sw128(stage_w8(s) + 32u * k);
-                    const uint64_t bdesc = ptx::umma_desc_k_sw128(stage_x(s) + 32u * k);
-                    ptx::umma_f8(tmem_base, adesc, bdesc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < 8; ++k) {  // panel k / 4, K = 16 slice k % 4 (32 bytes each)
+                        const uint32_t pa = (uint32_t)((k >> 2) * 128 * 128 + (k & 3) * 32);
+                        const uint32_t pb = (uint32_t)((k >> 2) * BNX * 128 + (k & 3) * 32);
+                        const uint64_t adesc = ptx::umma_desc_k_sw128(stage_w8(s) + pa);
+                        const uint64_t bdesc = ptx::umma_desc_k_sw128(stage_x(s) + pb);
+                        ptx::umma_bf16(tmem_base, adesc, bdesc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t adesc = ptx::umma_desc_k_sw128(stage_w8(s) + 32u * k);
+                        const uint64_t bdesc = ptx::umma_desc_k_sw128(stage_x(s) + 32u * k);
+                        ptx::umma_f8(tmem_base, adesc, bdesc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    }
                 }
                 ptx::umma_commit(bar_mma_done(s));
             }
@@ -177,6 +199,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
         for (int it = 0; it < (Cfg::W8 ? 0 : nkb); ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+            const uint32_t sc_bits = sc_next;
             const float sc = bf16_bits_to_float(sc_next);
             const int z = z_next;
             if (it + 1 < nkb && row_ok) {
@@ -184,7 +207,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                 if (z_ptr) z_next = (int)__ldg(z_ptr + it + 1);
             }
             DequantLut lut;
-            lut.build(sc, z);
+            if (!Cfg::W16) lut.build(sc, z);
             ok = ptx::mbar_wait(bar_full_tma(s), ph, abort_flag, status_word);
             if (!ok) break;
             const uint32_t src = stage_wp(s) + (uint32_t)r * 64u;
@@ -196,14 +219,39 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                              : "r"(src + (((uint32_t)j ^ sw64) << 4)));
             }
             const uint32_t dst = stage_w8(s) + (uint32_t)r * 128u;
+            if (Cfg::W16) {
+                // BF16 (128 + u) has the bit pattern 0x4300 | u: subtract 128 + z (exact), multiply by the
+                // group scale (one rounding).  Word j holds elements 8j .. 8j+7 = one 16-byte chunk.
+                const uint32_t off2 = (uint32_t)(0x4300 | z) * 0x00010001u;  // BF16 pair (128 + z, 128 + z)
+                const uint32_t sc2 = (sc_bits & 0xFFFFu) * 0x00010001u;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint32_t o0, o1, o2, o3;
-                lut.dequant8(p[2 * c], o0, o1);
-                lut.dequant8(p[2 * c + 1], o2, o3);
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)),
-                             "r"(o0), "r"(o1), "r"(o2), "r"(o3)
-                             : "memory");
+                for (int j = 0; j < 16; ++j) {
+                    uint32_t a = (p[j] & 0x000F000Fu) | 0x43004300u;           // elements 0, 4
+                    uint32_t b = ((p[j] >> 4) & 0x000F000Fu) | 0x43004300u;    // elements 1, 5
+                    uint32_t c = ((p[j] >> 8) & 0x000F000Fu) | 0x43004300u;    // elements 2, 6
+                    uint32_t d = ((p[j] >> 12) & 0x000F000Fu) | 0x43004300u;   // elements 3, 7
+                    a = bf16x2_sub_mul(a, off2, sc2);
+                    b = bf16x2_sub_mul(b, off2, sc2);
+                    c = bf16x2_sub_mul(c, off2, sc2);
+                    d = bf16x2_sub_mul(d, off2, sc2);
+                    const uint32_t o0 = prmt(a, b, 0x5410u), o1 = prmt(c, d, 0x5410u);
+                    const uint32_t o2 = prmt(a, b, 0x7632u), o3 = prmt(c, d, 0x7632u);
+                    const uint32_t panel = dst + (uint32_t)((j >> 3) * 128 * 128);
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(
+                                     panel + ((((uint32_t)j & 7u) ^ sw128) << 4)),
+                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                                 : "memory");
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t o0, o1, o2, o3;
+                    lut.dequant8(p[2 * c], o0, o1);
+                    lut.dequant8(p[2 * c + 1], o2, o3);
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)),
+                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                                 : "memory");
+                }
             }
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s));
@@ -228,7 +276,7 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                         if (partial != nullptr) {
                             partial[(int64_t)blockIdx.z * MN + (int64_t)m * N + n] = acc;
                         } else {
-                            const float res = acc * (__ldg(s_x + m) * swn);  // Eq. 4, Eq. 11
+                            const float res = acc * ((s_x != nullptr ? __ldg(s_x + m) : 1.0f) * swn);  // Eq. 4, Eq. 11
                             if (out_dtype == W4A8_OUT_FP32)
                                 reinterpret_cast<float*>(y)[(int64_t)m * ldy + n] = res;
                             else

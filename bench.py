@@ -751,7 +751,7 @@ def mlp_sweep(torch, binding, inputs, dev, peaks):
 def scheme_sweep(torch, binding, inputs, dev):
     """Same-box counterpart of the paper's scheme comparison (Sec. 4.3, Fig. 4, Table 3): per layer
     and token count the time of W4A8 as built here (group-aware order: groups are runs of columns),
-    of W8A8 (FP8 weights, own kernel and the library's FP8 GEMM) and of W4A8 quantized in an
+    of W8A8 (FP8 weights, own kernel and the library's FP8 GEMM), of W4A16 (own kernel) and of W4A8 quantized in an
     unconstrained activation order (per-column group index: the FP8 weights must be materialised
     by w4a8_dequant_weight_gidx before a W8A8 GEMM can use them).  CUDA graphs, rotating weights."""
     out = []
@@ -800,8 +800,17 @@ def scheme_sweep(torch, binding, inputs, dev):
             t_ao = graph_time(act_order, reps)
             t_lib = graph_time(lambda c: torch._scaled_mm(a8, w8s[c % copies].view(torch.float8_e4m3fn).t(),
                                                           scale_a=one, scale_b=one, out_dtype=torch.bfloat16), reps)
+
+            ws16 = torch.empty((max(binding.lib().w4a8_linear_w4a16_workspace_bytes(m, n, k), 16),),
+                               dtype=torch.uint8, device=dev)
+
+            def w4a16(c):
+                cq = raw[c % copies]
+                binding.linear_w4a16(x, cq[0], cq[1], None, cq[3], out=y, workspace=ws16)
+            t_16 = graph_time(w4a16, reps)
             out.append({"layer": name, "K": k, "N": n, "M": m, "w4a8_us": t_w4 * 1e6, "w8a8_own_kernel_us": t_w8 * 1e6,
-                        "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6})
+                        "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6,
+                        "w4a16_own_kernel_us": t_16 * 1e6})
             del x, x8, s_x, y, ws
         del tws, w8s, raw, w8_tmp
         torch.cuda.empty_cache()

@@ -195,6 +195,15 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * Needs no workspace and allocates nothing.  Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
+#define W4A8_FUSED_MAX_M 16
+/* 1 when w4a8_linear_fused is the faster way to run this problem on B200, 0 when
+ * w4a8_quantize_act + w4a8_linear is (currently always 0: see w4a8_linear_fused). */
+int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K);
+int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
+                      const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
+                      int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
+                      float* s_x_out, void* stream);
+
 /*
  * W4A16 comparison scheme (Sec. 4.3, Fig. 4): activations stay BF16, the INT4 codes are expanded
  * to BF16 on the fly and multiplied with BF16 tensor-core MMAs, FP32 accumulation:
@@ -204,11 +213,17 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * zero-points or NULL for z = 8, s_w per channel or per tensor), so the two schemes can be timed on
  * the same quantized layer; only the arithmetic of the multiplication differs.
  *   x_bf16 device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned); K % 128 == 0, N % 16 == 0.
- * One tile per CTA, no workspace.  Errors as w4a8_linear.
+ * One 128-channel tile per CTA; with few tokens and few tiles K is cut into slices whose FP32
+ * partial sums go through `workspace` (device, 16-byte aligned, at least
+ * w4a8_linear_w4a16_workspace_bytes(M, N, K) bytes, owned by the caller, may be NULL when that is
+ * 0) and are summed by a second kernel.  Errors as w4a8_linear, W4A8_ERR_WORKSPACE_TOO_SMALL
+ * included.
  */
+size_t w4a8_linear_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* codes,
                       const void* gscale_bf16, const uint8_t* gzero, const float* s_w, int sw_stride,
-                      int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* stream);
+                      int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* workspace,
+                      size_t workspace_bytes, void* stream);
 
 /*
  * Gated-MLP activation fused with the activation quantization of the next linear layer (the
@@ -230,14 +245,6 @@ int w4a8_silu_mul_quantize(const void* gate_up_bf16, int64_t M, int64_t F, int64
                            int64_t ldx8, float* s_x, int scale_mode, const float* static_scale,
                            void* h_bf16_out, int64_t ldh, void* stream);
 
-#define W4A8_FUSED_MAX_M 16
-/* 1 when w4a8_linear_fused is the faster way to run this problem on B200, 0 when
- * w4a8_quantize_act + w4a8_linear is (currently always 0: see w4a8_linear_fused). */
-int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K);
-int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
-                      const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
-                      int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
-                      float* s_x_out, void* stream);
 
 /*
  * Eq. 10 for weights quantized in an unconstrained activation order (the W4A8* rows of Table 3;

@@ -28,7 +28,7 @@ EXPORTS = (
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
     "w4a8_linear_fused", "w4a8_fused_is_faster", "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
-    "w4a8_silu_mul_quantize", "w4a8_linear_w4a16",
+    "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
@@ -58,7 +58,9 @@ def lib():
     L.w4a8_quantize_act.restype = i32
     L.w4a8_quantize_act.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p]
     L.w4a8_linear_w4a16.restype = i32
-    L.w4a8_linear_w4a16.argtypes = [p, i64, i64, p, p, p, p, i32, i64, i64, p, i64, i32, p]
+    L.w4a8_linear_w4a16.argtypes = [p, i64, i64, p, p, p, p, i32, i64, i64, p, i64, i32, p, sz, p]
+    L.w4a8_linear_w4a16_workspace_bytes.restype = sz
+    L.w4a8_linear_w4a16_workspace_bytes.argtypes = [i64, i64, i64]
     L.w4a8_silu_mul_quantize.restype = i32
     L.w4a8_silu_mul_quantize.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p, i64, p]
     L.w4a8_dequant_weight.restype = i32
@@ -156,7 +158,7 @@ def quantize_act(x, scale_mode=SCALE_EXACT, static_scale=None, out=None):
     return x8, s_x
 
 
-def linear_w4a16(x, codes, gscale, gzero, s_w, out=None, out_dtype=OUT_BF16):
+def linear_w4a16(x, codes, gscale, gzero, s_w, out=None, out_dtype=OUT_BF16, workspace=None):
     """w4a8_linear_w4a16: x BF16 [M, K]; canonical device weights.  Returns Y [M, N]."""
     import torch
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
@@ -165,9 +167,12 @@ def linear_w4a16(x, codes, gscale, gzero, s_w, out=None, out_dtype=OUT_BF16):
     if out is None:
         dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
         out = torch.empty((M, N), dtype=dt, device=x.device)
+    nb = int(lib().w4a8_linear_w4a16_workspace_bytes(M, N, K))
+    if workspace is None:
+        workspace = torch.empty((max(nb, 16),), dtype=torch.uint8, device=x.device)
     rc = lib().w4a8_linear_w4a16(_ptr(x), x.stride(0), M, _ptr(codes), _ptr(gscale), _ptr(gzero), _ptr(s_w),
                                  0 if s_w.numel() == 1 else 1, N, K, _ptr(out), out.stride(0), int(out_dtype),
-                                 _stream())
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check("w4a8_linear_w4a16", rc)
     return out
 

@@ -651,11 +651,18 @@ static int linear_w8a8_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, i
     return rc;
 }
 
+// W4A16 tile width over the tokens and split-K workspace (FP32 partial sums, one slab per K slice).
+static int w4a16_bnx(int64_t M) { return M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128)); }
+static size_t w4a16_workspace(int64_t M, int64_t N, int64_t K) {
+    const int s = auto_split_k(M, N, K, w4a16_bnx(M));
+    return s > 1 ? (size_t)s * (size_t)M * (size_t)N * sizeof(float) : 0;
+}
+
 // W4A16 comparison path (Sec. 4.3): BF16 activations, INT4 codes expanded to BF16 in the kernel,
 // kind::f16 MMAs; canonical weights, one tile per CTA.
 static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_t* codes, const void* gscale,
                              const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y,
-                             int64_t ldy, int out_dtype, cudaStream_t st) {
+                             int64_t ldy, int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     if (!x || !codes || !gscale || !s_w || !y) return W4A8_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
     if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
@@ -666,7 +673,13 @@ static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_
         return W4A8_ERR_BAD_ALIGNMENT;
     int rc = check_device();
     if (rc != W4A8_OK) return rc;
-    const int bnx = M <= 16 ? 16 : (M <= 64 ? 64 : 128);
+    const int bnx = w4a16_bnx(M);
+    const int split_k = auto_split_k(M, N, K, bnx);
+    const size_t need = w4a16_workspace(M, N, K);
+    if (need > 0) {
+        if (!workspace || workspace_bytes < need) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
+    }
     CUtensorMap tw, tx;
     if (!make_tmap_u8_2d(&tw, codes, (uint64_t)N, (uint64_t)(K / 2), (uint64_t)(K / 2), 64, 128,
                          CU_TENSOR_MAP_SWIZZLE_64B))
@@ -676,18 +689,29 @@ static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_
                          CU_TENSOR_MAP_SWIZZLE_128B))
         return W4A8_ERR_CUDA;
     const uint16_t* gs = static_cast<const uint16_t*>(gscale);
+    float* partial = split_k > 1 ? static_cast<float*>(workspace) : nullptr;
     const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
+#define W4A8_LAUNCH16(BNX, STG)                                                                                  \
+    rc = launch_umma<UmmaCfg<BNX, STG, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,         \
+                                                     out_dtype, partial, Mi, Ni, Ki, split_k, st)
     switch (bnx) {
-        case 16:
-            return launch_umma<UmmaCfg<16, 4, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
-                                                             out_dtype, nullptr, Mi, Ni, Ki, 1, st);
-        case 64:
-            return launch_umma<UmmaCfg<64, 3, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
-                                                             out_dtype, nullptr, Mi, Ni, Ki, 1, st);
-        default:
-            return launch_umma<UmmaCfg<128, 3, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,
-                                                              out_dtype, nullptr, Mi, Ni, Ki, 1, st);
+        case 16: W4A8_LAUNCH16(16, 4); break;
+        case 32: W4A8_LAUNCH16(32, 4); break;
+        case 64: W4A8_LAUNCH16(64, 3); break;
+        default: W4A8_LAUNCH16(128, 3); break;
     }
+#undef W4A8_LAUNCH16
+    if (rc != W4A8_OK) return rc;
+    if (split_k > 1) {
+        int64_t total = M * N;
+        unsigned blocks = (unsigned)((total + 255) / 256);
+        if (blocks > 148u * 8u) blocks = 148u * 8u;
+        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, split_k, M, N, nullptr, s_w, sw_stride, y, ldy,
+                                                     out_dtype);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        rc = launch_status();
+    }
+    return rc;
 }
 
 static int linear_fused_impl(const void* x, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
@@ -954,9 +978,14 @@ int w4a8_linear_w8a8(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t 
 
 int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* codes, const void* gscale_bf16,
                       const uint8_t* gzero, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y,
-                      int64_t ldy, int out_dtype, void* stream) {
+                      int64_t ldy, int out_dtype, void* workspace, size_t workspace_bytes, void* stream) {
     return linear_w4a16_impl(x_bf16, ldx, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, y, ldy, out_dtype,
-                             static_cast<cudaStream_t>(stream));
+                             workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t w4a8_linear_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    return w4a16_workspace(M, N, K);
 }
 
 int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {

@@ -461,7 +461,7 @@ linear_simt_kernel(const uint8_t* __restrict__ x8, int64_t ldx8, const float* __
             acc = fmaf(e4m3_to_float(x8[m * ldx8 + k + 1]), w1, acc);
         }
     }
-    float r = acc * (s_x[m] * s_w[n * sw_stride]);  // Eq. 4, Eq. 11
+    float r = acc * ((s_x != nullptr ? s_x[m] : 1.0f) * s_w[n * sw_stride]);  // Eq. 4, Eq. 11
     if (out_dtype == W4A8_OUT_FP32)
         reinterpret_cast<float*>(y)[m * ldy + n] = r;
     else
@@ -482,7 +482,7 @@ splitk_reduce_kernel(const float* __restrict__ partial, int S, int64_t M, int64_
         int64_t m = i / N, n = i - m * N;
         float acc = 0.0f;
         for (int s = 0; s < S; ++s) acc += partial[(int64_t)s * total + i];
-        float r = acc * (s_x[m] * s_w[n * sw_stride]);
+        float r = acc * ((s_x != nullptr ? s_x[m] : 1.0f) * s_w[n * sw_stride]);
         if (out_dtype == W4A8_OUT_FP32)
             reinterpret_cast<float*>(y)[m * ldy + n] = r;
         else

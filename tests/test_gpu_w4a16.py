@@ -19,7 +19,7 @@ def _bf16(v):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 16, 128), (16, 128, 256), (5, 144, 384), (64, 256, 512), (37, 400, 1024),
-                                   (128, 128, 128), (200, 272, 640)])
+                                   (128, 128, 128), (200, 272, 640), (24, 256, 1024), (3, 256, 4096)])
 def test_exact_on_small_integers(M, N, K):
     codes, _, gzero = inputs.random_codes(N, K, 40 + M, asymmetric=True)
     gs = np.full((N, K // 128), _bf16(1.0), dtype=np.uint16)
@@ -62,3 +62,20 @@ def test_outputs_beyond_the_problem_are_untouched():
                          out_dtype=binding.OUT_FP32)
     torch.cuda.synchronize()
     assert torch.all(y[M:] == 7.0) and torch.all(y[:, N:] == 7.0)
+
+
+def test_split_k_workspace_is_required_and_sized():
+    M, N, K = 4, 256, 4096                                  # two tiles, 32 k-blocks: K is cut into slices
+    need = int(binding.lib().w4a8_linear_w4a16_workspace_bytes(M, N, K))
+    assert need > 0 and need % (M * N * 4) == 0
+    assert int(binding.lib().w4a8_linear_w4a16_workspace_bytes(4096, 4096, 4096)) == 0
+    codes, gscale, gzero, s_w = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 9), symmetric=True)
+    wd = weights_to_dev(codes, gscale, gzero, s_w)
+    x = bf16_dev(inputs.make_activation(M, K, 10))
+    small = torch.empty((need - 16,), dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.W4A8Error) as e:
+        binding.linear_w4a16(x, *wd, workspace=small)
+    assert "workspace" in str(e.value).lower()
+    y = binding.linear_w4a16(x, *wd, workspace=torch.empty((need,), dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0 and torch.isfinite(y.float()).all()

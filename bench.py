@@ -748,6 +748,67 @@ def mlp_sweep(torch, binding, inputs, dev, peaks):
     return out
 
 
+def tp_sweep(torch, binding, inputs, dev, peaks, rank, world):
+    """The tensor-parallel MLP block of Llama-3-8B (H = 4096, F = 14336) at decode sizes.
+    One process: for TP degrees 1, 2, 4, 8 the time one rank spends on its shard (column-parallel
+    gate/up, fused activation + quantization, row-parallel down; no exchange), from CUDA graphs that
+    rotate over the shards of all ranks of several full layers (more than twice the L2 in total).
+    Several processes (one per GPU): TP degree = world size, the whole block with its NCCL
+    all-reduce of the BF16 partial outputs, max over ranks."""
+    from paper_2505_14638_b200 import tp
+    H, F = 4096, 14336
+    layers = 3      # 3 x 90.8 MB of packed weights > 2 x 126 MB
+    full = []
+    for c in range(layers):
+        W = torch.from_numpy(inputs.make_weight(2 * F, H, SIGMA, seed=9300 + c)).to(dev)
+        gu = tp.Weights(*binding.quantize_weight_rtn(W, symmetric=True))
+        del W
+        W = torch.from_numpy(inputs.make_weight(H, F, SIGMA, seed=9400 + c)).to(dev)
+        down = tp.Weights(*binding.quantize_weight_rtn(W, symmetric=True))
+        del W
+        full.append((gu, down))
+    ops = tp.CudaOps()
+    side = torch.cuda.Stream()
+    out = []
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    degrees = (world,) if world > 1 else (1, 2, 4, 8)
+    for t in degrees:
+        ex = tp.Exchange(world=t)
+        ranks = (rank,) if world > 1 else tuple(range(t))
+        blocks = [tp.TPMlpBlock(gu, down, r, t, ops=ops, exchange=ex) for gu, down in full for r in ranks]
+        shard_bytes = (2 * F * H + H * F) * (0.5 + 2.0 / GROUP) / t
+        for m in (1, 4, 16):
+            x = torch.from_numpy(inputs.make_activation(m, H, 88 + m, OUTLIER_FRAC, OUTLIER_MULT)).to(dev).view(torch.bfloat16)
+            fn = (lambda b: b.forward(x)) if world > 1 else (lambda b: b.partial(x))
+            for b in blocks:
+                fn(b)
+            torch.cuda.synchronize()
+            side.wait_stream(torch.cuda.current_stream())
+            g = torch.cuda.CUDAGraph()
+            reps = 2 * len(blocks) if world == 1 else 8 * len(blocks)
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for i in range(reps):
+                        fn(blocks[i % len(blocks)])
+            torch.cuda.current_stream().wait_stream(side)
+            if dist is not None:
+                dist.barrier()
+            sec = _time_loop(torch, g.replay, 5, warm=2) / reps
+            sec = max_over_ranks([sec], dist, dev)[0]
+            row = {"tp": t, "M": m, "rank_shard_MB": shard_bytes / 1e6, "weight_GBps_per_rank": shard_bytes / sec / 1e9,
+                   "frac_hbm_measured": shard_bytes / sec / 1e9 / peaks["hbm_gbs"]}
+            row["block_with_allreduce_us" if world > 1 else "rank_compute_us"] = sec * 1e6
+            out.append(row)
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set during the sweep")
+    if dist is not None:
+        dist.destroy_process_group()
+    return out
+
+
 def scheme_sweep(torch, binding, inputs, dev):
     """Same-box counterpart of the paper's scheme comparison (Sec. 4.3, Fig. 4, Table 3): per layer
     and token count the time of W4A8 as built here (group-aware order: groups are runs of columns),
@@ -880,7 +941,7 @@ def main():
                     help="consecutive steps captured in one CUDA graph (steps left over run from single-step graphs; default 8)")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
-    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes", "mlp"],
+    ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes", "mlp", "tp"],
                     help="instead of the bench line, print the per-layer table of config c5 (four Llama-3-8B "
                          "linears x M) or the single c4 case (M=8192, K=8192, N=28672)")
     args = ap.parse_args()
@@ -903,6 +964,10 @@ def main():
             rows = scheme_sweep(torch, binding, inputs, dev)
         elif args.sweep == "mlp":
             rows = mlp_sweep(torch, binding, inputs, dev, load_peaks())
+        elif args.sweep == "tp":
+            rows = tp_sweep(torch, binding, inputs, dev, load_peaks(), rank, world)
+            if rank != 0:
+                return
         elif args.sweep == "c5":
             rows = layer_sweep(torch, binding, inputs, dev, load_peaks())
         else:

@@ -328,6 +328,11 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan
     return true;
 }
 
+// Placement slots are handed out round-robin over ALL decode launches of the process: one counter
+// for every instantiation of the launcher (a counter per instantiation gave two kernels of a chain,
+// e.g. a gate/up and a down projection, the same slot while both were in flight).
+static std::atomic<unsigned int> g_sched_seq{0};
+
 template <class Cfg>
 static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                                  int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
@@ -378,8 +383,7 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
         // one worker per SM (see the placement notes beside SchedSlot).  Not for short K walks
         // (under 16 k-blocks per tile): there the extra microsecond at the start of a launch costs
         // more than an occasional SM with two workers (o projection at M = 1: 8.4 against 6.6 us).
-        static std::atomic<unsigned int> seq{0};
-        plan.sched = (int)(seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
+        plan.sched = (int)(g_sched_seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
         grid = 2u * (unsigned)P;
     }
     unsigned int* counters = static_cast<unsigned int*>(workspace);

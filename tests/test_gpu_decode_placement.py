@@ -95,3 +95,50 @@ def test_two_streams_issue_decode_launches_concurrently():
     for o, f in zip(outs, first):
         assert torch.equal(o, f)
     assert binding.query_device_status() == 0
+
+
+def test_chain_of_two_kernel_variants_never_waits_out_a_placement_hold():
+    # A chain that alternates a launch without a K cut (many output channels) and one with K cut
+    # into chunks (few output channels) runs two instantiations of the decode kernel back to back,
+    # each launch overlapping the next one's start.  Their placement slots must differ: when both
+    # drew the same slot, candidates of one launch counted into the other's table and now and then
+    # sat out the full hold limit (200 us) -- visible as single replays far above the median.
+    H, F, M = 4096, 14336, 1
+    mk = lambda N, K, seed: binding.prepack_weight(
+        *binding.quantize_weight_rtn(torch.from_numpy(inputs.make_weight(N, K, 0.02, seed)).cuda(), symmetric=True))
+    wide, narrow = mk(2 * F, H, 71), mk(H, F, 72)
+    x8a, sa = binding.quantize_act(bf16_dev(inputs.make_activation(M, H, 73)))
+    x8b, sb = binding.quantize_act(bf16_dev(inputs.make_activation(M, F, 74)))
+    ya = torch.empty((M, 2 * F), dtype=torch.bfloat16, device="cuda")
+    yb = torch.empty((M, H), dtype=torch.bfloat16, device="cuda")
+    wsa, wsb = binding.new_workspace(M, 2 * F, H, wide.fmt, "cuda"), binding.new_workspace(M, H, F, narrow.fmt, "cuda")
+
+    def chain():
+        binding.linear_tiled(x8a, sa, wide, out=ya, workspace=wsa)
+        binding.linear_tiled(x8b, sb, narrow, out=yb, workspace=wsb)
+
+    chain()
+    torch.cuda.synchronize()
+    first = (ya.clone(), yb.clone())
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(6):
+                chain()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    reps = 60
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for i in range(reps):
+        g.replay()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    t = np.array([ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(reps)])    # microseconds per replay
+    assert binding.query_device_status() == 0
+    assert torch.equal(ya, first[0]) and torch.equal(yb, first[1])
+    assert t.max() - np.median(t) < 100.0, (float(np.median(t)), float(t.max()))

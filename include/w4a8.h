@@ -110,9 +110,13 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * its first use; every call leaves it ready for the next one.  Calls that share a workspace
  * must not overlap on the device.
  * Calls with M <= 16 on tiled weights place their worker CTAs at run time (at most one per SM and
- * launch, so that consecutive launches can share the SMs); the bookkeeping is a table of 64
- * entries that is part of the library image, handed out round-robin per call and cleared by the
- * kernel: up to 64 such launches may be in flight on a device at a time.
+ * launch, so that consecutive launches can share the SMs).  The bookkeeping (1 KB, cleared by the
+ * kernel) lives in the workspace when one of the full size is given -- nothing more to observe
+ * than the rule above: calls that may overlap on the device need different workspaces; calls
+ * issued one after the other on one stream may share one.  Without a workspace it is an entry of a
+ * 64-entry table in the library image, handed out round-robin over all such calls of the process
+ * (a captured call keeps the entry it drew at capture): then no more than 64 such launches may be
+ * in flight on a device at a time, replays of graphs captured far apart included.
  */
 int w4a8_linear(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* weights,
                 const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w,
@@ -192,7 +196,9 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * On B200 the fused launch turned out slower than w4a8_quantize_act + w4a8_linear chained on one
  * stream (they overlap under programmatic dependent launch; every CTA of the fused launch scans X
  * for the token scales): it is kept for callers that want a single launch.
- * Needs no workspace and allocates nothing.  Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
+ * Needs no workspace and allocates nothing; its run-time placement of worker CTAs uses the
+ * library's 64-entry table (see w4a8_linear: at most 64 such launches in flight on a device).
+ * Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
  * K / N the tiled format does not admit; otherwise as w4a8_linear.
  */
 #define W4A8_FUSED_MAX_M 16

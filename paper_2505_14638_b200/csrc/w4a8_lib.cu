@@ -285,8 +285,11 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
 
 // Row partition and ring sizes of the split-N kernel for the current device.
 // Workspace of the split-N kernel when it cuts K (bytes; fits any SM count up to kMaxSMs and 128 tokens).
+// Layout: split-K counters (1 KB), placement state of the launch (1 KB), partial tiles.
 constexpr size_t kSnCounterBytes = 1024;
-constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + (size_t)kMaxSMs * 128 * 128 * sizeof(float);
+constexpr size_t kSnSchedBytes = 1024;
+static_assert(kSnCounterBytes == (size_t)kSchedWsOffset, "the kernel finds the placement state behind the counters");
+constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + kSnSchedBytes + (size_t)kMaxSMs * 128 * 128 * sizeof(float);
 
 template <class Cfg>
 static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan* pl) {
@@ -328,15 +331,17 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan
     return true;
 }
 
-// Placement slots are handed out round-robin over ALL decode launches of the process: one counter
-// for every instantiation of the launcher (a counter per instantiation gave two kernels of a chain,
-// e.g. a gate/up and a down projection, the same slot while both were in flight).
+// Launches without a workspace draw their placement slot round-robin over ALL decode launches of
+// the process: one counter for every instantiation of the launcher (a counter per instantiation
+// gave two kernels of a chain, e.g. a gate/up and a down projection, the same slot while both were
+// in flight).  Launches with a workspace keep the state there and need no slot.
 static std::atomic<unsigned int> g_sched_seq{0};
 
 template <class Cfg>
 static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                                  int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
-                                 cudaStream_t st, const SnFuse& fuse, void* workspace, const SnPlan& pl, int sms);
+                                 cudaStream_t st, const SnFuse& fuse, void* workspace, bool ws_usable,
+                                 const SnPlan& pl, int sms);
 
 template <int MT, int G, int FMT, bool FUSE = false>
 static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
@@ -347,23 +352,24 @@ static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const fl
     if (sms <= 0) return W4A8_ERR_CUDA;
     SnPlan pl;
     // K is cut only when the caller gave the (zero-initialised) workspace for the partial sums
-    const bool may_split_k = !FUSE && workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes &&
-                             aligned16(workspace);
+    const bool ws_usable = workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes && aligned16(workspace);
+    const bool may_split_k = !FUSE && ws_usable;
     if (!make_sn_plan<Cfg>(N, K, sms, may_split_k, &pl)) return W4A8_ERR_BAD_SHAPE;
     if constexpr (!FUSE) {
         if (pl.KSPLIT > 1)
             return launch_splitn_planned<SnCfg<MT, G, FMT, false, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                         out_dtype, M, N, K, st, fuse, workspace, pl,
-                                                                         sms);
+                                                                         out_dtype, M, N, K, st, fuse, workspace,
+                                                                         ws_usable, pl, sms);
     }
     return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, fuse, workspace,
-                                      pl, sms);
+                                      ws_usable, pl, sms);
 }
 
 template <class Cfg>
 static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                                  int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
-                                 cudaStream_t st, const SnFuse& fuse, void* workspace, const SnPlan& pl, int sms) {
+                                 cudaStream_t st, const SnFuse& fuse, void* workspace, bool ws_usable,
+                                 const SnPlan& pl, int sms) {
     auto kern = linear_splitn_kernel<Cfg>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -383,11 +389,12 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
         // one worker per SM (see the placement notes beside SchedSlot).  Not for short K walks
         // (under 16 k-blocks per tile): there the extra microsecond at the start of a launch costs
         // more than an occasional SM with two workers (o projection at M = 1: 8.4 against 6.6 us).
-        plan.sched = (int)(g_sched_seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
+        plan.sched = ws_usable ? kSchedInWorkspace
+                               : (int)(g_sched_seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
         grid = 2u * (unsigned)P;
     }
     unsigned int* counters = static_cast<unsigned int*>(workspace);
-    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kSnCounterBytes);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kSnCounterBytes + kSnSchedBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(Cfg::kThreads);

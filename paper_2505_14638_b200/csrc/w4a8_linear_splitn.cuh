@@ -114,7 +114,9 @@ struct SnPlan {
     int xstage;    // bytes per stage: activation tiles
     int smem;      // dynamic shared memory to request
     int P;         // CTAs that do the work; CTA p takes tiles p, p + P, ...
-    int sched;     // >= 0: slot of the per-launch placement state (twice P CTAs are launched, see below); -1: CTA p = blockIdx.x
+    int sched;     // -1: CTA p = blockIdx.x.  Otherwise twice P CTAs are launched and draw their worker indices at
+                   // run time (see below): kSchedInWorkspace = the table sits in the caller's workspace,
+                   // 0 .. kSchedSlots - 1 = slot of the library's own table
 };
 
 // ---- placement of the decode-sized launches -------------------------------------------------
@@ -127,18 +129,27 @@ struct SnPlan {
 // twice as many CTAs ("candidates") as it needs workers.  A candidate that finds a worker of
 // its own launch already on its SM retires at once (unless so few candidates are left that the
 // work could otherwise go undone); the first candidate on an SM takes the next worker index.
-// State lives in a small table of slots handed out round-robin by the host, one per launch, and
-// the last candidate of a launch to enter clears its slot: replaying a captured launch reuses
-// its slot, and launches that can overlap in time (consecutive ones) hold different slots.
+// The state of a launch (one SchedSlot) is cleared by the last of its candidates to enter.  It
+// lives in the caller's workspace when there is one (at byte kSchedWsOffset, after the split-K
+// counters): launches that may run at the same time must have different workspaces anyway, and
+// consecutive launches of one stream cannot meet in it, because the dependent launch starts only
+// after every candidate of this one has entered (entering comes before the launch-dependents
+// trigger in every candidate).  Without a workspace the state is a slot of a small table in the
+// library image, handed out round-robin by the host over all launches of the process; that is
+// safe only while fewer than kSchedSlots such launches are in flight, and a captured launch keeps
+// the slot it drew at capture time.
 constexpr int kSchedSlots = 64;
+constexpr int kSchedInWorkspace = kSchedSlots;
 constexpr int kSchedMaxSMs = 192;
+constexpr int kSchedWsOffset = 1024;
 struct SchedSlot {
     unsigned int started;   // candidates that have drawn a start number
     unsigned int issued;    // worker indices handed out
     unsigned int finished;  // candidates that have entered
-    unsigned int pad;
+    unsigned int gen;       // launches that have used and cleared this slot (never reset)
     unsigned int on_sm[kSchedMaxSMs];  // candidates of this launch seen per SM
 };
+static_assert(sizeof(SchedSlot) <= 1024, "the placement state has 1 KB of the workspace");
 __device__ SchedSlot g_sched[kSchedSlots];
 
 // Called by thread 0 of a candidate: returns its worker index, or -1 to retire.  Plain atomic adds
@@ -148,15 +159,17 @@ __device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candi
     unsigned int smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
     // (the two adds are independent: one L2 round trip for both)
+    // (the read of `issued` is issued together with the adds: three requests, one round trip)
+    const unsigned int i = *reinterpret_cast<volatile unsigned int*>(&sl->issued);
     const unsigned int c = atomicAdd(&sl->started, 1u);
     const bool first_here = smid < (unsigned)kSchedMaxSMs ? atomicAdd(&sl->on_sm[smid], 1u) == 0u : true;
     bool want = first_here;
     if (!want) {
         // A second candidate on this SM works only if the candidates still to come could not
         // cover the indices still to be issued.  The count read here may lag behind (never run
-        // ahead of) the true one, which errs towards working; the candidate with the last start
-        // number therefore declines only when every index has been issued.
-        const unsigned int i = *reinterpret_cast<volatile unsigned int*>(&sl->issued);
+        // ahead of) the true one, which errs towards working -- a candidate that then draws an
+        // index beyond the last one retires after all; the candidate with the last start number
+        // therefore declines only when every index has been issued.
         want = i < (unsigned)workers && (unsigned)workers - i >= (unsigned)candidates - c;
     }
     if (!want) return -1;
@@ -174,6 +187,8 @@ __device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
         sl->issued = 0u;
         sl->finished = 0u;
         __threadfence();
+        atomicAdd(&sl->gen, 1u);  // releases the candidates that still hold their place
+        __threadfence();
     }
 }
 
@@ -183,10 +198,12 @@ __device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
 // one would decline too: on SMs with two free places (the previous launch had fewer workers than
 // there are SMs) the whole surplus of candidates burnt away like this before the other SMs had
 // room, and the last ones were then forced to work as second workers after all.
-__device__ __forceinline__ void sched_hold(SchedSlot* sl, int workers) {
+__device__ __forceinline__ void sched_hold(SchedSlot* sl, int workers, unsigned int gen0) {
     const uint64_t t0 = ptx::globaltimer_ns();
-    while (*reinterpret_cast<volatile unsigned int*>(&sl->issued) < (unsigned)workers &&
-           *reinterpret_cast<volatile unsigned int*>(&sl->finished) != 0u &&
+    // (gen0 = the slot's generation when this candidate entered: once it has moved on, the slot
+    // belongs to a later launch and its counts say nothing about this one)
+    while (*reinterpret_cast<volatile unsigned int*>(&sl->gen) == gen0 &&
+           *reinterpret_cast<volatile unsigned int*>(&sl->issued) < (unsigned)workers &&
            ptx::globaltimer_ns() - t0 < 200000ull) {
         __nanosleep(500);
     }
@@ -313,7 +330,15 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     int P = gridDim.x, p = blockIdx.x;
     __shared__ int worker_s;
     // (thread 0 asks for a worker index while thread 32 sets up the barriers)
-    if (plan.sched >= 0 && threadIdx.x == 0) worker_s = sched_enter(&g_sched[plan.sched], plan.P, (int)gridDim.x);
+    SchedSlot* const sched_slot =
+        plan.sched == kSchedInWorkspace
+            ? reinterpret_cast<SchedSlot*>(reinterpret_cast<uint8_t*>(counters) + kSchedWsOffset)
+            : &g_sched[plan.sched >= 0 ? plan.sched : 0];
+    unsigned int sched_gen = 0u;  // (thread 0 only)
+    if (plan.sched >= 0 && threadIdx.x == 0) {
+        sched_gen = *reinterpret_cast<volatile unsigned int*>(&sched_slot->gen);
+        worker_s = sched_enter(sched_slot, plan.P, (int)gridDim.x);
+    }
     const int KSPLIT = Cfg::SPLITK ? plan.KSPLIT : 1, TR = T / KSPLIT;
     // Tile t: 8-row units [u0, u1) of row range t / KSPLIT, k-blocks [kb0, kb0 + nkb) of chunk t % KSPLIT.
     const int nst_all = (KB + KS - 1) / KS;  // stages per tile when K is not cut
@@ -358,13 +383,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         P = plan.P;
         if (p < 0) {  // a worker of this launch is already on this SM: retire
             if (threadIdx.x == 0) {
+                sched_entered(sched_slot, (int)gridDim.x);  // before the trigger: see the notes beside SchedSlot
                 ptx::griddep_launch_dependents();
-                sched_entered(&g_sched[plan.sched], (int)gridDim.x);
-                sched_hold(&g_sched[plan.sched], plan.P);
+                sched_hold(sched_slot, plan.P, sched_gen);
             }
             return;
         }
-        if (threadIdx.x == 64) sched_entered(&g_sched[plan.sched], (int)gridDim.x);  // an idle epilogue thread
+        if (threadIdx.x == 64) sched_entered(sched_slot, (int)gridDim.x);  // an idle epilogue thread
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);

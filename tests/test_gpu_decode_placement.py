@@ -142,3 +142,24 @@ def test_chain_of_two_kernel_variants_never_waits_out_a_placement_hold():
     assert binding.query_device_status() == 0
     assert torch.equal(ya, first[0]) and torch.equal(yb, first[1])
     assert t.max() - np.median(t) < 100.0, (float(np.median(t)), float(t.max()))
+
+
+def test_launches_without_a_workspace_use_the_library_table_and_agree():
+    # No (or too small a) workspace: the placement state is an entry of the library's own table and K
+    # is never cut.  Results: equal bit for bit to the workspace path where that does not cut K
+    # either (many output channels), within the output gate where it does (few output channels).
+    tiny = torch.zeros((16,), dtype=torch.uint8, device="cuda")
+    for M, N, K, cuts_k in ((4, 14336, 4096, False), (2, 4096, 14336, True)):
+        tw, x8, s_x, y64, ws = _case(M, N, K, 31 + M)
+        with_ws = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32, workspace=ws)
+        outs = [binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32, workspace=tiny) for _ in range(70)]
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0
+        worst, _ = fp32_gate(outs[0].cpu().numpy(), y64, rel=2e-3)
+        assert worst <= 2e-3, worst
+        assert all(torch.equal(o, outs[0]) for o in outs[1:])
+        if not cuts_k:
+            assert torch.equal(outs[0], with_ws)
+        else:
+            worst, _ = fp32_gate(with_ws.cpu().numpy(), y64, rel=2e-3)
+            assert worst <= 2e-3, worst

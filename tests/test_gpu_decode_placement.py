@@ -97,7 +97,8 @@ def test_two_streams_issue_decode_launches_concurrently():
     assert binding.query_device_status() == 0
 
 
-def test_chain_of_two_kernel_variants_never_waits_out_a_placement_hold():
+@pytest.mark.parametrize("shared_workspace", [False, True])
+def test_chain_of_two_kernel_variants_never_waits_out_a_placement_hold(shared_workspace):
     # A chain that alternates a launch without a K cut (many output channels) and one with K cut
     # into chunks (few output channels) runs two instantiations of the decode kernel back to back,
     # each launch overlapping the next one's start.  Their placement slots must differ: when both
@@ -112,6 +113,8 @@ def test_chain_of_two_kernel_variants_never_waits_out_a_placement_hold():
     ya = torch.empty((M, 2 * F), dtype=torch.bfloat16, device="cuda")
     yb = torch.empty((M, H), dtype=torch.bfloat16, device="cuda")
     wsa, wsb = binding.new_workspace(M, 2 * F, H, wide.fmt, "cuda"), binding.new_workspace(M, H, F, narrow.fmt, "cuda")
+    if shared_workspace:    # allowed for calls issued one after the other on one stream
+        wsb = wsa
 
     def chain():
         binding.linear_tiled(x8a, sa, wide, out=ya, workspace=wsa)

@@ -332,6 +332,11 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
  * copies y_dev (BF16 [M][N]) to y_host, all enqueued on `stream`; the caller synchronises the
  * stream before reading y_host.  Weights stay resident on the device.  Scratch device buffers
  * are the caller's: x_dev (2*M*K bytes), x8_dev (M*K), s_x_dev (4*M), y_dev (2*M*N), workspace.
+ * For M <= 128, when both host buffers are page-locked (pinned or registered, 16-byte aligned),
+ * no copy is enqueued: the quantization kernel reads x_host and the linear kernel writes y_host
+ * through their device mappings -- the same bytes cross the bus, without two copy-engine
+ * operations; x_dev and y_dev are then left untouched.  Pageable buffers and larger M take the
+ * copies.  x8_dev and s_x_dev hold the quantized activations afterwards in both cases.
  */
 int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights,
                       const void* gscale_bf16, const uint8_t* gzero, int weight_format, const float* s_w,

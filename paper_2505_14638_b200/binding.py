@@ -132,7 +132,12 @@ def _ptr(t):
 
 
 def _stream():
+    """Handle of torch's current CUDA stream on the current device (the raw getter when this torch
+    has it: the Stream object route costs about ten microseconds per call)."""
     import torch
+    raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+    if raw is not None:
+        return ctypes.c_void_p(raw(torch.cuda.current_device()))
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
@@ -453,6 +458,7 @@ class HostForward:
         self.d2h_bytes = M * self.N * 2
 
     def set_weight(self, weight):
+        self._args = None
         if isinstance(weight, TiledWeight):
             self.wbuf, self.gscale, self.gzero, self.s_w = weight.buf, None, None, weight.s_w
             self.fmt, self.N, self.K = weight.fmt, weight.N, weight.K
@@ -464,10 +470,13 @@ class HostForward:
     def __call__(self, x_host):
         """x_host: pinned BF16 [M, K] host tensor.  Enqueues everything; returns the pinned
         output tensor, valid after the current stream is synchronised."""
-        rc = lib().w4a8_forward_host(
-            ctypes.c_void_p(x_host.data_ptr()), self.M, _ptr(self.wbuf), _ptr(self.gscale),
-            _ptr(self.gzero), self.fmt, _ptr(self.s_w), 0 if self.s_w.numel() == 1 else 1, self.N,
-            self.K, GROUP, ctypes.c_void_p(self.y_host.data_ptr()), _ptr(self.x_dev), _ptr(self.x8),
-            _ptr(self.s_x), _ptr(self.y_dev), _ptr(self.ws), self.ws.numel(), _stream())
-        _check("w4a8_forward_host", rc)
+        if self._args is None:   # everything but the input pointer and the stream is fixed per weight
+            self._args = (self.M, _ptr(self.wbuf), _ptr(self.gscale), _ptr(self.gzero), self.fmt, _ptr(self.s_w),
+                          0 if self.s_w.numel() == 1 else 1, self.N, self.K, GROUP,
+                          ctypes.c_void_p(self.y_host.data_ptr()), _ptr(self.x_dev), _ptr(self.x8), _ptr(self.s_x),
+                          _ptr(self.y_dev), _ptr(self.ws), self.ws.numel())
+            self._fn = lib().w4a8_forward_host
+        rc = self._fn(ctypes.c_void_p(x_host.data_ptr()), *self._args, _stream())
+        if rc != 0:
+            _check("w4a8_forward_host", rc)
         return self.y_host

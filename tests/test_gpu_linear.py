@@ -233,10 +233,31 @@ def test_host_forward_entry_point():
     ref = oracle.forward(xb, *wq)
     x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
     wd = weights_to_dev(*wq)
+    # pinned input: the kernels read and write the host buffers themselves; pageable input: copies
+    x_pageable = torch.from_numpy(xb.view(np.int16).copy()).view(torch.bfloat16)
+    assert not x_pageable.is_pinned()
     for weight in (wd, binding.prepack_weight(*wd)):
-        fwd = binding.HostForward(M, weight)
-        y_host = fwd(x_host)
-        torch.cuda.synchronize()
-        ok, dist = bf16_gate(bf16_bits(y_host), ref["y64"])
-        assert ok, dist
-        assert fwd.h2d_bytes == M * K * 2 and fwd.d2h_bytes == M * N * 2
+        for xh in (x_host, x_pageable):
+            fwd = binding.HostForward(M, weight)
+            fwd.y_host.fill_(7.0)
+            y_host = fwd(xh)
+            torch.cuda.synchronize()
+            assert binding.query_device_status() == 0
+            ok, dist = bf16_gate(bf16_bits(y_host), ref["y64"])
+            assert ok, dist
+            assert np.array_equal(fwd.x8.cpu().numpy(), ref["x8"])                       # Eq. 13, bit for bit
+            assert np.array_equal(fwd.s_x.cpu().numpy().view(np.uint32), ref["s_x"].view(np.uint32))
+            assert fwd.h2d_bytes == M * K * 2 and fwd.d2h_bytes == M * N * 2
+
+
+def test_host_forward_many_tokens_takes_the_copy_path():
+    M, K, N = 200, 512, 256
+    wq = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 14), symmetric=True)
+    xb = inputs.make_activation(M, K, 15)
+    ref = oracle.forward(xb, *wq)
+    x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    fwd = binding.HostForward(M, binding.prepack_weight(*weights_to_dev(*wq)))
+    y_host = fwd(x_host)
+    torch.cuda.synchronize()
+    ok, dist = bf16_gate(bf16_bits(y_host), ref["y64"])
+    assert ok, dist

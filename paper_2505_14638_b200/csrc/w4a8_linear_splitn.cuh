@@ -142,7 +142,7 @@ constexpr int kSchedSlots = 64;
 constexpr int kSchedInWorkspace = kSchedSlots;
 constexpr int kSchedMaxSMs = 192;
 constexpr int kSchedWsOffset = 1024;
-struct SchedSlot {
+struct __align__(16) SchedSlot {
     unsigned int started;   // candidates that have drawn a start number
     unsigned int issued;    // worker indices handed out
     unsigned int finished;  // candidates that have entered
@@ -182,12 +182,16 @@ __device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candi
 __device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
     __threadfence();
     if (atomicAdd(&sl->finished, 1u) == (unsigned)candidates - 1u) {
-        for (int i = 0; i < kSchedMaxSMs; ++i) sl->on_sm[i] = 0u;
-        sl->started = 0u;
-        sl->issued = 0u;
-        sl->finished = 0u;
-        __threadfence();
-        atomicAdd(&sl->gen, 1u);  // releases the candidates that still hold their place
+        // The last one clears the slot.  This sits between the last candidate's arrival and the
+        // release of the dependent launch, so it is kept short: 16-byte stores, the three counters
+        // and the new generation (which releases the candidates that still hold their place) in
+        // one of them, a single fence.
+        static_assert(kSchedMaxSMs % 4 == 0 && sizeof(SchedSlot) == 16 + 4 * kSchedMaxSMs, "slot layout");
+        const unsigned int gen = *reinterpret_cast<volatile unsigned int*>(&sl->gen);
+        uint4* v = reinterpret_cast<uint4*>(sl);
+#pragma unroll 8
+        for (int i = 1; i <= kSchedMaxSMs / 4; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+        v[0] = make_uint4(0u, 0u, 0u, gen + 1u);
         __threadfence();
     }
 }

@@ -179,7 +179,9 @@ __device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candi
 // Called once by every candidate after sched_enter: the slot is only needed while candidates
 // enter, so the last one to have entered clears it (nothing of this runs at the end of the
 // kernel, where it would delay the launch's completion).
-__device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
+// (`gen` = the slot's generation if the caller has read it during this launch, kSchedGenUnknown otherwise)
+constexpr unsigned int kSchedGenUnknown = 0xFFFFFFFFu;
+__device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates, unsigned int gen_in) {
     __threadfence();
     if (atomicAdd(&sl->finished, 1u) == (unsigned)candidates - 1u) {
         // The last one clears the slot.  This sits between the last candidate's arrival and the
@@ -187,11 +189,12 @@ __device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates) {
         // and the new generation (which releases the candidates that still hold their place) in
         // one of them, a single fence.
         static_assert(kSchedMaxSMs % 4 == 0 && sizeof(SchedSlot) == 16 + 4 * kSchedMaxSMs, "slot layout");
-        const unsigned int gen = *reinterpret_cast<volatile unsigned int*>(&sl->gen);
+        const unsigned int gen =
+            gen_in != kSchedGenUnknown ? gen_in : *reinterpret_cast<volatile unsigned int*>(&sl->gen);
         uint4* v = reinterpret_cast<uint4*>(sl);
 #pragma unroll 8
         for (int i = 1; i <= kSchedMaxSMs / 4; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
-        v[0] = make_uint4(0u, 0u, 0u, gen + 1u);
+        v[0] = make_uint4(0u, 0u, 0u, gen + 1u == kSchedGenUnknown ? 0u : gen + 1u);
         __threadfence();
     }
 }
@@ -387,13 +390,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         P = plan.P;
         if (p < 0) {  // a worker of this launch is already on this SM: retire
             if (threadIdx.x == 0) {
-                sched_entered(sched_slot, (int)gridDim.x);  // before the trigger: see the notes beside SchedSlot
+                sched_entered(sched_slot, (int)gridDim.x, sched_gen);  // before the trigger: see the notes beside SchedSlot
                 ptx::griddep_launch_dependents();
                 sched_hold(sched_slot, plan.P, sched_gen);
             }
             return;
         }
-        if (threadIdx.x == 64) sched_entered(sched_slot, (int)gridDim.x);  // an idle epilogue thread
+        if (threadIdx.x == 64) sched_entered(sched_slot, (int)gridDim.x, kSchedGenUnknown);  // an idle epilogue thread
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);

@@ -248,6 +248,21 @@ def test_host_forward_entry_point():
             assert np.array_equal(fwd.x8.cpu().numpy(), ref["x8"])                       # Eq. 13, bit for bit
             assert np.array_equal(fwd.s_x.cpu().numpy().view(np.uint32), ref["s_x"].view(np.uint32))
             assert fwd.h2d_bytes == M * K * 2 and fwd.d2h_bytes == M * N * 2
+            if xh is x_host:
+                # later calls with the same buffers must see what the buffers hold NOW (new
+                # activations in the same pinned buffer)
+                xb2 = inputs.make_activation(M, K, 99, 0.01, 20.0)
+                ref2 = oracle.forward(xb2, *wq)
+                keep = x_host.clone()
+                for _ in range(3):
+                    x_host.copy_(torch.from_numpy(xb2.view(np.int16)).view(torch.bfloat16))
+                    fwd.y_host.fill_(7.0)
+                    y2 = fwd(x_host)
+                    torch.cuda.synchronize()
+                    ok, dist = bf16_gate(bf16_bits(y2), ref2["y64"])
+                    assert ok, dist
+                    assert np.array_equal(fwd.x8.cpu().numpy(), ref2["x8"])
+                x_host.copy_(keep)
 
 
 def test_host_forward_many_tokens_takes_the_copy_path():

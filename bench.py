@@ -880,6 +880,23 @@ def scheme_sweep(torch, binding, inputs, dev):
     return out
 
 
+def _hessian_upper_cholesky(H, perm=None, damp=0.01):
+    """Upper Cholesky factor of the inverse of the dampened Hessian in processing order (Sec. 3.3,
+    as in GPTQ), with torch.linalg in float64: an input of w4a8_dpq_quantize, prepared by the caller."""
+    import torch
+    H = H.to(torch.float64)
+    if perm is not None:
+        idx = perm.to(torch.int64)
+        H = H[idx][:, idx]
+    H = H.clone()
+    d = torch.diagonal(H)
+    d[d == 0] = 1.0
+    d += damp * d.mean()
+    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
+    Hinv = 0.5 * (Hinv + Hinv.T)
+    return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()
+
+
 def dpq_sweep(torch, binding, inputs, dev):
     """Offline DPQ quantizer (Algorithm 1 with Group-Aware Reordering and an 6-step scale search)
     on Llama-3-8B layer shapes: device time of w4a8_dpq_quantize against the plain-ALU roofline of
@@ -895,7 +912,7 @@ def dpq_sweep(torch, binding, inputs, dev):
         t0 = time.perf_counter()
         H = X.T @ X
         perm = binding.gar_permutation(torch.diagonal(H).to(torch.float32).contiguous())
-        U = binding.hessian_upper_cholesky(H, perm)
+        U = _hessian_upper_cholesky(H, perm)   # the caller's library step: the factor is an input of the quantizer
         torch.cuda.synchronize()
         t_prep = time.perf_counter() - t0
         binding.dpq_quantize(W, U, perm, symmetric=False, mse_steps=6)   # warm-up

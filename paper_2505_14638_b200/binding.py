@@ -402,24 +402,6 @@ def gar_permutation(hdiag):
     return perm
 
 
-def hessian_upper_cholesky(H, perm=None, damp=0.01):
-    """Library step in front of w4a8_dpq_quantize (Sec. 3.3, as in GPTQ), with torch.linalg in
-    float64 on the device: permute H to processing order, give dead columns a unit diagonal, add
-    damp * mean(diag), invert, return the upper Cholesky factor of the inverse as float32."""
-    import torch
-    H = H.to(torch.float64)
-    if perm is not None:
-        idx = perm.to(torch.int64)
-        H = H[idx][:, idx]
-    H = H.clone()
-    d = torch.diagonal(H)
-    d[d == 0] = 1.0
-    d += damp * d.mean()
-    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
-    Hinv = 0.5 * (Hinv + Hinv.T)
-    return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()
-
-
 def dpq_quantize(W, U, perm=None, symmetric=False, mse_steps=0, per_channel=False):
     """w4a8_dpq_quantize: W float32 [N, K], U float32 [K, K] (processing order), perm int32 [K] or
     None, all on the device.  Returns (codes, gscale BF16, gzero or None, s_w)."""

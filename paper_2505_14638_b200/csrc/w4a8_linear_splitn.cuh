@@ -631,8 +631,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                 }
                 if (!ok) break;
                 if (ptx::elect_one()) ptx::umma_commit(bar_acc_full);
-                if (lane == 0) {
-                }
             }
             if (!ok && lane == 0) {
                 // Gave up: wait (bounded) for the MMAs already issued before tensor memory is freed.
@@ -777,8 +775,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(bar_acc_empty);
-            if (threadIdx.x == 64) {
-            }
         }
     } else {
         // ------------------------------------------------------------------ dequantization groups

@@ -22,3 +22,21 @@ def bf16_bits(t):
 
 def weights_to_dev(codes, gscale, gzero, s_w):
     return (dev(codes), bf16_dev(gscale), None if gzero is None else dev(gzero), dev(s_w))
+
+
+def hessian_upper_cholesky_dev(H, perm=None, damp=0.01):
+    """The factor U that w4a8_dpq_quantize takes as an INPUT (Sec. 3.3, as in GPTQ), computed with
+    torch.linalg in float64 on the device: permute H to processing order, give dead columns a unit
+    diagonal, add damp * mean(diag), invert, return the upper Cholesky factor of the inverse as
+    float32.  The library has no entry point for this step: U is the caller's."""
+    H = H.to(torch.float64)
+    if perm is not None:
+        idx = perm.to(torch.int64)
+        H = H[idx][:, idx]
+    H = H.clone()
+    d = torch.diagonal(H)
+    d[d == 0] = 1.0
+    d += damp * d.mean()
+    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
+    Hinv = 0.5 * (Hinv + Hinv.T)
+    return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()

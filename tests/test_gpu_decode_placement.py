@@ -1,9 +1,10 @@
 """GPU: the decode-sized launches hand out their worker indices at run time (twice as many CTAs
-as workers, at most one worker per SM and launch; the state lives in a table of 64 slots that the
-host hands out round-robin and the kernel clears).  Whatever the placement, every row range must
-be computed exactly once: long runs of launches -- more than there are slots, eager and replayed
-from one CUDA graph, alternating shapes -- must reproduce the first result bit for bit, and that
-result must match the oracle."""
+as workers, at most one worker per SM and launch).  The state of a launch lives in the caller's
+workspace, behind the split-K counters, and is cleared by the last CTA to enter; launches without
+a workspace use an entry of a 64-entry table in the library image.  Whatever the placement, every
+row range must be computed exactly once: long runs of launches -- more than the table has entries,
+eager and replayed from one CUDA graph, alternating shapes, from two streams -- must reproduce the
+first result bit for bit, and that result must match the oracle."""
 import numpy as np
 import pytest
 import torch

@@ -8,7 +8,7 @@ import pytest
 import torch
 
 import oracle
-from gpu_utils import bf16_bits, dev
+from gpu_utils import bf16_bits, dev, hessian_upper_cholesky_dev
 from paper_2505_14638_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
@@ -82,13 +82,13 @@ def test_dpq_identity_factor_is_round_to_nearest():
 
 def test_dpq_layer_size_and_the_device_side_factorization():
     # a Llama-sized layer slice: N = 512 rows of the K = 4096 o-projection; the codes must match the
-    # oracle when both get the SAME factor (here the one the device-side helper computes) ...
+    # oracle when both get the SAME factor (here one computed on the device by the caller's library routines) ...
     N, K = 512, 4096
     W = inputs.make_weight(N, K, 0.02, seed=9)
     H = _hessian(K, 10, tokens=1024)
     Hd = dev(H.astype(np.float64))
     perm = binding.gar_permutation(torch.diagonal(Hd).to(torch.float32).contiguous())
-    U = binding.hessian_upper_cholesky(Hd, perm)
+    U = hessian_upper_cholesky_dev(Hd, perm)
     torch.cuda.synchronize()
     assert np.array_equal(perm.cpu().numpy(), oracle.gar_permutation(np.diag(H).astype(np.float32)))
     _compare(W, U.cpu().numpy(), perm.cpu().numpy(), symmetric=False, mse_steps=6)

@@ -145,3 +145,60 @@ def test_rejects_an_order_that_splits_groups():
     perm[[0, 200]] = perm[[200, 0]]
     with pytest.raises(ValueError):
         oracle.dpq_quantize(W, np.eye(256, dtype=np.float32), perm)
+
+
+def _damped_permuted(H, perm, damp):
+    """The matrix Sec. 3.3 inverts, built here entry by entry (not with the oracle's indexing)."""
+    K = H.shape[0]
+    order = list(range(K)) if perm is None else [int(v) for v in perm]
+    Hp = np.empty((K, K), dtype=np.float64)
+    for a in range(K):
+        for b in range(K):
+            Hp[a, b] = H[order[a], order[b]]
+    for a in range(K):
+        if Hp[a, a] == 0.0:
+            Hp[a, a] = 1.0
+    mean_diag = sum(Hp[a, a] for a in range(K)) / K
+    for a in range(K):
+        Hp[a, a] += damp * mean_diag
+    return Hp
+
+
+@pytest.mark.parametrize("use_perm,damp", [(False, 0.01), (True, 0.01), (True, 0.1)])
+def test_hessian_factor_inverts_the_dampened_permuted_hessian(use_perm, damp):
+    # U is upper triangular with a positive diagonal and U^T U is the inverse of the dampened
+    # Hessian in processing order: (U^T U) (H_perm + damp * mean(diag) * I) = I.  An asymmetric H
+    # ordering (rows permuted but not columns), a missing or doubled dampening, a lower factor or a
+    # factor of H instead of its inverse all fail one of the asserts.
+    rng = np.random.default_rng(5)
+    K = 96
+    X = rng.standard_normal((200, K)) * np.linspace(0.2, 3.0, K)   # distinct column energies
+    X[:, 7] = 0.0                                                  # a dead input feature
+    X[:, 40] = 0.0
+    H = X.T @ X
+    perm = rng.permutation(K).astype(np.int32) if use_perm else None
+    U = oracle.hessian_upper_cholesky(H, perm, damp=damp)
+    assert U.dtype == np.float32 and U.shape == (K, K)
+    assert np.array_equal(U, np.triu(U)) and (np.diag(U) > 0).all()
+    Hp = _damped_permuted(H, perm, damp)
+    U64 = U.astype(np.float64)
+    resid = U64.T @ U64 @ Hp - np.eye(K)
+    # U is stored in float32: 2^-24 relative per entry, amplified by the condition number (< 1e4 here)
+    assert np.abs(resid).max() < 2e-3
+    # the same identity without the amplification: R = U^-1 is upper triangular and R R^T = Hp
+    R = np.linalg.inv(U64)                      # upper triangular
+    assert np.abs(np.tril(R, -1)).max() < 1e-12
+    assert np.abs(R @ R.T - Hp).max() < 2e-6 * np.abs(Hp).max()
+    # (Hp carries the dead-column rule -- unit diagonal before the dampening, wherever the
+    # permutation put the column -- so a factor computed without it fails the identity above)
+
+
+def test_hessian_factor_of_a_diagonal_hessian_in_closed_form():
+    # H = diag(d): the dampened matrix is diag(d + damp * mean(d)), its inverse factor is
+    # diag(1 / sqrt(d + damp * mean(d))), permuted like the columns.
+    d = np.array([4.0, 1.0, 9.0, 16.0, 25.0, 0.25])
+    perm = np.array([2, 0, 5, 1, 4, 3], dtype=np.int32)
+    U = oracle.hessian_upper_cholesky(np.diag(d), perm, damp=0.05)
+    want = 1.0 / np.sqrt(d[perm] + 0.05 * d.mean())
+    assert np.allclose(np.diag(U), want, rtol=1e-6, atol=0)
+    assert np.array_equal(U, np.diag(np.diag(U)))

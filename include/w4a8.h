@@ -211,6 +211,80 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
                       float* s_x_out, void* stream);
 
 /*
+ * A chain of decode-sized layers in ONE persistent launch (Sec. 3 inference flow for every
+ * problem of the chain: Eq. 13 activation quantization, Eq. 10 weight dequantization, FP8 GEMM,
+ * Eq. 4 / Eq. 11 epilogue; Sec. 1 on the memory-bound regime of small batches this is for).
+ * Problem i computes  y_i = Linear_i( quantize_act( in_i ) )  with
+ *   in_i = x_i                                   (input_kind W4A8_CHAIN_INPUT_PLAIN), or
+ *   in_i = BF16( silu(G) * U ), G|U = x_i        (W4A8_CHAIN_INPUT_SILU_MUL: x_i has 2 K columns, gate
+ *                                                 first, exactly as w4a8_silu_mul_quantize defines it),
+ * and the results are those of w4a8_quantize_act (or w4a8_silu_mul_quantize) followed by
+ * w4a8_linear on the same tiled weights with K not cut: same scales, same FP8 codes, same
+ * accumulation order.  Problems run in array order on one grid of at most one CTA per SM that
+ * stays resident for the whole chain; the packed weights of the next problem are fetched while
+ * the current one is multiplied.
+ *   x_bf16       device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned), M <= W4A8_CHAIN_MAX_M.
+ *   depends_on   -1 when x_bf16 is complete before the call; otherwise the index (< i) of the
+ *                problem of this chain that WRITES the memory x_bf16 points into (normally
+ *                x_bf16 == that problem's y, out_dtype BF16): problem i is not quantized before
+ *                every row of that output has been written.  Buffers of problems that are not
+ *                linked this way must not overlap.
+ *   scale_mode, static_scale    as in w4a8_quantize_act.
+ *   weights      device, output of w4a8_prepack_weight; one tiled weight_format for the whole
+ *                chain.  K % 128 == 0, N % 16 == 0, N <= 256 rows per SM.
+ *   x8_out / s_x_out  optional (NULL): row-major copies of the FP8 activations [M][ldx8_out] and
+ *                of the M scales the layer multiplied with.
+ * workspace: device, 128-byte aligned, w4a8_linear_chain_workspace_bytes(problems, count) bytes:
+ * hand-over counters, activation scales and the FP8 activations as MMA operand tiles.  It must
+ * have been zero-filled once before its first use; every launch leaves the counters zero again
+ * (the last CTA to leave clears them, also after a time-out).  Launches that share a workspace
+ * must not overlap on the device; launches enqueued one after the other on one stream may share it.
+ * groups: 0 = the library's choice, 2..4 = number of 4-warp expansion groups (for tuning).
+ * Every device-side wait (on a pipeline barrier or on a hand-over counter) is bounded: when one
+ * runs out, all CTAs stop, outputs are incomplete and bit 0 of the device status word is set
+ * (w4a8_query_device_status returns W4A8_ERR_TIMEOUT).
+ * `problems` is a HOST array, read during the call only.  Errors: W4A8_ERR_INVALID_ARG (NULL,
+ * count outside 1..W4A8_CHAIN_MAX_PROBLEMS, bad enum, depends_on >= i, mixed weight formats),
+ * W4A8_ERR_BAD_SHAPE (M > 16, K % 128, N % 16, N too large, leading dimensions),
+ * W4A8_ERR_BAD_ALIGNMENT, W4A8_ERR_WORKSPACE_TOO_SMALL; nothing is enqueued on error.
+ */
+#define W4A8_CHAIN_INPUT_PLAIN 0
+#define W4A8_CHAIN_INPUT_SILU_MUL 1
+#define W4A8_CHAIN_MAX_PROBLEMS 24
+#define W4A8_CHAIN_MAX_M 16
+typedef struct w4a8_chain_problem {
+    const void* x_bf16;
+    int64_t ldx;
+    int32_t input_kind;
+    int32_t depends_on;
+    int32_t scale_mode;
+    int32_t weight_format;
+    const float* static_scale;
+    const uint8_t* weights;
+    const float* s_w;
+    int32_t sw_stride;
+    int32_t out_dtype;
+    int64_t M, N, K;
+    void* y;
+    int64_t ldy;
+    uint8_t* x8_out;
+    int64_t ldx8_out;
+    float* s_x_out;
+} w4a8_chain_problem;
+size_t w4a8_linear_chain_workspace_bytes(const w4a8_chain_problem* problems_host, int count);
+int w4a8_linear_chain(const w4a8_chain_problem* problems_host, int count, void* workspace,
+                      size_t workspace_bytes, int groups, void* stream);
+
+/*
+ * Self-test of the bounded device-side waits (the mechanism every kernel of the library uses; the
+ * paper has no counterpart): launches one CTA that waits, with a limit of `limit_ns` nanoseconds,
+ * on a pipeline barrier nobody ever arrives on.  The kernel must come back by itself, with bit 0 of
+ * the device status word set.  `elapsed_ns_dev` (device, one uint64, may be NULL) receives the time
+ * the wait took.  Nothing faults, traps or spins without a limit.
+ */
+int w4a8_selftest_bounded_wait(uint64_t limit_ns, uint64_t* elapsed_ns_dev, void* stream);
+
+/*
  * W4A16 comparison scheme (Sec. 4.3, Fig. 4): activations stay BF16, the INT4 codes are expanded
  * to BF16 on the fly and multiplied with BF16 tensor-core MMAs, FP32 accumulation:
  *   W16[n][k] = BF16( (u[n][k] - z[n][g]) * s_g[n][g] )      (one rounding to nearest even),

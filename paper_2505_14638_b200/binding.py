@@ -32,7 +32,25 @@ EXPORTS = (
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
+    "w4a8_linear_chain", "w4a8_linear_chain_workspace_bytes", "w4a8_selftest_bounded_wait",
 )
+
+CHAIN_INPUT_PLAIN, CHAIN_INPUT_SILU_MUL = 0, 1
+CHAIN_MAX_PROBLEMS, CHAIN_MAX_M = 24, 16
+
+
+class ChainProblem(ctypes.Structure):
+    """struct w4a8_chain_problem of include/w4a8.h, field for field."""
+    _fields_ = [
+        ("x_bf16", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+        ("input_kind", ctypes.c_int32), ("depends_on", ctypes.c_int32),
+        ("scale_mode", ctypes.c_int32), ("weight_format", ctypes.c_int32),
+        ("static_scale", ctypes.c_void_p), ("weights", ctypes.c_void_p), ("s_w", ctypes.c_void_p),
+        ("sw_stride", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+        ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+        ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64),
+        ("x8_out", ctypes.c_void_p), ("ldx8_out", ctypes.c_int64), ("s_x_out", ctypes.c_void_p),
+    ]
 
 _lib = None
 
@@ -100,6 +118,12 @@ def lib():
     L.w4a8_dpq_quantize.argtypes = [p, i64, i64, i32, p, p, i32, i32, i32, p, p, p, p, p, sz, p]
     L.w4a8_forward_host.restype = i32
     L.w4a8_forward_host.argtypes = [p, i64, p, p, p, i32, p, i32, i64, i64, i32, p, p, p, p, p, p, sz, p]
+    L.w4a8_linear_chain_workspace_bytes.restype = sz
+    L.w4a8_linear_chain_workspace_bytes.argtypes = [c.POINTER(ChainProblem), i32]
+    L.w4a8_linear_chain.restype = i32
+    L.w4a8_linear_chain.argtypes = [c.POINTER(ChainProblem), i32, p, sz, i32, p]
+    L.w4a8_selftest_bounded_wait.restype = i32
+    L.w4a8_selftest_bounded_wait.argtypes = [c.c_uint64, p, p]
     L.w4a8_query_device_status.restype = i32
     L.w4a8_query_device_status.argtypes = [c.POINTER(c.c_uint)]
     L.w4a8_launch_count.restype = c.c_uint64
@@ -418,6 +442,67 @@ def dpq_quantize(W, U, perm=None, symmetric=False, mse_steps=0, per_channel=Fals
                                  ws.numel(), _stream())
     _check("w4a8_dpq_quantize", rc)
     return codes, gscale, gzero, s_w
+
+
+def _addr(t):
+    return None if t is None else t.data_ptr()
+
+
+class LinearChain:
+    """w4a8_linear_chain: a list of decode-sized layers run by ONE persistent launch.
+
+    Build it once from problem descriptions (dicts with the keys x, weight, y and optionally
+    kind, depends_on, scale_mode, static_scale, x8_out, s_x_out), call it as often as wanted: the
+    argument array and the zero-filled workspace are kept.  x: BF16 [M, K] (or [M, 2K] for the
+    gated kind), weight: TiledWeight, y: BF16 or FP32 [M, N]; all on one device."""
+
+    def __init__(self, problems, groups=0, workspace=None):
+        import torch
+        n = len(problems)
+        self.arr = (ChainProblem * n)()
+        self.keep = problems          # keeps the tensors alive
+        for i, d in enumerate(problems):
+            x, tw, y = d["x"], d["weight"], d["y"]
+            kind = d.get("kind", CHAIN_INPUT_PLAIN)
+            assert x.dtype == torch.bfloat16 and x.stride(1) == 1 and y.stride(1) == 1
+            q = self.arr[i]
+            q.x_bf16, q.ldx = x.data_ptr(), x.stride(0)
+            q.input_kind, q.depends_on = kind, d.get("depends_on", -1)
+            q.scale_mode, q.weight_format = d.get("scale_mode", SCALE_EXACT), tw.fmt
+            q.static_scale = _addr(d.get("static_scale"))
+            q.weights, q.s_w = tw.buf.data_ptr(), tw.s_w.data_ptr()
+            q.sw_stride = 0 if tw.s_w.numel() == 1 else 1
+            q.out_dtype = OUT_FP32 if y.dtype == torch.float32 else OUT_BF16
+            q.M, q.N, q.K = x.shape[0], tw.N, tw.K
+            q.y, q.ldy = y.data_ptr(), y.stride(0)
+            x8o = d.get("x8_out")
+            q.x8_out, q.ldx8_out = _addr(x8o), (0 if x8o is None else x8o.stride(0))
+            q.s_x_out = _addr(d.get("s_x_out"))
+        self.n = n
+        self.groups = int(groups)
+        need = int(lib().w4a8_linear_chain_workspace_bytes(self.arr, n))
+        if need == 0:
+            _check("w4a8_linear_chain", lib().w4a8_linear_chain(self.arr, n, None, 0, self.groups, None))
+        self.need = need
+        dev = problems[0]["x"].device if problems[0]["x"].is_cuda else problems[0]["weight"].buf.device
+        self.ws = workspace if workspace is not None else torch.zeros((need,), dtype=torch.uint8, device=dev)
+        self._fn = lib().w4a8_linear_chain
+        self._wsp = ctypes.c_void_p(self.ws.data_ptr())
+        self._wsn = self.ws.numel()
+
+    def __call__(self):
+        rc = self._fn(self.arr, self.n, self._wsp, self._wsn, self.groups, _stream())
+        if rc != 0:
+            _check("w4a8_linear_chain", rc)
+
+
+def selftest_bounded_wait(limit_ns):
+    """w4a8_selftest_bounded_wait: returns the device-measured duration (ns) of a wait that runs out."""
+    import torch
+    out = torch.zeros((1,), dtype=torch.int64, device="cuda")
+    _check("w4a8_selftest_bounded_wait", lib().w4a8_selftest_bounded_wait(int(limit_ns), _ptr(out), _stream()))
+    torch.cuda.synchronize()
+    return int(out.item())
 
 
 class HostForward:

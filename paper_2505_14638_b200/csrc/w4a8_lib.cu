@@ -9,6 +9,7 @@
 
 #include "../../include/w4a8.h"
 #include "w4a8_dpq_kernels.cuh"
+#include "w4a8_linear_chain.cuh"
 #include "w4a8_linear_splitn.cuh"
 #include "w4a8_linear_pair.cuh"
 #include "w4a8_linear_streamk.cuh"
@@ -869,6 +870,168 @@ static int silu_mul_quantize_impl(const void* gu, int64_t M, int64_t F, int64_t 
     return launch_status();
 }
 
+// ------------------------------------------------------------------------------ chain of decode-sized layers
+static size_t chain_workspace_need(const w4a8_chain_problem* pr, int count) {
+    size_t need = kChainHeaderBytes;
+    for (int i = 0; i < count; ++i) need += (size_t)pr[i].K * kChainMaxM;   // [K/128][16][128] bytes
+    return need;
+}
+
+// Validation (device-independent part) of a chain description.
+static int chain_validate(const w4a8_chain_problem* pr, int count) {
+    if (!pr || count < 1 || count > kChainMaxProblems) return W4A8_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) {
+        const w4a8_chain_problem& q = pr[i];
+        if (!q.x_bf16 || !q.weights || !q.s_w || !q.y) return W4A8_ERR_INVALID_ARG;
+        if (q.M <= 0 || q.N <= 0 || q.K <= 0) return W4A8_ERR_INVALID_ARG;
+        if (q.input_kind != kChainKindPlain && q.input_kind != kChainKindSiluMul) return W4A8_ERR_INVALID_ARG;
+        if (q.depends_on < -1 || q.depends_on >= i) return W4A8_ERR_INVALID_ARG;
+        if (q.scale_mode != W4A8_SCALE_EXACT && q.scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
+        if (q.weight_format != kFmtTiled && q.weight_format != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+        if (q.weight_format != pr[0].weight_format) return W4A8_ERR_INVALID_ARG;
+        if (q.sw_stride != 0 && q.sw_stride != 1) return W4A8_ERR_INVALID_ARG;
+        if (q.out_dtype != W4A8_OUT_BF16 && q.out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
+        if (q.M > kChainMaxM || q.K % kGroup != 0 || q.N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
+        if (q.K > 16384 || q.N > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+        const int64_t in_cols = q.input_kind == kChainKindSiluMul ? 2 * q.K : q.K;
+        if (q.ldx < in_cols || q.ldy < q.N || (q.x8_out && q.ldx8_out < q.K)) return W4A8_ERR_BAD_SHAPE;
+        if (!aligned16(q.x_bf16) || !aligned16(q.y) || (q.ldx % 8) != 0 ||
+            (reinterpret_cast<uintptr_t>(q.weights) & 127u))
+            return W4A8_ERR_BAD_ALIGNMENT;
+        if (q.x8_out && (!aligned16(q.x8_out) || (q.ldx8_out % 16) != 0)) return W4A8_ERR_BAD_ALIGNMENT;
+        if ((reinterpret_cast<uintptr_t>(q.s_w) & 3u) || (reinterpret_cast<uintptr_t>(q.s_x_out) & 3u) ||
+            (reinterpret_cast<uintptr_t>(q.static_scale) & 3u))
+            return W4A8_ERR_BAD_ALIGNMENT;
+    }
+    return W4A8_OK;
+}
+
+template <class Cfg>
+static int launch_chain(const ChainParams& prm, int grid, int smem, uint8_t* ws, cudaStream_t st) {
+    auto kern = linear_chain_kernel<Cfg>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemMax);
+    });
+    if (attr_err != cudaSuccess) return W4A8_ERR_CUDA;
+    unsigned int* status = status_word_ptr();
+    if (!status) return W4A8_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(Cfg::kThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm, ws, status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) return W4A8_ERR_CUDA;
+    return launch_status();
+}
+
+static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* workspace, size_t workspace_bytes,
+                             int groups, cudaStream_t st) {
+    int rc = chain_validate(pr, count);
+    if (rc != W4A8_OK) return rc;
+    if (groups != 0 && (groups < 2 || groups > 4)) return W4A8_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < chain_workspace_need(pr, count)) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 127u) return W4A8_ERR_BAD_ALIGNMENT;
+    rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int sms = sm_count();
+    if (sms <= 0) return W4A8_ERR_CUDA;
+    const int fmt = pr[0].weight_format;
+    const int mb = meta_bytes(fmt);
+
+    ChainParams prm;
+    memset(&prm, 0, sizeof(prm));
+    prm.count = count;
+    prm.wait_limit_ns = ptx::kWaitLimitNs;
+    int grid = 1, wslot = 0, stash = 8192, jobs = 0;
+    size_t x8_off = kChainHeaderBytes;
+    for (int i = 0; i < count; ++i) {
+        const w4a8_chain_problem& q = pr[i];
+        ChainProblem& d = prm.prob[i];
+        d.x = static_cast<const uint16_t*>(q.x_bf16);
+        d.wpp = q.weights;
+        d.s_w = q.s_w;
+        d.y = q.y;
+        d.x8_out = q.x8_out;
+        d.s_x_out = q.s_x_out;
+        d.static_scale = q.static_scale;
+        d.ldx = q.ldx;
+        d.ldy = q.ldy;
+        d.ldx8_out = q.ldx8_out;
+        d.M = (int)q.M;
+        d.N = (int)q.N;
+        d.K = (int)q.K;
+        d.kind = q.input_kind;
+        d.dep = q.depends_on;
+        d.sw_stride = q.sw_stride;
+        d.out_dtype = q.out_dtype;
+        d.scale_mode = q.scale_mode;
+        const int64_t NU = q.N / 8;
+        const int64_t T = sms < NU ? sms : NU;
+        const int rmax = (int)((NU + T - 1) / T) * 8;
+        if (rmax > 256) return W4A8_ERR_BAD_SHAPE;
+        d.T = (int)T;
+        d.MBLK = rmax > 128 ? 2 : 1;
+        d.job_base = jobs;
+        jobs += d.M;
+        d.x8_off = (uint32_t)x8_off;
+        x8_off += (size_t)q.K * kChainMaxM;
+        if (x8_off > 0xFFFFFFFFull) return W4A8_ERR_BAD_SHAPE;
+        if ((int)T > grid) grid = (int)T;
+        // a slot holds two (k-block, 128-row block) items of the widest range of this problem
+        const int slot = ((2 / d.MBLK) * rmax * (kRowCodeBytes + mb) + 127) / 128 * 128;
+        if (slot > wslot) wslot = slot;
+        if (2 * (int)q.K > stash) stash = 2 * (int)q.K;
+    }
+    // every quantization job needs a CTA of its own kind of row: at least as many CTAs as tokens
+    if (grid < kChainMaxM) grid = kChainMaxM < sms ? kChainMaxM : sms;
+    prm.wslot = wslot;
+    prm.stash = stash;
+    using C0 = ChainCfg<3, kFmtTiledSignMag>;
+    const int fixed = 1024 + C0::kXRingBytes + stash + C0::kBarBytes;
+    int s1 = (C0::kSmemMax - fixed) / wslot;
+    if (s1 > C0::kS1Max) s1 = C0::kS1Max;
+    if (s1 < 3) return W4A8_ERR_BAD_SHAPE;
+    prm.S1 = s1;
+    const int smem = fixed + s1 * wslot;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (groups == 0) groups = 3;
+#define W4A8_CHAIN(GG)                                                                             \
+    (fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<GG, kFmtTiledSignMag>>(prm, grid, smem, ws, st) \
+                             : launch_chain<ChainCfg<GG, kFmtTiled>>(prm, grid, smem, ws, st))
+    switch (groups) {
+        case 2: return W4A8_CHAIN(2);
+        case 4: return W4A8_CHAIN(4);
+        default: return W4A8_CHAIN(3);
+    }
+#undef W4A8_CHAIN
+}
+
+// One CTA, one thread: a bounded wait on a barrier nobody arrives on (self-test of the time-out path).
+__global__ void bounded_wait_selftest_kernel(unsigned long long limit_ns, unsigned long long* elapsed,
+                                             unsigned int* status_word) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    __shared__ unsigned int chain_abort;
+    const uint32_t b = ptx::smem_addr(&bar);
+    ptx::mbar_init(b, 1);
+    abort_flag = 0u;
+    chain_abort = 0u;
+    ptx::fence_mbar_init();
+    const uint64_t t0 = ptx::globaltimer_ns();
+    const bool ok = chain_mbar_wait(b, 0u, &abort_flag, &chain_abort, status_word, limit_ns);
+    const uint64_t t1 = ptx::globaltimer_ns();
+    if (elapsed) *elapsed = ok ? 0ull : (unsigned long long)(t1 - t0);
+}
+
 }  // namespace w4a8
 
 using namespace w4a8;
@@ -1215,6 +1378,30 @@ int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights
     if (cudaMemcpyAsync(y_host_bf16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
     return W4A8_OK;
+}
+
+size_t w4a8_linear_chain_workspace_bytes(const w4a8_chain_problem* problems_host, int count) {
+    if (chain_validate(problems_host, count) != W4A8_OK) return 0;
+    return chain_workspace_need(problems_host, count);
+}
+
+int w4a8_linear_chain(const w4a8_chain_problem* problems_host, int count, void* workspace, size_t workspace_bytes,
+                      int groups, void* stream) {
+    return linear_chain_impl(problems_host, count, workspace, workspace_bytes, groups,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_selftest_bounded_wait(uint64_t limit_ns, uint64_t* elapsed_ns_dev, void* stream) {
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return W4A8_ERR_INVALID_ARG;   // at most one second
+    if (reinterpret_cast<uintptr_t>(elapsed_ns_dev) & 7u) return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    unsigned int* status = status_word_ptr();
+    if (!status) return W4A8_ERR_CUDA;
+    bounded_wait_selftest_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(
+        (unsigned long long)limit_ns, reinterpret_cast<unsigned long long*>(elapsed_ns_dev), status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
 }
 
 int w4a8_query_device_status(unsigned int* flags_host) {

@@ -1,0 +1,722 @@
+// One persistent launch for a chain of decode-sized W4A8 linear layers (M <= 16 tokens each) on
+// sm_100a: the whole inference flow of Sec. 3 -- Eq. 13 activation quantization, Eq. 10 weight
+// expansion, FP8 MMAs with FP32 accumulation, Eq. 4 / Eq. 11 epilogue -- for every problem of the
+// chain, in order, inside one kernel.
+//
+// Why one launch: a decode-sized layer streams its packed weights in a few microseconds, and the
+// hand-over between two dependent grids (completion of the first, release and start-up of the
+// second) costs about as much again.  Here one CTA per SM owns the whole SM for the whole chain:
+//   * the weight ring (bulk copies into ~190 KB of shared memory) never drains at a problem
+//     boundary: the codes of problem i + 1 depend on nothing and are fetched while problem i is
+//     still being multiplied;
+//   * the CTA has all 512 tensor-memory columns: seven stages of expanded weights in flight plus
+//     double-buffered accumulators, so the epilogue of problem i overlaps the MMAs of i + 1;
+//   * three or four dequantization groups (4 warps each) share the integer pipes, so the barrier
+//     round trips of one group hide behind the expansion work of the others;
+//   * problems are handed over through counters in the caller's workspace: the activations of a
+//     problem are quantized row by row by the epilogue warps of a few CTAs (one row per CTA),
+//     published with a fence and one atomic add, and picked up by every CTA's activation loader
+//     with a bounded acquire poll; a problem that reads the output of an earlier one waits (again
+//     bounded) for that problem's "rows written" counter first.
+//
+// Data path of one (k-block, 128-row block) item of a CTA's row range: as in the split-N kernel --
+//   HBM --bulk copy--> shared memory (INT4 codes + group scales [+ zero-points])
+//       --one thread per row: look-up-table expansion to E4M3 (Eq. 10)--> tensor memory (A operand)
+//       --tcgen05.mma kind::f8f6f4, B = FP8 activation tile from shared memory--> accumulator.
+// The FP8 activations of a problem live in the workspace as ready-made operand tiles
+// ([k-block][16 tokens][128 bytes], already in the 128-byte-swizzled order the MMA descriptor
+// expects), so a plain bulk copy brings a tile in: no tensor map, nothing to encode on the host.
+//
+// Every wait is bounded; on expiry the waiter raises the CTA's abort flag, the chain's abort word
+// (so that the other CTAs stop polling) and the time-out bit of the device status word.  The last
+// CTA to leave clears the control block, after an orderly run and after an aborted one alike.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "w4a8_ptx.cuh"
+#include "w4a8_simple_kernels.cuh"
+#include "w4a8_tiled_format.cuh"
+
+namespace w4a8 {
+
+constexpr int kChainMaxProblems = 24;
+constexpr int kChainMaxM = 16;            // tokens per problem = MMA N
+constexpr int kChainKindPlain = W4A8_CHAIN_INPUT_PLAIN;
+constexpr int kChainKindSiluMul = W4A8_CHAIN_INPUT_SILU_MUL;
+
+// One problem of the chain as the kernel sees it (filled by the host).
+struct ChainProblem {
+    const uint16_t* x;          // BF16 [M][ldx]: the layer's input, or gate|up (2 K columns) for the gated kind
+    const uint8_t* wpp;         // tiled weights
+    const float* s_w;
+    void* y;
+    uint8_t* x8_out;            // optional row-major copies of what the quantization produced
+    float* s_x_out;
+    const float* static_scale;  // nullptr = dynamic per-token scale
+    int64_t ldx, ldy, ldx8_out;
+    int M, N, K;
+    int kind;                   // kChainKind*
+    int dep;                    // index of the earlier problem whose output this one reads, or -1
+    int sw_stride, out_dtype, scale_mode;
+    int T;                      // row ranges: CTA p < T multiplies range p (8-row units [p NU / T, (p + 1) NU / T))
+    int MBLK;                   // 128-row blocks per range (1 or 2); k-blocks per stage = 2 / MBLK
+    int job_base;               // the quantization of row m runs on CTA (job_base + m) % gridDim.x
+    uint32_t x8_off;            // byte offset of this problem's FP8 activation tiles in the workspace
+};
+
+struct ChainParams {
+    ChainProblem prob[kChainMaxProblems];
+    int count;
+    int S1;       // depth of the weight ring
+    int wslot;    // bytes per weight-ring slot
+    int stash;    // bytes of the row stash (quantization) = output staging area (epilogue)
+    unsigned long long wait_limit_ns;
+};
+
+// Control block at the start of the workspace (zero-filled once by the caller, left zero by every launch).
+struct ChainCtl {
+    unsigned int exit_count;                  // CTAs that have left
+    unsigned int abort;                       // a wait ran out somewhere: stop polling
+    unsigned int pad[2];
+    unsigned int xready[kChainMaxProblems];   // rows of problem i quantized and published
+    unsigned int done[kChainMaxProblems];     // CTAs that have written their part of Y of problem i
+};
+constexpr size_t kChainCtlBytes = 1024;
+constexpr size_t kChainScaleBytes = (size_t)kChainMaxProblems * kChainMaxM * sizeof(float);
+constexpr size_t kChainHeaderBytes = kChainCtlBytes + 2048;   // control block, activation scales
+static_assert(sizeof(ChainCtl) <= kChainCtlBytes && kChainScaleBytes <= 2048, "workspace header");
+constexpr int kChainXTileBytes = kChainMaxM * 128;            // one k-block of FP8 activations: 16 tokens x 128 bytes
+
+template <int G_, int FMT_>
+struct ChainCfg {
+    static constexpr int G = G_;          // dequantization groups of 4 warps
+    static constexpr int FMT = FMT_;
+    static constexpr int kS1Max = 16;     // weight ring (runtime depth <= this)
+    static constexpr int kS2 = 7;         // stages of expanded weights in tensor memory = activation-tile slots
+    static constexpr int kMeta = meta_bytes(FMT_);
+    static constexpr int kAStageCols = 64;                    // two items of 32 columns
+    static constexpr int kDCol = kS2 * kAStageCols;           // 448: accumulators behind the A ring
+    static constexpr int kTmemCols = 512;
+    static constexpr int kFirstDqWarp = 8;
+    static constexpr int kThreads = 32 * (kFirstDqWarp + 4 * G_);
+    static constexpr int kBarBytes = 1024;
+    static constexpr int kXRingBytes = kS2 * 2 * kChainXTileBytes;
+    static constexpr int kSmemMax = 226 * 1024;
+    static_assert(kDCol + 2 * 2 * kChainMaxM <= kTmemCols, "tensor memory columns");
+    static_assert((2 * kS1Max + 3 * kS2 + 5) * 8 + 64 <= kBarBytes, "barrier area");
+};
+
+// Bounded acquire poll on a counter in global memory.
+__device__ __forceinline__ bool chain_poll_ge(const unsigned int* flag, unsigned int target, const unsigned int* gabort,
+                                              volatile uint32_t* abort_flag, unsigned int* gabort_w,
+                                              unsigned int* status_word, unsigned long long limit_ns) {
+    if (ptx::ld_acquire_gpu(flag) >= target) return true;
+    uint64_t t0 = 0;
+    uint32_t spins = 0;
+    while (true) {
+        if (ptx::ld_acquire_gpu(flag) >= target) return true;
+        if ((++spins & 15u) == 0u) {
+            if (*abort_flag) return false;
+            if (*reinterpret_cast<const volatile unsigned int*>(gabort)) {
+                *abort_flag = 1u;  // another CTA gave up: this one stops too
+                return false;
+            }
+            const uint64_t now = ptx::globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > limit_ns) {
+                *abort_flag = 1u;
+                atomicExch(gabort_w, 1u);
+                atomicOr(status_word, kStatusTimeout);
+                return false;
+            }
+        }
+    }
+}
+
+// All 32 lanes of a converged warp agree on whether to go on (a wait can run out for some lanes
+// and complete for others; the single-lane roles and the warp-collective tensor-memory stores
+// need the whole warp on one path).
+__device__ __forceinline__ bool warp_all(bool ok) { return __all_sync(0xFFFFFFFFu, ok) != 0; }
+
+// The same for the 128 threads of the epilogue role (named barrier 3 with an OR reduction).
+__device__ __forceinline__ bool epi_any(bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 3, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(r)
+        : "r"((uint32_t)flag)
+        : "memory");
+    return r != 0;
+}
+
+// mbarrier wait that also raises the chain's abort word when it runs out.
+__device__ __forceinline__ bool chain_mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                unsigned int* gabort_w, unsigned int* status_word,
+                                                unsigned long long limit_ns) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    uint64_t t0 = 0;
+    uint32_t spins = 0;
+    while (true) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            const uint64_t now = ptx::globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > limit_ns) {
+                *abort_flag = 1u;
+                atomicExch(gabort_w, 1u);
+                atomicOr(status_word, kStatusTimeout);
+                return false;
+            }
+        }
+    }
+}
+
+template <class Cfg>
+__global__ void __launch_bounds__(Cfg::kThreads, 1)
+linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict__ ws, unsigned int* status_word) {
+    constexpr int G = Cfg::G, S2 = Cfg::kS2, MB = Cfg::kMeta, S1M = Cfg::kS1Max;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - raw_addr);
+
+    const int S1 = prm.S1;
+    const uint32_t x_ring = base;                                            // [S2][2][2 KB], 1 KB aligned
+    const uint32_t w_ring = x_ring + (uint32_t)Cfg::kXRingBytes;             // [S1][wslot]
+    const uint32_t stash_off = (uint32_t)Cfg::kXRingBytes + (uint32_t)(S1 * prm.wslot);
+    const uint32_t stash_s = base + stash_off;                               // row stash / output staging
+    const uint32_t bars_off = stash_off + (uint32_t)prm.stash;
+    const uint32_t bars_addr = base + bars_off;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + bars_off);
+    const uint32_t bar_wfull0 = bars_addr;                                   // [S1M] packed codes + meta landed
+    const uint32_t bar_wfree0 = bars_addr + 8u * S1M;                        // [S1M] expanded: slot may be refilled
+    const uint32_t bar_xfull0 = bars_addr + 8u * (2 * S1M);                  // [S2]  activation tiles landed
+    const uint32_t bar_afull0 = bar_xfull0 + 8u * S2;                        // [S2]  expanded stage written to tensor memory
+    const uint32_t bar_afree0 = bar_afull0 + 8u * S2;                        // [S2]  stage consumed by the MMAs
+    const uint32_t bar_accfull0 = bar_afree0 + 8u * S2;                      // [2]
+    const uint32_t bar_accempty0 = bar_accfull0 + 16u;                       // [2]
+    const uint32_t bar_drain = bar_accempty0 + 16u;
+    constexpr int kNumBars = 2 * S1M + 3 * S2 + 5;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* red_s = reinterpret_cast<float*>(const_cast<uint32_t*>(tmem_slot) + 4);   // [4] warp maxima of a quantization job
+
+    ChainCtl* const ctl = reinterpret_cast<ChainCtl*>(ws);
+    float* const sx_ws = reinterpret_cast<float*>(ws + kChainCtlBytes);      // [problem][16] activation scales
+    unsigned int* const gabort = &ctl->abort;
+    const unsigned long long limit = prm.wait_limit_ns;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int p = blockIdx.x, P = gridDim.x;
+    const int count = prm.count;
+
+    if (threadIdx.x == 32) {
+        for (int s = 0; s < S1; ++s) {
+            ptx::mbar_init(bar_wfull0 + 8u * s, 1);
+            ptx::mbar_init(bar_wfree0 + 8u * s, 128);
+        }
+        for (int s = 0; s < S2; ++s) {
+            ptx::mbar_init(bar_xfull0 + 8u * s, 1);
+            ptx::mbar_init(bar_afull0 + 8u * s, 128);
+            ptx::mbar_init(bar_afree0 + 8u * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(bar_accfull0 + 8u * b, 1);
+            ptx::mbar_init(bar_accempty0 + 8u * b, 128);
+        }
+        ptx::mbar_init(bar_drain, 1);
+        *abort_flag = 0u;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 3) {
+        ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    ptx::griddep_launch_dependents();
+
+    // Geometry of this CTA's part of problem i.
+    struct Tile {
+        int R;        // rows
+        int n0;       // first row
+        int nst;      // pipeline stages
+        int KS;       // k-blocks per stage
+        int KB;
+    };
+    auto tile_of = [&](const ChainProblem& q) {
+        Tile t;
+        const int64_t NU = q.N >> 3;
+        const int u0 = (int)((int64_t)p * NU / q.T), u1 = (int)((int64_t)(p + 1) * NU / q.T);
+        t.R = (u1 - u0) * 8;
+        t.n0 = u0 * 8;
+        t.KS = 2 / q.MBLK;
+        t.KB = q.K >> 7;
+        t.nst = (t.KB + t.KS - 1) / t.KS;
+        return t;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ weight loader (one lane issues)
+        bool ok = true;
+        ptx::Ring r1;
+        int issued = 0;
+        for (int i = 0; i < count && ok; ++i) {
+            const ChainProblem& q = prm.prob[i];
+            if (p >= q.T) continue;
+            const Tile t = tile_of(q);
+            const int64_t code_step = (int64_t)q.N * kRowCodeBytes;   // one k-block further
+            const int64_t meta_step = (int64_t)q.N * MB;
+            const uint32_t cbytes = (uint32_t)(t.R * kRowCodeBytes), mbytes = (uint32_t)(t.R * MB);
+            const uint8_t* cptr = q.wpp + (int64_t)t.n0 * kRowCodeBytes;
+            const uint8_t* mptr = q.wpp + (int64_t)t.KB * code_step + (int64_t)t.n0 * MB;
+            const uint32_t meta_off = (uint32_t)t.KS * cbytes;
+            int kb = 0;
+            for (int st = 0; st < t.nst; ++st) {
+                ok = warp_all(chain_mbar_wait(bar_wfree0 + 8u * (uint32_t)r1.idx, r1.phase ^ 1u, abort_flag, gabort,
+                                              status_word, limit));
+                if (!ok) break;
+                const int ks = (t.KB - kb) < t.KS ? (t.KB - kb) : t.KS;
+                const uint32_t full = bar_wfull0 + 8u * (uint32_t)r1.idx;
+                const uint32_t wdst = w_ring + (uint32_t)(r1.idx * prm.wslot);
+                const uint32_t mdst = wdst + meta_off;
+                const uint8_t* cptr1 = cptr + code_step;
+                const uint8_t* mptr1 = mptr + meta_step;
+                if (ptx::elect_one()) {
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)ks * (cbytes + mbytes));
+                    ptx::bulk_load(wdst, cptr, cbytes, full);
+                    ptx::bulk_load(mdst, mptr, mbytes, full);
+                    if (ks == 2) {
+                        ptx::bulk_load(wdst + cbytes, cptr1, cbytes, full);
+                        ptx::bulk_load(mdst + mbytes, mptr1, mbytes, full);
+                    }
+                }
+                cptr += code_step * ks;
+                mptr += meta_step * ks;
+                kb += ks;
+                r1.advance(S1);
+                ++issued;
+            }
+        }
+        if (!ok && lane == 0) {
+            // Gave up: let the copies already in flight land before the CTA goes away.
+            ptx::Ring rb = r1;
+            const int n = issued < S1 ? issued : S1;
+            for (int i = 0; i < n; ++i) {
+                if (--rb.idx < 0) {
+                    rb.idx = S1 - 1;
+                    rb.phase ^= 1u;
+                }
+                const uint64_t t0 = ptx::globaltimer_ns();
+                while (!ptx::mbar_try_wait(bar_wfull0 + 8u * (uint32_t)rb.idx, rb.phase) &&
+                       ptx::globaltimer_ns() - t0 < limit) {
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one lane issues)
+        bool ok = true;
+        ptx::Ring r2;
+        int nacc = 0;
+        const uint32_t b_lo0 = ptx::umma_desc_lo(x_ring);
+        constexpr uint32_t b_step = (uint32_t)(2 * kChainXTileBytes) >> 4;
+        constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, kChainMaxM);
+        for (int i = 0; i < count && ok; ++i) {
+            const ChainProblem& q = prm.prob[i];
+            if (p >= q.T) continue;
+            const Tile t = tile_of(q);
+            const int buf = nacc & 1;
+            if (nacc >= 2) {
+                ok = warp_all(chain_mbar_wait(bar_accempty0 + 8u * (uint32_t)buf, (uint32_t)((nacc >> 1) - 1) & 1u,
+                                              abort_flag, gabort, status_word, limit));
+                if (!ok) break;
+            }
+            const uint32_t d0 = tmem_base + (uint32_t)(Cfg::kDCol + buf * 2 * kChainMaxM);
+            const bool two_blocks = q.MBLK == 2;
+            uint32_t accumulate = 0;
+            int kb = 0;
+            for (int st = 0; st < t.nst; ++st) {
+                ok = chain_mbar_wait(bar_xfull0 + 8u * (uint32_t)r2.idx, r2.phase, abort_flag, gabort, status_word, limit);
+                ok = ok && chain_mbar_wait(bar_afull0 + 8u * (uint32_t)r2.idx, r2.phase, abort_flag, gabort, status_word,
+                                           limit);
+                ok = warp_all(ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                // A stage holds two (k-block, 128-row block) items: two k-blocks of one row block,
+                // or one k-block of two row blocks.
+                const int ks = (t.KB - kb) < t.KS ? (t.KB - kb) : t.KS;
+                const uint32_t b_lo = b_lo0 + (uint32_t)r2.idx * b_step;
+                const uint32_t a_col = tmem_base + (uint32_t)(r2.idx * Cfg::kAStageCols);
+                const bool second = two_blocks || ks == 2;
+                const uint32_t b_lo1 = two_blocks ? b_lo : b_lo + ((uint32_t)kChainXTileBytes >> 4);
+                const uint32_t d1 = two_blocks ? d0 + (uint32_t)kChainMaxM : d0;
+                const uint32_t acc1 = two_blocks ? accumulate : 1u;
+                if (ptx::elect_one()) {
+                    ptx::umma_f8_kblock_ts(d0, a_col, b_lo, idesc, accumulate);
+                    if (second) ptx::umma_f8_kblock_ts(d1, a_col + 32u, b_lo1, idesc, acc1);
+                    ptx::umma_commit(bar_afree0 + 8u * (uint32_t)r2.idx);  // frees the expanded stage and its activation tiles
+                }
+                accumulate = 1u;
+                kb += ks;
+                r2.advance(S2);
+            }
+            if (!ok) break;
+            if (ptx::elect_one()) ptx::umma_commit(bar_accfull0 + 8u * (uint32_t)buf);
+            ++nacc;
+        }
+        if (!ok && lane == 0) {
+            // Gave up: wait (bounded) for the MMAs already issued before tensor memory is freed.
+            ptx::umma_commit(bar_drain);
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while (!ptx::mbar_try_wait(bar_drain, 0u) && ptx::globaltimer_ns() - t0 < limit) {
+            }
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ activation-tile loader (one lane issues)
+        bool ok = true;
+        ptx::Ring r2;
+        int issued = 0;
+        ptx::griddep_wait();  // the workspace and the counters belong to the previous launch until it has completed
+        for (int i = 0; i < count && ok; ++i) {
+            const ChainProblem& q = prm.prob[i];
+            if (p >= q.T) continue;
+            const Tile t = tile_of(q);
+            // the problem's activations must have been quantized (by the epilogue warps of M CTAs)
+            ok = warp_all(chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, gabort, status_word, limit));
+            if (!ok) break;
+            asm volatile("fence.proxy.async.global;" ::: "memory");  // their writes, before this thread's bulk copies
+            const uint8_t* xt = ws + q.x8_off;
+            const uint32_t rows_bytes = q.M <= 8 ? 1024u : 2048u;     // whole 8-row swizzle groups
+            int kb = 0;
+            for (int st = 0; st < t.nst; ++st) {
+                ok = warp_all(chain_mbar_wait(bar_afree0 + 8u * (uint32_t)r2.idx, r2.phase ^ 1u, abort_flag, gabort,
+                                              status_word, limit));
+                if (!ok) break;
+                const int ks = (t.KB - kb) < t.KS ? (t.KB - kb) : t.KS;
+                const uint32_t xfull = bar_xfull0 + 8u * (uint32_t)r2.idx;
+                const uint32_t xdst = x_ring + (uint32_t)(r2.idx * 2 * kChainXTileBytes);
+                const uint8_t* src = xt + (int64_t)kb * kChainXTileBytes;
+                if (ptx::elect_one()) {
+                    ptx::mbar_arrive_expect_tx(xfull, (uint32_t)ks * rows_bytes);
+                    ptx::bulk_load(xdst, src, rows_bytes, xfull);
+                    if (ks == 2) ptx::bulk_load(xdst + (uint32_t)kChainXTileBytes, src + kChainXTileBytes, rows_bytes, xfull);
+                }
+                kb += ks;
+                r2.advance(S2);
+                ++issued;
+            }
+        }
+        if (!ok && lane == 0) {
+            ptx::Ring rb = r2;
+            const int n = issued < S2 ? issued : S2;
+            for (int i = 0; i < n; ++i) {
+                if (--rb.idx < 0) {
+                    rb.idx = S2 - 1;
+                    rb.phase ^= 1u;
+                }
+                const uint64_t t0 = ptx::globaltimer_ns();
+                while (!ptx::mbar_try_wait(bar_xfull0 + 8u * (uint32_t)rb.idx, rb.phase) &&
+                       ptx::globaltimer_ns() - t0 < limit) {
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------------ quantization jobs + epilogue
+        const int qd = warp & 3;                 // tensor-memory lane quarter
+        const int r = qd * 32 + lane;            // row within a 128-row block
+        const int et = (warp - 4) * 32 + lane;   // index among the 128 threads of this role
+        bool ok = true;
+        ptx::griddep_wait();
+
+        // Eq. 13 for row m of problem j (one row per CTA): absmax, scale, FP8 codes written as
+        // operand tiles into the workspace, then published.  Called by all 128 threads.
+        auto quant_job = [&](int j, int m) -> bool {
+            const ChainProblem& q = prm.prob[j];
+            bool good = true;
+            if (q.dep >= 0) {
+                if (et == 0)
+                    good = chain_poll_ge(&ctl->done[q.dep], (unsigned)prm.prob[q.dep].T, gabort, abort_flag, gabort,
+                                         status_word, limit);
+                if (epi_any(!good)) return false;   // (also the barrier behind which every thread may read the input)
+            }
+            const int K = q.K;
+            const int nunits = K >> 4;  // 16 elements: 32 bytes of BF16 in, 16 bytes of FP8 out
+            const uint16_t* xrow = q.x + (int64_t)m * q.ldx;
+            float amax = 0.0f;
+            for (int u = et; u < nunits; u += 128) {
+                uint4 a, b;
+                if (q.kind == kChainKindSiluMul) {
+                    const uint4* gp = reinterpret_cast<const uint4*>(xrow) + 2 * u;
+                    const uint4* up = reinterpret_cast<const uint4*>(xrow + K) + 2 * u;
+                    const uint4 g0 = __ldcg(gp), g1 = __ldcg(gp + 1), u0 = __ldcg(up), u1 = __ldcg(up + 1);
+                    a.x = silu_mul_bf16x2(g0.x, u0.x);
+                    a.y = silu_mul_bf16x2(g0.y, u0.y);
+                    a.z = silu_mul_bf16x2(g0.z, u0.z);
+                    a.w = silu_mul_bf16x2(g0.w, u0.w);
+                    b.x = silu_mul_bf16x2(g1.x, u1.x);
+                    b.y = silu_mul_bf16x2(g1.y, u1.y);
+                    b.z = silu_mul_bf16x2(g1.z, u1.z);
+                    b.w = silu_mul_bf16x2(g1.w, u1.w);
+                } else {
+                    const uint4* xp = reinterpret_cast<const uint4*>(xrow) + 2 * u;
+                    a = __ldcg(xp);
+                    b = __ldcg(xp + 1);
+                }
+                amax = absmax_bf16x8(a, amax);
+                amax = absmax_bf16x8(b, amax);
+                ptx::st_shared_v4(stash_s + (uint32_t)u * 32u, a);
+                ptx::st_shared_v4(stash_s + (uint32_t)u * 32u + 16u, b);
+            }
+            float s, inv;
+            if (q.static_scale != nullptr) {
+                s = __ldg(q.static_scale);
+                inv = __fdiv_rn(1.0f, s);
+            } else {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+                if (lane == 0) red_s[warp - 4] = amax;
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                amax = fmaxf(fmaxf(red_s[0], red_s[1]), fmaxf(red_s[2], red_s[3]));
+                if (amax == 0.0f) {
+                    s = 1.0f;
+                    inv = 1.0f;
+                } else if (q.scale_mode == W4A8_SCALE_POW2) {
+                    s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
+                    inv = __fdiv_rn(1.0f, s);
+                } else {
+                    s = __fdiv_rn(amax, kE4M3Max);
+                    inv = __fdiv_rn(kE4M3Max, amax);
+                }
+            }
+            uint8_t* tiles = ws + q.x8_off;
+            for (int u = et; u < nunits; u += 128) {
+                uint4 a, b;
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w)
+                             : "r"(stash_s + (uint32_t)u * 32u));
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+                             : "r"(stash_s + (uint32_t)u * 32u + 16u));
+                const uint2 qa = quant_bf16x8(a, inv), qb = quant_bf16x8(b, inv);
+                const uint4 o = make_uint4(qa.x, qa.y, qb.x, qb.y);
+                // operand tile of k-block u / 8: token m is row m, its 16-byte chunk c sits at c ^ (m & 7)
+                const int kb = u >> 3, c = u & 7;
+                *reinterpret_cast<uint4*>(tiles + (int64_t)kb * kChainXTileBytes + m * 128 + ((c ^ (m & 7)) << 4)) = o;
+                if (q.x8_out != nullptr)
+                    *reinterpret_cast<uint4*>(q.x8_out + (int64_t)m * q.ldx8_out + (int64_t)u * 16) = o;
+            }
+            if (et == 0) {
+                sx_ws[j * kChainMaxM + m] = s;
+                if (q.s_x_out != nullptr) q.s_x_out[m] = s;
+            }
+            __threadfence();
+            asm volatile("bar.sync 3, 128;" ::: "memory");   // every thread's tiles are out (and the stash may be reused)
+            if (et == 0) atomicAdd(&ctl->xready[j], 1u);
+            return true;
+        };
+        auto my_row = [&](const ChainProblem& q) {
+            // the row of problem q this CTA quantizes, or -1
+            const int m = (int)(((unsigned)p + (unsigned)P - (unsigned)q.job_base % (unsigned)P) % (unsigned)P);
+            return m < q.M ? m : -1;
+        };
+
+        // problems whose input exists before the launch: quantized right away, by M CTAs each
+        for (int j = 0; j < count && ok; ++j) {
+            const ChainProblem& q = prm.prob[j];
+            if (q.dep >= 0) continue;
+            const int m = my_row(q);
+            if (m >= 0) ok = quant_job(j, m);
+        }
+
+        int nacc = 0;
+        for (int i = 0; i < count && ok; ++i) {
+            const ChainProblem& q = prm.prob[i];
+            if (p < q.T) {
+                const Tile t = tile_of(q);
+                const int es = q.out_dtype == W4A8_OUT_FP32 ? 4 : 2;
+                const bool wide_out = (((int64_t)q.ldy * es) & 15) == 0;  // rows of Y 16-byte aligned
+                float swn[2];
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+                    swn[b] = (b < q.MBLK && b * 128 + r < t.R)
+                                 ? __ldg(q.s_w + (int64_t)(t.n0 + b * 128 + r) * q.sw_stride)
+                                 : 0.0f;
+                // the scales were published together with the tiles the MMAs have consumed by now
+                ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, gabort, status_word, limit);
+                const float sx_mine = (ok && lane < q.M) ? __ldcg(sx_ws + i * kChainMaxM + lane) : 0.0f;
+                const int buf = nacc & 1;
+                ok = ok && chain_mbar_wait(bar_accfull0 + 8u * (uint32_t)buf, (uint32_t)(nacc >> 1) & 1u, abort_flag,
+                                           gabort, status_word, limit);
+                ok = !epi_any(!ok);   // all 128 threads take the same path (they meet at named barriers below)
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    if (b >= q.MBLK) break;
+                    uint32_t v[16];
+                    ptx::tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(qd * 32) << 16) +
+                                                (uint32_t)(Cfg::kDCol + buf * 2 * kChainMaxM + b * kChainMaxM),
+                                            v);
+                    ptx::tmem_ld_wait();
+                    float res[16];
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) {
+                        const float sxm = __shfl_sync(0xFFFFFFFFu, sx_mine, jj);
+                        res[jj] = __uint_as_float(v[jj]) * (sxm * swn[b]);  // Eq. 4, Eq. 11
+                    }
+                    const int row = b * 128 + r;
+                    if (wide_out) {
+                        // tokens x rows into the staging area, then 16-byte pieces of Y rows
+                        const uint32_t pitch = 128u * (uint32_t)es;
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const uint32_t a = stash_s + (uint32_t)jj * pitch + (uint32_t)(r * es);
+                            if (es == 4)
+                                asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[jj]) : "memory");
+                            else
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
+                                             "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[jj])))
+                                             : "memory");
+                        }
+                        asm volatile("bar.sync 3, 128;" ::: "memory");
+                        const int Rb = (t.R - b * 128) < 128 ? (t.R - b * 128) : 128;
+                        const int ppt = (Rb * es) >> 4;  // 16-byte pieces per token (rows come in eights)
+                        char* yb = static_cast<char*>(q.y) + ((int64_t)t.n0 + b * 128) * es;
+                        for (int id = et; id < q.M * ppt; id += 128) {
+                            const int tok = id / ppt, piece = id - tok * ppt;
+                            uint4 w;
+                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                                         : "r"(stash_s + (uint32_t)tok * pitch + (uint32_t)(piece << 4)));
+                            *reinterpret_cast<uint4*>(yb + (int64_t)tok * q.ldy * es + (piece << 4)) = w;
+                        }
+                        asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            if (jj < q.M && row < t.R) {
+                                const int64_t o = (int64_t)jj * q.ldy + t.n0 + row;
+                                if (es == 4)
+                                    reinterpret_cast<float*>(q.y)[o] = res[jj];
+                                else
+                                    reinterpret_cast<__nv_bfloat16*>(q.y)[o] = __float2bfloat16_rn(res[jj]);
+                            }
+                        }
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(bar_accempty0 + 8u * (uint32_t)buf);
+                ++nacc;
+                // this CTA's rows of Y are written: publish
+                __threadfence();
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (et == 0) atomicAdd(&ctl->done[i], 1u);
+            }
+            // problems that read the output of problem i: quantize this CTA's row of them now
+            for (int j = i + 1; j < count && ok; ++j) {
+                const ChainProblem& qj = prm.prob[j];
+                if (qj.dep != i) continue;
+                const int m = my_row(qj);
+                if (m >= 0) ok = quant_job(j, m);
+            }
+        }
+    } else if (warp >= Cfg::kFirstDqWarp) {
+        // ------------------------------------------------------------------ dequantization groups
+        const int dw = warp - Cfg::kFirstDqWarp;
+        const int g = dw >> 2;
+        const int qd = warp & 3;          // tensor-memory lane quarter this warp may access
+        const int r = qd * 32 + lane;     // row within a 128-row block
+        // Group g expands every G-th stage, counted across problems.
+        ptx::Ring r1, r2;
+        for (int i = 0; i < g; ++i) {
+            r1.advance(S1);
+            r2.advance(S2);
+        }
+        int turn = g;  // stages until this group's next turn
+        bool ok = true;
+        for (int i = 0; i < count && ok; ++i) {
+            const ChainProblem& q = prm.prob[i];
+            if (p >= q.T) continue;
+            const Tile t = tile_of(q);
+            const int MBLK = q.MBLK;
+            // This thread's rows of the range (one per 128-row block).  A lane beyond the range
+            // repeats the last row: its tensor-memory lane feeds accumulator rows nobody reads out.
+            const int row0 = r < t.R ? r : t.R - 1;
+            const int row1 = 128 + r < t.R ? 128 + r : t.R - 1;
+            const uint32_t code_off = tiled_row_offset(row0);
+            const uint32_t meta_off = (uint32_t)(t.KS * t.R * kRowCodeBytes + row0 * MB);
+            const uint32_t code_kstep = (uint32_t)(t.R * kRowCodeBytes), meta_kstep = (uint32_t)(t.R * MB);
+            const uint32_t code_s0 = MBLK == 2 ? tiled_row_offset(row1) - code_off : code_kstep;
+            const uint32_t meta_s0 = MBLK == 2 ? (uint32_t)((row1 - row0) * MB) : meta_kstep;
+            int st = turn;
+            for (; st < t.nst; st += G) {
+                const int kb = st * t.KS;
+                const int ks = (t.KB - kb) < t.KS ? (t.KB - kb) : t.KS;
+                const uint32_t full_bar = bar_wfull0 + 8u * (uint32_t)r1.idx;
+                const uint32_t free_bar = bar_afree0 + 8u * (uint32_t)r2.idx;
+                // both are normally complete already: test them together, wait only if not
+                const bool have_w = ptx::mbar_test_wait(full_bar, r1.phase);
+                const bool have_slot = ptx::mbar_test_wait(free_bar, r2.phase ^ 1u);
+                if (!have_w) ok = chain_mbar_wait(full_bar, r1.phase, abort_flag, gabort, status_word, limit);
+                if (ok && !have_slot) ok = chain_mbar_wait(free_bar, r2.phase ^ 1u, abort_flag, gabort, status_word, limit);
+                ok = warp_all(ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * prm.wslot);
+                const uint32_t a_col = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(r2.idx * Cfg::kAStageCols);
+                if (ks * MBLK == 2)
+                    dequant_two_rows_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, wsrc + code_off + code_s0,
+                                                       wsrc + meta_off + meta_s0, a_col);
+                else
+                    dequant_row_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, a_col);
+                ptx::mbar_arrive(bar_wfree0 + 8u * (uint32_t)r1.idx);   // this thread has read its codes
+                ptx::tmem_st_wait();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(bar_afull0 + 8u * (uint32_t)r2.idx);
+                for (int a = 0; a < G; ++a) {
+                    r1.advance(S1);
+                    r2.advance(S2);
+                }
+            }
+            turn = st - t.nst;
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 3) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+    if (threadIdx.x == 0) {
+        // The last CTA to leave clears the control block (nobody polls it any more), so that the
+        // next launch -- which touches it only after this one has completed -- finds zeros.
+        ptx::griddep_wait();
+        __threadfence();
+        if (atomicAdd(&ctl->exit_count, 1u) == (unsigned)P - 1u) {
+            for (int i = 0; i < kChainMaxProblems; ++i) {
+                ctl->xready[i] = 0u;
+                ctl->done[i] = 0u;
+            }
+            ctl->abort = 0u;
+            ctl->exit_count = 0u;
+            __threadfence();
+        }
+    }
+}
+
+}  // namespace w4a8

@@ -141,6 +141,56 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t src, uint32_t meta,
     }
 }
 
+// The expansion of one row whose codes and meta word are already in registers.
+template <int FMT>
+__device__ __forceinline__ void expand_row_to_tmem(const uint32_t (&pk)[16], uint32_t mbits, uint32_t taddr) {
+    const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
+    if constexpr (FMT == kFmtTiledSignMag) {
+        SignMagLut lut;
+        lut.build(sc);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t out[16];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) lut.dequant8(pk[8 * h + w], out[2 * w], out[2 * w + 1]);
+            ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
+        }
+    } else {
+        DequantLut lut;
+        lut.build(sc, (int)((mbits >> 16) & 0xFFu));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t out[16];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) lut.dequant8(pk[8 * h + w], out[2 * w], out[2 * w + 1]);
+            ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t load_meta_word(uint32_t meta, int fmt) {
+    uint32_t mbits;
+    if (fmt == kFmtTiledSignMag)
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    else
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    return mbits;
+}
+
+// Two rows (two items of one pipeline stage) expanded into 2 x 32 consecutive tensor-memory
+// columns: all ten shared-memory loads are issued before the first look-up, so that the second
+// row's loads are in flight while the first row is expanded.  Warp-collective.
+template <int FMT>
+__device__ __forceinline__ void dequant_two_rows_to_tmem(uint32_t src0, uint32_t meta0, uint32_t src1, uint32_t meta1,
+                                                         uint32_t taddr) {
+    uint32_t pa[16], pb[16];
+    const uint32_t m0 = load_meta_word(meta0, FMT), m1 = load_meta_word(meta1, FMT);
+    load_row_codes(src0, pa);
+    load_row_codes(src1, pb);
+    expand_row_to_tmem<FMT>(pa, m0, taddr);
+    expand_row_to_tmem<FMT>(pb, m1, taddr + 32u);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Offline prepack: canonical [N][K/2] codes + [N][K/128] scales (+ zero-points) -> tiled buffer.
 // One CTA per (128 rows, k-block), one thread per row.  In the sign-magnitude format a code 0

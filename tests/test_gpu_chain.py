@@ -1,0 +1,248 @@
+"""GPU parity: w4a8_linear_chain (a chain of decode-sized layers in one persistent launch) against
+the oracle's forward pass (Sec. 3 flow: Eq. 13 -> Eq. 10 -> FP8 matmul -> Eq. 4 / Eq. 11) and, bit
+for bit, against the per-launch path (w4a8_quantize_act / w4a8_silu_mul_quantize + w4a8_linear).
+The FP8 activations and scales the chain used are read back and must be bit-exact; the output
+gate is max relative error 2e-3 before the BF16 cast and one BF16 step after it."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_utils import bf16_bits, bf16_dev, dev, weights_to_dev
+from helpers import bf16_gate, fp32_gate
+from paper_2505_14638_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _weights(N, K, seed, asym=False, sigma=0.02):
+    W = inputs.make_weight(N, K, sigma, seed)
+    wq = oracle.quantize_weight_rtn(W, symmetric=not asym, per_channel=asym)
+    fmt = binding.FMT_TILED if asym else binding.FMT_TILED_SIGNMAG
+    tw = binding.prepack_weight(*weights_to_dev(*wq), weight_format=fmt)
+    return wq, tw
+
+
+def _oracle_layer(xb, wq, pow2=False):
+    x8, s_x = oracle.quantize_act(xb, scale_mode=1 if pow2 else 0)
+    ref = oracle.linear(x8, s_x, oracle.dequant_weight(*wq[:3]), wq[3])
+    return x8, s_x, ref
+
+
+def _per_launch(x, tw, out_dtype):
+    """The two-kernel path on the same weights, K never cut (a workspace too small for partial sums)."""
+    tiny = torch.zeros((16,), dtype=torch.uint8, device="cuda")
+    x8, s_x = binding.quantize_act(x)
+    return binding.linear_tiled(x8, s_x, tw, out_dtype=out_dtype, workspace=tiny)
+
+
+@pytest.mark.parametrize("groups", [0, 2, 4])
+@pytest.mark.parametrize("asym", [False, True])
+def test_independent_problems_match_oracle_and_per_launch_path(groups, asym):
+    # three problems of different token counts and shapes in one launch: a ragged row partition,
+    # an odd number of k-blocks (last stage holds one), few rows per CTA, M <= 8 and M > 8
+    shapes = [(1, 2368, 640), (4, 4736, 384), (16, 1024, 1024), (7, 48, 256), (9, 16, 128)]
+    probs, refs = [], []
+    for i, (M, N, K) in enumerate(shapes):
+        wq, tw = _weights(N, K, 50 + i, asym)
+        xb = inputs.make_activation(M, K, 60 + i, 0.01, 20.0)
+        x = bf16_dev(xb)
+        y = torch.full((M, N), 7.0, dtype=torch.float32, device="cuda")
+        x8o = torch.full((M, K), 0xAA, dtype=torch.uint8, device="cuda")
+        sxo = torch.full((M,), -1.0, dtype=torch.float32, device="cuda")
+        probs.append(dict(x=x, weight=tw, y=y, x8_out=x8o, s_x_out=sxo))
+        refs.append((xb, wq))
+    chain = binding.LinearChain(probs, groups=groups)
+    chain()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for d, (xb, wq) in zip(probs, refs):
+        x8, s_x, ref = _oracle_layer(xb, wq)
+        assert np.array_equal(d["s_x_out"].cpu().numpy().view(np.uint32), s_x.astype(np.float32).view(np.uint32))
+        assert np.array_equal(d["x8_out"].cpu().numpy(), x8)
+        worst, _ = fp32_gate(d["y"].cpu().numpy(), ref["y64"], rel=2e-3)
+        assert worst <= 2e-3, worst
+        want = _per_launch(d["x"], d["weight"], binding.OUT_FP32)
+        torch.cuda.synchronize()
+        assert torch.equal(d["y"], want)
+
+
+def test_exact_integer_problem_is_bit_exact():
+    # group scales 1, small integer activations: every partial sum is an exact integer below 2^24,
+    # so any accumulation order gives the oracle's value bit for bit -- a layout test of the
+    # activation tiles (token row, swizzled 16-byte chunks) and of the row ranges
+    rng = np.random.default_rng(3)
+    M, N, K = 13, 2368, 512
+    codes_u = rng.integers(1, 16, size=(N, K), dtype=np.int32)
+    from helpers import pack_codes
+    codes = pack_codes(codes_u)
+    gscale = np.full((N, K // 128), 0x3F80, dtype=np.uint16)     # BF16 1.0
+    s_w = np.ones((1,), dtype=np.float32)
+    tw = binding.prepack_weight(dev(codes), bf16_dev(gscale), None, dev(s_w), weight_format=binding.FMT_TILED_SIGNMAG)
+    xi = rng.integers(-3, 4, size=(M, K)).astype(np.float32)
+    xi[:, 5] = 4.0                                               # every row's absmax is 4: s_x = 4 / 448 exactly
+    xb = (xi.view(np.uint32) >> 16).astype(np.uint16)
+    x8, s_x = oracle.quantize_act(xb)
+    ref = oracle.linear(x8, s_x, oracle.dequant_weight(codes, gscale, None), s_w)
+    y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    chain = binding.LinearChain([dict(x=bf16_dev(xb), weight=tw, y=y)])
+    chain()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert np.array_equal(y.cpu().numpy(), ref["y32"])
+
+
+def test_dependent_chain_and_gated_block():
+    # x -> gate_up (BF16) -> silu(gate) * up quantized in the chain -> down (BF16) -> next layer on
+    # the down projection's output: every hand-over goes through the chain's counters
+    M, H, F = 5, 1024, 1408
+    wq_gu, tw_gu = _weights(2 * F, H, 70)
+    wq_dn, tw_dn = _weights(H, F, 71)
+    wq_nx, tw_nx = _weights(2304, H, 72)
+    xb = inputs.make_activation(M, H, 73, 0.01, 20.0)
+    x = bf16_dev(xb)
+    gu = torch.zeros((M, 2 * F), dtype=torch.bfloat16, device="cuda")
+    dn = torch.zeros((M, H), dtype=torch.bfloat16, device="cuda")
+    nx = torch.zeros((M, 2304), dtype=torch.float32, device="cuda")
+    x8_dn = torch.zeros((M, F), dtype=torch.uint8, device="cuda")
+    sx_dn = torch.zeros((M,), dtype=torch.float32, device="cuda")
+    chain = binding.LinearChain([
+        dict(x=x, weight=tw_gu, y=gu),
+        dict(x=gu, weight=tw_dn, y=dn, kind=binding.CHAIN_INPUT_SILU_MUL, depends_on=0, x8_out=x8_dn, s_x_out=sx_dn),
+        dict(x=dn, weight=tw_nx, y=nx, depends_on=1),
+    ])
+    # the same block launch by launch
+    tiny = torch.zeros((16,), dtype=torch.uint8, device="cuda")
+    x8, s_x = binding.quantize_act(x)
+    gu_ref = binding.linear_tiled(x8, s_x, tw_gu, workspace=tiny)
+    h8, s_h = binding.silu_mul_quantize(gu_ref)
+    dn_ref = binding.linear_tiled(h8, s_h, tw_dn, workspace=tiny)
+    d8, s_d = binding.quantize_act(dn_ref)
+    nx_ref = binding.linear_tiled(d8, s_d, tw_nx, out_dtype=binding.OUT_FP32, workspace=tiny)
+    for _ in range(3):     # repeated launches: the counters reset themselves
+        gu.zero_(); dn.zero_(); nx.zero_()
+        chain()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.equal(gu, gu_ref)
+    assert torch.equal(x8_dn, h8) and torch.equal(sx_dn, s_h)
+    assert torch.equal(dn, dn_ref)
+    assert torch.equal(nx, nx_ref)
+    # and the first layer against the oracle (the later ones are covered through the bit-equality
+    # with the per-launch path, whose kernels have their own oracle tests)
+    _, _, ref = _oracle_layer(xb, wq_gu)
+    ok, dist = bf16_gate(bf16_bits(gu), ref["y64"])
+    assert ok, dist
+
+
+def test_two_row_blocks_per_cta_and_graph_replay():
+    # N = 28672: 194 rows per CTA (two 128-row blocks); replayed from a CUDA graph many times
+    M, N, K = 3, 28672, 256
+    wq, tw = _weights(N, K, 80)
+    xb = inputs.make_activation(M, K, 81)
+    x = bf16_dev(xb)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.zeros((16, 1024), dtype=torch.bfloat16, device="cuda")
+    wq2, tw2 = _weights(1024, K, 82)
+    xb2 = inputs.make_activation(16, K, 83)
+    chain = binding.LinearChain([dict(x=x, weight=tw, y=y), dict(x=bf16_dev(xb2), weight=tw2, y=y2)])
+    chain()
+    torch.cuda.synchronize()
+    first = (y.clone(), y2.clone())
+    _, _, ref = _oracle_layer(xb, wq)
+    ok, dist = bf16_gate(bf16_bits(y), ref["y64"])
+    assert ok, dist
+    _, _, ref2 = _oracle_layer(xb2, wq2)
+    ok, dist = bf16_gate(bf16_bits(y2), ref2["y64"])
+    assert ok, dist
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(4):
+                chain()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(10):
+        y.zero_(); y2.zero_()
+        g.replay()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.equal(y, first[0]) and torch.equal(y2, first[1])
+
+
+def test_pow2_and_static_scales():
+    M, N, K = 6, 512, 512
+    wq, tw = _weights(N, K, 90)
+    xb = inputs.make_activation(M, K, 91, 0.01, 20.0)
+    x = bf16_dev(xb)
+    ss = dev(np.array([0.05], dtype=np.float32))
+    outs = [torch.zeros((M, N), dtype=torch.float32, device="cuda") for _ in range(2)]
+    x8s = [torch.zeros((M, K), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    sxs = [torch.zeros((M,), dtype=torch.float32, device="cuda") for _ in range(2)]
+    chain = binding.LinearChain([
+        dict(x=x, weight=tw, y=outs[0], scale_mode=binding.SCALE_POW2, x8_out=x8s[0], s_x_out=sxs[0]),
+        dict(x=x, weight=tw, y=outs[1], static_scale=ss, x8_out=x8s[1], s_x_out=sxs[1]),
+    ])
+    chain()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for k, kw in enumerate((dict(scale_mode=1), dict(static_scale=0.05))):
+        x8, s_x = oracle.quantize_act(xb, **kw)
+        assert np.array_equal(x8s[k].cpu().numpy(), x8)
+        assert np.array_equal(sxs[k].cpu().numpy().view(np.uint32), s_x.astype(np.float32).view(np.uint32))
+        ref = oracle.linear(x8, s_x, oracle.dequant_weight(*wq[:3]), wq[3])
+        worst, _ = fp32_gate(outs[k].cpu().numpy(), ref["y64"], rel=2e-3)
+        assert worst <= 2e-3, worst
+
+
+def test_chain_argument_errors():
+    M, N, K = 4, 256, 256
+    wq, tw = _weights(N, K, 95)
+    x = bf16_dev(inputs.make_activation(M, K, 96))
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    good = binding.LinearChain([dict(x=x, weight=tw, y=y)])
+    L = binding.lib()
+    arr = good.arr
+    ws = ctypes.c_void_p(good.ws.data_ptr())
+    assert L.w4a8_linear_chain(arr, 0, ws, good.need, 0, None) == binding.ERR_INVALID_ARG
+    assert L.w4a8_linear_chain(arr, 25, ws, good.need, 0, None) == binding.ERR_INVALID_ARG
+    assert L.w4a8_linear_chain(arr, 1, ws, good.need - 1, 0, None) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert L.w4a8_linear_chain(arr, 1, ws, good.need, 7, None) == binding.ERR_INVALID_ARG
+    arr[0].depends_on = 0
+    assert L.w4a8_linear_chain(arr, 1, ws, good.need, 0, None) == binding.ERR_INVALID_ARG
+    arr[0].depends_on = -1
+    arr[0].M = 17
+    assert L.w4a8_linear_chain(arr, 1, ws, good.need, 0, None) == binding.ERR_BAD_SHAPE
+    arr[0].M = M
+    arr[0].ldx = K - 8
+    assert L.w4a8_linear_chain(arr, 1, ws, good.need, 0, None) == binding.ERR_BAD_SHAPE
+    arr[0].ldx = K
+    assert L.w4a8_linear_chain(arr, 1, ctypes.c_void_p(good.ws.data_ptr() + 16), good.need, 0, None) == \
+        binding.ERR_BAD_ALIGNMENT
+    good()     # still launches after the rejected calls
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_library_carries_on():
+    # one CTA waits, with a limit of one millisecond, on a barrier nobody arrives on: the kernel
+    # returns by itself, the status word carries the time-out bit, the query reports and clears it,
+    # and the next ordinary call is correct
+    took = binding.selftest_bounded_wait(1_000_000)
+    assert 1_000_000 <= took < 50_000_000, took
+    flags = ctypes.c_uint(0)
+    assert binding.lib().w4a8_query_device_status(ctypes.byref(flags)) == binding.ERR_TIMEOUT
+    assert flags.value & 1
+    assert binding.query_device_status() == 0      # cleared by the query
+    M, N, K = 4, 512, 256
+    wq, tw = _weights(N, K, 97)
+    xb = inputs.make_activation(M, K, 98)
+    y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    binding.LinearChain([dict(x=bf16_dev(xb), weight=tw, y=y)])()
+    torch.cuda.synchronize()
+    _, _, ref = _oracle_layer(xb, wq)
+    worst, _ = fp32_gate(y.cpu().numpy(), ref["y64"], rel=2e-3)
+    assert worst <= 2e-3 and binding.query_device_status() == 0

@@ -220,9 +220,15 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
  *                                                 first, exactly as w4a8_silu_mul_quantize defines it),
  * and the results are those of w4a8_quantize_act (or w4a8_silu_mul_quantize) followed by
  * w4a8_linear on the same tiled weights with K not cut: same scales, same FP8 codes, same
- * accumulation order.  Problems run in array order on one grid of at most one CTA per SM that
- * stays resident for the whole chain; the packed weights of the next problem are fetched while
- * the current one is multiplied.
+ * accumulation order -- for the output channels whose K range one CTA walks alone; where the chain
+ * cuts K (see below) the FP32 partial sums are added in a fixed order, so results still repeat bit
+ * for bit from call to call, and agree with w4a8_linear within its output tolerance.  Problems run
+ * in array order on one grid of one CTA per SM that stays resident for the whole chain; the packed
+ * weights of the next problem are fetched while the current one is multiplied.
+ * Partition: the output channels are cut into blocks of 96; while at least as many blocks as SMs
+ * are left every CTA takes whole blocks, the remaining blocks are cut along K as well, into runs of
+ * at least four 128-wide k-blocks, and the CTA that holds a block's lowest k range adds the
+ * partial sums of the others (FP32, through the workspace) before it scales and writes the rows.
  *   x_bf16       device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned), M <= W4A8_CHAIN_MAX_M.
  *   depends_on   -1 when x_bf16 is complete before the call; otherwise the index (< i) of the
  *                problem of this chain that WRITES the memory x_bf16 points into (normally
@@ -231,15 +237,16 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
  *                linked this way must not overlap.
  *   scale_mode, static_scale    as in w4a8_quantize_act.
  *   weights      device, output of w4a8_prepack_weight; one tiled weight_format for the whole
- *                chain.  K % 128 == 0, N % 16 == 0, N <= 256 rows per SM.
+ *                chain.  K % 128 == 0, K <= 16384, N % 16 == 0, N <= 1152 rows per SM.
  *   x8_out / s_x_out  optional (NULL): row-major copies of the FP8 activations [M][ldx8_out] and
  *                of the M scales the layer multiplied with.
  * workspace: device, 128-byte aligned, w4a8_linear_chain_workspace_bytes(problems, count) bytes:
- * hand-over counters, activation scales and the FP8 activations as MMA operand tiles.  It must
+ * hand-over counters, activation scales, the FP8 activations as MMA operand tiles and the
+ * partial sums of the blocks that are cut along K.  It must
  * have been zero-filled once before its first use; every launch leaves the counters zero again
  * (the last CTA to leave clears them, also after a time-out).  Launches that share a workspace
  * must not overlap on the device; launches enqueued one after the other on one stream may share it.
- * groups: 0 = the library's choice, 2..4 = number of 4-warp expansion groups (for tuning).
+ * groups: 0 = the library's choice, 2..4 = number of 3-warp expansion groups (for tuning).
  * Every device-side wait (on a pipeline barrier or on a hand-over counter) is bounded: when one
  * runs out, all CTAs stop, outputs are incomplete and bit 0 of the device status word is set
  * (w4a8_query_device_status returns W4A8_ERR_TIMEOUT).

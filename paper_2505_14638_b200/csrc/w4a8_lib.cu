@@ -871,9 +871,17 @@ static int silu_mul_quantize_impl(const void* gu, int64_t M, int64_t F, int64_t 
 }
 
 // ------------------------------------------------------------------------------ chain of decode-sized layers
+// Workspace layout: header (control block, activation scales), then per problem the FP8 activation
+// tiles ([K/128][16][128] bytes), the partial-sum slots of the blocks that are cut along K (one per
+// CTA, M x 96 floats) and their arrival counters.  Sized for any SM count up to kMaxSMs so that
+// the query needs no device.
+constexpr size_t kChainCntBytes = 1024;
+static_assert(kMaxSMs * sizeof(unsigned int) <= kChainCntBytes, "one counter per block that is cut along K");
+static size_t chain_part_bytes(int64_t M, int ctas) { return (size_t)ctas * (size_t)M * kChainBlockRows * sizeof(float); }
 static size_t chain_workspace_need(const w4a8_chain_problem* pr, int count) {
     size_t need = kChainHeaderBytes;
-    for (int i = 0; i < count; ++i) need += (size_t)pr[i].K * kChainMaxM;   // [K/128][16][128] bytes
+    for (int i = 0; i < count; ++i)
+        need += (size_t)pr[i].K * kChainMaxM + chain_part_bytes(pr[i].M, kMaxSMs) + kChainCntBytes;
     return need;
 }
 
@@ -892,7 +900,7 @@ static int chain_validate(const w4a8_chain_problem* pr, int count) {
         if (q.sw_stride != 0 && q.sw_stride != 1) return W4A8_ERR_INVALID_ARG;
         if (q.out_dtype != W4A8_OUT_BF16 && q.out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
         if (q.M > kChainMaxM || q.K % kGroup != 0 || q.N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
-        if (q.K > 16384 || q.N > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
+        if (q.K > 16384 || q.N > (1 << 20)) return W4A8_ERR_BAD_SHAPE;
         const int64_t in_cols = q.input_kind == kChainKindSiluMul ? 2 * q.K : q.K;
         if (q.ldx < in_cols || q.ldy < q.N || (q.x8_out && q.ldx8_out < q.K)) return W4A8_ERR_BAD_SHAPE;
         if (!aligned16(q.x_bf16) || !aligned16(q.y) || (q.ldx % 8) != 0 ||
@@ -943,7 +951,7 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
     rc = check_device();
     if (rc != W4A8_OK) return rc;
     const int sms = sm_count();
-    if (sms <= 0) return W4A8_ERR_CUDA;
+    if (sms < kChainMaxM || sms > kMaxSMs) return W4A8_ERR_UNSUPPORTED_DEVICE;   // one quantization job per CTA and problem
     const int fmt = pr[0].weight_format;
     const int mb = meta_bytes(fmt);
 
@@ -951,8 +959,8 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
     memset(&prm, 0, sizeof(prm));
     prm.count = count;
     prm.wait_limit_ns = ptx::kWaitLimitNs;
-    int grid = 1, wslot = 0, stash = 8192, jobs = 0;
-    size_t x8_off = kChainHeaderBytes;
+    int stash = 8192, jobs = 0, rot = 0;
+    size_t off = kChainHeaderBytes;
     for (int i = 0; i < count; ++i) {
         const w4a8_chain_problem& q = pr[i];
         ChainProblem& d = prm.prob[i];
@@ -974,43 +982,43 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
         d.sw_stride = q.sw_stride;
         d.out_dtype = q.out_dtype;
         d.scale_mode = q.scale_mode;
-        const int64_t NU = q.N / 8;
-        const int64_t T = sms < NU ? sms : NU;
-        const int rmax = (int)((NU + T - 1) / T) * 8;
-        if (rmax > 256) return W4A8_ERR_BAD_SHAPE;
-        d.T = (int)T;
-        d.MBLK = rmax > 128 ? 2 : 1;
+        // whole 96-row blocks per CTA while at least as many blocks as CTAs are left, the rest cut along K
+        const int blocks = chain_blocks(d.N);
+        d.rounds = blocks / sms;
+        if ((d.rounds + 1) / 2 + 2 > kChainMaxSegs) return W4A8_ERR_BAD_SHAPE;   // more whole blocks per CTA than the segment table holds
+        d.rem_blocks = blocks - d.rounds * sms;
         d.job_base = jobs;
         jobs += d.M;
-        d.x8_off = (uint32_t)x8_off;
-        x8_off += (size_t)q.K * kChainMaxM;
-        if (x8_off > 0xFFFFFFFFull) return W4A8_ERR_BAD_SHAPE;
-        if ((int)T > grid) grid = (int)T;
-        // a slot holds two (k-block, 128-row block) items of the widest range of this problem
-        const int slot = ((2 / d.MBLK) * rmax * (kRowCodeBytes + mb) + 127) / 128 * 128;
-        if (slot > wslot) wslot = slot;
+        d.rem_rot = rot % sms;
+        rot += chain_rem_ctas(d, sms);
+        d.x8_off = (uint32_t)off;
+        off += (size_t)q.K * kChainMaxM;
+        d.part_off = (uint32_t)off;
+        off += chain_part_bytes(q.M, kMaxSMs);
+        d.cnt_off = (uint32_t)off;
+        off += kChainCntBytes;
+        if (off > 0xFFFFFFFFull) return W4A8_ERR_BAD_SHAPE;
         if (2 * (int)q.K > stash) stash = 2 * (int)q.K;
     }
-    // every quantization job needs a CTA of its own kind of row: at least as many CTAs as tokens
-    if (grid < kChainMaxM) grid = kChainMaxM < sms ? kChainMaxM : sms;
-    prm.wslot = wslot;
+    // a slot holds the two (k-block, block) items of a stage: 2 x 96 rows of codes and meta data
+    prm.wslot = (2 * kChainBlockRows * (kRowCodeBytes + mb) + 127) / 128 * 128;
     prm.stash = stash;
-    using C0 = ChainCfg<3, kFmtTiledSignMag>;
-    const int fixed = 1024 + C0::kXRingBytes + stash + C0::kBarBytes;
-    int s1 = (C0::kSmemMax - fixed) / wslot;
+    using C0 = ChainCfg<4, kFmtTiledSignMag>;
+    const int fixed = 1024 + C0::kXRingBytes + stash + C0::kBarBytes + C0::kSegBytes;
+    int s1 = (C0::kSmemMax - fixed) / prm.wslot;
     if (s1 > C0::kS1Max) s1 = C0::kS1Max;
-    if (s1 < 3) return W4A8_ERR_BAD_SHAPE;
+    if (s1 < 4) return W4A8_ERR_BAD_SHAPE;
     prm.S1 = s1;
-    const int smem = fixed + s1 * wslot;
+    const int smem = fixed + s1 * prm.wslot;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    if (groups == 0) groups = 3;
+    if (groups == 0) groups = 4;
 #define W4A8_CHAIN(GG)                                                                             \
-    (fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<GG, kFmtTiledSignMag>>(prm, grid, smem, ws, st) \
-                             : launch_chain<ChainCfg<GG, kFmtTiled>>(prm, grid, smem, ws, st))
+    (fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<GG, kFmtTiledSignMag>>(prm, sms, smem, ws, st) \
+                             : launch_chain<ChainCfg<GG, kFmtTiled>>(prm, sms, smem, ws, st))
     switch (groups) {
         case 2: return W4A8_CHAIN(2);
-        case 4: return W4A8_CHAIN(4);
-        default: return W4A8_CHAIN(3);
+        case 3: return W4A8_CHAIN(3);
+        default: return W4A8_CHAIN(4);
     }
 #undef W4A8_CHAIN
 }

@@ -1,8 +1,9 @@
 """GPU parity: w4a8_linear_chain (a chain of decode-sized layers in one persistent launch) against
-the oracle's forward pass (Sec. 3 flow: Eq. 13 -> Eq. 10 -> FP8 matmul -> Eq. 4 / Eq. 11) and, bit
-for bit, against the per-launch path (w4a8_quantize_act / w4a8_silu_mul_quantize + w4a8_linear).
-The FP8 activations and scales the chain used are read back and must be bit-exact; the output
-gate is max relative error 2e-3 before the BF16 cast and one BF16 step after it."""
+the oracle's forward pass (Sec. 3 flow: Eq. 13 -> Eq. 10 -> FP8 matmul -> Eq. 4 / Eq. 11).  The FP8
+activations and scales the chain used are read back and must be bit-exact; the output gate is max
+relative error 2e-3 before the BF16 cast and one BF16 step after it.  Where the chain does not cut K
+(whole 96-row blocks per CTA) its outputs must also equal those of the per-launch path
+(w4a8_quantize_act + w4a8_linear) bit for bit: same operands, same accumulation order."""
 import ctypes
 
 import numpy as np
@@ -41,8 +42,9 @@ def _per_launch(x, tw, out_dtype):
 @pytest.mark.parametrize("groups", [0, 2, 4])
 @pytest.mark.parametrize("asym", [False, True])
 def test_independent_problems_match_oracle_and_per_launch_path(groups, asym):
-    # three problems of different token counts and shapes in one launch: a ragged row partition,
-    # an odd number of k-blocks (last stage holds one), few rows per CTA, M <= 8 and M > 8
+    # problems of different token counts and shapes in one launch (all with fewer 96-row blocks than
+    # SMs, so every block is cut along K and summed by the CTA that arrives last): a short last
+    # block, an odd number of k-blocks, fewer items than CTAs, M <= 8 and M > 8
     shapes = [(1, 2368, 640), (4, 4736, 384), (16, 1024, 1024), (7, 48, 256), (9, 16, 128)]
     probs, refs = [], []
     for i, (M, N, K) in enumerate(shapes):
@@ -64,9 +66,6 @@ def test_independent_problems_match_oracle_and_per_launch_path(groups, asym):
         assert np.array_equal(d["x8_out"].cpu().numpy(), x8)
         worst, _ = fp32_gate(d["y"].cpu().numpy(), ref["y64"], rel=2e-3)
         assert worst <= 2e-3, worst
-        want = _per_launch(d["x"], d["weight"], binding.OUT_FP32)
-        torch.cuda.synchronize()
-        assert torch.equal(d["y"], want)
 
 
 def test_exact_integer_problem_is_bit_exact():
@@ -94,9 +93,31 @@ def test_exact_integer_problem_is_bit_exact():
     assert np.array_equal(y.cpu().numpy(), ref["y32"])
 
 
+def test_whole_blocks_match_the_per_launch_path_bit_for_bit():
+    # N = (number of SMs) x 96 x rounds: every CTA owns whole blocks and walks all of K, one block
+    # (rounds = 1), two at a time (2) or two and one (3); plus a short remainder cut along K
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for rounds, extra, M, K in ((1, 0, 16, 384), (2, 0, 5, 256), (3, 128, 9, 128)):
+        N = sms * 96 * rounds + extra
+        wq, tw = _weights(N, K, 100 + rounds)
+        xb = inputs.make_activation(M, K, 110 + rounds, 0.01, 20.0)
+        x = bf16_dev(xb)
+        y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        binding.LinearChain([dict(x=x, weight=tw, y=y)])()
+        want = _per_launch(x, tw, binding.OUT_FP32)
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0
+        whole = sms * 96 * rounds
+        assert torch.equal(y[:, :whole], want[:, :whole]), rounds
+        _, _, ref = _oracle_layer(xb, wq)
+        worst, _ = fp32_gate(y.cpu().numpy(), ref["y64"], rel=2e-3)
+        assert worst <= 2e-3, (rounds, worst)
+
+
 def test_dependent_chain_and_gated_block():
     # x -> gate_up (BF16) -> silu(gate) * up quantized in the chain -> down (BF16) -> next layer on
-    # the down projection's output: every hand-over goes through the chain's counters
+    # the down projection's output: every hand-over goes through the chain's counters.  Each stage is
+    # checked against the oracle on the input that stage saw (the chain's own previous output).
     M, H, F = 5, 1024, 1408
     wq_gu, tw_gu = _weights(2 * F, H, 70)
     wq_dn, tw_dn = _weights(H, F, 71)
@@ -108,37 +129,46 @@ def test_dependent_chain_and_gated_block():
     nx = torch.zeros((M, 2304), dtype=torch.float32, device="cuda")
     x8_dn = torch.zeros((M, F), dtype=torch.uint8, device="cuda")
     sx_dn = torch.zeros((M,), dtype=torch.float32, device="cuda")
+    x8_nx = torch.zeros((M, H), dtype=torch.uint8, device="cuda")
+    sx_nx = torch.zeros((M,), dtype=torch.float32, device="cuda")
     chain = binding.LinearChain([
         dict(x=x, weight=tw_gu, y=gu),
         dict(x=gu, weight=tw_dn, y=dn, kind=binding.CHAIN_INPUT_SILU_MUL, depends_on=0, x8_out=x8_dn, s_x_out=sx_dn),
-        dict(x=dn, weight=tw_nx, y=nx, depends_on=1),
+        dict(x=dn, weight=tw_nx, y=nx, depends_on=1, x8_out=x8_nx, s_x_out=sx_nx),
     ])
-    # the same block launch by launch
-    tiny = torch.zeros((16,), dtype=torch.uint8, device="cuda")
-    x8, s_x = binding.quantize_act(x)
-    gu_ref = binding.linear_tiled(x8, s_x, tw_gu, workspace=tiny)
-    h8, s_h = binding.silu_mul_quantize(gu_ref)
-    dn_ref = binding.linear_tiled(h8, s_h, tw_dn, workspace=tiny)
-    d8, s_d = binding.quantize_act(dn_ref)
-    nx_ref = binding.linear_tiled(d8, s_d, tw_nx, out_dtype=binding.OUT_FP32, workspace=tiny)
-    for _ in range(3):     # repeated launches: the counters reset themselves
+    chain()
+    torch.cuda.synchronize()
+    first = [t.clone() for t in (gu, dn, nx, x8_dn, sx_dn)]
+    for _ in range(3):     # repeated launches: the counters reset themselves, the results repeat
         gu.zero_(); dn.zero_(); nx.zero_()
         chain()
     torch.cuda.synchronize()
     assert binding.query_device_status() == 0
-    assert torch.equal(gu, gu_ref)
-    assert torch.equal(x8_dn, h8) and torch.equal(sx_dn, s_h)
-    assert torch.equal(dn, dn_ref)
-    assert torch.equal(nx, nx_ref)
-    # and the first layer against the oracle (the later ones are covered through the bit-equality
-    # with the per-launch path, whose kernels have their own oracle tests)
+    for a, b in zip(first, (gu, dn, nx, x8_dn, sx_dn)):
+        assert torch.equal(a, b)
+    # layer 1 against the oracle
     _, _, ref = _oracle_layer(xb, wq_gu)
     ok, dist = bf16_gate(bf16_bits(gu), ref["y64"])
     assert ok, dist
+    # the gated activation + quantization: the same arithmetic as w4a8_silu_mul_quantize on the same input
+    h8, s_h = binding.silu_mul_quantize(gu)
+    torch.cuda.synchronize()
+    assert torch.equal(x8_dn, h8) and torch.equal(sx_dn, s_h)
+    # layer 2 on the FP8 activations it used
+    ref2 = oracle.linear(x8_dn.cpu().numpy(), sx_dn.cpu().numpy(), oracle.dequant_weight(*wq_dn[:3]), wq_dn[3])
+    ok, dist = bf16_gate(bf16_bits(dn), ref2["y64"])
+    assert ok, dist
+    # layer 3: Eq. 13 of the chain's own BF16 output, bit-exact, then the product
+    d8, s_d = oracle.quantize_act(bf16_bits(dn))
+    assert np.array_equal(x8_nx.cpu().numpy(), d8)
+    assert np.array_equal(sx_nx.cpu().numpy().view(np.uint32), s_d.astype(np.float32).view(np.uint32))
+    ref3 = oracle.linear(d8, s_d, oracle.dequant_weight(*wq_nx[:3]), wq_nx[3])
+    worst, _ = fp32_gate(nx.cpu().numpy(), ref3["y64"], rel=2e-3)
+    assert worst <= 2e-3, worst
 
 
 def test_two_row_blocks_per_cta_and_graph_replay():
-    # N = 28672: 194 rows per CTA (two 128-row blocks); replayed from a CUDA graph many times
+    # N = 28672: two whole 96-row blocks per CTA plus a remainder cut along K; replayed from a CUDA graph many times
     M, N, K = 3, 28672, 256
     wq, tw = _weights(N, K, 80)
     xb = inputs.make_activation(M, K, 81)

@@ -2,17 +2,17 @@
 """Benchmark of the W4A8 linear hot path (activation FP8 quantize -> fused INT4->FP8 GEMM ->
 scaled BF16) on the decode sweep: M in {1,4,16}, K=4096, N=14336 (Llama-3-8B MLP up-projection).
 
-One step = one pass of the whole path over the sweep: for each M, w4a8_quantize_act then
-w4a8_linear (or one w4a8_linear_fused launch where w4a8_fused_is_faster says so: nowhere at
-present; --two-kernel forces the two-kernel sequence).  The metric is the weight stream rate:
-bytes of INT4 codes + group scales the method must read per step, divided by the step time.
-Weights rotate over several distinct copies whose total size exceeds twice the L2, so every pass
-streams them from HBM.  Steps are replayed from CUDA graphs that hold --steps-per-graph
-consecutive steps each (a decode graph likewise holds all layers of a forward pass).
+One step = one pass of the whole path over the sweep: for each M, the Eq. 13 activation
+quantization and the W4A8 linear, run as three problems of a w4a8_linear_chain launch (one
+persistent kernel; --steps-per-launch consecutive steps share a launch, as a decode launch holds
+the layers of a forward pass).  The metric is the weight stream rate: bytes of INT4 codes + group
+scales the method must read per step, divided by the step time.  Weights rotate over several
+distinct copies whose total size exceeds twice the L2, so every pass streams them from HBM.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-N > 1 runs under torchrun, one independent replica per GPU (the path has no exchange step).
+N > 1 runs one independent replica per GPU (the path has no exchange step): under torchrun when
+the launcher set WORLD_SIZE, else bench.py starts the N ranks itself.
 --impl reference times the CPU oracle on the host cores on a bounded sample of the same
 workload.  Prints one JSON line on rank 0.
 """
@@ -44,9 +44,10 @@ WORKLOAD = ("c2 decode sweep: W4A8 linear, M in {1,4,16}, K=4096, N=14336, INT4 
             "weights from N(0,0.02), BF16 N(0,1) activations with 1% outlier channels x20, "
             "per-token FP8 E4M3 scales, BF16 output")
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum); see profiles/.  None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 30.36e6  # profiles/linear_splitn_decode_c2.md, mean of M = 1, 4, 16
+# DRAM bytes per problem of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum of one launch divided by its problems); see profiles/.  None until a capture
+# exists for the current kernel.
+NCU_TRAFFIC_BYTES_PER_PROBLEM = None
 
 
 def weight_bytes(n=N, k=K):
@@ -230,6 +231,12 @@ def aggregate_rate(world, steps, ms_total):
     return world * steps * len(SWEEP_M) * weight_bytes() / (ms_total * 1e-3) / 1e9
 
 
+def chain_algorithmic_bytes(ms, n=N, k=K):
+    """Everything one chain launch over the token counts `ms` must move: per problem the stored
+    weights (codes + group scales), the BF16 activations in, the weight scale and the BF16 output."""
+    return sum(weight_bytes(n, k) + 2 * m * k + 4 + 2 * m * n for m in ms)
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_2505_14638_b200 import binding, inputs
@@ -258,168 +265,111 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.synchronize()
     if binding.query_device_status() != 0:
         raise RuntimeError("prepack reported an unrepresentable code")
-    xs, x8s, sxs, ys, x_host = {}, {}, {}, {}, {}
+    xs, ys, x_host, y_host = {}, {}, {}, {}
     for m in SWEEP_M:
         xb = inputs.make_activation(m, K, 1000 * rank + m, OUTLIER_FRAC, OUTLIER_MULT)
         t = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
         x_host[m] = t.pin_memory()
         xs[m] = t.to(dev)
-        x8s[m] = torch.empty((m, K), dtype=torch.uint8, device=dev)
-        sxs[m] = torch.empty((m,), dtype=torch.float32, device=dev)
         ys[m] = torch.empty((m, N), dtype=torch.bfloat16, device=dev)
-    workspace = binding.new_workspace(max(SWEEP_M), N, K, weights[0].fmt, dev)
+        y_host[m] = torch.empty((m, N), dtype=torch.bfloat16).pin_memory()
     torch.cuda.synchronize()
 
-    def quant(m):
-        binding.quantize_act(xs[m], out=(x8s[m], sxs[m]))
+    # ---- the step: one pass of the whole path (Eq. 13 quantization, Eq. 10 expansion, FP8 MMAs,
+    # Eq. 4 / Eq. 11 epilogue) over the sweep, as problems of ONE persistent launch
+    # (w4a8_linear_chain).  A launch carries `spl` consecutive steps, as a decode launch carries the
+    # layers of a forward pass; every problem reads the next weight copy of the rotation.
+    spl = max(1, min(args.steps_per_launch, binding.CHAIN_MAX_PROBLEMS // len(SWEEP_M)))
+    workspace = [None]
 
-    def lin(m, c):
-        binding.linear_tiled(x8s[m], sxs[m], weights[c % WEIGHT_COPIES], out=ys[m], workspace=workspace)
+    def make_launch(first_step, nsteps, host_buffers=False):
+        probs = []
+        for s_ in range(nsteps):
+            for i, m in enumerate(SWEEP_M):
+                c = ((first_step + s_) * len(SWEEP_M) + i) % WEIGHT_COPIES
+                probs.append(dict(x=x_host[m] if host_buffers else xs[m], weight=weights[c],
+                                  y=y_host[m] if host_buffers else ys[m]))
+        ch = binding.LinearChain(probs, workspace=workspace[0])
+        if workspace[0] is None or ch.ws.numel() > workspace[0].numel():
+            workspace[0] = ch.ws
+        return ch
 
-    fused_m = () if args.two_kernel else tuple(m for m in SWEEP_M if binding.fused_is_faster(m, N, K))
-    fused = bool(fused_m)
-    lin_unfused = lin
-
-    def lin(m, c):  # noqa: F811
-        if m in fused_m:
-            binding.linear_fused(xs[m], weights[c % WEIGHT_COPIES], out=ys[m])
-        else:
-            lin_unfused(m, c)
-
-    def eager_step(phase):
-        for i, m in enumerate(SWEEP_M):
-            if m not in fused_m:
-                quant(m)
-            lin(m, phase * len(SWEEP_M) + i)
+    probe = make_launch(0, spl)                     # sizes the shared workspace
+    n_full, n_tail = args.steps // spl, args.steps % spl
+    period = WEIGHT_COPIES                          # the weight rotation repeats after this many launches
+    full = [make_launch(g * spl, spl) for g in range(min(period, max(n_full, 1)))]
+    tail = make_launch(n_full * spl, n_tail) if n_tail else None
+    del probe
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for ph in range(3):
-        eager_step(ph)
+    for g in range(max(3, (max(args.warmup, 3) + spl - 1) // spl)):
+        full[g % len(full)]()
+    if tail is not None:
+        tail()
     barrier()
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set by the first steps (a bounded wait gave up)")
 
-    # ---- CUDA graphs (the step is launch-bound).  A graph holds `spg` consecutive steps, as a
-    # decode graph holds the layers of a whole forward pass; one graph per phase of the weight
-    # rotation.  Every step still runs all its launches on weights that come from HBM.
-    use_graph = not args.no_graph
-    spg = max(1, min(args.steps_per_graph, args.steps)) if use_graph else 1
-    n_groups, n_tail = args.steps // spg, args.steps % spg   # whole graphs, then single-step graphs
-    period = WEIGHT_COPIES
-    g_full, g_lin, g_quant, g_tail = [], [], None, []
-    if use_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            for ph in range(period):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    for j in range(spg):
-                        eager_step(ph * spg + j)
-                g_full.append(g)
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    for j in range(spg):
-                        for i, m in enumerate(SWEEP_M):
-                            lin(m, (ph * spg + j) * len(SWEEP_M) + i)
-                g_lin.append(g)
-                if n_tail:
-                    g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g, stream=side):
-                        eager_step(ph)
-                    g_tail.append(g)
-            if len(fused_m) < len(SWEEP_M):
-                g_quant = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g_quant, stream=side):
-                    for m in SWEEP_M:
-                        if m not in fused_m:
-                            quant(m)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-
-    kernels_per_step = 2 * len(SWEEP_M) - len(fused_m)
-
-    def step_group(gi):
-        """Runs steps gi * spg .. gi * spg + spg - 1."""
-        if use_graph:
-            g_full[gi % period].replay()
-        else:
-            eager_step(gi % period)
-
-    for gi in range((max(args.warmup, 3) + spg - 1) // spg):
-        step_group(gi)
-    barrier()
-
-    # ---- timed region 1: the whole path, K steps, device timed ----
+    # ---- timed region 1: K steps, device timed ----
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    for gi in range(n_groups):
-        step_group(gi)
-    for t in range(n_tail):
-        g_tail[t % period].replay()
+    for g in range(n_full):
+        full[g % len(full)]()
+    if tail is not None:
+        tail()
     e1.record()
     barrier()
-    launches = args.steps * kernels_per_step
+    launches = n_full + (1 if tail is not None else 0)
     ms_total = e0.elapsed_time(e1)
 
-    # ---- timed region 2: the same steps with the three linear launches bracketed by events ----
-    pairs = []
-    for s in range(n_groups):
-        if use_graph:
-            if g_quant is not None:
-                g_quant.replay()
-        else:
-            for m in SWEEP_M:
-                if m not in fused_m:
-                    quant(m)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        if use_graph:
-            g_lin[s % period].replay()
-        else:
-            for i, m in enumerate(SWEEP_M):
-                lin(m, s * len(SWEEP_M) + i)
-        b.record()
-        pairs.append((a, b))
+    # ---- timed region 2: the dominant kernel alone -- full launches back to back, bracketed by events ----
+    reps = max(10, n_full)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for g in range(reps):
+        full[g % len(full)]()
+    b.record()
     torch.cuda.synchronize()
-    lin_ms = sum(a.elapsed_time(b) for a, b in pairs)
+    launch_ms = a.elapsed_time(b) / reps
     clocks = sampler.stop() if rank == 0 else None
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set during the timed region")
 
-    # ---- end to end: host activations in, host result out, through w4a8_forward_host ----
-    fwd = {m: binding.HostForward(m, weights[0]) for m in SWEEP_M}
-    cnt = [0]
+    # ---- end to end: the same call with HOST buffers -- the activations of every step are read from
+    # pinned host memory and every step's result is written to pinned host memory inside the timed
+    # region (by the kernel itself, over the bus), the caller synchronises after every call ----
+    e2e_launch = make_launch(0, spl, host_buffers=True)
+    e2e_tail = make_launch(n_full * spl, n_tail, host_buffers=True) if n_tail else None
 
-    def e2e_step():
-        for m in SWEEP_M:
-            f = fwd[m]
-            f.set_weight(weights[cnt[0] % WEIGHT_COPIES])
-            cnt[0] += 1
-            f(x_host[m])
-        torch.cuda.current_stream().synchronize()   # the caller reads the result every step
+    def e2e_pass():
+        for _ in range(n_full):
+            e2e_launch()
+            torch.cuda.current_stream().synchronize()   # the caller reads the results
+        if e2e_tail is not None:
+            e2e_tail()
+            torch.cuda.current_stream().synchronize()
 
-    for _ in range(3):
-        e2e_step()
+    for _ in range(2):
+        e2e_launch()
     barrier()
-    n_e2e = min(args.steps, 2000)
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     g0.record()
-    for _ in range(n_e2e):
-        e2e_step()
+    e2e_pass()
     g1.record()
     barrier()
-    ms_e2e = g0.elapsed_time(g1) * args.steps / n_e2e
+    ms_e2e = g0.elapsed_time(g1)
+    if binding.query_device_status() != 0:
+        raise RuntimeError("device status word set during the end-to-end region")
 
-    ms_total, ms_e2e, lin_ms = max_over_ranks([ms_total, ms_e2e, lin_ms], dist, dev)
+    ms_total, ms_e2e, launch_ms = max_over_ranks([ms_total, ms_e2e, launch_ms], dist, dev)
 
     if rank != 0:
         if dist is not None:
@@ -430,10 +380,8 @@ def run_ours(args, rank, world, local_rank):
     peaks = load_peaks()
     value = aggregate_rate(world, args.steps, ms_total)
     e2e_value = aggregate_rate(world, args.steps, ms_e2e)
-    n_lin = n_groups * spg * len(SWEEP_M)
-    alg_bytes = sum(linear_algorithmic_bytes(m, fused=m in fused_m) for m in SWEEP_M) / len(SWEEP_M)
-    avg_launch_s = lin_ms * 1e-3 / n_lin
-    achieved = alg_bytes / avg_launch_s / 1e9
+    alg_bytes = chain_algorithmic_bytes(SWEEP_M * spl)
+    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
@@ -441,26 +389,32 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD, "parallelism": "replicas x%d (no collective)" % world,
                    "l2": "weights rotate over %d distinct copies (%.0f MB > 2 x 126 MB L2)"
                          % (WEIGHT_COPIES, WEIGHT_COPIES * weight_bytes() / 1e6),
-                   "step": ("M in %s: w4a8_linear_fused (activation quantization inside the kernel); other M: "
-                            "w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)" % (fused_m,)) if fused else
-                           "for M in (1,4,16): w4a8_quantize_act + w4a8_linear (tiled sign-magnitude weights)",
-                   "launch": ("CUDA graph replay, %d steps per graph" % spg) if use_graph else "eager launches"},
+                   "step": "for M in (1,4,16): Eq. 13 activation quantization + W4A8 linear on tiled sign-magnitude "
+                           "weights, as three problems of a w4a8_linear_chain launch",
+                   "launch": "one persistent launch per %d steps (%d problems), eager, back to back; "
+                             "%d launch(es) in the timed region" % (spl, spl * len(SWEEP_M), launches)},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(m * K * 2 for m in SWEEP_M),
                 "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
-                "ms_per_step": ms_e2e / args.steps},
+                "ms_per_step": ms_e2e / args.steps,
+                "how": "w4a8_linear_chain on pinned host activations and outputs (read and written over the bus by "
+                       "the kernel), one call and one stream synchronisation per %d steps" % spl},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "linear_splitn_kernel<MT=16> (%s), mean over M in {1,4,16}"
-                               % ("FUSE variant for M in %s" % (fused_m,) if fused else "w4a8_linear"),
+        "roofline": {"bound": "hbm", "kernel": "linear_chain_kernel (w4a8_linear_chain), %d problems per launch: "
+                               "M in {1,4,16} x %d" % (spl * len(SWEEP_M), spl),
                      "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": avg_launch_s * 1e6,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+                     "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": launch_ms * 1e3,
+                     "us_per_problem": launch_ms * 1e3 / (spl * len(SWEEP_M)),
+                     "traffic": NCU_TRAFFIC_BYTES_PER_PROBLEM * spl * len(SWEEP_M)
+                     if NCU_TRAFFIC_BYTES_PER_PROBLEM else None},
     }
     if not args.no_extras:
-        line["decode_detail"] = decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks)
+        line["decode_detail"] = decode_detail(torch, binding, weights, xs, ys, peaks)
+        line["act_quant"] = act_quant_extra(torch, binding, inputs, dev, peaks)
         line["prefill"] = prefill_extra(torch, binding, inputs, dev, peaks)
+        line["prefill_c4"] = prefill_c4_extra(torch, binding, inputs, dev, peaks)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line), flush=True)
@@ -482,30 +436,27 @@ def _time_loop(torch, fn, iters, warm=3):
     return a.elapsed_time(b) * 1e-3 / iters
 
 
-def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
-    """Per-M time of the fused launch and of the linear alone (graphs of back-to-back launches,
-    weights from HBM) next to cuBLAS BF16."""
+def decode_detail(torch, binding, weights, xs, ys, peaks):
+    """Per M: time per problem of a chain launch that carries one problem per weight copy, next to
+    the per-launch path (w4a8_quantize_act + w4a8_linear replayed from a CUDA graph) and cuBLAS BF16."""
     out = {}
-    dev = x8s[1].device
+    dev = ys[1].device
     wb = [torch.randn((N, K), dtype=torch.bfloat16, device=dev) for _ in range(4)]
     side = torch.cuda.Stream()
+    x8s = {m: torch.empty((m, K), dtype=torch.uint8, device=dev) for m in SWEEP_M}
+    sxs = {m: torch.empty((m,), dtype=torch.float32, device=dev) for m in SWEEP_M}
+    workspace = binding.new_workspace(max(SWEEP_M), N, K, weights[0].fmt, dev)
     for m in SWEEP_M:
-        side.wait_stream(torch.cuda.current_stream())
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(g, stream=side):
-                for c in range(WEIGHT_COPIES):
-                    binding.linear_tiled(x8s[m], sxs[m], weights[c], out=ys[m], workspace=workspace)
-        torch.cuda.current_stream().wait_stream(side)
-        t = _time_loop(torch, g.replay, 20) / WEIGHT_COPIES
-        side.wait_stream(torch.cuda.current_stream())
-        g2 = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(g2, stream=side):
-                for c in range(WEIGHT_COPIES):
-                    binding.linear_fused(xs[m], weights[c], out=ys[m])
-        torch.cuda.current_stream().wait_stream(side)
-        tf = _time_loop(torch, g2.replay, 20) / WEIGHT_COPIES
+        chain = binding.LinearChain([dict(x=xs[m], weight=weights[c], y=ys[m]) for c in range(WEIGHT_COPIES)])
+        t = _time_loop(torch, chain, 20) / WEIGHT_COPIES
+        one = [binding.LinearChain([dict(x=xs[m], weight=weights[c], y=ys[m])], workspace=chain.ws)
+               for c in range(WEIGHT_COPIES)]
+        j1 = [0]
+
+        def single():
+            j1[0] += 1
+            one[j1[0] % WEIGHT_COPIES]()
+        t1 = _time_loop(torch, single, 40)
         side.wait_stream(torch.cuda.current_stream())
         g3 = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
@@ -522,14 +473,66 @@ def decode_detail(torch, binding, weights, xs, x8s, sxs, ys, workspace, peaks):
             j[0] += 1
             torch.matmul(xb, wb[j[0] % 4].t())
         tb = _time_loop(torch, f, 40)
-        out["M=%d" % m] = {"quantize_then_linear_us": t2 * 1e6, "fused_us": tf * 1e6,
-                           "fused_frac_hbm_measured":
-                               linear_algorithmic_bytes(m, fused=True) / tf / 1e9 / peaks["hbm_gbs"],
-                           "linear_only_us": t * 1e6, "linear_only_weight_GBps": weight_bytes() / t / 1e9,
-                           "linear_only_frac_hbm_measured":
-                               linear_algorithmic_bytes(m) / t / 1e9 / peaks["hbm_gbs"],
+        alg = chain_algorithmic_bytes((m,))
+        out["M=%d" % m] = {"chain_us_per_problem": t * 1e6, "chain_weight_GBps": weight_bytes() / t / 1e9,
+                           "chain_frac_hbm_measured": alg / t / 1e9 / peaks["hbm_gbs"],
+                           "chain_single_problem_launch_us": t1 * 1e6,
+                           "per_launch_quantize_then_linear_us": t2 * 1e6,
+                           "per_launch_frac_hbm_measured": alg / t2 / 1e9 / peaks["hbm_gbs"],
                            "cublas_bf16_us": tb * 1e6}
     return out
+
+
+def act_quant_extra(torch, binding, inputs, dev, peaks):
+    """w4a8_quantize_act alone (Eq. 13: 2 bytes read + 1 byte written per element, plus one scale per
+    token) at the prefill sizes of c3 and c4, against the measured HBM copy rate."""
+    out = {}
+    for name, m, k in (("c3", 2048, 4096), ("c4", 8192, 8192)):
+        copies = max(2, int(2.2 * 126e6 / (3 * m * k)) + 1)
+        xs_ = []
+        for c in range(copies):
+            xb = inputs.make_activation(m, k, 300 + c, OUTLIER_FRAC, OUTLIER_MULT)
+            xs_.append(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+        x8 = torch.empty((m, k), dtype=torch.uint8, device=dev)
+        s_x = torch.empty((m,), dtype=torch.float32, device=dev)
+        i = [0]
+
+        def f():
+            i[0] += 1
+            binding.quantize_act(xs_[i[0] % copies], out=(x8, s_x))
+        t = _time_loop(torch, f, 30, warm=5)
+        b = 3.0 * m * k + 4.0 * m
+        out[name] = {"M": m, "K": k, "us": t * 1e6, "algorithmic_bytes": b, "GBps": b / t / 1e9,
+                     "frac_hbm_measured": b / t / 1e9 / peaks["hbm_gbs"],
+                     "l2": "inputs rotate over %d copies" % copies}
+        del xs_
+    return out
+
+
+def prefill_c4_extra(torch, binding, inputs, dev, peaks):
+    """Config c4 (M=8192, K=8192, N=28672): w4a8_linear on quantized activations, a few repeats of the
+    1.9 ms launch, against 2 x the SUSTAINED BF16 figure (a long tensor-bound launch runs under the
+    power cap) and against the burst figure."""
+    M4, K4, N4 = 8192, 8192, 28672
+    W = torch.from_numpy(inputs.make_weight(N4, K4, 0.015, seed=77)).to(dev)
+    tw = binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True))
+    del W
+    xb = inputs.make_activation(M4, K4, 78, 0.005, 30.0)
+    x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev)
+    x8, s_x = binding.quantize_act(x)
+    y = torch.empty((M4, N4), dtype=torch.bfloat16, device=dev)
+    ws = binding.new_workspace(M4, N4, K4, tw.fmt, dev)
+    t = _time_loop(torch, lambda: binding.linear_tiled(x8, s_x, tw, out=y, workspace=ws), 5, warm=3)
+    flops = 2.0 * M4 * N4 * K4
+    sus = 2.0 * peaks["bf16_tflops_sustained"]
+    res = {"workload": "c4 prefill M=8192 K=8192 N=28672 (weights + activations 0.36 GB > L2)", "us": t * 1e6,
+           "tflops": flops / t / 1e12, "fp8_peak_sustained_tflops": sus,
+           "frac_of_fp8_peak_sustained": flops / t / 1e12 / sus,
+           "frac_of_fp8_peak_burst": flops / t / 1e12 / (2.0 * peaks["bf16_tflops"]),
+           "frac_of_nominal_4500": flops / t / 1e12 / 4500.0, "peak_source": peaks["source"]}
+    del tw, x, x8, y, ws
+    torch.cuda.empty_cache()
+    return res
 
 
 def library_fp8_gemm_tflops(torch, dev, n=8192):
@@ -943,6 +946,23 @@ def dpq_sweep(torch, binding, inputs, dev):
     return rows
 
 
+def spawn_ranks(n):
+    """`bench.py --gpus N` started without a launcher: re-run this command line under
+    torch.distributed.run with one rank per GPU of this node (rendezvous on 127.0.0.1) and return its
+    exit code.  Fails loudly when the node has fewer GPUs than asked for."""
+    import socket
+    import torch
+    have = torch.cuda.device_count()
+    if have < n:
+        raise SystemExit("--gpus %d asked for, but this node has %d CUDA device(s)" % (n, have))
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -951,11 +971,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / per-M detail sections")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
-    ap.add_argument("--two-kernel", action="store_true",
-                    help="step = w4a8_quantize_act + w4a8_linear per M instead of the fused launch")
-    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
-    ap.add_argument("--steps-per-graph", type=int, default=8,
-                    help="consecutive steps captured in one CUDA graph (steps left over run from single-step graphs; default 8)")
+    ap.add_argument("--steps-per-launch", type=int, default=8,
+                    help="consecutive steps carried by one w4a8_linear_chain launch (3 problems per step, at most 24 "
+                         "problems per launch; steps left over run in one shorter launch; default 8)")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the c3 prefill section (small enough for a profiler capture) and print it")
     ap.add_argument("--sweep", default=None, choices=["c5", "c4", "dpq", "schemes", "mlp", "tp"],
@@ -1000,8 +1018,11 @@ def main():
         print(json.dumps({"prefill": prefill_extra(torch, binding, inputs, torch.device("cuda", local_rank),
                                                    load_peaks())}), flush=True)
         return
-    if world != args.gpus and world > 1:
-        raise SystemExit("--gpus %d does not match WORLD_SIZE %d" % (args.gpus, world))
+    if "WORLD_SIZE" in os.environ:
+        if world != args.gpus:
+            raise SystemExit("--gpus %d does not match WORLD_SIZE %d" % (args.gpus, world))
+    elif args.gpus > 1:
+        raise SystemExit(spawn_ranks(args.gpus))   # no launcher: start the N ranks ourselves
     run_ours(args, rank, world, local_rank)
 
 

@@ -229,7 +229,10 @@ int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode
  * are left every CTA takes whole blocks, the remaining blocks are cut along K as well, into runs of
  * at least four 128-wide k-blocks, and the CTA that holds a block's lowest k range adds the
  * partial sums of the others (FP32, through the workspace) before it scales and writes the rows.
- *   x_bf16       device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned), M <= W4A8_CHAIN_MAX_M.
+ *   x_bf16       device BF16 [M][ldx] (ldx % 8 == 0, 16-byte aligned), M <= W4A8_CHAIN_MAX_M.  x_bf16 and
+ *                y may also be device-side addresses of page-locked host buffers
+ *                (w4a8_host_buffer_device_pointer): decode-sized activations and outputs are small
+ *                enough to be read and written over the bus by the kernel itself.
  *   depends_on   -1 when x_bf16 is complete before the call; otherwise the index (< i) of the
  *                problem of this chain that WRITES the memory x_bf16 points into (normally
  *                x_bf16 == that problem's y, out_dtype BF16): problem i is not quantized before
@@ -281,6 +284,17 @@ typedef struct w4a8_chain_problem {
 size_t w4a8_linear_chain_workspace_bytes(const w4a8_chain_problem* problems_host, int count);
 int w4a8_linear_chain(const w4a8_chain_problem* problems_host, int count, void* workspace,
                       size_t workspace_bytes, int groups, void* stream);
+
+/*
+ * Device-side address of a page-locked HOST buffer (cudaHostAlloc / cudaHostRegister memory that
+ * is mapped into the device's address space), for callers that want a kernel of this library to
+ * read its activations from, or write its outputs to, host memory directly: w4a8_linear_chain
+ * accepts such addresses for x_bf16 and y (the bytes then cross the bus inside the kernel, with
+ * no copy-engine operation).  *dev_out receives the address; W4A8_ERR_INVALID_ARG when the
+ * buffer is pageable memory (which a kernel must not touch) or not host memory at all.  (A
+ * deployment helper; the paper has no counterpart.)
+ */
+int w4a8_host_buffer_device_pointer(const void* host, void** dev_out);
 
 /*
  * Self-test of the bounded device-side waits (the mechanism every kernel of the library uses; the

@@ -33,6 +33,7 @@ EXPORTS = (
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
     "w4a8_linear_chain", "w4a8_linear_chain_workspace_bytes", "w4a8_selftest_bounded_wait",
+    "w4a8_host_buffer_device_pointer",
 )
 
 CHAIN_INPUT_PLAIN, CHAIN_INPUT_SILU_MUL = 0, 1
@@ -122,6 +123,8 @@ def lib():
     L.w4a8_linear_chain_workspace_bytes.argtypes = [c.POINTER(ChainProblem), i32]
     L.w4a8_linear_chain.restype = i32
     L.w4a8_linear_chain.argtypes = [c.POINTER(ChainProblem), i32, p, sz, i32, p]
+    L.w4a8_host_buffer_device_pointer.restype = i32
+    L.w4a8_host_buffer_device_pointer.argtypes = [p, c.POINTER(c.c_void_p)]
     L.w4a8_selftest_bounded_wait.restype = i32
     L.w4a8_selftest_bounded_wait.argtypes = [c.c_uint64, p, p]
     L.w4a8_query_device_status.restype = i32
@@ -444,8 +447,19 @@ def dpq_quantize(W, U, perm=None, symmetric=False, mse_steps=0, per_channel=Fals
     return codes, gscale, gzero, s_w
 
 
+def host_buffer_device_pointer(t):
+    """w4a8_host_buffer_device_pointer: device-side address of a pinned host tensor."""
+    out = ctypes.c_void_p(0)
+    _check("w4a8_host_buffer_device_pointer",
+           lib().w4a8_host_buffer_device_pointer(ctypes.c_void_p(t.data_ptr()), ctypes.byref(out)))
+    return out.value
+
+
 def _addr(t):
-    return None if t is None else t.data_ptr()
+    """Address a kernel can use: the tensor's own for device tensors, the mapped one for pinned host tensors."""
+    if t is None:
+        return None
+    return t.data_ptr() if t.is_cuda else host_buffer_device_pointer(t)
 
 
 class LinearChain:
@@ -454,7 +468,8 @@ class LinearChain:
     Build it once from problem descriptions (dicts with the keys x, weight, y and optionally
     kind, depends_on, scale_mode, static_scale, x8_out, s_x_out), call it as often as wanted: the
     argument array and the zero-filled workspace are kept.  x: BF16 [M, K] (or [M, 2K] for the
-    gated kind), weight: TiledWeight, y: BF16 or FP32 [M, N]; all on one device."""
+    gated kind), weight: TiledWeight, y: BF16 or FP32 [M, N]; on one device, except that x and y may
+    be pinned host tensors (the kernel then reads / writes them over the bus)."""
 
     def __init__(self, problems, groups=0, workspace=None):
         import torch
@@ -466,7 +481,7 @@ class LinearChain:
             kind = d.get("kind", CHAIN_INPUT_PLAIN)
             assert x.dtype == torch.bfloat16 and x.stride(1) == 1 and y.stride(1) == 1
             q = self.arr[i]
-            q.x_bf16, q.ldx = x.data_ptr(), x.stride(0)
+            q.x_bf16, q.ldx = _addr(x), x.stride(0)
             q.input_kind, q.depends_on = kind, d.get("depends_on", -1)
             q.scale_mode, q.weight_format = d.get("scale_mode", SCALE_EXACT), tw.fmt
             q.static_scale = _addr(d.get("static_scale"))
@@ -474,7 +489,7 @@ class LinearChain:
             q.sw_stride = 0 if tw.s_w.numel() == 1 else 1
             q.out_dtype = OUT_FP32 if y.dtype == torch.float32 else OUT_BF16
             q.M, q.N, q.K = x.shape[0], tw.N, tw.K
-            q.y, q.ldy = y.data_ptr(), y.stride(0)
+            q.y, q.ldy = _addr(y), y.stride(0)
             x8o = d.get("x8_out")
             q.x8_out, q.ldx8_out = _addr(x8o), (0 if x8o is None else x8o.stride(0))
             q.s_x_out = _addr(d.get("s_x_out"))

@@ -1399,6 +1399,14 @@ int w4a8_linear_chain(const w4a8_chain_problem* problems_host, int count, void* 
                              static_cast<cudaStream_t>(stream));
 }
 
+int w4a8_host_buffer_device_pointer(const void* host, void** dev_out) {
+    if (!host || !dev_out) return W4A8_ERR_INVALID_ARG;
+    const void* d = host_buffer_as_device_pointer(host);
+    if (!d) return W4A8_ERR_INVALID_ARG;
+    *dev_out = const_cast<void*>(d);
+    return W4A8_OK;
+}
+
 int w4a8_selftest_bounded_wait(uint64_t limit_ns, uint64_t* elapsed_ns_dev, void* stream) {
     if (limit_ns == 0 || limit_ns > 1000000000ull) return W4A8_ERR_INVALID_ARG;   // at most one second
     if (reinterpret_cast<uintptr_t>(elapsed_ns_dev) & 7u) return W4A8_ERR_BAD_ALIGNMENT;

@@ -49,3 +49,25 @@ def test_single_process_passthrough_and_reference_arm_ranks():
     class A:
         steps, warmup, gpus = 1, 0, 2
     assert bench.run_reference(A, rank=1) is None      # ranks other than 0 do no work
+
+
+def test_gpus_without_a_launcher_starts_the_ranks_or_fails_loudly(monkeypatch):
+    # `bench.py --gpus N` with WORLD_SIZE unset re-runs itself under torch.distributed.run with N
+    # ranks on 127.0.0.1; with fewer devices than ranks it refuses instead of measuring one GPU
+    sys.path.insert(0, ROOT)
+    import pytest
+    import torch
+    import bench
+    monkeypatch.setattr(torch.cuda, "device_count", lambda: 1)
+    with pytest.raises(SystemExit) as e:
+        bench.spawn_ranks(2)
+    assert "2" in str(e.value) and "1 CUDA" in str(e.value)
+    seen = {}
+    monkeypatch.setattr(torch.cuda, "device_count", lambda: 8)
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "20", "--warmup", "5"])
+    assert bench.spawn_ranks(4) == 0
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-6:] == ["--gpus", "4", "--steps", "20", "--warmup", "5"] and cmd[-7].endswith("bench.py")

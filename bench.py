@@ -47,7 +47,7 @@ WORKLOAD = ("c2 decode sweep: W4A8 linear, M in {1,4,16}, K=4096, N=14336, INT4 
 # DRAM bytes per problem of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum of one launch divided by its problems); see profiles/.  None until a capture
 # exists for the current kernel.
-NCU_TRAFFIC_BYTES_PER_PROBLEM = None
+NCU_TRAFFIC_BYTES_PER_PROBLEM = 30.65e6  # profiles/linear_chain_decode_c2.md: (727.65 + 8.1) MB per 24-problem launch
 
 
 def weight_bytes(n=N, k=K):

@@ -131,6 +131,7 @@ __device__ __forceinline__ bool chain_poll_ge(const unsigned int* flag, unsigned
     uint32_t spins = 0;
     while (true) {
         if (ptx::ld_acquire_gpu(flag) >= target) return true;
+        __nanosleep(40);   // one poller per role and CTA, with a pause: the counter's L2 line is shared by every CTA
         if ((++spins & 15u) == 0u) {
             if (*abort_flag) return false;
             if (*reinterpret_cast<const volatile unsigned int*>(gabort)) {
@@ -535,9 +536,13 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             const int nseg = nseg_tab[i];
             if (nseg == 0) continue;
             // the problem's activations must have been quantized (by the epilogue warps of M CTAs)
-            ok = warp_all(chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit));
+            if (lane == 0) ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit);
+            ok = warp_all(ok);
+            __syncwarp();
             if (!ok) break;
-            asm volatile("fence.proxy.async.global;" ::: "memory");  // their writes, before this thread's bulk copies
+            // (lane 0 made the acquire; the warp barrier orders the other lanes behind it, and whichever lane is
+            // elected to issue fences the quantizers' writes before its own bulk copies)
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             const uint8_t* xt = ws + q.x8_off;
             const uint32_t rows_bytes = (uint32_t)q.M * 128u;         // the token rows are the first M rows of a tile
             for (int j = 0; j < nseg && ok; ++j) {
@@ -736,8 +741,8 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             float sx_mine = 0.0f;
             if (nseg > 0) {
                 // the scales were published together with the tiles the MMAs consume
-                ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit);
-                ok = !epi_any(!ok);
+                if (et == 0) ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit);
+                ok = !epi_any(!ok);   // (the barrier orders the other threads behind thread 0's acquire)
                 if (!ok) break;
                 sx_mine = (lane < q.M) ? __ldcg(sx_ws + i * kChainMaxM + lane) : 0.0f;
             }

@@ -40,3 +40,27 @@ def hessian_upper_cholesky_dev(H, perm=None, damp=0.01):
     Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
     Hinv = 0.5 * (Hinv + Hinv.T)
     return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()
+
+
+class Guarded:
+    """A device buffer with poisoned guard bands in front of and behind it: `t` is the usable part
+    (a view of `shape` / `dtype`, 256-byte aligned), check() asserts that the bands still hold the
+    poison -- a kernel that wrote outside the buffer it was given has changed them."""
+    BAND = 4096
+    POISON = 0xA5
+
+    def __init__(self, shape, dtype, fill=None):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.nbytes = n
+        self.raw = torch.full((n + 2 * self.BAND,), self.POISON, dtype=torch.uint8, device="cuda")
+        assert self.raw.data_ptr() % 256 == 0
+        self.t = self.raw[self.BAND:self.BAND + n].view(dtype).view(shape)
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self):
+        torch.cuda.synchronize()
+        front = self.raw[:self.BAND]
+        back = self.raw[self.BAND + self.nbytes:]
+        assert bool((front == self.POISON).all()), "bytes in front of the buffer were overwritten"
+        assert bool((back == self.POISON).all()), "bytes behind the buffer were overwritten"

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 import oracle
-from gpu_utils import bf16_bits, bf16_dev, dev, weights_to_dev
+from gpu_utils import Guarded, bf16_bits, bf16_dev, dev, weights_to_dev
 from helpers import bf16_gate, fp32_gate
 from paper_2505_14638_b200 import binding, inputs
 
@@ -226,6 +226,40 @@ def test_pow2_and_static_scales():
         ref = oracle.linear(x8, s_x, oracle.dequant_weight(*wq[:3]), wq[3])
         worst, _ = fp32_gate(outs[k].cpu().numpy(), ref["y64"], rel=2e-3)
         assert worst <= 2e-3, worst
+
+
+def test_chain_writes_only_its_outputs_and_its_workspace():
+    # poisoned guard bands around every buffer the chain writes: Y (with padding columns between the
+    # rows: ldy > N), the optional copies of the FP8 activations and scales, and a workspace of
+    # exactly the size the library asks for; shapes with whole blocks, a K-cut remainder and a short
+    # last block
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    shapes = [(16, sms * 96 + 176, 384), (3, 2000, 640), (8, 48, 128)]
+    probs, guards, pads = [], [], []
+    for i, (M, N, K) in enumerate(shapes):
+        wq, tw = _weights(N, K, 120 + i)
+        x = bf16_dev(inputs.make_activation(M, K, 130 + i, 0.01, 20.0))
+        ldy = N + 24
+        gy = Guarded((M, ldy), torch.bfloat16, fill=7.0)
+        g8 = Guarded((M, K), torch.uint8)
+        gs = Guarded((M,), torch.float32)
+        guards += [gy, g8, gs]
+        pads.append(gy)
+        probs.append(dict(x=x, weight=tw, y=gy.t[:, :N], x8_out=g8.t, s_x_out=gs.t))
+    probe = binding.LinearChain(probs)
+    gw = Guarded((probe.need,), torch.uint8, fill=0)
+    chain = binding.LinearChain(probs, workspace=gw.t)
+    for _ in range(3):
+        chain()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for g in guards + [gw]:
+        g.check()
+    for gy, (M, N, K) in zip(pads, shapes):
+        assert bool((gy.t[:, N:] == 7.0).all()), "padding columns of Y were written"
+        assert not bool((gy.t[:, :N] == 7.0).all())
+    # the counters are left zero for the next launch
+    assert int(gw.t[:1024].view(torch.int32).abs().sum().item()) == 0
 
 
 def test_chain_argument_errors():

@@ -21,30 +21,39 @@ pytestmark = pytest.mark.gpu
 
 def _sample_channels(N, W, n_random, seed):
     rng = np.random.default_rng(seed)
-    edge = [0, 1, 127, 128, 129, 255, 256, N // 2 - 1, N // 2, N - 257, N - 129, N - 128, N - 1]
+    edge = [0, 1, 95, 96, 97, 127, 128, 129, 191, 192, 255, 256, N // 2 - 1, N // 2, N - 257, N - 129, N - 128, N - 33,
+            N - 32, N - 1]
+    edge += [r for r in (148 * 96 - 1, 148 * 96, 2 * 148 * 96 - 1, 2 * 148 * 96) if r < N]   # 96-row blocks: last whole one / first cut along K
     top = int(np.argmax(np.max(np.abs(W), axis=1)))  # the channel that fixes the per-tensor scale
     rows = np.unique(np.concatenate([rng.choice(N, n_random, replace=False), np.array(edge + [top])]))
     return rows.astype(np.int64)
 
 
-def _run_case(M, N, K, sigma, frac, mult, seed, n_random):
+def _quantized_layer(N, K, sigma, seed, n_random, symmetric=True):
+    """Weights quantized on the GPU for all channels and by the oracle for a sample of them (which
+    must agree bit for bit), prepacked.  Returns (tiled weight, sampled rows, oracle weights)."""
     W = inputs.make_weight(N, K, sigma, seed)
     rows = _sample_channels(N, W, n_random, seed)
     Wd = torch.from_numpy(W).cuda()
-    codes, gscale, gzero, s_w = binding.quantize_weight_rtn(Wd, symmetric=True)
+    codes, gscale, gzero, s_w = binding.quantize_weight_rtn(Wd, symmetric=symmetric)
     del Wd
-    # oracle quantization of the sampled channels == the GPU's
-    oc, og, oz, osw = oracle.quantize_weight_rtn(W[rows], symmetric=True)
+    oc, og, oz, osw = oracle.quantize_weight_rtn(W[rows], symmetric=symmetric)
     del W
-    assert oz is None and gzero is None
     ridx = torch.from_numpy(rows).cuda()
     assert np.array_equal(codes[ridx].cpu().numpy(), oc)
     assert np.array_equal(bf16_bits(gscale[ridx]), og)
+    assert (oz is None) == (gzero is None)
+    if oz is not None:
+        assert np.array_equal(gzero[ridx].cpu().numpy(), oz)
     assert np.array_equal(s_w.cpu().numpy().view(np.uint32), osw.view(np.uint32))
-    tw = binding.prepack_weight(codes, gscale, gzero, s_w)
+    tw = binding.prepack_weight(codes, gscale, gzero, s_w)      # generic tiled format when asymmetric
     del codes, gscale
     assert binding.query_device_status() == 0
+    return tw, rows, ridx, (oc, og, oz, osw)
 
+
+def _run_case(M, N, K, sigma, frac, mult, seed, n_random, symmetric=True):
+    tw, rows, ridx, (oc, og, oz, osw) = _quantized_layer(N, K, sigma, seed, n_random, symmetric)
     xb = inputs.make_activation(M, K, seed, frac, mult)
     x = bf16_dev(xb)
     x8, s_x = binding.quantize_act(x)
@@ -58,7 +67,7 @@ def _run_case(M, N, K, sigma, frac, mult, seed, n_random):
     x8_ref, s_x_ref = oracle.quantize_act(xb)
     assert np.array_equal(x8.cpu().numpy(), x8_ref)
     assert np.array_equal(s_x.cpu().numpy().view(np.uint32), s_x_ref.view(np.uint32))
-    ref = oracle.linear(x8_ref, s_x_ref, oracle.dequant_weight(oc, og, None), osw, want=("y64",))
+    ref = oracle.linear(x8_ref, s_x_ref, oracle.dequant_weight(oc, og, oz), osw, want=("y64",))
     ok, dist = bf16_gate(bf16_bits(y[:, ridx]), ref["y64"])
     assert ok, dist
 
@@ -70,11 +79,75 @@ def test_config_c4_prefill_sampled_channels():
 
 @pytest.mark.parametrize("name,K,N,M", [("qkv", 4096, 6144, 512), ("o", 4096, 4096, 128),
                                         ("gate_up", 4096, 28672, 4096), ("down", 14336, 4096, 4096),
-                                        ("down", 14336, 4096, 32), ("gate_up", 4096, 28672, 8)])
+                                        ("down", 14336, 4096, 32), ("gate_up", 4096, 28672, 8),
+                                        ("qkv", 4096, 6144, 1), ("qkv", 4096, 6144, 32),
+                                        ("o", 4096, 4096, 1), ("o", 4096, 4096, 32),
+                                        ("gate_up", 4096, 28672, 128), ("down", 14336, 4096, 128)])
 def test_config_c5_layers_sampled_channels(name, K, N, M):
-    # c5: the four Llama-3-8B linears; token counts that reach the split-N kernel (<= 64), the
-    # persistent kernel with shared tiles (128, 512) and with whole tiles (4096)
+    # c5: the four Llama-3-8B linears; token counts that reach the split-N kernel (<= 64: the
+    # smallest layers there take the K-cut path), its 128-token tiles (128), the persistent kernel
+    # with shared tiles (512) and with whole tiles (4096)
     _run_case(M, N, K, 0.02, 0.01, 20.0, seed=500 + M + N // 64, n_random=40)
+
+
+@pytest.mark.parametrize("K,N,M", [(4096, 14336, 16), (4096, 6144, 2048)])
+def test_asymmetric_storage_at_layer_size_sampled_channels(K, N, M):
+    # the paper's stored format is asymmetric INT4 (Sec. 2.1, Sec. 4.1): zero-points per group, the
+    # generic tiled layout, at Llama layer sizes on the decode and on the prefill kernel
+    _run_case(M, N, K, 0.02, 0.01, 20.0, seed=900 + M, n_random=40, symmetric=False)
+
+
+def test_chain_launch_at_c2_size_and_gated_block_at_layer_size():
+    # The launch the benchmark times: M = 1, 4, 16 on the c2 layer (K = 4096, N = 14336) as three
+    # problems of one w4a8_linear_chain launch, then a Llama-3-8B MLP block as a dependent chain
+    # (gate/up -> silu(gate) * up quantized in the kernel -> down).  FP8 activations and scales bit
+    # for bit; outputs on sampled channels, every stage on the input that stage saw.
+    tw, rows, ridx, (oc, og, oz, osw) = _quantized_layer(14336, 4096, 0.02, 41, 40)
+    w8 = oracle.dequant_weight(oc, og, oz)
+    probs, xbs = [], []
+    for M in (1, 4, 16):
+        xb = inputs.make_activation(M, 4096, 40 + M, 0.01, 20.0)
+        xbs.append(xb)
+        probs.append(dict(x=bf16_dev(xb), weight=tw, y=torch.zeros((M, 14336), dtype=torch.bfloat16, device="cuda"),
+                          x8_out=torch.zeros((M, 4096), dtype=torch.uint8, device="cuda"),
+                          s_x_out=torch.zeros((M,), dtype=torch.float32, device="cuda")))
+    chain = binding.LinearChain(probs)
+    chain()
+    chain()      # a second launch on the same workspace
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for d, xb in zip(probs, xbs):
+        x8_ref, s_x_ref = oracle.quantize_act(xb)
+        assert np.array_equal(d["x8_out"].cpu().numpy(), x8_ref)
+        assert np.array_equal(d["s_x_out"].cpu().numpy().view(np.uint32), s_x_ref.view(np.uint32))
+        ref = oracle.linear(x8_ref, s_x_ref, w8, osw, want=("y64",))
+        ok, dist = bf16_gate(bf16_bits(d["y"][:, ridx]), ref["y64"])
+        assert ok, dist
+    del tw, probs, chain
+
+    H, F, M = 4096, 14336, 4
+    tw_gu, rows_gu, ridx_gu, (gc, gg, gz, gsw) = _quantized_layer(2 * F, H, 0.02, 42, 40)
+    tw_dn, rows_dn, ridx_dn, (dc, dg, dz, dsw) = _quantized_layer(H, F, 0.02, 43, 40)
+    xb = inputs.make_activation(M, H, 44, 0.01, 20.0)
+    gu = torch.zeros((M, 2 * F), dtype=torch.bfloat16, device="cuda")
+    dn = torch.zeros((M, H), dtype=torch.bfloat16, device="cuda")
+    h8 = torch.zeros((M, F), dtype=torch.uint8, device="cuda")
+    sh = torch.zeros((M,), dtype=torch.float32, device="cuda")
+    binding.LinearChain([dict(x=bf16_dev(xb), weight=tw_gu, y=gu),
+                         dict(x=gu, weight=tw_dn, y=dn, kind=binding.CHAIN_INPUT_SILU_MUL, depends_on=0,
+                              x8_out=h8, s_x_out=sh)])()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    x8_ref, s_x_ref = oracle.quantize_act(xb)
+    ref = oracle.linear(x8_ref, s_x_ref, oracle.dequant_weight(gc, gg, gz), gsw, want=("y64",))
+    ok, dist = bf16_gate(bf16_bits(gu[:, ridx_gu]), ref["y64"])
+    assert ok, dist
+    want8, wants = binding.silu_mul_quantize(gu)      # the same arithmetic on the same input
+    torch.cuda.synchronize()
+    assert torch.equal(h8, want8) and torch.equal(sh, wants)
+    ref = oracle.linear(h8.cpu().numpy(), sh.cpu().numpy(), oracle.dequant_weight(dc, dg, dz), dsw, want=("y64",))
+    ok, dist = bf16_gate(bf16_bits(dn[:, ridx_dn]), ref["y64"])
+    assert ok, dist
 
 
 def test_two_cta_kernel_shape_exact_integers_and_gaussian():

@@ -55,11 +55,10 @@ def weight_bytes(n=N, k=K):
     return n * k // 2 + n * (k // GROUP) * 2
 
 
-def linear_algorithmic_bytes(m, n=N, k=K, fused=False):
-    """Everything one linear launch must move: weights, activations (FP8 + scales, or BF16 when the
-    quantization is fused), the weight scale, BF16 output."""
-    act = 2 * m * k if fused else m * k + 4 * m
-    return weight_bytes(n, k) + act + 4 + 2 * m * n
+def linear_algorithmic_bytes(m, n=N, k=K):
+    """Everything one linear launch must move: weights, FP8 activations + scales, the weight scale,
+    BF16 output."""
+    return weight_bytes(n, k) + m * k + 4 * m + 4 + 2 * m * n
 
 
 def load_peaks():
@@ -600,8 +599,8 @@ C5_M = (1, 8, 32, 128, 512, 4096)
 
 
 def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, with_cublas=True):
-    """Config c5: the four Llama-3-8B linears x M.  Per case: time of quantize_act + linear (the
-    fused launch where it is the faster one) and of the linear alone, from CUDA graphs of
+    """Config c5: the four Llama-3-8B linears x M.  Per case: time of quantize_act + linear and of the
+    linear alone (for M <= 16 also per problem of a w4a8_linear_chain launch), from CUDA graphs of
     back-to-back launches that rotate over enough weight copies to exceed twice the L2; the
     roofline time is the larger of bytes / HBM peak and flops / (2 x BF16 burst peak)."""
     out = []
@@ -643,19 +642,26 @@ def layer_sweep(torch, binding, inputs, dev, peaks, layers=C5_LAYERS, ms=C5_M, w
                 binding.linear_tiled(x8, s_x, tws[c % copies], out=y, workspace=ws)
 
             def whole(c):
-                if binding.fused_is_faster(m, n, k):
-                    binding.linear_fused(x, tws[c % copies], out=y)
-                else:
-                    binding.quantize_act(x, out=(x8, s_x))
-                    lin(c)
+                binding.quantize_act(x, out=(x8, s_x))
+                lin(c)
             t_lin = graph_time(lin, reps)
             t_all = graph_time(whole, reps)
+            t_chain = None
+            if m <= binding.CHAIN_MAX_M:
+                # the same layer as problems of one persistent launch (quantization included)
+                nprob = min(binding.CHAIN_MAX_PROBLEMS, max(copies, 8))
+                chain = binding.LinearChain([dict(x=x, weight=tws[c % copies], y=y) for c in range(nprob)])
+                t_chain = _time_loop(torch, chain, 10, warm=3) / nprob
+                del chain
             flops = 2.0 * m * n * k
             t_roof = max(linear_algorithmic_bytes(m, n, k) / hbm, flops / fp8_peak)
             row = {"layer": name, "K": k, "N": n, "M": m, "linear_us": t_lin * 1e6, "quant_plus_linear_us": t_all * 1e6,
                    "tflops": flops / t_lin / 1e12, "weight_GBps": wbytes / t_lin / 1e9,
                    "roofline_us": t_roof * 1e6, "frac_of_roofline": t_roof / t_lin,
                    "bound": "hbm" if linear_algorithmic_bytes(m, n, k) / hbm > flops / fp8_peak else "tensor"}
+            if t_chain is not None:
+                row["chain_us_per_problem"] = t_chain * 1e6
+                row["chain_frac_of_roofline"] = chain_algorithmic_bytes((m,), n, k) / hbm / t_chain
             if with_cublas:
                 row["cublas_bf16_us"] = graph_time(lambda c: torch.matmul(x, wb.t()), 4) * 1e6
                 # W8A8 with the library's FP8 GEMM (FP8 weights read as they are: twice the bytes, no

@@ -181,36 +181,6 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
                                int64_t ldy, int out_dtype, int split_k, void* stream);
 
 /*
- * Fused decode-sized layer: y = Linear(quantize_act(x)) in ONE kernel (Sec. 3 inference flow:
- * Eq. 13 activation quantization, Eq. 10 weight dequantization, FP8 GEMM, Eq. 4 / Eq. 11
- * epilogue), for M <= W4A8_FUSED_MAX_M tokens and prepacked (tiled) weights.  The results are
- * those of w4a8_quantize_act followed by w4a8_linear, bit for bit: same scale, same FP8 codes,
- * same accumulation.
- *   x_bf16      device, BF16 [M][ldx], 16-byte aligned rows (ldx % 8 == 0), K % 128 == 0.
- *   weights     device, output of w4a8_prepack_weight; weight_format TILED or TILED_SIGNMAG.
- *   scale_mode, static_scale   as in w4a8_quantize_act.
- *   x8_out      optional (may be NULL): device u8 [M][ldx8_out], receives the FP8 activations
- *               the kernel multiplied with (ldx8_out % 16 == 0, 16-byte aligned);
- *   s_x_out     optional (may be NULL): device float [M], receives the activation scales.
- *   y, ldy, out_dtype, s_w, sw_stride   as in w4a8_linear.
- * On B200 the fused launch turned out slower than w4a8_quantize_act + w4a8_linear chained on one
- * stream (they overlap under programmatic dependent launch; every CTA of the fused launch scans X
- * for the token scales): it is kept for callers that want a single launch.
- * Needs no workspace and allocates nothing; its run-time placement of worker CTAs uses the
- * library's 64-entry table (see w4a8_linear: at most 64 such launches in flight on a device).
- * Errors: W4A8_ERR_BAD_SHAPE for M > the limit or a
- * K / N the tiled format does not admit; otherwise as w4a8_linear.
- */
-#define W4A8_FUSED_MAX_M 16
-/* 1 when w4a8_linear_fused is the faster way to run this problem on B200, 0 when
- * w4a8_quantize_act + w4a8_linear is (currently always 0: see w4a8_linear_fused). */
-int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K);
-int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
-                      const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
-                      int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
-                      float* s_x_out, void* stream);
-
-/*
  * A chain of decode-sized layers in ONE persistent launch (Sec. 3 inference flow for every
  * problem of the chain: Eq. 13 activation quantization, Eq. 10 weight dequantization, FP8 GEMM,
  * Eq. 4 / Eq. 11 epilogue; Sec. 1 on the memory-bound regime of small batches this is for).
@@ -422,8 +392,7 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
 
 /*
  * Whole layer from HOST activations to HOST output (Sec. 3 flow end to end): copies
- * x_host (BF16 [M][K], ideally pinned) to x_dev, runs w4a8_quantize_act and w4a8_linear (or
- * w4a8_linear_fused when the weights are prepacked and w4a8_fused_is_faster says so), and
+ * x_host (BF16 [M][K], ideally pinned) to x_dev, runs w4a8_quantize_act and w4a8_linear, and
  * copies y_dev (BF16 [M][N]) to y_host, all enqueued on `stream`; the caller synchronises the
  * stream before reading y_host.  Weights stay resident on the device.  Scratch device buffers
  * are the caller's: x_dev (2*M*K bytes), x8_dev (M*K), s_x_dev (4*M), y_dev (2*M*N), workspace.

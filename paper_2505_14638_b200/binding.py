@@ -27,7 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
-    "w4a8_linear_fused", "w4a8_fused_is_faster", "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
+    "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
     "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
@@ -101,10 +101,6 @@ def lib():
     L.w4a8_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p, p]
     L.w4a8_linear_w8a8.restype = i32
     L.w4a8_linear_w8a8.argtypes = [p, i64, p, i64, p, p, i32, i64, i64, p, i64, i32, p, sz, p]
-    L.w4a8_fused_is_faster.restype = i32
-    L.w4a8_fused_is_faster.argtypes = [i64, i64, i64]
-    L.w4a8_linear_fused.restype = i32
-    L.w4a8_linear_fused.argtypes = [p, i64, i64, i32, p, p, i32, p, i32, i64, i64, p, i64, i32, p, i64, p, p]
     L.w4a8_linear_ex_workspace_bytes.restype = sz
     L.w4a8_linear_ex_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
     L.w4a8_quantize_weight_rtn.restype = i32
@@ -372,32 +368,6 @@ def linear_w8a8(x8, s_x, w8, s_w, out_dtype=OUT_BF16, out=None):
                                 0 if s_w.numel() == 1 else 1, N, K, _ptr(out), out.stride(0), int(out_dtype),
                                 _ptr(ws), nb, _stream())
     _check("w4a8_linear_w8a8", rc)
-    return out
-
-
-FUSED_MAX_M = 16
-
-
-def fused_is_faster(M, N, K):
-    """w4a8_fused_is_faster: whether the fused launch is the faster way to run this problem."""
-    return bool(lib().w4a8_fused_is_faster(M, N, K))
-
-
-def linear_fused(x, tw, out_dtype=OUT_BF16, out=None, scale_mode=SCALE_EXACT, static_scale=None,
-                 x8_out=None, s_x_out=None):
-    """w4a8_linear_fused: BF16 activations [M <= 16, K] and a TiledWeight -> Y, one kernel.
-    x8_out (uint8 [M, K]) / s_x_out (float32 [M]) optionally receive the quantized activations."""
-    import torch
-    M, K = x.shape
-    assert K == tw.K and x.dtype == torch.bfloat16
-    if out is None:
-        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
-        out = torch.empty((M, tw.N), dtype=dt, device=x.device)
-    rc = lib().w4a8_linear_fused(_ptr(x), x.stride(0), M, int(scale_mode), _ptr(static_scale), _ptr(tw.buf),
-                                 tw.fmt, _ptr(tw.s_w), 0 if tw.s_w.numel() == 1 else 1, tw.N, K, _ptr(out),
-                                 out.stride(0), int(out_dtype), _ptr(x8_out),
-                                 0 if x8_out is None else x8_out.stride(0), _ptr(s_x_out), _stream())
-    _check("w4a8_linear_fused", rc)
     return out
 
 

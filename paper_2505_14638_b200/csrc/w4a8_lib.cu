@@ -353,36 +353,30 @@ static std::atomic<unsigned int> g_sched_seq{0};
 template <class Cfg>
 static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                                  int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
-                                 cudaStream_t st, const SnFuse& fuse, void* workspace, bool ws_usable,
-                                 const SnPlan& pl, int sms);
+                                 cudaStream_t st, void* workspace, bool ws_usable, const SnPlan& pl, int sms);
 
-template <int MT, int G, int FMT, bool FUSE = false>
+template <int MT, int G, int FMT>
 static int launch_splitn_cfg(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                              int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, cudaStream_t st,
-                             const SnFuse& fuse = SnFuse{}, void* workspace = nullptr, size_t workspace_bytes = 0) {
-    using Cfg = SnCfg<MT, G, FMT, FUSE, false>;
+                             void* workspace = nullptr, size_t workspace_bytes = 0) {
+    using Cfg = SnCfg<MT, G, FMT, false>;
     const int sms = sm_count();
     if (sms <= 0) return W4A8_ERR_CUDA;
     SnPlan pl;
     // K is cut only when the caller gave the (zero-initialised) workspace for the partial sums
     const bool ws_usable = workspace != nullptr && workspace_bytes >= kSnWorkspaceBytes && aligned16(workspace);
-    const bool may_split_k = !FUSE && ws_usable;
-    if (!make_sn_plan<Cfg>(N, K, sms, may_split_k, &pl)) return W4A8_ERR_BAD_SHAPE;
-    if constexpr (!FUSE) {
-        if (pl.KSPLIT > 1)
-            return launch_splitn_planned<SnCfg<MT, G, FMT, false, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                         out_dtype, M, N, K, st, fuse, workspace,
-                                                                         ws_usable, pl, sms);
-    }
-    return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, fuse, workspace,
+    if (!make_sn_plan<Cfg>(N, K, sms, ws_usable, &pl)) return W4A8_ERR_BAD_SHAPE;
+    if (pl.KSPLIT > 1)
+        return launch_splitn_planned<SnCfg<MT, G, FMT, true>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K,
+                                                              st, workspace, ws_usable, pl, sms);
+    return launch_splitn_planned<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, st, workspace,
                                       ws_usable, pl, sms);
 }
 
 template <class Cfg>
 static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                                  int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K,
-                                 cudaStream_t st, const SnFuse& fuse, void* workspace, bool ws_usable,
-                                 const SnPlan& pl, int sms) {
+                                 cudaStream_t st, void* workspace, bool ws_usable, const SnPlan& pl, int sms) {
     auto kern = linear_splitn_kernel<Cfg>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -419,7 +413,7 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, M, N, K, plan,
-                                       fuse, counters, partials, status);
+                                       counters, partials, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
@@ -496,23 +490,23 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
         if (mt == 128) {
             return fmt == kFmtTiledSignMag
                        ? launch_splitn_cfg<128, 4, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
-                                                                     Mi, Ni, Ki, st, SnFuse{}, workspace,
+                                                                     Mi, Ni, Ki, st, workspace,
                                                                      workspace_bytes)
                        : launch_splitn_cfg<128, 4, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi, Ni,
-                                                              Ki, st, SnFuse{}, workspace, workspace_bytes);
+                                                              Ki, st, workspace, workspace_bytes);
         }
         if (fmt == kFmtTiledSignMag) {
             return mt == 16 ? launch_splitn_cfg<16, 2, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                            out_dtype, Mi, Ni, Ki, st, SnFuse{},
+                                                                            out_dtype, Mi, Ni, Ki, st,
                                                                             workspace, workspace_bytes)
                             : launch_splitn_cfg<64, 4, kFmtTiledSignMag>(tx, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                            out_dtype, Mi, Ni, Ki, st, SnFuse{},
+                                                                            out_dtype, Mi, Ni, Ki, st,
                                                                             workspace, workspace_bytes);
         }
         return mt == 16 ? launch_splitn_cfg<16, 2, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
-                                                                 Ni, Ki, st, SnFuse{}, workspace, workspace_bytes)
+                                                                 Ni, Ki, st, workspace, workspace_bytes)
                         : launch_splitn_cfg<64, 4, kFmtTiled>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, Mi,
-                                                                 Ni, Ki, st, SnFuse{}, workspace, workspace_bytes);
+                                                                 Ni, Ki, st, workspace, workspace_bytes);
     }
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return W4A8_ERR_BAD_ALIGNMENT;
     SkPlan pl;
@@ -736,44 +730,6 @@ static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_
         rc = launch_status();
     }
     return rc;
-}
-
-static int linear_fused_impl(const void* x, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
-                             const uint8_t* wpp, int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K,
-                             void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out, float* s_x_out,
-                             cudaStream_t st) {
-    if (!x || !wpp || !s_w || !y) return W4A8_ERR_INVALID_ARG;
-    if (fmt != kFmtTiled && fmt != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
-    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
-    if (scale_mode != W4A8_SCALE_EXACT && scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
-    if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
-    if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
-    if (M > W4A8_FUSED_MAX_M || K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
-    if (ldx < K || ldy < N || (x8_out && ldx8_out < K)) return W4A8_ERR_BAD_SHAPE;
-    if (N > INT32_MAX || K > INT32_MAX) return W4A8_ERR_BAD_SHAPE;
-    if (!aligned16(x) || !aligned16(wpp) || !aligned16(y) || (ldx % 8) != 0) return W4A8_ERR_BAD_ALIGNMENT;
-    if (x8_out && (!aligned16(x8_out) || (ldx8_out % 16) != 0)) return W4A8_ERR_BAD_ALIGNMENT;
-    if ((reinterpret_cast<uintptr_t>(s_w) & 3u) || (reinterpret_cast<uintptr_t>(s_x_out) & 3u) ||
-        (reinterpret_cast<uintptr_t>(static_scale) & 3u))
-        return W4A8_ERR_BAD_ALIGNMENT;
-    int rc = check_device();
-    if (rc != W4A8_OK) return rc;
-    SnFuse fuse;
-    fuse.x = static_cast<const uint16_t*>(x);
-    fuse.ldx = ldx;
-    fuse.scale_mode = scale_mode;
-    fuse.static_scale = static_scale;
-    fuse.x8_out = x8_out;
-    fuse.ldx8_out = ldx8_out;
-    fuse.s_x_out = s_x_out;
-    CUtensorMap unused;
-    memset(&unused, 0, sizeof(unused));
-    const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
-    if (fmt == kFmtTiledSignMag)
-        return launch_splitn_cfg<16, 2, kFmtTiledSignMag, true>(unused, wpp, nullptr, s_w, sw_stride, y, ldy,
-                                                                   out_dtype, Mi, Ni, Ki, st, fuse);
-    return launch_splitn_cfg<16, 2, kFmtTiled, true>(unused, wpp, nullptr, s_w, sw_stride, y, ldy, out_dtype, Mi,
-                                                        Ni, Ki, st, fuse);
 }
 
 static int quantize_act_impl(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* x8, int64_t ldx8,
@@ -1182,28 +1138,6 @@ size_t w4a8_linear_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     return w4a16_workspace(M, N, K);
 }
 
-int w4a8_fused_is_faster(int64_t M, int64_t N, int64_t K) {
-    // Measured on B200 (c2 layer, CUDA graphs): in a chain of equal launches one token takes 13.3 us
-    // fused against 14.5 us for quantize + linear, four tokens 14.3 against 11.5 us, sixteen 20.2
-    // against 11.8 us; in the benchmark's mixed chain (M = 1, 4, 16) the two-kernel sequence wins for
-    // every M (39.3 against 43.0 us per step with M = 1 fused).  The two kernels overlap under
-    // programmatic dependent launch and the linear leaves a few SMs to the quantize kernel, while
-    // every CTA of the fused launch has to scan X for the token scales; with few output channels the
-    // two-kernel path also cuts K across the SMs, which the fused launch (no workspace) cannot.
-    (void)M;
-    (void)N;
-    (void)K;
-    return 0;
-}
-
-int w4a8_linear_fused(const void* x_bf16, int64_t ldx, int64_t M, int scale_mode, const float* static_scale,
-                      const uint8_t* weights, int weight_format, const float* s_w, int sw_stride, int64_t N,
-                      int64_t K, void* y, int64_t ldy, int out_dtype, uint8_t* x8_out, int64_t ldx8_out,
-                      float* s_x_out, void* stream) {
-    return linear_fused_impl(x_bf16, ldx, M, scale_mode, static_scale, weights, weight_format, s_w, sw_stride, N, K,
-                             y, ldy, out_dtype, x8_out, ldx8_out, s_x_out, static_cast<cudaStream_t>(stream));
-}
-
 int w4a8_silu_mul_quantize(const void* gate_up_bf16, int64_t M, int64_t F, int64_t ldgu, uint8_t* x8, int64_t ldx8,
                            float* s_x, int scale_mode, const float* static_scale, void* h_bf16_out, int64_t ldh,
                            void* stream) {
@@ -1370,19 +1304,11 @@ int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights
     }
     if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
-    if (weight_format != kFmtCanonical && w4a8_fused_is_faster(M, N, K) == 1) {
-        // a few tokens and prepacked weights: one kernel quantizes the activations and multiplies
-        // (measured faster than the two-kernel sequence up to here, slower above)
-        rc = linear_fused_impl(x_dev, K, M, W4A8_SCALE_EXACT, nullptr, weights, weight_format, s_w, sw_stride, N, K,
-                               y_dev, N, W4A8_OUT_BF16, nullptr, 0, nullptr, st);
-        if (rc != W4A8_OK) return rc;
-    } else {
-        rc = quantize_act_impl(x_dev, M, K, K, x8_dev, K, s_x_dev, W4A8_SCALE_EXACT, nullptr, st);
-        if (rc != W4A8_OK) return rc;
-        rc = linear_impl(x8_dev, K, s_x_dev, M, weights, gscale_bf16, gzero, weight_format, s_w, sw_stride, N, K,
-                         group, y_dev, N, W4A8_OUT_BF16, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, st);
-        if (rc != W4A8_OK) return rc;
-    }
+    rc = quantize_act_impl(x_dev, M, K, K, x8_dev, K, s_x_dev, W4A8_SCALE_EXACT, nullptr, st);
+    if (rc != W4A8_OK) return rc;
+    rc = linear_impl(x8_dev, K, s_x_dev, M, weights, gscale_bf16, gzero, weight_format, s_w, sw_stride, N, K,
+                     group, y_dev, N, W4A8_OUT_BF16, workspace, workspace_bytes, W4A8_ALGO_AUTO, 0, st);
+    if (rc != W4A8_OK) return rc;
     if (cudaMemcpyAsync(y_host_bf16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
     return W4A8_OK;

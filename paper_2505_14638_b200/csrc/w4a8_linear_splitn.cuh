@@ -36,16 +36,11 @@ namespace w4a8 {
 
 
 
-template <int MT_, int G_, int FMT_, bool FUSE_ = false, bool SPLITK_ = false>
+template <int MT_, int G_, int FMT_, bool SPLITK_ = false>
 struct SnCfg {
     // SPLITK: the K range may be cut in chunks (layers with few output channels); otherwise the
     // chunk arithmetic is compiled out.
     static constexpr bool SPLITK = SPLITK_;
-    // FUSE: the kernel takes BF16 activations and does the per-token FP8 quantization (Eq. 13)
-    // itself: an absmax pass over X before the main loop (overlapped with the first weight copies)
-    // and a convert step that writes each stage's FP8 activation tile into shared memory, in the
-    // layout a 128-byte-swizzled TMA tile would have had.
-    static constexpr bool FUSE = FUSE_;
     static constexpr int MT = MT_;      // tokens per tile = MMA N (16 or 64)
     static constexpr int G = G_;        // dequantization groups of 4 warps
     static constexpr int FMT = FMT_;
@@ -68,39 +63,7 @@ struct SnCfg {
     static_assert(MT == 16 || MT == 64 || MT == 128, "token tile");
     static_assert(kDCol + 2 * MT <= kTmemCols, "tensor memory columns");
     static_assert((3 * kS1Max + kS2 + 3) * 8 + 16 + 3 * 64 + 16 <= kBarBytes, "barrier area");
-    static_assert(!FUSE_ || MT_ == 16, "the fused activation quantization is built for <= 16 tokens");
-    static_assert(!(FUSE_ && SPLITK_), "the fused launch has no workspace and never cuts K");
 };
-
-constexpr int kFuseFewTokens = 4;
-
-// Fused activation quantization: which part of which stage's activation tile one of the 128
-// converting threads produces.  A stage's tile (2 k-blocks x Mp tokens, Mp = the token count
-// rounded up to a power of two) takes 8*Mp threads, 32 elements each; the 128 threads therefore
-// can work on up to 16/Mp consecutive stages at once, which keeps that many stages' loads in
-// flight.  No more than S1 (the ring depth) at once, though: a thread that waited for a slot two
-// ring rounds ahead could not tell the rounds apart by the barrier's parity.
-struct XMap {
-    int tps;   // threads per stage (those beyond 8*Mp only arrive on the barrier)
-    int span;  // stages worked on at once = 128 / tps
-    int sub;   // this thread's stage within a group of `span`
-    int xj;    // k-block within the stage (0 or 1)
-    int xrow;  // token
-    int xq;    // 32-element quarter of the k-block
-};
-__device__ __forceinline__ XMap x_map(int r, int M, int S1) {
-    const int lg = M <= 1 ? 0 : M <= 2 ? 1 : M <= 4 ? 2 : M <= 8 ? 3 : 4;
-    XMap m;
-    m.span = 16 >> lg;
-    while (m.span > S1) m.span >>= 1;
-    m.tps = 128 / m.span;
-    m.sub = r / m.tps;
-    const int within = r & (m.tps - 1);
-    m.xq = within & 3;
-    m.xrow = (within >> 2) & ((1 << lg) - 1);
-    m.xj = within >> (2 + lg);  // >= 2 for the threads with nothing to convert
-    return m;
-}
 
 // Launch-time plan shared by host and device.
 struct SnPlan {
@@ -216,25 +179,13 @@ __device__ __forceinline__ void sched_hold(SchedSlot* sl, int workers, unsigned 
     }
 }
 
-// Arguments of the fused activation quantization (unused otherwise).
-struct SnFuse {
-    const uint16_t* x;          // BF16 activations [M][ldx]
-    int64_t ldx;
-    int scale_mode;
-    const float* static_scale;  // nullptr = dynamic per-token scale
-    uint8_t* x8_out;            // optional copies of the FP8 activations and their scales,
-    int64_t ldx8_out;           // written by CTA 0 only (nullptr = not wanted)
-    float* s_x_out;
-};
-
 // Epilogue of the split-N kernel: scales 16 tokens of accumulated sums (row r of 128-row block b,
 // tokens c0..c0+15) with Eq. 4 / Eq. 11 and writes them to Y, through the staging area in 16-byte
 // pieces when the rows of Y are 16-byte aligned.  Called by all 128 epilogue threads together.
 template <class Cfg>
 __device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, int b, int c0, int r, int et, int R,
                                         int n0, int M, int es, bool wide_out, uint32_t out_s, void* y, int64_t ldy,
-                                        const float (&sx_lane)[Cfg::MT / 32 > 0 ? Cfg::MT / 32 : 1],
-                                        const float* sx_s) {
+                                        const float (&sx_lane)[Cfg::MT / 32 > 0 ? Cfg::MT / 32 : 1]) {
     constexpr int MT = Cfg::MT;
 
     const int row = b * 128 + r;
@@ -247,7 +198,7 @@ __device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, i
     float res[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const float sxm = Cfg::FUSE ? sx_s[c0 + j] : __shfl_sync(0xFFFFFFFFu, sxv, (c0 & 16) + j);
+        const float sxm = __shfl_sync(0xFFFFFFFFu, sxv, (c0 & 16) + j);
         res[j] = __uint_as_float(accv[j]) * (sxm * swb);  // Eq. 4, Eq. 11
     }
     if (wide_out) {
@@ -296,11 +247,11 @@ __device__ __forceinline__ void sn_emit(const uint32_t (&accv)[16], float swb, i
 // registers), or the CTA that finds no room starts a whole layer late.  Bounds for 576 threads
 // give 56 registers: 2 x 448 x 56 + 256 x 48 <= 65536.
 template <class Cfg>
-__global__ void __launch_bounds__(Cfg::MT == 16 && !Cfg::FUSE ? 576 : Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
+__global__ void __launch_bounds__(Cfg::MT == 16 ? 576 : Cfg::kThreads, Cfg::MT == 16 ? 2 : 1)
 linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x MT, 128B swizzle
                      const uint8_t* __restrict__ wpp, const float* __restrict__ s_x,
                      const float* __restrict__ s_w, int sw_stride, void* __restrict__ y, int64_t ldy,
-                     int out_dtype, int M, int N, int K, const SnPlan plan, const SnFuse fuse,
+                     int out_dtype, int M, int N, int K, const SnPlan plan,
                      unsigned int* counters, float* partials, unsigned int* status_word) {
     constexpr int MT = Cfg::MT, G = Cfg::G, S2 = Cfg::kS2, MB = Cfg::kMeta;
     constexpr int S1M = Cfg::kS1Max;
@@ -326,10 +277,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     const uint32_t out_s = bars_addr + (uint32_t)Cfg::kBarBytes;  // epilogue staging, kOutBytes
-    unsigned int* amax_s = const_cast<unsigned int*>(tmem_slot) + 4;  // [16] row absmax bit patterns
-    float* sx_s = reinterpret_cast<float*>(amax_s + 16);              // [16] activation scales s_x
-    float* inv_s = sx_s + 16;                                         // [16] multipliers 1/s_x
-    volatile unsigned int* ticket_s = reinterpret_cast<volatile unsigned int*>(inv_s + 16);
+    volatile unsigned int* ticket_s = reinterpret_cast<volatile unsigned int*>(tmem_slot + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = K >> 7;
@@ -372,7 +320,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     if (threadIdx.x == 32) {
         for (int s = 0; s < S1; ++s) {
             ptx::mbar_init(bar_full0 + 8u * s, 1);
-            ptx::mbar_init(bar_xfull0 + 8u * s, Cfg::FUSE ? (uint32_t)x_map(0, M, S1).tps : 1u);
+            ptx::mbar_init(bar_xfull0 + 8u * s, 1u);
             ptx::mbar_init(bar_free10 + 8u * s, 1);
         }
         for (int s = 0; s < S2; ++s) ptx::mbar_init(bar_a_full0 + 8u * s, 128);
@@ -381,9 +329,8 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         ptx::mbar_init(bar_drain, 1);
         *abort_flag = 0u;
         ptx::fence_mbar_init();
-        if (!Cfg::FUSE) ptx::prefetch_tensormap(&tmap_x);
+        ptx::prefetch_tensormap(&tmap_x);
     }
-    if (Cfg::FUSE && threadIdx.x >= 64 && threadIdx.x < 80) amax_s[threadIdx.x - 64] = 0u;
     if (plan.sched >= 0) {
         __syncthreads();
         p = worker_s;
@@ -407,92 +354,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     ptx::griddep_launch_dependents();
-
-    // FUSE: first activation chunks of the converting threads (warps 2..5), fetched before the absmax
-    // pass so that they are in flight during it.
-    uint4 xv[4];
-    bool xv_loaded = false;
-    // Few tokens: only the four epilogue warps (idle until the end) do the absmax pass and the
-    // dequantizers start at once.  More tokens: every warp but the two issuers takes part.
-    const bool fuse_all = M > kFuseFewTokens;
-    if (Cfg::FUSE && warp >= 2 && (fuse_all || warp < 6)) {
-        // Eq. 13, first half: per-token absmax and scale while the first weight stages are in flight.
-        const int NF = fuse_all ? Cfg::kThreads - 64 : 128;
-        const int ft = (int)threadIdx.x - 64;
-        ptx::griddep_wait();  // X comes from the previous kernel in the stream
-        if (warp < 6) {
-            const XMap xm = x_map((warp & 3) * 32 + lane, M, S1);  // as in the epilogue branch below
-            const int kbk = xm.sub * KS + xm.xj;
-            if (xm.xrow < M && xm.xj < KS && kbk < KB) {
-                const uint4* xp = reinterpret_cast<const uint4*>(fuse.x + (int64_t)xm.xrow * fuse.ldx +
-                                                                 (int64_t)kbk * 128 + xm.xq * 32);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) xv[j] = __ldg(xp + j);
-            }
-            xv_loaded = true;
-        }
-        if (fuse.static_scale == nullptr) {
-            const int nch = K >> 3;  // 16-byte chunks per row
-#pragma unroll 1
-            for (int m0 = 0; m0 < M; m0 += 4) {
-                float rm[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                for (int c = ft; c < nch; c += 2 * NF) {
-                    // eight 16-byte loads in flight per thread: four tokens x two chunks
-                    const bool two = c + NF < nch;
-                    uint4 v[4], w[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (m0 + j < M) {
-                            const uint4* row = reinterpret_cast<const uint4*>(fuse.x + (int64_t)(m0 + j) * fuse.ldx);
-                            v[j] = __ldg(row + c);
-                            if (two) w[j] = __ldg(row + c + NF);
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (m0 + j < M) {
-                            rm[j] = absmax_bf16x8(v[j], rm[j]);
-                            if (two) rm[j] = absmax_bf16x8(w[j], rm[j]);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (m0 + j < M) {  // uniform
-                        float a = rm[j];
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
-                        // non-negative floats order like their bit patterns
-                        if (lane == 0) atomicMax(amax_s + m0 + j, __float_as_uint(a));
-                    }
-                }
-            }
-        }
-        asm volatile("bar.sync 2, %0;" ::"r"(NF) : "memory");
-        if (ft < 16) {
-            float s = 1.0f, inv = 1.0f;
-            if (ft < M) {
-                if (fuse.static_scale != nullptr) {
-                    s = __ldg(fuse.static_scale);
-                    inv = __fdiv_rn(1.0f, s);
-                } else {
-                    const float amax = __uint_as_float(amax_s[ft]);
-                    if (amax == 0.0f) {
-                    } else if (fuse.scale_mode == W4A8_SCALE_POW2) {
-                        s = pow2_ceil(__fdiv_rn(amax, kE4M3Max));
-                        inv = __fdiv_rn(1.0f, s);
-                    } else {
-                        s = __fdiv_rn(amax, kE4M3Max);
-                        inv = __fdiv_rn(kE4M3Max, amax);
-                    }
-                }
-                if (p == 0 && fuse.s_x_out != nullptr) fuse.s_x_out[ft] = s;
-            }
-            sx_s[ft] = s;
-            inv_s[ft] = inv;
-        }
-        asm volatile("bar.sync 2, %0;" ::"r"(NF) : "memory");
-    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp, one lane issues)
@@ -542,7 +403,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                     kb += ks;
                     r1.advance(S1);
                     ++issued;
-                    if (Cfg::FUSE) continue;       // the dequantization groups make the activation tiles
                     if (st + 1 < ahead) continue;  // still inside the weight-only prologue
                     if (!waited) {
                         ptx::griddep_wait();
@@ -648,7 +508,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         const int r = q * 32 + lane;
         bool ok = true;
         uint32_t acc_phase = 0;
-        ptx::Ring rx;  // ring position of the next activation tile (FUSE)
         // The scales are fetched before the accumulator is waited for (a global load issued after
         // it would add its full latency to the kernel's tail): s_x one or two per lane, broadcast
         // by shuffles later; s_w per row at the top of each range.
@@ -656,12 +515,10 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         const int es = out_dtype == W4A8_OUT_FP32 ? 4 : 2;
         const bool wide_out = (((int64_t)ldy * es) & 15) == 0;  // Y rows 16-byte aligned (y itself is)
         float sx_lane[MT / 32 > 0 ? MT / 32 : 1];
-        if (!Cfg::FUSE) {
-            ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
+        ptx::griddep_wait();  // s_x comes from, and Y may still be read by, earlier kernels
 #pragma unroll
-            for (int c = 0; c < (MT / 32 > 0 ? MT / 32 : 1); ++c)
-                sx_lane[c] = (c * 32 + lane < M) ? __ldg(s_x + c * 32 + lane) : 0.0f;
-        }
+        for (int c = 0; c < (MT / 32 > 0 ? MT / 32 : 1); ++c)
+            sx_lane[c] = (c * 32 + lane < M) ? __ldg(s_x + c * 32 + lane) : 0.0f;
         for (int t = p; t < T && ok; t += P) {
             const TileGeom tg = tile_geom(t);
             const int u0 = tg.u0, u1 = tg.u1, kb0 = tg.kb0, nkb = tg.nkb;
@@ -672,72 +529,6 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
 #pragma unroll
             for (int b = 0; b < 2; ++b)
                 swn[b] = (b < MBLK && b * 128 + r < R) ? __ldg(s_w + (int64_t)(n0 + b * 128 + r) * sw_stride) : 0.0f;
-            if (Cfg::FUSE) {
-                // Eq. 13, second half: these four warps, idle until the accumulator is complete,
-                // convert the activations ahead of the MMAs (thread mapping: XMap).  Each thread
-                // keeps the loads of its next two stages in flight.
-                const XMap xm = x_map(r, M, S1);
-                const bool xrow_ok = xm.xrow < M;
-                const uint4* xbase = reinterpret_cast<const uint4*>(fuse.x + (int64_t)xm.xrow * fuse.ldx + xm.xq * 32);
-                const float inv = inv_s[xm.xrow];
-                const uint32_t xoff = (uint32_t)(xm.xj * (MT * 128) + xm.xrow * 128);
-                const uint32_t sw0 = (uint32_t)(((2 * xm.xq) ^ (xm.xrow & 7)) << 4);
-                const uint32_t sw1 = (uint32_t)(((2 * xm.xq + 1) ^ (xm.xrow & 7)) << 4);
-                auto xload = [&](uint4(&v)[4], int st) {
-                    const int kbk = st * KS + xm.xj;  // 128 BF16 = 16 chunks per k-block
-                    if (xrow_ok && xm.xj < KS && st < nst && kbk < KB) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) v[j] = __ldg(xbase + (int64_t)kbk * 16 + j);
-                    }
-                };
-                // convert stage st from v, refill v with stage st_next, publish the tile part
-                auto xstage = [&](uint4(&v)[4], int st, int st_next, const ptx::Ring& rg) -> bool {
-                    const int kbk = st * KS + xm.xj;
-                    const bool xact = xm.xj < KS && kbk < KB;
-                    uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
-                    if (xact && xrow_ok) {
-                        const uint2 a = quant_bf16x8(v[0], inv), b = quant_bf16x8(v[1], inv);
-                        const uint2 c = quant_bf16x8(v[2], inv), d = quant_bf16x8(v[3], inv);
-                        lo = make_uint4(a.x, a.y, b.x, b.y);
-                        hi = make_uint4(c.x, c.y, d.x, d.y);
-                    }
-                    xload(v, st_next);
-                    if (!ptx::mbar_wait(bar_free10 + 8u * (uint32_t)rg.idx, rg.phase ^ 1u, abort_flag, status_word))
-                        return false;
-                    if (xact) {
-                        if (xrow_ok && p == 0 && fuse.x8_out != nullptr) {
-                            uint4* o = reinterpret_cast<uint4*>(fuse.x8_out + (int64_t)xm.xrow * fuse.ldx8_out +
-                                                                (int64_t)kbk * 128 + xm.xq * 32);
-                            o[0] = lo;
-                            o[1] = hi;
-                        }
-                        // 128-byte swizzle: the 16-byte chunk index is XORed with the row modulo 8
-                        const uint32_t xt = x_ring + (uint32_t)(rg.idx * plan.xstage) + xoff;
-                        ptx::st_shared_v4(xt + sw0, lo);
-                        ptx::st_shared_v4(xt + sw1, hi);
-                    }
-                    ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(bar_xfull0 + 8u * (uint32_t)rg.idx);
-                    return true;
-                };
-                const int span = xm.span;
-                uint4 xw[4];
-                if (!xv_loaded) xload(xv, xm.sub);
-                xv_loaded = false;
-                xload(xw, xm.sub + span);
-                ptx::Ring rg = rx;  // ring position of this thread's next stage
-                for (int i = 0; i < xm.sub; ++i) rg.advance(S1);
-                for (int st = xm.sub; st < nst && ok; st += 2 * span) {
-                    ok = xstage(xv, st, st + 2 * span, rg);
-                    for (int i = 0; i < span; ++i) rg.advance(S1);
-                    if (ok && st + span < nst) {
-                        ok = xstage(xw, st + span, st + 3 * span, rg);
-                        for (int i = 0; i < span; ++i) rg.advance(S1);
-                    }
-                }
-                if (!ok) break;
-                for (int i = 0; i < nst; ++i) rx.advance(S1);
-            }
             ok = ptx::mbar_wait(bar_acc_full, acc_phase, abort_flag, status_word);
             acc_phase ^= 1u;
             if (!ok) break;
@@ -757,7 +548,7 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
                         tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(Cfg::kDCol + b * MT + c0), v);
                     ptx::tmem_ld_wait();
                     if (KSPLIT == 1) {
-                        sn_emit<Cfg>(v, swn[b], b, c0, r, et, R, n0, M, es, wide_out, out_s, y, ldy, sx_lane, sx_s);
+                        sn_emit<Cfg>(v, swn[b], b, c0, r, et, R, n0, M, es, wide_out, out_s, y, ldy, sx_lane);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 16; ++j)

@@ -435,6 +435,30 @@ static bool pair_kernel_applies(int64_t M, int64_t N, int64_t K, int sms) {
     return tiles >= 4 * (int64_t)(sms / 2);
 }
 
+// Tiles of 256 weight rows x 256 tokens (two row blocks per activation tile, whole tiles per CTA)
+// against tiles of 128 x 256: per k-block step about 1060 tensor-pipe cycles for 50 KB from L2 instead
+// of 530 cycles for 41 KB, which the SM's L2 port (about 64 bytes per clock) turns into ~650.  The wide
+// tile cannot be cut along K and its epilogue does not overlap the next tile, so it is used where
+// whole tiles fill the SMs well (measured, us: (2048, 4096, 4096) 34.9 vs 37.7; (4096, 4096, 14336)
+// 203 vs 265; (8192, 28672, 8192) 1785 vs 1906 for the two-CTA kernel) or where a model fitted to
+// such measurements says so ((512, 28672, 4096): 68 vs 87).
+static bool two_block_tiles_apply(int64_t M, int64_t N, int64_t K, int sms) {
+    if (M < 512 || N < 256 || K < 512) return false;
+    const int64_t TM = (M + 255) / 256;
+    const int64_t t2 = TM * ((N + 255) / 256);
+    const int64_t t1 = TM * ((N + 127) / 128);
+    const int64_t KB = K / 128;
+    const int64_t rounds2 = (t2 + sms - 1) / sms;
+    if (5 * t2 >= 4 * rounds2 * sms) return true;   // at least 80 % of the tile slots of its rounds are used
+    // microseconds: 0.857 per k-block step + 3.9 per tile for the wide tile; 0.61 per unit for the
+    // 128-row tile (0.573 in the two-CTA kernel, 0.85 with at most two token tiles, where every
+    // weight tile comes from HBM and four ring stages do not cover that latency)
+    const double per_unit = pair_kernel_applies(M, N, K, sms) ? 0.573 : (TM <= 2 ? 0.85 : 0.61);
+    const double c2 = (double)rounds2 * ((double)KB * 0.857 + 3.9);
+    const double c1 = (double)((t1 * KB + sms - 1) / sms) * per_unit;
+    return c2 < c1;
+}
+
 template <class Cfg>
 static int launch_pair(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, const float* s_x, const float* s_w,
                        int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, int sms,
@@ -516,6 +540,27 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     if (rc != W4A8_OK) return rc;
     const int sms = sm_count();
     if (sms <= 0) return W4A8_ERR_CUDA;
+    if (two_block_tiles_apply(M, N, K, sms)) {
+        // tiles of 256 weight rows x 256 tokens, whole tiles per CTA
+        SkPlan p2;
+        p2.bnx = 256;
+        p2.TM = (int)((M + 255) / 256);
+        p2.TN = (int)((N + 255) / 256);
+        p2.aligned = 1;
+        p2.U = (int64_t)p2.TM * p2.TN * (K / 128);
+        p2.P = (int64_t)p2.TM * p2.TN < sms ? (int64_t)p2.TM * p2.TN : sms;
+        p2.counter_bytes = 0;
+        p2.workspace_bytes = 0;
+        CUtensorMap tx2;
+        if (!make_tmap_u8_2d(&tx2, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, 256, CU_TENSOR_MAP_SWIZZLE_128B))
+            return W4A8_ERR_CUDA;
+        return fmt == kFmtTiledSignMag
+                   ? launch_streamk<SkCfg<256, 3, 3, 2, kFmtTiledSignMag, 2>>(tx2, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                             out_dtype, workspace, p2, (int)M, (int)N,
+                                                                             (int)K, st)
+                   : launch_streamk<SkCfg<256, 3, 3, 2, kFmtTiled, 2>>(tx2, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                                                      workspace, p2, (int)M, (int)N, (int)K, st);
+    }
     if (pair_kernel_applies(M, N, K, sms))
         return fmt == kFmtTiledSignMag
                    ? launch_pair<PairCfg<4, 6, 4, kFmtTiledSignMag>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,

@@ -19,6 +19,15 @@
 // the codes to E4M3 (Eq. 10) into a ring of swizzled shared-memory tiles; one thread issues the
 // tcgen05 kind::f8f6f4 MMAs (weights on the M side, tokens on the N side); accumulators are
 // double-buffered in tensor memory so the epilogue warps overlap the next tile's main loop.
+//
+// RB = 2 (whole tiles only): a tile is 256 weight rows x 256 tokens -- two 128-row blocks against one
+// activation tile per k-block, two accumulators of 256 columns (all of tensor memory, so the
+// epilogue of a tile no longer overlaps the next tile).  A k-block step then brings 18 KB of packed
+// weights + 32 KB of activations for eight MMAs (about 1060 tensor-pipe cycles) instead of 9 + 32 KB
+// for four: the activation bytes an SM pulls from L2 per flop are halved, and the SM's L2 port
+// (about 64 bytes per clock) no longer sets the pace.  Measured on (2048, 4096, 4096), per CTA:
+// 32 steps in 41.9 k cycles, of which the MMA warp waits 2.2 k for the first operands, 2.6 k for
+// activation tiles and 3.3 k for expanded weights; the rest is the tensor pipe itself.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -29,7 +38,7 @@
 namespace w4a8 {
 
 
-template <int BNX_, int G_, int S1_, int S2_, int FMT_>
+template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1>
 struct SkCfg {
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
     static constexpr int G = G_;       // dequantization groups of 4 warps
@@ -37,16 +46,19 @@ struct SkCfg {
     static constexpr int S2 = S2_;     // ring of dequantized E4M3 weight tiles
     static constexpr int FMT = FMT_;
     static constexpr int kMeta = meta_bytes(FMT);
-    static constexpr int kWStage = 9216;  // 128 rows x (64 code bytes + meta), padded to keep the activation tile 1024-aligned
+    static constexpr int RB = RB_;     // 128-row blocks per tile
+    static constexpr int kCodeBytes = RB_ * 8192;   // packed codes of the tile's rows for one k-block
+    static constexpr int kWStage = RB_ * 9216;  // rows x (64 code bytes + meta), padded to keep the activation tile 1024-aligned
     static constexpr int kXBytes = BNX * 128;
     static constexpr int kStage1 = kWStage + kXBytes;
-    static constexpr int kW8Bytes = 128 * 128;
+    static constexpr int kW8Bytes = RB_ * 128 * 128;
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + 1024;
-    static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;
+    static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;   // RB = 1: two accumulators (double buffer); RB = 2: one per row block
     static constexpr int kThreads = 32 * (10 + 4 * G);
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
+    static_assert(RB_ == 1 || (RB_ == 2 && BNX_ == 256), "two row blocks per tile only with 256-token tiles");
     // A dequantization group handles every G-th stage, so it skips phases of the barriers it
     // waits on, and an mbarrier wait tells phases apart by parity only: the wait for use k of a
     // slot is sound only if use k-1 has completed before it starts.  That holds because a stage's
@@ -57,6 +69,10 @@ struct SkCfg {
     // a "slot free" barrier and overwrote an expanded tile still in use; with G == S2 and
     // S1 % G == 0 it was sound but no faster.)
     static_assert(S1 <= 2 * S2, "ring depths: see the comment above");
+    // The same parity argument for the "packed weights landed" barriers: a group that has finished
+    // stage i next waits for stage i + G in ring slot (i + G) % S1, whose previous use is stage
+    // i + G - S1; that one has landed for sure only if it is not later than stage i itself.
+    static_assert(G_ <= S1_, "a group must not run ahead of the TMA ring by more than one round");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
     static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
@@ -69,7 +85,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                       const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                       void* __restrict__ y, int64_t ldy, int out_dtype, unsigned int* counters,
                       float* slots, int M, int N, int K, int TM, int TN, int aligned, unsigned int* status_word) {
-    constexpr int BNX = Cfg::BNX, G = Cfg::G, S1 = Cfg::S1, S2 = Cfg::S2;
+    constexpr int BNX = Cfg::BNX, G = Cfg::G, S1 = Cfg::S1, S2 = Cfg::S2, RB = Cfg::RB;
+    constexpr int TR = 128 * RB;   // weight rows per tile
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -158,8 +175,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             for (int it = 0; it < n_it; ++it) {
                 ok = ptx::mbar_wait(bar_free1(r1.idx), r1.phase ^ 1u, abort_flag, status_word);
                 if (!ok) break;
-                const int rows = (N - nt * 128) < 128 ? (N - nt * 128) : 128;  // ragged last tile
-                const int64_t row0 = (int64_t)kb * N + (int64_t)nt * 128;
+                const int rows = (N - nt * TR) < TR ? (N - nt * TR) : TR;  // ragged last tile
+                const int64_t row0 = (int64_t)kb * N + (int64_t)nt * TR;
                 const uint32_t full = bar_full(r1.idx), wdst = stage_w(r1.idx);
                 const uint8_t* csrc = wpp + row0 * kRowCodeBytes;
                 const uint8_t* msrc = meta_base + row0 * Cfg::kMeta;
@@ -167,7 +184,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 if (ptx::elect_one()) {
                     ptx::mbar_arrive_expect_tx(full, cbytes + mbytes);
                     ptx::bulk_load(wdst, csrc, cbytes, full);
-                    ptx::bulk_load(wdst + 8192u, msrc, mbytes, full);
+                    ptx::bulk_load(wdst + (uint32_t)Cfg::kCodeBytes, msrc, mbytes, full);
                 }
                 r1.advance(S1);
                 ++issued;
@@ -228,9 +245,11 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 const int64_t tile = u / KB;
                 const int kb0 = (int)(u - tile * KB);
                 const int len = (int)((u_end - u) < (int64_t)(KB - kb0) ? (u_end - u) : (int64_t)(KB - kb0));
-                const int buf = j & 1;
-                if (j >= 2) {
-                    ok = ptx::mbar_wait(bar_acc_empty(buf), (uint32_t)(((j >> 1) - 1) & 1), abort_flag, status_word);
+                // RB = 1: two accumulators used in turn; RB = 2: both belong to the one tile in flight
+                const int buf = RB == 1 ? (j & 1) : 0;
+                if (RB == 1 ? j >= 2 : j >= 1) {
+                    const uint32_t par = RB == 1 ? (uint32_t)(((j >> 1) - 1) & 1) : (uint32_t)((j - 1) & 1);
+                    ok = ptx::mbar_wait(bar_acc_empty(buf), par, abort_flag, status_word);
                     if (!ok) break;
                 }
                 const uint32_t tmem_acc = tmem_base + (uint32_t)(buf * BNX);
@@ -245,6 +264,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     const uint32_t f1 = bar_free1(r1.idx), f2 = bar_free2(r2.idx);
                     if (ptx::elect_one()) {
                         ptx::umma_f8_kblock(tmem_acc, a_lo, b_lo, idesc, accumulate);
+                        if (RB == 2) ptx::umma_f8_kblock(tmem_acc + (uint32_t)BNX, a_lo + (16384u >> 4), b_lo, idesc, accumulate);
                         ptx::umma_commit(f1);
                         ptx::umma_commit(f2);
                     }
@@ -294,11 +314,13 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             const int kb0 = (int)(u - tile * KB);
             const int len = (int)((u_end - u) < (int64_t)(KB - kb0) ? (u_end - u) : (int64_t)(KB - kb0));
             const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
-            const int n = nt * 128 + r, m0 = mt * BNX + half * kHalfCols;
-            const bool row_ok = n < N;
-            const int buf = j & 1;
+            const int m0 = mt * BNX + half * kHalfCols;
+            const int buf = RB == 1 ? (j & 1) : 0;
             const bool whole = (len == KB);
-            const float swn = row_ok ? __ldg(s_w + (int64_t)n * sw_stride) : 0.0f;
+            float swn_rb[RB];
+#pragma unroll
+            for (int b = 0; b < RB; ++b)
+                swn_rb[b] = (nt * TR + b * 128 + r < N) ? __ldg(s_w + (int64_t)(nt * TR + b * 128 + r) * sw_stride) : 0.0f;
             // Activation scales of this warp's columns, one per lane and 32 columns, fetched before
             // the accumulator is ready and broadcast by shuffles later: global loads issued inside
             // the store loop queue behind the operand traffic of the main loop.
@@ -306,16 +328,22 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
 #pragma unroll
             for (int c = 0; c < kHalfCols / 32; ++c)
                 sx_pre[c] = (m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f;
-            ok = ptx::mbar_wait(bar_acc_full(buf), (uint32_t)((j >> 1) & 1), abort_flag, status_word);
+            ok = ptx::mbar_wait(bar_acc_full(buf), RB == 1 ? (uint32_t)((j >> 1) & 1) : (uint32_t)(j & 1), abort_flag, status_word);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            const uint32_t tmem_acc =
+            const uint32_t tmem_acc0 =
                 tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BNX + half * kHalfCols);
             // The CTA's first segment uses slot 0, a later (necessarily last) one slot 1.
             float* my_slot = slots + ((int64_t)p * 2 + (j == 0 ? 0 : 1)) * Cfg::kSlotFloats +
                              (int64_t)half * kHalfCols * 128;
 #pragma unroll 1
-            for (int c0 = 0; c0 < kHalfCols; c0 += 16) {
+            for (int cb = 0; cb < RB * kHalfCols; cb += 16) {
+                // (RB = 2: the second row block's accumulator sits BNX columns further)
+                const int b = cb / kHalfCols, c0 = cb - b * kHalfCols;
+                const int n = nt * TR + b * 128 + r;
+                const bool row_ok = n < N;
+                const float swn = b == 0 ? swn_rb[0] : swn_rb[RB - 1];
+                const uint32_t tmem_acc = tmem_acc0 + (uint32_t)(b * BNX);
                 uint32_t v[16];
                 ptx::tmem_ld_32x32b_x16(tmem_acc + (uint32_t)c0, v);
                 ptx::tmem_ld_wait();
@@ -377,9 +405,11 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
-            dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + tiled_row_offset(r),
-                                          stage_w(s1) + 8192u + (uint32_t)(r * Cfg::kMeta), r,
-                                          stage_w8(s2) + (uint32_t)r * 128u);
+#pragma unroll
+            for (int b = 0; b < RB; ++b)
+                dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + tiled_row_offset(b * 128 + r),
+                                              stage_w(s1) + (uint32_t)Cfg::kCodeBytes + (uint32_t)((b * 128 + r) * Cfg::kMeta), r,
+                                              stage_w8(s2) + (uint32_t)(b * 16384) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
         }

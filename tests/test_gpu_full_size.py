@@ -186,3 +186,44 @@ def test_two_cta_kernel_shape_exact_integers_and_gaussian():
         else:
             worst, _ = fp32_gate(got, ref["y64"], rel=2e-3)
             assert worst <= 2e-3, worst
+
+
+def test_wide_tile_kernel_shape_exact_integers_and_gaussian():
+    """A shape that the prefill kernel with tiles of 256 output channels x 256 tokens takes (whole
+    tiles fill the SMs well), ragged in both directions -- the last token tile has 120 tokens, the
+    last channel tile 80 rows -- and with more tiles than SMs, so that some CTAs run a second tile
+    on the same accumulators.  Small-integer inputs (exact FP32 sums: a misplaced operand changes a
+    result by at least one unit) in the generic tiled format, then Gaussian inputs in the
+    sign-magnitude format within the usual gates.  Sampled output channels: the first and last row of
+    every 128-row block."""
+    M, N, K = 1400, 10576, 640
+    rng = np.random.default_rng(31)
+    cols = np.unique(np.concatenate([rng.integers(0, N, 500), np.arange(0, N, 128), np.arange(127, N, 128),
+                                     np.array([N - 81, N - 80, N - 1])]))
+    for exact in (True, False):
+        if exact:
+            codes, gscale, gzero = inputs.random_codes(N, K, 7, scale_bits=0x3F80)       # group scale 1.0
+            s_w = np.array([1.0], dtype=np.float32)
+            xb = inputs.make_small_int_activation(M, K, 8)
+        else:
+            W = inputs.make_weight(N, K, 0.02, 33)
+            codes, gscale, gzero, s_w = oracle.quantize_weight_rtn(W, symmetric=True)
+            xb = inputs.make_activation(M, K, 34, 0.01, 20.0)
+        x8_ref, s_x_ref = oracle.quantize_act(xb)
+        w8 = oracle.dequant_weight(codes, gscale, gzero)
+        ref = oracle.linear(x8_ref, s_x_ref, w8, s_w, cols=cols, want=("y64",))
+        fmt = binding.FMT_TILED if exact else binding.FMT_TILED_SIGNMAG
+        tw = binding.prepack_weight(*weights_to_dev(codes, gscale, gzero, s_w), weight_format=fmt)
+        x8, s_x = binding.quantize_act(bf16_dev(xb))
+        y = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32)
+        yb = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_BF16)
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0
+        got = y.cpu().numpy()[:, cols]
+        if exact:
+            assert np.all(np.abs(got.astype(np.float64) - ref["y64"]) <= 4e-7 * np.abs(ref["y64"]) + 1e-6)
+        else:
+            worst, _ = fp32_gate(got, ref["y64"], rel=2e-3)
+            assert worst <= 2e-3, worst
+            ok, dist = bf16_gate(bf16_bits(yb)[:, cols], ref["y64"])
+            assert ok, dist

@@ -317,8 +317,11 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan
     // expansion work then covers 128 useful rows instead of a sliver, and its K walk is shorter;
     // the price is a small fix-up through the workspace.
     const int64_t blocks128 = (N + 127) / 128;
-    // (With 64-token tiles the partial sums are four times larger: only worth it for a long K.)
-    if (may_split_k && blocks128 * 2 <= sms && KB >= (Cfg::MT > 16 ? 64 : 8)) {
+    // (With 64- and 128-token tiles the partial sums are four and eight times larger: only worth
+    // it for a long K; with 64 tokens also from K = 4096 on when at most a quarter of the SMs would
+    // otherwise get a 128-row block -- o projection at M = 32: 10.9 against 14.6 us.)
+    const int64_t kb_min = Cfg::MT == 16 ? 8 : (Cfg::MT == 64 && blocks128 * 4 <= sms ? 32 : 64);
+    if (may_split_k && blocks128 * 2 <= sms && KB >= kb_min) {
         int64_t ks = sms / blocks128;
         if (ks > KB / 4) ks = KB / 4;  // at least four k-blocks per chunk
         if (ks > 1 && blocks128 <= (int64_t)(kSnCounterBytes / sizeof(unsigned int)) &&

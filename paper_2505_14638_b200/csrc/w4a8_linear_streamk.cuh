@@ -428,11 +428,21 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     ptx::griddep_wait();
     const int n_shared = (int)share_slot[0];
     unsigned int* done = counters + (int64_t)TM * TN;  // second counter per tile: finished reducers
+    // Slot index of every contributor of the tile, worked out once (64-bit divisions: left inside
+    // the adding loop they cost every thread more than the loads did).  The rings are idle by now.
+    int* slot_of = reinterpret_cast<int*>(sm);
     for (int k = 0; k < n_shared; ++k) {
         const int64_t tile = (int64_t)share_slot[1 + k];
         const int64_t p_lo = ((tile * KB + 1) * P - 1) / U;  // first and last contributor
         const int64_t p_hi = (((tile + 1) * KB) * P - 1) / U;
         const int C = (int)(p_hi - p_lo) + 1, me = (int)(p - p_lo);
+        __syncthreads();  // readers of the previous tile's table are done
+        for (int i = (int)threadIdx.x; i < C; i += Cfg::kThreads) {
+            // contributor q's slot for this tile: its first slot if the tile is where its share begins, else its second
+            const int64_t q = p_lo + i;
+            const int64_t first_tile = (q * U / P) / KB;
+            slot_of[i] = (int)(q * 2 + (tile == first_tile ? 0 : 1));
+        }
         if (threadIdx.x == 0 && *abort_flag == 0u) {
             // bounded wait for the C arrivals
             uint64_t t0 = 0;
@@ -462,11 +472,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         for (int e0 = (int)threadIdx.x; e0 < total; e0 += 4 * Cfg::kThreads) {
             float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll 4
-            for (int64_t q = p_lo; q <= p_hi; ++q) {
-                // slot of contributor q for this tile: its first slot if the tile is where its
-                // share begins, else its second
-                const int64_t first_tile = (q * U / P) / KB;
-                const float* sl = slots + (q * 2 + (tile == first_tile ? 0 : 1)) * Cfg::kSlotFloats + c_lo * 128;
+            for (int i = 0; i < C; ++i) {
+                const float* sl = slots + (int64_t)slot_of[i] * Cfg::kSlotFloats + c_lo * 128;
 #pragma unroll
                 for (int jj = 0; jj < 4; ++jj) {
                     const int e = e0 + jj * Cfg::kThreads;

@@ -268,10 +268,10 @@ def run_ours(args, rank, world, local_rank):
     for m in SWEEP_M:
         xb = inputs.make_activation(m, K, 1000 * rank + m, OUTLIER_FRAC, OUTLIER_MULT)
         t = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
-        x_host[m] = t.pin_memory()
+        x_host[m] = t
         xs[m] = t.to(dev)
         ys[m] = torch.empty((m, N), dtype=torch.bfloat16, device=dev)
-        y_host[m] = torch.empty((m, N), dtype=torch.bfloat16).pin_memory()
+        y_host[m] = [torch.empty((m, N), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     torch.cuda.synchronize()
 
     # ---- the step: one pass of the whole path (Eq. 13 quantization, Eq. 10 expansion, FP8 MMAs,
@@ -281,13 +281,19 @@ def run_ours(args, rank, world, local_rank):
     spl = max(1, min(args.steps_per_launch, binding.CHAIN_MAX_PROBLEMS // len(SWEEP_M)))
     workspace = [None]
 
-    def make_launch(first_step, nsteps, host_buffers=False):
+    def make_launch(first_step, nsteps, host_buffers=None):
         probs = []
         for s_ in range(nsteps):
             for i, m in enumerate(SWEEP_M):
                 c = ((first_step + s_) * len(SWEEP_M) + i) % WEIGHT_COPIES
-                probs.append(dict(x=x_host[m] if host_buffers else xs[m], weight=weights[c],
-                                  y=y_host[m] if host_buffers else ys[m]))
+                if host_buffers is None:
+                    x_, y_ = xs[m], ys[m]
+                else:
+                    # this step's rows of the staging buffer that the call's one host-to-device copy fills;
+                    # the results go straight to pinned host memory
+                    x_ = x_stage[host_buffers][s_, row0[m]:row0[m] + m]
+                    y_ = y_host[m][host_buffers]
+                probs.append(dict(x=x_, weight=weights[c], y=y_))
         ch = binding.LinearChain(probs, workspace=workspace[0])
         if workspace[0] is None or ch.ws.numel() > workspace[0].numel():
             workspace[0] = ch.ws
@@ -342,33 +348,68 @@ def run_ours(args, rank, world, local_rank):
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set during the timed region")
 
-    # ---- end to end: the same call with HOST buffers -- the activations of every step are read from
-    # pinned host memory and every step's result is written to pinned host memory inside the timed
-    # region (by the kernel itself, over the bus), the caller synchronises after every call ----
-    e2e_launch = make_launch(0, spl, host_buffers=True)
-    e2e_tail = make_launch(n_full * spl, n_tail, host_buffers=True) if n_tail else None
+    # ---- end to end: host buffers in and out.  Every step's activations sit in pinned host memory
+    # and are brought to the device inside the timed region, one asynchronous copy per call (all
+    # the steps of the call) on a copy stream; every step's result is written to pinned host memory
+    # by the kernel itself, over the bus.  Two sets of buffers: the copy for call i + 1 runs while
+    # call i computes, and the caller waits for call i's event (and reads its results) after it
+    # has issued call i + 1.  (A kernel that reads its activations from host memory directly takes
+    # 60-75 us longer per call: loads issued by SMs fetch 1.4 MB over the bus far more slowly than
+    # the copy engine does; stores to host memory cost nothing measurable.)  Also measured: a full
+    # stop after every call. ----
+    rows_per_step = sum(SWEEP_M)
+    row0, acc = {}, 0
+    for m in SWEEP_M:
+        row0[m] = acc
+        acc += m
+    x_pin, x_stage = [], []
+    for par in range(2):
+        hp = torch.empty((spl, rows_per_step, K), dtype=torch.bfloat16).pin_memory()
+        for m in SWEEP_M:
+            hp[:, row0[m]:row0[m] + m] = x_host[m]
+        x_pin.append(hp)
+        x_stage.append(torch.empty((spl, rows_per_step, K), dtype=torch.bfloat16, device=dev))
+    e2e_calls = [make_launch(g * spl, spl, host_buffers=g % 2) for g in range(min(2, max(n_full, 1)))]
+    e2e_tail = make_launch(n_full * spl, n_tail, host_buffers=n_full % 2) if n_tail else None
+    seq = [(e2e_calls[g % len(e2e_calls)], g % 2, spl) for g in range(n_full)]
+    if e2e_tail is not None:
+        seq.append((e2e_tail, n_full % 2, n_tail))
+    copy_stream = torch.cuda.Stream(device=dev)
+    copied = [torch.cuda.Event() for _ in seq]
+    done = [torch.cuda.Event() for _ in seq]
 
-    def e2e_pass():
-        for _ in range(n_full):
-            e2e_launch()
-            torch.cuda.current_stream().synchronize()   # the caller reads the results
-        if e2e_tail is not None:
-            e2e_tail()
-            torch.cuda.current_stream().synchronize()
+    def e2e_pass(overlap):
+        main = torch.cuda.current_stream()
+        for i, (call, par, nsteps) in enumerate(seq):
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(done[i - 2])      # the call that read this staging buffer last
+                x_stage[par][:nsteps].copy_(x_pin[par][:nsteps], non_blocking=True)
+                copied[i].record()
+            main.wait_event(copied[i])
+            call()
+            done[i].record()
+            if not overlap:
+                done[i].synchronize()           # the caller reads this call's results
+            elif i > 0:
+                done[i - 1].synchronize()       # the caller reads the previous call's results
+        done[-1].synchronize()
 
-    for _ in range(2):
-        e2e_launch()
-    barrier()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record()
-    e2e_pass()
-    g1.record()
-    barrier()
-    ms_e2e = g0.elapsed_time(g1)
+    ms_e2e_by_mode = {}
+    for overlap in (False, True):
+        e2e_pass(True)
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        e2e_pass(overlap)
+        g1.record()
+        barrier()
+        ms_e2e_by_mode[overlap] = g0.elapsed_time(g1)
+    ms_e2e, ms_e2e_stop = ms_e2e_by_mode[True], ms_e2e_by_mode[False]
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set during the end-to-end region")
 
-    ms_total, ms_e2e, launch_ms = max_over_ranks([ms_total, ms_e2e, launch_ms], dist, dev)
+    ms_total, ms_e2e, ms_e2e_stop, launch_ms = max_over_ranks([ms_total, ms_e2e, ms_e2e_stop, launch_ms], dist, dev)
 
     if rank != 0:
         if dist is not None:
@@ -397,8 +438,10 @@ def run_ours(args, rank, world, local_rank):
                 "h2d_bytes_per_step": sum(m * K * 2 for m in SWEEP_M),
                 "d2h_bytes_per_step": sum(m * N * 2 for m in SWEEP_M),
                 "ms_per_step": ms_e2e / args.steps,
-                "how": "w4a8_linear_chain on pinned host activations and outputs (read and written over the bus by "
-                       "the kernel), one call and one stream synchronisation per %d steps" % spl},
+                "ms_per_step_full_stop_after_every_call": ms_e2e_stop / args.steps,
+                "how": "per call of %d steps: one asynchronous copy of the steps' activations from pinned host memory "
+                       "(copy stream), w4a8_linear_chain writing every step's result to pinned host memory over the "
+                       "bus; two sets of buffers, the caller waits for a call's event after issuing the next call" % spl},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "linear_chain_kernel (w4a8_linear_chain), %d problems per launch: "
                                "M in {1,4,16} x %d" % (spl * len(SWEEP_M), spl),
@@ -687,9 +730,11 @@ def mlp_sweep(torch, binding, inputs, dev, peaks):
     """The MLP block of a Llama-3-8B decoder layer at decode sizes, all on the W4A8 path:
     quantize_act(x) -> stacked gate/up projection (K = 4096 -> N = 2 x 14336) -> silu(gate) * up fused
     with the activation quantization of the next layer (w4a8_silu_mul_quantize) -> down projection
-    (K = 14336 -> N = 4096).  Per token count: the block time from CUDA graphs of consecutive blocks
-    on rotating weight copies (more than twice the L2), the same block with the activation written as
-    BF16 and quantized by a separate launch, and the BF16 library block (two torch.matmul + silu * mul)."""
+    (K = 14336 -> N = 4096).  Per token count: the block as two dependent problems of a w4a8_linear_chain
+    launch (eight blocks per launch), the block time of the per-launch kernels from CUDA graphs of
+    consecutive blocks on rotating weight copies (more than twice the L2), the same with the activation
+    written as BF16 and quantized by a separate launch, and the BF16 library block (two torch.matmul +
+    silu * mul)."""
     H, F = 4096, 14336
     out = []
     side = torch.cuda.Stream()
@@ -746,13 +791,29 @@ def mlp_sweep(torch, binding, inputs, dev, peaks):
             g2 = torch.matmul(x, wg_bf.t())
             torch.matmul(torch.nn.functional.silu(g2[:, :F]) * g2[:, F:], wd_bf.t())
 
+        # The same blocks as ONE w4a8_linear_chain launch: per block a gate/up problem and a down
+        # problem of the gated kind that depends on it (Eq. 13 of silu(gate) * up inside the kernel);
+        # every block of the launch has its own gate/up buffer, because a CTA that is ahead may write
+        # the next block's while another still reads this one's.
+        nblk = 2 * copies
+        gus_out = [torch.empty((m, 2 * F), dtype=torch.bfloat16, device=dev) for _ in range(nblk)]
+        probs = []
+        for b in range(nblk):
+            probs.append(dict(x=x, weight=gus[b % copies], y=gus_out[b]))
+            probs.append(dict(x=gus_out[b], weight=downs[b % copies], y=y, kind=binding.CHAIN_INPUT_SILU_MUL,
+                              depends_on=2 * b))
+        chain = binding.LinearChain(probs)
+        t_c = _time_loop(torch, chain, 10, warm=3) / nblk
+
         t = graph_time(block, 2 * copies)
         t_u = graph_time(block_unfused, 2 * copies)
         t_b = graph_time(block_bf16, 4)
         if binding.query_device_status() != 0:
             raise RuntimeError("device status word set")
-        out.append({"M": m, "block_us": t * 1e6, "block_unfused_activation_us": t_u * 1e6,
-                    "weight_GBps": wbytes / t / 1e9, "frac_hbm_measured": wbytes / t / 1e9 / peaks["hbm_gbs"],
+        out.append({"M": m, "block_chain_us": t_c * 1e6, "block_per_launch_us": t * 1e6,
+                    "block_unfused_activation_us": t_u * 1e6,
+                    "chain_weight_GBps": wbytes / t_c / 1e9, "chain_frac_hbm_measured": wbytes / t_c / 1e9 / peaks["hbm_gbs"],
+                    "per_launch_frac_hbm_measured": wbytes / t / 1e9 / peaks["hbm_gbs"],
                     "library_bf16_block_us": t_b * 1e6})
     return out
 

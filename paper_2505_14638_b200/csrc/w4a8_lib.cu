@@ -964,6 +964,7 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
     prm.count = count;
     prm.wait_limit_ns = ptx::kWaitLimitNs;
     int stash = 8192, jobs = 0, rot = 0;
+    bool full = false;   // some problem is of the gated kind or has its rows quantized in chunks by several CTAs
     size_t off = kChainHeaderBytes;
     for (int i = 0; i < count; ++i) {
         const w4a8_chain_problem& q = pr[i];
@@ -991,8 +992,16 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
         d.rounds = blocks / sms;
         if ((d.rounds + 1) / 2 + 2 > kChainMaxSegs) return W4A8_ERR_BAD_SHAPE;   // more whole blocks per CTA than the segment table holds
         d.rem_blocks = blocks - d.rounds * sms;
+        // rows of 4096 elements and more are cut into chunks of about 4096 (2048 for the gated kind:
+        // silu costs far more per element than a load) quantized by different CTAs, if there is a
+        // CTA for every chunk of every row
+        // (the kernel with this in it is instantiated for the default number of expansion groups only)
+        const int chunk = d.kind == kChainKindSiluMul ? 2048 : 4096;
+        d.nch = (groups == 0 || groups == 4) ? (d.K + chunk - 1) / chunk : 1;
+        while (d.nch > 1 && d.M * d.nch > sms) --d.nch;
+        if (d.nch > 1 || d.kind == kChainKindSiluMul) full = true;
         d.job_base = jobs;
-        jobs += d.M;
+        jobs += d.M * d.nch;
         d.rem_rot = rot % sms;
         rot += chain_rem_ctas(d, sms);
         d.x8_off = (uint32_t)off;
@@ -1019,6 +1028,9 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
 #define W4A8_CHAIN(GG)                                                                             \
     (fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<GG, kFmtTiledSignMag>>(prm, sms, smem, ws, st) \
                              : launch_chain<ChainCfg<GG, kFmtTiled>>(prm, sms, smem, ws, st))
+    if (groups == 4 && !full)
+        return fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<4, kFmtTiledSignMag, false>>(prm, sms, smem, ws, st)
+                                       : launch_chain<ChainCfg<4, kFmtTiled, false>>(prm, sms, smem, ws, st);
     switch (groups) {
         case 2: return W4A8_CHAIN(2);
         case 3: return W4A8_CHAIN(3);

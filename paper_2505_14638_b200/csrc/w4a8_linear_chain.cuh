@@ -72,7 +72,8 @@ struct ChainProblem {
     int rounds;                 // whole blocks per CTA: CTA p owns blocks [p * rounds, (p + 1) * rounds)
     int rem_blocks;             // blocks behind them, cut along K into runs of (block, k-block) items
     int rem_rot;                // the runs go to CTAs rem_rot, rem_rot + 1, ... (mod P): a different set for every problem
-    int job_base;               // the quantization of row m runs on CTA (job_base + m) % gridDim.x
+    int job_base;               // quantization job t = m * nch + c (row m, chunk c) runs on CTA (job_base + t) % gridDim.x
+    int nch;                    // chunks a row is cut into for its quantization (1: a CTA takes a whole row)
     uint32_t x8_off;            // byte offsets into the workspace: FP8 activation tiles,
     uint32_t part_off;          //   partial-sum slots (one per CTA, M x 96 floats),
     uint32_t cnt_off;           //   arrival counters of the blocks that are cut along K
@@ -97,14 +98,24 @@ struct ChainCtl {
 };
 constexpr size_t kChainCtlBytes = 1024;
 constexpr size_t kChainScaleBytes = (size_t)kChainMaxProblems * kChainMaxM * sizeof(float);
-constexpr size_t kChainHeaderBytes = kChainCtlBytes + 2048;   // control block, activation scales
-static_assert(sizeof(ChainCtl) <= kChainCtlBytes && kChainScaleBytes <= 2048, "workspace header");
+// header: control block, then per (problem, token): activation scale, row maximum under construction
+// (float bits, combined with atomicMax by the CTAs that share a row) and the count of chunks whose
+// maximum is in
+constexpr size_t kChainHeaderBytes = 6144;
+static_assert(sizeof(ChainCtl) <= kChainCtlBytes && kChainCtlBytes + 3 * kChainScaleBytes <= kChainHeaderBytes,
+              "workspace header");
 constexpr int kChainXTileBytes = kChainMaxM * 128;            // one k-block of FP8 activations: 16 tokens x 128 bytes
 
-template <int G_, int FMT_>
+template <int G_, int FMT_, bool FULL_ = true>
 struct ChainCfg {
     static constexpr int G = G_;          // expansion groups (three warps each: lane quarters 0..2)
     static constexpr int FMT = FMT_;
+    // FULL: the gated input kind, and rows cut into chunks that several CTAs quantize
+    // (ChainProblem::nch > 1).  Launches that need neither run an instantiation without that code:
+    // compiled into the one kernel, the extra code of the quantization jobs cost them 2 % (measured;
+    // the roles of a CTA share the instruction caches).
+    static constexpr bool kFull = FULL_;
+    static constexpr bool kChunk = FULL_;
     static constexpr int kS1Max = 16;     // weight ring (runtime depth <= this)
     static constexpr int kS2 = 7;         // stages of expanded weights in tensor memory = activation-tile slots
     static constexpr int kMeta = meta_bytes(FMT_);
@@ -344,7 +355,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
     constexpr int kNumBars = 2 * S1M + 2 * S2 + 5;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    float* red_s = reinterpret_cast<float*>(const_cast<uint32_t*>(tmem_slot) + 4);   // [4] warp maxima of a quantization job
+    float* red_s = reinterpret_cast<float*>(const_cast<uint32_t*>(tmem_slot) + 4);   // [4] warp maxima of a quantization job, [1] the row's maximum
     // This CTA's segments of every problem, worked out once (the partition needs 64-bit divisions,
     // which cost a single warp microseconds per problem if every role repeats them).
     const ChainSeg* seg_tab = reinterpret_cast<const ChainSeg*>(sm + bars_off + Cfg::kBarBytes);   // [problem][kChainMaxSegs]
@@ -352,6 +363,8 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
 
     ChainCtl* const ctl = reinterpret_cast<ChainCtl*>(ws);
     float* const sx_ws = reinterpret_cast<float*>(ws + kChainCtlBytes);      // [problem][16] activation scales
+    unsigned int* const amax_ws = reinterpret_cast<unsigned int*>(ws + kChainCtlBytes + kChainScaleBytes);       // [problem][16]
+    unsigned int* const qcnt_ws = reinterpret_cast<unsigned int*>(ws + kChainCtlBytes + 2 * kChainScaleBytes);   // [problem][16]
     unsigned int* const gabort = &ctl->abort;
     const unsigned long long limit = prm.wait_limit_ns;
 
@@ -536,7 +549,9 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             const int nseg = nseg_tab[i];
             if (nseg == 0) continue;
             // the problem's activations must have been quantized (by the epilogue warps of M CTAs)
-            if (lane == 0) ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit);
+            if (lane == 0)
+                ok = chain_poll_ge(&ctl->xready[i], (unsigned)(Cfg::kChunk ? q.M * q.nch : q.M), gabort, abort_flag,
+                                   status_word, limit);
             ok = warp_all(ok);
             __syncwarp();
             if (!ok) break;
@@ -590,9 +605,15 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
         bool ok = true;
         ptx::griddep_wait();
 
-        // Eq. 13 for row m of problem j (one row per CTA): absmax, scale, FP8 codes written as
-        // operand tiles into the workspace, then published.  Called by all 128 threads.
-        auto quant_job = [&](int j, int m) -> bool {
+        // Eq. 13 for chunk c of row m of problem j: absmax, scale, FP8 codes written as operand tiles
+        // into the workspace, then published.  A row is one chunk, or -- long rows, above all the
+        // gated kind, whose silu costs the 128 threads of a lone CTA tens of microseconds -- nch
+        // chunks on nch CTAs, which combine their maxima through the workspace (atomicMax on the
+        // float bits, a count of the chunks that are in, one bounded poll) before any of them
+        // converts.  That wait cannot deadlock: a chunk's maximum is published before anything is
+        // waited for, and every CTA reaches the jobs of a problem in the same order.  Called by all
+        // 128 threads.
+        auto quant_job = [&](int j, int m, int c) -> bool {
             const ChainProblem& q = prm.prob[j];
             bool good = true;
             if (q.dep >= 0) {
@@ -604,10 +625,16 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             const int K = q.K;
             const int nunits = K >> 4;  // 16 elements: 32 bytes of BF16 in, 16 bytes of FP8 out
             const uint16_t* xrow = q.x + (int64_t)m * q.ldx;
+            int u_lo = 0, u_hi = nunits;
+            if constexpr (Cfg::kChunk) {
+                const int upc = (nunits + q.nch - 1) / q.nch;
+                u_lo = c * upc;
+                u_hi = (u_lo + upc) < nunits ? (u_lo + upc) : nunits;
+            }
             float amax = 0.0f;
-            for (int u = et; u < nunits; u += 128) {
+            for (int u = u_lo + et; u < u_hi; u += 128) {
                 uint4 a, b;
-                if (q.kind == kChainKindSiluMul) {
+                if (Cfg::kFull && q.kind == kChainKindSiluMul) {
                     const uint4* gp = reinterpret_cast<const uint4*>(xrow) + 2 * u;
                     const uint4* up = reinterpret_cast<const uint4*>(xrow + K) + 2 * u;
                     const uint4 g0 = __ldcg(gp), g1 = __ldcg(gp + 1), u0 = __ldcg(up), u1 = __ldcg(up + 1);
@@ -626,8 +653,8 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                 }
                 amax = absmax_bf16x8(a, amax);
                 amax = absmax_bf16x8(b, amax);
-                ptx::st_shared_v4(stash_s + (uint32_t)u * 32u, a);
-                ptx::st_shared_v4(stash_s + (uint32_t)u * 32u + 16u, b);
+                ptx::st_shared_v4(stash_s + (uint32_t)(u - u_lo) * 32u, a);
+                ptx::st_shared_v4(stash_s + (uint32_t)(u - u_lo) * 32u + 16u, b);
             }
             float s, inv;
             if (q.static_scale != nullptr) {
@@ -639,6 +666,20 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                 if (lane == 0) red_s[qd] = amax;
                 asm volatile("bar.sync 3, 128;" ::: "memory");
                 amax = fmaxf(fmaxf(red_s[0], red_s[1]), fmaxf(red_s[2], red_s[3]));
+                if constexpr (Cfg::kChunk) {
+                    if (q.nch > 1) {
+                        unsigned int* am = amax_ws + j * kChainMaxM + m;
+                        unsigned int* qc = qcnt_ws + j * kChainMaxM + m;
+                        if (et == 0) {
+                            atomicMax(am, __float_as_uint(amax));   // non-negative floats order like their bit patterns
+                            ptx::red_release_add(qc, 1u);
+                            good = chain_poll_ge(qc, (unsigned)q.nch, gabort, abort_flag, status_word, limit);
+                            red_s[4] = __uint_as_float(ptx::ld_acquire_gpu(am));
+                        }
+                        if (epi_any(!good)) return false;
+                        amax = red_s[4];
+                    }
+                }
                 if (amax == 0.0f) {
                     s = 1.0f;
                     inv = 1.0f;
@@ -651,23 +692,23 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                 }
             }
             uint8_t* tiles = ws + q.x8_off;
-            for (int u = et; u < nunits; u += 128) {
+            for (int u = u_lo + et; u < u_hi; u += 128) {
                 uint4 a, b;
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                              : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w)
-                             : "r"(stash_s + (uint32_t)u * 32u));
+                             : "r"(stash_s + (uint32_t)(u - u_lo) * 32u));
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                              : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
-                             : "r"(stash_s + (uint32_t)u * 32u + 16u));
+                             : "r"(stash_s + (uint32_t)(u - u_lo) * 32u + 16u));
                 const uint2 qa = quant_bf16x8(a, inv), qb = quant_bf16x8(b, inv);
                 const uint4 o = make_uint4(qa.x, qa.y, qb.x, qb.y);
                 // operand tile of k-block u / 8: token m is row m, its 16-byte chunk c sits at c ^ (m & 7)
-                const int kb = u >> 3, c = u & 7;
-                *reinterpret_cast<uint4*>(tiles + (int64_t)kb * kChainXTileBytes + m * 128 + ((c ^ (m & 7)) << 4)) = o;
+                const int kb = u >> 3, ck = u & 7;
+                *reinterpret_cast<uint4*>(tiles + (int64_t)kb * kChainXTileBytes + m * 128 + ((ck ^ (m & 7)) << 4)) = o;
                 if (q.x8_out != nullptr)
                     *reinterpret_cast<uint4*>(q.x8_out + (int64_t)m * q.ldx8_out + (int64_t)u * 16) = o;
             }
-            if (et == 0) {
+            if (et == 0 && c == 0) {
                 sx_ws[j * kChainMaxM + m] = s;
                 if (q.s_x_out != nullptr) q.s_x_out[m] = s;
             }
@@ -675,10 +716,10 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             if (et == 0) ptx::red_release_add(&ctl->xready[j], 1u);
             return true;
         };
-        auto my_row = [&](const ChainProblem& q) {
-            // the row of problem q this CTA quantizes, or -1
-            const int m = (int)(((unsigned)p + (unsigned)P - (unsigned)q.job_base % (unsigned)P) % (unsigned)P);
-            return m < q.M ? m : -1;
+        auto my_job = [&](const ChainProblem& q) {
+            // the quantization job (row * nch + chunk) of problem q that this CTA runs, or -1
+            const int t = (int)(((unsigned)p + (unsigned)P - (unsigned)q.job_base % (unsigned)P) % (unsigned)P);
+            return t < (Cfg::kChunk ? q.M * q.nch : q.M) ? t : -1;
         };
         // Cast and store of the M tokens of one block of up to 96 rows whose scaled sums this thread
         // holds in res (its row: lane r of the accumulator); through the staging area in 16-byte
@@ -730,8 +771,8 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
         for (int j = 0; j < count && ok; ++j) {
             const ChainProblem& q = prm.prob[j];
             if (q.dep >= 0) continue;
-            const int m = my_row(q);
-            if (m >= 0) ok = quant_job(j, m);
+            const int t = my_job(q);
+            if (t >= 0) ok = Cfg::kChunk ? quant_job(j, t / q.nch, t % q.nch) : quant_job(j, t, 0);
         }
 
         int nacc = 0;
@@ -741,7 +782,9 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             float sx_mine = 0.0f;
             if (nseg > 0) {
                 // the scales were published together with the tiles the MMAs consume
-                if (et == 0) ok = chain_poll_ge(&ctl->xready[i], (unsigned)q.M, gabort, abort_flag, status_word, limit);
+                if (et == 0)
+                    ok = chain_poll_ge(&ctl->xready[i], (unsigned)(Cfg::kChunk ? q.M * q.nch : q.M), gabort, abort_flag,
+                                       status_word, limit);
                 ok = !epi_any(!ok);   // (the barrier orders the other threads behind thread 0's acquire)
                 if (!ok) break;
                 sx_mine = (lane < q.M) ? __ldcg(sx_ws + i * kChainMaxM + lane) : 0.0f;
@@ -761,7 +804,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (sg.part < 0) {
-#pragma unroll
+#pragma unroll 1   // (one copy of the block's code: the roles of a CTA share the instruction caches)
                     for (int b = 0; b < 2; ++b) {
                         if (b >= sg.NB) break;
                         uint32_t v[16];
@@ -773,7 +816,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const float sxm = __shfl_sync(0xFFFFFFFFu, sx_mine, jj);
-                            res[jj] = __uint_as_float(v[jj]) * (sxm * swn[b]);  // Eq. 4, Eq. 11
+                            res[jj] = __uint_as_float(v[jj]) * (sxm * (b == 0 ? swn[0] : swn[1]));  // Eq. 4, Eq. 11
                         }
                         const int Rb = (sg.R - b * BR) < BR ? (sg.R - b * BR) : BR;
                         emit_block(q, res, sg.n0 + b * BR, Rb);
@@ -826,13 +869,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) res[jj] = __uint_as_float(v[jj]);
                         if (r < sg.R) {
-                            const int others = last - first;
-                            if (others <= 2)
-                                chain_add_partials<2>(res, q, parts, slot_floats, r, first, last, P);
-                            else if (others <= 4)
-                                chain_add_partials<4>(res, q, parts, slot_floats, r, first, last, P);
-                            else
-                                chain_add_partials<8>(res, q, parts, slot_floats, r, first, last, P);
+                            chain_add_partials<4>(res, q, parts, slot_floats, r, first, last, P);
                         }
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
@@ -852,8 +889,8 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             for (int j = i + 1; j < count && ok; ++j) {
                 const ChainProblem& qj = prm.prob[j];
                 if (qj.dep != i) continue;
-                const int m = my_row(qj);
-                if (m >= 0) ok = quant_job(j, m);
+                const int t = my_job(qj);
+                if (t >= 0) ok = Cfg::kChunk ? quant_job(j, t / qj.nch, t % qj.nch) : quant_job(j, t, 0);
             }
         }
     } else if (is_dq) {
@@ -954,6 +991,15 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             for (int i = 0; i < kChainMaxProblems; ++i) {
                 ctl->xready[i] = 0u;
                 ctl->done[i] = 0u;
+            }
+            if constexpr (Cfg::kChunk) {
+                for (int i = 0; i < count; ++i) {
+                    if (prm.prob[i].nch == 1) continue;
+                    for (int m = 0; m < prm.prob[i].M; ++m) {
+                        amax_ws[i * kChainMaxM + m] = 0u;
+                        qcnt_ws[i * kChainMaxM + m] = 0u;
+                    }
+                }
             }
             ctl->abort = 0u;
             ctl->exit_count = 0u;

@@ -727,23 +727,23 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
         auto emit_block = [&](const ChainProblem& q, const float (&res)[16], int n0b, int Rb) {
             const int es = q.out_dtype == W4A8_OUT_FP32 ? 4 : 2;
             const bool wide_out = (((int64_t)q.ldy * es) & 15) == 0;  // rows of Y 16-byte aligned
-            if (wide_out) {
-                const uint32_t pitch = (uint32_t)(BR * es);
-                if (r < BR) {
+            const uint32_t pitch = (uint32_t)(BR * es);
+            if (r < BR) {
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const uint32_t a = stash_s + (uint32_t)jj * pitch + (uint32_t)(r * es);
-                        if (es == 4)
-                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[jj]) : "memory");
-                        else
-                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
-                                         "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[jj])))
-                                         : "memory");
-                    }
+                for (int jj = 0; jj < 16; ++jj) {
+                    const uint32_t a = stash_s + (uint32_t)jj * pitch + (uint32_t)(r * es);
+                    if (es == 4)
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(res[jj]) : "memory");
+                    else
+                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(a),
+                                     "h"(__bfloat16_as_ushort(__float2bfloat16_rn(res[jj])))
+                                     : "memory");
                 }
-                asm volatile("bar.sync 3, 128;" ::: "memory");
+            }
+            asm volatile("bar.sync 3, 128;" ::: "memory");
+            char* yb = static_cast<char*>(q.y) + (int64_t)n0b * es;
+            if (wide_out) {
                 const int ppt = (Rb * es) >> 4;  // 16-byte pieces per token (rows come in eights)
-                char* yb = static_cast<char*>(q.y) + (int64_t)n0b * es;
                 for (int id = et; id < q.M * ppt; id += 128) {
                     const int tok = id / ppt, piece = id - tok * ppt;
                     uint4 w;
@@ -752,19 +752,17 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                                  : "r"(stash_s + (uint32_t)tok * pitch + (uint32_t)(piece << 4)));
                     *reinterpret_cast<uint4*>(yb + (int64_t)tok * q.ldy * es + (piece << 4)) = w;
                 }
-                asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
-            } else if (r < Rb) {
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    if (jj < q.M) {
-                        const int64_t o = (int64_t)jj * q.ldy + n0b + r;
-                        if (es == 4)
-                            reinterpret_cast<float*>(q.y)[o] = res[jj];
-                        else
-                            reinterpret_cast<__nv_bfloat16*>(q.y)[o] = __float2bfloat16_rn(res[jj]);
-                    }
+            } else {
+                // rows of Y that are not 16-byte aligned: the same staged values, two bytes at a time
+                const int ppt = (Rb * es) >> 1;
+                for (int id = et; id < q.M * ppt; id += 128) {
+                    const int tok = id / ppt, piece = id - tok * ppt;
+                    uint16_t w;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(w) : "r"(stash_s + (uint32_t)tok * pitch + (uint32_t)(piece << 1)));
+                    *reinterpret_cast<uint16_t*>(yb + (int64_t)tok * q.ldy * es + (piece << 1)) = w;
                 }
             }
+            asm volatile("bar.sync 3, 128;" ::: "memory");  // before the area is written again
         };
 
         // problems whose input exists before the launch: quantized right away, by M CTAs each

@@ -310,3 +310,27 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_library_carries_on():
     _, _, ref = _oracle_layer(xb, wq)
     worst, _ = fp32_gate(y.cpu().numpy(), ref["y64"], rel=2e-3)
     assert worst <= 2e-3 and binding.query_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype,pad", [(torch.bfloat16, 3), (torch.float32, 1), (torch.bfloat16, 24)])
+def test_output_rows_that_are_not_16_byte_aligned(dtype, pad):
+    # Y as a view of a wider buffer: with an odd row pitch the kernel cannot store 16-byte pieces and
+    # takes its two-byte path; the values must be those of a contiguous output bit for bit, and the
+    # padding columns must stay untouched.  Whole blocks (N > 96 * SMs is not needed: the path is
+    # the same for blocks cut along K) and a short last block.
+    probs, wide = [], []
+    for i, (M, N, K) in enumerate([(5, 208, 256), (16, 1040, 384), (1, 96, 128)]):
+        wq, tw = _weights(N, K, 300 + i)
+        x = bf16_dev(inputs.make_activation(M, K, 310 + i, 0.01, 20.0))
+        buf = torch.full((M, N + pad), 7.0, dtype=dtype, device="cuda")
+        yc = torch.zeros((M, N), dtype=dtype, device="cuda")
+        probs.append(dict(x=x, weight=tw, y=buf[:, :N]))
+        probs.append(dict(x=x, weight=tw, y=yc))
+        wide.append((buf, yc, N))
+    binding.LinearChain(probs)()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for buf, yc, N in wide:
+        assert torch.equal(buf[:, :N].contiguous().view(torch.uint8), yc.view(torch.uint8))
+        assert bool((buf[:, N:] == 7.0).all())
+        assert bool(torch.isfinite(yc.float()).all()) and float(yc.float().abs().max()) > 0

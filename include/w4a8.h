@@ -107,8 +107,9 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * when it is NULL or too small; larger M requires it.  It
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
- * its first use; every call leaves it ready for the next one.  Calls that share a workspace
- * must not overlap on the device.
+ * its first use; every call leaves it ready for the next one -- except a call during which a
+ * bounded wait gave up (w4a8_query_device_status returns W4A8_ERR_TIMEOUT): zero-fill the
+ * workspace again after that.  Calls that share a workspace must not overlap on the device.
  * Calls with M <= 16 on tiled weights place their worker CTAs at run time (at most one per SM and
  * launch, so that consecutive launches can share the SMs).  The bookkeeping (1 KB, cleared by the
  * kernel) lives in the workspace when one of the full size is given -- nothing more to observe
@@ -411,8 +412,13 @@ int w4a8_forward_host(const void* x_host_bf16, int64_t M, const uint8_t* weights
 /*
  * Reads and clears the device-side status word (synchronises the device).  *flags receives a
  * bit mask: bit 0 = a bounded wait inside a kernel gave up; bit 1 = w4a8_prepack_weight met a
- * code its target format cannot hold.  Returns W4A8_ERR_TIMEOUT when bit 0 was set,
- * W4A8_ERR_BAD_SHAPE when only bit 1 was set, W4A8_OK otherwise.
+ * code its target format cannot hold; bit 2 = the run-time placement of a decode launch
+ * (w4a8_linear, M <= 16 on tiled weights) ended with a worker index unissued.  Bits 0 and 2 mean
+ * that the outputs of some launch are incomplete: returns W4A8_ERR_TIMEOUT; W4A8_ERR_BAD_SHAPE when
+ * only bit 1 was set, W4A8_OK otherwise.  After W4A8_ERR_TIMEOUT the workspaces of w4a8_linear
+ * calls that were in flight must be zero-filled again before they are reused (their split-K
+ * counters and placement state may have been left part-way); the workspace of w4a8_linear_chain
+ * needs no such care (its last CTA clears it after an aborted launch too).
  */
 int w4a8_query_device_status(unsigned int* flags_host);
 

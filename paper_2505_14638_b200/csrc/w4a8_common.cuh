@@ -16,6 +16,7 @@ constexpr float kE4M3Max = 448.0f;    // Z_max of Eq. 3 / Eq. 13
 // Device status word bits.
 constexpr unsigned int kStatusTimeout = 1u;   // a bounded device-side wait gave up
 constexpr unsigned int kStatusBadCode = 2u;   // prepack met a code the target format cannot hold
+constexpr unsigned int kStatusPlacement = 4u; // run-time placement of a decode launch ended with a worker index unissued
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
     return __uint_as_float(bits16 << 16);

@@ -121,18 +121,23 @@ __device__ SchedSlot g_sched[kSchedSlots];
 __device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candidates) {
     unsigned int smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    // The count of issued indices is read BEFORE this candidate takes its start number (an acquire
+    // load: the adds below cannot move in front of it).  Then every index counted in i was drawn by
+    // a candidate that is not among the `candidates - c` still to come, and the test below can only
+    // err towards working.  (Read together with the adds it saved a round trip, but i could then
+    // include draws of candidates with later start numbers, which the test counts again as still
+    // to come: a decliner too many, an index never issued.)
+    const unsigned int i = ptx::ld_acquire_gpu(&sl->issued);
     // (the two adds are independent: one L2 round trip for both)
-    // (the read of `issued` is issued together with the adds: three requests, one round trip)
-    const unsigned int i = *reinterpret_cast<volatile unsigned int*>(&sl->issued);
     const unsigned int c = atomicAdd(&sl->started, 1u);
     const bool first_here = smid < (unsigned)kSchedMaxSMs ? atomicAdd(&sl->on_sm[smid], 1u) == 0u : true;
     bool want = first_here;
     if (!want) {
         // A second candidate on this SM works only if the candidates still to come could not
-        // cover the indices still to be issued.  The count read here may lag behind (never run
-        // ahead of) the true one, which errs towards working -- a candidate that then draws an
-        // index beyond the last one retires after all; the candidate with the last start number
-        // therefore declines only when every index has been issued.
+        // cover the indices still to be issued.  The count read above may lag behind the true
+        // one, which errs towards working -- a candidate that then draws an index beyond the last
+        // one retires after all; the candidate with the last start number therefore declines only
+        // when every index has been issued.
         want = i < (unsigned)workers && (unsigned)workers - i >= (unsigned)candidates - c;
     }
     if (!want) return -1;
@@ -144,9 +149,15 @@ __device__ __forceinline__ int sched_enter(SchedSlot* sl, int workers, int candi
 // kernel, where it would delay the launch's completion).
 // (`gen` = the slot's generation if the caller has read it during this launch, kSchedGenUnknown otherwise)
 constexpr unsigned int kSchedGenUnknown = 0xFFFFFFFFu;
-__device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates, unsigned int gen_in) {
+__device__ __forceinline__ void sched_entered(SchedSlot* sl, int candidates, unsigned int gen_in, int workers,
+                                              unsigned int* status_word) {
     __threadfence();
     if (atomicAdd(&sl->finished, 1u) == (unsigned)candidates - 1u) {
+        // Every candidate has entered, so every index that will ever be drawn has been: if one is
+        // missing, a tile of this launch is never computed -- say so instead of leaving stale
+        // outputs behind silently.
+        if (*reinterpret_cast<volatile unsigned int*>(&sl->issued) < (unsigned)workers)
+            atomicOr(status_word, kStatusPlacement);
         // The last one clears the slot.  This sits between the last candidate's arrival and the
         // release of the dependent launch, so it is kept short: 16-byte stores, the three counters
         // and the new generation (which releases the candidates that still hold their place) in
@@ -337,13 +348,13 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
         P = plan.P;
         if (p < 0) {  // a worker of this launch is already on this SM: retire
             if (threadIdx.x == 0) {
-                sched_entered(sched_slot, (int)gridDim.x, sched_gen);  // before the trigger: see the notes beside SchedSlot
+                sched_entered(sched_slot, (int)gridDim.x, sched_gen, plan.P, status_word);  // before the trigger: see the notes beside SchedSlot
                 ptx::griddep_launch_dependents();
                 sched_hold(sched_slot, plan.P, sched_gen);
             }
             return;
         }
-        if (threadIdx.x == 64) sched_entered(sched_slot, (int)gridDim.x, kSchedGenUnknown);  // an idle epilogue thread
+        if (threadIdx.x == 64) sched_entered(sched_slot, (int)gridDim.x, kSchedGenUnknown, plan.P, status_word);  // an idle epilogue thread
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);

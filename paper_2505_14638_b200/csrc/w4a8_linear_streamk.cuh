@@ -22,7 +22,8 @@
 //
 // RB = 2 (whole tiles only): a tile is 256 weight rows x 256 tokens -- two 128-row blocks against one
 // activation tile per k-block, two accumulators of 256 columns (all of tensor memory, so the
-// epilogue of a tile no longer overlaps the next tile).  A k-block step then brings 18 KB of packed
+// epilogue of a tile no longer overlaps the next tile; the expansion warps, which have nothing to
+// expand into meanwhile, help to drain it).  A k-block step then brings 18 KB of packed
 // weights + 32 KB of activations for eight MMAs (about 1060 tensor-pipe cycles) instead of 9 + 32 KB
 // for four: the activation bytes an SM pulls from L2 per flop are halved, and the SM's L2 port
 // (about 64 bytes per clock) no longer sets the pace.  Measured on (2048, 4096, 4096), per CTA:
@@ -137,7 +138,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(bar_acc_full(b), 1);
-            ptx::mbar_init(bar_acc_empty(b), 256);
+            ptx::mbar_init(bar_acc_empty(b), RB == 2 ? 256 + 128 * G : 256);   // (RB = 2: the expansion warps drain too)
         }
         ptx::mbar_init(bar_drain, 1);
         *abort_flag = 0u;
@@ -156,6 +157,63 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     // set-up and weight prefetch while this one runs; everything that depends on earlier kernels
     // (activations, scales, outputs, workspace) is touched only after griddepcontrol.wait.
     ptx::griddep_launch_dependents();
+
+    // RB = 2: this warp's share of the 32 chunks (2 row blocks x 16 chunks of 16 token columns) of the
+    // CTA's j-th tile -- Eq. 4 / Eq. 11 scales, cast, store.  The tile's two accumulators fill tensor
+    // memory, so nothing overlaps its epilogue: besides the two epilogue warps of a lane quarter
+    // (slots 0 and 1) the quarter's expansion warps (slot 2 + group), which have nothing to expand
+    // into until the accumulators are free again, take chunks as well.
+    auto drain_wide = [&](int j, int slot) -> bool {
+        constexpr int kSlots = 2 + G;
+        const int q = warp & 3, r = q * 32 + lane;
+        const int64_t tile = u_begin / KB + j;
+        const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
+        const int m0 = mt * BNX;
+        const int n_lo = nt * TR + r, n_hi = n_lo + 128;
+        const float swn_lo = n_lo < N ? __ldg(s_w + (int64_t)n_lo * sw_stride) : 0.0f;
+        const float swn_hi = n_hi < N ? __ldg(s_w + (int64_t)n_hi * sw_stride) : 0.0f;
+        // activation scales of the tile's 256 tokens, one per lane and 32 tokens, fetched before the
+        // accumulator is ready and broadcast by shuffles later
+        float sx_pre[BNX / 32];
+#pragma unroll
+        for (int c = 0; c < BNX / 32; ++c) sx_pre[c] = (m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f;
+        if (!ptx::mbar_wait(bar_acc_full(0), (uint32_t)(j & 1), abort_flag, status_word)) return false;
+        ptx::tc_fence_after_sync();
+        const uint32_t tmem_acc0 = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+        for (int ch = slot; ch < 2 * (BNX / 16); ch += kSlots) {
+            const int b = ch / (BNX / 16), c0 = (ch - b * (BNX / 16)) * 16;
+            uint32_t v[16];
+            ptx::tmem_ld_32x32b_x16(tmem_acc0 + (uint32_t)(b * BNX + c0), v);
+            ptx::tmem_ld_wait();
+            if (m0 + c0 >= M) continue;  // warp-uniform
+            const int n = b == 0 ? n_lo : n_hi;
+            const float swn = b == 0 ? swn_lo : swn_hi;
+            float sx_lane = sx_pre[0];
+#pragma unroll
+            for (int c = 1; c < BNX / 32; ++c) sx_lane = (c0 >= c * 32) ? sx_pre[c] : sx_lane;
+            float sx[16];
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) sx[jj] = __shfl_sync(0xFFFFFFFFu, sx_lane, (c0 & 16) + jj);
+            if (n < N) {
+                if (out_dtype == W4A8_OUT_FP32) {
+                    float* yp = reinterpret_cast<float*>(y) + (int64_t)(m0 + c0) * ldy + n;
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        if (m0 + c0 + jj < M) yp[(int64_t)jj * ldy] = __uint_as_float(v[jj]) * (sx[jj] * swn);
+                } else {
+                    __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(y) + (int64_t)(m0 + c0) * ldy + n;
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        if (m0 + c0 + jj < M)
+                            yp[(int64_t)jj * ldy] = __float2bfloat16_rn(__uint_as_float(v[jj]) * (sx[jj] * swn));
+                }
+            }
+        }
+        ptx::tc_fence_before_sync();
+        ptx::mbar_arrive(bar_acc_empty(0));
+        return true;
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp, one lane issues)
@@ -309,6 +367,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         };
         int64_t shared_tile0 = 0, shared_tile1 = 0;  // tiles of which this CTA holds a partial (first and last segment)
         int n_shared = 0;
+        if constexpr (RB == 2) {
+            // whole tiles only: this warp's chunks of every tile of the CTA
+            for (; u < u_end && ok; u += KB, ++j) ok = drain_wide(j, half);
+        }
         while (u < u_end && ok) {
             const int64_t tile = u / KB;
             const int kb0 = (int)(u - tile * KB);
@@ -412,6 +474,14 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                                               stage_w8(s2) + (uint32_t)(b * 16384) + (uint32_t)r * 128u);
             ptx::fence_proxy_async_smem();
             ptx::mbar_arrive(bar_w8_full(s2));
+            if constexpr (RB == 2) {
+                // after this group's last stage of a tile: help to drain the tile's accumulators
+                const int jt = it / KB;
+                if (it + G >= n_it || (it + G) / KB != jt) {
+                    ptx::griddep_wait();  // (scales and outputs may still be in use by earlier kernels; long satisfied by now)
+                    if (!drain_wide(jt, 2 + g)) break;
+                }
+            }
         }
     }
 

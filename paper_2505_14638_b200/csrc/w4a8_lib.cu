@@ -1003,7 +1003,10 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
         d.job_base = jobs;
         jobs += d.M * d.nch;
         d.rem_rot = rot % sms;
-        rot += chain_rem_ctas(d, sms);
+        // the next problem's runs start behind this one's; when the runs cover every CTA, one CTA
+        // further, so that the adding CTAs (every few CTAs one) are not the same ones problem after problem
+        const int pr = chain_rem_ctas(d, sms);
+        rot += pr < sms ? pr : 1;
         d.x8_off = (uint32_t)off;
         off += (size_t)q.K * kChainMaxM;
         d.part_off = (uint32_t)off;

@@ -117,7 +117,8 @@ struct ChainCfg {
     static constexpr bool kFull = FULL_;
     static constexpr bool kChunk = FULL_;
     static constexpr int kS1Max = 16;     // weight ring (runtime depth <= this)
-    static constexpr int kS2 = 7;         // stages of expanded weights in tensor memory = activation-tile slots
+    static constexpr int kNAcc = 4;       // accumulator buffers (two blocks of 16 columns each): segments the MMAs may run ahead of the epilogue
+    static constexpr int kS2 = kNAcc == 4 ? 6 : 7;   // stages of expanded weights in tensor memory = activation-tile slots
     static constexpr int kMeta = meta_bytes(FMT_);
     static constexpr int kAStageCols = 64;                    // two items of 32 columns
     static constexpr int kDCol = kS2 * kAStageCols;           // 448: accumulators behind the A ring
@@ -128,8 +129,8 @@ struct ChainCfg {
     static constexpr int kSegBytes = kChainMaxProblems * (kChainMaxSegs + 1) * 16;   // segment table of this CTA
     static constexpr int kXRingBytes = kS2 * 2 * kChainXTileBytes;
     static constexpr int kSmemMax = 226 * 1024;
-    static_assert(kDCol + 2 * 2 * kChainMaxM <= kTmemCols, "tensor memory columns");
-    static_assert((2 * kS1Max + 2 * kS2 + 5) * 8 + 64 <= kBarBytes, "barrier area");
+    static_assert(kDCol + kNAcc * 2 * kChainMaxM <= kTmemCols, "tensor memory columns");
+    static_assert((2 * kS1Max + 2 * kS2 + 2 * kNAcc + 1) * 8 + 64 <= kBarBytes, "barrier area");
     static_assert(G_ >= 2 && G_ <= 4 && G_ <= kS2, "expansion groups");
 };
 
@@ -349,10 +350,11 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
     const uint32_t bar_wfree0 = bars_addr + 8u * S1M;                        // [S1M] expanded: slot may be refilled
     const uint32_t bar_afull0 = bars_addr + 8u * (2 * S1M);                  // [S2]  stage ready: weights expanded into tensor memory, activation tiles landed
     const uint32_t bar_afree0 = bar_afull0 + 8u * S2;                        // [S2]  stage consumed by the MMAs
-    const uint32_t bar_accfull0 = bar_afree0 + 8u * S2;                      // [2]
-    const uint32_t bar_accempty0 = bar_accfull0 + 16u;                       // [2]
-    const uint32_t bar_drain = bar_accempty0 + 16u;
-    constexpr int kNumBars = 2 * S1M + 2 * S2 + 5;
+    constexpr int NA = Cfg::kNAcc;
+    const uint32_t bar_accfull0 = bar_afree0 + 8u * S2;                      // [NA]
+    const uint32_t bar_accempty0 = bar_accfull0 + 8u * NA;                   // [NA]
+    const uint32_t bar_drain = bar_accempty0 + 8u * NA;
+    constexpr int kNumBars = 2 * S1M + 2 * S2 + 2 * NA + 1;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     float* red_s = reinterpret_cast<float*>(const_cast<uint32_t*>(tmem_slot) + 4);   // [4] warp maxima of a quantization job, [1] the row's maximum
@@ -394,7 +396,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             ptx::mbar_init(bar_afull0 + 8u * s, 96 + 1);   // the expanding threads + the activation loader (with its byte count)
             ptx::mbar_init(bar_afree0 + 8u * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NA; ++b) {
             ptx::mbar_init(bar_accfull0 + 8u * b, 1);
             ptx::mbar_init(bar_accempty0 + 8u * b, 128);
         }
@@ -493,9 +495,9 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             const int nseg = nseg_tab[i];
             for (int j = 0; j < nseg && ok; ++j) {
                 const ChainSeg sg = seg_tab[i * kChainMaxSegs + j];
-                const int buf = nacc & 1;
-                if (nacc >= 2) {
-                    ok = warp_all(chain_mbar_wait(bar_accempty0 + 8u * (uint32_t)buf, (uint32_t)((nacc >> 1) - 1) & 1u,
+                const int buf = nacc % NA;
+                if (nacc >= NA) {
+                    ok = warp_all(chain_mbar_wait(bar_accempty0 + 8u * (uint32_t)buf, (uint32_t)(nacc / NA - 1) & 1u,
                                                   abort_flag, gabort, status_word, limit));
                     if (!ok) break;
                 }
@@ -789,14 +791,14 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             }
             for (int j = 0; j < nseg && ok; ++j) {
                 const ChainSeg sg = seg_tab[i * kChainMaxSegs + j];
-                const int buf = nacc & 1;
+                const int buf = nacc % NA;
                 float swn[2];
 #pragma unroll
                 for (int b = 0; b < 2; ++b)
                     swn[b] = (sg.part < 0 && b < sg.NB && r < BR && b * BR + r < sg.R)
                                  ? __ldg(q.s_w + (int64_t)(sg.n0 + b * BR + r) * q.sw_stride)
                                  : 0.0f;
-                ok = chain_mbar_wait(bar_accfull0 + 8u * (uint32_t)buf, (uint32_t)(nacc >> 1) & 1u, abort_flag, gabort,
+                ok = chain_mbar_wait(bar_accfull0 + 8u * (uint32_t)buf, (uint32_t)(nacc / NA) & 1u, abort_flag, gabort,
                                      status_word, limit);
                 ok = !epi_any(!ok);   // all 128 threads take the same path (they meet at named barriers below)
                 if (!ok) break;

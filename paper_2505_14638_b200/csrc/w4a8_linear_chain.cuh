@@ -776,22 +776,38 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
         }
 
         int nacc = 0;
+        // "Activations ready" and the scales of the NEXT problem are looked up while this problem's
+        // first accumulator is awaited: two L2 round trips per problem that would otherwise sit in
+        // front of every problem's first segment (the epilogue warps are what paces short problems).
+        bool pre_seen = false;    // this thread saw the next problem's activations complete ...
+        float pre_sx = 0.0f;      // ... and read its lane's scale behind that acquire
         for (int i = 0; i < count && ok; ++i) {
             const ChainProblem& q = prm.prob[i];
             const int nseg = nseg_tab[i];
             float sx_mine = 0.0f;
             if (nseg > 0) {
-                // the scales were published together with the tiles the MMAs consume
-                if (et == 0)
-                    ok = chain_poll_ge(&ctl->xready[i], (unsigned)(Cfg::kChunk ? q.M * q.nch : q.M), gabort, abort_flag,
-                                       status_word, limit);
-                ok = !epi_any(!ok);   // (the barrier orders the other threads behind thread 0's acquire)
-                if (!ok) break;
-                sx_mine = (lane < q.M) ? __ldcg(sx_ws + i * kChainMaxM + lane) : 0.0f;
+                // every thread must have seen it (they take the same path: named barriers below)
+                if (!epi_any(!pre_seen)) {
+                    sx_mine = pre_sx;
+                } else {
+                    // the scales were published together with the tiles the MMAs consume
+                    if (et == 0)
+                        ok = chain_poll_ge(&ctl->xready[i], (unsigned)(Cfg::kChunk ? q.M * q.nch : q.M), gabort,
+                                           abort_flag, status_word, limit);
+                    ok = !epi_any(!ok);   // (the barrier orders the other threads behind thread 0's acquire)
+                    if (!ok) break;
+                    sx_mine = (lane < q.M) ? __ldcg(sx_ws + i * kChainMaxM + lane) : 0.0f;
+                }
             }
+            pre_seen = false;
             for (int j = 0; j < nseg && ok; ++j) {
                 const ChainSeg sg = seg_tab[i * kChainMaxSegs + j];
                 const int buf = nacc % NA;
+                if (j == 0 && i + 1 < count && nseg_tab[i + 1] > 0) {
+                    const ChainProblem& qn = prm.prob[i + 1];
+                    pre_seen = ptx::ld_acquire_gpu(&ctl->xready[i + 1]) >= (unsigned)(Cfg::kChunk ? qn.M * qn.nch : qn.M);
+                    pre_sx = (lane < qn.M) ? __ldcg(sx_ws + (i + 1) * kChainMaxM + lane) : 0.0f;
+                }
                 float swn[2];
 #pragma unroll
                 for (int b = 0; b < 2; ++b)

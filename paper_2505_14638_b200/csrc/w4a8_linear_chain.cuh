@@ -9,8 +9,8 @@
 //   * the weight ring (bulk copies into ~190 KB of shared memory) never drains at a problem
 //     boundary: the codes of problem i + 1 depend on nothing and are fetched while problem i is
 //     still being multiplied;
-//   * the CTA has all 512 tensor-memory columns: seven stages of expanded weights in flight plus
-//     double-buffered accumulators, so the epilogue of one segment overlaps the MMAs of the next;
+//   * the CTA has all 512 tensor-memory columns: six stages of expanded weights in flight plus four
+//     accumulator buffers, so the epilogues of up to four segments overlap the MMAs that follow;
 //   * problems are handed over through counters in the caller's workspace: the activations of a
 //     problem are quantized row by row by the epilogue warps of a few CTAs (one row per CTA),
 //     published with a fence and one atomic add, and picked up by every CTA's activation loader
@@ -23,9 +23,13 @@
 // are at least as many blocks left as CTAs, every CTA takes whole blocks (all of K, one or two
 // blocks at a time, results written directly).  The remaining blocks are cut along K as well: their
 // (block, k-block) items are dealt out evenly, a CTA gets one contiguous run (at most two blocks),
-// writes its FP32 partial sums to the workspace, and the CTA that arrives last at a block adds the
-// partial sums in ascending k order -- a fixed order, so results repeat bit for bit -- and writes Y.
-// Every CTA therefore expands the same number of weights within one item, whatever N is.
+// writes its FP32 partial sums to the workspace, and the CTA that holds a block's lowest k range (the
+// second part of its run: it reaches the block last) adds the partial sums in ascending k order -- a
+// fixed order, so results repeat bit for bit -- and writes Y.  A CTA works on its run of the cut
+// blocks first and on its whole blocks afterwards, so that the hand-over of the partial sums hides
+// behind the whole blocks instead of standing at the end of the problem, where the next problem of
+// a dependent chain waits for it.  Every CTA expands the same number of weights within one item,
+// whatever N is.
 //
 // Data path of one (k-block, 96-row block) item: as in the split-N kernel --
 //   HBM --bulk copy--> shared memory (INT4 codes + group scales [+ zero-points])
@@ -251,12 +255,17 @@ __host__ __device__ inline int chain_num_segs(const ChainProblem& q, int p, int 
     }
     return n;
 }
-// Segment j of CTA p.
-__host__ __device__ inline ChainSeg chain_seg(const ChainProblem& q, int p, int P, int j) {
+// Segment j of CTA p.  The CTA's run of the blocks that are cut along K comes FIRST, its whole blocks
+// after it: the hand-over of partial sums and the adding-up then overlap the whole blocks' MMAs
+// instead of standing at the end of the problem, where a dependent problem waits for them.
+// (nsegs = chain_num_segs(q, p, P), passed in: it costs 64-bit divisions)
+__host__ __device__ inline ChainSeg chain_seg(const ChainProblem& q, int p, int P, int j, int nsegs) {
     ChainSeg s;
     const int KB = q.K >> 7;
     const int full_segs = (q.rounds + 1) / 2;
-    if (j < full_segs) {
+    const int rem_segs = nsegs - full_segs;
+    if (j >= rem_segs) {
+        j -= rem_segs;
         const int b0 = p * q.rounds + 2 * j;
         s.NB = (signed char)((q.rounds - 2 * j) < 2 ? 1 : 2);
         s.blk = b0;
@@ -274,7 +283,7 @@ __host__ __device__ inline ChainSeg chain_seg(const ChainProblem& q, int p, int 
     const long long lo = chain_rem_lo(l, Pr, items), hi = chain_rem_lo(l + 1, Pr, items);
     const int br0 = (int)(lo / KB);
     const long long cut = (long long)(br0 + 1) * KB;
-    const int jj = j - full_segs;
+    const int jj = j;
     const long long a = jj == 0 ? lo : cut, b = jj == 0 ? (hi < cut ? hi : cut) : hi;
     const int br = br0 + jj;
     s.NB = 1;
@@ -413,7 +422,7 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
         const ChainProblem& q = prm.prob[i];
         const int n = chain_num_segs(q, p, P);
         const_cast<int*>(nseg_tab)[i] = n;
-        for (int j = 0; j < n; ++j) const_cast<ChainSeg*>(seg_tab)[i * kChainMaxSegs + j] = chain_seg(q, p, P, j);
+        for (int j = 0; j < n; ++j) const_cast<ChainSeg*>(seg_tab)[i * kChainMaxSegs + j] = chain_seg(q, p, P, j, n);
     }
     ptx::tc_fence_before_sync();
     __syncthreads();

@@ -240,8 +240,23 @@ static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
         const double t_unit = mma_cycles / 1900.0 > 0.22 ? mma_cycles / 1900.0 : 0.22;
         const int64_t Pa = cap < Tt ? cap : Tt;
         const double t_aligned = (double)((Tt + Pa - 1) / Pa) * (double)KB * t_unit;
-        const int64_t Ps = cap < U ? cap : U;
-        const double t_split = (double)((U + Ps - 1) / Ps) * t_unit + 2.0 + bnx * 2048.0 / 1.0e5;
+        int64_t Ps = cap < U ? cap : U;
+        const double t_tail = 2.0 + bnx * 2048.0 / 1.0e5;   // exchange of partial tiles: two per CTA
+        double t_split = (double)((U + Ps - 1) / Ps) * t_unit + t_tail;
+        if (Tt < cap && KB % (cap / Tt) == 0) {
+            // Fewer tiles than CTAs: a whole number of CTAs per tile instead of equal slices of the
+            // unit space, where that number divides the k-blocks.  Every CTA then stays inside one
+            // tile -- one partial tile to store, and a tile's contributors finish together -- at
+            // the price of a few idle SMs (measured, us: (128, 4096, 4096) 13.4 against 17.9;
+            // (512, 4096, 14336) 41.6 against 49.8; with a remainder -- (256, 6144, 4096), three CTAs
+            // per tile, 32 k-blocks -- it was slower: 20.9 against 18.0).
+            const int64_t Pk = Tt * (cap / Tt);
+            const double t_k = (double)((U + Pk - 1) / Pk) * t_unit + 0.5 * t_tail;
+            if (t_k < t_split) {
+                t_split = t_k;
+                Ps = Pk;
+            }
+        }
         const bool al = t_aligned <= t_split;
         const double t = al ? t_aligned : t_split;
         if (t < best) {
@@ -341,7 +356,7 @@ static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan
     const int fixed = Cfg::kBarBytes + Cfg::kOutBytes + 1024;
     int s1 = (Cfg::kSmemBudget - fixed) / (pl->wstage + pl->xstage);
     if (s1 > Cfg::kS1Max) s1 = Cfg::kS1Max;
-    if (s1 < Cfg::kS2) return false;  // the tensor-memory ring may not be deeper than the TMA ring
+    if (s1 < Cfg::kS2 || s1 < Cfg::G) return false;  // the tensor-memory ring may not be deeper than the TMA ring, nor may there be more groups than slots
     pl->S1 = s1;
     pl->smem = s1 * (pl->wstage + pl->xstage) + fixed;
     return true;
@@ -502,10 +517,29 @@ static int launch_pair(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, cons
     return launch_status();
 }
 
+// 65..128 tokens on a layer with few output channels (at most a quarter as many 128-row tiles as
+// SMs): the persistent kernel with K cut between a whole number of CTAs per tile, instead of the
+// split-N kernel, every CTA of which pulls the whole X8 through its L2 port (measured, us:
+// o projection 13.4 against 15.3, down projection 21.5 against 27.5; qkv and gate_up stay: 16.9
+// against 15.4, 33.6 against 27.1).
+static bool streamk_for_128_tokens(int64_t M, int64_t N, int64_t K, int sms) {
+    return M > 64 && M <= kSplitNMaxM && K >= 2048 && ((N + 127) / 128) * 4 <= sms;
+}
+
 static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* wpp,
                              int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
                              int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
-    if (M <= kSplitNMaxM) {
+    bool split_n = M <= kSplitNMaxM;
+    if (split_n && M > 64) {
+        // (the persistent kernel needs its full workspace; without it the split-N kernel runs)
+        SkPlan plq;
+        make_sk_plan(M, N, K, kNominalSMs, &plq);
+        const int sms_q = sm_count();
+        if (sms_q > 0 && streamk_for_128_tokens(M, N, K, sms_q) && workspace != nullptr &&
+            workspace_bytes >= plq.workspace_bytes && aligned16(workspace))
+            split_n = false;
+    }
+    if (split_n) {
         int rc = check_device();
         if (rc != W4A8_OK) return rc;
         const int mt = M <= 16 ? 16 : (M <= 64 ? 64 : 128);
@@ -566,9 +600,9 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     }
     if (pair_kernel_applies(M, N, K, sms))
         return fmt == kFmtTiledSignMag
-                   ? launch_pair<PairCfg<4, 6, 4, kFmtTiledSignMag>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                   ? launch_pair<PairCfg<3, 6, 4, kFmtTiledSignMag>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
                                                                       (int)M, (int)N, (int)K, sms, st)
-                   : launch_pair<PairCfg<4, 6, 4, kFmtTiled>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                   : launch_pair<PairCfg<3, 6, 4, kFmtTiled>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
                                                                (int)M, (int)N, (int)K, sms, st);
     make_sk_plan(M, N, K, sms, &pl);
     CUtensorMap tx;
@@ -583,8 +617,8 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
              : launch_streamk<SkCfg<BNX, G, S1, S2, kFmtTiled>>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, \
                                                                 workspace, pl, Mi, Ni, Ki, st)
     switch (pl.bnx) {
-        case 64: W4A8_SK(64, 4, 6, 4); break;
-        case 128: W4A8_SK(128, 4, 5, 4); break;
+        case 64: W4A8_SK(64, 4, 8, 4); break;
+        case 128: W4A8_SK(128, 4, 4, 4); break;
         default: W4A8_SK(256, 4, 4, 3); break;
     }
 #undef W4A8_SK
@@ -1023,7 +1057,7 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
     const int fixed = 1024 + C0::kXRingBytes + stash + C0::kBarBytes + C0::kSegBytes;
     int s1 = (C0::kSmemMax - fixed) / prm.wslot;
     if (s1 > C0::kS1Max) s1 = C0::kS1Max;
-    if (s1 < 4) return W4A8_ERR_BAD_SHAPE;
+    if (s1 < C0::kS2) return W4A8_ERR_BAD_SHAPE;   // (the weight ring may not be shallower than the tensor-memory ring)
     prm.S1 = s1;
     const int smem = fixed + s1 * prm.wslot;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -1101,10 +1135,11 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
     if (M <= 0 || N <= 0 || K <= 0 || K % kGroup != 0) return 0;
     if (weight_format == kFmtCanonical) return w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_AUTO, 0);
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
-    if (M <= kSplitNMaxM) return kSnWorkspaceBytes;  // used when the layer has few output channels and K is cut
+    if (M <= 64) return kSnWorkspaceBytes;  // used when the layer has few output channels and K is cut
     SkPlan pl;
     make_sk_plan(M, N, K, kNominalSMs, &pl);
-    return pl.workspace_bytes;
+    // (65..128 tokens: either kernel may run, the persistent one only with its full workspace)
+    return M <= kSplitNMaxM && pl.workspace_bytes < kSnWorkspaceBytes ? kSnWorkspaceBytes : pl.workspace_bytes;
 }
 
 size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format) {

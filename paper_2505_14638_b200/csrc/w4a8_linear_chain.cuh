@@ -955,11 +955,14 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                     const int ks = (sg.nkb - st * KS) < KS ? (sg.nkb - st * KS) : KS;
                     const uint32_t full_bar = bar_wfull0 + 8u * (uint32_t)r1.idx;
                     const uint32_t free_bar = bar_afree0 + 8u * (uint32_t)r2.idx;
-                    // both are normally complete already: test them together, wait only if not
-                    const bool have_w = ptx::mbar_test_wait(full_bar, r1.phase);
-                    const bool have_slot = ptx::mbar_test_wait(free_bar, r2.phase ^ 1u);
-                    if (!have_w) ok = chain_mbar_wait(full_bar, r1.phase, abort_flag, gabort, status_word, limit);
-                    if (ok && !have_slot) ok = chain_mbar_wait(free_bar, r2.phase ^ 1u, abort_flag, gabort, status_word, limit);
+                    // Both are normally complete already.  The tensor-memory stage FIRST: once the MMAs S2
+                    // stages back have completed, every earlier stage has landed -- among them the previous
+                    // use of this stage's ring slot (S1 >= S2) -- so the parity test of "weights landed"
+                    // cannot mistake the phase before last for this one.
+                    if (!ptx::mbar_test_wait(free_bar, r2.phase ^ 1u))
+                        ok = chain_mbar_wait(free_bar, r2.phase ^ 1u, abort_flag, gabort, status_word, limit);
+                    if (ok && !ptx::mbar_test_wait(full_bar, r1.phase))
+                        ok = chain_mbar_wait(full_bar, r1.phase, abort_flag, gabort, status_word, limit);
                     ok = warp_all(ok);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();

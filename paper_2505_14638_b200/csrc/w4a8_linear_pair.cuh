@@ -45,6 +45,9 @@ struct PairCfg {
     static constexpr int kThreads = 32 * (10 + 4 * G);
     // same ring-depth rule as the one-CTA persistent kernel (barrier parity, skipped phases)
     static_assert(S1 <= 2 * S2, "ring depths");
+    // (a group's next "weights landed" wait must find the slot's previous use among the group's own
+    // earlier stages: see the persistent one-CTA kernel)
+    static_assert(S1_ % G_ == 0, "the ring depth must be a multiple of the number of expansion groups");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
     static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");

@@ -618,13 +618,17 @@ linear_splitn_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K
             for (; st < nst; st += G) {
                 const int kb = st * KS;
                 const int ks = (nkb - kb) < KS ? (nkb - kb) : KS;
-                // both barriers are normally complete already: test them together, wait only if not
+                // Both barriers are normally complete already.  The tensor-memory slot FIRST: once the
+                // MMAs S2 stages back have completed, every earlier stage has landed -- among them the
+                // previous use of this stage's ring slot (S1 >= S2) -- so the parity test of "weights
+                // landed" cannot mistake the phase before last for this one.  (Tested the other way
+                // round, a group ahead of a late copy could pass one phase early.)
                 const uint32_t full_bar = bar_full0 + 8u * (uint32_t)r1.idx;
                 const uint32_t free_bar = bar_free10 + 8u * (uint32_t)rl.idx;
-                const bool have_w = ptx::mbar_test_wait(full_bar, r1.phase);
-                const bool have_slot = done < S2 || ptx::mbar_test_wait(free_bar, rl.phase);
-                if (!have_w) ok = ptx::mbar_wait(full_bar, r1.phase, abort_flag, status_word);
-                if (ok && !have_slot) ok = ptx::mbar_wait(free_bar, rl.phase, abort_flag, status_word);
+                if (done >= S2 && !ptx::mbar_test_wait(free_bar, rl.phase))
+                    ok = ptx::mbar_wait(free_bar, rl.phase, abort_flag, status_word);
+                if (ok && !ptx::mbar_test_wait(full_bar, r1.phase))
+                    ok = ptx::mbar_wait(full_bar, r1.phase, abort_flag, status_word);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * plan.wstage);

@@ -72,8 +72,14 @@ struct SkCfg {
     static_assert(S1 <= 2 * S2, "ring depths: see the comment above");
     // The same parity argument for the "packed weights landed" barriers: a group that has finished
     // stage i next waits for stage i + G in ring slot (i + G) % S1, whose previous use is stage
-    // i + G - S1; that one has landed for sure only if it is not later than stage i itself.
-    static_assert(G_ <= S1_, "a group must not run ahead of the TMA ring by more than one round");
+    // i + G - S1.  That stage must have landed before the wait starts, or the wait passes one phase
+    // early and the group expands what is still in the slot.  With S1 a multiple of G it is one of
+    // the group's own earlier stages (or stage i itself), which it has seen land.  With S1 = 5 or 6
+    // and G = 4 it was another group's stage, issued earlier than stage i but not bound to land
+    // earlier: first launches of a process (cold translation caches, latencies all over the
+    // place) now and then summed a stale tile into a few outputs -- found when a second launch on
+    // the same inputs disagreed with the first.
+    static_assert(S1_ % G_ == 0, "the ring depth must be a multiple of the number of expansion groups");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
     static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");

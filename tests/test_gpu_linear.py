@@ -120,7 +120,10 @@ def test_persistent_kernel_split_tiles_and_reuse_of_workspace(M, N, K):
     assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
     worst, _ = fp32_gate(outs[0].cpu().numpy()[:, cols], ref["y64"])
     assert worst <= 2e-3, worst
-    n_counter_bytes = 1024 if M <= 128 else 8 * ((M + 255) // 256) * ((N + 127) // 128)
+    # (65..128 tokens on a layer with few output channels run on the persistent kernel as well)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    persistent = M > 128 or (M > 64 and K >= 2048 and ((N + 127) // 128) * 4 <= sms)
+    n_counter_bytes = 8 * ((M + 255) // 256) * ((N + 127) // 128) if persistent else 1024
     assert np.all(ws[:n_counter_bytes].cpu().numpy() == 0)     # tile counters are back to zero
 
 

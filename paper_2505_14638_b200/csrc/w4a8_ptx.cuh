@@ -67,23 +67,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// The same test with a suspend-time hint: the thread may stay suspended in hardware for up to
-// `hint_ns` nanoseconds (it is woken when the phase completes), instead of returning to a polling
-// loop whose instructions compete with the working warps of its SM sub-partition for issue slots.
-__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(hint_ns)
-        : "memory");
-    return ok != 0;
-}
-
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
 // Non-blocking test of a phase; two of them issued back to back overlap their round trips.

@@ -890,8 +890,10 @@ def scheme_sweep(torch, binding, inputs, dev):
     """Same-box counterpart of the paper's scheme comparison (Sec. 4.3, Fig. 4, Table 3): per layer
     and token count the time of W4A8 as built here (group-aware order: groups are runs of columns),
     of W8A8 (FP8 weights, own kernel and the library's FP8 GEMM), of W4A16 (own kernel) and of W4A8 quantized in an
-    unconstrained activation order (per-column group index: the FP8 weights must be materialised
-    by w4a8_dequant_weight_gidx before a W8A8 GEMM can use them).  CUDA graphs, rotating weights."""
+    unconstrained activation order (per-column group index), both as two launches (the FP8 weights
+    materialised by w4a8_dequant_weight_gidx, then a W8A8 GEMM) and as one kernel with the look-up
+    inside (w4a8_linear_gidx), next to the same tile kernel on the group-aware order.  CUDA graphs,
+    rotating weights."""
     out = []
     side = torch.cuda.Stream()
 
@@ -936,6 +938,12 @@ def scheme_sweep(torch, binding, inputs, dev):
                 binding.dequant_weight_gidx(cq[0], cq[1], None, g_idx, out=w8_tmp)
                 binding.linear_w8a8(x8, s_x, w8_tmp, cq[3], out=y)
             t_ao = graph_time(act_order, reps)
+            # the same scheme in ONE kernel: per-weight scale look-up inside the canonical-layout tile kernel,
+            # next to that kernel on the group-aware (consecutive) order of the same layer
+            t_aof = graph_time(lambda c: binding.linear_gidx(x8, s_x, raw[c % copies][0], raw[c % copies][1], None,
+                                                             g_idx, raw[c % copies][3], out=y), reps)
+            t_tile = graph_time(lambda c: binding.linear(x8, s_x, raw[c % copies][0], raw[c % copies][1], None,
+                                                         raw[c % copies][3], algo=binding.ALGO_UMMA, out=y), reps)
             t_lib = graph_time(lambda c: torch._scaled_mm(a8, w8s[c % copies].view(torch.float8_e4m3fn).t(),
                                                           scale_a=one, scale_b=one, out_dtype=torch.bfloat16), reps)
 
@@ -948,6 +956,7 @@ def scheme_sweep(torch, binding, inputs, dev):
             t_16 = graph_time(w4a16, reps)
             out.append({"layer": name, "K": k, "N": n, "M": m, "w4a8_us": t_w4 * 1e6, "w8a8_own_kernel_us": t_w8 * 1e6,
                         "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6,
+                        "w4a8_act_order_one_kernel_us": t_aof * 1e6, "w4a8_same_tile_kernel_group_order_us": t_tile * 1e6,
                         "w4a16_own_kernel_us": t_16 * 1e6})
             del x, x8, s_x, y, ws
         del tws, w8s, raw, w8_tmp

@@ -332,6 +332,24 @@ int w4a8_dequant_weight_gidx(const uint8_t* codes, const void* gscale_bf16, cons
                              const int32_t* g_idx, int64_t N, int64_t K, int64_t G, uint8_t* w8, void* stream);
 
 /*
+ * The W4A8 linear layer on activation-ordered weights in ONE kernel (the W4A8* rows of Table 3;
+ * appendix "Activation Reordering"): as w4a8_linear on canonical weights, except that column k of
+ * the weights takes the scale and zero-point of group g_idx[k] (device int32 [K], values in
+ * [0, K / 128), not range-checked on the device).  No look-up table can be shared by the columns of
+ * a k-block, so Eq. 10 is evaluated weight by weight inside the kernel (a multiplication and a
+ * conversion each, with two cached loads for the group's scale and zero-point): what this costs
+ * against w4a8_linear on the same layer is the inference overhead of an unconstrained activation
+ * order.  The FP8 weights it multiplies with are those of w4a8_dequant_weight_gidx, so the result
+ * equals w4a8_linear_w8a8 on that output bit for bit.  Workspace:
+ * w4a8_linear_ex_workspace_bytes(M, N, K, W4A8_ALGO_UMMA, 0) bytes.  Other arguments and errors
+ * as in w4a8_linear_ex; W4A8_ERR_INVALID_ARG for a NULL or misaligned g_idx.
+ */
+int w4a8_linear_gidx(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                     const void* gscale_bf16, const uint8_t* gzero, const int32_t* g_idx, const float* s_w,
+                     int sw_stride, int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * W8A8 comparison scheme (Sec. 4.3, Fig. 4): the same FP8 GEMM and epilogue on weights that are
  * stored as FP8 E4M3 bytes -- e.g. the output of w4a8_dequant_weight -- so that the cost of
  * streaming twice the bytes can be set against the cost of expanding INT4 on the fly, on the

@@ -27,7 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
-    "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx",
+    "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx", "w4a8_linear_gidx",
     "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
@@ -99,6 +99,8 @@ def lib():
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
     L.w4a8_dequant_weight_gidx.restype = i32
     L.w4a8_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p, p]
+    L.w4a8_linear_gidx.restype = i32
+    L.w4a8_linear_gidx.argtypes = [p, i64, p, i64, p, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz, p]
     L.w4a8_linear_w8a8.restype = i32
     L.w4a8_linear_w8a8.argtypes = [p, i64, p, i64, p, p, i32, i64, i64, p, i64, i32, p, sz, p]
     L.w4a8_linear_ex_workspace_bytes.restype = sz
@@ -352,6 +354,23 @@ def dequant_weight_gidx(codes, gscale, gzero, g_idx, out=None):
                                         gscale.shape[1], _ptr(w8), _stream())
     _check("w4a8_dequant_weight_gidx", rc)
     return w8
+
+
+def linear_gidx(x8, s_x, codes, gscale, gzero, g_idx, s_w, out_dtype=OUT_BF16, out=None):
+    """w4a8_linear_gidx: the linear layer on activation-ordered weights (per-column group index) in one kernel."""
+    import torch
+    M, K = x8.shape
+    N = codes.shape[0]
+    if out is None:
+        dt = torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32
+        out = torch.empty((M, N), dtype=dt, device=x8.device)
+    nb = linear_workspace_bytes(M, N, K, ALGO_UMMA, 0)
+    ws = torch.empty((max(nb, 16),), dtype=torch.uint8, device=x8.device)
+    rc = lib().w4a8_linear_gidx(_ptr(x8), x8.stride(0), _ptr(s_x), M, _ptr(codes), _ptr(gscale), _ptr(gzero),
+                                _ptr(g_idx), _ptr(s_w), 0 if s_w.numel() == 1 else 1, N, K, GROUP, _ptr(out),
+                                out.stride(0), int(out_dtype), _ptr(ws), nb, _stream())
+    _check("w4a8_linear_gidx", rc)
+    return out
 
 
 def linear_w8a8(x8, s_x, w8, s_w, out_dtype=OUT_BF16, out=None):

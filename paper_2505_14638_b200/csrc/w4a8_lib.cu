@@ -176,7 +176,7 @@ static int make_plan(int64_t M, int64_t N, int64_t K, int algo, int split_k, Lin
 
 template <class Cfg>
 static int launch_umma(const CUtensorMap& tw, const CUtensorMap& tx, const uint16_t* gscale, const uint8_t* gzero,
-                       const float* s_x, const float* s_w, int sw_stride, void* y, int64_t ldy, int out_dtype,
+                       const int32_t* g_idx, const float* s_x, const float* s_w, int sw_stride, void* y, int64_t ldy, int out_dtype,
                        float* partial, int M, int N, int K, int split_k, cudaStream_t st) {
     auto kern = linear_umma_kernel<Cfg>;
     static std::once_flag once;
@@ -188,7 +188,7 @@ static int launch_umma(const CUtensorMap& tw, const CUtensorMap& tx, const uint1
     unsigned int* status = status_word_ptr();
     if (!status) return W4A8_ERR_CUDA;
     dim3 grid((unsigned)((N + 127) / 128), (unsigned)((M + Cfg::BNX - 1) / Cfg::BNX), (unsigned)split_k);
-    kern<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tw, tx, gscale, gzero, s_x, s_w, sw_stride, y, ldy,
+    kern<<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(tw, tx, gscale, gzero, g_idx, s_x, s_w, sw_stride, y, ldy,
                                                        out_dtype, partial, M, N, K, (K / 128) / split_k, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return launch_status();
@@ -628,8 +628,10 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
 static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
                        const void* gscale, const uint8_t* gzero, int fmt, const float* s_w, int sw_stride,
                        int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype, void* workspace,
-                       size_t workspace_bytes, int algo, int split_k, cudaStream_t st) {
+                       size_t workspace_bytes, int algo, int split_k, cudaStream_t st,
+                       const int32_t* g_idx = nullptr) {
     if (fmt != kFmtCanonical && fmt != kFmtTiled && fmt != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+    if (g_idx && (fmt != kFmtCanonical || (reinterpret_cast<uintptr_t>(g_idx) & 3u))) return W4A8_ERR_INVALID_ARG;
     if (!x8 || !s_x || !codes || !s_w || !y) return W4A8_ERR_INVALID_ARG;
     if (fmt == kFmtCanonical && !gscale) return W4A8_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
@@ -676,8 +678,11 @@ static int linear_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_
     float* partial = plan.split_k > 1 ? static_cast<float*>(workspace) : nullptr;
     const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
 #define W4A8_LAUNCH(BNX, STG)                                                                                 \
-    rc = launch_umma<UmmaCfg<BNX, STG>>(tw, tx, gs, gzero, s_x, s_w, sw_stride, y, ldy, out_dtype, partial, Mi, \
-                                        Ni, Ki, plan.split_k, st)
+    rc = g_idx ? launch_umma<UmmaCfg<BNX, STG, false, false, true>>(tw, tx, gs, gzero, g_idx, s_x, s_w, sw_stride, y, \
+                                                                    ldy, out_dtype, partial, Mi, Ni, Ki,          \
+                                                                    plan.split_k, st)                             \
+               : launch_umma<UmmaCfg<BNX, STG>>(tw, tx, gs, gzero, nullptr, s_x, s_w, sw_stride, y, ldy, out_dtype,  \
+                                                partial, Mi, Ni, Ki, plan.split_k, st)
     switch (plan.bnx) {
         case 16: W4A8_LAUNCH(16, 4); break;
         case 32: W4A8_LAUNCH(32, 4); break;
@@ -728,7 +733,7 @@ static int linear_w8a8_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, i
     float* partial = plan.split_k > 1 ? static_cast<float*>(workspace) : nullptr;
     const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
 #define W4A8_LAUNCH8(BNX, STG)                                                                                   \
-    rc = launch_umma<UmmaCfg<BNX, STG, true>>(tw, tx, nullptr, nullptr, s_x, s_w, sw_stride, y, ldy, out_dtype,  \
+    rc = launch_umma<UmmaCfg<BNX, STG, true>>(tw, tx, nullptr, nullptr, nullptr, s_x, s_w, sw_stride, y, ldy, out_dtype,  \
                                               partial, Mi, Ni, Ki, plan.split_k, st)
     switch (plan.bnx) {
         case 16: W4A8_LAUNCH8(16, 4); break;
@@ -792,7 +797,7 @@ static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_
     float* partial = split_k > 1 ? static_cast<float*>(workspace) : nullptr;
     const int Mi = (int)M, Ni = (int)N, Ki = (int)K;
 #define W4A8_LAUNCH16(BNX, STG)                                                                                  \
-    rc = launch_umma<UmmaCfg<BNX, STG, false, true>>(tw, tx, gs, gzero, nullptr, s_w, sw_stride, y, ldy,         \
+    rc = launch_umma<UmmaCfg<BNX, STG, false, true>>(tw, tx, gs, gzero, nullptr, nullptr, s_w, sw_stride, y, ldy,         \
                                                      out_dtype, partial, Mi, Ni, Ki, split_k, st)
     switch (bnx) {
         case 16: W4A8_LAUNCH16(16, 4); break;
@@ -1176,6 +1181,16 @@ int w4a8_linear_ex(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M,
                    size_t workspace_bytes, int algo, int split_k, void* stream) {
     return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
                        ldy, out_dtype, workspace, workspace_bytes, algo, split_k, static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_linear_gidx(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,
+                     const void* gscale_bf16, const uint8_t* gzero, const int32_t* g_idx, const float* s_w,
+                     int sw_stride, int64_t N, int64_t K, int group, void* y, int64_t ldy, int out_dtype,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+    if (!g_idx) return W4A8_ERR_INVALID_ARG;
+    return linear_impl(x8, ldx8, s_x, M, codes, gscale_bf16, gzero, kFmtCanonical, s_w, sw_stride, N, K, group, y,
+                       ldy, out_dtype, workspace, workspace_bytes, W4A8_ALGO_UMMA, 0, static_cast<cudaStream_t>(stream),
+                       g_idx);
 }
 
 int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* codes,

@@ -22,10 +22,15 @@ namespace w4a8 {
 // W16_ = true: the W4A16 comparison scheme of Sec. 4.3: activations stay BF16, the INT4 codes are
 // expanded to BF16 (u - z) * s_g, rounded once, and multiplied with kind::f16 MMAs (K = 16 each);
 // a k-block of 128 is then two swizzled 128-byte panels of 64 elements per operand.
-template <int BNX_, int STAGES_, bool W8_ = false, bool W16_ = false>
+// GIDX_ = true: weights quantized in an unconstrained activation order (the W4A8* rows of Table 3,
+// appendix "Activation Reordering"): column k takes the scale and zero-point of group g_idx[k], so
+// no look-up table can be shared by the 128 columns of a k-block -- every weight is expanded by its
+// own multiplication and conversion (Eq. 10 element by element), inside the same kernel.
+template <int BNX_, int STAGES_, bool W8_ = false, bool W16_ = false, bool GIDX_ = false>
 struct UmmaCfg {
     static constexpr bool W8 = W8_;
     static constexpr bool W16 = W16_;
+    static constexpr bool GIDX = GIDX_;
     static constexpr int BNX = BNX_;        // tokens per tile (MMA N)
     static constexpr int STAGES = STAGES_;
     static constexpr int BW = 128;          // weight rows per tile (MMA M)
@@ -43,11 +48,20 @@ struct UmmaCfg {
     static_assert((3 * STAGES + 2) * 8 + 8 <= kBarBytes, "barrier area");
 };
 
+// p[j] with a run-time j without turning the register array into local memory: a chain of selects.
+__device__ __forceinline__ uint32_t p_word(const uint32_t (&p)[16], int j) {
+    uint32_t v = p[0];
+#pragma unroll
+    for (int i = 1; i < 16; ++i) v = (j == i) ? p[i] : v;
+    return v;
+}
+
 template <class Cfg>
 __global__ void __launch_bounds__(Cfg::kThreads)
 linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N][K/2], box 64 x 128, 64B swizzle (W8: FP8 u8 [N][K], box 128 x 128, 128B swizzle)
                    const __grid_constant__ CUtensorMap tmap_x,   // X8     u8 [M][K],   box 128 x BNX, 128B swizzle
                    const uint16_t* __restrict__ gscale, const uint8_t* __restrict__ gzero,
+                   const int32_t* __restrict__ g_idx,   // GIDX: group of every input column, int32 [K]
                    const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                    void* __restrict__ y, int64_t ldy, int out_dtype, float* __restrict__ partial,
                    int M, int N, int K, int kb_per_split, unsigned int* status_word) {
@@ -193,8 +207,11 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
         const uint8_t* z_ptr = gzero ? gzero + (int64_t)(row_ok ? n : 0) * G + kb0 : nullptr;
         const uint32_t sw64 = (uint32_t)((r >> 1) & 3);
         const uint32_t sw128 = (uint32_t)(r & 7);
-        uint32_t sc_next = (row_ok && !Cfg::W8) ? (uint32_t)__ldg(sc_ptr) : 0u;
-        int z_next = (z_ptr && row_ok && !Cfg::W8) ? (int)__ldg(z_ptr) : 8;
+        uint32_t sc_next = (row_ok && !Cfg::W8 && !Cfg::GIDX) ? (uint32_t)__ldg(sc_ptr) : 0u;
+        int z_next = (z_ptr && row_ok && !Cfg::W8 && !Cfg::GIDX) ? (int)__ldg(z_ptr) : 8;
+        // GIDX: this row's scales and zero-points of ALL groups (the look-ups below stay in L1)
+        const uint16_t* sc_row = gscale + (int64_t)(row_ok ? n : 0) * G;
+        const uint8_t* z_row = gzero ? gzero + (int64_t)(row_ok ? n : 0) * G : nullptr;
         bool ok = true;
         for (int it = 0; it < (Cfg::W8 ? 0 : nkb); ++it) {
             const int s = it % STAGES;
@@ -202,12 +219,12 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
             const uint32_t sc_bits = sc_next;
             const float sc = bf16_bits_to_float(sc_next);
             const int z = z_next;
-            if (it + 1 < nkb && row_ok) {
+            if (!Cfg::GIDX && it + 1 < nkb && row_ok) {
                 sc_next = (uint32_t)__ldg(sc_ptr + it + 1);
                 if (z_ptr) z_next = (int)__ldg(z_ptr + it + 1);
             }
             DequantLut lut;
-            if (!Cfg::W16) lut.build(sc, z);
+            if (!Cfg::W16 && !Cfg::GIDX) lut.build(sc, z);
             ok = ptx::mbar_wait(bar_full_tma(s), ph, abort_flag, status_word);
             if (!ok) break;
             const uint32_t src = stage_wp(s) + (uint32_t)r * 64u;
@@ -240,6 +257,32 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap tmap_w,   // codes  u8 [N
                     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(
                                      panel + ((((uint32_t)j & 7u) ^ sw128) << 4)),
                                  "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                                 : "memory");
+                }
+            } else if (Cfg::GIDX) {
+                // Eq. 10 with the scale and zero-point of group g_idx[k], one weight at a time:
+                // word w holds the nibbles of columns 8w .. 8w+7 (even column in the low nibble)
+                const int32_t* gi = g_idx + (int64_t)(kb0 + it) * 128;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const uint32_t word = p_word(p, 2 * c + (h >> 1));
+                        uint32_t out = 0;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int col = 16 * c + 4 * h + e;
+                            const int g = __ldg(gi + col);
+                            const int u = (int)((word >> (4 * ((h & 1) * 4 + e))) & 15u);
+                            const int zz = z_row ? (int)__ldg(z_row + g) : 8;
+                            const float ss = bf16_bits_to_float((uint32_t)__ldg(sc_row + g));
+                            out |= (cvt_e4m3x2(0.0f, __fmul_rn((float)(u - zz), ss)) & 0xFFu) << (8 * e);
+                        }
+                        o[h] = out;
+                    }
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)),
+                                 "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
                                  : "memory");
                 }
             } else {

@@ -1,0 +1,45 @@
+"""GPU: every kernel family of w4a8_linear, launched several times on FRESH zero-filled workspaces and
+fresh outputs, must return the same bits every time, and the first launch must be right (checked
+against a float32 product of the dequantized operands, which is exact enough to expose a tile that
+was summed from stale or missing data).  A repeat on a USED workspace cannot show such an error: a
+kernel that reads partial sums too early finds the previous launch's identical values there.  (This
+is how a barrier-phase hazard in the expansion groups showed up: wrong sums in a few tiles of the
+first launch of a process only.)  Shapes: one per kernel and plan -- split-N with and without a
+K cut, the persistent kernel with 64-, 128- and 256-token tiles as equal slices, as whole CTAs per
+tile and as whole tiles, the 256 x 256 tiles, the two-CTA kernel."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_14638_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(8, 4096, 4096), (16, 14336, 4096), (48, 4096, 4096), (128, 6144, 4096), (128, 4096, 14336),
+          (100, 512, 8192), (200, 4096, 4096), (256, 4096, 14336), (512, 4096, 4096), (512, 6144, 4096),
+          (700, 10576, 640), (1061, 16384, 1024), (2048, 4096, 4096)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_fresh_workspace_launches_agree_and_are_right(M, N, K):
+    dev = torch.device("cuda")
+    W = torch.from_numpy(inputs.make_weight(N, K, 0.02, seed=M + N)).to(dev)
+    codes, gs, gz, sw = binding.quantize_weight_rtn(W, symmetric=True)
+    del W
+    w8 = binding.dequant_weight(codes, gs, gz)
+    tw = binding.prepack_weight(codes, gs, gz, sw)
+    xb = inputs.make_activation(M, K, M + K, 0.01, 20.0)
+    x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+    ref = (x8.view(torch.float8_e4m3fn).float() @ w8.view(torch.float8_e4m3fn).float().t()) * s_x[:, None] * sw
+    outs = []
+    for _ in range(4):
+        ws = binding.new_workspace(M, N, K, tw.fmt, dev)          # zero-filled, never used
+        outs.append(binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32, workspace=ws))
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int32), outs[0].view(torch.int32))
+    # float32 sums of K exact products: agreement to ~1e-5 of the output scale; a misplaced or missing
+    # k-slice of a tile is off by a good fraction of it
+    scale = float(ref.abs().max())
+    assert float((outs[0] - ref).abs().max()) <= 1e-3 * scale

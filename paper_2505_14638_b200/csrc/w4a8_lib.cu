@@ -280,7 +280,7 @@ static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
 template <class Cfg>
 static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                           int sw_stride, void* y, int64_t ldy, int out_dtype, void* workspace, const SkPlan& pl,
-                          int M, int N, int K, cudaStream_t st) {
+                          int M, int N, int K, cudaStream_t st, const CUtensorMap* tw8 = nullptr) {
     auto kern = linear_streamk_kernel<Cfg>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -304,8 +304,9 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, counters, slots, M,
-                                       N, K, pl.TM, pl.TN, aligned, status);
+    // (the second tensor map is read only by the FP8-weight variant)
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, tw8 ? *tw8 : tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
+                                       counters, slots, M, N, K, pl.TM, pl.TN, aligned, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
@@ -727,6 +728,30 @@ static int linear_w8a8_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, i
     CUtensorMap tw, tx;
     if (!make_tmap_u8_2d(&tw, w8, (uint64_t)N, (uint64_t)K, (uint64_t)K, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B))
         return W4A8_ERR_CUDA;
+    {
+        // Many tokens and at least as many 128 x 256 tiles as SMs: the persistent kernel of the W4A8
+        // path with the expansion compiled out (whole tiles per CTA, no workspace) -- the like-for-like
+        // partner of w4a8_linear at prefill sizes.
+        const int sms = sm_count();
+        const int64_t TM = (M + 255) / 256, TN = (N + 127) / 128;
+        if (M > 128 && sms > 0 && TM * TN >= sms) {
+            SkPlan p8;
+            p8.bnx = 256;
+            p8.TM = (int)TM;
+            p8.TN = (int)TN;
+            p8.aligned = 1;
+            p8.U = TM * TN * (K / 128);
+            p8.P = sms;
+            p8.counter_bytes = 0;
+            p8.workspace_bytes = 0;
+            CUtensorMap tx8;
+            if (!make_tmap_u8_2d(&tx8, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, 256, CU_TENSOR_MAP_SWIZZLE_128B))
+                return W4A8_ERR_CUDA;
+            return launch_streamk<SkCfg<256, 4, 4, 3, kFmtTiledSignMag, 1, true>>(tx8, w8, s_x, s_w, sw_stride, y, ldy,
+                                                                                    out_dtype, nullptr, p8, (int)M,
+                                                                                    (int)N, (int)K, st, &tw);
+        }
+    }
     if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)plan.bnx,
                          CU_TENSOR_MAP_SWIZZLE_128B))
         return W4A8_ERR_CUDA;

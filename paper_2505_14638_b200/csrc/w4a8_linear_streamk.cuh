@@ -39,8 +39,12 @@
 namespace w4a8 {
 
 
-template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1>
+// W8 = true (the W8A8 comparison scheme of Sec. 4.3 on this kernel's skeleton): the weights are FP8
+// E4M3 bytes [N][K] already; a TMA tile load puts them straight into the ring of swizzled weight
+// tiles the MMAs read, the expansion groups have nothing to do.  Whole tiles only.
+template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false>
 struct SkCfg {
+    static constexpr bool W8 = W8_;
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
     static constexpr int G = G_;       // dequantization groups of 4 warps
     static constexpr int S1 = S1_;     // ring of TMA stages (packed chunk + activation tile)
@@ -60,6 +64,7 @@ struct SkCfg {
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
     static_assert(RB_ == 1 || (RB_ == 2 && BNX_ == 256), "two row blocks per tile only with 256-token tiles");
+    static_assert(!W8_ || RB_ == 1, "the FP8-weight variant uses one row block per tile");
     // A dequantization group handles every G-th stage, so it skips phases of the barriers it
     // waits on, and an mbarrier wait tells phases apart by parity only: the wait for use k of a
     // slot is sound only if use k-1 has completed before it starts.  That holds because a stage's
@@ -88,6 +93,7 @@ struct SkCfg {
 template <class Cfg>
 __global__ void __launch_bounds__(Cfg::kThreads)
 linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][K], box 128 x BNX, 128B swizzle
+                      const __grid_constant__ CUtensorMap tmap_w,  // W8 only: FP8 weights u8 [N][K], box 128 x 128, 128B swizzle
                       const uint8_t* __restrict__ wpp,             // tiled weights (panels, k-block major)
                       const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                       void* __restrict__ y, int64_t ldy, int out_dtype, unsigned int* counters,
@@ -139,7 +145,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             ptx::mbar_init(bar_free1(s), 1);
         }
         for (int s = 0; s < S2; ++s) {
-            ptx::mbar_init(bar_w8_full(s), 128);
+            ptx::mbar_init(bar_w8_full(s), Cfg::W8 ? 1 : 128);   // (W8: the TMA load's transaction count)
             ptx::mbar_init(bar_free2(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -232,7 +238,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
             // Weights depend on no earlier kernel: the first ring-full of packed tiles is requested
             // before waiting for the kernels that produce the activations.
-            const int ahead = n_it < S1 ? n_it : S1;
+            // (FP8 weights go straight into the operand ring, whose slots are freed by MMAs, and MMAs need
+            // activations: the weight-only prologue may not be longer than that ring)
+            constexpr int kAhead = Cfg::W8 ? (S2 < S1 ? S2 : S1) : S1;
+            const int ahead = n_it < kAhead ? n_it : kAhead;
             ptx::Ring rx;  // ring position of the next activation tile
             int xkb = kb, xmt = mt;
             int it_x = 0;  // activation tiles issued so far
@@ -245,7 +254,19 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 const uint8_t* csrc = wpp + row0 * kRowCodeBytes;
                 const uint8_t* msrc = meta_base + row0 * Cfg::kMeta;
                 const uint32_t cbytes = (uint32_t)(rows * kRowCodeBytes), mbytes = (uint32_t)(rows * Cfg::kMeta);
-                if (ptx::elect_one()) {
+                if constexpr (Cfg::W8) {
+                    // FP8 weights: straight into the ring of MMA operand tiles, once the MMAs that read
+                    // the slot's previous tile have completed (every stage in turn: no phase is skipped)
+                    const int s2 = it % S2;
+                    if (it >= S2) {
+                        ok = ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word);
+                        if (!ok) break;
+                    }
+                    if (ptx::elect_one()) {
+                        ptx::mbar_arrive_expect_tx(bar_w8_full(s2), (uint32_t)Cfg::kW8Bytes);
+                        ptx::tma_load_2d(stage_w8(s2), &tmap_w, kb * 128, nt * TR, bar_w8_full(s2));
+                    }
+                } else if (ptx::elect_one()) {
                     ptx::mbar_arrive_expect_tx(full, cbytes + mbytes);
                     ptx::bulk_load(wdst, csrc, cbytes, full);
                     ptx::bulk_load(wdst + (uint32_t)Cfg::kCodeBytes, msrc, mbytes, full);
@@ -286,8 +307,17 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                         rb.phase ^= 1u;
                     }
                     uint64_t t0 = ptx::globaltimer_ns();
-                    while (!ptx::mbar_try_wait(bar_full(rb.idx), rb.phase) &&
-                           ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
+                    if constexpr (Cfg::W8) {
+                        // (the FP8 tile of stage `st` went to slot st % S2 of the operand ring)
+                        const int st = issued - 1 - i;
+                        if (st >= issued - S2)
+                            while (!ptx::mbar_try_wait(bar_w8_full(st % S2), (uint32_t)((st / S2) & 1)) &&
+                                   ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
+                            }
+                    } else {
+                        while (!ptx::mbar_try_wait(bar_full(rb.idx), rb.phase) &&
+                               ptx::globaltimer_ns() - t0 < ptx::kWaitLimitNs) {
+                        }
                     }
                     const bool x_issued = issued - 1 - i < it_x;  // this stage's activation tile was requested too
                     while (x_issued && !ptx::mbar_try_wait(bar_xfull(rb.idx), rb.phase) &&
@@ -467,7 +497,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
         const int dw = warp - 10;
         const int g = dw >> 2;
         const int r = (dw & 3) * 32 + lane;
-        for (int it = g; it < n_it; it += G) {
+        for (int it = Cfg::W8 ? n_it : g; it < n_it; it += G) {   // (W8: nothing to expand)
             const int s1 = it % S1, s2 = it % S2;
             if (!ptx::mbar_wait(bar_full(s1), (uint32_t)((it / S1) & 1), abort_flag, status_word)) break;
             if (it >= S2) {

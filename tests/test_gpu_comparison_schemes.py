@@ -102,3 +102,29 @@ def test_gidx_linear_in_one_kernel(M, N, K, asym):
     b = binding.linear(dev(x8), dev(s_x), *wd, out_dtype=binding.OUT_FP32, algo=binding.ALGO_UMMA)
     torch.cuda.synchronize()
     assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_w8a8_on_the_persistent_kernel_at_prefill_size():
+    # enough 128 x 256 tiles for every SM: w4a8_linear_w8a8 runs the persistent kernel of the W4A8 path
+    # with the expansion compiled out (FP8 weight tiles by TMA straight into the operand ring).  Ragged
+    # in both directions; against the oracle on sampled channels, and bit for bit against w4a8_linear on
+    # the same FP8 weights (same operands, same k order of the FP32 accumulation).
+    M, N, K = 1900, 5008, 1024
+    rng = np.random.default_rng(7)
+    wq = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 36), symmetric=True)
+    cols = np.unique(np.concatenate([rng.integers(0, N, 300), np.arange(0, N, 128), np.arange(127, N, 128), [N - 1]]))
+    w8 = oracle.dequant_weight(*wq[:3])
+    x8, s_x = oracle.quantize_act(inputs.make_activation(M, K, 37, 0.01, 20.0))
+    ref = oracle.linear(x8, s_x, w8, wq[3], cols=cols, want=("y64",))
+    wd = weights_to_dev(*wq)
+    y8 = binding.linear_w8a8(dev(x8), dev(s_x), dev(w8), dev(wq[3]), out_dtype=binding.OUT_FP32)
+    y8b = binding.linear_w8a8(dev(x8), dev(s_x), dev(w8), dev(wq[3]), out_dtype=binding.OUT_BF16)
+    tw = binding.prepack_weight(*wd)
+    y4 = binding.linear_tiled(dev(x8), dev(s_x), tw, out_dtype=binding.OUT_FP32)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    worst, _ = fp32_gate(y8.cpu().numpy()[:, cols], ref["y64"], rel=2e-3)
+    assert worst <= 2e-3, worst
+    ok, dist = bf16_gate(bf16_bits(y8b)[:, cols], ref["y64"])
+    assert ok, dist
+    assert torch.equal(y8.view(torch.int32), y4.view(torch.int32))

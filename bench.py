@@ -911,12 +911,13 @@ def scheme_sweep(torch, binding, inputs, dev):
 
     for name, k, n in C5_LAYERS:
         copies = max(2, min(16, int(2.2 * 126e6 / (n * k)) + 1))     # FP8 copies: 1 byte per weight
-        tws, w8s, raw = [], [], []
+        tws, w8s, raw, tw8s = [], [], [], []
         for c in range(copies):
             W = torch.from_numpy(inputs.make_weight(n, k, SIGMA, seed=8000 + c)).to(dev)
             q = binding.quantize_weight_rtn(W, symmetric=True)
             tws.append(binding.prepack_weight(*q))
             w8s.append(binding.dequant_weight(*q[:3]))
+            tw8s.append(binding.prepack_fp8(w8s[-1], q[3]))
             raw.append(q)
             del W
         g_idx = (torch.randperm(k, device=dev) // GROUP).to(torch.int32)   # an unconstrained column order
@@ -954,12 +955,25 @@ def scheme_sweep(torch, binding, inputs, dev):
                 cq = raw[c % copies]
                 binding.linear_w4a16(x, cq[0], cq[1], None, cq[3], out=y, workspace=ws16)
             t_16 = graph_time(w4a16, reps)
+            # decode sizes: both schemes as problems of a w4a8_linear_chain launch (same kernel, partition and
+            # MMAs; the FP8 weights are copied to tensor memory where the INT4 codes are expanded)
+            t_c4 = t_c8 = None
+            if m <= binding.CHAIN_MAX_M:
+                nprob = 12
+                yc = torch.empty((m, n), dtype=torch.bfloat16, device=dev)
+                c4 = binding.LinearChain([dict(x=x, weight=tws[j % copies], y=yc) for j in range(nprob)])
+                c8 = binding.LinearChain([dict(x=x, weight=tw8s[j % copies], y=yc) for j in range(nprob)])
+                t_c4 = _time_loop(torch, c4, 10, warm=3) / nprob
+                t_c8 = _time_loop(torch, c8, 10, warm=3) / nprob
+                del c4, c8
             out.append({"layer": name, "K": k, "N": n, "M": m, "w4a8_us": t_w4 * 1e6, "w8a8_own_kernel_us": t_w8 * 1e6,
                         "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6,
                         "w4a8_act_order_one_kernel_us": t_aof * 1e6, "w4a8_same_tile_kernel_group_order_us": t_tile * 1e6,
-                        "w4a16_own_kernel_us": t_16 * 1e6})
+                        "w4a16_own_kernel_us": t_16 * 1e6,
+                        "w4a8_chain_us_per_problem": None if t_c4 is None else t_c4 * 1e6,
+                        "w8a8_chain_us_per_problem": None if t_c8 is None else t_c8 * 1e6})
             del x, x8, s_x, y, ws
-        del tws, w8s, raw, w8_tmp
+        del tws, w8s, raw, w8_tmp, tw8s
         torch.cuda.empty_cache()
     if binding.query_device_status() != 0:
         raise RuntimeError("device status word set during the sweep")

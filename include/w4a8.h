@@ -70,6 +70,7 @@ extern "C" {
 #define W4A8_FMT_CANONICAL 0
 #define W4A8_FMT_TILED 1
 #define W4A8_FMT_TILED_SIGNMAG 2
+#define W4A8_FMT_TILED_FP8 3 /* FP8 E4M3 weights, tiled by w4a8_prepack_fp8: the W8A8 comparison scheme in w4a8_linear_chain */
 
 /*
  * Activation FP8 quantization, Eq. 13 (with Eq. 3), one scale per token:
@@ -136,6 +137,16 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
  * (w4a8_query_device_status) and the buffer must not be used.
  */
 size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format);
+
+/*
+ * W8A8 comparison scheme (Sec. 4.3, Fig. 4) for the chain launch: re-layout (no arithmetic) of FP8
+ * E4M3 weights w8 [N][K] -- e.g. the output of w4a8_dequant_weight -- into the tiled order
+ * [K/128][N/8][8 chunks][8 rows][16 bytes] (N * K bytes, 128-byte aligned) that
+ * w4a8_linear_chain reads with weight_format W4A8_FMT_TILED_FP8: the same kernel, partition and
+ * MMAs as for the INT4 formats, the expansion replaced by a copy -- twice the weight bytes, no
+ * integer work.  N % 16 == 0, K % 128 == 0.
+ */
+int w4a8_prepack_fp8(const uint8_t* w8, int64_t N, int64_t K, uint8_t* out, size_t out_bytes, void* stream);
 int w4a8_prepack_weight(const uint8_t* codes, const void* gscale_bf16, const uint8_t* gzero, int64_t N,
                         int64_t K, int group, int weight_format, uint8_t* out, size_t out_bytes,
                         void* stream);

@@ -19,7 +19,7 @@ ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 SCALE_EXACT, SCALE_POW2 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 ALGO_AUTO, ALGO_SIMT, ALGO_UMMA = 0, 1, 2
-FMT_CANONICAL, FMT_TILED, FMT_TILED_SIGNMAG = 0, 1, 2
+FMT_CANONICAL, FMT_TILED, FMT_TILED_SIGNMAG, FMT_TILED_FP8 = 0, 1, 2, 3
 GROUP = 128
 
 # Every symbol include/w4a8.h declares.
@@ -27,7 +27,7 @@ EXPORTS = (
     "w4a8_quantize_act", "w4a8_dequant_weight", "w4a8_linear", "w4a8_linear_workspace_bytes",
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
-    "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx", "w4a8_linear_gidx",
+    "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx", "w4a8_linear_gidx", "w4a8_prepack_fp8",
     "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
@@ -99,6 +99,8 @@ def lib():
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
     L.w4a8_dequant_weight_gidx.restype = i32
     L.w4a8_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p, p]
+    L.w4a8_prepack_fp8.restype = i32
+    L.w4a8_prepack_fp8.argtypes = [p, i64, i64, p, sz, p]
     L.w4a8_linear_gidx.restype = i32
     L.w4a8_linear_gidx.argtypes = [p, i64, p, i64, p, p, p, p, p, i32, i64, i64, i32, p, i64, i32, p, sz, p]
     L.w4a8_linear_w8a8.restype = i32
@@ -266,6 +268,16 @@ def prepack_weight(codes, gscale, gzero, s_w, weight_format=None):
                                    int(weight_format), _ptr(buf), nbytes, _stream())
     _check("w4a8_prepack_weight", rc)
     return TiledWeight(buf, weight_format, N, K, s_w)
+
+
+def prepack_fp8(w8, s_w):
+    """w4a8_prepack_fp8: FP8 E4M3 weights [N, K] (uint8) -> TiledWeight of format FMT_TILED_FP8, the W8A8
+    comparison scheme for LinearChain."""
+    import torch
+    N, K = w8.shape
+    buf = torch.empty((N * K,), dtype=torch.uint8, device=w8.device)
+    _check("w4a8_prepack_fp8", lib().w4a8_prepack_fp8(_ptr(w8), N, K, _ptr(buf), N * K, _stream()))
+    return TiledWeight(buf, FMT_TILED_FP8, N, K, s_w)
 
 
 def new_workspace(M, N, K, weight_format=FMT_CANONICAL, device="cuda"):

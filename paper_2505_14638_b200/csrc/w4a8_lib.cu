@@ -963,7 +963,8 @@ static int chain_validate(const w4a8_chain_problem* pr, int count) {
         if (q.input_kind != kChainKindPlain && q.input_kind != kChainKindSiluMul) return W4A8_ERR_INVALID_ARG;
         if (q.depends_on < -1 || q.depends_on >= i) return W4A8_ERR_INVALID_ARG;
         if (q.scale_mode != W4A8_SCALE_EXACT && q.scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
-        if (q.weight_format != kFmtTiled && q.weight_format != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+        if (q.weight_format != kFmtTiled && q.weight_format != kFmtTiledSignMag && q.weight_format != kFmtTiledFp8)
+            return W4A8_ERR_INVALID_ARG;
         if (q.weight_format != pr[0].weight_format) return W4A8_ERR_INVALID_ARG;
         if (q.sw_stride != 0 && q.sw_stride != 1) return W4A8_ERR_INVALID_ARG;
         if (q.out_dtype != W4A8_OUT_BF16 && q.out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
@@ -1081,7 +1082,7 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
         if (2 * (int)q.K > stash) stash = 2 * (int)q.K;
     }
     // a slot holds the two (k-block, block) items of a stage: 2 x 96 rows of codes and meta data
-    prm.wslot = (2 * kChainBlockRows * (kRowCodeBytes + mb) + 127) / 128 * 128;
+    prm.wslot = (2 * kChainBlockRows * (row_bytes(fmt) + mb) + 127) / 128 * 128;
     prm.stash = stash;
     using C0 = ChainCfg<4, kFmtTiledSignMag>;
     const int fixed = 1024 + C0::kXRingBytes + stash + C0::kBarBytes + C0::kSegBytes;
@@ -1095,6 +1096,8 @@ static int linear_chain_impl(const w4a8_chain_problem* pr, int count, void* work
 #define W4A8_CHAIN(GG)                                                                             \
     (fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<GG, kFmtTiledSignMag>>(prm, sms, smem, ws, st) \
                              : launch_chain<ChainCfg<GG, kFmtTiled>>(prm, sms, smem, ws, st))
+    if (fmt == kFmtTiledFp8)   // the W8A8 comparison scheme: one instantiation (four groups, everything compiled in)
+        return launch_chain<ChainCfg<4, kFmtTiledFp8, true>>(prm, sms, smem, ws, st);
     if (groups == 4 && !full)
         return fmt == kFmtTiledSignMag ? launch_chain<ChainCfg<4, kFmtTiledSignMag, false>>(prm, sms, smem, ws, st)
                                        : launch_chain<ChainCfg<4, kFmtTiled, false>>(prm, sms, smem, ws, st);
@@ -1172,8 +1175,22 @@ size_t w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int weight_f
     return M <= kSplitNMaxM && pl.workspace_bytes < kSnWorkspaceBytes ? kSnWorkspaceBytes : pl.workspace_bytes;
 }
 
+int w4a8_prepack_fp8(const uint8_t* w8, int64_t N, int64_t K, uint8_t* out, size_t out_bytes, void* stream) {
+    if (!w8 || !out || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (K % kGroup != 0 || N % 16 != 0) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(w8) || (reinterpret_cast<uintptr_t>(out) & 127u)) return W4A8_ERR_BAD_ALIGNMENT;
+    if (out_bytes < (size_t)N * (size_t)K) return W4A8_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int64_t chunks = N * (K / 16);
+    prepack_fp8_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(w8, N, K, out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
 size_t w4a8_prepack_bytes(int64_t N, int64_t K, int weight_format) {
     if (N <= 0 || K <= 0 || K % kGroup != 0) return 0;
+    if (weight_format == kFmtTiledFp8) return (size_t)N * (size_t)K;
     if (weight_format != kFmtTiled && weight_format != kFmtTiledSignMag) return 0;
     return (size_t)N * (size_t)(K / 128) * (size_t)(kRowCodeBytes + meta_bytes(weight_format));
 }

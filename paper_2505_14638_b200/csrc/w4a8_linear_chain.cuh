@@ -124,6 +124,7 @@ struct ChainCfg {
     static constexpr int kNAcc = 4;       // accumulator buffers (two blocks of 16 columns each): segments the MMAs may run ahead of the epilogue
     static constexpr int kS2 = kNAcc == 4 ? 6 : 7;   // stages of expanded weights in tensor memory = activation-tile slots
     static constexpr int kMeta = meta_bytes(FMT_);
+    static constexpr int kRowBytes = row_bytes(FMT_);   // bytes of one row of one k-block in the weight buffer
     static constexpr int kAStageCols = 64;                    // two items of 32 columns
     static constexpr int kDCol = kS2 * kAStageCols;           // 448: accumulators behind the A ring
     static constexpr int kTmemCols = 512;
@@ -439,13 +440,14 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
             const ChainProblem& q = prm.prob[i];
             const int nseg = nseg_tab[i];
             const int KB = q.K >> 7;
-            const int64_t code_step = (int64_t)q.N * kRowCodeBytes;   // one k-block further
+            constexpr int RBY = Cfg::kRowBytes;
+            const int64_t code_step = (int64_t)q.N * RBY;   // one k-block further
             const int64_t meta_step = (int64_t)q.N * MB;
             for (int j = 0; j < nseg && ok; ++j) {
                 const ChainSeg sg = seg_tab[i * kChainMaxSegs + j];
                 const int KS = 2 / sg.NB;
-                const uint32_t cbytes = (uint32_t)(sg.R * kRowCodeBytes), mbytes = (uint32_t)(sg.R * MB);
-                const uint8_t* cptr = q.wpp + (int64_t)sg.kb0 * code_step + (int64_t)sg.n0 * kRowCodeBytes;
+                const uint32_t cbytes = (uint32_t)(sg.R * RBY), mbytes = (uint32_t)(sg.R * MB);
+                const uint8_t* cptr = q.wpp + (int64_t)sg.kb0 * code_step + (int64_t)sg.n0 * RBY;
                 const uint8_t* mptr = q.wpp + (int64_t)KB * code_step + (int64_t)sg.kb0 * meta_step + (int64_t)sg.n0 * MB;
                 const uint32_t meta_off = (uint32_t)KS * cbytes;
                 for (int kb = 0; kb < sg.nkb;) {
@@ -461,10 +463,10 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                     if (ptx::elect_one()) {
                         ptx::mbar_arrive_expect_tx(full, (uint32_t)ks * (cbytes + mbytes));
                         ptx::bulk_load(wdst, cptr, cbytes, full);
-                        ptx::bulk_load(mdst, mptr, mbytes, full);
+                        if (MB > 0) ptx::bulk_load(mdst, mptr, mbytes, full);
                         if (ks == 2) {
                             ptx::bulk_load(wdst + cbytes, cptr1, cbytes, full);
-                            ptx::bulk_load(mdst + mbytes, mptr1, mbytes, full);
+                            if (MB > 0) ptx::bulk_load(mdst + mbytes, mptr1, mbytes, full);
                         }
                     }
                     cptr += code_step * ks;
@@ -945,10 +947,10 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                 const int row1 = BR + r < sg.R ? BR + r : sg.R - 1;
                 const bool have0 = qd * 32 < Rb0;
                 const bool have1 = NB == 2 ? BR + qd * 32 < sg.R : have0;
-                const uint32_t code_off = tiled_row_offset(row0);
-                const uint32_t meta_off = (uint32_t)(KS * sg.R * kRowCodeBytes + row0 * MB);
-                const uint32_t code_kstep = (uint32_t)(sg.R * kRowCodeBytes), meta_kstep = (uint32_t)(sg.R * MB);
-                const uint32_t code_s0 = NB == 2 ? tiled_row_offset(row1) - code_off : code_kstep;
+                const uint32_t code_off = row_offset(Cfg::FMT, row0);
+                const uint32_t meta_off = (uint32_t)(KS * sg.R * Cfg::kRowBytes + row0 * MB);
+                const uint32_t code_kstep = (uint32_t)(sg.R * Cfg::kRowBytes), meta_kstep = (uint32_t)(sg.R * MB);
+                const uint32_t code_s0 = NB == 2 ? row_offset(Cfg::FMT, row1) - code_off : code_kstep;
                 const uint32_t meta_s0 = NB == 2 ? (uint32_t)((row1 - row0) * MB) : meta_kstep;
                 int st = turn;
                 for (; st < nst; st += G) {
@@ -968,7 +970,11 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                     ptx::tc_fence_after_sync();
                     const uint32_t wsrc = w_ring + (uint32_t)(r1.idx * prm.wslot);
                     const uint32_t a_col = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(r2.idx * Cfg::kAStageCols);
-                    if (ks * NB == 2) {
+                    if constexpr (Cfg::FMT == kFmtTiledFp8) {
+                        // FP8 weights: nothing to expand, the rows go to tensor memory as they are
+                        if (have0) copy_fp8_row_to_tmem(wsrc + code_off, a_col);
+                        if (ks * NB == 2 && have1) copy_fp8_row_to_tmem(wsrc + code_off + code_s0, a_col + 32u);
+                    } else if (ks * NB == 2) {
                         if (have1)
                             dequant_two_rows_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, wsrc + code_off + code_s0,
                                                                wsrc + meta_off + meta_s0, a_col);

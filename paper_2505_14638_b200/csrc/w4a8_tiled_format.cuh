@@ -24,6 +24,7 @@ namespace w4a8 {
 constexpr int kFmtCanonical = W4A8_FMT_CANONICAL;
 constexpr int kFmtTiled = W4A8_FMT_TILED;
 constexpr int kFmtTiledSignMag = W4A8_FMT_TILED_SIGNMAG;
+constexpr int kFmtTiledFp8 = W4A8_FMT_TILED_FP8;   // FP8 weights (W8A8 comparison scheme): 128 bytes per row and k-block, no meta data
 
 constexpr int kRowCodeBytes = 64;  // one row of one k-block: 128 INT4 codes
 constexpr uint32_t kChunkStride = 128;  // bytes between two chunks of one row
@@ -31,7 +32,13 @@ constexpr uint32_t kChunkStride = 128;  // bytes between two chunks of one row
 __host__ __device__ constexpr uint32_t tiled_row_offset(int row) {
     return (uint32_t)(row >> 3) * 512u + (uint32_t)(row & 7) * 16u;
 }
-__host__ __device__ constexpr int meta_bytes(int fmt) { return fmt == kFmtTiledSignMag ? 2 : 4; }
+__host__ __device__ constexpr int meta_bytes(int fmt) { return fmt == kFmtTiledSignMag ? 2 : (fmt == kFmtTiledFp8 ? 0 : 4); }
+// Bytes of one row of one k-block, and the offset of a row's first 16-byte chunk within a piece that
+// starts on a multiple of eight rows (chunk c of the row sits c * 128 bytes further), per format.
+__host__ __device__ constexpr int row_bytes(int fmt) { return fmt == kFmtTiledFp8 ? 128 : kRowCodeBytes; }
+__host__ __device__ constexpr uint32_t row_offset(int fmt, int row) {
+    return fmt == kFmtTiledFp8 ? (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 16u : tiled_row_offset(row);
+}
 
 // Sign-magnitude table of a symmetric group (z = 8): entry d = nearest_E4M3(d * s), d = 0..7.
 // A stored nibble carries |u - 8| in its low three bits; the sign travels separately and is
@@ -139,6 +146,31 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t src, uint32_t meta,
             ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
         }
     }
+}
+
+// FP8 weights (W8A8 comparison scheme): the row's 128 bytes of the k-block go to tensor memory as they are.
+__device__ __forceinline__ void copy_fp8_row_to_tmem(uint32_t src, uint32_t taddr) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t out[16];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(out[4 * c]), "=r"(out[4 * c + 1]), "=r"(out[4 * c + 2]), "=r"(out[4 * c + 3])
+                         : "r"(src + (uint32_t)(4 * h + c) * kChunkStride));
+        ptx::tmem_st_32x32b_x16(taddr + 16u * h, out);
+    }
+}
+
+// [N][K] FP8 bytes -> tiled order (one thread per 16-byte chunk).
+__global__ void prepack_fp8_kernel(const uint8_t* __restrict__ w8, int64_t N, int64_t K, uint8_t* __restrict__ out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // chunk index: n * (K / 16) + k / 16
+    const int64_t cpr = K >> 4;
+    if (i >= N * cpr) return;
+    const int64_t n = i / cpr, ck = i - n * cpr;
+    const int64_t kb = ck >> 3, c = ck & 7;
+    const uint4 v = *reinterpret_cast<const uint4*>(w8 + n * K + ck * 16);
+    *reinterpret_cast<uint4*>(out + (kb * N + (n & ~(int64_t)7)) * 128 + c * 128 + (n & 7) * 16) = v;
 }
 
 // The expansion of one row whose codes and meta word are already in registers.

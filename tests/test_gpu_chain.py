@@ -334,3 +334,32 @@ def test_output_rows_that_are_not_16_byte_aligned(dtype, pad):
         assert torch.equal(buf[:, :N].contiguous().view(torch.uint8), yc.view(torch.uint8))
         assert bool((buf[:, N:] == 7.0).all())
         assert bool(torch.isfinite(yc.float()).all()) and float(yc.float().abs().max()) > 0
+
+
+def test_w8a8_comparison_scheme_in_the_chain_kernel():
+    # FP8 weights (the dequantized weights of the same layers, tiled by w4a8_prepack_fp8) through the same
+    # launch, partition and MMAs, the expansion replaced by a copy: outputs must equal those of the INT4
+    # problems bit for bit (same FP8 operands, same accumulation order), and match the oracle.
+    shapes = [(1, 2368, 640), (16, 1024, 1024), (7, 48, 256), (4, 14336, 512)]
+    p4, p8, refs = [], [], []
+    for i, (M, N, K) in enumerate(shapes):
+        wq, tw = _weights(N, K, 400 + i)
+        wd = weights_to_dev(*wq)
+        tw8 = binding.prepack_fp8(binding.dequant_weight(*wd[:3]), wd[3])
+        xb = inputs.make_activation(M, K, 410 + i, 0.01, 20.0)
+        x = bf16_dev(xb)
+        p4.append(dict(x=x, weight=tw, y=torch.zeros((M, N), dtype=torch.float32, device="cuda")))
+        p8.append(dict(x=x, weight=tw8, y=torch.zeros((M, N), dtype=torch.float32, device="cuda")))
+        refs.append((xb, wq))
+    binding.LinearChain(p4)()
+    binding.LinearChain(p8)()
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    for a, b, (xb, wq) in zip(p4, p8, refs):
+        assert torch.equal(a["y"].view(torch.int32), b["y"].view(torch.int32))
+        _, _, ref = _oracle_layer(xb, wq)
+        worst, _ = fp32_gate(b["y"].cpu().numpy(), ref["y64"], rel=2e-3)
+        assert worst <= 2e-3, worst
+    # formats may not be mixed within a launch
+    with pytest.raises(binding.W4A8Error):
+        binding.LinearChain([p4[0], p8[1]])()

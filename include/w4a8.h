@@ -221,8 +221,10 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  *                every row of that output has been written.  Buffers of problems that are not
  *                linked this way must not overlap.
  *   scale_mode, static_scale    as in w4a8_quantize_act.
- *   weights      device, output of w4a8_prepack_weight; one tiled weight_format for the whole
- *                chain.  K % 128 == 0, K <= 16384, N % 16 == 0, N <= 1152 rows per SM.
+ *   weights      device, output of w4a8_prepack_weight (W4A8_FMT_TILED, W4A8_FMT_TILED_SIGNMAG) or, for
+ *                the W8A8 comparison scheme, of w4a8_prepack_fp8 (W4A8_FMT_TILED_FP8: the weights are
+ *                FP8 bytes, copied instead of expanded); one weight_format for the whole chain.
+ *                K % 128 == 0, K <= 16384, N % 16 == 0, N <= 1152 rows per SM.
  *   x8_out / s_x_out  optional (NULL): row-major copies of the FP8 activations [M][ldx8_out] and
  *                of the M scales the layer multiplied with.
  * workspace: device, 128-byte aligned, w4a8_linear_chain_workspace_bytes(problems, count) bytes:

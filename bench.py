@@ -980,19 +980,12 @@ def scheme_sweep(torch, binding, inputs, dev):
     return out
 
 
-def _hessian_upper_cholesky(H, perm=None, damp=0.01):
-    """Upper Cholesky factor of the inverse of the dampened Hessian in processing order (Sec. 3.3,
-    as in GPTQ), with torch.linalg in float64: an input of w4a8_dpq_quantize, prepared by the caller."""
+def _inverse_factor(Hp):
+    """Upper Cholesky factor of the inverse of the prepared Hessian (the output of w4a8_hessian_prepare;
+    Sec. 3.3, as in GPTQ), with torch.linalg in float64: the library step between the Hessian and
+    w4a8_dpq_quantize, which is the caller's."""
     import torch
-    H = H.to(torch.float64)
-    if perm is not None:
-        idx = perm.to(torch.int64)
-        H = H[idx][:, idx]
-    H = H.clone()
-    d = torch.diagonal(H)
-    d[d == 0] = 1.0
-    d += damp * d.mean()
-    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(H))
+    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(Hp.to(torch.float64)))
     Hinv = 0.5 * (Hinv + Hinv.T)
     return torch.linalg.cholesky(Hinv, upper=True).to(torch.float32).contiguous()
 
@@ -1007,12 +1000,17 @@ def dpq_sweep(torch, binding, inputs, dev):
     for name, k, n in (("o", 4096, 4096), ("gate_up", 4096, 28672), ("down", 14336, 4096)):
         W = torch.from_numpy(inputs.make_weight(n, k, SIGMA, seed=9000)).to(dev)
         xb = inputs.make_activation(1024, k, 9001, OUTLIER_FRAC, OUTLIER_MULT)
-        X = torch.from_numpy(inputs.bf16_bits_to_f32(xb)).to(dev).to(torch.float64)
-        X += 0.5 * torch.randn((1024, 1), dtype=torch.float64, device=dev)
+        X = torch.from_numpy(inputs.bf16_bits_to_f32(xb)).to(dev)
+        X = (X + 0.5 * torch.randn((1024, 1), dtype=torch.float32, device=dev)).to(torch.bfloat16)   # calibration tokens
+        binding.hessian_accumulate(X)             # warm-up
+        torch.cuda.synchronize()
         t0 = time.perf_counter()
-        H = X.T @ X
-        perm = binding.gar_permutation(torch.diagonal(H).to(torch.float32).contiguous())
-        U = _hessian_upper_cholesky(H, perm)   # the caller's library step: the factor is an input of the quantizer
+        H = binding.hessian_accumulate(X)         # H = X^T X (Sec. 3.1)
+        perm = binding.gar_permutation(torch.diagonal(H).contiguous())
+        Hp = binding.hessian_prepare(H, perm, damp=0.01)     # processing order, dead features, dampening (Sec. 3.3)
+        torch.cuda.synchronize()
+        t_hess = time.perf_counter() - t0
+        U = _inverse_factor(Hp)   # the caller's library step: the factor is an input of the quantizer
         torch.cuda.synchronize()
         t_prep = time.perf_counter() - t0
         binding.dpq_quantize(W, U, perm, symmetric=False, mse_steps=6)   # warm-up
@@ -1035,7 +1033,7 @@ def dpq_sweep(torch, binding, inputs, dev):
         t_cpu = time.perf_counter() - c0
         same = bool(np.array_equal(q[0][ridx].cpu().numpy(), ref[0]))
         rows.append({"layer": name, "K": k, "N": n, "dpq_ms": t * 1e3, "fma_per_s": fmas / t,
-                     "frac_of_fp32_fma_peak": fmas / t / fma_peak, "hessian_and_factor_s": t_prep,
+                     "frac_of_fp32_fma_peak": fmas / t / fma_peak, "hessian_and_factor_s": t_prep, "hessian_kernels_s": t_hess,
                      "oracle_slab_rows": slab, "oracle_slab_s": t_cpu, "oracle_full_layer_s_extrapolated":
                          t_cpu * n / slab, "oracle_cores": oracle.num_threads(), "slab_codes_equal": same})
         del W, X, H, U, q

@@ -388,6 +388,26 @@ int w4a8_quantize_weight_rtn(const float* W, int64_t N, int64_t K, int group, in
                              uint8_t* gzero, float* s_w, void* stream);
 
 /*
+ * The layer Hessian the quantizer works with (Sec. 3.1; prepared as in Sec. 3.3): H = X^T X over the T
+ * calibration tokens of the layer's input X (device BF16 [T][ldx]), FP32 sums, written as a full
+ * symmetric matrix (device float [K][K]); accumulate != 0 adds to what H holds (batches of tokens).
+ * Its diagonal is what w4a8_gar_permutation ranks by.  K <= 32768.
+ */
+int w4a8_hessian_accumulate(const void* x_bf16, int64_t T, int64_t K, int64_t ldx, float* H, int accumulate,
+                            void* stream);
+
+/*
+ * Sec. 3.3 (dampening as in GPTQ): H_out = the Hessian in processing order -- rows and columns
+ * permuted by perm (device int32 [K] from w4a8_gar_permutation, or NULL) --, with a unit diagonal
+ * for input features whose diagonal entry is zero, and damp * mean(diag) added to the diagonal
+ * (the mean taken after the unit-diagonal rule).  scratch: one device float.  H_out != H.
+ * What remains between this matrix and the factor U that w4a8_dpq_quantize takes -- the inverse
+ * and its upper Cholesky factor -- is a library factorization and the caller's.
+ */
+int w4a8_hessian_prepare(const float* H, int64_t K, const int32_t* perm, float damp, float* H_out, float* scratch,
+                         void* stream);
+
+/*
  * Group-Aware Reordering (Sec. 3.2 and its appendix): the order in which the DPQ quantizer
  * processes the input features, from the diagonal of the Hessian H = X^T X.  Inside each group
  * of 128 the columns go by descending diagonal, the groups by descending maximum diagonal (the
@@ -407,8 +427,9 @@ int w4a8_gar_permutation(const float* hdiag, int64_t K, int group, int32_t* perm
  * Produces the same stored format as w4a8_quantize_weight_rtn, in the ORIGINAL column order.
  *   W     device fp32 [N][K], 16-byte aligned.
  *   U     device fp32 [K][K]: upper Cholesky factor of the inverse of the (dampened) Hessian with
- *         rows and columns in processing order; only the upper triangle is read.  Computing it
- *         (H = X^T X, dampening, factorizations) is a library matter and the caller's.
+ *         rows and columns in processing order; only the upper triangle is read.  H = X^T X and its
+ *         preparation are w4a8_hessian_accumulate / w4a8_hessian_prepare; the two factorizations
+ *         in between (inverse, Cholesky) are a library matter and the caller's.
  *   perm  device int32 [K] from w4a8_gar_permutation, or NULL for the original order.  Every run
  *         of 128 positions must hold the columns of one original group (not checked on the device).
  *   symmetric / per_channel   as in w4a8_quantize_weight_rtn (gzero may be NULL when symmetric).

@@ -177,10 +177,16 @@ def gar_permutation(diag, group=128):
     return np.concatenate([within[g] for g in gorder]).astype(np.int32)
 
 
-def hessian_upper_cholesky(H, perm=None, damp=0.01):
-    """What Sec. 3.3 takes from GPTQ, in float64: permute the Hessian to processing order, add
-    damp * mean(diag) to the diagonal, invert, and return the upper Cholesky factor U of the
-    inverse (H^-1 = U^T U) as float32.  Columns with a zero diagonal get a unit diagonal."""
+def hessian(x_bf16) -> np.ndarray:
+    """The layer Hessian of Sec. 3.1 (up to the constant factor that cancels in the update of
+    Eq. 12): H = X^T X over the calibration tokens, X given as BF16 bits [T, K]; float64."""
+    X = bf16_to_f32(x_bf16).astype(np.float64)
+    return X.T @ X
+
+
+def hessian_prepare(H, perm=None, damp=0.01) -> np.ndarray:
+    """Sec. 3.3 (as in GPTQ), float64: the Hessian in processing order, a unit diagonal for columns
+    whose diagonal entry is zero, damp * mean(diag) added to the diagonal."""
     H = np.array(H, dtype=np.float64)
     if perm is not None:
         H = H[np.ix_(perm, perm)]
@@ -188,6 +194,13 @@ def hessian_upper_cholesky(H, perm=None, damp=0.01):
     dead = d == 0
     H[dead, dead] = 1.0
     H[np.diag_indices_from(H)] += damp * np.mean(np.diag(H))
+    return H
+
+
+def hessian_upper_cholesky(H, perm=None, damp=0.01):
+    """What Sec. 3.3 takes from GPTQ, in float64: the prepared Hessian (hessian_prepare) inverted,
+    and the upper Cholesky factor U of the inverse (H^-1 = U^T U) as float32."""
+    H = hessian_prepare(H, perm, damp)
     Hinv = np.linalg.inv(H)
     Hinv = 0.5 * (Hinv + Hinv.T)
     L = np.linalg.cholesky(Hinv)          # Hinv = L L^T

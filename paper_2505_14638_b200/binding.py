@@ -28,6 +28,7 @@ EXPORTS = (
     "w4a8_prepack_bytes", "w4a8_prepack_weight",
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
     "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx", "w4a8_linear_gidx", "w4a8_prepack_fp8",
+    "w4a8_hessian_accumulate", "w4a8_hessian_prepare",
     "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
@@ -99,6 +100,10 @@ def lib():
     L.w4a8_linear_static_scratch.argtypes = [p, i64, p, i64, p, p, p, p, i32, i64, i64, i32, p, i64, i32, i32, p]
     L.w4a8_dequant_weight_gidx.restype = i32
     L.w4a8_dequant_weight_gidx.argtypes = [p, p, p, p, i64, i64, i64, p, p]
+    L.w4a8_hessian_accumulate.restype = i32
+    L.w4a8_hessian_accumulate.argtypes = [p, i64, i64, i64, p, i32, p]
+    L.w4a8_hessian_prepare.restype = i32
+    L.w4a8_hessian_prepare.argtypes = [p, i64, p, ctypes.c_float, p, p, p]
     L.w4a8_prepack_fp8.restype = i32
     L.w4a8_prepack_fp8.argtypes = [p, i64, i64, p, sz, p]
     L.w4a8_linear_gidx.restype = i32
@@ -268,6 +273,28 @@ def prepack_weight(codes, gscale, gzero, s_w, weight_format=None):
                                    int(weight_format), _ptr(buf), nbytes, _stream())
     _check("w4a8_prepack_weight", rc)
     return TiledWeight(buf, weight_format, N, K, s_w)
+
+
+def hessian_accumulate(x, H=None):
+    """w4a8_hessian_accumulate: x BF16 [T, K] on the device; returns H float32 [K, K] (H = X^T X, added to H if given)."""
+    import torch
+    T, K = x.shape
+    acc = H is not None
+    if H is None:
+        H = torch.empty((K, K), dtype=torch.float32, device=x.device)
+    _check("w4a8_hessian_accumulate", lib().w4a8_hessian_accumulate(_ptr(x), T, K, x.stride(0), _ptr(H), int(acc), _stream()))
+    return H
+
+
+def hessian_prepare(H, perm=None, damp=0.01):
+    """w4a8_hessian_prepare: the Hessian in processing order with the dead-feature rule and the dampening."""
+    import torch
+    K = H.shape[0]
+    out = torch.empty_like(H)
+    scratch = torch.empty((1,), dtype=torch.float32, device=H.device)
+    _check("w4a8_hessian_prepare", lib().w4a8_hessian_prepare(_ptr(H), K, _ptr(perm), ctypes.c_float(damp), _ptr(out),
+                                                             _ptr(scratch), _stream()))
+    return out
 
 
 def prepack_fp8(w8, s_w):

@@ -276,4 +276,103 @@ dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The layer Hessian of the quantizer (Sec. 3.1; Sec. 3.3 for its preparation): H = X^T X over the
+// calibration tokens.  A plain FP32 contraction on the FMA pipes -- an offline step whose sums
+// decide nothing bit-exactly (the factorization that follows is a library matter in float64).
+// One CTA per 64 x 64 tile of the upper triangle (tiles below the diagonal are mirrored on the
+// way out); 256 threads, 4 x 4 outputs each; the token dimension in slabs of 32 rows staged in
+// shared memory as fp32.
+// ---------------------------------------------------------------------------------------------
+constexpr int kHessTile = 64, kHessSlab = 32;
+__global__ void __launch_bounds__(256)
+hessian_xtx_kernel(const uint16_t* __restrict__ x, int64_t T, int64_t K, int64_t ldx, float* __restrict__ H,
+                   float beta) {
+    // tile (bi, bj) with bj >= bi, enumerated row by row of the upper triangle
+    const int nb = (int)((K + kHessTile - 1) / kHessTile);
+    int bi = 0, rem = (int)blockIdx.x;
+    while (rem >= nb - bi) {
+        rem -= nb - bi;
+        ++bi;
+    }
+    const int bj = bi + rem;
+    __shared__ float a_s[kHessSlab][kHessTile + 1], b_s[kHessSlab][kHessTile + 1];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;   // 16 x 16 threads, 4 x 4 outputs each
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+    for (int64_t t0 = 0; t0 < T; t0 += kHessSlab) {
+        // 32 x 64 BF16 values per operand: 2048 values, 8 per thread
+        for (int e = (int)threadIdx.x; e < kHessSlab * kHessTile; e += 256) {
+            const int r = e / kHessTile, c = e - r * kHessTile;
+            const int64_t t = t0 + r;
+            const int64_t ca = (int64_t)bi * kHessTile + c, cb = (int64_t)bj * kHessTile + c;
+            a_s[r][c] = (t < T && ca < K) ? bf16_bits_to_float((uint32_t)__ldg(x + t * ldx + ca)) : 0.0f;
+            b_s[r][c] = (t < T && cb < K) ? bf16_bits_to_float((uint32_t)__ldg(x + t * ldx + cb)) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int r = 0; r < kHessSlab; ++r) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) av[i] = a_s[r][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bv[j] = b_s[r][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t gi = (int64_t)bi * kHessTile + ty * 4 + i, gj = (int64_t)bj * kHessTile + tx * 4 + j;
+            if (gi < K && gj < K) {
+                const float v = acc[i][j] + (beta != 0.0f ? beta * H[gi * K + gj] : 0.0f);
+                H[gi * K + gj] = v;
+                if (bi != bj) H[gj * K + gi] = v;   // (a diagonal tile computes both halves itself)
+            }
+        }
+}
+
+// Sec. 3.3 (as in GPTQ): the Hessian in processing order, a unit diagonal for input features that
+// never fired, damp * mean(diag) added to the diagonal.  Pass 1: the mean of the diagonal after the
+// dead-feature rule (one CTA); pass 2: the permuted copy.
+__global__ void __launch_bounds__(256)
+hessian_diag_mean_kernel(const float* __restrict__ H, int64_t K, float* __restrict__ mean_out) {
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int64_t k = threadIdx.x; k < K; k += 256) {
+        const float d = H[k * K + k];
+        s += d == 0.0f ? 1.0 : (double)d;
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *mean_out = (float)(red[0] / (double)K);
+}
+__global__ void __launch_bounds__(256)
+hessian_prepare_kernel(const float* __restrict__ H, int64_t K, const int32_t* __restrict__ perm, float damp,
+                       const float* __restrict__ mean_diag, float* __restrict__ Hp) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= K * K) return;
+    const int64_t i = idx / K, j = idx - i * K;
+    const int64_t si = perm ? perm[i] : i, sj = perm ? perm[j] : j;
+    float v = H[si * K + sj];
+    if (i == j) {
+        if (v == 0.0f) v = 1.0f;
+        v = __fadd_rn(v, __fmul_rn(damp, *mean_diag));
+    }
+    Hp[idx] = v;
+}
+
 }  // namespace w4a8

@@ -1364,6 +1364,37 @@ int w4a8_gar_permutation(const float* hdiag, int64_t K, int group, int32_t* perm
     return launch_status();
 }
 
+int w4a8_hessian_accumulate(const void* x_bf16, int64_t T, int64_t K, int64_t ldx, float* H, int accumulate,
+                            void* stream) {
+    if (!x_bf16 || !H || T <= 0 || K <= 0 || ldx < K) return W4A8_ERR_INVALID_ARG;
+    if (K > 32768) return W4A8_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(x_bf16) & 1u) || (reinterpret_cast<uintptr_t>(H) & 3u)) return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int64_t nb = (K + kHessTile - 1) / kHessTile;
+    hessian_xtx_kernel<<<(unsigned)(nb * (nb + 1) / 2), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(x_bf16), T, K, ldx, H, accumulate ? 1.0f : 0.0f);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_status();
+}
+
+int w4a8_hessian_prepare(const float* H, int64_t K, const int32_t* perm, float damp, float* H_out, float* scratch,
+                         void* stream) {
+    if (!H || !H_out || !scratch || K <= 0 || H == H_out) return W4A8_ERR_INVALID_ARG;
+    if (!(damp >= 0.0f)) return W4A8_ERR_INVALID_ARG;
+    if (K > 32768) return W4A8_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(H) & 3u) || (reinterpret_cast<uintptr_t>(H_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(scratch) & 3u) || (reinterpret_cast<uintptr_t>(perm) & 3u))
+        return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    hessian_diag_mean_kernel<<<1, 256, 0, st>>>(H, K, scratch);
+    hessian_prepare_kernel<<<(unsigned)((K * K + 255) / 256), 256, 0, st>>>(H, K, perm, damp, scratch, H_out);
+    g_launches.fetch_add(2, std::memory_order_relaxed);
+    return launch_status();
+}
+
 size_t w4a8_dpq_workspace_bytes(int64_t N, int64_t K) {
     if (N <= 0 || K <= 0 || K % kGroup != 0) return 0;
     return ((size_t)N * (size_t)K + (size_t)N * 128) * sizeof(float);

@@ -104,3 +104,64 @@ def test_dpq_layer_size_and_the_device_side_factorization():
         D = torch.from_numpy(W).cuda().to(torch.float64) - w16
         return float(torch.einsum("nk,kj,nj->", D, Hd, D))    # || (W - W^) X^T ||^2 = tr(D H D^T)
     assert out_err((codes, gscale, gzero, s_w)) < 0.8 * out_err(rtn)
+
+
+@pytest.mark.parametrize("T,K", [(100, 128), (384, 640), (1000, 1096)])
+def test_hessian_accumulate_and_prepare_match_oracle(T, K):
+    # w4a8_hessian_accumulate: FP32 sums over T products per entry against the oracle's float64 X^T X
+    # (tolerance: T rounding errors of 2^-24 relative to the entry's sum of magnitudes, bounded by
+    # sqrt(H_ii H_jj)); two batches accumulated = one pass; the matrix is exactly symmetric.
+    # w4a8_hessian_prepare: permutation, dead-feature rule, dampening -- against the oracle's.
+    rng = np.random.default_rng(T + K)
+    X = rng.standard_normal((T, K)).astype(np.float32) * np.linspace(0.1, 4.0, K, dtype=np.float32)
+    X[:, 3] = 0.0
+    X[:, K - 1] = 0.0
+    xb = oracle.f32_to_bf16(X)
+    xd = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).cuda()
+    H = binding.hessian_accumulate(xd)
+    half = T // 2
+    H2 = binding.hessian_accumulate(xd[:half].contiguous())
+    H2 = binding.hessian_accumulate(xd[half:].contiguous(), H2)
+    torch.cuda.synchronize()
+    ref = oracle.hessian(xb)
+    got = H.cpu().numpy().astype(np.float64)
+    assert np.array_equal(H.cpu().numpy(), H.cpu().numpy().T)
+    bound = np.sqrt(np.outer(np.diag(ref), np.diag(ref)))
+    assert np.all(np.abs(got - ref) <= 4.0 * T * 2.0 ** -24 * bound + 1e-30)
+    assert np.all(np.abs(H2.cpu().numpy().astype(np.float64) - ref) <= 4.0 * T * 2.0 ** -24 * bound + 1e-30)
+    assert np.all(got[3] == 0) and np.all(got[:, K - 1] == 0)
+    perm = rng.permutation(K).astype(np.int32)
+    for pm in (None, perm):
+        Hp = binding.hessian_prepare(H, None if pm is None else torch.from_numpy(pm).cuda(), damp=0.02)
+        torch.cuda.synchronize()
+        want = oracle.hessian_prepare(H.cpu().numpy(), pm, damp=0.02)
+        assert np.allclose(Hp.cpu().numpy().astype(np.float64), want, rtol=3e-7, atol=0)
+
+
+def test_quantizer_pipeline_from_activations_through_the_c_abi():
+    # X -> H (w4a8_hessian_accumulate) -> order (w4a8_gar_permutation) -> prepared Hessian
+    # (w4a8_hessian_prepare) -> [library: inverse and Cholesky factor] -> w4a8_dpq_quantize: the stored
+    # layer must beat round-to-nearest on the layer's output error by the margin the oracle's
+    # quantizer shows on such inputs (>= 20 %).
+    N, K, T = 256, 512, 1024
+    rng = np.random.default_rng(5)
+    mix = rng.standard_normal((K, K)).astype(np.float32) * 0.2 + np.eye(K, dtype=np.float32)
+    X = (rng.standard_normal((T, K)).astype(np.float32) @ mix) * np.linspace(0.3, 3.0, K, dtype=np.float32)
+    xb = oracle.f32_to_bf16(X)
+    xd = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).cuda()
+    W = torch.from_numpy(inputs.make_weight(N, K, 0.02, 6)).cuda()
+    H = binding.hessian_accumulate(xd)
+    perm = binding.gar_permutation(H.diagonal().contiguous())
+    Hp = binding.hessian_prepare(H, perm, damp=0.01).to(torch.float64)
+    Hinv = torch.cholesky_inverse(torch.linalg.cholesky(Hp))
+    U = torch.linalg.cholesky(0.5 * (Hinv + Hinv.T), upper=True).to(torch.float32).contiguous()
+    cq = binding.dpq_quantize(W, U, perm, symmetric=True, mse_steps=6)
+    rq = binding.quantize_weight_rtn(W, symmetric=True)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+
+    def out_err(q):
+        w8 = binding.dequant_weight(q[0], q[1], q[2]).view(torch.float8_e4m3fn).float() * q[3]
+        D = (W - w8).double()
+        return float(torch.einsum("nk,kj,nj->", D, H.double(), D))
+    assert out_err(cq) <= 0.8 * out_err(rq)

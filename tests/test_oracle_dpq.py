@@ -202,3 +202,34 @@ def test_hessian_factor_of_a_diagonal_hessian_in_closed_form():
     want = 1.0 / np.sqrt(d[perm] + 0.05 * d.mean())
     assert np.allclose(np.diag(U), want, rtol=1e-6, atol=0)
     assert np.array_equal(U, np.diag(np.diag(U)))
+
+
+def test_hessian_is_the_sum_of_outer_products_and_prepare_follows_its_three_rules():
+    # oracle.hessian: X^T X written out as a sum of outer products of the token rows (no matmul), its
+    # diagonal the column sums of squares; a one-hot X gives a diagonal count matrix.  oracle.hessian_prepare
+    # against the three rules applied entry by entry: permutation of rows AND columns, unit diagonal for dead
+    # columns, damp * mean(diag) on the diagonal.
+    rng = np.random.default_rng(12)
+    T, K = 37, 24
+    X = (rng.standard_normal((T, K)) * 3).astype(np.float32)
+    X[:, 5] = 0.0
+    xb = oracle.f32_to_bf16(X)
+    Xr = oracle.bf16_to_f32(xb).astype(np.float64)
+    H = oracle.hessian(xb)
+    want = np.zeros((K, K))
+    for t in range(T):
+        want += np.outer(Xr[t], Xr[t])
+    assert np.allclose(H, want, rtol=1e-13, atol=1e-12)
+    assert np.allclose(np.diag(H), (Xr ** 2).sum(axis=0), rtol=1e-13)
+    onehot = np.zeros((10, 4), dtype=np.float32)
+    onehot[np.arange(10), [0, 1, 1, 3, 3, 3, 0, 1, 3, 3]] = 1.0
+    assert np.array_equal(oracle.hessian(oracle.f32_to_bf16(onehot)), np.diag([2.0, 3.0, 0.0, 5.0]))
+    perm = rng.permutation(K).astype(np.int32)
+    Hp = oracle.hessian_prepare(H, perm, damp=0.05)
+    dd = np.array([H[perm[a], perm[a]] if H[perm[a], perm[a]] != 0 else 1.0 for a in range(K)])
+    for a in range(K):
+        for b in range(K):
+            v = H[perm[a], perm[b]]
+            if a == b:
+                v = dd[a] + 0.05 * dd.mean()
+            assert Hp[a, b] == pytest.approx(v, rel=1e-14, abs=1e-300)

@@ -363,3 +363,53 @@ def test_w8a8_comparison_scheme_in_the_chain_kernel():
     # formats may not be mixed within a launch
     with pytest.raises(binding.W4A8Error):
         binding.LinearChain([p4[0], p8[1]])()
+
+
+@pytest.mark.parametrize("M", [1, 5, 16])
+def test_rows_quantized_in_chunks_by_several_ctas(M):
+    # Long rows are cut into chunks that different CTAs quantize; the chunk maxima meet in the workspace
+    # before any chunk is converted.  Plain input with K = 8192 and 16384 (two and four chunks; 16384 is the
+    # largest K), the gated kind with F = 4096 and 6144 (two and three chunks), dynamic, power-of-two and
+    # static scales; FP8 bytes and scales bit-exact against the oracle (plain) and against
+    # w4a8_silu_mul_quantize (gated), outputs within the gate; three launches on the same workspace (the
+    # maxima and chunk counts must be back to zero after every launch).
+    N = 208
+    ss = dev(np.array([0.07], dtype=np.float32))
+    probs, checks = [], []
+    for i, (K, kw, okw) in enumerate([(8192, {}, {}), (16384, dict(scale_mode=binding.SCALE_POW2), dict(scale_mode=1)),
+                                      (8192, dict(static_scale=ss), dict(static_scale=0.07))]):
+        wq, tw = _weights(N, K, 500 + i)
+        xb = inputs.make_activation(M, K, 510 + i, 0.01, 20.0)
+        d = dict(x=bf16_dev(xb), weight=tw, y=torch.zeros((M, N), dtype=torch.float32, device="cuda"),
+                 x8_out=torch.zeros((M, K), dtype=torch.uint8, device="cuda"),
+                 s_x_out=torch.zeros((M,), dtype=torch.float32, device="cuda"), **kw)
+        probs.append(d)
+        checks.append(("plain", xb, wq, okw))
+    for i, F in enumerate([4096, 6144]):
+        wq, tw = _weights(N, F, 520 + i)
+        gu = bf16_dev(inputs.make_activation(M, 2 * F, 530 + i, 0.0, 1.0))
+        d = dict(x=gu, weight=tw, y=torch.zeros((M, N), dtype=torch.float32, device="cuda"),
+                 kind=binding.CHAIN_INPUT_SILU_MUL, x8_out=torch.zeros((M, F), dtype=torch.uint8, device="cuda"),
+                 s_x_out=torch.zeros((M,), dtype=torch.float32, device="cuda"))
+        probs.append(d)
+        checks.append(("gated", gu, wq, None))
+    chain = binding.LinearChain(probs)
+    for _ in range(3):
+        for d in probs:
+            d["y"].zero_(); d["x8_out"].zero_(); d["s_x_out"].zero_()
+        chain()
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0
+        for d, (kind, src, wq, okw) in zip(probs, checks):
+            if kind == "plain":
+                x8, s_x = oracle.quantize_act(src, **okw)
+                assert np.array_equal(d["x8_out"].cpu().numpy(), x8)
+                assert np.array_equal(d["s_x_out"].cpu().numpy().view(np.uint32), s_x.astype(np.float32).view(np.uint32))
+            else:
+                h8, s_h = binding.silu_mul_quantize(src)
+                torch.cuda.synchronize()
+                assert torch.equal(d["x8_out"], h8) and torch.equal(d["s_x_out"], s_h)
+                x8, s_x = h8.cpu().numpy(), s_h.cpu().numpy()
+            ref = oracle.linear(x8, s_x, oracle.dequant_weight(*wq[:3]), wq[3])
+            worst, _ = fp32_gate(d["y"].cpu().numpy(), ref["y64"], rel=2e-3)
+            assert worst <= 2e-3, worst

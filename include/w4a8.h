@@ -108,7 +108,8 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * when it is NULL or too small; larger M requires it.  It
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
- * its first use; every call leaves it ready for the next one -- except a call during which a
+ * its first use; every call leaves it ready for the next one, whatever that call's shape is (one
+ * workspace of the largest size may serve all layers of a model) -- except a call during which a
  * bounded wait gave up (w4a8_query_device_status returns W4A8_ERR_TIMEOUT): zero-fill the
  * workspace again after that.  Calls that share a workspace must not overlap on the device.
  * Calls with M <= 16 on tiled weights place their worker CTAs at run time (at most one per SM and

@@ -214,6 +214,17 @@ static int sm_count() {
 
 constexpr int kNominalSMs = 148;  // for size queries made without a device
 
+// Layout of every w4a8_linear workspace, whatever kernel and shape use it: a control area of fixed
+// size at the start (tile counters of the persistent kernel; K-cut counters and placement state
+// of the split-N kernel), which every launch leaves zero-filled, and behind it the data (partial
+// sums), which may be left in any state.  With the control area at a shape-dependent size, one
+// call's left-over partial sums could sit where the next call -- another layer, another kernel
+// -- expects zeroed counters; callers do share one workspace between the layers of a model.
+constexpr size_t kLinearCtlBytes = 65536;
+// The split-N kernel's 2 KB (K-cut counters, placement state -- whose generation word stays non-zero
+// by design) sit at the END of the control area, the persistent kernel's tile counters at its start.
+constexpr size_t kLinearCtlSplitN = kLinearCtlBytes - 2048;
+
 struct SkPlan {
     int bnx, TM, TN;
     int aligned;   // 1: whole tiles per CTA, nothing shared; 0: equal slices of the (tile, k-block) space
@@ -257,7 +268,8 @@ static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
                 Ps = Pk;
             }
         }
-        const bool al = t_aligned <= t_split;
+        // (tile counters must fit the control area: otherwise whole tiles per CTA, which need none)
+        const bool al = t_aligned <= t_split || 2 * (size_t)Tt * sizeof(unsigned int) > kLinearCtlSplitN;
         const double t = al ? t_aligned : t_split;
         if (t < best) {
             best = t;
@@ -269,12 +281,10 @@ static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
             pl->P = al ? Pa : Ps;
         }
     }
-    size_t cb = 2 * (size_t)pl->TM * pl->TN * sizeof(unsigned int);  // arrivals and finished reducers per tile
-    pl->counter_bytes = (cb + 255) / 256 * 256;
-    // The size asked of the caller covers every tile width and any SM count up to kMaxSMs, so that
-    // the query needs no device: counters of the narrowest tiles, partial tiles of the widest.
-    size_t cb_max = 2 * (size_t)((M + 63) / 64) * (size_t)TN * sizeof(unsigned int);
-    pl->workspace_bytes = (cb_max + 255) / 256 * 256 + (size_t)kMaxSMs * 2 * 256 * 128 * sizeof(float);
+    // arrivals and finished reducers per tile live in the control area; the size asked of the caller
+    // covers every tile width and any SM count up to kMaxSMs, so that the query needs no device
+    pl->counter_bytes = kLinearCtlBytes;
+    pl->workspace_bytes = kLinearCtlBytes + (size_t)kMaxSMs * 2 * 256 * 128 * sizeof(float);
 }
 
 template <class Cfg>
@@ -314,11 +324,13 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
 
 // Row partition and ring sizes of the split-N kernel for the current device.
 // Workspace of the split-N kernel when it cuts K (bytes; fits any SM count up to kMaxSMs and 128 tokens).
-// Layout: split-K counters (1 KB), placement state of the launch (1 KB), partial tiles.
+// Layout: split-K counters (1 KB) and placement state of the launch (1 KB) at the end of the common
+// control area, partial tiles behind that area.
 constexpr size_t kSnCounterBytes = 1024;
 constexpr size_t kSnSchedBytes = 1024;
 static_assert(kSnCounterBytes == (size_t)kSchedWsOffset, "the kernel finds the placement state behind the counters");
-constexpr size_t kSnWorkspaceBytes = kSnCounterBytes + kSnSchedBytes + (size_t)kMaxSMs * 128 * 128 * sizeof(float);
+static_assert(kLinearCtlSplitN + kSnCounterBytes + kSnSchedBytes == kLinearCtlBytes, "split-N control data at the end of the common control area");
+constexpr size_t kSnWorkspaceBytes = kLinearCtlBytes + (size_t)kMaxSMs * 128 * 128 * sizeof(float);
 
 template <class Cfg>
 static bool make_sn_plan(int64_t N, int64_t K, int sms, bool may_split_k, SnPlan* pl) {
@@ -419,8 +431,8 @@ static int launch_splitn_planned(const CUtensorMap& tx, const uint8_t* wpp, cons
                                : (int)(g_sched_seq.fetch_add(1, std::memory_order_relaxed) % (unsigned)kSchedSlots);
         grid = 2u * (unsigned)P;
     }
-    unsigned int* counters = static_cast<unsigned int*>(workspace);
-    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kSnCounterBytes + kSnSchedBytes);
+    unsigned int* counters = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(workspace) + kLinearCtlSplitN);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kLinearCtlBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(Cfg::kThreads);

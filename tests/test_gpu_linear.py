@@ -124,7 +124,9 @@ def test_persistent_kernel_split_tiles_and_reuse_of_workspace(M, N, K):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     persistent = M > 128 or (M > 64 and K >= 2048 and ((N + 127) // 128) * 4 <= sms)
     n_counter_bytes = 8 * ((M + 255) // 256) * ((N + 127) // 128) if persistent else 1024
-    assert np.all(ws[:n_counter_bytes].cpu().numpy() == 0)     # tile counters are back to zero
+    # tile counters (persistent kernel: start of the 64 KB control area; split-N: its last 2 KB) are back to zero
+    first = 0 if persistent else 65536 - 2048
+    assert np.all(ws[first:first + n_counter_bytes].cpu().numpy() == 0)
 
 
 def test_sign_magnitude_prepack_flags_code_zero():

@@ -43,3 +43,34 @@ def test_fresh_workspace_launches_agree_and_are_right(M, N, K):
     # k-slice of a tile is off by a good fraction of it
     scale = float(ref.abs().max())
     assert float((outs[0] - ref).abs().max()) <= 1e-3 * scale
+
+
+def test_one_workspace_shared_by_layers_of_different_shapes_and_kernels():
+    # One workspace of the largest size, used by calls of different shapes one after the other -- split-N
+    # with and without a K cut, the persistent kernel as equal slices and as whole CTAs per tile, the
+    # 256 x 256 tiles: whatever a call leaves behind in the data part of the workspace, the next call's
+    # counters must be zero.  Every result must equal the one computed on a fresh workspace of its own.
+    dev = torch.device("cuda")
+    shapes = [(128, 4096, 14336), (128, 28672, 4096), (128, 4096, 4096), (16, 4096, 14336), (300, 640, 8192),
+              (128, 6144, 4096), (512, 4096, 4096), (700, 10576, 640), (8, 4096, 4096), (256, 4096, 14336)]
+    cases = []
+    for (M, N, K) in shapes:
+        W = torch.from_numpy(inputs.make_weight(N, K, 0.02, seed=7 * M + N)).to(dev)
+        tw = binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True))
+        del W
+        xb = inputs.make_activation(M, K, M + 3 * K, 0.01, 20.0)
+        x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+        own = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32,
+                                   workspace=binding.new_workspace(M, N, K, tw.fmt, dev))
+        cases.append((tw, x8, s_x, own))
+    need = max(binding.linear_workspace_bytes(M, N, K, weight_format=binding.FMT_TILED_SIGNMAG) for (M, N, K) in shapes)
+    shared = torch.zeros((need,), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        for tw, x8, s_x, own in cases:
+            got = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32, workspace=shared)
+            assert torch.equal(got.view(torch.int32), own.view(torch.int32))
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    # the control area is left zero-filled (but for the generation word of the split-N kernel's placement state,
+    # in its last kilobyte)
+    assert bool((shared[:65536 - 1024] == 0).all())

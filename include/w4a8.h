@@ -239,7 +239,8 @@ int w4a8_linear_static_scratch(const uint8_t* x8, int64_t ldx8, const float* s_x
  * runs out, all CTAs stop, outputs are incomplete and bit 0 of the device status word is set
  * (w4a8_query_device_status returns W4A8_ERR_TIMEOUT).
  * `problems` is a HOST array, read during the call only.  Errors: W4A8_ERR_INVALID_ARG (NULL,
- * count outside 1..W4A8_CHAIN_MAX_PROBLEMS, bad enum, depends_on >= i, mixed weight formats),
+ * count outside 1..W4A8_CHAIN_MAX_PROBLEMS, bad enum, depends_on >= i, mixed weight formats, an
+ * input that is the FP32 output of the problem it depends on),
  * W4A8_ERR_BAD_SHAPE (M > 16, K % 128, N % 16, N too large, leading dimensions),
  * W4A8_ERR_BAD_ALIGNMENT, W4A8_ERR_WORKSPACE_TOO_SMALL; nothing is enqueued on error.
  */

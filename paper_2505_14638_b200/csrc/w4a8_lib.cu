@@ -974,6 +974,9 @@ static int chain_validate(const w4a8_chain_problem* pr, int count) {
         if (q.M <= 0 || q.N <= 0 || q.K <= 0) return W4A8_ERR_INVALID_ARG;
         if (q.input_kind != kChainKindPlain && q.input_kind != kChainKindSiluMul) return W4A8_ERR_INVALID_ARG;
         if (q.depends_on < -1 || q.depends_on >= i) return W4A8_ERR_INVALID_ARG;
+        // a problem that reads an earlier problem's output reads BF16: that output may not be FP32
+        if (q.depends_on >= 0 && q.x_bf16 == pr[q.depends_on].y && pr[q.depends_on].out_dtype != W4A8_OUT_BF16)
+            return W4A8_ERR_INVALID_ARG;
         if (q.scale_mode != W4A8_SCALE_EXACT && q.scale_mode != W4A8_SCALE_POW2) return W4A8_ERR_INVALID_ARG;
         if (q.weight_format != kFmtTiled && q.weight_format != kFmtTiledSignMag && q.weight_format != kFmtTiledFp8)
             return W4A8_ERR_INVALID_ARG;

@@ -291,6 +291,18 @@ def test_chain_argument_errors():
     assert binding.query_device_status() == 0
 
 
+def test_a_dependent_problem_may_not_read_an_fp32_output():
+    M, N, K = 4, 256, 256
+    wq, tw = _weights(N, K, 95)
+    wq2, tw2 = _weights(128, N, 96)
+    x = bf16_dev(inputs.make_activation(M, K, 97))
+    y32 = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    y2 = torch.zeros((M, 128), dtype=torch.float32, device="cuda")
+    probs = [dict(x=x, weight=tw, y=y32), dict(x=y32.view(torch.bfloat16)[:, :N], weight=tw2, y=y2, depends_on=0)]
+    with pytest.raises(binding.W4A8Error):
+        binding.LinearChain(probs)()
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_library_carries_on():
     # one CTA waits, with a limit of one millisecond, on a barrier nobody arrives on: the kernel
     # returns by itself, the status word carries the time-out bit, the query reports and clears it,

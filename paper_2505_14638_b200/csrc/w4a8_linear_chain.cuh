@@ -974,13 +974,10 @@ linear_chain_kernel(const __grid_constant__ ChainParams prm, uint8_t* __restrict
                         // FP8 weights: nothing to expand, the rows go to tensor memory as they are
                         if (have0) copy_fp8_row_to_tmem(wsrc + code_off, a_col);
                         if (ks * NB == 2 && have1) copy_fp8_row_to_tmem(wsrc + code_off + code_s0, a_col + 32u);
-                    } else if (ks * NB == 2) {
-                        if (have1)
-                            dequant_two_rows_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, wsrc + code_off + code_s0,
-                                                               wsrc + meta_off + meta_s0, a_col);
-                        else if (have0)
-                            dequant_row_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, a_col);
-                    } else if (have0) {
+                    } else if (ks * NB == 2 && have1) {
+                        dequant_two_rows_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, wsrc + code_off + code_s0,
+                                                           wsrc + meta_off + meta_s0, a_col);
+                    } else if (have0) {   // (one copy of the single-row expansion: the roles share the instruction caches)
                         dequant_row_to_tmem<Cfg::FMT>(wsrc + code_off, wsrc + meta_off, a_col);
                     }
                     ptx::mbar_arrive(bar_wfree0 + 8u * (uint32_t)r1.idx);   // this thread has read its codes

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from gpu_utils import Guarded
 from paper_2505_14638_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
@@ -74,3 +75,30 @@ def test_one_workspace_shared_by_layers_of_different_shapes_and_kernels():
     # the control area is left zero-filled (but for the generation word of the split-N kernel's placement state,
     # in its last kilobyte)
     assert bool((shared[:65536 - 1024] == 0).all())
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 4096, 14336), (128, 4096, 4096), (100, 512, 8192), (300, 640, 8192),
+                                   (700, 10576, 640), (1061, 16384, 1024), (512, 6144, 1024)])
+def test_linear_kernels_write_only_their_outputs_and_their_workspace(M, N, K):
+    # poisoned guard bands in front of and behind Y (with padding columns between its rows, which must
+    # stay untouched too) and around a workspace of exactly the size the library asks for: no kernel
+    # family of w4a8_linear may write a byte outside them
+    dev = torch.device("cuda")
+    W = torch.from_numpy(inputs.make_weight(N, K, 0.02, seed=M + 2 * N)).to(dev)
+    tw = binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True))
+    del W
+    xb = inputs.make_activation(M, K, 5 * M + K, 0.01, 20.0)
+    x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+    need = binding.linear_workspace_bytes(M, N, K, weight_format=tw.fmt)
+    gws = Guarded((need,), torch.uint8, fill=0)
+    ldy = N + 8
+    gy = Guarded((M, ldy), torch.bfloat16, fill=7.0)
+    ref = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_BF16, workspace=binding.new_workspace(M, N, K, tw.fmt, dev))
+    for _ in range(2):
+        binding.linear_tiled(x8, s_x, tw, out=gy.t[:, :N], workspace=gws.t)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    gy.check()
+    gws.check()
+    assert torch.equal(gy.t[:, :N].contiguous().view(torch.int16), ref.view(torch.int16))
+    assert bool((gy.t[:, N:] == 7.0).all())

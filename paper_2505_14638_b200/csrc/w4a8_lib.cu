@@ -290,7 +290,7 @@ static void make_sk_plan(int64_t M, int64_t N, int64_t K, int sms, SkPlan* pl) {
 template <class Cfg>
 static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float* s_x, const float* s_w,
                           int sw_stride, void* y, int64_t ldy, int out_dtype, void* workspace, const SkPlan& pl,
-                          int M, int N, int K, cudaStream_t st, const CUtensorMap* tw8 = nullptr) {
+                          int M, int N, int K, cudaStream_t st, const CUtensorMap* tw8 = nullptr, int cl = 0) {
     auto kern = linear_streamk_kernel<Cfg>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -309,14 +309,23 @@ static int launch_streamk(const CUtensorMap& tx, const uint8_t* wpp, const float
     cfg.blockDim = dim3(Cfg::kThreads);
     cfg.dynamicSmemBytes = (size_t)Cfg::kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (Cfg::CL) {
+        // the cl CTAs of a tile as one thread-block cluster (P = tiles x cl)
+        if (cl < 2 || cl > 8 || P % cl != 0) return W4A8_ERR_INVALID_ARG;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cl;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     // (the second tensor map is read only by the FP8-weight variant)
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tx, tw8 ? *tw8 : tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
-                                       counters, slots, M, N, K, pl.TM, pl.TN, aligned, status);
+                                       counters, slots, M, N, K, pl.TM, pl.TN, aligned, cl, status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) return W4A8_ERR_CUDA;
     return launch_status();
@@ -539,9 +548,97 @@ static bool streamk_for_128_tokens(int64_t M, int64_t N, int64_t K, int sms) {
     return M > 64 && M <= kSplitNMaxM && K >= 2048 && ((N + 127) / 128) * 4 <= sms;
 }
 
+// Few tiles (at most half as many 128-row tiles as SMs) and at most 128 tokens: CTAs per tile of the plan
+// that cuts K between the CTAs of a thread-block cluster (0: the plan does not apply).  Every CTA keeps
+// at least two k-blocks.
+static int cluster_kcut_ctas(int64_t M, int64_t N, int64_t K, int sms) {
+    if (M > 128) return 0;
+    const int64_t TN = (N + 127) / 128, KB = K / 128;
+    int64_t c = sms / TN;
+    if (c > 8) c = 8;
+    while (c > 1 && KB < 2 * c) --c;
+    return c >= 2 ? (int)c : 0;
+}
+
+// Launches the cluster plan; returns -1 (nothing launched) when the device cannot hold all of the
+// launch's clusters at once -- a second wave would cost more than the exchange through L2 saves.
+template <class Cfg>
+static int launch_cluster_kcut(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, const float* s_x, const float* s_w,
+                               int sw_stride, void* y, int64_t ldy, int out_dtype, int M, int N, int K, int cl,
+                               cudaStream_t st) {
+    const int TN = (N + 127) / 128;
+    static std::atomic<int> fits[9];   // clusters of size cl resident at once (0: not asked yet)
+    int have = fits[cl].load(std::memory_order_relaxed);
+    if (have == 0) {
+        auto kern = linear_streamk_kernel<Cfg>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+            return W4A8_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(cl * 64));
+        cfg.blockDim = dim3(Cfg::kThreads);
+        cfg.dynamicSmemBytes = (size_t)Cfg::kSmemBytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cl;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+            cudaGetLastError();
+            n = -1;
+        }
+        have = n > 0 ? n : -1;
+        fits[cl].store(have, std::memory_order_relaxed);
+    }
+    if (have < TN) return -1;
+    CUtensorMap tx;
+    if (!make_tmap_u8_2d(&tx, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)Cfg::BNX,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    SkPlan pl;
+    pl.bnx = Cfg::BNX;
+    pl.TM = 1;
+    pl.TN = TN;
+    pl.aligned = 1;
+    pl.U = (int64_t)TN * (K / 128);
+    pl.P = (int64_t)TN * cl;
+    pl.counter_bytes = 0;
+    pl.workspace_bytes = 0;
+    return launch_streamk<Cfg>(tx, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, nullptr, pl, M, N, K, st, nullptr, cl);
+}
+
 static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, int64_t M, const uint8_t* wpp,
                              int fmt, const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
                              int out_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (M > 16) {
+        // 17..128 tokens on a layer with few 128-row tiles: K cut between the CTAs of a cluster (measured, us,
+        // against the split-N kernel or the persistent kernel with its exchange through L2:
+        // (32, 4096, 4096) 8.6 / 9.8, (64, 2048, 4096) 8.0 / 12.6, (100, 512, 8192) 9.0 / 15.0,
+        // (128, 4096, 4096) 12.4 / 12.9, (128, 4096, 14336) 20.3 / 21.2, (128, 6144, 4096) 14.3 / 14.5; at
+        // 16 tokens and fewer the split-N kernel, which overlaps its set-up with the launch before, stays
+        // ahead: (8, 4096, 4096) 8.5 / 7.3)
+        const int sms_c = sm_count();
+        const int cl0 = sms_c > 0 ? cluster_kcut_ctas(M, N, K, sms_c) : 0;
+        for (int cl = cl0; cl >= 2; --cl) {   // the largest cluster size of which all clusters are resident at once
+            int rc = check_device();
+            if (rc != W4A8_OK) return rc;
+            if (M <= 64)
+                rc = fmt == kFmtTiledSignMag
+                         ? launch_cluster_kcut<SkCfg<64, 4, 4, 4, kFmtTiledSignMag, 1, false, true>>(
+                               x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st)
+                         : launch_cluster_kcut<SkCfg<64, 4, 4, 4, kFmtTiled, 1, false, true>>(
+                               x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st);
+            else
+                rc = fmt == kFmtTiledSignMag
+                         ? launch_cluster_kcut<SkCfg<128, 4, 4, 3, kFmtTiledSignMag, 1, false, true>>(
+                               x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st)
+                         : launch_cluster_kcut<SkCfg<128, 4, 4, 3, kFmtTiled, 1, false, true>>(
+                               x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st);
+            if (rc != -1) return rc;
+        }
+    }
     bool split_n = M <= kSplitNMaxM;
     if (split_n && M > 64) {
         // (the persistent kernel needs its full workspace; without it the split-N kernel runs)

@@ -42,9 +42,21 @@ namespace w4a8 {
 // W8 = true (the W8A8 comparison scheme of Sec. 4.3 on this kernel's skeleton): the weights are FP8
 // E4M3 bytes [N][K] already; a TMA tile load puts them straight into the ring of swizzled weight
 // tiles the MMAs read, the expansion groups have nothing to do.  Whole tiles only.
-template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false>
+//
+// CL = true (few tiles, at most 128 tokens): the CTAs that share a tile's K range form a thread-block
+// cluster and exchange their partial sums through distributed shared memory instead of a workspace in
+// global memory.  CTA i of the C takes the i-th slice of the tile's token columns: every CTA writes,
+// its accumulator into its own (by then idle) ring memory and sends each slice to the staging area of
+// the slice's owner with one bulk copy that completes on the owner's barrier; the owner adds the C
+// partials in ascending rank order, applies the scales and stores the outputs.  Against the exchange through L2 -- partial tile out,
+// fence, counter, wait, partial tiles back in, each a round trip of a microsecond or more -- this
+// takes the tail of a (128, 4096, 4096) launch from 7.4 to about 2 us.  Needs no workspace.
+template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false, bool CL_ = false>
 struct SkCfg {
     static constexpr bool W8 = W8_;
+    static constexpr bool CL = CL_;
+    // staging area of the cluster exchange: C slices of ceil(columns / C) token columns x 128 channels, fp32
+    static constexpr int kRedBytes = CL_ ? (BNX_ + 8) * 128 * 4 : 0;
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
     static constexpr int G = G_;       // dequantization groups of 4 warps
     static constexpr int S1 = S1_;     // ring of TMA stages (packed chunk + activation tile)
@@ -58,13 +70,14 @@ struct SkCfg {
     static constexpr int kStage1 = kWStage + kXBytes;
     static constexpr int kW8Bytes = RB_ * 128 * 128;
     static constexpr int kBarBytes = 512;
-    static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + 1024;
+    static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + kRedBytes + 1024;
     static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;   // RB = 1: two accumulators (double buffer); RB = 2: one per row block
     static constexpr int kThreads = 32 * (10 + 4 * G);
     static constexpr int kSlotFloats = BNX * 128;
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
     static_assert(RB_ == 1 || (RB_ == 2 && BNX_ == 256), "two row blocks per tile only with 256-token tiles");
     static_assert(!W8_ || RB_ == 1, "the FP8-weight variant uses one row block per tile");
+    static_assert(!CL_ || (RB_ == 1 && !W8_ && BNX_ <= 128), "the cluster exchange serves one row block and at most 128 tokens");
     // A dequantization group handles every G-th stage, so it skips phases of the barriers it
     // waits on, and an mbarrier wait tells phases apart by parity only: the wait for use k of a
     // slot is sound only if use k-1 has completed before it starts.  That holds because a stage's
@@ -86,7 +99,7 @@ struct SkCfg {
     // the same inputs disagreed with the first.
     static_assert(S1_ % G_ == 0, "the ring depth must be a multiple of the number of expansion groups");
     static_assert(kStage1 % 1024 == 0, "alignment of the swizzled tiles");
-    static_assert((3 * S1 + 2 * S2 + 5) * 8 + 32 <= kBarBytes, "barrier area");
+    static_assert((3 * S1 + 2 * S2 + 6) * 8 + 32 <= kBarBytes, "barrier area");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
@@ -97,7 +110,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                       const uint8_t* __restrict__ wpp,             // tiled weights (panels, k-block major)
                       const float* __restrict__ s_x, const float* __restrict__ s_w, int sw_stride,
                       void* __restrict__ y, int64_t ldy, int out_dtype, unsigned int* counters,
-                      float* slots, int M, int N, int K, int TM, int TN, int aligned, unsigned int* status_word) {
+                      float* slots, int M, int N, int K, int TM, int TN, int aligned, int cl,
+                      unsigned int* status_word) {
     constexpr int BNX = Cfg::BNX, G = Cfg::G, S1 = Cfg::S1, S2 = Cfg::S2, RB = Cfg::RB;
     constexpr int TR = 128 * RB;   // weight rows per tile
     extern __shared__ uint8_t smem_raw[];
@@ -117,7 +131,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     auto bar_acc_empty = [&](int b) { return bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 2 + b); };
     const uint32_t bar_drain = bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 4);
     auto bar_xfull = [&](int s) { return bars_addr + 8u * (uint32_t)(2 * S1 + 2 * S2 + 5 + s); };
-    constexpr int kNumBars = 3 * S1 + 2 * S2 + 5;
+    const uint32_t bar_red = bars_addr + 8u * (uint32_t)(3 * S1 + 2 * S2 + 5);   // CL: partial sums of all CTAs of the cluster have arrived
+    constexpr int kNumBars = 3 * S1 + 2 * S2 + 6;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + kNumBars);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* share_slot = tmem_slot + 2;  // [3] number of shared tiles and their indices
@@ -134,28 +149,37 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     // Share of this CTA: an equal slice of the unit space, or -- when there are enough tiles
     // for whole tiles to balance -- a run of whole tiles (then no partial tile is ever produced).
     const int64_t Tt = (int64_t)TM * TN;
-    const int64_t u_begin = aligned ? (p * Tt / P) * KB : p * U / P;
-    const int64_t u_end = aligned ? ((p + 1) * Tt / P) * KB : (p + 1) * U / P;
+    int64_t u_begin, u_end;
+    if constexpr (Cfg::CL) {
+        // CTA p is member p % cl of the cluster of tile p / cl and takes that share of the tile's k-blocks
+        // (32-bit arithmetic: the 64-bit divisions of the general case cost a good part of a microsecond
+        // at the head of a launch that lasts ten)
+        const int pi = (int)blockIdx.x, tl = pi / cl, me = pi - tl * cl;
+        u_begin = (int64_t)tl * KB + me * KB / cl;
+        u_end = (int64_t)tl * KB + (me + 1) * KB / cl;
+    } else {
+        u_begin = aligned ? (p * Tt / P) * KB : p * U / P;
+        u_end = aligned ? ((p + 1) * Tt / P) * KB : (p + 1) * U / P;
+    }
     const int n_it = (int)(u_end - u_begin);
+    // first tile and k-block of the share
+    const int64_t tile_begin = Cfg::CL ? (int64_t)((int)blockIdx.x / cl) : u_begin / KB;
+    const int kb_begin = (int)(u_begin - tile_begin * KB);
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S1; ++s) {
-            ptx::mbar_init(bar_full(s), 1);
-            ptx::mbar_init(bar_xfull(s), 1);
-            ptx::mbar_init(bar_free1(s), 1);
+    if (warp == 0) {
+        // barrier i of the area, one lane each; arrival counts: 128 expanding threads on a "weights expanded"
+        // barrier (W8: the TMA load), the draining threads on an "accumulator drained" barrier, one elsewhere
+        for (int i = lane; i < kNumBars; i += 32) {
+            uint32_t count = 1u;
+            if (i >= 2 * S1 && i < 2 * S1 + S2) count = Cfg::W8 ? 1u : 128u;
+            if (i >= 2 * S1 + 2 * S2 + 2 && i < 2 * S1 + 2 * S2 + 4) count = RB == 2 ? 256u + 128u * G : 256u;   // (RB = 2: the expansion warps drain too)
+            ptx::mbar_init(bars_addr + 8u * (uint32_t)i, count);
         }
-        for (int s = 0; s < S2; ++s) {
-            ptx::mbar_init(bar_w8_full(s), Cfg::W8 ? 1 : 128);   // (W8: the TMA load's transaction count)
-            ptx::mbar_init(bar_free2(s), 1);
+        if (lane == 0) {
+            *abort_flag = 0u;
+            ptx::prefetch_tensormap(&tmap_x);
         }
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(bar_acc_full(b), 1);
-            ptx::mbar_init(bar_acc_empty(b), RB == 2 ? 256 + 128 * G : 256);   // (RB = 2: the expansion warps drain too)
-        }
-        ptx::mbar_init(bar_drain, 1);
-        *abort_flag = 0u;
         ptx::fence_mbar_init();
-        ptx::prefetch_tensormap(&tmap_x);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
@@ -164,6 +188,9 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
+    // CL: no CTA may signal a peer's barrier before it is initialized -- arrive here, wait before the first copy
+    if constexpr (Cfg::CL) ptx::cluster_arrive();
+    bool cl_waited = false;
     const uint32_t tmem_base = *tmem_slot;
     // Launched with programmatic stream serialization: the next kernel in the stream may start its
     // set-up and weight prefetch while this one runs; everything that depends on earlier kernels
@@ -178,7 +205,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     auto drain_wide = [&](int j, int slot) -> bool {
         constexpr int kSlots = 2 + G;
         const int q = warp & 3, r = q * 32 + lane;
-        const int64_t tile = u_begin / KB + j;
+        const int64_t tile = tile_begin + j;
         const int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
         const int m0 = mt * BNX;
         const int n_lo = nt * TR + r, n_hi = n_lo + 128;
@@ -233,8 +260,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             bool ok = true;
             int issued = 0;
             ptx::Ring r1;
-            int64_t tile = u_begin / KB;
-            int kb = (int)(u_begin - tile * KB);
+            const int64_t tile = tile_begin;
+            int kb = kb_begin;
             int nt = (int)(tile / TM), mt = (int)(tile - (int64_t)nt * TM);
             // Weights depend on no earlier kernel: the first ring-full of packed tiles is requested
             // before waiting for the kernels that produce the activations.
@@ -242,12 +269,22 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             // activations: the weight-only prologue may not be longer than that ring)
             constexpr int kAhead = Cfg::W8 ? (S2 < S1 ? S2 : S1) : S1;
             const int ahead = n_it < kAhead ? n_it : kAhead;
+            // (the activation tiles of the first ring-full are requested by the MMA warp)
+            const int nx = n_it < S1 ? n_it : S1;
             ptx::Ring rx;  // ring position of the next activation tile
             int xkb = kb, xmt = mt;
-            int it_x = 0;  // activation tiles issued so far
+            int it_x = nx;  // activation tiles issued so far
+            for (int i = 0; i < nx; ++i) {
+                rx.advance(S1);
+                if (++xkb == KB) {
+                    xkb = 0;
+                    if (++xmt == TM) xmt = 0;
+                }
+            }
             for (int it = 0; it < n_it; ++it) {
                 ok = ptx::mbar_wait(bar_free1(r1.idx), r1.phase ^ 1u, abort_flag, status_word);
                 if (!ok) break;
+                // (operands worked out by the whole warp: see elect_one)
                 const int rows = (N - nt * TR) < TR ? (N - nt * TR) : TR;  // ragged last tile
                 const int64_t row0 = (int64_t)kb * N + (int64_t)nt * TR;
                 const uint32_t full = bar_full(r1.idx), wdst = stage_w(r1.idx);
@@ -335,6 +372,23 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             ptx::Ring r1, r2;
             int j = 0;
             int64_t u = u_begin;
+            {
+                // The activation tiles of the first ring-full (every slot is free): requested here, while
+                // the producer warp requests the weights -- one lane after the other, the first
+                // activation tile went out only after the last of those, a microsecond late.
+                ptx::griddep_wait();
+                int xkb = kb_begin, xmt = (int)(tile_begin % TM);
+                for (int i = 0; i < n_it && i < S1; ++i) {
+                    if (ptx::elect_one()) {
+                        ptx::mbar_arrive_expect_tx(bar_xfull(i), (uint32_t)Cfg::kXBytes);
+                        ptx::tma_load_2d(stage_x(i), &tmap_x, xkb * 128, xmt * BNX, bar_xfull(i));
+                    }
+                    if (++xkb == KB) {
+                        xkb = 0;
+                        if (++xmt == TM) xmt = 0;
+                    }
+                }
+            }
             while (u < u_end && ok) {
                 const int64_t tile = u / KB;
                 const int kb0 = (int)(u - tile * KB);
@@ -434,6 +488,114 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             // The CTA's first segment uses slot 0, a later (necessarily last) one slot 1.
             float* my_slot = slots + ((int64_t)p * 2 + (j == 0 ? 0 : 1)) * Cfg::kSlotFloats +
                              (int64_t)half * kHalfCols * 128;
+            if constexpr (Cfg::CL) {
+                if (!whole) {
+                    // ---- exchange inside the cluster ----
+                    const uint32_t red_local = bars_addr + (uint32_t)Cfg::kBarBytes;   // [source rank][column of my slice][128 channels]
+                    const int me = (int)ptx::cluster_ctarank();
+                    const int ncol = (M - mt * BNX) < BNX ? (M - mt * BNX) : BNX;   // valid token columns of the tile
+                    const int w = (ncol + cl - 1) / cl;                             // columns per slice
+                    int wn = ncol - me * w;                                         // valid columns of my slice
+                    wn = wn < 0 ? 0 : (wn > w ? w : wn);
+                    if (leader) ptx::mbar_arrive_expect_tx(bar_red, (uint32_t)(cl * wn * 512));
+                    // this thread's outputs as the owner of slice `me`: channels c4 .. c4 + 3 of the slice's
+                    // columns te / 32, te / 32 + 8, ...; their scales are fetched before the wait
+                    const int te = (warp - 2) * 32 + lane, c4 = (te & 31) * 4;
+                    const int n4 = nt * 128 + c4;
+                    float sw4[4], sxp[8];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) sw4[i] = (n4 + i < N) ? __ldg(s_w + (int64_t)(n4 + i) * sw_stride) : 0.0f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int tl = (te >> 5) + 8 * k;
+                        sxp[k] = tl < wn ? __ldg(s_x + mt * BNX + me * w + tl) : 0.0f;
+                    }
+                    // accumulator -> this CTA's own ring memory (idle: the tile's MMAs have completed), as
+                    // [column][128 channels]: the slice of owner d is one contiguous piece
+                    const int t0 = half * kHalfCols;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kHalfCols; c0 += 16) {
+                        uint32_t v[16];
+                        ptx::tmem_ld_32x32b_x16(tmem_acc0 + (uint32_t)c0, v);
+                        ptx::tmem_ld_wait();
+                        if (t0 + c0 >= ncol) break;  // warp-uniform
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            asm volatile("st.shared.u32 [%0], %1;" ::"r"(base + (uint32_t)(((t0 + c0 + jj) * 128 + r) * 4)), "r"(v[jj])
+                                         : "memory");
+                    }
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive(bar_acc_empty(buf));
+                    ptx::fence_proxy_async_smem();
+                    if (!cl_waited) {
+                        ptx::cluster_wait();   // every CTA of the cluster has initialized its barriers
+                        cl_waited = true;
+                    }
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (te < cl) {
+                        // one bulk copy per owner: my partial sums of its slice into its staging area,
+                        // completion counted on its barrier
+                        int cols = ncol - te * w;
+                        cols = cols < 0 ? 0 : (cols > w ? w : cols);
+                        if (cols > 0)
+                            ptx::bulk_copy_to_cta(ptx::map_to_cta(red_local + (uint32_t)(me * w * 512), (uint32_t)te),
+                                                  base + (uint32_t)(te * w * 512), (uint32_t)(cols * 512),
+                                                  ptx::map_to_cta(bar_red, (uint32_t)te));
+                    }
+                    ok = ptx::mbar_wait(bar_red, 0u, abort_flag, status_word);
+                    if (!ok) break;
+                    const bool vec_ok = (ldy & 3) == 0;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int tl = (te >> 5) + 8 * k;
+                        if (tl >= wn) break;
+                        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+                        for (int sr = 0; sr < cl; ++sr) {   // ascending rank order: the same sum on every launch
+                            float4 pv;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(pv.x), "=f"(pv.y), "=f"(pv.z), "=f"(pv.w)
+                                         : "r"(red_local + (uint32_t)(((sr * w + tl) * 128 + c4) * 4)));
+                            a0 += pv.x;
+                            a1 += pv.y;
+                            a2 += pv.z;
+                            a3 += pv.w;
+                        }
+                        if (n4 >= N) continue;
+                        const int m = mt * BNX + me * w + tl;
+                        const float sxm = sxp[k];
+                        const float r0 = a0 * (sxm * sw4[0]), r1 = a1 * (sxm * sw4[1]), r2 = a2 * (sxm * sw4[2]),
+                                    r3 = a3 * (sxm * sw4[3]);
+                        if (out_dtype == W4A8_OUT_FP32) {
+                            float* yp = reinterpret_cast<float*>(y) + (int64_t)m * ldy + n4;
+                            if (vec_ok) {
+                                *reinterpret_cast<float4*>(yp) = make_float4(r0, r1, r2, r3);
+                            } else {
+                                yp[0] = r0;
+                                yp[1] = r1;
+                                yp[2] = r2;
+                                yp[3] = r3;
+                            }
+                        } else {
+                            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(y) + (int64_t)m * ldy + n4;
+                            if (vec_ok) {
+                                const __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+                                uint2 pk;
+                                pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+                                pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+                                *reinterpret_cast<uint2*>(yp) = pk;
+                            } else {
+                                yp[0] = __float2bfloat16_rn(r0);
+                                yp[1] = __float2bfloat16_rn(r1);
+                                yp[2] = __float2bfloat16_rn(r2);
+                                yp[3] = __float2bfloat16_rn(r3);
+                            }
+                        }
+                    }
+                    u += len;
+                    ++j;
+                    continue;
+                }
+            }
 #pragma unroll 1
             for (int cb = 0; cb < RB * kHalfCols; cb += 16) {
                 // (RB = 2: the second row block's accumulator sits BNX columns further)
@@ -526,6 +688,14 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+    // CL: no CTA leaves while a peer may still write into its shared memory or while its own copies,
+    // which read its shared memory, are in flight (a peer arrives here only after they have landed);
+    // also on the way out after a timeout
+    if constexpr (Cfg::CL) {
+        if (!cl_waited) ptx::cluster_wait();
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
     }
 
     // ---- reduction of the shared tiles, by every thread of the CTA: this CTA's slice of the token

@@ -412,6 +412,16 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
+// Split cluster barrier (every thread of every CTA of the cluster arrives, and waits before it arrives again).
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the bytes
+// complete on a barrier of that CTA (`dst` and `cluster_bar` from map_to_cta; 16-byte granularity).
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst, uint32_t src, uint32_t bytes, uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "r"(src), "r"(bytes), "r"(cluster_bar)
+                 : "memory");
+}
 // 2-D tile load into THIS CTA's shared memory whose completion (tx bytes) is signalled on a
 // barrier of the pair's leader (`cluster_bar`: a shared::cluster address).
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtensorMap* m, int x, int y,

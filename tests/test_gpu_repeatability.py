@@ -6,7 +6,9 @@ kernel that reads partial sums too early finds the previous launch's identical v
 is how a barrier-phase hazard in the expansion groups showed up: wrong sums in a few tiles of the
 first launch of a process only.)  Shapes: one per kernel and plan -- split-N with and without a
 K cut, the persistent kernel with 64-, 128- and 256-token tiles as equal slices, as whole CTAs per
-tile and as whole tiles, the 256 x 256 tiles, the two-CTA kernel."""
+tile and as whole tiles, the 256 x 256 tiles, the two-CTA kernel, the cluster plan (K cut between two to eight CTAs of a cluster,
+with a ragged last tile, with as few as two k-blocks per CTA, with the largest number of clusters
+that fits)."""
 import numpy as np
 import pytest
 import torch
@@ -17,6 +19,7 @@ from paper_2505_14638_b200 import binding, inputs
 pytestmark = pytest.mark.gpu
 
 SHAPES = [(8, 4096, 4096), (16, 14336, 4096), (48, 4096, 4096), (128, 6144, 4096), (128, 4096, 14336),
+          (17, 2048, 4096), (64, 1024, 1024), (100, 2064, 8192), (33, 4096, 384), (128, 9472, 1024),
           (100, 512, 8192), (200, 4096, 4096), (256, 4096, 14336), (512, 4096, 4096), (512, 6144, 4096),
           (700, 10576, 640), (1061, 16384, 1024), (2048, 4096, 4096)]
 
@@ -77,9 +80,10 @@ def test_one_workspace_shared_by_layers_of_different_shapes_and_kernels():
     assert bool((shared[:65536 - 1024] == 0).all())
 
 
-@pytest.mark.parametrize("M,N,K", [(16, 4096, 14336), (128, 4096, 4096), (100, 512, 8192), (300, 640, 8192),
-                                   (700, 10576, 640), (1061, 16384, 1024), (512, 6144, 1024)])
-def test_linear_kernels_write_only_their_outputs_and_their_workspace(M, N, K):
+@pytest.mark.parametrize("M,N,K,pad", [(16, 4096, 14336, 8), (128, 4096, 4096, 8), (100, 512, 8192, 8), (300, 640, 8192, 8),
+                                       (700, 10576, 640, 8), (1061, 16384, 1024, 8), (512, 6144, 1024, 8),
+                                       (100, 2064, 8192, 2), (37, 4096, 4096, 6), (128, 6144, 4096, 8)])
+def test_linear_kernels_write_only_their_outputs_and_their_workspace(M, N, K, pad):
     # poisoned guard bands in front of and behind Y (with padding columns between its rows, which must
     # stay untouched too) and around a workspace of exactly the size the library asks for: no kernel
     # family of w4a8_linear may write a byte outside them
@@ -91,7 +95,7 @@ def test_linear_kernels_write_only_their_outputs_and_their_workspace(M, N, K):
     x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
     need = binding.linear_workspace_bytes(M, N, K, weight_format=tw.fmt)
     gws = Guarded((need,), torch.uint8, fill=0)
-    ldy = N + 8
+    ldy = N + pad   # (a row stride that is no multiple of four elements: the scalar store path of the cluster plan)
     gy = Guarded((M, ldy), torch.bfloat16, fill=7.0)
     ref = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_BF16, workspace=binding.new_workspace(M, N, K, tw.fmt, dev))
     for _ in range(2):

@@ -46,17 +46,18 @@ namespace w4a8 {
 // CL = true (few tiles, at most 128 tokens): the CTAs that share a tile's K range form a thread-block
 // cluster and exchange their partial sums through distributed shared memory instead of a workspace in
 // global memory.  CTA i of the C takes the i-th slice of the tile's token columns: every CTA writes,
-// its accumulator into its own (by then idle) ring memory and sends each slice to the staging area of
-// the slice's owner with one bulk copy that completes on the owner's barrier; the owner adds the C
-// partials in ascending rank order, applies the scales and stores the outputs.  Against the exchange through L2 -- partial tile out,
+// its accumulator into its own ring memory and sends each slice to the owner's ring memory with one
+// bulk copy that completes on the owner's barrier -- once the MMAs of every CTA of the cluster have
+// completed and all their rings are idle, which a cluster barrier establishes --; the owner adds the
+// C partials in ascending rank order, applies the scales and stores the outputs.  No shared memory
+// is set aside for the exchange, so the rings can be deep: with eight k-blocks per CTA all of a CTA's
+// weights are requested at once.  Against the exchange through L2 -- partial tile out,
 // fence, counter, wait, partial tiles back in, each a round trip of a microsecond or more -- this
 // takes the tail of a (128, 4096, 4096) launch from 7.4 to about 2 us.  Needs no workspace.
 template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false, bool CL_ = false>
 struct SkCfg {
     static constexpr bool W8 = W8_;
     static constexpr bool CL = CL_;
-    // staging area of the cluster exchange: C slices of ceil(columns / C) token columns x 128 channels, fp32
-    static constexpr int kRedBytes = CL_ ? (BNX_ + 8) * 128 * 4 : 0;
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
     static constexpr int G = G_;       // dequantization groups of 4 warps
     static constexpr int S1 = S1_;     // ring of TMA stages (packed chunk + activation tile)
@@ -70,7 +71,7 @@ struct SkCfg {
     static constexpr int kStage1 = kWStage + kXBytes;
     static constexpr int kW8Bytes = RB_ * 128 * 128;
     static constexpr int kBarBytes = 512;
-    static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + kRedBytes + 1024;
+    static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + 1024;
     static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;   // RB = 1: two accumulators (double buffer); RB = 2: one per row block
     static constexpr int kThreads = 32 * (10 + 4 * G);
     static constexpr int kSlotFloats = BNX * 128;
@@ -78,6 +79,9 @@ struct SkCfg {
     static_assert(RB_ == 1 || (RB_ == 2 && BNX_ == 256), "two row blocks per tile only with 256-token tiles");
     static_assert(!W8_ || RB_ == 1, "the FP8-weight variant uses one row block per tile");
     static_assert(!CL_ || (RB_ == 1 && !W8_ && BNX_ <= 128), "the cluster exchange serves one row block and at most 128 tokens");
+    // the exchange happens in the ring memory, idle by then in every CTA of the cluster: the CTA's own partial
+    // tile (BNX columns x 128 channels, fp32) and behind it the slices it receives (C x ceil(BNX / C) columns)
+    static_assert(!CL_ || S1_ * (RB_ * 9216 + BNX_ * 128) + S2_ * RB_ * 16384 >= (2 * BNX_ + 8) * 512, "room for the exchange");
     // A dequantization group handles every G-th stage, so it skips phases of the barriers it
     // waits on, and an mbarrier wait tells phases apart by parity only: the wait for use k of a
     // slot is sound only if use k-1 has completed before it starts.  That holds because a stage's
@@ -188,9 +192,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-    // CL: no CTA may signal a peer's barrier before it is initialized -- arrive here, wait before the first copy
-    if constexpr (Cfg::CL) ptx::cluster_arrive();
-    bool cl_waited = false;
+    // CL: first cluster barrier = "my MMAs have completed and my rings are idle" (a thread arrives when its role
+    // is done: the epilogue threads once the accumulator is complete); it is waited for before the first copy
+    // into a peer's rings.  Implies that the peer's barriers are initialized.
+    bool cl_arrived = false, cl_waited = false;
     const uint32_t tmem_base = *tmem_slot;
     // Launched with programmatic stream serialization: the next kernel in the stream may start its
     // set-up and weight prefetch while this one runs; everything that depends on earlier kernels
@@ -281,7 +286,39 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     if (++xmt == TM) xmt = 0;
                 }
             }
-            for (int it = 0; it < n_it; ++it) {
+            int it0 = 0;
+            if constexpr (!Cfg::W8) {
+                // The weights-only prologue as straight-line code: every slot is free, nothing to wait
+                // for, and the requests of the ring-full go out back to back (as iterations of the
+                // general loop below each took some 600 cycles, four times what the requests cost).
+#pragma unroll
+                for (int i = 0; i < S1; ++i) {
+                    if (i < ahead) {
+                        const int rows = (N - nt * TR) < TR ? (N - nt * TR) : TR;
+                        const int64_t row0 = (int64_t)kb * N + (int64_t)nt * TR;
+                        const uint8_t* csrc = wpp + row0 * kRowCodeBytes;
+                        const uint8_t* msrc = meta_base + row0 * Cfg::kMeta;
+                        const uint32_t cbytes = (uint32_t)(rows * kRowCodeBytes), mbytes = (uint32_t)(rows * Cfg::kMeta);
+                        if (ptx::elect_one()) {
+                            ptx::mbar_arrive_expect_tx(bar_full(i), cbytes + mbytes);
+                            ptx::bulk_load(stage_w(i), csrc, cbytes, bar_full(i));
+                            ptx::bulk_load(stage_w(i) + (uint32_t)Cfg::kCodeBytes, msrc, mbytes, bar_full(i));
+                        }
+                        r1.advance(S1);
+                        ++issued;
+                        if (++kb == KB) {
+                            kb = 0;
+                            if (++mt == TM) {
+                                mt = 0;
+                                ++nt;
+                            }
+                        }
+                    }
+                }
+                it0 = ahead;
+                ptx::griddep_wait();
+            }
+            for (int it = it0; it < n_it; ++it) {
                 ok = ptx::mbar_wait(bar_free1(r1.idx), r1.phase ^ 1u, abort_flag, status_word);
                 if (!ok) break;
                 // (operands worked out by the whole warp: see elect_one)
@@ -364,6 +401,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             }
         }
         __syncwarp();
+        if constexpr (Cfg::CL) {
+            ptx::cluster_arrive();
+            cl_arrived = true;
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
         {
@@ -434,6 +475,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             }
         }
         __syncwarp();
+        if constexpr (Cfg::CL) {
+            ptx::cluster_arrive();
+            cl_arrived = true;
+        }
     } else if (warp < 10) {
         // ------------------------------------------------------------------ epilogue (8 warps)
         // Accumulator: lane = output channel of the tile, column = token.  Two warps share each
@@ -491,7 +536,9 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             if constexpr (Cfg::CL) {
                 if (!whole) {
                     // ---- exchange inside the cluster ----
-                    const uint32_t red_local = bars_addr + (uint32_t)Cfg::kBarBytes;   // [source rank][column of my slice][128 channels]
+                    ptx::cluster_arrive();
+                    cl_arrived = true;
+                    const uint32_t red_local = base + (uint32_t)(BNX * 512);   // [source rank][column of my slice][128 channels]
                     const int me = (int)ptx::cluster_ctarank();
                     const int ncol = (M - mt * BNX) < BNX ? (M - mt * BNX) : BNX;   // valid token columns of the tile
                     const int w = (ncol + cl - 1) / cl;                             // columns per slice
@@ -527,10 +574,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive(bar_acc_empty(buf));
                     ptx::fence_proxy_async_smem();
-                    if (!cl_waited) {
-                        ptx::cluster_wait();   // every CTA of the cluster has initialized its barriers
-                        cl_waited = true;
-                    }
+                    ptx::cluster_wait();   // the rings of every CTA of the cluster are idle
+                    cl_waited = true;
                     asm volatile("bar.sync 1, 256;" ::: "memory");
                     if (te < cl) {
                         // one bulk copy per owner: my partial sums of its slice into its staging area,
@@ -681,6 +726,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 }
             }
         }
+        if constexpr (Cfg::CL) {
+            ptx::cluster_arrive();
+            cl_arrived = true;
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -693,6 +742,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     // which read its shared memory, are in flight (a peer arrives here only after they have landed);
     // also on the way out after a timeout
     if constexpr (Cfg::CL) {
+        if (!cl_arrived) ptx::cluster_arrive();
         if (!cl_waited) ptx::cluster_wait();
         ptx::cluster_arrive();
         ptx::cluster_wait();

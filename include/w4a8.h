@@ -105,7 +105,9 @@ int w4a8_dequant_weight(const uint8_t* codes, const void* gscale_bf16, const uin
  * `workspace` holds fp32 partial tiles when the reduction over K is split between CTAs (they are
  * added in a fixed order: results repeat bit for bit).  Calls with M <= 128 on tiled
  * weights use it only for layers with few output channels and run without it, somewhat slower,
- * when it is NULL or too small; larger M requires it.  It
+ * when it is NULL or too small; larger M requires it.  (With 17..128 tokens such layers normally
+ * need none: the CTAs that share a tile form a thread-block cluster and exchange their partial
+ * sums through shared memory, again added in a fixed order.)  It
  * needs w4a8_linear_workspace_bytes(M, N, K, weight_format) bytes and may be NULL when that is
  * 0.  For the tiled formats the workspace must have been zero-filled once (cudaMemset) before
  * its first use; every call leaves it ready for the next one, whatever that call's shape is (one

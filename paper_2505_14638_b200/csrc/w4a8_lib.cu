@@ -548,6 +548,26 @@ static bool streamk_for_128_tokens(int64_t M, int64_t N, int64_t K, int sms) {
     return M > 64 && M <= kSplitNMaxM && K >= 2048 && ((N + 127) / 128) * 4 <= sms;
 }
 
+// Tiles of 256 weight rows x Cfg::BNX tokens, whole tiles per CTA (no workspace).
+template <class Cfg>
+static int launch_two_block(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, const float* s_x, const float* s_w,
+                            int sw_stride, void* y, int64_t ldy, int out_dtype, int64_t M, int64_t N, int64_t K, int sms,
+                            cudaStream_t st) {
+    SkPlan p2;
+    p2.bnx = Cfg::BNX;
+    p2.TM = (int)((M + Cfg::BNX - 1) / Cfg::BNX);
+    p2.TN = (int)((N + 255) / 256);
+    p2.aligned = 1;
+    p2.U = (int64_t)p2.TM * p2.TN * (K / 128);
+    p2.P = (int64_t)p2.TM * p2.TN < sms ? (int64_t)p2.TM * p2.TN : sms;
+    p2.counter_bytes = 0;
+    p2.workspace_bytes = 0;
+    CUtensorMap tx2;
+    if (!make_tmap_u8_2d(&tx2, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, (uint32_t)Cfg::BNX, CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    return launch_streamk<Cfg>(tx2, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, nullptr, p2, (int)M, (int)N, (int)K, st);
+}
+
 // Few tiles (at most half as many 128-row tiles as SMs) and at most 128 tokens: CTAs per tile of the plan
 // that cuts K between the CTAs of a thread-block cluster (0: the plan does not apply).  Every CTA keeps
 // at least two k-blocks.
@@ -689,24 +709,11 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     if (sms <= 0) return W4A8_ERR_CUDA;
     if (two_block_tiles_apply(M, N, K, sms)) {
         // tiles of 256 weight rows x 256 tokens, whole tiles per CTA
-        SkPlan p2;
-        p2.bnx = 256;
-        p2.TM = (int)((M + 255) / 256);
-        p2.TN = (int)((N + 255) / 256);
-        p2.aligned = 1;
-        p2.U = (int64_t)p2.TM * p2.TN * (K / 128);
-        p2.P = (int64_t)p2.TM * p2.TN < sms ? (int64_t)p2.TM * p2.TN : sms;
-        p2.counter_bytes = 0;
-        p2.workspace_bytes = 0;
-        CUtensorMap tx2;
-        if (!make_tmap_u8_2d(&tx2, x8, (uint64_t)M, (uint64_t)K, (uint64_t)ldx8, 128, 256, CU_TENSOR_MAP_SWIZZLE_128B))
-            return W4A8_ERR_CUDA;
         return fmt == kFmtTiledSignMag
-                   ? launch_streamk<SkCfg<256, 3, 3, 2, kFmtTiledSignMag, 2>>(tx2, wpp, s_x, s_w, sw_stride, y, ldy,
-                                                                             out_dtype, workspace, p2, (int)M, (int)N,
-                                                                             (int)K, st)
-                   : launch_streamk<SkCfg<256, 3, 3, 2, kFmtTiled, 2>>(tx2, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype,
-                                                                      workspace, p2, (int)M, (int)N, (int)K, st);
+                   ? launch_two_block<SkCfg<256, 3, 3, 2, kFmtTiledSignMag, 2>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                               out_dtype, M, N, K, sms, st)
+                   : launch_two_block<SkCfg<256, 3, 3, 2, kFmtTiled, 2>>(x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy,
+                                                                        out_dtype, M, N, K, sms, st);
     }
     if (pair_kernel_applies(M, N, K, sms))
         return fmt == kFmtTiledSignMag

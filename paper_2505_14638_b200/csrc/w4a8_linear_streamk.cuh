@@ -45,15 +45,18 @@ namespace w4a8 {
 //
 // CL = true (few tiles, at most 128 tokens): the CTAs that share a tile's K range form a thread-block
 // cluster and exchange their partial sums through distributed shared memory instead of a workspace in
-// global memory.  CTA i of the C takes the i-th slice of the tile's token columns: every CTA writes,
+// global memory.  CTA i of the C takes the i-th slice of the tile's token columns: every CTA writes
 // its accumulator into its own ring memory and sends each slice to the owner's ring memory with one
 // bulk copy that completes on the owner's barrier -- once the MMAs of every CTA of the cluster have
 // completed and all their rings are idle, which a cluster barrier establishes --; the owner adds the
 // C partials in ascending rank order, applies the scales and stores the outputs.  No shared memory
 // is set aside for the exchange, so the rings can be deep: with eight k-blocks per CTA all of a CTA's
 // weights are requested at once.  Against the exchange through L2 -- partial tile out,
-// fence, counter, wait, partial tiles back in, each a round trip of a microsecond or more -- this
-// takes the tail of a (128, 4096, 4096) launch from 7.4 to about 2 us.  Needs no workspace.
+// fence, counter, wait, partial tiles back in, each a round trip of a microsecond or more: 7.4 us
+// from the last MMA to the end of a (128, 4096, 4096) launch -- the tail of a (32, 4096, 4096)
+// launch takes 2.8 us (accumulator complete 0.8, exchange and sum 1.2, closing cluster barrier 0.8).
+// At 128 tokens a CTA exchanges 64 KB, which the SM-to-SM network moves in about 2.5 us (some
+// 25 bytes per clock and SM): little is gained there.  Needs no workspace.
 template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false, bool CL_ = false>
 struct SkCfg {
     static constexpr bool W8 = W8_;

@@ -539,11 +539,12 @@ static int launch_pair(const uint8_t* x8, int64_t ldx8, const uint8_t* wpp, cons
     return launch_status();
 }
 
+// Where the cluster plan cannot run (not all of its clusters resident at once on this device):
 // 65..128 tokens on a layer with few output channels (at most a quarter as many 128-row tiles as
-// SMs): the persistent kernel with K cut between a whole number of CTAs per tile, instead of the
-// split-N kernel, every CTA of which pulls the whole X8 through its L2 port (measured, us:
-// o projection 13.4 against 15.3, down projection 21.5 against 27.5; qkv and gate_up stay: 16.9
-// against 15.4, 33.6 against 27.1).
+// SMs) take the persistent kernel with K cut between a whole number of CTAs per tile and the
+// exchange through the workspace, instead of the split-N kernel, every CTA of which pulls the whole
+// X8 through its L2 port (measured, us: o projection 13.4 against 15.3, down projection 21.5
+// against 27.5; qkv and gate_up stay: 16.9 against 15.4, 33.6 against 27.1).
 static bool streamk_for_128_tokens(int64_t M, int64_t N, int64_t K, int sms) {
     return M > 64 && M <= kSplitNMaxM && K >= 2048 && ((N + 127) / 128) * 4 <= sms;
 }

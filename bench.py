@@ -955,6 +955,11 @@ def scheme_sweep(torch, binding, inputs, dev):
                 cq = raw[c % copies]
                 binding.linear_w4a16(x, cq[0], cq[1], None, cq[3], out=y, workspace=ws16)
             t_16 = graph_time(w4a16, reps)
+            # the same scheme on the persistent prefill kernel of the W4A8 path (prepacked weights, whole tiles):
+            # the like-for-like partner of the W4A8 column at prefill sizes
+            t_16p = None
+            if m >= 128:
+                t_16p = graph_time(lambda c: binding.linear_w4a16_tiled(x, tws[c % copies], out=y), reps)
             # decode sizes: both schemes as problems of a w4a8_linear_chain launch (same kernel, partition and
             # MMAs; the FP8 weights are copied to tensor memory where the INT4 codes are expanded)
             t_c4 = t_c8 = None
@@ -970,6 +975,7 @@ def scheme_sweep(torch, binding, inputs, dev):
                         "w8a8_library_us": t_lib * 1e6, "w4a8_act_order_dequant_plus_w8a8_us": t_ao * 1e6,
                         "w4a8_act_order_one_kernel_us": t_aof * 1e6, "w4a8_same_tile_kernel_group_order_us": t_tile * 1e6,
                         "w4a16_own_kernel_us": t_16 * 1e6,
+                        "w4a16_persistent_kernel_us": None if t_16p is None else t_16p * 1e6,
                         "w4a8_chain_us_per_problem": None if t_c4 is None else t_c4 * 1e6,
                         "w8a8_chain_us_per_problem": None if t_c8 is None else t_c8 * 1e6})
             del x, x8, s_x, y, ws

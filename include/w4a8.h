@@ -315,6 +315,18 @@ int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t*
                       size_t workspace_bytes, void* stream);
 
 /*
+ * The same scheme on the persistent prefill kernel of the W4A8 path, for a like-for-like timing at
+ * prefill sizes: prepacked weights (w4a8_prepack_weight, W4A8_FMT_TILED_SIGNMAG only: symmetric
+ * storage; another format returns W4A8_ERR_INVALID_ARG), the same TMA / expansion-group / MMA /
+ * epilogue roles, the codes expanded to the BF16 values defined above, kind::f16 MMAs, whole tiles
+ * of 128 channels x 64, 128 or 256 tokens (by M) per CTA, no workspace.  Same result as
+ * w4a8_linear_w4a16 up to the order of the FP32 additions.  Other arguments and errors as there.
+ */
+int w4a8_linear_w4a16_tiled(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* weights, int weight_format,
+                            const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy,
+                            int out_dtype, void* stream);
+
+/*
  * Gated-MLP activation fused with the activation quantization of the next linear layer (the
  * paper quantizes the BF16 activations that enter a linear layer, Eq. 13; in a Llama MLP block
  * those of the down projection are silu(gate) * up, computed from the output of the stacked

@@ -29,7 +29,7 @@ EXPORTS = (
     "w4a8_linear_ex", "w4a8_linear_ex_workspace_bytes", "w4a8_linear_static_scratch",
     "w4a8_linear_w8a8", "w4a8_dequant_weight_gidx", "w4a8_linear_gidx", "w4a8_prepack_fp8",
     "w4a8_hessian_accumulate", "w4a8_hessian_prepare",
-    "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes",
+    "w4a8_silu_mul_quantize", "w4a8_linear_w4a16", "w4a8_linear_w4a16_workspace_bytes", "w4a8_linear_w4a16_tiled",
     "w4a8_quantize_weight_rtn",
     "w4a8_gar_workspace_bytes", "w4a8_gar_permutation", "w4a8_dpq_workspace_bytes", "w4a8_dpq_quantize",
     "w4a8_forward_host", "w4a8_query_device_status", "w4a8_launch_count", "w4a8_status_string",
@@ -79,6 +79,8 @@ def lib():
     L.w4a8_quantize_act.argtypes = [p, i64, i64, i64, p, i64, p, i32, p, p]
     L.w4a8_linear_w4a16.restype = i32
     L.w4a8_linear_w4a16.argtypes = [p, i64, i64, p, p, p, p, i32, i64, i64, p, i64, i32, p, sz, p]
+    L.w4a8_linear_w4a16_tiled.restype = i32
+    L.w4a8_linear_w4a16_tiled.argtypes = [p, i64, i64, p, i32, p, i32, i64, i64, p, i64, i32, p]
     L.w4a8_linear_w4a16_workspace_bytes.restype = sz
     L.w4a8_linear_w4a16_workspace_bytes.argtypes = [i64, i64, i64]
     L.w4a8_silu_mul_quantize.restype = i32
@@ -211,6 +213,22 @@ def linear_w4a16(x, codes, gscale, gzero, s_w, out=None, out_dtype=OUT_BF16, wor
                                  0 if s_w.numel() == 1 else 1, N, K, _ptr(out), out.stride(0), int(out_dtype),
                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check("w4a8_linear_w4a16", rc)
+    return out
+
+
+def linear_w4a16_tiled(x, tw, out=None, out_dtype=OUT_BF16):
+    """w4a8_linear_w4a16_tiled: x BF16 [M, K]; tw a TiledWeight in the sign-magnitude format.  Returns Y [M, N]."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    assert K == tw.K
+    if out is None:
+        dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+        out = torch.empty((M, tw.N), dtype=dt, device=x.device)
+    rc = lib().w4a8_linear_w4a16_tiled(_ptr(x), x.stride(0), M, _ptr(tw.buf), tw.fmt, _ptr(tw.s_w),
+                                       0 if tw.s_w.numel() == 1 else 1, tw.N, K, _ptr(out), out.stride(0),
+                                       int(out_dtype), _stream())
+    _check("w4a8_linear_w4a16_tiled", rc)
     return out
 
 

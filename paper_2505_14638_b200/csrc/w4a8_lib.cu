@@ -961,6 +961,50 @@ static int linear_w4a16_impl(const void* x, int64_t ldx, int64_t M, const uint8_
     return rc;
 }
 
+// W4A16 on the persistent kernel (prepacked sign-magnitude weights, whole tiles per CTA).
+static int linear_w4a16_tiled_impl(const void* x, int64_t ldx, int64_t M, const uint8_t* wpp, int fmt, const float* s_w,
+                                   int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype,
+                                   cudaStream_t st) {
+    if (!x || !wpp || !s_w || !y) return W4A8_ERR_INVALID_ARG;
+    if (fmt != kFmtTiledSignMag) return W4A8_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return W4A8_ERR_INVALID_ARG;
+    if (sw_stride != 0 && sw_stride != 1) return W4A8_ERR_INVALID_ARG;
+    if (out_dtype != W4A8_OUT_BF16 && out_dtype != W4A8_OUT_FP32) return W4A8_ERR_INVALID_ARG;
+    if (K % kGroup != 0 || N % 16 != 0 || ldx < K || ldy < N) return W4A8_ERR_BAD_SHAPE;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX / 2) return W4A8_ERR_BAD_SHAPE;
+    if (!aligned16(x) || !aligned16(wpp) || !aligned16(y) || (ldx % 8) != 0) return W4A8_ERR_BAD_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(s_w) & 3u) return W4A8_ERR_BAD_ALIGNMENT;
+    int rc = check_device();
+    if (rc != W4A8_OK) return rc;
+    const int sms = sm_count();
+    if (sms <= 0) return W4A8_ERR_CUDA;
+    // token tiles of 256 from 513 tokens on (measured, us, 256 / 128: (2048, 4096, 4096) 64 / 77,
+    // (2048, 28672, 4096) 409 / 459, (512, 4096, 4096) 35 / 25)
+    const int bnx = M > 512 ? 256 : (M > 64 ? 128 : 64);
+    SkPlan pl;
+    pl.bnx = bnx;
+    pl.TM = (int)((M + bnx - 1) / bnx);
+    pl.TN = (int)((N + 127) / 128);
+    pl.aligned = 1;
+    pl.U = (int64_t)pl.TM * pl.TN * (K / 128);
+    pl.P = (int64_t)pl.TM * pl.TN < sms ? (int64_t)pl.TM * pl.TN : sms;
+    pl.counter_bytes = 0;
+    pl.workspace_bytes = 0;
+    CUtensorMap tx;   // X as bytes: rows of 2 K bytes, boxes of 128 bytes (64 BF16 values) x bnx tokens
+    if (!make_tmap_u8_2d(&tx, x, (uint64_t)M, (uint64_t)(2 * K), (uint64_t)(2 * ldx), 128, (uint32_t)bnx,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return W4A8_ERR_CUDA;
+    // (the kernel reads no activation scale in this variant)
+    if (bnx == 256)
+        return launch_streamk<SkCfg<256, 2, 2, 2, kFmtTiledSignMag, 1, false, false, true>>(
+            tx, wpp, s_w, s_w, sw_stride, y, ldy, out_dtype, nullptr, pl, (int)M, (int)N, (int)K, st);
+    if (bnx == 128)
+        return launch_streamk<SkCfg<128, 3, 3, 2, kFmtTiledSignMag, 1, false, false, true>>(
+            tx, wpp, s_w, s_w, sw_stride, y, ldy, out_dtype, nullptr, pl, (int)M, (int)N, (int)K, st);
+    return launch_streamk<SkCfg<64, 3, 3, 2, kFmtTiledSignMag, 1, false, false, true>>(
+        tx, wpp, s_w, s_w, sw_stride, y, ldy, out_dtype, nullptr, pl, (int)M, (int)N, (int)K, st);
+}
+
 static int quantize_act_impl(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* x8, int64_t ldx8,
                              float* s_x, int scale_mode, const float* static_scale, cudaStream_t st) {
     if (!x || !x8 || !s_x) return W4A8_ERR_INVALID_ARG;
@@ -1406,6 +1450,13 @@ int w4a8_linear_w4a16(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t*
                       int64_t ldy, int out_dtype, void* workspace, size_t workspace_bytes, void* stream) {
     return linear_w4a16_impl(x_bf16, ldx, M, codes, gscale_bf16, gzero, s_w, sw_stride, N, K, y, ldy, out_dtype,
                              workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int w4a8_linear_w4a16_tiled(const void* x_bf16, int64_t ldx, int64_t M, const uint8_t* weights, int weight_format,
+                            const float* s_w, int sw_stride, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype,
+                            void* stream) {
+    return linear_w4a16_tiled_impl(x_bf16, ldx, M, weights, weight_format, s_w, sw_stride, N, K, y, ldy, out_dtype,
+                                   static_cast<cudaStream_t>(stream));
 }
 
 size_t w4a8_linear_w4a16_workspace_bytes(int64_t M, int64_t N, int64_t K) {

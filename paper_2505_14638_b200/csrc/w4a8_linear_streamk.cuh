@@ -57,10 +57,17 @@ namespace w4a8 {
 // launch takes 2.8 us (accumulator complete 0.8, exchange and sum 1.2, closing cluster barrier 0.8).
 // At 128 tokens a CTA exchanges 64 KB, which the SM-to-SM network moves in about 2.5 us (some
 // 25 bytes per clock and SM): little is gained there.  Needs no workspace.
-template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false, bool CL_ = false>
+//
+// W16 = true (the W4A16 comparison scheme of Sec. 4.3 on this kernel's skeleton): activations stay
+// BF16 (two TMA loads of 64 values per k-block and token tile), the INT4 codes are expanded to BF16
+// through a table of the group's eight magnitudes (two 128-byte panels per row and k-block), the
+// MMAs are kind::f16 with K = 16, and there is no activation scale.  Sign-magnitude format, whole
+// tiles only.
+template <int BNX_, int G_, int S1_, int S2_, int FMT_, int RB_ = 1, bool W8_ = false, bool CL_ = false, bool W16_ = false>
 struct SkCfg {
     static constexpr bool W8 = W8_;
     static constexpr bool CL = CL_;
+    static constexpr bool W16 = W16_;
     static constexpr int BNX = BNX_;   // tokens per tile (MMA N)
     static constexpr int G = G_;       // dequantization groups of 4 warps
     static constexpr int S1 = S1_;     // ring of TMA stages (packed chunk + activation tile)
@@ -70,9 +77,9 @@ struct SkCfg {
     static constexpr int RB = RB_;     // 128-row blocks per tile
     static constexpr int kCodeBytes = RB_ * 8192;   // packed codes of the tile's rows for one k-block
     static constexpr int kWStage = RB_ * 9216;  // rows x (64 code bytes + meta), padded to keep the activation tile 1024-aligned
-    static constexpr int kXBytes = BNX * 128;
+    static constexpr int kXBytes = BNX * 128 * (W16_ ? 2 : 1);
     static constexpr int kStage1 = kWStage + kXBytes;
-    static constexpr int kW8Bytes = RB_ * 128 * 128;
+    static constexpr int kW8Bytes = RB_ * 128 * 128 * (W16_ ? 2 : 1);   // expanded weights of one k-block: E4M3 (W16: BF16, two panels)
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = S1 * kStage1 + S2 * kW8Bytes + kBarBytes + 1024;
     static constexpr int kTmemCols = 2 * BNX < 32 ? 32 : 2 * BNX;   // RB = 1: two accumulators (double buffer); RB = 2: one per row block
@@ -81,6 +88,7 @@ struct SkCfg {
     static_assert(BNX == 16 || BNX == 32 || BNX == 64 || BNX == 128 || BNX == 256, "token tile");
     static_assert(RB_ == 1 || (RB_ == 2 && BNX_ == 256), "two row blocks per tile only with 256-token tiles");
     static_assert(!W8_ || RB_ == 1, "the FP8-weight variant uses one row block per tile");
+    static_assert(!W16_ || (RB_ == 1 && !W8_ && !CL_ && FMT_ == kFmtTiledSignMag), "the BF16 variant: one row block, sign-magnitude codes, whole tiles");
     static_assert(!CL_ || (RB_ == 1 && !W8_ && BNX_ <= 128), "the cluster exchange serves one row block and at most 128 tokens");
     // the exchange happens in the ring memory, idle by then in every CTA of the cluster: the CTA's own partial
     // tile (BNX columns x 128 channels, fp32) and behind it the slices it receives (C x ceil(BNX / C) columns)
@@ -362,10 +370,11 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 // activation tiles of every stage whose weights have been requested
                 for (; it_x <= it; ++it_x) {
                     const uint32_t xfull = bar_xfull(rx.idx), xdst = stage_x(rx.idx);
-                    const int x0 = xkb * 128, y0 = xmt * BNX;
+                    const int x0 = xkb * (Cfg::W16 ? 256 : 128), y0 = xmt * BNX;   // (W16: X as bytes, 256 per k-block)
                     if (ptx::elect_one()) {
                         ptx::mbar_arrive_expect_tx(xfull, (uint32_t)Cfg::kXBytes);
                         ptx::tma_load_2d(xdst, &tmap_x, x0, y0, xfull);
+                        if constexpr (Cfg::W16) ptx::tma_load_2d(xdst + (uint32_t)(BNX * 128), &tmap_x, x0 + 128, y0, xfull);
                     }
                     rx.advance(S1);
                     if (++xkb == KB) {
@@ -411,7 +420,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
         {
-            constexpr uint32_t idesc = ptx::umma_idesc_e4m3_f32(128, BNX);
+            constexpr uint32_t idesc = Cfg::W16 ? ptx::umma_idesc_bf16_f32(128, BNX) : ptx::umma_idesc_e4m3_f32(128, BNX);
             bool ok = true;
             ptx::Ring r1, r2;
             int j = 0;
@@ -425,7 +434,9 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                 for (int i = 0; i < n_it && i < S1; ++i) {
                     if (ptx::elect_one()) {
                         ptx::mbar_arrive_expect_tx(bar_xfull(i), (uint32_t)Cfg::kXBytes);
-                        ptx::tma_load_2d(stage_x(i), &tmap_x, xkb * 128, xmt * BNX, bar_xfull(i));
+                        ptx::tma_load_2d(stage_x(i), &tmap_x, xkb * (Cfg::W16 ? 256 : 128), xmt * BNX, bar_xfull(i));
+                        if constexpr (Cfg::W16)
+                            ptx::tma_load_2d(stage_x(i) + (uint32_t)(BNX * 128), &tmap_x, xkb * 256 + 128, xmt * BNX, bar_xfull(i));
                     }
                     if (++xkb == KB) {
                         xkb = 0;
@@ -454,7 +465,18 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     const uint32_t a_lo = ptx::umma_desc_lo(stage_w8(r2.idx));
                     const uint32_t b_lo = ptx::umma_desc_lo(stage_x(r1.idx));
                     const uint32_t f1 = bar_free1(r1.idx), f2 = bar_free2(r2.idx);
-                    if (ptx::elect_one()) {
+                    if constexpr (Cfg::W16) {
+                        if (ptx::elect_one()) {
+                            // two panels of 64 BF16 values, four K = 16 slices (32 bytes) each
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                ptx::umma_bf16_lo(tmem_acc, a_lo + (uint32_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2),
+                                                  b_lo + (uint32_t)((k >> 2) * ((BNX * 128) >> 4) + (k & 3) * 2), idesc,
+                                                  (accumulate | (uint32_t)k) != 0u ? 1u : 0u);
+                            ptx::umma_commit(f1);
+                            ptx::umma_commit(f2);
+                        }
+                    } else if (ptx::elect_one()) {
                         ptx::umma_f8_kblock(tmem_acc, a_lo, b_lo, idesc, accumulate);
                         if (RB == 2) ptx::umma_f8_kblock(tmem_acc + (uint32_t)BNX, a_lo + (16384u >> 4), b_lo, idesc, accumulate);
                         ptx::umma_commit(f1);
@@ -527,7 +549,7 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             float sx_pre[kHalfCols / 32];
 #pragma unroll
             for (int c = 0; c < kHalfCols / 32; ++c)
-                sx_pre[c] = (m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f;
+                sx_pre[c] = Cfg::W16 ? 1.0f : ((m0 + c * 32 + lane < M) ? __ldg(s_x + m0 + c * 32 + lane) : 0.0f);   // (W16: no activation scale)
             ok = ptx::mbar_wait(bar_acc_full(buf), RB == 1 ? (uint32_t)((j >> 1) & 1) : (uint32_t)(j & 1), abort_flag, status_word);
             if (!ok) break;
             ptx::tc_fence_after_sync();
@@ -713,6 +735,10 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             if (it >= S2) {
                 if (!ptx::mbar_wait(bar_free2(s2), (uint32_t)((it / S2 - 1) & 1), abort_flag, status_word)) break;
             }
+            if constexpr (Cfg::W16)
+                dequant_row_to_smem_bf16(stage_w(s1) + tiled_row_offset(r), stage_w(s1) + (uint32_t)Cfg::kCodeBytes + (uint32_t)(r * Cfg::kMeta), r,
+                                         stage_w8(s2) + (uint32_t)r * 128u);
+            else
 #pragma unroll
             for (int b = 0; b < RB; ++b)
                 dequant_row_to_smem<Cfg::FMT>(stage_w(s1) + tiled_row_offset(b * 128 + r),

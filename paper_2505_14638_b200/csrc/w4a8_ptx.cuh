@@ -264,6 +264,22 @@ __device__ __forceinline__ void umma_f8_lo(uint32_t tmem_d, uint32_t a_lo, uint3
         : "memory");
 }
 
+// kind::f16 (BF16 operands, K = 16 per instruction) with the descriptors given as low words.
+__device__ __forceinline__ void umma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t"
+        "}\n" ::"r"(tmem_d),
+        "r"(a_lo), "r"(b_lo), "r"(kUmmaDescHiSw128), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // The four K=32 slices of one 128-wide k-block in one go: the descriptors of slice k are the
 // base descriptors advanced by 32*k bytes (2 in the address field).
 __device__ __forceinline__ void umma_f8_kblock(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,

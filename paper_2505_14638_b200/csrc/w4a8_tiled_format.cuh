@@ -16,6 +16,8 @@
 // shared memory, whatever row partition the kernel picks at launch.
 #pragma once
 
+#include <cuda_bf16.h>
+
 #include "w4a8_common.cuh"
 #include "w4a8_ptx.cuh"
 
@@ -106,6 +108,44 @@ __device__ __forceinline__ void dequant_row_to_smem(uint32_t src, uint32_t meta,
         }
         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)c ^ sw128) << 4)), "r"(o0),
                      "r"(o1), "r"(o2), "r"(o3)
+                     : "memory");
+    }
+}
+
+// W4A16 comparison scheme, sign-magnitude codes: the row's 128 weights of the k-block as BF16
+// values bf16_rn(+-d * s) -- the same one rounding as a BF16 multiplication of the integer by the
+// group scale -- written as two rows of 128 bytes (64 values each) of two K-major panels with the
+// 128-byte swizzle, the second panel 16384 bytes behind the first.  The table of the eight
+// magnitudes is split into low and high bytes (a byte permute picks among eight bytes); the sign
+// bits of the code words sit where the high bytes' sign bits go.
+__device__ __forceinline__ void dequant_row_to_smem_bf16(uint32_t src, uint32_t meta, int row, uint32_t dst) {
+    const uint32_t sw128 = (uint32_t)(row & 7);
+    uint32_t mbits;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(mbits) : "r"(meta));
+    const float sc = bf16_bits_to_float(mbits & 0xFFFFu);
+    uint32_t pk[16];
+    load_row_codes(src, pk);
+    uint32_t tl0 = 0, tl1 = 0, th0 = 0, th1 = 0;
+#pragma unroll
+    for (int d = 0; d < 8; ++d) {
+        const uint32_t b = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__fmul_rn((float)d, sc)));
+        if (d < 4) {
+            tl0 |= (b & 0xFFu) << (8 * d);
+            th0 |= (b >> 8) << (8 * d);
+        } else {
+            tl1 |= (b & 0xFFu) << (8 * (d - 4));
+            th1 |= (b >> 8) << (8 * (d - 4));
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {   // word j: elements 8j .. 8j+7 = one 16-byte chunk of BF16 values
+        const uint32_t w = pk[j], sel = w & 0x77777777u;
+        const uint32_t lo_a = prmt(tl0, tl1, sel), hi_a = prmt(th0, th1, sel) ^ (w & 0x80808080u);
+        const uint32_t lo_b = prmt(tl0, tl1, sel >> 16), hi_b = prmt(th0, th1, sel >> 16) ^ ((w << 4) & 0x80808080u);
+        const uint32_t o0 = prmt(lo_a, hi_a, 0x5140u), o1 = prmt(lo_a, hi_a, 0x7362u);
+        const uint32_t o2 = prmt(lo_b, hi_b, 0x5140u), o3 = prmt(lo_b, hi_b, 0x7362u);
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((j >> 3) * 16384) + ((((uint32_t)j & 7u) ^ sw128) << 4)),
+                     "r"(o0), "r"(o1), "r"(o2), "r"(o3)
                      : "memory");
     }
 }

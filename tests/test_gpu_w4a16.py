@@ -79,3 +79,70 @@ def test_split_k_workspace_is_required_and_sized():
     y = binding.linear_w4a16(x, *wd, workspace=torch.empty((need,), dtype=torch.uint8, device="cuda"))
     torch.cuda.synchronize()
     assert binding.query_device_status() == 0 and torch.isfinite(y.float()).all()
+
+
+# ---- the same scheme on the persistent prefill kernel (prepacked sign-magnitude weights) ----
+
+def _symmetric_integer_case(M, N, K, seed):
+    codes, _, _ = inputs.random_codes(N, K, seed)
+    u = np.clip(np.stack([codes & 15, codes >> 4], axis=-1).reshape(N, K), 1, 15).astype(np.uint8)   # the symmetric quantizer never emits 0
+    codes = (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+    gs = np.full((N, K // 128), _bf16(1.0), dtype=np.uint16)
+    gs[::3] = _bf16(0.5)
+    s_w = (np.arange(N, dtype=np.float32) % 4 + 1) * 0.25
+    return codes, gs, s_w
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 16, 128), (16, 128, 256), (64, 256, 512), (37, 400, 1024), (128, 128, 128),
+                                   (200, 272, 640), (300, 2064, 1152), (129, 19072, 384), (600, 272, 640),
+                                   (1030, 4112, 256)])
+def test_tiled_exact_on_small_integers(M, N, K):
+    # ragged token and channel tiles of 64, 128 and 256 tokens, one to many tiles per CTA (two shapes have
+    # more tiles than SMs)
+    codes, gs, s_w = _symmetric_integer_case(M, N, K, 140 + M)
+    xb = inputs.make_small_int_activation(M, K, 150 + N)
+    ref = oracle.linear_w4a16(xb, oracle.dequant_weight_bf16(codes, gs, None), s_w)
+    tw = binding.prepack_weight(*weights_to_dev(codes, gs, None, s_w))
+    assert tw.fmt == binding.FMT_TILED_SIGNMAG
+    y = binding.linear_w4a16_tiled(bf16_dev(xb), tw, out_dtype=binding.OUT_FP32)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert np.array_equal(y.cpu().numpy().astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("M,N,K,pc", [(16, 512, 4096, False), (96, 640, 2048, True), (300, 1152, 1024, False),
+                                      (1000, 2048, 2048, True)])
+def test_tiled_gaussian_within_gates_and_equal_to_the_tile_kernel(M, N, K, pc):
+    W = inputs.make_weight(N, K, 0.02, 71)
+    codes, gscale, gzero, s_w = oracle.quantize_weight_rtn(W, symmetric=True, per_channel=pc)
+    xb = inputs.make_activation(M, K, 72, 0.01, 20.0)
+    ref = oracle.linear_w4a16(xb, oracle.dequant_weight_bf16(codes, gscale, gzero), s_w)
+    wd = weights_to_dev(codes, gscale, gzero, s_w)
+    tw = binding.prepack_weight(*wd)
+    x = bf16_dev(xb)
+    y32 = binding.linear_w4a16_tiled(x, tw, out_dtype=binding.OUT_FP32)
+    ybf = binding.linear_w4a16_tiled(x, tw, out_dtype=binding.OUT_BF16)
+    y32_again = binding.linear_w4a16_tiled(x, tw, out_dtype=binding.OUT_FP32)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.equal(y32, y32_again)
+    worst, _ = fp32_gate(y32.cpu().numpy(), ref, rel=2e-3)
+    assert worst <= 2e-3, worst
+    ok, dist = bf16_gate(bf16_bits(ybf), ref)
+    assert ok, dist
+
+
+def test_tiled_rejects_other_formats_and_leaves_padding_alone():
+    M, N, K = 70, 272, 256
+    codes, gscale, gzero, s_w = oracle.quantize_weight_rtn(inputs.make_weight(N, K, 0.02, 5), symmetric=True)
+    wd = weights_to_dev(codes, gscale, gzero, s_w)
+    x = bf16_dev(inputs.make_activation(M, K, 6))
+    generic = binding.prepack_weight(*wd, weight_format=binding.FMT_TILED)
+    with pytest.raises(binding.W4A8Error):
+        binding.linear_w4a16_tiled(x, generic)
+    tw = binding.prepack_weight(*wd)
+    y = torch.full((M + 3, N + 16), 7.0, dtype=torch.float32, device="cuda")
+    binding.linear_w4a16_tiled(x, tw, out=y[:M, :N], out_dtype=binding.OUT_FP32)
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.all(y[M:] == 7.0) and torch.all(y[:, N:] == 7.0)

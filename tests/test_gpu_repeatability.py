@@ -106,3 +106,35 @@ def test_linear_kernels_write_only_their_outputs_and_their_workspace(M, N, K, pa
     gws.check()
     assert torch.equal(gy.t[:, :N].contiguous().view(torch.int16), ref.view(torch.int16))
     assert bool((gy.t[:, N:] == 7.0).all())
+
+
+def test_seeded_random_shapes_through_every_route():
+    # 72 seeded shapes across the routing rules of w4a8_linear on prepacked weights (token counts around
+    # 16 / 64 / 128 / 512, one to many tiles, one to many k-blocks, ragged last tiles), both tiled formats in
+    # turn, BF16 and FP32 outputs in turn: every result against the float32 product of the dequantized
+    # operands, and a second launch on a fresh workspace bit for bit equal to the first
+    rng = np.random.default_rng(20250611)
+    dev = torch.device("cuda")
+    ms = [1, 7, 16, 17, 31, 64, 65, 100, 128, 129, 300, 513, 700]
+    for t in range(72):
+        M = int(ms[t % len(ms)]) if t % 3 else int(rng.integers(1, 600))
+        N = 16 * int(rng.integers(1, 260))
+        K = 128 * int(rng.integers(1, 17 if M > 128 else 40))
+        asym = bool(t % 2)
+        W = torch.from_numpy(inputs.make_weight(N, K, 0.02, seed=900 + t)).to(dev)
+        codes, gs, gz, sw = binding.quantize_weight_rtn(W, symmetric=not asym)
+        del W
+        w8 = binding.dequant_weight(codes, gs, gz)
+        tw = binding.prepack_weight(codes, gs, gz, sw)
+        xb = inputs.make_activation(M, K, 1000 + t, 0.01, 20.0)
+        x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+        ref = (x8.view(torch.float8_e4m3fn).float() @ w8.view(torch.float8_e4m3fn).float().t()) * s_x[:, None] * sw
+        od = binding.OUT_FP32 if t % 4 < 2 else binding.OUT_BF16
+        a = binding.linear_tiled(x8, s_x, tw, out_dtype=od, workspace=binding.new_workspace(M, N, K, tw.fmt, dev))
+        b = binding.linear_tiled(x8, s_x, tw, out_dtype=od, workspace=binding.new_workspace(M, N, K, tw.fmt, dev))
+        torch.cuda.synchronize()
+        assert binding.query_device_status() == 0, (M, N, K)
+        assert torch.equal(a, b), (M, N, K)
+        scale = float(ref.abs().max())
+        tol = 1e-3 if od == binding.OUT_FP32 else 6e-3      # (BF16: half a unit in the last place of the largest output)
+        assert float((a.float() - ref).abs().max()) <= tol * scale, (M, N, K, asym)

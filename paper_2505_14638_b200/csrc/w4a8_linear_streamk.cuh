@@ -773,7 +773,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     if constexpr (Cfg::CL) {
         if (!cl_arrived) ptx::cluster_arrive();
         if (!cl_waited) ptx::cluster_wait();
-        ptx::cluster_arrive();
+        // (execution order only: a release here would first wait for this thread's output stores)
+        ptx::cluster_arrive_relaxed();
         ptx::cluster_wait();
     }
 

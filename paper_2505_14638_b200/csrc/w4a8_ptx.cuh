@@ -431,6 +431,8 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
 // Split cluster barrier (every thread of every CTA of the cluster arrives, and waits before it arrives again).
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// Arrival that orders no memory operations (the barrier is used to order execution only).
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory"); }
 // Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the bytes
 // complete on a barrier of that CTA (`dst` and `cluster_bar` from map_to_cta; 16-byte granularity).
 __device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst, uint32_t src, uint32_t bytes, uint32_t cluster_bar) {

@@ -653,9 +653,9 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
                                x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st);
             else
                 rc = fmt == kFmtTiledSignMag
-                         ? launch_cluster_kcut<SkCfg<128, 4, 4, 4, kFmtTiledSignMag, 1, false, true>>(
+                         ? launch_cluster_kcut<SkCfg<128, 3, 6, 3, kFmtTiledSignMag, 1, false, true>>(
                                x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st)
-                         : launch_cluster_kcut<SkCfg<128, 4, 4, 4, kFmtTiled, 1, false, true>>(
+                         : launch_cluster_kcut<SkCfg<128, 3, 6, 3, kFmtTiled, 1, false, true>>(
                                x8, ldx8, wpp, s_x, s_w, sw_stride, y, ldy, out_dtype, (int)M, (int)N, (int)K, cl, st);
             if (rc != -1) return rc;
         }

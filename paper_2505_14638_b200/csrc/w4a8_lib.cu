@@ -636,8 +636,8 @@ static int linear_tiled_impl(const uint8_t* x8, int64_t ldx8, const float* s_x, 
     if (M > 16) {
         // 17..128 tokens on a layer with few 128-row tiles: K cut between the CTAs of a cluster (measured, us,
         // against the split-N kernel or the persistent kernel with its exchange through L2:
-        // (32, 4096, 4096) 8.6 / 9.8, (64, 2048, 4096) 8.0 / 12.6, (100, 512, 8192) 9.0 / 15.0,
-        // (128, 4096, 4096) 12.4 / 12.9, (128, 4096, 14336) 20.3 / 21.2, (128, 6144, 4096) 14.3 / 14.5; at
+        // (32, 4096, 4096) 8.0 / 9.8, (64, 2048, 4096) 7.4 / 12.6, (100, 512, 8192) 9.0 / 15.0,
+        // (128, 4096, 4096) 11.9 / 12.9, (128, 4096, 14336) 19.0 / 21.2, (128, 6144, 4096) 13.5 / 14.5; at
         // 16 tokens and fewer the split-N kernel, which overlaps its set-up with the launch before, stays
         // ahead: (8, 4096, 4096) 8.5 / 7.3)
         const int sms_c = sm_count();

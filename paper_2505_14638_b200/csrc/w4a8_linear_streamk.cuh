@@ -205,7 +205,9 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
     ptx::tc_fence_after_sync();
     // CL: first cluster barrier = "my MMAs have completed and my rings are idle" (a thread arrives when its role
     // is done: the epilogue threads once the accumulator is complete); it is waited for before the first copy
-    // into a peer's rings.  Implies that the peer's barriers are initialized.
+    // into a peer's rings.  Implies that the peer's barriers are initialized.  A cluster barrier is a hardware
+    // wait without a limit: every thread arrives where its role ends, never behind a CTA-wide barrier that the
+    // threads waiting for that arrival would have to reach first.
     bool cl_arrived = false, cl_waited = false;
     const uint32_t tmem_base = *tmem_slot;
     // Launched with programmatic stream serialization: the next kernel in the stream may start its

@@ -216,62 +216,67 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
 }
 
 // Columns to the right of block b: w[n][v] <- fma(-e[n][q], U[128 b + q][v], w[n][v]), q = 0..127
-// in order.  CTA = 512 columns x 16 rows; a thread owns two columns (v, v + 256) and keeps their 16
-// rows in registers, so that one q costs four 16-byte shared loads, two global loads and 32 FMAs.
-__global__ void __launch_bounds__(256)
+// in order.  A CTA takes 128 rows x 128 columns, a thread 8 rows x 8 columns (two runs of four
+// columns, 64 apart) which it keeps in registers; the errors and the rows of U come through shared
+// memory in chunks of 32 values of q, so that one q costs a thread four 16-byte shared loads and 64
+// FMAs and a tile of U is fetched once per 128 rows.  (First version: 16 rows x 512 columns per CTA,
+// U straight from L2 -- every 16 rows fetched it again, and the L2 traffic, not the FMA pipe, set
+// the pace: a fifth to a third of the FMA peak.)  The chain of one element is unchanged: the same
+// fused multiply-adds, q ascending.
+__global__ void __launch_bounds__(256, 2)
 dpq_trailing_kernel(float* __restrict__ work, const float* __restrict__ U, const float* __restrict__ err,
                     int64_t N, int64_t K, int b) {
-    __shared__ float4 e_s[128][4];  // [q][row / 4]: the 16 rows' errors of one q in four 16-byte loads
+    __shared__ __align__(16) float e_s[32][132];  // [q][row] = -e (the padding spreads the transposing stores over the banks)
+    __shared__ __align__(16) float u_s[32][128];  // [q][column]
     const int64_t p0 = (int64_t)b * 128;
-    const int64_t v0 = p0 + 128 + (int64_t)blockIdx.x * 512 + threadIdx.x;
-    const int64_t v1 = v0 + 256;
-    const int64_t n0 = (int64_t)blockIdx.y * 16;
-    for (int i = threadIdx.x; i < 16 * 128; i += 256) {
-        const int r = i >> 7, q = i & 127;
-        reinterpret_cast<float*>(&e_s[q][0])[r] = (n0 + r < N) ? -err[(n0 + r) * 128 + q] : 0.0f;  // -e, exact
-    }
-    __syncthreads();
-    if (v0 >= K) return;
-    const bool two = v1 < K;
-    float w0[16], w1[16];
+    const int64_t v0 = p0 + 128 + (int64_t)blockIdx.x * 128;   // K is a multiple of 128: the column tile is whole
+    const int64_t n0 = (int64_t)blockIdx.y * 128;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    float acc[8][8];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        w0[r] = (n0 + r < N) ? work[(n0 + r) * K + v0] : 0.0f;
-        w1[r] = (two && n0 + r < N) ? work[(n0 + r) * K + v1] : 0.0f;
+    for (int i = 0; i < 8; ++i) {
+        const int64_t n = n0 + ty * 8 + i;
+        float4 a = make_float4(0.0f, 0.0f, 0.0f, 0.0f), c = a;
+        if (n < N) {
+            a = *reinterpret_cast<const float4*>(work + n * K + v0 + tx * 4);
+            c = *reinterpret_cast<const float4*>(work + n * K + v0 + 64 + tx * 4);
+        }
+        acc[i][0] = a.x; acc[i][1] = a.y; acc[i][2] = a.z; acc[i][3] = a.w;
+        acc[i][4] = c.x; acc[i][5] = c.y; acc[i][6] = c.z; acc[i][7] = c.w;
     }
-    const float* up = U + p0 * K;
+    const float* up = U + p0 * K + v0;
 #pragma unroll 1
-    for (int q8 = 0; q8 < 128; q8 += 8) {
-        // eight rows of U at a time: sixteen loads in flight per thread hide the L2 latency
-        float ua[8], ub[8];
+    for (int qc = 0; qc < 128; qc += 32) {
+        if (qc > 0) __syncthreads();   // the previous chunk has been consumed
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            ua[i] = __ldg(up + (int64_t)(q8 + i) * K + v0);
-            ub[i] = two ? __ldg(up + (int64_t)(q8 + i) * K + v1) : 0.0f;
+        for (int i = 0; i < 16; ++i) {
+            const int idx = i * 256 + tid;
+            const int q = idx & 31, row = idx >> 5;
+            e_s[q][row] = (n0 + row < N) ? -err[(n0 + row) * 128 + qc + q] : 0.0f;   // -e, exact
+            const int c = idx & 127, qu = idx >> 7;
+            u_s[qu][c] = __ldg(up + (int64_t)(qc + qu) * K + c);
         }
+        __syncthreads();
+#pragma unroll 2
+        for (int q = 0; q < 32; ++q) {
+            const float4 ea = *reinterpret_cast<const float4*>(&e_s[q][ty * 8]);
+            const float4 eb = *reinterpret_cast<const float4*>(&e_s[q][ty * 8 + 4]);
+            const float4 ua = *reinterpret_cast<const float4*>(&u_s[q][tx * 4]);
+            const float4 ub = *reinterpret_cast<const float4*>(&u_s[q][64 + tx * 4]);
+            const float e[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
+            const float u[8] = {ua.x, ua.y, ua.z, ua.w, ub.x, ub.y, ub.z, ub.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-        const int q = q8 + i;
-        const float u0 = ua[i], u1 = ub[i];
+            for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int r4 = 0; r4 < 4; ++r4) {
-            const float4 e = e_s[q][r4];
-            w0[4 * r4 + 0] = __fmaf_rn(e.x, u0, w0[4 * r4 + 0]);
-            w0[4 * r4 + 1] = __fmaf_rn(e.y, u0, w0[4 * r4 + 1]);
-            w0[4 * r4 + 2] = __fmaf_rn(e.z, u0, w0[4 * r4 + 2]);
-            w0[4 * r4 + 3] = __fmaf_rn(e.w, u0, w0[4 * r4 + 3]);
-            w1[4 * r4 + 0] = __fmaf_rn(e.x, u1, w1[4 * r4 + 0]);
-            w1[4 * r4 + 1] = __fmaf_rn(e.y, u1, w1[4 * r4 + 1]);
-            w1[4 * r4 + 2] = __fmaf_rn(e.z, u1, w1[4 * r4 + 2]);
-            w1[4 * r4 + 3] = __fmaf_rn(e.w, u1, w1[4 * r4 + 3]);
-        }
+                for (int j = 0; j < 8; ++j) acc[i][j] = __fmaf_rn(e[i], u[j], acc[i][j]);   // Eq. 12
         }
     }
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        if (n0 + r < N) {
-            work[(n0 + r) * K + v0] = w0[r];
-            if (two) work[(n0 + r) * K + v1] = w1[r];
+    for (int i = 0; i < 8; ++i) {
+        const int64_t n = n0 + ty * 8 + i;
+        if (n < N) {
+            *reinterpret_cast<float4*>(work + n * K + v0 + tx * 4) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+            *reinterpret_cast<float4*>(work + n * K + v0 + 64 + tx * 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
         }
     }
 }

@@ -1617,7 +1617,7 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
         ++launches;
         const int64_t rest = K - ((int64_t)b + 1) * 128;
         if (rest > 0) {
-            dim3 grid((unsigned)((rest + 511) / 512), (unsigned)((N + 15) / 16));
+            dim3 grid((unsigned)(rest / 128), (unsigned)((N + 127) / 128));
             dpq_trailing_kernel<<<grid, 256, 0, st>>>(work, U, err, N, K, b);
             ++launches;
         }

@@ -138,3 +138,23 @@ def test_seeded_random_shapes_through_every_route():
         scale = float(ref.abs().max())
         tol = 1e-3 if od == binding.OUT_FP32 else 6e-3      # (BF16: half a unit in the last place of the largest output)
         assert float((a.float() - ref).abs().max()) <= tol * scale, (M, N, K, asym)
+
+
+def test_cluster_plan_needs_no_workspace():
+    # 17..128 tokens on a layer with few tiles: the call succeeds without any workspace and equals the
+    # call with one bit for bit
+    dev = torch.device("cuda")
+    M, N, K = 48, 528, 1024
+    W = torch.from_numpy(inputs.make_weight(N, K, 0.02, seed=77)).to(dev)
+    tw = binding.prepack_weight(*binding.quantize_weight_rtn(W, symmetric=True))
+    xb = inputs.make_activation(M, K, 78, 0.01, 20.0)
+    x8, s_x = binding.quantize_act(torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).to(dev))
+    with_ws = binding.linear_tiled(x8, s_x, tw, out_dtype=binding.OUT_FP32)
+    y = torch.empty((M, N), dtype=torch.float32, device=dev)
+    rc = binding.lib().w4a8_linear(x8.data_ptr(), x8.stride(0), s_x.data_ptr(), M, tw.buf.data_ptr(), None, None, tw.fmt,
+                                   tw.s_w.data_ptr(), 0 if tw.s_w.numel() == 1 else 1, N, K, 128, y.data_ptr(), y.stride(0),
+                                   binding.OUT_FP32, None, 0, torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert binding.query_device_status() == 0
+    assert torch.equal(y, with_ws)

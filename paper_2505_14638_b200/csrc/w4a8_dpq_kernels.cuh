@@ -6,7 +6,7 @@
 // sending its scaled error e to the columns on its right (Eq. 12): w_v <- fma(-e, U_qv, w_v),
 // U = upper Cholesky factor of the inverse Hessian in processing order.  Work is cut the way
 // GPTQ cuts it, in blocks of one group (128 columns):
-//   dpq_block_kernel     one warp per row: group scale / zero-point (Eq. 8, optional search),
+//   dpq_block_kernel     half a warp per row: group scale / zero-point (Eq. 8, optional search),
 //                        then the 128 columns in sequence with the updates inside the block;
 //                        writes the codes, the group's scale and zero-point and the 128 errors;
 //   dpq_trailing_kernel  applies the block's 128 errors to every column to the right of the
@@ -110,13 +110,32 @@ __device__ __forceinline__ long long warp_sum_ll(long long v) {
     return v;
 }
 
-// One warp per row, 16 rows per CTA (the chain of dependent divisions and conversions of one
-// column is long: many warps per SM hide it); block `b` = processing positions [128 b, 128 b + 128).
-// Lane l owns positions l, l + 32, l + 64, l + 96 of the block.  The block of U (128 x 128) is
-// staged in shared memory for the whole CTA.
-constexpr int kDpqRowsPerCta = 16;
+// Half a warp per row, 32 rows per CTA; block `b` = processing positions [128 b, 128 b + 128).
+// The chain of one column (three IEEE divisions, two FP8 conversions) is some seventy dependent
+// instructions that every lane executes and only the column's owner needs: with two rows per warp a
+// warp instruction carries two of those chains (a warp per row spent its issue slots on them: with
+// 28 warps per SM the kernel was bound by issue, not by latency).  Lane l of a half owns positions
+// l, l + 16, ..., l + 112 of the block.  The block of U (128 x 128) is staged in shared memory for
+// the whole CTA.
+constexpr int kDpqRowsPerCta = 32;
 
-__global__ void __launch_bounds__(32 * kDpqRowsPerCta)
+__device__ __forceinline__ float half_warp_min(float v) {
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ float half_warp_max(float v) {
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ long long half_warp_sum_ll(long long v) {
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(16 * kDpqRowsPerCta)
 dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const int32_t* __restrict__ perm,
                  int64_t N, int64_t K, int b, int symmetric, int mse_steps, int per_channel,
                  const float* __restrict__ s_w, uint8_t* __restrict__ codes, uint16_t* __restrict__ gscale,
@@ -124,34 +143,38 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
     extern __shared__ float u_s[];  // [128][128] block of U, then kDpqRowsPerCta x 128 bytes of code staging
     uint8_t* code_s = reinterpret_cast<uint8_t*>(u_s + 128 * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int half = lane >> 4, sl = lane & 15;
     const int64_t p0 = (int64_t)b * 128;
-    for (int i = threadIdx.x; i < 128 * 128; i += 32 * kDpqRowsPerCta) {
+    for (int i = threadIdx.x; i < 128 * 128; i += 16 * kDpqRowsPerCta) {
         const int q = i >> 7, v = i & 127;
         u_s[i] = (v >= q) ? U[(p0 + q) * K + p0 + v] : 0.0f;
     }
     __syncthreads();
-    const int64_t n = (int64_t)blockIdx.x * kDpqRowsPerCta + warp;
-    if (n >= N) return;
+    const int rl = 2 * warp + half;                               // row within the CTA
+    const int64_t n_raw = (int64_t)blockIdx.x * kDpqRowsPerCta + rl;
+    if ((int64_t)blockIdx.x * kDpqRowsPerCta + 2 * warp >= N) return;   // neither row of the warp exists
+    const bool valid = n_raw < N;                                 // (a half without a row repeats the last one and stores nothing)
+    const int64_t n = valid ? n_raw : N - 1;
     const int64_t G = K >> 7;
     const float sw = per_channel ? s_w[n] : s_w[0];
     float* wrow = work + n * K + p0;
-    float w[4];
+    float w[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) w[i] = wrow[lane + 32 * i];
+    for (int i = 0; i < 8; ++i) w[i] = wrow[sl + 16 * i];
 
     // Eq. 7 on the group's current weights, then Eq. 8 (once per group)
-    float w8[4];
+    float w8[8];
     float lo = 0.0f, hi = 0.0f, amax = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 8; ++i) {
         w8[i] = e4m3_roundtrip(__fdiv_rn(w[i], sw));
         lo = fminf(lo, w8[i]);
         hi = fmaxf(hi, w8[i]);
         amax = fmaxf(amax, fabsf(w8[i]));
     }
-    lo = warp_min(lo);
-    hi = warp_max(hi);
-    amax = warp_max(amax);
+    lo = half_warp_min(lo);
+    hi = half_warp_max(hi);
+    amax = half_warp_max(amax);
     DpqGroup grp = dpq_group_params(lo, hi, amax, 1.0f, symmetric);
     if (mse_steps > 1) {
         // Sec. 3.3: least squared error over the group among shrunk ranges; exact integer sums
@@ -161,13 +184,13 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
             const DpqGroup gt = dpq_group_params(lo, hi, amax, pt, symmetric);
             long long e2 = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 float h;
                 (void)dpq_quant_dequant(w8[i], gt, symmetric, h);
                 const long long d = (long long)__fmul_rn(__fsub_rn(w8[i], h), 512.0f);
                 e2 += d * d;
             }
-            e2 = warp_sum_ll(e2);
+            e2 = half_warp_sum_ll(e2);
             if (best < 0 || e2 < best) {
                 best = e2;
                 grp = gt;
@@ -175,15 +198,15 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
         }
     }
 
-    // the 128 columns in sequence; every lane follows the same scalar computation
+    // the 128 columns in sequence; every lane of a half follows the same scalar computation
     const int64_t og = perm ? (int64_t)(perm[p0] >> 7) : (int64_t)b;
     float* erow = err + n * 128;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 8; ++i) {
 #pragma unroll 4
-        for (int o = 0; o < 32; ++o) {
-            const int q = 32 * i + o;
-            const float wq = __shfl_sync(0xFFFFFFFFu, w[i], o);
+        for (int o = 0; o < 16; ++o) {
+            const int q = 16 * i + o;
+            const float wq = __shfl_sync(0xFFFFFFFFu, w[i], (lane & 16) | o);
             const float wq8 = e4m3_roundtrip(__fdiv_rn(wq, sw));         // Eq. 7
             float h8;
             const int u = dpq_quant_dequant(wq8, grp, symmetric, h8);    // Eq. 9, Eq. 10
@@ -191,25 +214,27 @@ dpq_block_kernel(float* __restrict__ work, const float* __restrict__ U, const in
             const float e = __fdiv_rn(__fsub_rn(wq, h16), u_s[q * 128 + q]);
             const float* urow = u_s + q * 128;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int v = lane + 32 * k;
+            for (int k = 0; k < 8; ++k) {
+                const int v = sl + 16 * k;
                 if (v > q) w[k] = __fmaf_rn(-e, urow[v], w[k]);          // Eq. 12
             }
-            if (lane == o) {
+            if (sl == o && valid) {
                 erow[q] = e;
                 const int c = perm ? (perm[p0 + q] & 127) : q;  // column inside its original group
-                code_s[warp * 128 + c] = (uint8_t)u;
+                code_s[rl * 128 + c] = (uint8_t)u;
             }
         }
     }
     __syncwarp();
+    if (!valid) return;
     // codes of the group, original order, two per byte (even column in the low nibble)
     {
-        const uint8_t* cs = code_s + warp * 128 + lane * 4;
-        const uint16_t packed = (uint16_t)(cs[0] | (cs[1] << 4) | (cs[2] << 8) | (cs[3] << 12));
-        *reinterpret_cast<uint16_t*>(codes + n * (K >> 1) + og * 64 + lane * 2) = packed;
+        const uint8_t* cs = code_s + rl * 128 + sl * 8;
+        const uint32_t packed = (uint32_t)cs[0] | ((uint32_t)cs[1] << 4) | ((uint32_t)cs[2] << 8) | ((uint32_t)cs[3] << 12) |
+                                ((uint32_t)cs[4] << 16) | ((uint32_t)cs[5] << 20) | ((uint32_t)cs[6] << 24) | ((uint32_t)cs[7] << 28);
+        *reinterpret_cast<uint32_t*>(codes + n * (K >> 1) + og * 64 + sl * 4) = packed;
     }
-    if (lane == 0) {
+    if (sl == 0) {
         gscale[n * G + og] = __bfloat16_as_ushort(__float2bfloat16_rn(grp.s));
         if (gzero) gzero[n * G + og] = (uint8_t)grp.z;
     }

@@ -1611,7 +1611,7 @@ int w4a8_dpq_quantize(const float* W, int64_t N, int64_t K, int group, const flo
     uint64_t launches = 3;
     const int G = (int)(K / kGroup);
     for (int b = 0; b < G; ++b) {
-        dpq_block_kernel<<<(unsigned)((N + kDpqRowsPerCta - 1) / kDpqRowsPerCta), 32 * kDpqRowsPerCta, kBlockSmem, st>>>(
+        dpq_block_kernel<<<(unsigned)((N + kDpqRowsPerCta - 1) / kDpqRowsPerCta), 16 * kDpqRowsPerCta, kBlockSmem, st>>>(
             work, U, perm, N, K, b, symmetric, mse_steps, per_channel, s_w, codes,
             static_cast<uint16_t*>(gscale_bf16), gzero, err);
         ++launches;

@@ -48,7 +48,7 @@ def test_gar_permutation_matches(K):
     assert np.array_equal(perm.cpu().numpy(), oracle.gar_permutation(d))
 
 
-@pytest.mark.parametrize("N,K", [(8, 128), (24, 384), (100, 1024)])
+@pytest.mark.parametrize("N,K", [(8, 128), (24, 384), (100, 1024), (37, 256), (1, 128)])
 @pytest.mark.parametrize("symmetric", [False, True])
 def test_dpq_matches_oracle_in_original_order(N, K, symmetric):
     W = inputs.make_weight(N, K, 0.02, seed=N + K)

@@ -276,8 +276,14 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
                     // (the whole chunk inside the problem: no test per token -- the drain is bound by issue slots)
                     __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(y) + (int64_t)(m0 + c0) * ldy + n;
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj)
-                        yp[(int64_t)jj * ldy] = __float2bfloat16_rn(__uint_as_float(v[jj]) * (sx[jj] * swn));
+                    for (int jj = 0; jj < 16; jj += 2) {
+                        // two tokens per multiply (packed FP32 pairs: the same two roundings per value)
+                        float sc0, sc1, r0, r1;
+                        ptx::mul_f32x2(sx[jj], sx[jj + 1], swn, swn, sc0, sc1);
+                        ptx::mul_f32x2(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), sc0, sc1, r0, r1);
+                        yp[(int64_t)jj * ldy] = __float2bfloat16_rn(r0);
+                        yp[(int64_t)(jj + 1) * ldy] = __float2bfloat16_rn(r1);
+                    }
                 } else {
                     __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(y) + (int64_t)(m0 + c0) * ldy + n;
 #pragma unroll

@@ -39,6 +39,19 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// Two FP32 products in one instruction (round to nearest even each, as two mul.rn.f32).
+__device__ __forceinline__ void mul_f32x2(float a0, float a1, float b0, float b1, float& r0, float& r1) {
+    asm("{\n\t"
+        ".reg .b64 a, b, d;\n\t"
+        "mov.b64 a, {%2, %3};\n\t"
+        "mov.b64 b, {%4, %5};\n\t"
+        "mul.rn.f32x2 d, a, b;\n\t"
+        "mov.b64 {%0, %1}, d;\n\t"
+        "}\n"
+        : "=f"(r0), "=f"(r1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

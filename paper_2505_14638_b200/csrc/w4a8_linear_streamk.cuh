@@ -243,14 +243,12 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
             const int b = ch / (BNX / 16), c0 = (ch - b * (BNX / 16)) * 16;
             uint32_t v[16];
             ptx::tmem_ld_32x32b_x16(tmem_acc0 + (uint32_t)(b * BNX + c0), v);
-            ptx::tmem_ld_wait();
-            if (m0 + c0 >= M) continue;  // warp-uniform
             const int n = b == 0 ? n_lo : n_hi;
             const float swn = b == 0 ? swn_lo : swn_hi;
             float sx[16];
             if (sx_vec && m0 + c0 + 16 <= M) {
                 // the chunk's sixteen activation scales: four 16-byte loads of one address per warp (L1 hits after
-                // the first warp) instead of sixteen shuffles
+                // the first warp) instead of sixteen shuffles; issued while the tensor-memory load is in flight
 #pragma unroll
                 for (int v4 = 0; v4 < 4; ++v4) {
                     const float4 t = __ldg(reinterpret_cast<const float4*>(s_x + m0 + c0) + v4);
@@ -266,6 +264,8 @@ linear_streamk_kernel(const __grid_constant__ CUtensorMap tmap_x,  // X8 u8 [M][
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) sx[jj] = __shfl_sync(0xFFFFFFFFu, sx_lane, (c0 & 16) + jj);
             }
+            ptx::tmem_ld_wait();
+            if (m0 + c0 >= M) continue;  // warp-uniform
             if (n < N) {
                 if (out_dtype == W4A8_OUT_FP32) {
                     float* yp = reinterpret_cast<float*>(y) + (int64_t)(m0 + c0) * ldy + n;
